@@ -1,0 +1,254 @@
+/*
+ * sailor.h — C ABI of the batched plan simulator and plan search (CUDA, sm_100a).
+ *
+ * The library evaluates candidate training-job configurations with the Sailor
+ * simulator (Sailor, SOSP'25, Sec. 4.3: memory footprint, 1F1B iteration time,
+ * cost per iteration) and reduces a whole search space to the best plan and the
+ * top-k under an objective and a constraint (Sec. 4.2, last two paragraphs of the
+ * planner overview).  Every candidate is simulated on the GPU; there is no CPU
+ * fallback.  All functions return 0 on success and a negative SAILOR_E_* code on
+ * failure; none throws, aborts or prints.
+ *
+ * Conventions
+ *   P      pipeline stages          D    data-parallel degree (same for all stages, H3)
+ *   tp     tensor-parallel degree   mbs  microbatch size
+ *   gbs    global batch size        N_b  = gbs / (D * mbs), microbatches per pipeline
+ *   T      GPU types                Z    zones; a "digit" d = zone * T + type
+ *   kinds  layer kinds: 0 = EMBED, 1 = BLOCK, 2 = HEAD
+ *
+ * Arithmetic.  Bytes and counts are unsigned integers (exact).  Times and costs
+ * are IEEE binary64 evaluated in one fixed order without fused multiply-add:
+ *   f_i   = sum over the layers of stage i (stage order) of fwd[kind][g_i][tp_i][mbs]
+ *   b_i   = same over bwd, then + f_i when recomputation is on
+ *   u_i   = same over upd[kind][g_i][tp_i]
+ *   c_i   = alpha(link_i) + (double)p2p_bytes[mbs] * inv_bw(link_i), 0 for the last stage
+ *   t_i   = (f_i + b_i) + 2 * c_i
+ *   T_pp  = (t_0 + t_1 + ... left to right) + (double)N_b * max_i t_i
+ *   sync_i= D == 1 ? 0 : ((2(D-1))/D * (double)gradbytes_i) * inv_bw_dp(i) + (2(D-1)) * alpha_dp(i)
+ *   T_iter= (T_pp + max_i sync_i) + max_i u_i                          (Sec. 4.3, Sec. 4.2.2)
+ *   rate  = sum_i (double)(D * tp_i) * (price_per_hour[z_i][g_i] / 3600)   left to right
+ *   C_comm= sum over stage boundaries that cross zones of
+ *           (double)(2 * N_b * D * p2p_bytes[mbs]) * egress[z_i][z_{i+1}]  left to right
+ *   C_iter= rate * T_iter + C_comm                                      (Sec. 4.3, Sec. 4.2.3)
+ *
+ * Threading.  A context is not thread-safe; use one context per host thread.
+ */
+#ifndef SAILOR_H
+#define SAILOR_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ---- limits --------------------------------------------------------------------------- */
+#define SAILOR_KINDS      3     /* EMBED, BLOCK, HEAD                                       */
+#define SAILOR_T_MAX      8     /* GPU types                                                */
+#define SAILOR_Z_MAX      8     /* zones                                                    */
+#define SAILOR_TP_MAX     8     /* entries of tp_values                                     */
+#define SAILOR_MBS_MAX    16    /* entries of mbs_values                                    */
+#define SAILOR_P_MAX      96    /* pipeline stages in one plan                              */
+#define SAILOR_RUN_MAX    16    /* runs in a plan record                                    */
+#define SAILOR_SEG_MAX    4     /* segments the enumerator varies per plan                  */
+#define SAILOR_K_MAX      32    /* top-k                                                    */
+#define SAILOR_NP_MAX     32    /* entries of sailor_space.p_values                         */
+#define SAILOR_ND_MAX     32    /* entries of sailor_space.d_values                         */
+
+/* ---- error codes ---------------------------------------------------------------------- */
+#define SAILOR_OK          0
+#define SAILOR_E_ARG      (-1)  /* null pointer, zero k, inconsistent sizes, bad record      */
+#define SAILOR_E_RANGE    (-2)  /* an index or a size is outside a table or a limit above    */
+#define SAILOR_E_CUDA     (-3)  /* a CUDA call failed; see sailor_last_cuda_error            */
+#define SAILOR_E_NOMEM    (-4)  /* host or device allocation failed                          */
+#define SAILOR_E_DEVICE   (-5)  /* a kernel reported an internal fault (bounded wait ran out) */
+
+/* ---- status bits of one simulated plan ------------------------------------------------- */
+#define SAILOR_ST_INVALID          1u   /* gbs % (D*mbs) != 0, tp > gpus_per_node, heads % tp != 0 (H1) */
+#define SAILOR_ST_OVER_AVAIL       2u   /* needs more GPUs of some (zone, type) than available           */
+#define SAILOR_ST_OOM              4u   /* some stage's peak memory exceeds its GPU's capacity (H2)     */
+#define SAILOR_ST_OVER_BUDGET      8u   /* C_iter > budget                                              */
+#define SAILOR_ST_UNDER_THROUGHPUT 16u  /* 1 / T_iter < min_iters_per_s                                 */
+#define SAILOR_ST_BAD_RECORD       32u  /* device-side record failed its bounds checks; nothing read    */
+
+/* ---- inputs --------------------------------------------------------------------------- */
+
+/* Training job (Sec. 4: "model training specifications").  Layers are n_blocks identical
+ * BLOCK layers, preceded by one EMBED layer when has_embed and followed by one HEAD layer
+ * when has_head.  A plan with P stages gives stage i  n_blocks / P  blocks, plus one more
+ * for the first n_blocks % P stages; EMBED goes to stage 0, HEAD to stage P-1. */
+typedef struct sailor_model {
+    uint32_t n_blocks;          /* >= 1                                                     */
+    uint32_t has_embed;         /* 0 / 1                                                    */
+    uint32_t has_head;          /* 0 / 1                                                    */
+    uint32_t heads;             /* attention heads; tp must divide it                       */
+    uint64_t gbs;               /* global batch size, never changed by the planner          */
+    uint32_t mul_factor;        /* copies of each parameter (weights, grads, optimizer), Sec. 4.3 */
+    uint32_t dtype_size;        /* bytes per parameter copy                                 */
+    uint32_t grad_dtype_size;   /* bytes per gradient element sent in the all-reduce        */
+    uint32_t _pad;
+} sailor_model;
+
+/* Per-layer profile (Sec. 4.1, training job profiling).  All pointers are HOST arrays,
+ * row-major in the index order shown, copied by sailor_create. */
+typedef struct sailor_profile {
+    uint32_t n_types, n_tp, n_mbs, _pad;
+    uint32_t tp_values[SAILOR_TP_MAX];    /* tensor-parallel degree of each tp index        */
+    uint32_t mbs_values[SAILOR_MBS_MAX];  /* microbatch size of each mbs index              */
+    const double*   fwd;        /* [kind][type][tp][mbs] seconds, finite, >= 0              */
+    const double*   bwd;        /* [kind][type][tp][mbs] seconds                            */
+    const double*   upd;        /* [kind][type][tp]      seconds                            */
+    const uint64_t* params;     /* [kind] parameters of one layer                           */
+    const uint64_t* act_saved;  /* [kind][tp][mbs] bytes kept per in-flight microbatch      */
+    const uint64_t* act_ckpt;   /* [kind][tp][mbs] bytes kept when recomputation is on      */
+    const uint64_t* act_work;   /* [kind][tp][mbs] transient working bytes                  */
+    const uint64_t* p2p_bytes;  /* [mbs] bytes one microbatch sends to the next stage       */
+} sailor_profile;
+
+/* Cluster (Sec. 4: quotas, prices; Sec. 4.1, cluster profiling).  A link is a degree-1
+ * time model  time(m) = alpha + m * inv_bw  (seconds, seconds per byte).  HOST arrays. */
+typedef struct sailor_cluster {
+    uint32_t n_types, n_zones;
+    const uint64_t* capacity;        /* [type] bytes of GPU memory                           */
+    const uint64_t* reserved;        /* [type] bytes unavailable to the job                  */
+    const uint32_t* gpus_per_node;   /* [type]                                               */
+    const double*   price_per_hour;  /* [zone][type] USD per GPU-hour                        */
+    const double*   intra_alpha;     /* [zone][type] link inside one node                    */
+    const double*   intra_inv_bw;    /* [zone][type]                                         */
+    const double*   inter_alpha;     /* [zone][type] link between nodes of one zone          */
+    const double*   inter_inv_bw;    /* [zone][type]                                         */
+    const double*   zone_alpha;      /* [zone][zone] link between zones (diagonal unused)    */
+    const double*   zone_inv_bw;     /* [zone][zone]                                         */
+    const double*   egress;          /* [zone][zone] USD per byte sent from row to column    */
+} sailor_cluster;
+
+/* One plan, stages run-length encoded: run r covers n_stages consecutive stages that share
+ * (type, zone, tp).  sum of n_stages == P.  72 bytes; arrays of records must be 8-byte aligned. */
+typedef struct sailor_run {
+    uint8_t type, zone, tp_idx, n_stages;
+} sailor_run;
+
+typedef struct sailor_plan_rec {
+    uint8_t  P;                 /* 1 .. SAILOR_P_MAX                                        */
+    uint8_t  mbs_idx;
+    uint8_t  rc;                /* 1 = activation recomputation                             */
+    uint8_t  n_runs;            /* 1 .. SAILOR_RUN_MAX                                      */
+    uint16_t D;                 /* >= 1                                                     */
+    uint16_t _pad;
+    sailor_run run[SAILOR_RUN_MAX];
+} sailor_plan_rec;
+
+/* Search space of sailor_plan.  Flat index, digits from low to high:
+ *   seg[nseg-1], ..., seg[0]   radix T*Z each, digit = zone*T + type
+ *   d_values index, rc_values index, tp_idx index, mbs_idx index
+ * and the sub-spaces of the entries of p_values are concatenated in that order.
+ * nseg = min(P, seg_max); stage i belongs to segment floor(i * nseg / P). */
+typedef struct sailor_space {
+    uint32_t n_p, n_mbs, n_tp, n_rc, n_d, seg_max;
+    uint8_t  p_values[SAILOR_NP_MAX];
+    uint8_t  mbs_idx[SAILOR_MBS_MAX];
+    uint8_t  tp_idx[SAILOR_TP_MAX];
+    uint8_t  rc_values[2];
+    uint8_t  _pad[6];
+    uint16_t d_values[SAILOR_ND_MAX];
+} sailor_space;
+
+#define SAILOR_OBJ_MAX_THROUGHPUT         0   /* minimise T_iter          */
+#define SAILOR_OBJ_MIN_COST               1   /* minimise C_iter          */
+#define SAILOR_OBJ_MAX_THROUGHPUT_PER_USD 2   /* minimise T_iter * C_iter */
+
+#define SAILOR_FLAG_EVAL_ALL 1u  /* compute time and cost of every candidate, skipping nothing;
+                                    results are identical with or without it                */
+
+typedef struct sailor_objective {
+    uint32_t kind;
+    uint32_t flags;
+    double   budget_usd_per_iter;          /* <= 0: none                                    */
+    double   min_iters_per_s;              /* <= 0: none                                    */
+    double   budget_factor_over_cheapest;  /* > 0: first find the cheapest feasible plan
+                                              (MIN_COST, no budget), then search with budget
+                                              = factor * that cost (two passes)             */
+} sailor_objective;
+
+typedef struct sailor_result {
+    uint64_t flat;
+    double   t_iter;
+    double   cost;
+    uint64_t peak_mem;
+    double   score;
+    uint32_t status;
+    uint32_t _pad;
+    sailor_plan_rec plan;
+} sailor_result;
+
+/* Every candidate falls in exactly one class: the first of invalid, oom, over_avail,
+ * over_constraint (budget or throughput) that applies, else feasible. */
+typedef struct sailor_stats {
+    uint64_t n_total, n_invalid, n_oom, n_over_avail, n_over_constraint, n_feasible;
+    double   budget_used;       /* the budget the (last) pass ran with; <= 0 if none         */
+    float    kernel_ms;         /* device time of the search kernels (CUDA events)          */
+    uint32_t n_launches;        /* kernels launched by this call                            */
+} sailor_stats;
+
+typedef struct sailor_ctx sailor_ctx;     /* opaque; owns device copies of the tables       */
+
+/* ---- entry points --------------------------------------------------------------------- */
+
+/* Build a context on `cuda_device`.  Copies and validates the tables (HOST pointers),
+ * uploads them, and precomputes on the device the left-to-right layer sums every stage
+ * composition needs.  `cuda_stream` is a cudaStream_t (NULL = default stream) on which all
+ * later work of this context is enqueued.  Availability starts at zero everywhere.
+ * Errors: E_ARG (null, n_types mismatch, zero sizes, non-finite or negative table entry),
+ * E_RANGE (a size beyond a limit), E_CUDA, E_NOMEM. */
+int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_cluster* c,
+                  int cuda_device, void* cuda_stream, sailor_ctx** out);
+
+int sailor_destroy(sailor_ctx* ctx);      /* NULL is accepted                               */
+
+/* Replace the availability snapshot (Sec. 4: "current availability of hardware resources").
+ * `avail` is a HOST array [zone][type] of GPU counts.  The only per-snapshot upload. */
+int sailor_set_availability(sailor_ctx* ctx, const uint16_t* avail);
+
+/* Simulate n explicit plans (Sec. 4.3).  Inputs and outputs are all HOST pointers when
+ * on_device == 0 (copied both ways, stream synchronised before return) or all DEVICE
+ * pointers when on_device == 1 (work is only enqueued on the context's stream).  Outputs are
+ * arrays of n; any of them may be NULL.  t_iter and cost are NaN when SAILOR_ST_INVALID
+ * or SAILOR_ST_BAD_RECORD is set; peak_mem is the maximum over stages of the per-GPU peak
+ * (with N_b taken as floor(gbs / (D*mbs))).  A different tp per run is accepted (Sec. 4.4).
+ * Errors: E_ARG (null ctx/plans, unaligned plans), E_RANGE (host records only: an index
+ * outside its table, n_runs or P outside limits, run lengths not summing to P), E_CUDA. */
+int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, int on_device,
+                    double* t_iter, uint64_t* peak_mem, double* cost, uint32_t* status);
+
+/* Number of candidates in a space (host arithmetic).  E_RANGE if it overflows 2^63. */
+int sailor_space_size(const sailor_ctx* ctx, const sailor_space* s, uint64_t* n_out);
+
+/* Flat index -> plan record (host arithmetic), the inverse of the enumeration order. */
+int sailor_decode(const sailor_ctx* ctx, const sailor_space* s, uint64_t flat,
+                  sailor_plan_rec* out);
+
+/* Search the whole space (Sec. 4.2: evaluate candidates, keep those within the constraint,
+ * order by the objective, return the best).  Candidates are generated on the device from
+ * their flat index.  `topk` is a HOST array of k records, filled best first in
+ * (score, flat) ascending order; *n_found <= k is how many are feasible.  An empty
+ * feasible set is not an error.  `stats` may be NULL.  Synchronises the stream.
+ * Errors: E_ARG (null, k == 0, empty radix list), E_RANGE (k > SAILOR_K_MAX, an index
+ * outside its table, P > SAILOR_P_MAX, seg_max outside 1..SAILOR_SEG_MAX), E_CUDA, E_DEVICE. */
+int sailor_plan(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o,
+                uint32_t k, sailor_result* topk, uint32_t* n_found, sailor_stats* stats);
+
+/* Same over the candidates with flat index in [flat_lo, flat_hi) only, so that a space can
+ * be split over several GPUs and the per-range top-k lists merged by (score, flat).
+ * With budget_factor_over_cheapest > 0 the cheapest plan is searched in this range only;
+ * a sharded caller runs the MIN_COST pass itself and passes an explicit budget. */
+int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o,
+                      uint64_t flat_lo, uint64_t flat_hi,
+                      uint32_t k, sailor_result* topk, uint32_t* n_found, sailor_stats* stats);
+
+const char* sailor_strerror(int code);
+int sailor_last_cuda_error(const sailor_ctx* ctx);   /* cudaError_t of the last E_CUDA      */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAILOR_H */

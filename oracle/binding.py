@@ -1,0 +1,290 @@
+"""ctypes binding of the CPU oracle — TEST INFRASTRUCTURE ONLY.
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this module.
+It compiles ``sailor_oracle.c`` with gcc on first use and marshals a workload (plain numbers
+and numpy arrays) into the oracle's own structures.  It imports nothing from the CUDA
+package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sailor_oracle.c")
+_HDR = os.path.join(_HERE, "sailor_oracle.h")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+STAGES_MAX = 128
+ST_INVALID, ST_OVER_AVAIL, ST_OOM, ST_OVER_BUDGET, ST_UNDER_THROUGHPUT = 1, 2, 4, 8, 16
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (contraction off, no fast-math) if the library is missing or stale."""
+    stale = (not os.path.exists(_LIB)
+             or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR)))
+    if force or stale:
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math",
+                               "-Wall", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_dp = C.POINTER(C.c_double)
+_u64p = C.POINTER(C.c_uint64)
+_u32p = C.POINTER(C.c_uint32)
+_u16p = C.POINTER(C.c_uint16)
+
+
+class OrcInputs(C.Structure):
+    _fields_ = [
+        ("n_blocks", C.c_uint32), ("has_embed", C.c_uint32), ("has_head", C.c_uint32), ("heads", C.c_uint32),
+        ("gbs", C.c_uint64),
+        ("mul_factor", C.c_uint32), ("dtype_size", C.c_uint32), ("grad_dtype_size", C.c_uint32),
+        ("n_types", C.c_uint32), ("n_zones", C.c_uint32), ("n_tp", C.c_uint32), ("n_mbs", C.c_uint32),
+        ("tp_values", _u32p), ("mbs_values", _u32p),
+        ("fwd", _dp), ("bwd", _dp), ("upd", _dp),
+        ("params", _u64p), ("act_saved", _u64p), ("act_ckpt", _u64p), ("act_work", _u64p), ("p2p_bytes", _u64p),
+        ("capacity", _u64p), ("reserved", _u64p), ("gpus_per_node", _u32p),
+        ("price_per_hour", _dp), ("intra_alpha", _dp), ("intra_inv_bw", _dp), ("inter_alpha", _dp),
+        ("inter_inv_bw", _dp), ("zone_alpha", _dp), ("zone_inv_bw", _dp), ("egress", _dp),
+        ("avail", _u16p),
+    ]
+
+
+class OrcPlan(C.Structure):
+    _fields_ = [("P", C.c_uint32), ("mbs_idx", C.c_uint32), ("rc", C.c_uint32), ("D", C.c_uint32),
+                ("type", C.c_uint32 * STAGES_MAX), ("zone", C.c_uint32 * STAGES_MAX),
+                ("tp_idx", C.c_uint32 * STAGES_MAX)]
+
+
+class OrcOut(C.Structure):
+    _fields_ = [("status", C.c_uint32), ("_pad", C.c_uint32), ("t_iter", C.c_double), ("cost", C.c_double),
+                ("peak_mem", C.c_uint64), ("t_pp", C.c_double), ("t_sync", C.c_double),
+                ("t_update", C.c_double), ("rate_per_s", C.c_double), ("c_comm", C.c_double),
+                ("n_b", C.c_uint64), ("stage_mem", C.c_uint64 * STAGES_MAX),
+                ("stage_t", C.c_double * STAGES_MAX), ("stage_c", C.c_double * STAGES_MAX),
+                ("stage_sync", C.c_double * STAGES_MAX)]
+
+
+class OrcSpace(C.Structure):
+    _fields_ = [("n_p", C.c_uint32), ("n_mbs", C.c_uint32), ("n_tp", C.c_uint32), ("n_rc", C.c_uint32),
+                ("n_d", C.c_uint32), ("seg_max", C.c_uint32),
+                ("p_values", _u32p), ("mbs_idx", _u32p), ("tp_idx", _u32p), ("rc_values", _u32p),
+                ("d_values", _u32p)]
+
+
+class OrcObjective(C.Structure):
+    _fields_ = [("kind", C.c_uint32), ("_pad", C.c_uint32), ("budget", C.c_double), ("min_rate", C.c_double)]
+
+
+class OrcHit(C.Structure):
+    _fields_ = [("flat", C.c_uint64), ("score", C.c_double), ("t_iter", C.c_double), ("cost", C.c_double),
+                ("peak_mem", C.c_uint64)]
+
+
+class OrcCounts(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in ("n_total", "n_invalid", "n_oom", "n_over_avail",
+                                          "n_over_constraint", "n_feasible")]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        L.orc_simulate.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcPlan), C.POINTER(OrcOut)]
+        L.orc_simulate.restype = None
+        L.orc_space_size.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcSpace)]
+        L.orc_space_size.restype = C.c_uint64
+        L.orc_decode.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcSpace), C.c_uint64, C.POINTER(OrcPlan)]
+        L.orc_decode.restype = C.c_int
+        L.orc_search.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcSpace), C.POINTER(OrcObjective),
+                                 C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint32, C.POINTER(OrcHit),
+                                 C.POINTER(OrcCounts)]
+        L.orc_search.restype = C.c_uint32
+        L.orc_simulate_flat.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcSpace), _u64p, C.c_uint64,
+                                        _u32p, _dp, _dp, _u64p]
+        L.orc_simulate_flat.restype = None
+        L.orc_simulate_batch.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcPlan), C.c_uint64,
+                                         _u32p, _dp, _dp, _u64p]
+        L.orc_simulate_batch.restype = None
+        _lib = L
+    return _lib
+
+
+def _arr(a, dtype, ptr_type):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    return a, a.ctypes.data_as(ptr_type)
+
+
+class Oracle:
+    """The oracle bound to one workload's tables (kept alive here)."""
+
+    def __init__(self, w, avail: Optional[np.ndarray] = None):
+        self._keep = []
+        self.w = w
+        i = OrcInputs()
+        for name in ("n_blocks", "has_embed", "has_head", "heads", "gbs", "mul_factor", "dtype_size",
+                     "grad_dtype_size", "n_types", "n_zones"):
+            setattr(i, name, int(getattr(w, name)))
+        if w.n_blocks > 1024:
+            raise ValueError("oracle supports at most 1024 blocks")
+        i.n_tp, i.n_mbs = len(w.tp_values), len(w.mbs_values)
+
+        def put(name, value, dtype, ptr):
+            a, p = _arr(value, dtype, ptr)
+            self._keep.append(a)
+            setattr(i, name, p)
+            return a
+
+        put("tp_values", w.tp_values, np.uint32, _u32p)
+        put("mbs_values", w.mbs_values, np.uint32, _u32p)
+        for name in ("fwd", "bwd", "upd", "price_per_hour", "intra_alpha", "intra_inv_bw", "inter_alpha",
+                     "inter_inv_bw", "zone_alpha", "zone_inv_bw", "egress"):
+            put(name, getattr(w, name), np.float64, _dp)
+        for name in ("params", "act_saved", "act_ckpt", "act_work", "p2p_bytes", "capacity", "reserved"):
+            put(name, getattr(w, name), np.uint64, _u64p)
+        put("gpus_per_node", w.gpus_per_node, np.uint32, _u32p)
+        self._avail = put("avail", w.avail if avail is None else avail, np.uint16, _u16p)
+        self.inputs = i
+
+        s = OrcSpace()
+        s.n_p, s.n_mbs, s.n_tp = len(w.p_values), len(w.mbs_idx), len(w.tp_idx)
+        s.n_rc, s.n_d, s.seg_max = len(w.rc_values), len(w.d_values), w.seg_max
+        for name in ("p_values", "mbs_idx", "tp_idx", "rc_values", "d_values"):
+            a, p = _arr(getattr(w, name), np.uint32, _u32p)
+            self._keep.append(a)
+            setattr(s, name, p)
+        self.space = s
+
+    def set_availability(self, avail) -> None:
+        self._avail[...] = np.asarray(avail, dtype=np.uint16).reshape(self._avail.shape)
+
+    # -- single plans -------------------------------------------------------------------
+    @staticmethod
+    def make_plan(P: int, mbs_idx: int, rc: int, D: int, types: Sequence[int], zones: Sequence[int],
+                  tp_idx: Sequence[int]) -> OrcPlan:
+        pl = OrcPlan()
+        pl.P, pl.mbs_idx, pl.rc, pl.D = P, mbs_idx, rc, D
+        for j in range(P):
+            pl.type[j], pl.zone[j], pl.tp_idx[j] = int(types[j]), int(zones[j]), int(tp_idx[j])
+        return pl
+
+    def simulate(self, plan: OrcPlan) -> OrcOut:
+        out = OrcOut()
+        lib().orc_simulate(C.byref(self.inputs), C.byref(plan), C.byref(out))
+        return out
+
+    def space_size(self) -> int:
+        return int(lib().orc_space_size(C.byref(self.inputs), C.byref(self.space)))
+
+    def decode(self, flat: int) -> OrcPlan:
+        pl = OrcPlan()
+        if lib().orc_decode(C.byref(self.inputs), C.byref(self.space), flat, C.byref(pl)) != 0:
+            raise IndexError(flat)
+        return pl
+
+    # -- batches ------------------------------------------------------------------------
+    def simulate_flat(self, flat) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+        flat = np.ascontiguousarray(flat, dtype=np.uint64)
+        n = flat.size
+        st = np.zeros(n, np.uint32); t = np.zeros(n); c = np.zeros(n); m = np.zeros(n, np.uint64)
+        lib().orc_simulate_flat(C.byref(self.inputs), C.byref(self.space), flat.ctypes.data_as(_u64p), n,
+                                st.ctypes.data_as(_u32p), t.ctypes.data_as(_dp), c.ctypes.data_as(_dp),
+                                m.ctypes.data_as(_u64p))
+        return st, t, c, m
+
+    def simulate_records(self, recs: dict):
+        """Simulate run-length encoded records (the dict layout of workloads.random_plans)."""
+        n = len(recs["P"])
+        plans = (OrcPlan * n)()
+        for j in range(n):
+            pl = plans[j]
+            pl.P, pl.mbs_idx, pl.rc, pl.D = (int(recs["P"][j]), int(recs["mbs_idx"][j]), int(recs["rc"][j]),
+                                             int(recs["D"][j]))
+            i = 0
+            for r in range(int(recs["n_runs"][j])):
+                for _ in range(int(recs["n_stages"][j, r])):
+                    pl.type[i] = int(recs["type"][j, r])
+                    pl.zone[i] = int(recs["zone"][j, r])
+                    pl.tp_idx[i] = int(recs["tp_idx"][j, r])
+                    i += 1
+        st = np.zeros(n, np.uint32); t = np.zeros(n); c = np.zeros(n); m = np.zeros(n, np.uint64)
+        lib().orc_simulate_batch(C.byref(self.inputs), plans, n, st.ctypes.data_as(_u32p),
+                                 t.ctypes.data_as(_dp), c.ctypes.data_as(_dp), m.ctypes.data_as(_u64p))
+        return st, t, c, m
+
+    # -- search -------------------------------------------------------------------------
+    def search(self, kind: int, k: int, *, budget: float = 0.0, min_rate: float = 0.0, lo: int = 0,
+               hi: Optional[int] = None, stride: int = 1):
+        """One exhaustive pass over [lo, hi): returns (hits as list of dicts, counts dict)."""
+        hi = self.space_size() if hi is None else hi
+        obj = OrcObjective(kind, 0, budget, min_rate)
+        hits = (OrcHit * max(k, 1))()
+        cnt = OrcCounts()
+        n = lib().orc_search(C.byref(self.inputs), C.byref(self.space), C.byref(obj), lo, hi, stride, k,
+                             hits, C.byref(cnt))
+        out = [dict(flat=int(h.flat), score=h.score, t_iter=h.t_iter, cost=h.cost, peak_mem=int(h.peak_mem))
+               for h in hits[:n]]
+        return out, {f: int(getattr(cnt, f)) for f, _ in OrcCounts._fields_}
+
+    def plan(self, k: int, *, lo: int = 0, hi: Optional[int] = None):
+        """The workload's own objective, with the cheapest-feasible budget rule when it has one:
+        pass 1 minimises cost without a budget, pass 2 runs the objective under
+        budget = factor x that cost (Sec. 5.2.4, scenario 2 shape)."""
+        w = self.w
+        budget = w.budget_usd_per_iter
+        if w.budget_factor_over_cheapest > 0.0:
+            cheapest, _ = self.search(1, 1, lo=lo, hi=hi)
+            if not cheapest:
+                return [], {"n_feasible": 0}, 0.0
+            budget = w.budget_factor_over_cheapest * cheapest[0]["cost"]
+        hits, counts = self.search(w.objective, k, budget=budget, min_rate=w.min_iters_per_s, lo=lo, hi=hi)
+        return hits, counts, budget
+
+
+def merge_hits(lists: List[list], k: int) -> list:
+    """Merge per-range top-k lists by (score, flat)."""
+    allh = [h for l in lists for h in l]
+    allh.sort(key=lambda h: (h["score"], h["flat"]))
+    return allh[:k]
+
+
+def _search_range(args):
+    w, avail, kind, k, budget, min_rate, lo, hi = args
+    o = Oracle(w, avail)
+    return o.search(kind, k, budget=budget, min_rate=min_rate, lo=lo, hi=hi)
+
+
+def parallel_search(w, kind: int, k: int, *, budget: float = 0.0, min_rate: float = 0.0, avail=None,
+                    procs: int = 0, pool=None):
+    """The same exhaustive pass split by flat range over worker processes (spawned)."""
+    import multiprocessing as mp
+    n = Oracle(w, avail).space_size()
+    procs = procs or os.cpu_count() or 1
+    chunks = max(procs * 8, 1)
+    edges = [n * j // chunks for j in range(chunks + 1)]
+    tasks = [(w, avail, kind, k, budget, min_rate, edges[j], edges[j + 1]) for j in range(chunks)]
+    own = pool is None
+    if own:
+        pool = mp.get_context("spawn").Pool(procs)
+    try:
+        parts = pool.map(_search_range, tasks)
+    finally:
+        if own:
+            pool.close()
+            pool.join()
+    hits = merge_hits([p[0] for p in parts], k)
+    counts = {}
+    for _, c in parts:
+        for key, v in c.items():
+            counts[key] = counts.get(key, 0) + v
+    return hits, counts

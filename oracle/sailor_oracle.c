@@ -1,0 +1,307 @@
+/*
+ * sailor_oracle.c — TEST INFRASTRUCTURE ONLY (see sailor_oracle.h).
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -shared -fPIC
+ * All times and costs are IEEE binary64, every sum runs left to right in stage order,
+ * bytes and counts are 64-bit unsigned integers.
+ */
+#include "sailor_oracle.h"
+
+#include <math.h>
+#include <string.h>
+
+static uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+static uint64_t min_u64(uint64_t a, uint64_t b) { return a < b ? a : b; }
+static double max_f64(double a, double b) { return a > b ? a : b; }
+
+/* table lookups, index order as declared in orc_inputs */
+static double tab4(const orc_inputs* in, const double* t, uint32_t kind, uint32_t g, uint32_t tp, uint32_t mbs) {
+    return t[((kind * in->n_types + g) * in->n_tp + tp) * in->n_mbs + mbs];
+}
+static double tab_upd(const orc_inputs* in, uint32_t kind, uint32_t g, uint32_t tp) {
+    return in->upd[(kind * in->n_types + g) * in->n_tp + tp];
+}
+static uint64_t tab_act(const orc_inputs* in, const uint64_t* t, uint32_t kind, uint32_t tp, uint32_t mbs) {
+    return t[(kind * in->n_tp + tp) * in->n_mbs + mbs];
+}
+
+/* The layers of stage i of a P-stage pipeline, as a list of kinds.
+ * Uniform split of the blocks, the remainder going one each to the first stages; the
+ * embedding opens stage 0 and the head closes stage P-1 (Sec. 4.1: repeated layers are
+ * profiled once, non-uniform ones separately). */
+static uint32_t stage_layers(const orc_inputs* in, uint32_t P, uint32_t i, uint8_t* kinds) {
+    uint32_t n = 0;
+    uint32_t blocks = in->n_blocks / P + (i < in->n_blocks % P ? 1u : 0u);
+    if (i == 0 && in->has_embed) kinds[n++] = 0;
+    for (uint32_t j = 0; j < blocks; ++j) kinds[n++] = 1;
+    if (i == P - 1 && in->has_head) kinds[n++] = 2;
+    return n;
+}
+
+/* time of one message of `bytes` over a link: degree-1 fit of Sec. 4.1's bandwidth profile */
+static double link_time(double alpha, double inv_bw, uint64_t bytes) {
+    return alpha + (double)bytes * inv_bw;
+}
+
+void orc_simulate(const orc_inputs* in, const orc_plan* pl, orc_out* out) {
+    static uint8_t kinds[ORC_STAGES_MAX][1024 + 2];
+    uint32_t nl[ORC_STAGES_MAX];
+    const uint32_t P = pl->P, T = in->n_types, Z = in->n_zones;
+    const uint32_t mbs_idx = pl->mbs_idx, D = pl->D, rc = pl->rc;
+    const uint64_t mbs = in->mbs_values[mbs_idx];
+    uint32_t status = 0;
+    out->t_pp = out->t_sync = out->t_update = out->rate_per_s = out->c_comm = 0.0;
+
+    /* validity: the global batch is never changed (Sec. 4.2), tensor parallelism stays in
+     * one node (H1), attention heads split evenly */
+    if (D == 0 || in->gbs % ((uint64_t)D * mbs) != 0) status |= ORC_INVALID;
+    for (uint32_t i = 0; i < P; ++i) {
+        uint32_t tp = in->tp_values[pl->tp_idx[i]];
+        if (tp > in->gpus_per_node[pl->type[i]]) status |= ORC_INVALID;
+        if (in->heads % tp != 0) status |= ORC_INVALID;
+    }
+    const uint64_t n_b = D ? in->gbs / ((uint64_t)D * mbs) : 0;
+    out->n_b = n_b;
+
+    /* resources: every stage takes D replicas of tp GPUs of its (zone, type) (H3: same D) */
+    uint64_t used[64 * 64];
+    memset(used, 0, sizeof(uint64_t) * Z * T);
+    for (uint32_t i = 0; i < P; ++i)
+        used[pl->zone[i] * T + pl->type[i]] += (uint64_t)D * in->tp_values[pl->tp_idx[i]];
+    for (uint32_t d = 0; d < Z * T; ++d)
+        if (used[d] > in->avail[d]) status |= ORC_OVER_AVAIL;
+
+    /* memory per worker of each stage, Sec. 4.3: M_peak = M_model + M_activation */
+    uint64_t params_stage[ORC_STAGES_MAX];
+    uint64_t peak = 0;
+    for (uint32_t i = 0; i < P; ++i) {
+        nl[i] = stage_layers(in, P, i, kinds[i]);
+        uint32_t g = pl->type[i], tpi = pl->tp_idx[i];
+        uint64_t tp = in->tp_values[tpi];
+        uint64_t params = 0, A = 0, W = 0;
+        for (uint32_t l = 0; l < nl[i]; ++l) {
+            uint32_t k = kinds[i][l];
+            params += in->params[k];
+            A += rc ? tab_act(in, in->act_ckpt, k, tpi, mbs_idx) : tab_act(in, in->act_saved, k, tpi, mbs_idx);
+            uint64_t w = rc ? tab_act(in, in->act_saved, k, tpi, mbs_idx) : tab_act(in, in->act_work, k, tpi, mbs_idx);
+            if (w > W) W = w;
+        }
+        params_stage[i] = params;
+        uint64_t m_model = ceil_div_u64(params, tp) * in->mul_factor * in->dtype_size;
+        uint64_t inflight = min_u64((uint64_t)(P - i), n_b);   /* 1F1B: stage i keeps P-i microbatches */
+        uint64_t m = m_model + inflight * A + W + in->reserved[g];
+        out->stage_mem[i] = m;
+        if (m > in->capacity[g]) status |= ORC_OOM;
+        if (m > peak) peak = m;
+    }
+    out->peak_mem = peak;
+    out->status = status;
+    if (status & ORC_INVALID) {
+        out->t_iter = NAN;
+        out->cost = NAN;
+        return;
+    }
+
+    /* iteration time, Sec. 4.3: T_iter = max(T_pp) + T_sync + T_update, all pipelines alike */
+    const uint64_t msg = in->p2p_bytes[mbs_idx];
+    double sum_t = 0.0, max_t = 0.0, max_sync = 0.0, max_u = 0.0;
+    for (uint32_t i = 0; i < P; ++i) {
+        uint32_t g = pl->type[i], z = pl->zone[i], tpi = pl->tp_idx[i];
+        uint32_t tp = in->tp_values[tpi];
+        double f = 0.0, b = 0.0, u = 0.0;
+        for (uint32_t l = 0; l < nl[i]; ++l) {
+            uint32_t k = kinds[i][l];
+            f = f + tab4(in, in->fwd, k, g, tpi, mbs_idx);
+            b = b + tab4(in, in->bwd, k, g, tpi, mbs_idx);
+            u = u + tab_upd(in, k, g, tpi);
+        }
+        if (rc) b = b + f;                 /* recomputation re-runs the forward pass */
+
+        /* activation to the next stage and its gradient back over the same link */
+        double c = 0.0;
+        if (i + 1 < P) {
+            uint32_t g2 = pl->type[i + 1], z2 = pl->zone[i + 1];
+            uint32_t tp2 = in->tp_values[pl->tp_idx[i + 1]];
+            if (z != z2) {
+                c = link_time(in->zone_alpha[z * Z + z2], in->zone_inv_bw[z * Z + z2], msg);
+            } else if (g == g2 && (uint64_t)D * (tp + tp2) <= in->gpus_per_node[g]) {
+                c = link_time(in->intra_alpha[z * T + g], in->intra_inv_bw[z * T + g], msg);
+            } else {
+                double c1 = link_time(in->inter_alpha[z * T + g], in->inter_inv_bw[z * T + g], msg);
+                double c2 = link_time(in->inter_alpha[z * T + g2], in->inter_inv_bw[z * T + g2], msg);
+                c = max_f64(c1, c2);
+            }
+        }
+        double t = (f + b) + 2.0 * c;
+        out->stage_c[i] = c;
+        out->stage_t[i] = t;
+        sum_t = sum_t + t;                 /* warm-up and cool-down: every stage once (Sec. 4.2.3) */
+        max_t = max_f64(max_t, t);         /* the straggler sets the steady phase */
+        max_u = max_f64(max_u, u);
+
+        /* ring all-reduce of the stage's gradients among its D replicas, inside one zone (H5) */
+        double sync = 0.0;
+        if (D > 1) {
+            uint64_t gradbytes = ceil_div_u64(params_stage[i], tp) * in->grad_dtype_size;
+            double alpha, inv;
+            if ((uint64_t)D * tp <= in->gpus_per_node[g]) {
+                alpha = in->intra_alpha[z * T + g];
+                inv = in->intra_inv_bw[z * T + g];
+            } else {
+                alpha = in->inter_alpha[z * T + g];
+                inv = in->inter_inv_bw[z * T + g];
+            }
+            double steps = (double)(2 * (uint64_t)(D - 1));
+            double coef = steps / (double)D;
+            sync = (coef * (double)gradbytes) * inv + steps * alpha;
+        }
+        out->stage_sync[i] = sync;
+        max_sync = max_f64(max_sync, sync);
+    }
+    double t_pp = sum_t + (double)n_b * max_t;          /* T_total of Sec. 4.2.2 without sync */
+    double t_iter = (t_pp + max_sync) + max_u;
+    out->t_pp = t_pp;
+    out->t_sync = max_sync;
+    out->t_update = max_u;
+    out->t_iter = t_iter;
+
+    /* cost per iteration, Sec. 4.3: C_iter = C_comp + C_comm */
+    double rate = 0.0;                                  /* dollars per second of all GPUs */
+    for (uint32_t i = 0; i < P; ++i) {
+        uint32_t n_gpus = D * in->tp_values[pl->tp_idx[i]];
+        double per_s = in->price_per_hour[pl->zone[i] * T + pl->type[i]] / 3600.0;
+        rate = rate + (double)n_gpus * per_s;
+    }
+    double c_comm = 0.0;
+    for (uint32_t i = 0; i + 1 < P; ++i) {
+        uint32_t z = pl->zone[i], z2 = pl->zone[i + 1];
+        if (z != z2) {
+            uint64_t bytes = 2 * n_b * (uint64_t)D * msg;    /* forward and backward, all microbatches, all replicas */
+            c_comm = c_comm + (double)bytes * in->egress[z * Z + z2];
+        }
+    }
+    out->rate_per_s = rate;
+    out->c_comm = c_comm;
+    out->cost = rate * t_iter + c_comm;
+}
+
+static uint64_t ipow_u64(uint64_t b, uint32_t e) {
+    uint64_t r = 1;
+    while (e--) r *= b;
+    return r;
+}
+static uint32_t nseg_of(const orc_space* sp, uint32_t P) { return P < sp->seg_max ? P : sp->seg_max; }
+
+uint64_t orc_space_size(const orc_inputs* in, const orc_space* sp) {
+    uint64_t radix = (uint64_t)in->n_types * in->n_zones;
+    uint64_t base = (uint64_t)sp->n_mbs * sp->n_tp * sp->n_rc * sp->n_d;
+    uint64_t n = 0;
+    for (uint32_t j = 0; j < sp->n_p; ++j) n += base * ipow_u64(radix, nseg_of(sp, sp->p_values[j]));
+    return n;
+}
+
+/* Flat index -> plan.  The sub-spaces of the P values follow one another; inside one, the
+ * digits from the lowest are: segment nseg-1 ... segment 0 (radix T*Z, digit = zone*T+type),
+ * D, recomputation, tp, mbs.  Stage i takes segment floor(i*nseg/P). */
+int orc_decode(const orc_inputs* in, const orc_space* sp, uint64_t flat, orc_plan* pl) {
+    uint64_t radix = (uint64_t)in->n_types * in->n_zones;
+    uint64_t base = (uint64_t)sp->n_mbs * sp->n_tp * sp->n_rc * sp->n_d;
+    for (uint32_t j = 0; j < sp->n_p; ++j) {
+        uint32_t P = sp->p_values[j];
+        uint32_t nseg = nseg_of(sp, P);
+        uint64_t sub = base * ipow_u64(radix, nseg);
+        if (flat >= sub) { flat -= sub; continue; }
+        uint32_t seg[ORC_SEG_MAX];
+        for (uint32_t s = nseg; s-- > 0;) { seg[s] = (uint32_t)(flat % radix); flat /= radix; }
+        uint32_t di = (uint32_t)(flat % sp->n_d);   flat /= sp->n_d;
+        uint32_t ri = (uint32_t)(flat % sp->n_rc);  flat /= sp->n_rc;
+        uint32_t ti = (uint32_t)(flat % sp->n_tp);  flat /= sp->n_tp;
+        uint32_t mi = (uint32_t)flat;
+        pl->P = P;
+        pl->mbs_idx = sp->mbs_idx[mi];
+        pl->rc = sp->rc_values[ri];
+        pl->D = sp->d_values[di];
+        for (uint32_t i = 0; i < P; ++i) {
+            uint32_t s = (uint32_t)(((uint64_t)i * nseg) / P);
+            pl->type[i] = seg[s] % in->n_types;
+            pl->zone[i] = seg[s] / in->n_types;
+            pl->tp_idx[i] = sp->tp_idx[ti];
+        }
+        return 0;
+    }
+    return -1;
+}
+
+static int hit_before(const orc_hit* a, double score, uint64_t flat) {
+    return a->score < score || (a->score == score && a->flat < flat);
+}
+
+uint32_t orc_search(const orc_inputs* in, const orc_space* sp, const orc_objective* obj,
+                    uint64_t lo, uint64_t hi, uint64_t stride, uint32_t k, orc_hit* hits,
+                    orc_counts* counts) {
+    orc_plan pl;
+    orc_out o;
+    uint32_t n_hits = 0;
+    orc_counts c;
+    memset(&c, 0, sizeof(c));
+    if (stride == 0) stride = 1;
+    for (uint64_t flat = lo; flat < hi; flat += stride) {
+        if (orc_decode(in, sp, flat, &pl) != 0) break;
+        orc_simulate(in, &pl, &o);
+        c.n_total++;
+        if (o.status & ORC_INVALID) { c.n_invalid++; continue; }
+        if (o.status & ORC_OOM) { c.n_oom++; continue; }
+        if (o.status & ORC_OVER_AVAIL) { c.n_over_avail++; continue; }
+        /* the planner keeps a configuration only when it is within the constraint (Sec. 4.2) */
+        int over = 0;
+        if (obj->budget > 0.0 && o.cost > obj->budget) over = 1;
+        if (obj->min_rate > 0.0 && 1.0 / o.t_iter < obj->min_rate) over = 1;
+        if (over) { c.n_over_constraint++; continue; }
+        c.n_feasible++;
+        double score = obj->kind == ORC_OBJ_TIME ? o.t_iter
+                     : obj->kind == ORC_OBJ_COST ? o.cost
+                                                 : o.t_iter * o.cost;
+        /* sorted insertion: (score, flat) ascending, keep k (Sec. 4.2: sort by objective) */
+        if (k == 0) continue;
+        if (n_hits == k && hit_before(&hits[k - 1], score, flat)) continue;
+        uint32_t pos = n_hits < k ? n_hits : k - 1;
+        while (pos > 0 && !hit_before(&hits[pos - 1], score, flat)) {
+            hits[pos] = hits[pos - 1];
+            pos--;
+        }
+        hits[pos].flat = flat;
+        hits[pos].score = score;
+        hits[pos].t_iter = o.t_iter;
+        hits[pos].cost = o.cost;
+        hits[pos].peak_mem = o.peak_mem;
+        if (n_hits < k) n_hits++;
+    }
+    if (counts) *counts = c;
+    return n_hits;
+}
+
+void orc_simulate_flat(const orc_inputs* in, const orc_space* sp, const uint64_t* flat, uint64_t n,
+                       uint32_t* status, double* t_iter, double* cost, uint64_t* peak_mem) {
+    orc_plan pl;
+    orc_out o;
+    for (uint64_t j = 0; j < n; ++j) {
+        if (orc_decode(in, sp, flat[j], &pl) != 0) { status[j] = 0xFFFFFFFFu; continue; }
+        orc_simulate(in, &pl, &o);
+        status[j] = o.status;
+        t_iter[j] = o.t_iter;
+        cost[j] = o.cost;
+        peak_mem[j] = o.peak_mem;
+    }
+}
+
+void orc_simulate_batch(const orc_inputs* in, const orc_plan* plans, uint64_t n,
+                        uint32_t* status, double* t_iter, double* cost, uint64_t* peak_mem) {
+    orc_out o;
+    for (uint64_t j = 0; j < n; ++j) {
+        orc_simulate(in, &plans[j], &o);
+        status[j] = o.status;
+        t_iter[j] = o.t_iter;
+        cost[j] = o.cost;
+        peak_mem[j] = o.peak_mem;
+    }
+}

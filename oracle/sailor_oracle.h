@@ -1,0 +1,137 @@
+/*
+ * sailor_oracle.h — TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-threaded CPU statement of what the Sailor plan simulator and the
+ * exhaustive plan search compute (Sailor, SOSP'25: Sec. 4.2 planner overview and H1-H5,
+ * Sec. 4.2.2 T_total, Sec. 4.2.3 cost constraint, Sec. 4.3 simulator).  It exists to check the
+ * CUDA library; it shares no source, header, table or helper with it and nothing in the
+ * product may call it.  Every stage of every plan is walked layer by layer; nothing is
+ * cached, blocked, fused or reordered.
+ *
+ * Pins (see tests, all run without a GPU): three hand-computed two-stage cases and one
+ * hand-computed three-stage case with embedding/head layers, recomputation, alpha > 0 and
+ * mixed tensor parallelism; the homogeneous closed form (P + N_b) * t; monotonicity and
+ * scaling invariants; an independent nested-loop enumeration and brute-force minimum on
+ * tiny clusters.
+ * Parity unpinned: the absolute realism of the outputs against real clusters (Sec. 5.1
+ * reports 4-6 % error on hardware this repository cannot reach).
+ */
+#ifndef SAILOR_ORACLE_H
+#define SAILOR_ORACLE_H
+
+#include <stdint.h>
+
+#define ORC_KINDS 3            /* 0 embedding, 1 transformer block, 2 head */
+#define ORC_STAGES_MAX 128
+#define ORC_SEG_MAX 8
+
+/* status bits */
+#define ORC_INVALID 1u
+#define ORC_OVER_AVAIL 2u
+#define ORC_OOM 4u
+#define ORC_OVER_BUDGET 8u
+#define ORC_UNDER_THROUGHPUT 16u
+
+/* objective kinds: what is minimised */
+#define ORC_OBJ_TIME 0           /* maximise throughput            */
+#define ORC_OBJ_COST 1           /* minimise cost per iteration    */
+#define ORC_OBJ_TIME_X_COST 2    /* maximise throughput per dollar */
+
+typedef struct orc_inputs {
+    /* training job */
+    uint32_t n_blocks, has_embed, has_head, heads;
+    uint64_t gbs;
+    uint32_t mul_factor, dtype_size, grad_dtype_size;
+    /* table shapes */
+    uint32_t n_types, n_zones, n_tp, n_mbs;
+    const uint32_t* tp_values;     /* [n_tp]  */
+    const uint32_t* mbs_values;    /* [n_mbs] */
+    /* per-layer profile, Sec. 4.1 */
+    const double* fwd;             /* [kind][type][tp][mbs] */
+    const double* bwd;             /* [kind][type][tp][mbs] */
+    const double* upd;             /* [kind][type][tp]      */
+    const uint64_t* params;        /* [kind]                */
+    const uint64_t* act_saved;     /* [kind][tp][mbs]       */
+    const uint64_t* act_ckpt;      /* [kind][tp][mbs]       */
+    const uint64_t* act_work;      /* [kind][tp][mbs]       */
+    const uint64_t* p2p_bytes;     /* [mbs]                 */
+    /* cluster */
+    const uint64_t* capacity;      /* [type] */
+    const uint64_t* reserved;      /* [type] */
+    const uint32_t* gpus_per_node; /* [type] */
+    const double* price_per_hour;  /* [zone][type] */
+    const double* intra_alpha;     /* [zone][type] */
+    const double* intra_inv_bw;
+    const double* inter_alpha;
+    const double* inter_inv_bw;
+    const double* zone_alpha;      /* [zone][zone] */
+    const double* zone_inv_bw;
+    const double* egress;          /* [zone][zone] dollars per byte */
+    const uint16_t* avail;         /* [zone][type] */
+} orc_inputs;
+
+/* a plan with every stage written out */
+typedef struct orc_plan {
+    uint32_t P, mbs_idx, rc, D;
+    uint32_t type[ORC_STAGES_MAX];
+    uint32_t zone[ORC_STAGES_MAX];
+    uint32_t tp_idx[ORC_STAGES_MAX];
+} orc_plan;
+
+typedef struct orc_out {
+    uint32_t status;
+    uint32_t _pad;
+    double t_iter;
+    double cost;
+    uint64_t peak_mem;
+    /* intermediate quantities, for the hand-computed pins */
+    double t_pp, t_sync, t_update, rate_per_s, c_comm;
+    uint64_t n_b;
+    uint64_t stage_mem[ORC_STAGES_MAX];
+    double stage_t[ORC_STAGES_MAX];
+    double stage_c[ORC_STAGES_MAX];
+    double stage_sync[ORC_STAGES_MAX];
+} orc_out;
+
+typedef struct orc_space {
+    uint32_t n_p, n_mbs, n_tp, n_rc, n_d, seg_max;
+    const uint32_t* p_values;
+    const uint32_t* mbs_idx;
+    const uint32_t* tp_idx;
+    const uint32_t* rc_values;
+    const uint32_t* d_values;
+} orc_space;
+
+typedef struct orc_objective {
+    uint32_t kind;
+    uint32_t _pad;
+    double budget;        /* dollars per iteration, <= 0: none */
+    double min_rate;      /* iterations per second, <= 0: none */
+} orc_objective;
+
+typedef struct orc_hit {
+    uint64_t flat;
+    double score, t_iter, cost;
+    uint64_t peak_mem;
+} orc_hit;
+
+typedef struct orc_counts {
+    uint64_t n_total, n_invalid, n_oom, n_over_avail, n_over_constraint, n_feasible;
+} orc_counts;
+
+void orc_simulate(const orc_inputs* in, const orc_plan* plan, orc_out* out);
+uint64_t orc_space_size(const orc_inputs* in, const orc_space* sp);
+int orc_decode(const orc_inputs* in, const orc_space* sp, uint64_t flat, orc_plan* plan);
+/* walk flat indices lo <= flat < hi in steps of `stride`; keep the k best feasible plans in
+ * (score, flat) ascending order; returns how many were kept */
+uint32_t orc_search(const orc_inputs* in, const orc_space* sp, const orc_objective* obj,
+                    uint64_t lo, uint64_t hi, uint64_t stride, uint32_t k, orc_hit* hits,
+                    orc_counts* counts);
+/* simulate chosen flat indices: out arrays of n */
+void orc_simulate_flat(const orc_inputs* in, const orc_space* sp, const uint64_t* flat, uint64_t n,
+                       uint32_t* status, double* t_iter, double* cost, uint64_t* peak_mem);
+/* simulate n written-out plans */
+void orc_simulate_batch(const orc_inputs* in, const orc_plan* plans, uint64_t n,
+                        uint32_t* status, double* t_iter, double* cost, uint64_t* peak_mem);
+
+#endif
