@@ -186,6 +186,7 @@ typedef struct sailor_result {
 typedef struct sailor_stats {
     uint64_t n_total, n_invalid, n_oom, n_over_avail, n_over_constraint, n_feasible;
     double   budget_used;       /* the budget the (last) pass ran with; <= 0 if none         */
+    double   min_feasible_cost; /* smallest C_iter among the feasible candidates; 0 if none */
     float    kernel_ms;         /* device time of the search kernels (CUDA events)          */
     uint32_t n_launches;        /* kernels launched by this call                            */
 } sailor_stats;

@@ -90,7 +90,7 @@ class OrcHit(C.Structure):
 
 class OrcCounts(C.Structure):
     _fields_ = [(n, C.c_uint64) for n in ("n_total", "n_invalid", "n_oom", "n_over_avail",
-                                          "n_over_constraint", "n_feasible")]
+                                          "n_over_constraint", "n_feasible")] + [("min_cost", C.c_double)]
 
 
 _lib = None
@@ -153,7 +153,8 @@ class Oracle:
         for name in ("params", "act_saved", "act_ckpt", "act_work", "p2p_bytes", "capacity", "reserved"):
             put(name, getattr(w, name), np.uint64, _u64p)
         put("gpus_per_node", w.gpus_per_node, np.uint32, _u32p)
-        self._avail = put("avail", w.avail if avail is None else avail, np.uint16, _u16p)
+        self._avail = put("avail", np.array(w.avail if avail is None else avail, dtype=np.uint16, copy=True),
+                          np.uint16, _u16p)
         self.inputs = i
 
         s = OrcSpace()
@@ -234,7 +235,7 @@ class Oracle:
                              hits, C.byref(cnt))
         out = [dict(flat=int(h.flat), score=h.score, t_iter=h.t_iter, cost=h.cost, peak_mem=int(h.peak_mem))
                for h in hits[:n]]
-        return out, {f: int(getattr(cnt, f)) for f, _ in OrcCounts._fields_}
+        return out, {f: (getattr(cnt, f) if f == "min_cost" else int(getattr(cnt, f))) for f, _ in OrcCounts._fields_}
 
     def plan(self, k: int, *, lo: int = 0, hi: Optional[int] = None):
         """The workload's own objective, with the cheapest-feasible budget rule when it has one:
@@ -286,5 +287,8 @@ def parallel_search(w, kind: int, k: int, *, budget: float = 0.0, min_rate: floa
     counts = {}
     for _, c in parts:
         for key, v in c.items():
-            counts[key] = counts.get(key, 0) + v
+            if key != "min_cost":
+                counts[key] = counts.get(key, 0) + v
+    costs = [c["min_cost"] for _, c in parts if c["n_feasible"]]
+    counts["min_cost"] = min(costs) if costs else 0.0
     return hits, counts

@@ -258,6 +258,7 @@ uint32_t orc_search(const orc_inputs* in, const orc_space* sp, const orc_objecti
         if (obj->min_rate > 0.0 && 1.0 / o.t_iter < obj->min_rate) over = 1;
         if (over) { c.n_over_constraint++; continue; }
         c.n_feasible++;
+        if (c.n_feasible == 1 || o.cost < c.min_cost) c.min_cost = o.cost;
         double score = obj->kind == ORC_OBJ_TIME ? o.t_iter
                      : obj->kind == ORC_OBJ_COST ? o.cost
                                                  : o.t_iter * o.cost;

@@ -117,6 +117,7 @@ typedef struct orc_hit {
 
 typedef struct orc_counts {
     uint64_t n_total, n_invalid, n_oom, n_over_avail, n_over_constraint, n_feasible;
+    double min_cost;      /* smallest cost among the feasible plans, 0 if there is none */
 } orc_counts;
 
 void orc_simulate(const orc_inputs* in, const orc_plan* plan, orc_out* out);

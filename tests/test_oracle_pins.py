@@ -290,7 +290,7 @@ def test_search_equals_brute_force(objective):
     assert [(h["score"], h["flat"]) for h in hits] == [r[:2] for r in rows[:10]]
     assert [(h["t_iter"], h["cost"], h["peak_mem"]) for h in hits] == [r[2:] for r in rows[:10]]
     assert counts == dict(n_total=o.space_size(), n_invalid=n_inv, n_oom=n_oom, n_over_avail=n_av,
-                          n_over_constraint=0, n_feasible=len(rows))
+                          n_over_constraint=0, n_feasible=len(rows), min_cost=min(r[3] for r in rows))
     # k larger than the feasible set returns them all, sorted
     hits_all, _ = o.search(objective, len(rows) + 5)
     assert [h["flat"] for h in hits_all] == [r[1] for r in rows]
