@@ -1,0 +1,268 @@
+"""ctypes binding of the C ABI in include/sailor.h: the same entry points, arguments marshalled
+from numpy arrays / raw device pointers.  No step of the simulation runs here, and there is no
+fallback: if the CUDA library is missing, loading it fails loudly."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import numpy as np
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libsailor_b200.so")
+
+KINDS, T_MAX, Z_MAX, TP_MAX, MBS_MAX, P_MAX, RUN_MAX, SEG_MAX, K_MAX, NP_MAX, ND_MAX = 3, 8, 8, 8, 16, 96, 16, 4, 32, 32, 32
+OK, E_ARG, E_RANGE, E_CUDA, E_NOMEM, E_DEVICE = 0, -1, -2, -3, -4, -5
+ST_INVALID, ST_OVER_AVAIL, ST_OOM, ST_OVER_BUDGET, ST_UNDER_THROUGHPUT, ST_BAD_RECORD = 1, 2, 4, 8, 16, 32
+OBJ_MAX_THROUGHPUT, OBJ_MIN_COST, OBJ_MAX_THROUGHPUT_PER_USD = 0, 1, 2
+FLAG_EVAL_ALL = 1
+
+EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
+           "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_strerror",
+           "sailor_last_cuda_error")
+
+_dp, _u64p, _u32p, _u16p = C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.POINTER(C.c_uint16)
+
+
+class Model(C.Structure):
+    _fields_ = [("n_blocks", C.c_uint32), ("has_embed", C.c_uint32), ("has_head", C.c_uint32), ("heads", C.c_uint32),
+                ("gbs", C.c_uint64), ("mul_factor", C.c_uint32), ("dtype_size", C.c_uint32),
+                ("grad_dtype_size", C.c_uint32), ("_pad", C.c_uint32)]
+
+
+class Profile(C.Structure):
+    _fields_ = [("n_types", C.c_uint32), ("n_tp", C.c_uint32), ("n_mbs", C.c_uint32), ("_pad", C.c_uint32),
+                ("tp_values", C.c_uint32 * TP_MAX), ("mbs_values", C.c_uint32 * MBS_MAX),
+                ("fwd", _dp), ("bwd", _dp), ("upd", _dp), ("params", _u64p), ("act_saved", _u64p),
+                ("act_ckpt", _u64p), ("act_work", _u64p), ("p2p_bytes", _u64p)]
+
+
+class Cluster(C.Structure):
+    _fields_ = [("n_types", C.c_uint32), ("n_zones", C.c_uint32), ("capacity", _u64p), ("reserved", _u64p),
+                ("gpus_per_node", _u32p), ("price_per_hour", _dp), ("intra_alpha", _dp), ("intra_inv_bw", _dp),
+                ("inter_alpha", _dp), ("inter_inv_bw", _dp), ("zone_alpha", _dp), ("zone_inv_bw", _dp),
+                ("egress", _dp)]
+
+
+class Run(C.Structure):
+    _fields_ = [("type", C.c_uint8), ("zone", C.c_uint8), ("tp_idx", C.c_uint8), ("n_stages", C.c_uint8)]
+
+
+class PlanRec(C.Structure):
+    _fields_ = [("P", C.c_uint8), ("mbs_idx", C.c_uint8), ("rc", C.c_uint8), ("n_runs", C.c_uint8),
+                ("D", C.c_uint16), ("_pad", C.c_uint16), ("run", Run * RUN_MAX)]
+
+
+class Space(C.Structure):
+    _fields_ = [("n_p", C.c_uint32), ("n_mbs", C.c_uint32), ("n_tp", C.c_uint32), ("n_rc", C.c_uint32),
+                ("n_d", C.c_uint32), ("seg_max", C.c_uint32), ("p_values", C.c_uint8 * NP_MAX),
+                ("mbs_idx", C.c_uint8 * MBS_MAX), ("tp_idx", C.c_uint8 * TP_MAX), ("rc_values", C.c_uint8 * 2),
+                ("_pad", C.c_uint8 * 6), ("d_values", C.c_uint16 * ND_MAX)]
+
+
+class Objective(C.Structure):
+    _fields_ = [("kind", C.c_uint32), ("flags", C.c_uint32), ("budget_usd_per_iter", C.c_double),
+                ("min_iters_per_s", C.c_double), ("budget_factor_over_cheapest", C.c_double)]
+
+
+class Result(C.Structure):
+    _fields_ = [("flat", C.c_uint64), ("t_iter", C.c_double), ("cost", C.c_double), ("peak_mem", C.c_uint64),
+                ("score", C.c_double), ("status", C.c_uint32), ("_pad", C.c_uint32), ("plan", PlanRec)]
+
+
+class Stats(C.Structure):
+    _fields_ = [("n_total", C.c_uint64), ("n_invalid", C.c_uint64), ("n_oom", C.c_uint64),
+                ("n_over_avail", C.c_uint64), ("n_over_constraint", C.c_uint64), ("n_feasible", C.c_uint64),
+                ("budget_used", C.c_double), ("min_feasible_cost", C.c_double), ("kernel_ms", C.c_float),
+                ("n_launches", C.c_uint32)]
+
+
+assert C.sizeof(PlanRec) == 72 and C.sizeof(Result) == 120 and C.sizeof(Space) == 152
+assert C.sizeof(Objective) == 32 and C.sizeof(Stats) == 72
+
+# numpy view of an array of plan records (same 72-byte layout)
+RUN_DTYPE = np.dtype([("type", "u1"), ("zone", "u1"), ("tp_idx", "u1"), ("n_stages", "u1")])
+REC_DTYPE = np.dtype([("P", "u1"), ("mbs_idx", "u1"), ("rc", "u1"), ("n_runs", "u1"), ("D", "<u2"), ("_pad", "<u2"),
+                      ("run", RUN_DTYPE, (RUN_MAX,))])
+assert REC_DTYPE.itemsize == 72
+
+
+class SailorError(RuntimeError):
+    def __init__(self, code: int, where: str, cuda: int = 0):
+        self.code = code
+        msg = f"{where}: {sailor_strerror(code)} ({code})"
+        if cuda:
+            msg += f" [cudaError {cuda}]"
+        super().__init__(msg)
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Load the CUDA library; raises if it has not been built (there is no other code path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2504_17096_b200.build` "
+                          "(this package has no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp = C.c_void_p
+    L.sailor_create.argtypes = [C.POINTER(Model), C.POINTER(Profile), C.POINTER(Cluster), C.c_int, vp, C.POINTER(vp)]
+    L.sailor_destroy.argtypes = [vp]
+    L.sailor_set_availability.argtypes = [vp, _u16p]
+    L.sailor_simulate.argtypes = [vp, vp, C.c_uint64, C.c_int, vp, vp, vp, vp]
+    L.sailor_space_size.argtypes = [vp, C.POINTER(Space), _u64p]
+    L.sailor_decode.argtypes = [vp, C.POINTER(Space), C.c_uint64, C.POINTER(PlanRec)]
+    L.sailor_plan.argtypes = [vp, C.POINTER(Space), C.POINTER(Objective), C.c_uint32, C.POINTER(Result), _u32p,
+                              C.POINTER(Stats)]
+    L.sailor_plan_range.argtypes = [vp, C.POINTER(Space), C.POINTER(Objective), C.c_uint64, C.c_uint64, C.c_uint32,
+                                    C.POINTER(Result), _u32p, C.POINTER(Stats)]
+    L.sailor_strerror.argtypes = [C.c_int]
+    L.sailor_strerror.restype = C.c_char_p
+    L.sailor_last_cuda_error.argtypes = [vp]
+    for name in EXPORTS:
+        if name != "sailor_strerror":
+            getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def sailor_strerror(code: int) -> str:
+    return load().sailor_strerror(code).decode()
+
+
+def _check(rc: int, where: str, ctx=None):
+    if rc != OK:
+        cuda = load().sailor_last_cuda_error(ctx) if (ctx and rc == E_CUDA) else 0
+        raise SailorError(rc, where, cuda)
+
+
+def _np(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+def make_space(w) -> Space:
+    """sailor_space from a workload's radix lists."""
+    s = Space()
+    s.n_p, s.n_mbs, s.n_tp, s.n_rc, s.n_d = len(w.p_values), len(w.mbs_idx), len(w.tp_idx), len(w.rc_values), len(w.d_values)
+    s.seg_max = w.seg_max
+    for name in ("p_values", "mbs_idx", "tp_idx", "rc_values", "d_values"):
+        arr = getattr(s, name)
+        for i, x in enumerate(getattr(w, name)):
+            arr[i] = int(x)
+    return s
+
+
+def make_objective(w, *, flags: int = 0, kind: Optional[int] = None, budget: Optional[float] = None,
+                   min_rate: Optional[float] = None, factor: Optional[float] = None) -> Objective:
+    return Objective(w.objective if kind is None else kind, flags,
+                     w.budget_usd_per_iter if budget is None else budget,
+                     w.min_iters_per_s if min_rate is None else min_rate,
+                     w.budget_factor_over_cheapest if factor is None else factor)
+
+
+def pack_records(recs: dict) -> np.ndarray:
+    """Dict of integer arrays (workloads.random_plans layout) -> array of 72-byte plan records."""
+    n = len(recs["P"])
+    out = np.zeros(n, dtype=REC_DTYPE)
+    for k in ("P", "mbs_idx", "rc", "n_runs", "D"):
+        out[k] = recs[k]
+    for k in ("type", "zone", "tp_idx", "n_stages"):
+        out["run"][k] = recs[k]
+    return out
+
+
+def sailor_create(w, device: int = 0, stream: int = 0) -> C.c_void_p:
+    """Context for a workload's model, profile and cluster tables (host arrays are copied)."""
+    m = Model(w.n_blocks, w.has_embed, w.has_head, w.heads, w.gbs, w.mul_factor, w.dtype_size, w.grad_dtype_size, 0)
+    keep = []
+
+    def ptr(a, dtype, ptype):
+        a = _np(a, dtype)
+        keep.append(a)
+        return a.ctypes.data_as(ptype)
+
+    p = Profile()
+    p.n_types, p.n_tp, p.n_mbs = w.n_types, len(w.tp_values), len(w.mbs_values)
+    for i, x in enumerate(w.tp_values):
+        p.tp_values[i] = x
+    for i, x in enumerate(w.mbs_values):
+        p.mbs_values[i] = x
+    p.fwd, p.bwd, p.upd = ptr(w.fwd, np.float64, _dp), ptr(w.bwd, np.float64, _dp), ptr(w.upd, np.float64, _dp)
+    p.params = ptr(w.params, np.uint64, _u64p)
+    p.act_saved, p.act_ckpt = ptr(w.act_saved, np.uint64, _u64p), ptr(w.act_ckpt, np.uint64, _u64p)
+    p.act_work, p.p2p_bytes = ptr(w.act_work, np.uint64, _u64p), ptr(w.p2p_bytes, np.uint64, _u64p)
+    c = Cluster()
+    c.n_types, c.n_zones = w.n_types, w.n_zones
+    c.capacity, c.reserved = ptr(w.capacity, np.uint64, _u64p), ptr(w.reserved, np.uint64, _u64p)
+    c.gpus_per_node = ptr(w.gpus_per_node, np.uint32, _u32p)
+    for name in ("price_per_hour", "intra_alpha", "intra_inv_bw", "inter_alpha", "inter_inv_bw", "zone_alpha",
+                 "zone_inv_bw", "egress"):
+        setattr(c, name, ptr(getattr(w, name), np.float64, _dp))
+    ctx = C.c_void_p()
+    _check(load().sailor_create(C.byref(m), C.byref(p), C.byref(c), device, C.c_void_p(stream), C.byref(ctx)),
+           "sailor_create")
+    return ctx
+
+
+def sailor_destroy(ctx) -> None:
+    _check(load().sailor_destroy(ctx), "sailor_destroy")
+
+
+def sailor_set_availability(ctx, avail) -> None:
+    a = _np(avail, np.uint16)
+    _check(load().sailor_set_availability(ctx, a.ctypes.data_as(_u16p)), "sailor_set_availability", ctx)
+
+
+def sailor_simulate(ctx, plans: np.ndarray):
+    """Host path: records (REC_DTYPE array) in, (t_iter, peak_mem, cost, status) numpy arrays out."""
+    plans = np.ascontiguousarray(plans, dtype=REC_DTYPE)
+    n = plans.size
+    t, c = np.empty(n, np.float64), np.empty(n, np.float64)
+    m, s = np.empty(n, np.uint64), np.empty(n, np.uint32)
+    _check(load().sailor_simulate(ctx, plans.ctypes.data, n, 0, t.ctypes.data, m.ctypes.data, c.ctypes.data,
+                                  s.ctypes.data), "sailor_simulate", ctx)
+    return t, m, c, s
+
+
+def sailor_simulate_device(ctx, plans_ptr: int, n: int, t_iter_ptr: int, peak_mem_ptr: int, cost_ptr: int,
+                           status_ptr: int) -> None:
+    """Device path: raw device pointers (e.g. torch tensors' data_ptr()); only enqueues work."""
+    _check(load().sailor_simulate(ctx, plans_ptr, n, 1, t_iter_ptr or None, peak_mem_ptr or None, cost_ptr or None,
+                                  status_ptr or None), "sailor_simulate", ctx)
+
+
+def sailor_space_size(ctx, space: Space) -> int:
+    n = C.c_uint64()
+    _check(load().sailor_space_size(ctx, C.byref(space), C.byref(n)), "sailor_space_size")
+    return int(n.value)
+
+
+def sailor_decode(ctx, space: Space, flat: int) -> PlanRec:
+    r = PlanRec()
+    _check(load().sailor_decode(ctx, C.byref(space), flat, C.byref(r)), "sailor_decode")
+    return r
+
+
+def sailor_plan_range(ctx, space: Space, obj: Objective, lo: int, hi: int, k: int):
+    res = (Result * k)()
+    n = C.c_uint32()
+    st = Stats()
+    _check(load().sailor_plan_range(ctx, C.byref(space), C.byref(obj), lo, hi, k, res, C.byref(n), C.byref(st)),
+           "sailor_plan_range", ctx)
+    return list(res[: n.value]), st
+
+
+def sailor_plan(ctx, space: Space, obj: Objective, k: int):
+    res = (Result * k)()
+    n = C.c_uint32()
+    st = Stats()
+    _check(load().sailor_plan(ctx, C.byref(space), C.byref(obj), k, res, C.byref(n), C.byref(st)), "sailor_plan", ctx)
+    return list(res[: n.value]), st
+
+
+def stats_dict(st: Stats) -> dict:
+    return {f: getattr(st, f) for f, _ in Stats._fields_}

@@ -1,0 +1,695 @@
+// C ABI of the library (see include/sailor.h): context management, argument checks, launches.
+// Every simulation step runs in the kernels; the host only validates, packs tables and
+// enqueues work on the caller's stream.
+#include <cmath>
+#include <cstddef>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "sailor_plan_kernels.cuh"
+
+using namespace sailor;
+
+namespace {
+
+constexpr int SIM_THREADS = 256;
+
+// ---- kernels of the explicit-batch path -----------------------------------------------------
+
+// Left-to-right layer sums for every stage composition: chain[n] = start + n blocks, where
+// start is 0 or the embedding layer's entry.  One thread per (table, start, type, tp[, mbs]).
+__global__ void chain_kernel(unsigned char* blob) {
+    TabView v;
+    v.bind(blob, blob);
+    const TabHdr* h = v.h;
+    const uint32_t gts = h->T * h->n_tp;
+    const uint32_t n4 = 2 * gts * h->n_mbs;                  // [start][type][tp][mbs]
+    const uint32_t n3 = 2 * gts;                             // [start][type][tp]
+    const uint32_t x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x < 2 * n4) {
+        const bool is_b = x >= n4;
+        const uint32_t y = is_b ? x - n4 : x;
+        const uint32_t mi = y % h->n_mbs, gt = (y / h->n_mbs) % gts, start = y / (h->n_mbs * gts);
+        const double* tab = is_b ? v.bwd : v.fwd;
+        double* out = reinterpret_cast<double*>(blob + (is_b ? h->off_chain_b : h->off_chain_f)) + (size_t)y * h->chain_len;
+        const double e = tab[((size_t)KIND_EMBED * gts + gt) * h->n_mbs + mi];
+        const double b = tab[((size_t)KIND_BLOCK * gts + gt) * h->n_mbs + mi];
+        double acc = start ? add_rn(0.0, e) : 0.0;
+        out[0] = acc;
+        for (uint32_t n = 1; n < h->chain_len; ++n) { acc = add_rn(acc, b); out[n] = acc; }
+    } else if (x < 2 * n4 + n3) {
+        const uint32_t y = x - 2 * n4;
+        const uint32_t gt = y % gts, start = y / gts;
+        double* out = reinterpret_cast<double*>(blob + h->off_chain_u) + (size_t)y * h->chain_len;
+        const double e = v.upd[(size_t)KIND_EMBED * gts + gt];
+        const double b = v.upd[(size_t)KIND_BLOCK * gts + gt];
+        double acc = start ? add_rn(0.0, e) : 0.0;
+        out[0] = acc;
+        for (uint32_t n = 1; n < h->chain_len; ++n) { acc = add_rn(acc, b); out[n] = acc; }
+    }
+}
+
+// One thread per explicit plan record (Sec. 4.3).  Records are staged through shared memory
+// with coalesced 8-byte loads; results leave as four structure-of-arrays streams.
+__global__ void __launch_bounds__(SIM_THREADS)
+simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
+                const sailor_plan_rec* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
+                uint64_t* __restrict__ peak_mem, double* __restrict__ cost, uint32_t* __restrict__ status,
+                unsigned int* error) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ uint64_t mbar;
+    constexpr uint32_t W = sizeof(sailor_plan_rec) / 8;      // 9 words per record
+    __shared__ uint64_t recs[SIM_THREADS * W];
+    const uint32_t tid = threadIdx.x;
+    const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(blob)->static_bytes;
+    if (!bulk_load(dyn, blob, static_bytes, &mbar)) {
+        if (tid == 0) atomicExch(error, 1u);
+        for (uint32_t x = tid; x < static_bytes / 16; x += SIM_THREADS)
+            reinterpret_cast<uint4*>(dyn)[x] = reinterpret_cast<const uint4*>(blob)[x];
+        __syncthreads();
+    }
+    TabView v;
+    v.bind(dyn, blob);
+    const uint64_t* src = reinterpret_cast<const uint64_t*>(plans);
+    for (uint64_t tile = (uint64_t)blockIdx.x * SIM_THREADS; tile < n; tile += (uint64_t)gridDim.x * SIM_THREADS) {
+        const uint64_t cnt = n - tile < SIM_THREADS ? n - tile : SIM_THREADS;
+        __syncthreads();
+        for (uint32_t x = tid; x < cnt * W; x += SIM_THREADS) recs[x] = src[tile * W + x];
+        __syncthreads();
+        if (tid < cnt) {
+            union { sailor_plan_rec r; uint64_t w[W]; } u;      // 8-byte aligned copy of the record
+#pragma unroll
+            for (uint32_t w = 0; w < W; ++w) u.w[w] = recs[tid * W + w];
+            const SimOut o = simulate_record(v, avail, u.r);
+            if (t_iter) t_iter[tile + tid] = o.t_iter;
+            if (peak_mem) peak_mem[tile + tid] = o.peak_mem;
+            if (cost) cost[tile + tid] = o.cost;
+            if (status) status[tile + tid] = o.status;
+        }
+    }
+}
+
+// ---- host state -----------------------------------------------------------------------------
+
+struct SpaceCache {
+    bool valid = false;
+    sailor_space key;
+    SpaceDesc desc;
+    uint32_t n_config = 0, n_chunks = 0, p_max = 0;
+    uint64_t n_total = 0;
+    std::vector<uint32_t> chunk_start;     // host copies, for range -> chunk lookup
+    std::vector<uint64_t> flat_base;
+    uint32_t* d_chunk_start = nullptr;
+    uint64_t* d_flat_base = nullptr;
+    size_t smem = 0;
+};
+
+struct OutBlock {                          // device -> pinned host
+    sailor_result results[SAILOR_K_MAX];
+    Ctrl ctrl;
+};
+
+}  // namespace
+
+struct sailor_ctx {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int last_cuda = 0;
+    int sm_count = 0;
+    TabHdr hdr;                            // host copy of the header
+    unsigned char* d_blob = nullptr;
+    uint16_t* d_avail = nullptr;
+    uint16_t* h_avail = nullptr;           // pinned
+    Ctrl* d_ctrl = nullptr;
+    sailor_result* d_results = nullptr;
+    OutBlock* h_out = nullptr;             // pinned
+    Hit* d_partial = nullptr;
+    uint32_t* d_partial_n = nullptr;
+    uint32_t max_grid = 0;                 // capacity of the partial-result buffers
+    uint32_t grid_of[6] = {0, 0, 0, 0, 0, 0};   // resident blocks per kernel variant, for the cached space
+    SpaceCache space;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    // explicit-batch staging (grow-only)
+    unsigned char* d_stage = nullptr;
+    size_t stage_bytes = 0;
+};
+
+namespace {
+
+#define CU(ctx, call)                                  \
+    do {                                               \
+        cudaError_t e_ = (call);                       \
+        if (e_ != cudaSuccess) {                       \
+            (ctx)->last_cuda = (int)e_;                \
+            return SAILOR_E_CUDA;                      \
+        }                                              \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        cudaGetDevice(&prev);
+        if (prev != dev) cudaSetDevice(dev);
+        else prev = -1;
+    }
+    ~DeviceGuard() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+bool finite_nonneg(const double* p, size_t n) {
+    for (size_t i = 0; i < n; ++i)
+        if (!(p[i] >= 0.0) || std::isinf(p[i])) return false;
+    return true;
+}
+
+uint32_t align16(uint32_t x) { return (x + 15u) & ~15u; }
+
+template <typename T>
+uint32_t put(std::vector<unsigned char>& blob, const T* src, size_t n) {
+    const uint32_t off = align16((uint32_t)blob.size());
+    blob.resize(off + n * sizeof(T));
+    if (src) memcpy(blob.data() + off, src, n * sizeof(T));
+    return off;
+}
+
+int check_space(const sailor_ctx* ctx, const sailor_space* s) {
+    if (!ctx || !s) return SAILOR_E_ARG;
+    if (s->n_p == 0 || s->n_mbs == 0 || s->n_tp == 0 || s->n_rc == 0 || s->n_d == 0) return SAILOR_E_ARG;
+    if (s->n_p > SAILOR_NP_MAX || s->n_mbs > SAILOR_MBS_MAX || s->n_tp > SAILOR_TP_MAX || s->n_rc > 2 ||
+        s->n_d > SAILOR_ND_MAX || s->seg_max < 1 || s->seg_max > SAILOR_SEG_MAX)
+        return SAILOR_E_RANGE;
+    for (uint32_t i = 0; i < s->n_p; ++i)
+        if (s->p_values[i] < 1 || s->p_values[i] > SAILOR_P_MAX) return SAILOR_E_RANGE;
+    for (uint32_t i = 0; i < s->n_mbs; ++i)
+        if (s->mbs_idx[i] >= ctx->hdr.n_mbs) return SAILOR_E_RANGE;
+    for (uint32_t i = 0; i < s->n_tp; ++i)
+        if (s->tp_idx[i] >= ctx->hdr.n_tp) return SAILOR_E_RANGE;
+    for (uint32_t i = 0; i < s->n_rc; ++i)
+        if (s->rc_values[i] > 1) return SAILOR_E_RANGE;
+    for (uint32_t i = 0; i < s->n_d; ++i)
+        if (s->d_values[i] < 1) return SAILOR_E_RANGE;
+    return SAILOR_OK;
+}
+
+SpaceDesc to_desc(const sailor_space* s) {
+    SpaceDesc d;
+    memset(&d, 0, sizeof(d));
+    d.n_p = s->n_p; d.n_mbs = s->n_mbs; d.n_tp = s->n_tp; d.n_rc = s->n_rc; d.n_d = s->n_d; d.seg_max = s->seg_max;
+    memcpy(d.p_values, s->p_values, sizeof(d.p_values));
+    memcpy(d.mbs_idx, s->mbs_idx, sizeof(d.mbs_idx));
+    memcpy(d.tp_idx, s->tp_idx, sizeof(d.tp_idx));
+    memcpy(d.rc_values, s->rc_values, sizeof(d.rc_values));
+    memcpy(d.d_values, s->d_values, sizeof(d.d_values));
+    return d;
+}
+
+// Candidate count with overflow check (limit 2^63).
+int space_total(const sailor_ctx* ctx, const SpaceDesc& d, uint64_t* out) {
+    const uint64_t R = ctx->hdr.R;
+    const uint64_t base = (uint64_t)d.n_mbs * d.n_tp * d.n_rc * d.n_d;
+    unsigned __int128 n = 0;
+    for (uint32_t j = 0; j < d.n_p; ++j) {
+        n += (unsigned __int128)base * ipow64(R, nseg_of(d.p_values[j], d.seg_max));
+        if (n >> 63) return SAILOR_E_RANGE;
+    }
+    *out = (uint64_t)n;
+    return SAILOR_OK;
+}
+
+bool same_space(const sailor_space& a, const sailor_space& b) {
+    if (a.n_p != b.n_p || a.n_mbs != b.n_mbs || a.n_tp != b.n_tp || a.n_rc != b.n_rc || a.n_d != b.n_d ||
+        a.seg_max != b.seg_max)
+        return false;
+    return !memcmp(a.p_values, b.p_values, a.n_p) && !memcmp(a.mbs_idx, b.mbs_idx, a.n_mbs) &&
+           !memcmp(a.tp_idx, b.tp_idx, a.n_tp) && !memcmp(a.rc_values, b.rc_values, a.n_rc) &&
+           !memcmp(a.d_values, b.d_values, a.n_d * sizeof(uint16_t));
+}
+
+// Per-configuration chunk and flat-index offsets; uploaded once per distinct space.
+int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
+    SpaceCache& sc = ctx->space;
+    if (sc.valid && same_space(sc.key, *s)) return SAILOR_OK;
+    int rc = check_space(ctx, s);
+    if (rc) return rc;
+    SpaceDesc d = to_desc(s);
+    uint64_t total = 0;
+    rc = space_total(ctx, d, &total);
+    if (rc) return rc;
+    const uint64_t R = ctx->hdr.R;
+    const uint32_t per_p = d.n_mbs * d.n_tp * d.n_rc * d.n_d;
+    const uint64_t n_config = (uint64_t)per_p * d.n_p;
+    if (n_config > (1u << 24)) return SAILOR_E_RANGE;
+    std::vector<uint32_t> cs(n_config + 1);
+    std::vector<uint64_t> fb(n_config);
+    uint64_t chunks = 0, flat = 0;
+    uint32_t p_max = 0;
+    for (uint32_t j = 0; j < d.n_p; ++j) {
+        const uint32_t nseg = nseg_of(d.p_values[j], d.seg_max);
+        p_max = d.p_values[j] > p_max ? d.p_values[j] : p_max;
+        const uint64_t items = ipow64(R, nseg - 1);
+        const uint64_t per_cfg = (items + PLAN_THREADS - 1) / PLAN_THREADS;
+        for (uint32_t c = 0; c < per_p; ++c) {
+            cs[(size_t)j * per_p + c] = (uint32_t)chunks;
+            fb[(size_t)j * per_p + c] = flat;
+            chunks += per_cfg;
+            flat += items * R;
+            if (chunks >= 0xfff00000ull) return SAILOR_E_RANGE;
+        }
+    }
+    cs[n_config] = (uint32_t)chunks;
+    const size_t smem = plan_smem_bytes(ctx->hdr.static_bytes, p_max, ctx->hdr.T, ctx->hdr.Z);
+    if (smem > 200 * 1024) return SAILOR_E_RANGE;
+
+    sc.valid = false;
+    cudaFree(sc.d_chunk_start);
+    cudaFree(sc.d_flat_base);
+    sc.d_chunk_start = nullptr;
+    sc.d_flat_base = nullptr;
+    CU(ctx, cudaMalloc(&sc.d_chunk_start, cs.size() * sizeof(uint32_t)));
+    CU(ctx, cudaMalloc(&sc.d_flat_base, fb.size() * sizeof(uint64_t)));
+    CU(ctx, cudaMemcpyAsync(sc.d_chunk_start, cs.data(), cs.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(sc.d_flat_base, fb.data(), fb.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(ctx, cudaStreamSynchronize(ctx->stream));       // the vectors are pageable
+    sc.key = *s;
+    sc.desc = d;
+    sc.n_config = (uint32_t)n_config;
+    sc.n_chunks = (uint32_t)chunks;
+    sc.n_total = total;
+    sc.p_max = p_max;
+    sc.chunk_start.swap(cs);
+    sc.flat_base.swap(fb);
+    sc.smem = smem;
+    sc.valid = true;
+    for (uint32_t& g : ctx->grid_of) g = 0;
+    return SAILOR_OK;
+}
+
+// Chunk that contains flat index f (f < n_total).
+uint32_t chunk_of(const sailor_ctx* ctx, uint64_t f) {
+    const SpaceCache& sc = ctx->space;
+    uint32_t lo = 0, hi = sc.n_config;
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) / 2;
+        if (sc.flat_base[mid] <= f) lo = mid; else hi = mid;
+    }
+    const uint64_t item = (f - sc.flat_base[lo]) / ctx->hdr.R;
+    return sc.chunk_start[lo] + (uint32_t)(item / PLAN_THREADS);
+}
+
+using PlanKernel = void (*)(const PlanParams);
+
+PlanKernel pick_kernel(uint32_t obj, bool constr) {
+    switch (obj) {
+        case SAILOR_OBJ_MAX_THROUGHPUT: return constr ? plan_kernel<0, true> : plan_kernel<0, false>;
+        case SAILOR_OBJ_MIN_COST: return constr ? plan_kernel<1, true> : plan_kernel<1, false>;
+        default: return constr ? plan_kernel<2, true> : plan_kernel<2, false>;
+    }
+}
+
+// Enqueue one search pass (clear, search, merge) on the context's stream.
+int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_ctrl, double min_rate,
+                 uint32_t flags, uint64_t lo, uint64_t hi, uint32_t k, double next_budget_factor,
+                 uint32_t* n_launches) {
+    SpaceCache& sc = ctx->space;
+    // clear the counters; ctrl->budget (the previous pass may have written it) and the sticky error stay
+    CU(ctx, cudaMemsetAsync(ctx->d_ctrl, 0, offsetof(Ctrl, min_cost_bits), ctx->stream));
+    CU(ctx, cudaMemsetAsync(&ctx->d_ctrl->min_cost_bits, 0x7f, sizeof(unsigned long long), ctx->stream));
+    PlanParams pp;
+    memset(&pp, 0, sizeof(pp));
+    pp.blob = ctx->d_blob;
+    pp.avail = ctx->d_avail;
+    pp.cfg_chunk_start = sc.d_chunk_start;
+    pp.cfg_flat_base = sc.d_flat_base;
+    pp.ctrl = ctx->d_ctrl;
+    pp.partial = ctx->d_partial;
+    pp.partial_n = ctx->d_partial_n;
+    pp.sp = sc.desc;
+    pp.n_config = sc.n_config;
+    pp.flat_lo = lo;
+    pp.flat_hi = hi;
+    pp.k = k;
+    pp.eval_all = (flags & SAILOR_FLAG_EVAL_ALL) ? 1u : 0u;
+    pp.budget_from_ctrl = budget_from_ctrl ? 1u : 0u;
+    pp.p_max = sc.p_max;
+    pp.budget = budget;
+    pp.min_rate = min_rate;
+    uint32_t grid = 0;
+    if (hi > lo) {
+        pp.chunk_lo = chunk_of(ctx, lo);
+        pp.chunk_hi = chunk_of(ctx, hi - 1) + 1;
+        const uint32_t n_chunks = pp.chunk_hi - pp.chunk_lo;
+        const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
+        PlanKernel kern = pick_kernel(obj, constr);
+        uint32_t& resident = ctx->grid_of[obj * 2 + (constr ? 1 : 0)];
+        if (resident == 0) {       // once per (space, kernel variant): opt in to the shared memory, size the grid
+            CU(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sc.smem));
+            int per_sm = 0;
+            CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, sc.smem));
+            if (per_sm < 1) return SAILOR_E_RANGE;
+            resident = (uint32_t)per_sm * (uint32_t)ctx->sm_count;
+            if (resident > ctx->max_grid) resident = ctx->max_grid;
+        }
+        grid = n_chunks < resident ? n_chunks : resident;
+        const uint32_t batch = n_chunks / (grid * 32u);
+        pp.batch = batch < 1 ? 1 : (batch > 16 ? 16 : batch);
+        kern<<<grid, PLAN_THREADS, sc.smem, ctx->stream>>>(pp);
+        CU(ctx, cudaGetLastError());
+        ++*n_launches;
+    }
+    MergeParams mp;
+    memset(&mp, 0, sizeof(mp));
+    mp.blob = ctx->d_blob;
+    mp.avail = ctx->d_avail;
+    mp.partial = ctx->d_partial;
+    mp.partial_n = ctx->d_partial_n;
+    mp.ctrl = ctx->d_ctrl;
+    mp.results = ctx->d_results;
+    mp.sp = sc.desc;
+    mp.n_partial = grid;
+    mp.k = k;
+    mp.obj = obj;
+    mp.budget_factor = next_budget_factor;
+    merge_kernel<<<1, MERGE_THREADS, 0, ctx->stream>>>(mp);
+    CU(ctx, cudaGetLastError());
+    ++*n_launches;
+    return SAILOR_OK;
+}
+
+int validate_host_record(const sailor_ctx* ctx, const sailor_plan_rec& r) {
+    const TabHdr& h = ctx->hdr;
+    if (r.P < 1 || r.P > SAILOR_P_MAX || r.n_runs < 1 || r.n_runs > SAILOR_RUN_MAX || r.D < 1) return SAILOR_E_RANGE;
+    if (r.mbs_idx >= h.n_mbs) return SAILOR_E_RANGE;
+    uint32_t tot = 0;
+    for (uint32_t q = 0; q < r.n_runs; ++q) {
+        if (r.run[q].type >= h.T || r.run[q].zone >= h.Z || r.run[q].tp_idx >= h.n_tp || r.run[q].n_stages < 1)
+            return SAILOR_E_RANGE;
+        tot += r.run[q].n_stages;
+    }
+    return tot == r.P ? SAILOR_OK : SAILOR_E_RANGE;
+}
+
+}  // namespace
+
+// ---- C ABI ------------------------------------------------------------------------------------
+
+extern "C" {
+
+const char* sailor_strerror(int code) {
+    switch (code) {
+        case SAILOR_OK: return "ok";
+        case SAILOR_E_ARG: return "invalid argument";
+        case SAILOR_E_RANGE: return "index or size out of range";
+        case SAILOR_E_CUDA: return "CUDA call failed";
+        case SAILOR_E_NOMEM: return "out of memory";
+        case SAILOR_E_DEVICE: return "kernel reported an internal fault";
+        default: return "unknown error";
+    }
+}
+
+int sailor_last_cuda_error(const sailor_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
+
+int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_cluster* c, int cuda_device,
+                  void* cuda_stream, sailor_ctx** out) {
+    if (!m || !p || !c || !out) return SAILOR_E_ARG;
+    *out = nullptr;
+    if (!p->fwd || !p->bwd || !p->upd || !p->params || !p->act_saved || !p->act_ckpt || !p->act_work ||
+        !p->p2p_bytes || !c->capacity || !c->reserved || !c->gpus_per_node || !c->price_per_hour ||
+        !c->intra_alpha || !c->intra_inv_bw || !c->inter_alpha || !c->inter_inv_bw || !c->zone_alpha ||
+        !c->zone_inv_bw || !c->egress)
+        return SAILOR_E_ARG;
+    const uint32_t T = p->n_types, Z = c->n_zones, n_tp = p->n_tp, n_mbs = p->n_mbs;
+    if (T == 0 || Z == 0 || n_tp == 0 || n_mbs == 0 || T != c->n_types || m->n_blocks == 0) return SAILOR_E_ARG;
+    if (m->gbs == 0 || m->heads == 0 || m->mul_factor == 0 || m->dtype_size == 0 || m->grad_dtype_size == 0)
+        return SAILOR_E_ARG;
+    if (T > SAILOR_T_MAX || Z > SAILOR_Z_MAX || n_tp > SAILOR_TP_MAX || n_mbs > SAILOR_MBS_MAX ||
+        m->n_blocks > 4096)
+        return SAILOR_E_RANGE;
+    for (uint32_t i = 0; i < n_tp; ++i)
+        if (p->tp_values[i] == 0) return SAILOR_E_ARG;
+    for (uint32_t i = 0; i < n_mbs; ++i)
+        if (p->mbs_values[i] == 0) return SAILOR_E_ARG;
+    for (uint32_t g = 0; g < T; ++g)
+        if (c->gpus_per_node[g] == 0) return SAILOR_E_ARG;
+    const size_t n4 = (size_t)SAILOR_KINDS * T * n_tp * n_mbs, n3 = (size_t)SAILOR_KINDS * T * n_tp;
+    const size_t na = (size_t)SAILOR_KINDS * n_tp * n_mbs, R = (size_t)T * Z;
+    if (!finite_nonneg(p->fwd, n4) || !finite_nonneg(p->bwd, n4) || !finite_nonneg(p->upd, n3) ||
+        !finite_nonneg(c->price_per_hour, R) || !finite_nonneg(c->intra_alpha, R) ||
+        !finite_nonneg(c->intra_inv_bw, R) || !finite_nonneg(c->inter_alpha, R) ||
+        !finite_nonneg(c->inter_inv_bw, R) || !finite_nonneg(c->zone_alpha, (size_t)Z * Z) ||
+        !finite_nonneg(c->zone_inv_bw, (size_t)Z * Z) || !finite_nonneg(c->egress, (size_t)Z * Z))
+        return SAILOR_E_ARG;
+
+    sailor_ctx* ctx = new (std::nothrow) sailor_ctx();
+    if (!ctx) return SAILOR_E_NOMEM;
+    ctx->device = cuda_device;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    DeviceGuard guard(cuda_device);
+
+    // pack the blob: header, raw tables, cluster tables (static part), then the chains
+    TabHdr& h = ctx->hdr;
+    memset(&h, 0, sizeof(h));
+    h.n_blocks = m->n_blocks; h.has_embed = m->has_embed ? 1 : 0; h.has_head = m->has_head ? 1 : 0;
+    h.heads = m->heads; h.gbs = m->gbs;
+    h.mul_bytes = (uint64_t)m->mul_factor * m->dtype_size;
+    h.grad_bytes = m->grad_dtype_size;
+    h.T = T; h.Z = Z; h.R = (uint32_t)R; h.n_tp = n_tp; h.n_mbs = n_mbs; h.chain_len = m->n_blocks + 1;
+    memcpy(h.tp_values, p->tp_values, n_tp * sizeof(uint32_t));
+    memcpy(h.mbs_values, p->mbs_values, n_mbs * sizeof(uint32_t));
+    for (uint32_t g = 0; g < T; ++g) {
+        h.gpn[g] = c->gpus_per_node[g];
+        h.capacity[g] = c->capacity[g];
+        h.reserved[g] = c->reserved[g];
+    }
+    for (int k = 0; k < SAILOR_KINDS; ++k) h.params[k] = p->params[k];
+
+    std::vector<unsigned char> blob(sizeof(TabHdr));
+    h.off_fwd = put(blob, p->fwd, n4);
+    h.off_bwd = put(blob, p->bwd, n4);
+    h.off_upd = put(blob, p->upd, n3);
+    h.off_saved = put(blob, p->act_saved, na);
+    h.off_ckpt = put(blob, p->act_ckpt, na);
+    h.off_work = put(blob, p->act_work, na);
+    h.off_p2p = put(blob, p->p2p_bytes, n_mbs);
+    std::vector<double> price_s(R);
+    for (size_t d = 0; d < R; ++d) price_s[d] = c->price_per_hour[d] / 3600.0;   // dollars per GPU-second
+    h.off_price_s = put(blob, price_s.data(), R);
+    h.off_intra_a = put(blob, c->intra_alpha, R);
+    h.off_intra_i = put(blob, c->intra_inv_bw, R);
+    h.off_inter_a = put(blob, c->inter_alpha, R);
+    h.off_inter_i = put(blob, c->inter_inv_bw, R);
+    h.off_zone_a = put(blob, c->zone_alpha, (size_t)Z * Z);
+    h.off_zone_i = put(blob, c->zone_inv_bw, (size_t)Z * Z);
+    h.off_egress = put(blob, c->egress, (size_t)Z * Z);
+    h.static_bytes = align16((uint32_t)blob.size());
+    blob.resize(h.static_bytes);
+    const size_t c4 = (size_t)2 * T * n_tp * n_mbs * h.chain_len, c3 = (size_t)2 * T * n_tp * h.chain_len;
+    if (h.static_bytes + (2 * c4 + c3) * sizeof(double) > (1ull << 30) || h.static_bytes > 96 * 1024) {
+        delete ctx;
+        return SAILOR_E_RANGE;
+    }
+    h.off_chain_f = put<double>(blob, nullptr, c4);
+    h.off_chain_b = put<double>(blob, nullptr, c4);
+    h.off_chain_u = put<double>(blob, nullptr, c3);
+    h.total_bytes = align16((uint32_t)blob.size());
+    blob.resize(h.total_bytes);
+    memcpy(blob.data(), &h, sizeof(h));
+
+    auto fail = [&](int code) { sailor_destroy(ctx); return code; };
+#define CUF(call)                                                   \
+    do {                                                            \
+        cudaError_t e_ = (call);                                    \
+        if (e_ != cudaSuccess) {                                    \
+            ctx->last_cuda = (int)e_;                               \
+            return fail(e_ == cudaErrorMemoryAllocation ? SAILOR_E_NOMEM : SAILOR_E_CUDA); \
+        }                                                           \
+    } while (0)
+    cudaDeviceProp prop;
+    CUF(cudaGetDeviceProperties(&prop, cuda_device));
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->max_grid = (uint32_t)ctx->sm_count * 8;
+    CUF(cudaMalloc(&ctx->d_blob, h.total_bytes));
+    CUF(cudaMalloc(&ctx->d_avail, R_MAX * sizeof(uint16_t)));
+    CUF(cudaMallocHost(&ctx->h_avail, R_MAX * sizeof(uint16_t)));
+    CUF(cudaMalloc(&ctx->d_ctrl, sizeof(Ctrl)));
+    CUF(cudaMalloc(&ctx->d_results, sizeof(sailor_result) * SAILOR_K_MAX));
+    CUF(cudaMallocHost(&ctx->h_out, sizeof(OutBlock)));
+    CUF(cudaMalloc(&ctx->d_partial, sizeof(Hit) * SAILOR_K_MAX * ctx->max_grid));
+    CUF(cudaMalloc(&ctx->d_partial_n, sizeof(uint32_t) * ctx->max_grid));
+    CUF(cudaEventCreate(&ctx->ev0));
+    CUF(cudaEventCreate(&ctx->ev1));
+    CUF(cudaMemcpyAsync(ctx->d_blob, blob.data(), h.total_bytes, cudaMemcpyHostToDevice, ctx->stream));
+    CUF(cudaMemsetAsync(ctx->d_avail, 0, R_MAX * sizeof(uint16_t), ctx->stream));
+    CUF(cudaMemsetAsync(ctx->d_ctrl, 0, sizeof(Ctrl), ctx->stream));
+    CUF(cudaMemsetAsync(ctx->d_results, 0, sizeof(sailor_result) * SAILOR_K_MAX, ctx->stream));
+    {
+        const uint32_t n_threads = 4 * T * n_tp * n_mbs + 2 * T * n_tp;
+        chain_kernel<<<(n_threads + 127) / 128, 128, 0, ctx->stream>>>(ctx->d_blob);
+        CUF(cudaGetLastError());
+    }
+    CUF(cudaStreamSynchronize(ctx->stream));           // `blob` is pageable host memory
+    if (h.static_bytes > 24 * 1024)
+        CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h.static_bytes));
+#undef CUF
+    *out = ctx;
+    return SAILOR_OK;
+}
+
+int sailor_destroy(sailor_ctx* ctx) {
+    if (!ctx) return SAILOR_OK;
+    DeviceGuard guard(ctx->device);
+    if (ctx->d_blob) cudaStreamSynchronize(ctx->stream);
+    cudaFree(ctx->d_blob);
+    cudaFree(ctx->d_avail);
+    cudaFreeHost(ctx->h_avail);
+    cudaFree(ctx->d_ctrl);
+    cudaFree(ctx->d_results);
+    cudaFreeHost(ctx->h_out);
+    cudaFree(ctx->d_partial);
+    cudaFree(ctx->d_partial_n);
+    cudaFree(ctx->space.d_chunk_start);
+    cudaFree(ctx->space.d_flat_base);
+    cudaFree(ctx->d_stage);
+    if (ctx->ev0) cudaEventDestroy(ctx->ev0);
+    if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+    delete ctx;
+    return SAILOR_OK;
+}
+
+int sailor_set_availability(sailor_ctx* ctx, const uint16_t* avail) {
+    if (!ctx || !avail) return SAILOR_E_ARG;
+    DeviceGuard guard(ctx->device);
+    // the pinned staging buffer may still feed the previous copy
+    CU(ctx, cudaStreamSynchronize(ctx->stream));
+    memcpy(ctx->h_avail, avail, ctx->hdr.R * sizeof(uint16_t));
+    CU(ctx, cudaMemcpyAsync(ctx->d_avail, ctx->h_avail, ctx->hdr.R * sizeof(uint16_t), cudaMemcpyHostToDevice,
+                            ctx->stream));
+    return SAILOR_OK;
+}
+
+int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, int on_device, double* t_iter,
+                    uint64_t* peak_mem, double* cost, uint32_t* status) {
+    if (!ctx || (!plans && n)) return SAILOR_E_ARG;
+    if (n == 0) return SAILOR_OK;
+    if ((uintptr_t)plans % 8 != 0) return SAILOR_E_ARG;
+    DeviceGuard guard(ctx->device);
+    const sailor_plan_rec* d_plans = plans;
+    double *d_t = t_iter, *d_c = cost;
+    uint64_t* d_m = peak_mem;
+    uint32_t* d_s = status;
+    if (!on_device) {
+        for (uint64_t j = 0; j < n; ++j) {
+            const int rc = validate_host_record(ctx, plans[j]);
+            if (rc) return rc;
+        }
+        const size_t need = n * (sizeof(sailor_plan_rec) + 32);
+        if (need > ctx->stage_bytes) {
+            CU(ctx, cudaStreamSynchronize(ctx->stream));
+            cudaFree(ctx->d_stage);
+            ctx->d_stage = nullptr;
+            ctx->stage_bytes = 0;
+            cudaError_t e = cudaMalloc(&ctx->d_stage, need);
+            if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
+            ctx->stage_bytes = need;
+        }
+        unsigned char* base = ctx->d_stage;
+        d_t = reinterpret_cast<double*>(base);
+        d_c = reinterpret_cast<double*>(base + 8 * n);
+        d_m = reinterpret_cast<uint64_t*>(base + 16 * n);
+        d_s = reinterpret_cast<uint32_t*>(base + 24 * n);
+        sailor_plan_rec* dp = reinterpret_cast<sailor_plan_rec*>(base + 32 * n);
+        CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_plan_rec), cudaMemcpyHostToDevice, ctx->stream));
+        d_plans = dp;
+    }
+    const uint64_t tiles = (n + SIM_THREADS - 1) / SIM_THREADS;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 16;
+    const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
+    simulate_kernel<<<grid, SIM_THREADS, ctx->hdr.static_bytes, ctx->stream>>>(
+        ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s, &ctx->d_ctrl->error);
+    CU(ctx, cudaGetLastError());
+    if (!on_device) {
+        if (t_iter) CU(ctx, cudaMemcpyAsync(t_iter, d_t, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
+        if (cost) CU(ctx, cudaMemcpyAsync(cost, d_c, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
+        if (peak_mem) CU(ctx, cudaMemcpyAsync(peak_mem, d_m, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
+        if (status) CU(ctx, cudaMemcpyAsync(status, d_s, 4 * n, cudaMemcpyDeviceToHost, ctx->stream));
+        CU(ctx, cudaStreamSynchronize(ctx->stream));
+    }
+    return SAILOR_OK;
+}
+
+int sailor_space_size(const sailor_ctx* ctx, const sailor_space* s, uint64_t* n_out) {
+    if (!n_out) return SAILOR_E_ARG;
+    int rc = check_space(ctx, s);
+    if (rc) return rc;
+    return space_total(ctx, to_desc(s), n_out);
+}
+
+int sailor_decode(const sailor_ctx* ctx, const sailor_space* s, uint64_t flat, sailor_plan_rec* out) {
+    if (!out) return SAILOR_E_ARG;
+    int rc = check_space(ctx, s);
+    if (rc) return rc;
+    return decode_flat(to_desc(s), ctx->hdr.T, ctx->hdr.Z, flat, out) ? SAILOR_OK : SAILOR_E_RANGE;
+}
+
+int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint64_t flat_lo,
+                      uint64_t flat_hi, uint32_t k, sailor_result* topk, uint32_t* n_found, sailor_stats* stats) {
+    if (!ctx || !s || !o || !topk || !n_found || k == 0) return SAILOR_E_ARG;
+    if (k > SAILOR_K_MAX || o->kind > SAILOR_OBJ_MAX_THROUGHPUT_PER_USD) return SAILOR_E_RANGE;
+    if (std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) ||
+        std::isnan(o->budget_factor_over_cheapest))
+        return SAILOR_E_ARG;
+    DeviceGuard guard(ctx->device);
+    int rc = prepare_space(ctx, s);
+    if (rc) return rc;
+    const uint64_t total = ctx->space.n_total;
+    if (flat_hi > total) flat_hi = total;
+    if (flat_lo > flat_hi) flat_lo = flat_hi;
+
+    uint32_t launches = 0;
+    CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
+    const bool two_pass = o->budget_factor_over_cheapest > 0.0;
+    if (two_pass) {
+        // cheapest feasible plan first; its merge step leaves factor * cost in ctrl->budget
+        rc = enqueue_pass(ctx, SAILOR_OBJ_MIN_COST, 0.0, false, 0.0, o->flags, flat_lo, flat_hi, 1,
+                          o->budget_factor_over_cheapest, &launches);
+        if (rc) return rc;
+    }
+    rc = enqueue_pass(ctx, o->kind, o->budget_usd_per_iter, two_pass, o->min_iters_per_s, o->flags, flat_lo,
+                      flat_hi, k, 0.0, &launches);
+    if (rc) return rc;
+    CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(ctx->h_out->results, ctx->d_results, sizeof(sailor_result) * k, cudaMemcpyDeviceToHost,
+                            ctx->stream));
+    CU(ctx, cudaMemcpyAsync(&ctx->h_out->ctrl, ctx->d_ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, cudaStreamSynchronize(ctx->stream));
+    const Ctrl& cr = ctx->h_out->ctrl;
+    if (cr.error) return SAILOR_E_DEVICE;
+    *n_found = cr.n_found;
+    memcpy(topk, ctx->h_out->results, sizeof(sailor_result) * cr.n_found);
+    if (stats) {
+        stats->n_total = cr.stats[0];
+        stats->n_invalid = cr.stats[1];
+        stats->n_oom = cr.stats[2];
+        stats->n_over_avail = cr.stats[3];
+        stats->n_over_constraint = cr.stats[4];
+        stats->n_feasible = cr.stats[5];
+        stats->budget_used = two_pass ? cr.budget : o->budget_usd_per_iter;
+        double mc;
+        memcpy(&mc, &cr.min_cost_bits, sizeof(mc));
+        stats->min_feasible_cost = cr.stats[5] ? mc : 0.0;
+        float ms = 0.f;
+        CU(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
+        stats->kernel_ms = ms;
+        stats->n_launches = launches;
+    }
+    return SAILOR_OK;
+}
+
+int sailor_plan(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint32_t k,
+                sailor_result* topk, uint32_t* n_found, sailor_stats* stats) {
+    return sailor_plan_range(ctx, s, o, 0, ~0ull >> 1, k, topk, n_found, stats);
+}
+
+}  // extern "C"

@@ -1,0 +1,333 @@
+// Device-side table layout, flat-index decoding and the per-record simulator.
+//
+// All tables of one context live in one contiguous device "blob": a fixed header followed
+// by the variable-size arrays at 16-byte aligned offsets.  The part up to `static_bytes`
+// (header + raw profile + cluster tables, a few KB) is what kernels stage in shared
+// memory; the left-to-right layer-sum chains are larger and stay in global memory (L2).
+#pragma once
+
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/sailor.h"
+
+namespace sailor {
+
+constexpr int KIND_EMBED = 0, KIND_BLOCK = 1, KIND_HEAD = 2;
+constexpr int R_MAX = SAILOR_T_MAX * SAILOR_Z_MAX;   // digits: zone * T + type
+
+struct alignas(16) TabHdr {
+    // model
+    uint32_t n_blocks, has_embed, has_head, heads;
+    uint64_t gbs;
+    uint64_t mul_bytes;        // mul_factor * dtype_size, bytes per parameter on a worker
+    uint64_t grad_bytes;       // bytes per gradient element
+    // shapes
+    uint32_t T, Z, R, n_tp, n_mbs, chain_len;   // chain_len = n_blocks + 1
+    uint32_t tp_values[SAILOR_TP_MAX];
+    uint32_t mbs_values[SAILOR_MBS_MAX];
+    uint32_t gpn[SAILOR_T_MAX];
+    uint64_t capacity[SAILOR_T_MAX];
+    uint64_t reserved[SAILOR_T_MAX];
+    uint64_t params[SAILOR_KINDS];
+    // byte offsets from the blob start
+    uint32_t off_fwd, off_bwd, off_upd;           // f64 [kind][type][tp][mbs], [kind][type][tp]
+    uint32_t off_saved, off_ckpt, off_work;       // u64 [kind][tp][mbs]
+    uint32_t off_p2p;                             // u64 [mbs]
+    uint32_t off_price_s;                         // f64 [digit]  price_per_hour / 3600
+    uint32_t off_intra_a, off_intra_i, off_inter_a, off_inter_i;   // f64 [digit]
+    uint32_t off_zone_a, off_zone_i, off_egress;  // f64 [zone][zone]
+    uint32_t static_bytes;                        // multiple of 16
+    uint32_t off_chain_f, off_chain_b;            // f64 [start][type][tp][mbs][chain_len]
+    uint32_t off_chain_u;                         // f64 [start][type][tp][chain_len]
+    uint32_t total_bytes;
+};
+static_assert(sizeof(TabHdr) % 16 == 0, "header must keep the arrays 16-byte aligned");
+
+// Typed view over a blob whose static part may sit in shared memory and whose chains sit in
+// global memory.
+struct TabView {
+    const TabHdr* h;
+    const double *fwd, *bwd, *upd;
+    const uint64_t *saved, *ckpt, *work, *p2p;
+    const double *price_s, *intra_a, *intra_i, *inter_a, *inter_i, *zone_a, *zone_i, *egress;
+    const double *chain_f, *chain_b, *chain_u;
+
+    __host__ __device__ void bind(const unsigned char* stat, const unsigned char* glob) {
+        h = reinterpret_cast<const TabHdr*>(stat);
+        fwd = reinterpret_cast<const double*>(stat + h->off_fwd);
+        bwd = reinterpret_cast<const double*>(stat + h->off_bwd);
+        upd = reinterpret_cast<const double*>(stat + h->off_upd);
+        saved = reinterpret_cast<const uint64_t*>(stat + h->off_saved);
+        ckpt = reinterpret_cast<const uint64_t*>(stat + h->off_ckpt);
+        work = reinterpret_cast<const uint64_t*>(stat + h->off_work);
+        p2p = reinterpret_cast<const uint64_t*>(stat + h->off_p2p);
+        price_s = reinterpret_cast<const double*>(stat + h->off_price_s);
+        intra_a = reinterpret_cast<const double*>(stat + h->off_intra_a);
+        intra_i = reinterpret_cast<const double*>(stat + h->off_intra_i);
+        inter_a = reinterpret_cast<const double*>(stat + h->off_inter_a);
+        inter_i = reinterpret_cast<const double*>(stat + h->off_inter_i);
+        zone_a = reinterpret_cast<const double*>(stat + h->off_zone_a);
+        zone_i = reinterpret_cast<const double*>(stat + h->off_zone_i);
+        egress = reinterpret_cast<const double*>(stat + h->off_egress);
+        chain_f = reinterpret_cast<const double*>(glob + h->off_chain_f);
+        chain_b = reinterpret_cast<const double*>(glob + h->off_chain_b);
+        chain_u = reinterpret_cast<const double*>(glob + h->off_chain_u);
+    }
+};
+
+// ---- arithmetic helpers: one rounding per operation, never contracted ---------------------
+__device__ __forceinline__ double add_rn(double a, double b) { return __dadd_rn(a, b); }
+__device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(a, b); }
+__host__ __device__ __forceinline__ double dmax(double a, double b) { return a > b ? a : b; }
+
+// Forward / backward / update time of one stage on (type g, tp index, mbs index): the
+// left-to-right sum over [embed?] + nb blocks + [head?], read from the chain tables.
+struct StageTimes { double f, b, u; };
+
+__device__ __forceinline__ StageTimes stage_times(const TabView& v, uint32_t g, uint32_t tpi, uint32_t mi,
+                                                  uint32_t nb, bool e, bool hd) {
+    const TabHdr* h = v.h;
+    const uint32_t gt = (g * h->n_tp + tpi);
+    const size_t tstride = (size_t)h->T * h->n_tp;
+    const size_t i3 = (size_t)(e ? tstride : 0) + gt;
+    const size_t i4 = i3 * h->n_mbs + mi;
+    StageTimes s;
+    s.f = v.chain_f[i4 * h->chain_len + nb];
+    s.b = v.chain_b[i4 * h->chain_len + nb];
+    s.u = v.chain_u[i3 * h->chain_len + nb];
+    if (hd) {
+        const size_t k4 = (((size_t)KIND_HEAD * h->T + g) * h->n_tp + tpi);
+        s.f = add_rn(s.f, v.fwd[k4 * h->n_mbs + mi]);
+        s.b = add_rn(s.b, v.bwd[k4 * h->n_mbs + mi]);
+        s.u = add_rn(s.u, v.upd[k4]);
+    }
+    return s;
+}
+
+__host__ __device__ __forceinline__ uint64_t ceil_div64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+
+// Parameters of stage i and its per-worker peak memory without the reserved bytes
+// (Sec. 4.3: M_peak = M_model + M_activation; stage i keeps min(P - i, N_b) microbatches).
+struct StageMem { uint64_t params, mem; };
+
+__device__ __forceinline__ StageMem stage_memory(const TabView& v, uint32_t tpi, uint32_t mi, uint32_t rc,
+                                                 uint32_t nb, bool e, bool hd, uint64_t inflight) {
+    const TabHdr* h = v.h;
+    const uint32_t tp = h->tp_values[tpi];
+    auto at = [&](const uint64_t* t, int kind) { return t[((size_t)kind * h->n_tp + tpi) * h->n_mbs + mi]; };
+    const uint64_t* keep = rc ? v.ckpt : v.saved;
+    const uint64_t* wset = rc ? v.saved : v.work;
+    uint64_t params = (uint64_t)nb * h->params[KIND_BLOCK];
+    uint64_t A = (uint64_t)nb * at(keep, KIND_BLOCK);
+    uint64_t W = nb ? at(wset, KIND_BLOCK) : 0;
+    if (e) {
+        params += h->params[KIND_EMBED];
+        A += at(keep, KIND_EMBED);
+        const uint64_t w = at(wset, KIND_EMBED);
+        W = w > W ? w : W;
+    }
+    if (hd) {
+        params += h->params[KIND_HEAD];
+        A += at(keep, KIND_HEAD);
+        const uint64_t w = at(wset, KIND_HEAD);
+        W = w > W ? w : W;
+    }
+    StageMem m;
+    m.params = params;
+    m.mem = ceil_div64(params, tp) * h->mul_bytes + inflight * A + W;
+    return m;
+}
+
+// Time of one message over the link between neighbouring stages (one direction).
+__device__ __forceinline__ double boundary_time(const TabView& v, uint32_t g, uint32_t z, uint32_t tp,
+                                                uint32_t g2, uint32_t z2, uint32_t tp2, uint32_t D, double msg) {
+    const TabHdr* h = v.h;
+    if (z != z2) return add_rn(v.zone_a[z * h->Z + z2], mul_rn(msg, v.zone_i[z * h->Z + z2]));
+    const uint32_t d = z * h->T + g;
+    if (g == g2 && (uint64_t)D * (tp + tp2) <= h->gpn[g]) return add_rn(v.intra_a[d], mul_rn(msg, v.intra_i[d]));
+    const uint32_t d2 = z * h->T + g2;
+    const double c1 = add_rn(v.inter_a[d], mul_rn(msg, v.inter_i[d]));
+    const double c2 = add_rn(v.inter_a[d2], mul_rn(msg, v.inter_i[d2]));
+    return dmax(c1, c2);
+}
+
+// Ring all-reduce of a stage's gradients among its D replicas (H5: inside one zone).
+__device__ __forceinline__ double sync_time(const TabView& v, uint32_t g, uint32_t z, uint32_t tp, uint32_t D,
+                                            uint64_t params) {
+    if (D <= 1) return 0.0;
+    const TabHdr* h = v.h;
+    const uint32_t d = z * h->T + g;
+    const bool intra = (uint64_t)D * tp <= h->gpn[g];
+    const double alpha = intra ? v.intra_a[d] : v.inter_a[d];
+    const double inv = intra ? v.intra_i[d] : v.inter_i[d];
+    const double gradbytes = (double)(ceil_div64(params, tp) * h->grad_bytes);
+    const double steps = (double)(2 * (uint64_t)(D - 1));
+    const double coef = steps / (double)D;
+    return add_rn(mul_rn(mul_rn(coef, gradbytes), inv), mul_rn(steps, alpha));
+}
+
+struct SimOut {
+    double t_iter, cost;
+    uint64_t peak_mem;
+    uint32_t status;
+};
+
+__device__ __forceinline__ double make_nan() { return __longlong_as_double(0x7ff8000000000000LL); }
+__device__ __forceinline__ double make_inf() { return __longlong_as_double(0x7ff0000000000000LL); }
+
+// Simulate one run-length encoded plan (Sec. 4.3).  Every index is checked before use; a
+// record that fails gets SAILOR_ST_BAD_RECORD and nothing is read through it.
+__device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __restrict__ avail,
+                                         const sailor_plan_rec& r) {
+    const TabHdr* h = v.h;
+    SimOut o;
+    o.t_iter = o.cost = make_nan();
+    o.peak_mem = 0;
+    o.status = SAILOR_ST_BAD_RECORD;
+    const uint32_t P = r.P, n_runs = r.n_runs, D = r.D, mi = r.mbs_idx, rc = r.rc ? 1u : 0u;
+    if (P < 1 || P > SAILOR_P_MAX || n_runs < 1 || n_runs > SAILOR_RUN_MAX || D < 1 || mi >= h->n_mbs) return o;
+    uint32_t tot = 0;
+    for (uint32_t q = 0; q < n_runs; ++q) {
+        const sailor_run& rr = r.run[q];
+        if (rr.type >= h->T || rr.zone >= h->Z || rr.tp_idx >= h->n_tp || rr.n_stages < 1) return o;
+        tot += rr.n_stages;
+    }
+    if (tot != P) return o;
+
+    uint32_t status = 0;
+    const uint64_t mbs = h->mbs_values[mi];
+    const uint64_t dm = (uint64_t)D * mbs;
+    if (h->gbs % dm != 0) status |= SAILOR_ST_INVALID;
+    const uint64_t n_b = h->gbs / dm;
+
+    // resources: total demand of every (zone, type) a run touches
+    for (uint32_t q = 0; q < n_runs; ++q) {
+        const sailor_run& a = r.run[q];
+        const uint32_t tp = h->tp_values[a.tp_idx];
+        if (tp > h->gpn[a.type] || h->heads % tp != 0) status |= SAILOR_ST_INVALID;
+        uint64_t need = 0;
+        for (uint32_t q2 = 0; q2 < n_runs; ++q2) {
+            const sailor_run& b = r.run[q2];
+            if (b.type == a.type && b.zone == a.zone)
+                need += (uint64_t)D * h->tp_values[b.tp_idx] * b.n_stages;
+        }
+        if (need > avail[a.zone * h->T + a.type]) status |= SAILOR_ST_OVER_AVAIL;
+    }
+
+    const uint32_t base = h->n_blocks / P, extra = h->n_blocks % P;
+    const double msg = (double)v.p2p[mi];
+    const uint64_t xbytes = 2 * n_b * (uint64_t)D * v.p2p[mi];
+    double sum_t = 0.0, max_t = 0.0, max_sync = 0.0, max_u = 0.0, rate = 0.0, c_comm = 0.0;
+    uint64_t peak = 0;
+    uint32_t i = 0;
+    for (uint32_t q = 0; q < n_runs; ++q) {
+        const sailor_run a = r.run[q];
+        const uint32_t g = a.type, z = a.zone, tpi = a.tp_idx, tp = h->tp_values[tpi];
+        const double gpu_rate = mul_rn((double)(D * tp), v.price_s[z * h->T + g]);
+        for (uint32_t j = 0; j < a.n_stages; ++j, ++i) {
+            const uint32_t nb = base + (i < extra ? 1u : 0u);
+            const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
+            const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
+            const StageMem sm = stage_memory(v, tpi, mi, rc, nb, e, hd, inflight);
+            const uint64_t m = sm.mem + h->reserved[g];
+            if (m > h->capacity[g]) status |= SAILOR_ST_OOM;
+            peak = m > peak ? m : peak;
+
+            const StageTimes st = stage_times(v, g, tpi, mi, nb, e, hd);
+            const double b = rc ? add_rn(st.b, st.f) : st.b;
+            double c = 0.0;
+            if (i + 1 < P) {
+                const sailor_run nx = (j + 1 < a.n_stages) ? a : r.run[q + 1];
+                c = boundary_time(v, g, z, tp, nx.type, nx.zone, h->tp_values[nx.tp_idx], D, msg);
+                if (nx.zone != z) c_comm = add_rn(c_comm, mul_rn((double)xbytes, v.egress[z * h->Z + nx.zone]));
+            }
+            const double t = add_rn(add_rn(st.f, b), mul_rn(2.0, c));
+            sum_t = add_rn(sum_t, t);
+            max_t = dmax(max_t, t);
+            max_u = dmax(max_u, st.u);
+            max_sync = dmax(max_sync, sync_time(v, g, z, tp, D, sm.params));
+            rate = add_rn(rate, gpu_rate);
+        }
+    }
+    o.peak_mem = peak;
+    o.status = status;
+    if (status & SAILOR_ST_INVALID) return o;
+    const double t_pp = add_rn(sum_t, mul_rn((double)n_b, max_t));
+    o.t_iter = add_rn(add_rn(t_pp, max_sync), max_u);
+    o.cost = add_rn(mul_rn(rate, o.t_iter), c_comm);
+    return o;
+}
+
+// ---- search space -------------------------------------------------------------------------
+struct SpaceDesc {
+    uint32_t n_p, n_mbs, n_tp, n_rc, n_d, seg_max;
+    uint8_t p_values[SAILOR_NP_MAX];
+    uint8_t mbs_idx[SAILOR_MBS_MAX];
+    uint8_t tp_idx[SAILOR_TP_MAX];
+    uint8_t rc_values[2];
+    uint16_t d_values[SAILOR_ND_MAX];
+};
+
+__host__ __device__ inline uint32_t nseg_of(uint32_t P, uint32_t seg_max) { return P < seg_max ? P : seg_max; }
+__host__ __device__ inline uint64_t ipow64(uint64_t b, uint32_t e) {
+    uint64_t r = 1;
+    while (e--) r *= b;
+    return r;
+}
+
+// One configuration = (P, mbs, tp, rc, D); index c counts them in enumeration order.
+struct Config {
+    uint32_t P, mi, tpi, rc, D, nseg;
+};
+__host__ __device__ inline Config config_of(const SpaceDesc& s, uint32_t c) {
+    Config k;
+    uint32_t x = c;
+    const uint32_t di = x % s.n_d;  x /= s.n_d;
+    const uint32_t ri = x % s.n_rc; x /= s.n_rc;
+    const uint32_t ti = x % s.n_tp; x /= s.n_tp;
+    const uint32_t mi = x % s.n_mbs; x /= s.n_mbs;
+    k.P = s.p_values[x];
+    k.mi = s.mbs_idx[mi];
+    k.tpi = s.tp_idx[ti];
+    k.rc = s.rc_values[ri];
+    k.D = s.d_values[di];
+    k.nseg = nseg_of(k.P, s.seg_max);
+    return k;
+}
+
+// Flat index -> record.  Runs are the segments (equal neighbours are not merged, so that a
+// record maps back to exactly one flat index).
+__host__ __device__ inline bool decode_flat(const SpaceDesc& s, uint32_t T, uint32_t Z, uint64_t flat,
+                                            sailor_plan_rec* out) {
+    const uint64_t R = (uint64_t)T * Z;
+    const uint64_t base = (uint64_t)s.n_mbs * s.n_tp * s.n_rc * s.n_d;
+    for (uint32_t j = 0; j < s.n_p; ++j) {
+        const uint32_t P = s.p_values[j];
+        const uint32_t nseg = nseg_of(P, s.seg_max);
+        const uint64_t sub = base * ipow64(R, nseg);
+        if (flat >= sub) { flat -= sub; continue; }
+        uint32_t seg[SAILOR_SEG_MAX];
+        for (uint32_t q = nseg; q-- > 0;) { seg[q] = (uint32_t)(flat % R); flat /= R; }
+        const uint32_t c = j * (uint32_t)base + (uint32_t)flat;
+        const Config k = config_of(s, c);
+        for (int q = 0; q < (int)sizeof(*out); ++q) reinterpret_cast<unsigned char*>(out)[q] = 0;
+        out->P = (uint8_t)P;
+        out->mbs_idx = (uint8_t)k.mi;
+        out->rc = (uint8_t)k.rc;
+        out->D = (uint16_t)k.D;
+        out->n_runs = (uint8_t)nseg;
+        for (uint32_t q = 0; q < nseg; ++q) {
+            // stages of segment q: floor(i*nseg/P) == q  <=>  ceil(q*P/nseg) <= i < ceil((q+1)*P/nseg)
+            const uint32_t a = (q * P + nseg - 1) / nseg, e = ((q + 1) * P + nseg - 1) / nseg;
+            out->run[q].type = (uint8_t)(seg[q] % T);
+            out->run[q].zone = (uint8_t)(seg[q] / T);
+            out->run[q].tp_idx = (uint8_t)k.tpi;
+            out->run[q].n_stages = (uint8_t)(e - a);
+        }
+        return true;
+    }
+    return false;
+}
+
+}  // namespace sailor
