@@ -1,0 +1,361 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.  Integer results (status, bytes, flat indices, counts) must be bit-exact; times
+and costs must agree within 1e-5 relative (binary64) — and, because both sides follow one
+written-down operation order without contraction, are also expected to be bit-identical."""
+import ctypes as C
+import math
+
+import numpy as np
+import pytest
+
+from helpers import REL_TOL_F64, golden_cases, rel_close, stages_to_records, workload_from_tables
+from oracle.binding import Oracle, parallel_search
+from paper_2504_17096_b200 import binding as B
+from paper_2504_17096_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def torch_cuda():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    return torch
+
+
+class Ctx:
+    def __init__(self, w, avail=None):
+        self.w = w
+        self.ctx = B.sailor_create(w, 0, 0)
+        B.sailor_set_availability(self.ctx, w.avail if avail is None else avail)
+        self.space = B.make_space(w)
+
+    def close(self):
+        B.sailor_destroy(self.ctx)
+
+
+@pytest.fixture
+def make_ctx(torch_cuda):
+    made = []
+
+    def _make(w, avail=None):
+        c = Ctx(w, avail)
+        made.append(c)
+        return c
+
+    yield _make
+    for c in made:
+        c.close()
+
+
+def assert_sim_equal(gpu, orc, what=""):
+    t, m, c, s = gpu
+    so, to, co, mo = orc
+    assert np.array_equal(s, so), f"{what}: status differs at {np.flatnonzero(s != so)[:5]}"
+    assert np.array_equal(m, mo), f"{what}: peak memory differs at {np.flatnonzero(m != mo)[:5]}"
+    assert rel_close(t, to, REL_TOL_F64), f"{what}: t_iter beyond {REL_TOL_F64}"
+    assert rel_close(c, co, REL_TOL_F64), f"{what}: cost beyond {REL_TOL_F64}"
+    # one operation order on both sides: identical bits
+    ok = ~np.isnan(to)
+    assert np.array_equal(np.isnan(t), np.isnan(to)) and np.array_equal(np.isnan(c), np.isnan(co))
+    assert np.array_equal(t[ok].view(np.uint64), to[ok].view(np.uint64)), f"{what}: t_iter bits"
+    assert np.array_equal(c[ok].view(np.uint64), co[ok].view(np.uint64)), f"{what}: cost bits"
+
+
+# ---- sailor_simulate -----------------------------------------------------------------------------
+
+@pytest.mark.parametrize("case", golden_cases(), ids=lambda c: c["name"])
+def test_simulate_hand_worked_cases(case, make_ctx):
+    w = workload_from_tables(case["tables"])
+    cx = make_ctx(w)
+    recs = B.pack_records(stages_to_records([case["plan"]]))
+    t, m, c, s = B.sailor_simulate(cx.ctx, recs)
+    e = case["expect"]
+    assert s[0] == e["status"] and m[0] == e["peak_mem"]
+    if e.get("nan"):
+        assert math.isnan(t[0]) and math.isnan(c[0])
+    else:
+        assert t[0] == pytest.approx(e["t_iter"], rel=1e-12)
+        assert c[0] == pytest.approx(e["cost"], rel=1e-12)
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 5])
+def test_simulate_random_records_match_oracle(cfg, make_ctx):
+    w = W.CONFIGS[cfg]()
+    cx = make_ctx(w)
+    n = 20011                         # several 256-record tiles and a ragged tail
+    recs = W.random_plans(w, n, seed=100 + cfg, hetero_tp=True)
+    gpu = B.sailor_simulate(cx.ctx, B.pack_records(recs))
+    orc = Oracle(w).simulate_records(recs)
+    assert_sim_equal(gpu, orc, f"cfg{cfg}")
+    assert len(np.unique(gpu[3])) >= 3          # the sample exercises several status combinations
+
+
+def test_simulate_tiny_with_latency_terms(make_ctx):
+    w = W.tiny(seed=5, n_types=3, n_zones=2)
+    cx = make_ctx(w)
+    recs = W.random_plans(w, 5000, seed=77, hetero_tp=True)
+    assert_sim_equal(B.sailor_simulate(cx.ctx, B.pack_records(recs)), Oracle(w).simulate_records(recs), "tiny")
+
+
+def test_simulate_device_pointers(make_ctx, torch_cuda):
+    torch = torch_cuda
+    w = W.config2()
+    cx = make_ctx(w)
+    n = 4099
+    recs = W.random_plans(w, n, seed=9, hetero_tp=False)
+    packed = B.pack_records(recs)
+    d_plans = torch.from_numpy(packed.view(np.uint8).reshape(n, 72).copy()).cuda()
+    t = torch.empty(n, dtype=torch.float64, device="cuda")
+    c = torch.empty(n, dtype=torch.float64, device="cuda")
+    m = torch.empty(n, dtype=torch.int64, device="cuda")
+    s = torch.empty(n, dtype=torch.int32, device="cuda")
+    B.sailor_simulate_device(cx.ctx, d_plans.data_ptr(), n, t.data_ptr(), m.data_ptr(), c.data_ptr(), s.data_ptr())
+    torch.cuda.synchronize()
+    gpu = (t.cpu().numpy(), m.cpu().numpy().view(np.uint64), c.cpu().numpy(), s.cpu().numpy().view(np.uint32))
+    assert_sim_equal(gpu, Oracle(w).simulate_records(recs), "device pointers")
+
+
+def test_simulate_empty_and_bad_records(make_ctx, torch_cuda):
+    torch = torch_cuda
+    w = W.config1()
+    cx = make_ctx(w)
+    t, m, c, s = B.sailor_simulate(cx.ctx, np.zeros(0, dtype=B.REC_DTYPE))
+    assert t.size == 0
+    good = stages_to_records([dict(P=2, mbs_idx=0, rc=0, D=1, type=[0, 1], zone=[0, 0], tp_idx=[0, 0])])
+    for field, value in (("P", 3), ("mbs_idx", 9), ("D", 0), ("n_runs", 17)):
+        bad = B.pack_records(good)
+        bad[field] = value
+        with pytest.raises(B.SailorError) as e:
+            B.sailor_simulate(cx.ctx, bad)
+        assert e.value.code == B.E_RANGE
+    bad = B.pack_records(good)
+    bad["run"]["type"][0, 1] = 5
+    with pytest.raises(B.SailorError):
+        B.sailor_simulate(cx.ctx, bad)
+    # the same records given on the device are flagged by the kernel's own bounds checks
+    both = np.concatenate([B.pack_records(good), bad])
+    d = torch.from_numpy(both.view(np.uint8).reshape(2, 72).copy()).cuda()
+    st = torch.zeros(2, dtype=torch.int32, device="cuda")
+    tt = torch.zeros(2, dtype=torch.float64, device="cuda")
+    B.sailor_simulate_device(cx.ctx, d.data_ptr(), 2, tt.data_ptr(), 0, 0, st.data_ptr())
+    torch.cuda.synchronize()
+    assert st.cpu().tolist()[1] == B.ST_BAD_RECORD and (st.cpu().tolist()[0] & B.ST_BAD_RECORD) == 0
+    assert math.isnan(tt.cpu().tolist()[1])
+
+
+# ---- enumeration ---------------------------------------------------------------------------------
+
+def _rec_stages(r):
+    types, zones, tps = [], [], []
+    for q in range(r.n_runs):
+        for _ in range(r.run[q].n_stages):
+            types.append(r.run[q].type); zones.append(r.run[q].zone); tps.append(r.run[q].tp_idx)
+    return (r.P, r.mbs_idx, r.rc, r.D, tuple(types), tuple(zones), tuple(tps))
+
+
+def _orc_stages(pl):
+    return (pl.P, pl.mbs_idx, pl.rc, pl.D, tuple(pl.type[: pl.P]), tuple(pl.zone[: pl.P]), tuple(pl.tp_idx[: pl.P]))
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 5])
+def test_space_size_and_decode_match_oracle(cfg, make_ctx):
+    w = W.CONFIGS[cfg]()
+    cx = make_ctx(w)
+    o = Oracle(w)
+    n = B.sailor_space_size(cx.ctx, cx.space)
+    assert n == o.space_size() == w.space_size()
+    rng = W.SplitMix64(cfg)
+    flats = [0, 1, n - 1] + [rng.next_u64() % n for _ in range(300)]
+    for f in flats:
+        assert _rec_stages(B.sailor_decode(cx.ctx, cx.space, f)) == _orc_stages(o.decode(f))
+    with pytest.raises(B.SailorError):
+        B.sailor_decode(cx.ctx, cx.space, n)
+
+
+# ---- sailor_plan ---------------------------------------------------------------------------------
+
+COUNT_KEYS = ("n_total", "n_invalid", "n_oom", "n_over_avail", "n_over_constraint", "n_feasible")
+
+
+def assert_plan_equal(res, st, hits, counts, oracle, what=""):
+    assert [r.flat for r in res] == [h["flat"] for h in hits], what
+    for r, h in zip(res, hits):
+        assert r.status == 0
+        assert r.peak_mem == h["peak_mem"]
+        assert rel_close([r.t_iter, r.cost, r.score], [h["t_iter"], h["cost"], h["score"]], REL_TOL_F64)
+        assert (r.t_iter, r.cost, r.score) == (h["t_iter"], h["cost"], h["score"])      # identical bits
+        assert _rec_stages(r.plan) == _orc_stages(oracle.decode(r.flat))
+    if counts is not None:
+        assert {k: getattr(st, k) for k in COUNT_KEYS} == {k: counts[k] for k in COUNT_KEYS}, what
+        assert st.min_feasible_cost == counts["min_cost"]
+
+
+@pytest.mark.parametrize("seed,T,Z,seg_max", [(1, 2, 2, 4), (2, 3, 2, 4), (3, 2, 1, 4), (4, 3, 3, 2), (5, 1, 1, 4), (6, 2, 2, 1)])
+@pytest.mark.parametrize("objective", [W.OBJ_MAX_THROUGHPUT, W.OBJ_MIN_COST, W.OBJ_MAX_THROUGHPUT_PER_USD])
+def test_plan_tiny_spaces_match_exhaustive_oracle(seed, T, Z, seg_max, objective, make_ctx):
+    w = W.tiny(seed=seed, n_types=T, n_zones=Z, seg_max=seg_max, objective=objective)
+    cx = make_ctx(w)
+    o = Oracle(w)
+    for k in (1, 7, 32):
+        hits, counts = o.search(objective, k)
+        for flags in (0, B.FLAG_EVAL_ALL):
+            res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=flags), k)
+            assert_plan_equal(res, st, hits, counts, o, f"k={k} flags={flags}")
+
+
+def test_plan_constraints_and_empty_results(make_ctx):
+    w = W.tiny(seed=8, n_types=2, n_zones=2)
+    cx = make_ctx(w)
+    o = Oracle(w)
+    allh, _ = o.search(w.objective, 32)
+    budget = sorted(h["cost"] for h in allh)[5]
+    rate = 1.0 / allh[10]["t_iter"]
+    for kw in (dict(budget=budget), dict(min_rate=rate), dict(budget=budget, min_rate=rate)):
+        hits, counts = o.search(w.objective, 9, **kw)
+        res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, **kw), 9)
+        assert_plan_equal(res, st, hits, counts, o, str(kw))
+    # nothing is available: an empty result, not an error
+    B.sailor_set_availability(cx.ctx, np.zeros_like(w.avail))
+    res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w), 4)
+    assert res == [] and st.n_feasible == 0 and st.n_total == o.space_size()
+    # k larger than the feasible set
+    B.sailor_set_availability(cx.ctx, w.avail)
+    cheap, _ = o.search(W.OBJ_MIN_COST, 6)
+    budget = cheap[-1]["cost"]
+    hits, counts = o.search(w.objective, 32, budget=budget)
+    res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, budget=budget), 32)
+    assert 6 <= len(res) == len(hits) < 32
+    assert_plan_equal(res, st, hits, counts, o)
+
+
+def test_plan_argument_errors(make_ctx):
+    w = W.tiny(seed=2)
+    cx = make_ctx(w)
+    L = B.load()
+    res = (B.Result * 40)()
+    n = C.c_uint32()
+    obj = B.make_objective(w)
+    assert L.sailor_plan(cx.ctx, C.byref(cx.space), C.byref(obj), 0, res, C.byref(n), None) == B.E_ARG
+    assert L.sailor_plan(cx.ctx, C.byref(cx.space), C.byref(obj), 33, res, C.byref(n), None) == B.E_RANGE
+    assert L.sailor_plan(cx.ctx, None, C.byref(obj), 1, res, C.byref(n), None) == B.E_ARG
+    bad = B.make_space(w)
+    bad.n_d = 0
+    assert L.sailor_plan(cx.ctx, C.byref(bad), C.byref(obj), 1, res, C.byref(n), None) == B.E_ARG
+    bad = B.make_space(w)
+    bad.tp_idx[0] = 7
+    assert L.sailor_plan(cx.ctx, C.byref(bad), C.byref(obj), 1, res, C.byref(n), None) == B.E_RANGE
+    bad = B.make_space(w)
+    bad.seg_max = 5
+    assert L.sailor_plan(cx.ctx, C.byref(bad), C.byref(obj), 1, res, C.byref(n), None) == B.E_RANGE
+
+
+def test_plan_range_split_merges_to_full(make_ctx):
+    w = W.config1()
+    cx = make_ctx(w)
+    o = Oracle(w)
+    n = o.space_size()
+    obj = B.make_objective(w)
+    full, st_full = B.sailor_plan(cx.ctx, cx.space, obj, 16)
+    edges = [0, 1, 143, 144, 1000, 3333, 6767, n]
+    merged, total = [], 0
+    for a, b in zip(edges[:-1], edges[1:]):
+        res, st = B.sailor_plan_range(cx.ctx, cx.space, obj, a, b, 16)
+        hits, counts = o.search(w.objective, 16, lo=a, hi=b)
+        assert_plan_equal(res, st, hits, counts, o, f"[{a},{b})")
+        merged += [(r.score, r.flat) for r in res]
+        total += st.n_total
+    assert total == n == st_full.n_total
+    assert sorted(merged)[:16] == [(r.score, r.flat) for r in full]
+
+
+def test_plan_config1_full(make_ctx):
+    w = W.config1()
+    cx = make_ctx(w)
+    o = Oracle(w)
+    hits, counts = o.search(w.objective, 32)
+    for flags in (0, B.FLAG_EVAL_ALL):
+        res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=flags), 32)
+        assert_plan_equal(res, st, hits, counts, o)
+
+
+def test_plan_config2_budget_factor_two_pass(make_ctx):
+    w = W.config2()
+    cx = make_ctx(w)
+    o = Oracle(w)
+    hits, counts, budget = o.plan(16)
+    res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w), 16)
+    assert st.budget_used == budget
+    assert_plan_equal(res, st, hits, counts, o)
+
+
+def test_plan_config4_snapshots_replan(make_ctx):
+    """Dynamic availability: re-plan per snapshot on one context; only the counts are uploaded."""
+    w = W.config4(n_snapshots=200)
+    cx = make_ctx(w)
+    o = Oracle(w)
+    obj = B.make_objective(w)
+    checked = 0
+    for t in range(0, 200, 8):                       # 25 of the 200 snapshots
+        snap = w.snapshots[t]
+        o.set_availability(snap)
+        B.sailor_set_availability(cx.ctx, snap)
+        hits, counts, budget = o.plan(4)
+        res, st = B.sailor_plan(cx.ctx, cx.space, obj, 4)
+        if hits:
+            assert st.budget_used == budget
+            assert_plan_equal(res, st, hits, counts, o, f"snapshot {t}")
+        else:
+            assert res == []
+        checked += 1
+    assert checked == 25
+
+
+def test_plan_config3_full_space(make_ctx):
+    """3.6e8 candidates: the whole space on the GPU, the oracle split over the host's cores."""
+    w = W.config3()
+    cx = make_ctx(w)
+    hits, counts = parallel_search(w, w.objective, 16)
+    o = Oracle(w)
+    for flags in (0, B.FLAG_EVAL_ALL):
+        res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=flags), 16)
+        assert_plan_equal(res, st, hits, counts, o, f"flags={flags}")
+
+
+def test_plan_config5_windows_and_sampled_winner(make_ctx):
+    """6.4e9 candidates.  Exact on windows the oracle can enumerate; for the full space the
+    winners are re-simulated by the oracle and no sampled candidate may beat them."""
+    w = W.config5()
+    cx = make_ctx(w)
+    o = Oracle(w)
+    n = o.space_size()
+    obj = B.make_objective(w, flags=B.FLAG_EVAL_ALL)
+    rng = W.SplitMix64(55)
+    res, st = B.sailor_plan(cx.ctx, cx.space, obj, 32)
+    res2, st2 = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w), 32)       # with pruning: same answer
+    assert [(r.flat, r.score) for r in res] == [(r.flat, r.score) for r in res2]
+    assert {k: getattr(st, k) for k in COUNT_KEYS} == {k: getattr(st2, k) for k in COUNT_KEYS}
+    assert st.n_total == n and len(res) == 32 and st.n_feasible > 0
+    flats = np.array([r.flat for r in res], dtype=np.uint64)
+    so, to, co, mo = o.simulate_flat(flats)
+    assert np.all(so == 0)
+    assert [r.t_iter for r in res] == list(to) and [r.cost for r in res] == list(co)
+    assert [r.peak_mem for r in res] == list(mo)
+    assert [(r.score, r.flat) for r in res] == sorted((r.score, r.flat) for r in res)
+    # windows the oracle enumerates in full: both ends, random places, and around the winner
+    best = int(res[0].flat)
+    windows = [(0, 300_000), (n - 250_000, n), (max(0, best - 200_000), min(n, best + 200_000))]
+    windows += [(s, s + 400_003) for s in (rng.next_u64() % (n - 500_000) for _ in range(3))]
+    for a, b in windows:
+        hits, counts = o.search(w.objective, 8, lo=a, hi=b)
+        r, s = B.sailor_plan_range(cx.ctx, cx.space, obj, a, b, 8)
+        assert_plan_equal(r, s, hits, counts, o, f"[{a},{b})")
+    # seeded uniform subsample of 1e6 flat indices: none is feasible and better than the k-th kept
+    sample = np.array(sorted({rng.next_u64() % n for _ in range(1_000_000)}), dtype=np.uint64)
+    ss, ts, cs_, ms = o.simulate_flat(sample)
+    feas = ss == 0
+    worst = (res[-1].score, res[-1].flat)
+    kept = {r.flat for r in res}
+    for f, t in zip(sample[feas], ts[feas]):
+        assert (t, int(f)) >= worst or int(f) in kept
