@@ -246,6 +246,37 @@ int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objec
                       uint64_t flat_lo, uint64_t flat_hi,
                       uint32_t k, sailor_result* topk, uint32_t* n_found, sailor_stats* stats);
 
+/* Search without allocating.  (The paper has no counterpart: this entry point exists for the
+ * sake of callers, not of the method.)
+ *
+ * sailor_plan allocates device memory whenever it meets a space it has not cached (two
+ * cudaMalloc / cudaFree pairs for the per-configuration index arrays).  Some callers cannot
+ * afford or are not allowed that: a re-planning loop inside a training process whose memory
+ * pool already owns the whole GPU, where a further cudaMalloc fails; a latency-critical
+ * controller for which cudaMalloc's device-wide synchronisation stalls every other stream;
+ * a thread that runs while another thread of the process captures a stream in the global
+ * capture mode, during which cudaMalloc is an error.  This variant computes exactly what
+ * sailor_plan computes (whole space, same results, same statistics) but calls no cudaMalloc,
+ * cudaFree or any other allocating routine: all of its working memory (work counter,
+ * statistics, per-block top-k lists, result records, per-configuration index arrays) lies in
+ * one array of about 0.6 MB that is part of the library image, so every GPU that loads the
+ * library holds it until the process exits.  The context must already exist (sailor_create
+ * allocates; call it at set-up).
+ *
+ * Limit: at most SAILOR_NOALLOC_CONFIG_MAX configurations, i.e.
+ * n_p * n_mbs * n_tp * n_rc * n_d <= 4096; a larger space returns SAILOR_E_RANGE and nothing
+ * is launched.  Other errors as sailor_plan.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call before any stream capture begins.
+ * All calls, from every context on a device, share the one array: it keeps the previous
+ * call's contents (the counters are cleared at the start of each call), and two calls that
+ * overlap on the GPU (different streams or threads) race on it and return garbage.  Issue
+ * them one after the other. */
+#define SAILOR_NOALLOC_CONFIG_MAX 4096
+int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint32_t k,
+                        sailor_result* topk, uint32_t* n_found, sailor_stats* stats);
+
 const char* sailor_strerror(int code);
 int sailor_last_cuda_error(const sailor_ctx* ctx);   /* cudaError_t of the last E_CUDA      */
 

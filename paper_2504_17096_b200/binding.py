@@ -19,8 +19,8 @@ OBJ_MAX_THROUGHPUT, OBJ_MIN_COST, OBJ_MAX_THROUGHPUT_PER_USD = 0, 1, 2
 FLAG_EVAL_ALL = 1
 
 EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
-           "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_strerror",
-           "sailor_last_cuda_error")
+           "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_plan_noalloc",
+           "sailor_strerror", "sailor_last_cuda_error")
 
 _dp, _u64p, _u32p, _u16p = C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.POINTER(C.c_uint16)
 
@@ -120,6 +120,7 @@ def load() -> C.CDLL:
                               C.POINTER(Stats)]
     L.sailor_plan_range.argtypes = [vp, C.POINTER(Space), C.POINTER(Objective), C.c_uint64, C.c_uint64, C.c_uint32,
                                     C.POINTER(Result), _u32p, C.POINTER(Stats)]
+    L.sailor_plan_noalloc.argtypes = L.sailor_plan.argtypes
     L.sailor_strerror.argtypes = [C.c_int]
     L.sailor_strerror.restype = C.c_char_p
     L.sailor_last_cuda_error.argtypes = [vp]
@@ -261,6 +262,18 @@ def sailor_plan(ctx, space: Space, obj: Objective, k: int):
     n = C.c_uint32()
     st = Stats()
     _check(load().sailor_plan(ctx, C.byref(space), C.byref(obj), k, res, C.byref(n), C.byref(st)), "sailor_plan", ctx)
+    return list(res[: n.value]), st
+
+
+def sailor_plan_noalloc(ctx, space: Space, obj: Objective, k: int):
+    """The search of sailor_plan for callers that must not allocate device memory: all working
+    memory comes from a fixed array inside the library (spaces of at most 4096 configurations;
+    calls on one GPU must not overlap).  Same return values as sailor_plan."""
+    res = (Result * k)()
+    n = C.c_uint32()
+    st = Stats()
+    _check(load().sailor_plan_noalloc(ctx, C.byref(space), C.byref(obj), k, res, C.byref(n), C.byref(st)),
+           "sailor_plan_noalloc", ctx)
     return list(res[: n.value]), st
 
 

@@ -693,3 +693,201 @@ int sailor_plan(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* 
 }
 
 }  // extern "C"
+
+// ---- search without device allocation ----------------------------------------------------------
+//
+// sailor_plan_range keeps its per-space index arrays in memory it allocates when a new space
+// arrives.  The variant below takes every byte of working memory from one fixed array that is
+// part of the library image instead, so it can serve callers that must not allocate.
+
+namespace {
+
+constexpr uint32_t NOALLOC_GRID_MAX = 1024;     // blocks whose partial lists fit the fixed scratch
+
+struct NoAllocScratch {                         // layout of the fixed scratch array
+    Ctrl ctrl;
+    sailor_result results[SAILOR_K_MAX];
+    uint32_t partial_n[NOALLOC_GRID_MAX];
+    Hit partial[(size_t)NOALLOC_GRID_MAX * SAILOR_K_MAX];
+    uint32_t cfg_chunk_start[SAILOR_NOALLOC_CONFIG_MAX + 1];
+    uint64_t cfg_flat_base[SAILOR_NOALLOC_CONFIG_MAX];
+};
+
+// About 0.6 MB, held by every GPU that loads the library until the process exits.  In host code
+// this name is only a handle for cudaGetSymbolAddress; it is never passed to a kernel.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+constexpr int NOALLOC_DEVICES_MAX = 64;
+NoAllocScratch* g_noalloc_ptr[NOALLOC_DEVICES_MAX] = {};     // device address of the array, per device
+
+// Device address of the scratch on the current device; resolved on first use per device.
+int noalloc_scratch(sailor_ctx* ctx, NoAllocScratch** out) {
+    if (ctx->device < 0 || ctx->device >= NOALLOC_DEVICES_MAX) return SAILOR_E_RANGE;
+    if (!g_noalloc_ptr[ctx->device]) {
+        void* p = nullptr;
+        CU(ctx, cudaGetSymbolAddress(&p, g_noalloc_scratch));
+        g_noalloc_ptr[ctx->device] = static_cast<NoAllocScratch*>(p);
+    }
+    *out = g_noalloc_ptr[ctx->device];
+    return SAILOR_OK;
+}
+
+// One pass (clear, search, merge) whose scratch all lies in `sc`.
+int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& desc, uint32_t n_config,
+                         uint32_t p_max, size_t smem, uint32_t chunk_lo, uint32_t chunk_hi, uint64_t total,
+                         uint32_t obj, double budget, bool budget_from_ctrl, double min_rate, uint32_t flags,
+                         uint32_t k, double next_budget_factor, uint32_t* n_launches) {
+    // the array keeps the previous call's contents: counters and the work counter restart at zero
+    CU(ctx, cudaMemsetAsync(&sc->ctrl, 0, offsetof(Ctrl, min_cost_bits), ctx->stream));
+    CU(ctx, cudaMemsetAsync(&sc->ctrl.min_cost_bits, 0x7f, sizeof(unsigned long long), ctx->stream));
+    PlanParams pp;
+    memset(&pp, 0, sizeof(pp));
+    pp.blob = ctx->d_blob;
+    pp.avail = ctx->d_avail;
+    pp.cfg_chunk_start = sc->cfg_chunk_start;
+    pp.cfg_flat_base = sc->cfg_flat_base;
+    pp.ctrl = &sc->ctrl;
+    pp.partial = sc->partial;
+    pp.partial_n = sc->partial_n;
+    pp.sp = desc;
+    pp.n_config = n_config;
+    pp.flat_lo = 0;
+    pp.flat_hi = total;
+    pp.k = k;
+    pp.eval_all = (flags & SAILOR_FLAG_EVAL_ALL) ? 1u : 0u;
+    pp.budget_from_ctrl = budget_from_ctrl ? 1u : 0u;
+    pp.p_max = p_max;
+    pp.budget = budget;
+    pp.min_rate = min_rate;
+    pp.chunk_lo = chunk_lo;
+    pp.chunk_hi = chunk_hi;
+    const uint32_t n_chunks = chunk_hi - chunk_lo;
+    const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
+    PlanKernel kern = pick_kernel(obj, constr);
+    // the opt-in is per kernel, not per call site: ask for the library-wide ceiling so that it also
+    // covers whatever another context's search set it to
+    CU(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    int per_sm = 0;
+    CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, smem));
+    if (per_sm < 1) return SAILOR_E_RANGE;
+    uint32_t grid = (uint32_t)per_sm * (uint32_t)ctx->sm_count;
+    if (grid > NOALLOC_GRID_MAX) grid = NOALLOC_GRID_MAX;
+    if (grid > n_chunks) grid = n_chunks;
+    const uint32_t batch = n_chunks / (grid * 32u);
+    pp.batch = batch < 1 ? 1 : (batch > 16 ? 16 : batch);
+    kern<<<grid, PLAN_THREADS, smem, ctx->stream>>>(pp);
+    CU(ctx, cudaGetLastError());
+    ++*n_launches;
+    MergeParams mp;
+    memset(&mp, 0, sizeof(mp));
+    mp.blob = ctx->d_blob;
+    mp.avail = ctx->d_avail;
+    mp.partial = sc->partial;
+    mp.partial_n = sc->partial_n;
+    mp.ctrl = &sc->ctrl;
+    mp.results = sc->results;
+    mp.sp = desc;
+    mp.n_partial = grid;
+    mp.k = k;
+    mp.obj = obj;
+    mp.budget_factor = next_budget_factor;
+    merge_kernel<<<1, MERGE_THREADS, 0, ctx->stream>>>(mp);
+    CU(ctx, cudaGetLastError());
+    ++*n_launches;
+    return SAILOR_OK;
+}
+
+}  // namespace
+
+extern "C" int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint32_t k,
+                                   sailor_result* topk, uint32_t* n_found, sailor_stats* stats) {
+    if (!ctx || !s || !o || !topk || !n_found || k == 0) return SAILOR_E_ARG;
+    if (k > SAILOR_K_MAX || o->kind > SAILOR_OBJ_MAX_THROUGHPUT_PER_USD) return SAILOR_E_RANGE;
+    if (std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) ||
+        std::isnan(o->budget_factor_over_cheapest))
+        return SAILOR_E_ARG;
+    int rc = check_space(ctx, s);
+    if (rc) return rc;
+    const SpaceDesc d = to_desc(s);
+    uint64_t total = 0;
+    rc = space_total(ctx, d, &total);
+    if (rc) return rc;
+    const uint32_t per_p = d.n_mbs * d.n_tp * d.n_rc * d.n_d;
+    const uint64_t n_config = (uint64_t)per_p * d.n_p;
+    if (n_config > SAILOR_NOALLOC_CONFIG_MAX) return SAILOR_E_RANGE;       // beyond the fixed scratch
+
+    // per-configuration offsets, built in fixed-size host arrays (thread-local: no heap, no device memory)
+    static thread_local uint32_t h_chunk_start[SAILOR_NOALLOC_CONFIG_MAX + 1];
+    static thread_local uint64_t h_flat_base[SAILOR_NOALLOC_CONFIG_MAX];
+    const uint64_t R = ctx->hdr.R;
+    uint64_t chunks = 0, flat = 0;
+    uint32_t p_max = 0;
+    for (uint32_t j = 0; j < d.n_p; ++j) {
+        const uint32_t nseg = nseg_of(d.p_values[j], d.seg_max);
+        p_max = d.p_values[j] > p_max ? d.p_values[j] : p_max;
+        const uint64_t items = ipow64(R, nseg - 1);
+        const uint64_t per_cfg = (items + PLAN_THREADS - 1) / PLAN_THREADS;
+        for (uint32_t c = 0; c < per_p; ++c) {
+            h_chunk_start[(size_t)j * per_p + c] = (uint32_t)chunks;
+            h_flat_base[(size_t)j * per_p + c] = flat;
+            chunks += per_cfg;
+            flat += items * R;
+            if (chunks >= 0xfff00000ull) return SAILOR_E_RANGE;
+        }
+    }
+    h_chunk_start[n_config] = (uint32_t)chunks;
+    const size_t smem = plan_smem_bytes(ctx->hdr.static_bytes, p_max, ctx->hdr.T, ctx->hdr.Z);
+    if (smem > 200 * 1024) return SAILOR_E_RANGE;
+
+    DeviceGuard guard(ctx->device);
+    NoAllocScratch* sc = nullptr;
+    rc = noalloc_scratch(ctx, &sc);
+    if (rc) return rc;
+    // the host arrays are reused by the next call on this thread: wait for the copies below at the end
+    CU(ctx, cudaMemcpyAsync(sc->cfg_chunk_start, h_chunk_start, (n_config + 1) * sizeof(uint32_t),
+                            cudaMemcpyHostToDevice, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(sc->cfg_flat_base, h_flat_base, n_config * sizeof(uint64_t), cudaMemcpyHostToDevice,
+                            ctx->stream));
+    CU(ctx, cudaMemsetAsync(&sc->ctrl, 0, sizeof(Ctrl), ctx->stream));      // also the sticky error word
+
+    uint32_t launches = 0;
+    CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
+    const bool two_pass = o->budget_factor_over_cheapest > 0.0;
+    if (total > 0) {
+        if (two_pass) {
+            rc = enqueue_pass_noalloc(ctx, sc, d, (uint32_t)n_config, p_max, smem, 0, (uint32_t)chunks, total,
+                                      SAILOR_OBJ_MIN_COST, 0.0, false, 0.0, o->flags, 1,
+                                      o->budget_factor_over_cheapest, &launches);
+            if (rc) return rc;
+        }
+        rc = enqueue_pass_noalloc(ctx, sc, d, (uint32_t)n_config, p_max, smem, 0, (uint32_t)chunks, total, o->kind,
+                                  o->budget_usd_per_iter, two_pass, o->min_iters_per_s, o->flags, k, 0.0, &launches);
+        if (rc) return rc;
+    }
+    CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(ctx->h_out->results, sc->results, sizeof(sailor_result) * k, cudaMemcpyDeviceToHost,
+                            ctx->stream));
+    CU(ctx, cudaMemcpyAsync(&ctx->h_out->ctrl, &sc->ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, cudaStreamSynchronize(ctx->stream));
+    const Ctrl& cr = ctx->h_out->ctrl;
+    if (cr.error) return SAILOR_E_DEVICE;
+    *n_found = cr.n_found;
+    memcpy(topk, ctx->h_out->results, sizeof(sailor_result) * cr.n_found);
+    if (stats) {
+        stats->n_total = cr.stats[0];
+        stats->n_invalid = cr.stats[1];
+        stats->n_oom = cr.stats[2];
+        stats->n_over_avail = cr.stats[3];
+        stats->n_over_constraint = cr.stats[4];
+        stats->n_feasible = cr.stats[5];
+        stats->budget_used = two_pass ? cr.budget : o->budget_usd_per_iter;
+        double mc;
+        memcpy(&mc, &cr.min_cost_bits, sizeof(mc));
+        stats->min_feasible_cost = cr.stats[5] ? mc : 0.0;
+        float ms = 0.f;
+        CU(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
+        stats->kernel_ms = ms;
+        stats->n_launches = launches;
+    }
+    return SAILOR_OK;
+}
