@@ -123,12 +123,31 @@ struct WarpTopK {
 };
 
 // ---- per-configuration tables in shared memory ---------------------------------------------
+//
+// Inside one segment all stages share (type, zone, tp), so their per-microbatch times take at
+// most four distinct values, in stage order: stage 0 (embedding), stages with one extra block,
+// plain stages, the final stage (head, sends nothing).  A segment is therefore stored as four
+// (count, value[digit]) runs; adding `count` copies of `value` one after the other is the same
+// sequence of additions as walking the stages.  The last stage of a non-final segment sends to
+// the next segment, so its time depends on two digits and is kept apart (fb_last + c2x).
+constexpr int N_RUNS = 4;
+
+struct alignas(16) SegRec {                  // one per (segment, digit); 64 bytes, read as broadcasts
+    double v[N_RUNS];            // t_i of each run (f + b + 2c with the next stage on the same digit)
+    double tmax;                 // max of v[] over the non-empty runs
+    double sync;                 // max all-reduce time over the segment's stages
+    double upd;                  // max update time over the segment's stages
+    double rate;                 // D * tp * price per second of one stage
+};
+
 struct CfgShared {
     // scalars (written by thread 0 / the build, read by all)
     Config cfg;
     uint32_t valid;              // gbs % (D*mbs) == 0 and heads % tp == 0
     uint32_t seg_a[SAILOR_SEG_MAX + 1];   // first stage of each segment; seg_a[nseg] = P
     uint32_t need[SAILOR_SEG_MAX];        // GPUs a segment takes of its digit: D * tp * stages
+    uint32_t n_run[SAILOR_SEG_MAX][N_RUNS];   // stages in each run (without a non-final segment's last stage)
+    uint32_t magic;              // floor(2^32 / R) + 1: x / R == umulhi(x, magic) for x < 2^26
     uint64_t n_b;
     uint64_t n_items;            // R^(nseg-1)
     uint64_t invalid_mask;       // digit d: tp > gpus_per_node[type(d)]
@@ -143,37 +162,43 @@ struct CfgShared {
 };
 
 struct CfgArrays {               // pointers into dynamic shared memory
-    double *fb, *uu;             // [P][T]   f+b (+f if rc), update
-    double* tself;               // [P][R]   t_i when stage i+1 has the same digit (last stage: no message)
-    double *seg_tmax, *seg_sync, *seg_upd;   // [nseg][R]
-    double* rate_d;              // [R]      D * tp * price per second
+    SegRec* rec;                 // [SEG_MAX][R]
     double* c2x;                 // [R][R]   2 * message time, index [next digit][this digit]
-    double* commx;               // [Z][Z]   transfer cost of one boundary, index [next zone][this zone]
+    double* commx;               // [R][Z]   transfer cost of one boundary, index [next digit][this zone]
+    double* fb_last;             // [SEG_MAX][T]  f+b of a segment's last stage, per type
+    double *fb, *uu;             // [P][T]   build scratch: f+b (+f if rc), update
     uint32_t* availv;            // [R]
+    uint32_t* tz;                // [R]      type | zone << 8 of a digit
 };
 
 __host__ __device__ inline size_t plan_smem_bytes(uint32_t static_bytes, uint32_t p_max, uint32_t T, uint32_t Z) {
     const size_t R = (size_t)T * Z;
     size_t n = static_bytes;
-    n += sizeof(double) * (2 * (size_t)p_max * T + (size_t)p_max * R + 3 * SAILOR_SEG_MAX * R + R + R * R + (size_t)Z * Z);
-    n += sizeof(uint32_t) * R;
+    n += sizeof(SegRec) * SAILOR_SEG_MAX * R;
+    n += sizeof(double) * (R * R + R * Z + (size_t)SAILOR_SEG_MAX * T + 2 * (size_t)p_max * T);
+    n += sizeof(uint32_t) * 2 * R;
     return (n + 15) & ~(size_t)15;
 }
 
 __device__ __forceinline__ void carve(unsigned char* dyn, uint32_t static_bytes, uint32_t p_max, uint32_t T,
                                       uint32_t Z, CfgArrays& a) {
     const uint32_t R = T * Z;
-    double* p = reinterpret_cast<double*>(dyn + static_bytes);
+    a.rec = reinterpret_cast<SegRec*>(dyn + static_bytes);           // static_bytes is a multiple of 16
+    double* p = reinterpret_cast<double*>(a.rec + (size_t)SAILOR_SEG_MAX * R);
+    a.c2x = p;       p += (size_t)R * R;
+    a.commx = p;     p += (size_t)R * Z;
+    a.fb_last = p;   p += (size_t)SAILOR_SEG_MAX * T;
     a.fb = p;        p += (size_t)p_max * T;
     a.uu = p;        p += (size_t)p_max * T;
-    a.tself = p;     p += (size_t)p_max * R;
-    a.seg_tmax = p;  p += SAILOR_SEG_MAX * R;
-    a.seg_sync = p;  p += SAILOR_SEG_MAX * R;
-    a.seg_upd = p;   p += SAILOR_SEG_MAX * R;
-    a.rate_d = p;    p += R;
-    a.c2x = p;       p += (size_t)R * R;
-    a.commx = p;     p += (size_t)Z * Z;
     a.availv = reinterpret_cast<uint32_t*>(p);
+    a.tz = a.availv + R;
+}
+
+// Run of stage i: 0 = stage 0 with the embedding, 1 = one extra block, 2 = plain, 3 = final stage.
+__device__ __forceinline__ uint32_t run_of(const TabHdr* h, uint32_t P, uint32_t i) {
+    if (i == P - 1) return 3;
+    if (i == 0 && h->has_embed) return 0;
+    return i < h->n_blocks % P ? 1 : 2;
 }
 
 // Build the tables of configuration `c`.  Called by the whole block; ends synchronised.
@@ -191,8 +216,12 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         for (uint32_t s = 0; s < k.nseg; ++s) {
             cs.need[s] = k.D * tp * (cs.seg_a[s + 1] - cs.seg_a[s]);
             cs.oom_mask[s] = 0;
+            for (int r = 0; r < N_RUNS; ++r) cs.n_run[s][r] = 0;
+            const uint32_t t_end = (s + 1 < k.nseg) ? cs.seg_a[s + 1] - 1 : cs.seg_a[s + 1];
+            for (uint32_t i = cs.seg_a[s]; i < t_end; ++i) cs.n_run[s][run_of(h, k.P, i)]++;
         }
         cs.n_items = ipow64(R, k.nseg - 1);
+        cs.magic = (uint32_t)(0x100000000ull / R) + 1u;
         uint64_t inv = 0;
         for (uint32_t d = 0; d < R; ++d)
             if (tp > h->gpn[d % T]) inv |= 1ull << d;
@@ -222,45 +251,51 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
     }
     for (uint32_t d = tid; d < R; d += PLAN_THREADS) {
         a.availv[d] = pp.avail[d];
-        a.rate_d[d] = mul_rn((double)(k.D * tp), v.price_s[d]);
+        a.tz[d] = (d % T) | ((d / T) << 8);
     }
     __syncthreads();
 
-    // phase B: t_i with the next stage on the same digit; boundary tables
+    // phase B: boundary tables and per-(segment, digit) records
     const double msg = (double)v.p2p[k.mi];
-    for (uint32_t x = tid; x < P * R; x += PLAN_THREADS) {
-        const uint32_t i = x / R, d = x % R, g = d % T, z = d / T;
-        double t = a.fb[i * T + g];
-        if (i + 1 < P) t = add_rn(t, mul_rn(2.0, boundary_time(v, g, z, tp, g, z, tp, k.D, msg)));
-        a.tself[x] = t;
-    }
     const uint64_t xbytes = 2 * cs.n_b * (uint64_t)k.D * v.p2p[k.mi];
     for (uint32_t x = tid; x < R * R; x += PLAN_THREADS) {
         const uint32_t dn = x / R, d = x % R;      // [next][this]
         a.c2x[x] = mul_rn(2.0, boundary_time(v, d % T, d / T, tp, dn % T, dn / T, tp, k.D, msg));
     }
-    for (uint32_t x = tid; x < Z * Z; x += PLAN_THREADS) {
-        const uint32_t zn = x / Z, z = x % Z;      // [next][this]
+    for (uint32_t x = tid; x < R * Z; x += PLAN_THREADS) {
+        const uint32_t dn = x / Z, z = x % Z, zn = dn / T;      // [next digit][this zone]
         a.commx[x] = (z != zn) ? mul_rn((double)xbytes, v.egress[z * Z + zn]) : 0.0;
     }
-    __syncthreads();
-    // phase C: per (segment, digit) maxima and memory masks
+    for (uint32_t x = tid; x < k.nseg * T; x += PLAN_THREADS) {
+        const uint32_t s = x / T, g = x % T;
+        a.fb_last[x] = a.fb[(cs.seg_a[s + 1] - 1) * T + g];
+    }
     for (uint32_t x = tid; x < k.nseg * R; x += PLAN_THREADS) {
         const uint32_t s = x / R, d = x % R, g = d % T, z = d / T;
         const uint32_t sa = cs.seg_a[s], se = cs.seg_a[s + 1];
-        // the last stage of a non-final segment talks to the next segment: its t is not in tself
+        // the last stage of a non-final segment talks to the next segment: its t is not in the runs
         const uint32_t t_end = (s + 1 < k.nseg) ? se - 1 : se;
+        const double c2self = mul_rn(2.0, boundary_time(v, g, z, tp, g, z, tp, k.D, msg));
+        SegRec r;
+        for (int q = 0; q < N_RUNS; ++q) r.v[q] = 0.0;
         double tm = 0.0, sy = 0.0, up = 0.0;
         bool oom = false;
         for (uint32_t i = sa; i < se; ++i) {
-            if (i < t_end) tm = dmax(tm, a.tself[i * R + d]);
+            if (i < t_end) {
+                const double fbi = a.fb[i * T + g];
+                const double t = (i + 1 < P) ? add_rn(fbi, c2self) : fbi;
+                r.v[run_of(h, P, i)] = t;
+                tm = dmax(tm, t);
+            }
             sy = dmax(sy, sync_time(v, g, z, tp, k.D, cs.params[i]));
             up = dmax(up, a.uu[i * T + g]);
             oom |= (cs.oom_stage[i] >> g) & 1u;
         }
-        a.seg_tmax[x] = tm;
-        a.seg_sync[x] = sy;
-        a.seg_upd[x] = up;
+        r.tmax = tm;
+        r.sync = sy;
+        r.upd = up;
+        r.rate = mul_rn((double)(k.D * tp), v.price_s[d]);
+        a.rec[x] = r;
         if (oom) atomicOr(reinterpret_cast<unsigned long long*>(&cs.oom_mask[s]), 1ull << d);
     }
     if (tid == 0) {
@@ -296,41 +331,49 @@ __device__ __forceinline__ void flush_counters(CfgShared& cs, Counters& cnt, uin
     }
 }
 
+// acc + v + v + ... (n times), one rounding per addition: the stage-by-stage sum of a run.
+__device__ __forceinline__ double add_n(double acc, double v, uint32_t n) {
+#pragma unroll 4
+    for (uint32_t j = 0; j < n; ++j) acc = add_rn(acc, v);
+    return acc;
+}
+
 // One item per lane: fixed prefix digits, walk the last segment's digit.
 template <int NSEG, int OBJ, bool CONSTR>
 __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared& cs, const CfgArrays& a,
-                                          uint32_t T, uint32_t Z, uint32_t R, uint64_t q, bool active,
+                                          uint32_t T, uint32_t Z, uint32_t R, uint32_t q, bool active,
                                           uint64_t item_flat, double budget, WarpTopK& top, Counters& cnt,
                                           uint32_t lane) {
     constexpr uint32_t last = NSEG - 1;
     // ---- prefix: segments 0 .. NSEG-2 --------------------------------------------------------
     uint32_t dg[NSEG > 1 ? NSEG - 1 : 1];
     {
-        uint64_t x = active ? q : 0;
+        uint32_t x = active ? q : 0;
 #pragma unroll
-        for (int s = NSEG - 2; s >= 0; --s) { dg[s] = (uint32_t)(x % R); x /= R; }
+        for (int s = NSEG - 2; s >= 0; --s) {
+            const uint32_t y = R == 1 ? x : __umulhi(x, cs.magic);     // x / R
+            dg[s] = x - y * R;
+            x = y;
+        }
     }
     double acc = 0.0, mx = 0.0, sy = 0.0, up = 0.0, rate = 0.0, cc = 0.0;
     bool p_inv = false, p_oom = false, p_over = false;
 #pragma unroll
     for (int s = 0; s < NSEG - 1; ++s) {
         const uint32_t d = dg[s];
-        const uint32_t sa = cs.seg_a[s], se = cs.seg_a[s + 1];
-        const double rd = a.rate_d[d];
-        for (uint32_t i = sa; i + 1 < se; ++i) {          // stages followed by the same digit
-            acc = add_rn(acc, a.tself[i * R + d]);
-            rate = add_rn(rate, rd);
-        }
-        mx = dmax(mx, a.seg_tmax[s * R + d]);
-        sy = dmax(sy, a.seg_sync[s * R + d]);
-        up = dmax(up, a.seg_upd[s * R + d]);
-        rate = add_rn(rate, rd);                          // the segment's last stage
-        if (s < NSEG - 2) {                               // its message goes to the next prefix digit
+        const SegRec& rc = a.rec[s * R + d];
+#pragma unroll
+        for (int r = 0; r < N_RUNS - 1; ++r) acc = add_n(acc, rc.v[r], cs.n_run[s][r]);   // run 3 is the final stage
+        mx = fmax(mx, rc.tmax);
+        sy = fmax(sy, rc.sync);
+        up = fmax(up, rc.upd);
+        rate = add_n(rate, rc.rate, cs.seg_a[s + 1] - cs.seg_a[s]);
+        if (s < NSEG - 2) {                               // the segment's last stage sends to the next prefix digit
             const uint32_t dn = dg[s + 1];
-            const double tb = add_rn(a.fb[(se - 1) * T + d % T], a.c2x[dn * R + d]);
+            const double tb = add_rn(a.fb_last[s * T + (a.tz[d] & 0xff)], a.c2x[dn * R + d]);
             acc = add_rn(acc, tb);
-            mx = dmax(mx, tb);
-            cc = add_rn(cc, a.commx[(dn / T) * Z + d / T]);
+            mx = fmax(mx, tb);
+            cc = add_rn(cc, a.commx[dn * Z + (a.tz[d] >> 8)]);
         }
         p_inv |= (cs.invalid_mask >> d) & 1;
         p_oom |= (cs.oom_mask[s] >> d) & 1;
@@ -378,49 +421,56 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     if (!CONSTR) cnt.feasible += n_ok;
 
     // ---- the candidates -----------------------------------------------------------------------
-    uint64_t walk = pp.eval_all ? warp_or64(range) : warp_or64(ok);   // warp-uniform: skip dead digits
-    const uint32_t la = cs.seg_a[last], le = cs.seg_a[last + 1];
+    const uint64_t walk = pp.eval_all ? warp_or64(range) : warp_or64(ok);   // warp-uniform: skip dead digits
+    const uint32_t n0 = cs.n_run[last][0], n1 = cs.n_run[last][1], n2 = cs.n_run[last][2], n3 = cs.n_run[last][3];
+    const uint32_t n_last = cs.seg_a[last + 1] - cs.seg_a[last];
     const double nb = (double)cs.n_b;
     double fb_b = 0.0;
     uint32_t d_prev = 0, z_prev = 0;
     if (NSEG > 1) {
         d_prev = dg[NSEG > 1 ? NSEG - 2 : 0];
-        z_prev = d_prev / T;
-        fb_b = a.fb[(la - 1) * T + d_prev % T];
+        z_prev = a.tz[d_prev] >> 8;
+        fb_b = a.fb_last[(NSEG > 1 ? NSEG - 2 : 0) * T + (a.tz[d_prev] & 0xff)];
     }
+    const SegRec* recs = a.rec + last * R;
+    const double* c2x_col = a.c2x + d_prev;
+    const double* comm_col = a.commx + z_prev;
     uint32_t feas = 0;
-    while (walk) {
-        const uint32_t d = __ffsll((long long)walk) - 1;
-        walk &= walk - 1;
-        double t_sum = acc, t_max = mx;
-        double c_comm = cc;
-        if (NSEG > 1) {                                   // last stage of the prefix sends to digit d
-            const double tb = add_rn(fb_b, a.c2x[d * R + d_prev]);
-            t_sum = add_rn(t_sum, tb);
-            t_max = dmax(t_max, tb);
-            c_comm = add_rn(c_comm, a.commx[(d / T) * Z + z_prev]);
+    for (uint32_t half = 0; half * 32 < R; ++half) {
+        const uint32_t wm = (uint32_t)(walk >> (32 * half)), om = (uint32_t)(ok >> (32 * half));
+        const uint32_t d_end = min(R - 32 * half, 32u);
+        for (uint32_t dd = 0; dd < d_end; ++dd) {
+            if (!((wm >> dd) & 1u)) continue;                 // warp-uniform
+            const uint32_t d = 32 * half + dd;
+            const SegRec& rc = recs[d];
+            double t_sum = acc, t_max = mx, c_comm = cc;
+            if (NSEG > 1) {                                   // last stage of the prefix sends to digit d
+                const double tb = add_rn(fb_b, c2x_col[d * R]);
+                t_sum = add_rn(t_sum, tb);
+                t_max = fmax(t_max, tb);
+                c_comm = add_rn(c_comm, comm_col[d * Z]);
+            }
+            t_sum = add_n(t_sum, rc.v[0], n0);
+            t_sum = add_n(t_sum, rc.v[1], n1);
+            t_sum = add_n(t_sum, rc.v[2], n2);
+            t_sum = add_n(t_sum, rc.v[3], n3);
+            const double r = add_n(rate, rc.rate, n_last);
+            t_max = fmax(t_max, rc.tmax);
+            const double t_pp = add_rn(t_sum, mul_rn(nb, t_max));
+            const double t_iter = add_rn(add_rn(t_pp, fmax(sy, rc.sync)), fmax(up, rc.upd));
+            const double cost = add_rn(mul_rn(r, t_iter), c_comm);
+            bool good = (om >> dd) & 1u;
+            if (CONSTR) {
+                if (budget > 0.0) good &= !(cost > budget);
+                if (pp.min_rate > 0.0) good &= !(1.0 / t_iter < pp.min_rate);
+                feas += good;
+            }
+            const double score = OBJ == SAILOR_OBJ_MAX_THROUGHPUT ? t_iter
+                               : OBJ == SAILOR_OBJ_MIN_COST ? cost : mul_rn(t_iter, cost);
+            if (good && cost < cnt.min_cost) cnt.min_cost = cost;
+            const bool want = good && score <= top.thr_score;
+            if (__any_sync(FULL, want)) top.offer(want, score, item_flat + d, pp.k, lane);
         }
-        double r = rate;
-        const double rd = a.rate_d[d];
-        for (uint32_t i = la; i < le; ++i) {
-            t_sum = add_rn(t_sum, a.tself[i * R + d]);
-            r = add_rn(r, rd);
-        }
-        t_max = dmax(t_max, a.seg_tmax[last * R + d]);
-        const double t_pp = add_rn(t_sum, mul_rn(nb, t_max));
-        const double t_iter = add_rn(add_rn(t_pp, dmax(sy, a.seg_sync[last * R + d])), dmax(up, a.seg_upd[last * R + d]));
-        const double cost = add_rn(mul_rn(r, t_iter), c_comm);
-        bool good = (ok >> d) & 1;
-        if (CONSTR) {
-            if (budget > 0.0) good &= !(cost > budget);
-            if (pp.min_rate > 0.0) good &= !(1.0 / t_iter < pp.min_rate);
-            feas += good;
-        }
-        const double score = OBJ == SAILOR_OBJ_MAX_THROUGHPUT ? t_iter
-                           : OBJ == SAILOR_OBJ_MIN_COST ? cost : mul_rn(t_iter, cost);
-        if (good && cost < cnt.min_cost) cnt.min_cost = cost;
-        const bool want = good && score <= top.thr_score;
-        if (__any_sync(FULL, want)) top.offer(want, score, item_flat + d, pp.k, lane);
     }
     if (CONSTR) {
         cnt.feasible += feas;
@@ -480,9 +530,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const __grid_constan
                 __syncthreads();
                 build_config(pp, v, cs, a, c);
             }
-            const uint64_t q = (uint64_t)(ch - pp.cfg_chunk_start[c]) * PLAN_THREADS + tid;
+            const uint32_t q = (ch - pp.cfg_chunk_start[c]) * PLAN_THREADS + tid;    // < R^3 + 256 <= 2^18 + 256
             const bool active = q < cs.n_items;
-            const uint64_t item_flat = pp.cfg_flat_base[c] + q * R;
+            const uint64_t item_flat = pp.cfg_flat_base[c] + (uint64_t)q * R;
             if (!cs.valid) {
                 // every candidate of the configuration is invalid; count those in range
                 if (active) {
