@@ -43,8 +43,12 @@ def mean_ops_per_candidate(w: W.Workload) -> float:
     return ops / tot
 
 
-def workload_by_name(name: str) -> W.Workload:
-    return W.CONFIGS[int(name.replace("cfg", ""))]()
+def workload_by_name(name: str, only_p=None) -> W.Workload:
+    w = W.CONFIGS[int(name.replace("cfg", ""))]()
+    if only_p:                       # a sub-space with the given stage counts only (small profiling cases)
+        w.p_values = [p for p in w.p_values if p in only_p]
+        w.name += "-P" + "_".join(str(p) for p in w.p_values)
+    return w
 
 
 class ClockSampler:
@@ -95,7 +99,7 @@ def run_reference(args) -> None:
     if int(os.environ.get("RANK", "0")) != 0:
         return
     from oracle.binding import Oracle
-    w = workload_by_name(args.workload)
+    w = workload_by_name(args.workload, args.only_p)
     o = Oracle(w)
     n = o.space_size()
     sample = min(n, args.ref_sample)
@@ -175,7 +179,7 @@ def run_ours(args) -> None:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    w = workload_by_name(args.workload)
+    w = workload_by_name(args.workload, args.only_p)
     # independent problems: every rank searches the whole space for its own availability snapshot
     avail = w.avail.copy()
     if rank:
@@ -290,6 +294,7 @@ def main() -> None:
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-sample", type=int, default=20_000_000, help="candidates the CPU baseline evaluates")
     ap.add_argument("--ref-sample", type=int, default=4_000_000, help="candidates per reference step")
+    ap.add_argument("--only-p", type=int, nargs="*", default=None, help="keep only these pipeline depths")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-aux", action="store_true")
     args = ap.parse_args()

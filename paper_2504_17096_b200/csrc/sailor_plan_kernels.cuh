@@ -338,8 +338,88 @@ __device__ __forceinline__ double add_n(double acc, double v, uint32_t n) {
     return acc;
 }
 
+// What a lane carries from its prefix into the walk over the last segment's digit.
+struct ItemState {
+    double acc, mx, sy, up, rate, cc;    // running sum / maxima / price rate / transfer cost of the prefix
+    double fb_b;                         // f+b of the prefix's last stage (its message goes to the last digit)
+    uint64_t ok, walk;                   // per last digit: feasible for this lane / worth visiting for the warp
+    const SegRec* recs;                  // records of the last segment
+    const double* c2x_col;               // c2x[.][d_prev]
+    const double* comm_col;              // commx[.][z_prev]
+};
+
+// Evaluate the candidates of one item.  OFFER == false: track the lane's best score, the class
+// counts and the cheapest cost.  OFFER == true: same arithmetic, but candidates that may enter
+// the warp's top-k list are offered to it (warp-synchronous), and nothing is counted.
+template <int NSEG, int OBJ, bool CONSTR, int N2, bool OFFER>
+__device__ __forceinline__ void walk_candidates(const PlanParams& pp, const CfgShared& cs, const ItemState& it,
+                                                uint32_t Z, uint32_t R, double budget, uint64_t item_flat,
+                                                double& best, uint32_t& feas, double& min_cost, WarpTopK& top,
+                                                uint32_t lane) {
+    constexpr uint32_t last = NSEG - 1;
+    const uint32_t n0 = cs.n_run[last][0], n1 = cs.n_run[last][1], n2 = cs.n_run[last][2], n3 = cs.n_run[last][3];
+    const double nb = (double)cs.n_b;
+    for (uint32_t half = 0; half * 32 < R; ++half) {
+        const uint32_t wm = (uint32_t)(it.walk >> (32 * half)), om = (uint32_t)(it.ok >> (32 * half));
+        const uint32_t d_end = min(R - 32 * half, 32u);
+        for (uint32_t dd = 0; dd < d_end; ++dd) {
+            if (!((wm >> dd) & 1u)) continue;                 // warp-uniform
+            const uint32_t d = 32 * half + dd;
+            const SegRec& rc = it.recs[d];
+            double t_sum = it.acc, t_max = it.mx, c_comm = it.cc;
+            if (NSEG > 1) {                                   // last stage of the prefix sends to digit d
+                const double tb = add_rn(it.fb_b, it.c2x_col[d * R]);
+                t_sum = add_rn(t_sum, tb);
+                t_max = dmax(t_max, tb);
+                c_comm = add_rn(c_comm, it.comm_col[d * Z]);
+            }
+            // the segment's stages in order: [stage 0] [stages with an extra block] [plain stages] [final stage];
+            // the price-rate sum takes one term per stage alongside
+            double r = it.rate;
+            const double rd = rc.rate;
+            if (N2 >= 0) {
+                const double v2 = rc.v[2];
+#pragma unroll
+                for (int j = 0; j < N2; ++j) { t_sum = add_rn(t_sum, v2); r = add_rn(r, rd); }
+                t_sum = add_rn(t_sum, rc.v[3]);
+                r = add_rn(r, rd);
+            } else {
+                if (n0) { t_sum = add_rn(t_sum, rc.v[0]); r = add_rn(r, rd); }
+                if (n1) {
+                    const double v1 = rc.v[1];
+                    for (uint32_t j = 0; j < n1; ++j) { t_sum = add_rn(t_sum, v1); r = add_rn(r, rd); }
+                }
+                const double v2 = rc.v[2];
+                for (uint32_t j = 0; j < n2; ++j) { t_sum = add_rn(t_sum, v2); r = add_rn(r, rd); }
+                if (n3) { t_sum = add_rn(t_sum, rc.v[3]); r = add_rn(r, rd); }
+            }
+            t_max = dmax(t_max, rc.tmax);
+            const double t_pp = add_rn(t_sum, mul_rn(nb, t_max));
+            const double t_iter = add_rn(add_rn(t_pp, dmax(it.sy, rc.sync)), dmax(it.up, rc.upd));
+            const double cost = add_rn(mul_rn(r, t_iter), c_comm);
+            bool good = (om >> dd) & 1u;
+            if (CONSTR) {
+                if (budget > 0.0) good &= !(cost > budget);
+                if (pp.min_rate > 0.0) good &= !(1.0 / t_iter < pp.min_rate);
+            }
+            const double score = OBJ == SAILOR_OBJ_MAX_THROUGHPUT ? t_iter
+                               : OBJ == SAILOR_OBJ_MIN_COST ? cost : mul_rn(t_iter, cost);
+            if (OFFER) {
+                const bool want = good && score <= top.thr_score;
+                if (__any_sync(FULL, want)) top.offer(want, score, item_flat + d, pp.k, lane);
+            } else {
+                if (CONSTR) feas += good;
+                min_cost = (good && cost < min_cost) ? cost : min_cost;
+                best = (good && score < best) ? score : best;
+            }
+        }
+    }
+}
+
 // One item per lane: fixed prefix digits, walk the last segment's digit.
-template <int NSEG, int OBJ, bool CONSTR>
+// N2 >= 0 fixes the shape of the last segment at compile time (N2 plain stages, then the final
+// stage, nothing else), which makes the candidate loop straight-line code; N2 < 0 is the general form.
+template <int NSEG, int OBJ, bool CONSTR, int N2>
 __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared& cs, const CfgArrays& a,
                                           uint32_t T, uint32_t Z, uint32_t R, uint32_t q, bool active,
                                           uint64_t item_flat, double budget, WarpTopK& top, Counters& cnt,
@@ -364,15 +444,15 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
         const SegRec& rc = a.rec[s * R + d];
 #pragma unroll
         for (int r = 0; r < N_RUNS - 1; ++r) acc = add_n(acc, rc.v[r], cs.n_run[s][r]);   // run 3 is the final stage
-        mx = fmax(mx, rc.tmax);
-        sy = fmax(sy, rc.sync);
-        up = fmax(up, rc.upd);
+        mx = dmax(mx, rc.tmax);
+        sy = dmax(sy, rc.sync);
+        up = dmax(up, rc.upd);
         rate = add_n(rate, rc.rate, cs.seg_a[s + 1] - cs.seg_a[s]);
         if (s < NSEG - 2) {                               // the segment's last stage sends to the next prefix digit
             const uint32_t dn = dg[s + 1];
             const double tb = add_rn(a.fb_last[s * T + (a.tz[d] & 0xff)], a.c2x[dn * R + d]);
             acc = add_rn(acc, tb);
-            mx = fmax(mx, tb);
+            mx = dmax(mx, tb);
             cc = add_rn(cc, a.commx[dn * Z + (a.tz[d] >> 8)]);
         }
         p_inv |= (cs.invalid_mask >> d) & 1;
@@ -421,61 +501,32 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     if (!CONSTR) cnt.feasible += n_ok;
 
     // ---- the candidates -----------------------------------------------------------------------
-    const uint64_t walk = pp.eval_all ? warp_or64(range) : warp_or64(ok);   // warp-uniform: skip dead digits
-    const uint32_t n0 = cs.n_run[last][0], n1 = cs.n_run[last][1], n2 = cs.n_run[last][2], n3 = cs.n_run[last][3];
-    const uint32_t n_last = cs.seg_a[last + 1] - cs.seg_a[last];
-    const double nb = (double)cs.n_b;
-    double fb_b = 0.0;
+    ItemState it;
+    it.acc = acc; it.mx = mx; it.sy = sy; it.up = up; it.rate = rate; it.cc = cc;
+    it.ok = ok;
+    it.walk = pp.eval_all ? warp_or64(range) : warp_or64(ok);   // warp-uniform: skip dead digits
+    it.fb_b = 0.0;
     uint32_t d_prev = 0, z_prev = 0;
     if (NSEG > 1) {
         d_prev = dg[NSEG > 1 ? NSEG - 2 : 0];
         z_prev = a.tz[d_prev] >> 8;
-        fb_b = a.fb_last[(NSEG > 1 ? NSEG - 2 : 0) * T + (a.tz[d_prev] & 0xff)];
+        it.fb_b = a.fb_last[(NSEG > 1 ? NSEG - 2 : 0) * T + (a.tz[d_prev] & 0xff)];
     }
-    const SegRec* recs = a.rec + last * R;
-    const double* c2x_col = a.c2x + d_prev;
-    const double* comm_col = a.commx + z_prev;
+    it.recs = a.rec + last * R;
+    it.c2x_col = a.c2x + d_prev;
+    it.comm_col = a.commx + z_prev;
+
+    // fast pass: no votes, no list updates; each lane keeps its item's best score
+    double best = make_inf();
     uint32_t feas = 0;
-    for (uint32_t half = 0; half * 32 < R; ++half) {
-        const uint32_t wm = (uint32_t)(walk >> (32 * half)), om = (uint32_t)(ok >> (32 * half));
-        const uint32_t d_end = min(R - 32 * half, 32u);
-        for (uint32_t dd = 0; dd < d_end; ++dd) {
-            if (!((wm >> dd) & 1u)) continue;                 // warp-uniform
-            const uint32_t d = 32 * half + dd;
-            const SegRec& rc = recs[d];
-            double t_sum = acc, t_max = mx, c_comm = cc;
-            if (NSEG > 1) {                                   // last stage of the prefix sends to digit d
-                const double tb = add_rn(fb_b, c2x_col[d * R]);
-                t_sum = add_rn(t_sum, tb);
-                t_max = fmax(t_max, tb);
-                c_comm = add_rn(c_comm, comm_col[d * Z]);
-            }
-            t_sum = add_n(t_sum, rc.v[0], n0);
-            t_sum = add_n(t_sum, rc.v[1], n1);
-            t_sum = add_n(t_sum, rc.v[2], n2);
-            t_sum = add_n(t_sum, rc.v[3], n3);
-            const double r = add_n(rate, rc.rate, n_last);
-            t_max = fmax(t_max, rc.tmax);
-            const double t_pp = add_rn(t_sum, mul_rn(nb, t_max));
-            const double t_iter = add_rn(add_rn(t_pp, fmax(sy, rc.sync)), fmax(up, rc.upd));
-            const double cost = add_rn(mul_rn(r, t_iter), c_comm);
-            bool good = (om >> dd) & 1u;
-            if (CONSTR) {
-                if (budget > 0.0) good &= !(cost > budget);
-                if (pp.min_rate > 0.0) good &= !(1.0 / t_iter < pp.min_rate);
-                feas += good;
-            }
-            const double score = OBJ == SAILOR_OBJ_MAX_THROUGHPUT ? t_iter
-                               : OBJ == SAILOR_OBJ_MIN_COST ? cost : mul_rn(t_iter, cost);
-            if (good && cost < cnt.min_cost) cnt.min_cost = cost;
-            const bool want = good && score <= top.thr_score;
-            if (__any_sync(FULL, want)) top.offer(want, score, item_flat + d, pp.k, lane);
-        }
-    }
+    walk_candidates<NSEG, OBJ, CONSTR, N2, false>(pp, cs, it, Z, R, budget, item_flat, best, feas, cnt.min_cost, top, lane);
     if (CONSTR) {
         cnt.feasible += feas;
         cnt.over_constr += n_ok - feas;
     }
+    // rare: some lane's item holds a candidate that may enter the warp's list; walk again and offer
+    if (__any_sync(FULL, best < make_inf() && best <= top.thr_score))     // best == inf: the item has no feasible candidate
+        walk_candidates<NSEG, OBJ, CONSTR, N2, true>(pp, cs, it, Z, R, budget, item_flat, best, feas, cnt.min_cost, top, lane);
 }
 
 template <int OBJ, bool CONSTR>
@@ -544,12 +595,25 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const __grid_constan
                 }
                 continue;
             }
+            // the bulk of every space has four segments: pick the straight-line loop for its common shapes
+            const int fixed = (cs.n_run[3][0] == 0 && cs.n_run[3][1] == 0 && cs.n_run[3][3] == 1 && cs.n_run[3][2] <= 3)
+                                  ? (int)cs.n_run[3][2] : -1;
+#define SAILOR_RUN(NS, NF) run_items<NS, OBJ, CONSTR, NF>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane)
             switch (cs.cfg.nseg) {
-                case 1: run_items<1, OBJ, CONSTR>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane); break;
-                case 2: run_items<2, OBJ, CONSTR>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane); break;
-                case 3: run_items<3, OBJ, CONSTR>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane); break;
-                default: run_items<4, OBJ, CONSTR>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane); break;
+                case 1: SAILOR_RUN(1, -1); break;
+                case 2: SAILOR_RUN(2, -1); break;
+                case 3: SAILOR_RUN(3, -1); break;
+                default:
+                    switch (fixed) {
+                        case 0: SAILOR_RUN(4, 0); break;
+                        case 1: SAILOR_RUN(4, 1); break;
+                        case 2: SAILOR_RUN(4, 2); break;
+                        case 3: SAILOR_RUN(4, 3); break;
+                        default: SAILOR_RUN(4, -1); break;
+                    }
+                    break;
             }
+#undef SAILOR_RUN
         }
         // per-thread counters are 32 bits wide: hand them to the block's 64-bit sums in time
         if (__any_sync(FULL, cnt.total > (1u << 30))) flush_counters(cs, cnt, lane);
