@@ -18,6 +18,9 @@ namespace sailor {
 
 constexpr int PLAN_THREADS = 256;
 constexpr int PLAN_WARPS = PLAN_THREADS / 32;
+#ifndef PLAN_MIN_BLOCKS
+#define PLAN_MIN_BLOCKS 3
+#endif
 constexpr unsigned FULL = 0xffffffffu;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;   // bound of every spin-wait in this file
 
@@ -154,7 +157,7 @@ struct CfgShared {
     uint64_t oom_mask[SAILOR_SEG_MAX];    // digit d: some stage of the segment does not fit type(d)
     uint64_t avail_last;         // digit d: need[last] <= avail[d]
     uint32_t cur_config;
-    uint32_t next_chunk;
+    uint32_t next_chunk, batch_len;
     uint32_t oom_stage[SAILOR_P_MAX];     // per stage: bit g set when the stage does not fit type g
     uint64_t params[SAILOR_P_MAX];
     unsigned long long stat[6];
@@ -530,7 +533,7 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
 }
 
 template <int OBJ, bool CONSTR>
-__global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const __grid_constant__ PlanParams pp) {
+__global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(const __grid_constant__ PlanParams pp) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ CfgShared cs;
     __shared__ Hit s_hits[PLAN_WARPS][SAILOR_K_MAX];
@@ -562,11 +565,20 @@ __global__ void __launch_bounds__(PLAN_THREADS) plan_kernel(const __grid_constan
 
     uint32_t c = 0;     // configuration of the current chunk (monotone within a batch)
     for (;;) {
-        if (tid == 0) cs.next_chunk = pp.chunk_lo + atomicAdd(&pp.ctrl->work_counter, pp.batch);
+        if (tid == 0) {
+            // guided self-scheduling: long runs of consecutive chunks first (a block then stays inside
+            // one configuration and rebuilds its tables rarely), single chunks at the end (even finish)
+            const uint32_t n_chunks = pp.chunk_hi - pp.chunk_lo;
+            const uint32_t seen = *reinterpret_cast<volatile unsigned int*>(&pp.ctrl->work_counter);
+            const uint32_t left = seen < n_chunks ? n_chunks - seen : 0u;
+            const uint32_t len = max(1u, left / (gridDim.x * 4u));
+            cs.next_chunk = pp.chunk_lo + atomicAdd(&pp.ctrl->work_counter, len);
+            cs.batch_len = len;
+        }
         __syncthreads();
         const uint32_t first = cs.next_chunk;
         if (first >= pp.chunk_hi) break;
-        const uint32_t end = min(first + pp.batch, pp.chunk_hi);
+        const uint32_t end = min(first + cs.batch_len, pp.chunk_hi);
         {   // configuration of the first chunk: binary search (uniform)
             uint32_t lo = 0, hi = pp.n_config;
             while (hi - lo > 1) {
