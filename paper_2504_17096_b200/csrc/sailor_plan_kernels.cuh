@@ -18,8 +18,11 @@ namespace sailor {
 
 constexpr int PLAN_THREADS = 256;
 constexpr int PLAN_WARPS = PLAN_THREADS / 32;
+#ifndef PLAN_DIGITS_PER_STEP
+#define PLAN_DIGITS_PER_STEP 4      // candidates evaluated side by side per thread (independent chains)
+#endif
 #ifndef PLAN_MIN_BLOCKS
-#define PLAN_MIN_BLOCKS 3
+#define PLAN_MIN_BLOCKS 2
 #endif
 constexpr unsigned FULL = 0xffffffffu;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;   // bound of every spin-wait in this file
@@ -134,6 +137,7 @@ struct WarpTopK {
 // sequence of additions as walking the stages.  The last stage of a non-final segment sends to
 // the next segment, so its time depends on two digits and is kept apart (fb_last + c2x).
 constexpr int N_RUNS = 4;
+constexpr uint32_t PLAN_PAD = PLAN_DIGITS_PER_STEP - 1;   // table entries past the last digit that a step may read
 
 struct alignas(16) SegRec {                  // one per (segment, digit); 64 bytes, read as broadcasts
     double v[N_RUNS];            // t_i of each run (f + b + 2c with the next stage on the same digit)
@@ -177,8 +181,8 @@ struct CfgArrays {               // pointers into dynamic shared memory
 __host__ __device__ inline size_t plan_smem_bytes(uint32_t static_bytes, uint32_t p_max, uint32_t T, uint32_t Z) {
     const size_t R = (size_t)T * Z;
     size_t n = static_bytes;
-    n += sizeof(SegRec) * SAILOR_SEG_MAX * R;
-    n += sizeof(double) * (R * R + R * Z + (size_t)SAILOR_SEG_MAX * T + 2 * (size_t)p_max * T);
+    n += sizeof(SegRec) * (SAILOR_SEG_MAX * R + PLAN_PAD);               // padding digits, see walk_fast
+    n += sizeof(double) * ((R + PLAN_PAD) * R + (R + PLAN_PAD) * Z + (size_t)SAILOR_SEG_MAX * T + 2 * (size_t)p_max * T);
     n += sizeof(uint32_t) * 2 * R;
     return (n + 15) & ~(size_t)15;
 }
@@ -187,9 +191,9 @@ __device__ __forceinline__ void carve(unsigned char* dyn, uint32_t static_bytes,
                                       uint32_t Z, CfgArrays& a) {
     const uint32_t R = T * Z;
     a.rec = reinterpret_cast<SegRec*>(dyn + static_bytes);           // static_bytes is a multiple of 16
-    double* p = reinterpret_cast<double*>(a.rec + (size_t)SAILOR_SEG_MAX * R);
-    a.c2x = p;       p += (size_t)R * R;
-    a.commx = p;     p += (size_t)R * Z;
+    double* p = reinterpret_cast<double*>(a.rec + (size_t)SAILOR_SEG_MAX * R + PLAN_PAD);
+    a.c2x = p;       p += (size_t)(R + PLAN_PAD) * R;
+    a.commx = p;     p += (size_t)(R + PLAN_PAD) * Z;
     a.fb_last = p;   p += (size_t)SAILOR_SEG_MAX * T;
     a.fb = p;        p += (size_t)p_max * T;
     a.uu = p;        p += (size_t)p_max * T;
@@ -351,71 +355,106 @@ struct ItemState {
     const double* comm_col;              // commx[.][z_prev]
 };
 
-// Evaluate the candidates of one item.  OFFER == false: track the lane's best score, the class
-// counts and the cheapest cost.  OFFER == true: same arithmetic, but candidates that may enter
-// the warp's top-k list are offered to it (warp-synchronous), and nothing is counted.
-template <int NSEG, int OBJ, bool CONSTR, int N2, bool OFFER>
-__device__ __forceinline__ void walk_candidates(const PlanParams& pp, const CfgShared& cs, const ItemState& it,
-                                                uint32_t Z, uint32_t R, double budget, uint64_t item_flat,
-                                                double& best, uint32_t& feas, double& min_cost, WarpTopK& top,
-                                                uint32_t lane) {
+// Time and cost of the candidate that extends item `it` with last digit d.
+template <int NSEG, int N2>
+__device__ __forceinline__ void eval_candidate(const CfgShared& cs, const ItemState& it, uint32_t Z, uint32_t R,
+                                               uint32_t d, double nb, double& t_iter, double& cost) {
     constexpr uint32_t last = NSEG - 1;
-    const uint32_t n0 = cs.n_run[last][0], n1 = cs.n_run[last][1], n2 = cs.n_run[last][2], n3 = cs.n_run[last][3];
+    const SegRec& rc = it.recs[d];
+    double t_sum = it.acc, t_max = it.mx, c_comm = it.cc;
+    if (NSEG > 1) {                                   // last stage of the prefix sends to digit d
+        const double tb = add_rn(it.fb_b, it.c2x_col[d * R]);
+        t_sum = add_rn(t_sum, tb);
+        t_max = dmax(t_max, tb);
+        c_comm = add_rn(c_comm, it.comm_col[d * Z]);
+    }
+    // the segment's stages in order: [stage 0] [stages with an extra block] [plain stages] [final stage];
+    // the price-rate sum takes one term per stage alongside
+    double r = it.rate;
+    const double rd = rc.rate;
+    if (N2 >= 0) {
+        const double v2 = rc.v[2];
+#pragma unroll
+        for (int j = 0; j < N2; ++j) { t_sum = add_rn(t_sum, v2); r = add_rn(r, rd); }
+        t_sum = add_rn(t_sum, rc.v[3]);
+        r = add_rn(r, rd);
+    } else {
+        const uint32_t n0 = cs.n_run[last][0], n1 = cs.n_run[last][1], n2 = cs.n_run[last][2], n3 = cs.n_run[last][3];
+        if (n0) { t_sum = add_rn(t_sum, rc.v[0]); r = add_rn(r, rd); }
+        if (n1) {
+            const double v1 = rc.v[1];
+            for (uint32_t j = 0; j < n1; ++j) { t_sum = add_rn(t_sum, v1); r = add_rn(r, rd); }
+        }
+        const double v2 = rc.v[2];
+        for (uint32_t j = 0; j < n2; ++j) { t_sum = add_rn(t_sum, v2); r = add_rn(r, rd); }
+        if (n3) { t_sum = add_rn(t_sum, rc.v[3]); r = add_rn(r, rd); }
+    }
+    t_max = dmax(t_max, rc.tmax);
+    const double t_pp = add_rn(t_sum, mul_rn(nb, t_max));
+    t_iter = add_rn(add_rn(t_pp, dmax(it.sy, rc.sync)), dmax(it.up, rc.upd));
+    cost = add_rn(mul_rn(r, t_iter), c_comm);
+}
+
+template <int OBJ>
+__device__ __forceinline__ double score_of(double t_iter, double cost) {
+    return OBJ == SAILOR_OBJ_MAX_THROUGHPUT ? t_iter : OBJ == SAILOR_OBJ_MIN_COST ? cost : mul_rn(t_iter, cost);
+}
+
+template <bool CONSTR>
+__device__ __forceinline__ bool within(const PlanParams& pp, double budget, double t_iter, double cost) {
+    bool good = true;
+    if (CONSTR) {
+        if (budget > 0.0) good &= !(cost > budget);
+        if (pp.min_rate > 0.0) good &= !(1.0 / t_iter < pp.min_rate);
+    }
+    return good;
+}
+
+// Fast pass over the candidates of one item, several digits per step (independent dependency
+// chains per thread): tracks the lane's best score, the feasible count and the cheapest cost.
+// No votes, no list updates.  Tables are padded, so a step may read (and mask out) digits >= R.
+template <int NSEG, int OBJ, bool CONSTR, int N2>
+__device__ __forceinline__ void walk_fast(const PlanParams& pp, const CfgShared& cs, const ItemState& it,
+                                          uint32_t Z, uint32_t R, double budget, double& best, uint32_t& feas,
+                                          double& min_cost) {
     const double nb = (double)cs.n_b;
+    constexpr uint32_t U = PLAN_DIGITS_PER_STEP;
     for (uint32_t half = 0; half * 32 < R; ++half) {
         const uint32_t wm = (uint32_t)(it.walk >> (32 * half)), om = (uint32_t)(it.ok >> (32 * half));
         const uint32_t d_end = min(R - 32 * half, 32u);
-        for (uint32_t dd = 0; dd < d_end; ++dd) {
-            if (!((wm >> dd) & 1u)) continue;                 // warp-uniform
+        for (uint32_t dd = 0; dd < d_end; dd += U) {
+            if (!((wm >> dd) & ((1u << U) - 1u))) continue;   // warp-uniform
             const uint32_t d = 32 * half + dd;
-            const SegRec& rc = it.recs[d];
-            double t_sum = it.acc, t_max = it.mx, c_comm = it.cc;
-            if (NSEG > 1) {                                   // last stage of the prefix sends to digit d
-                const double tb = add_rn(it.fb_b, it.c2x_col[d * R]);
-                t_sum = add_rn(t_sum, tb);
-                t_max = dmax(t_max, tb);
-                c_comm = add_rn(c_comm, it.comm_col[d * Z]);
-            }
-            // the segment's stages in order: [stage 0] [stages with an extra block] [plain stages] [final stage];
-            // the price-rate sum takes one term per stage alongside
-            double r = it.rate;
-            const double rd = rc.rate;
-            if (N2 >= 0) {
-                const double v2 = rc.v[2];
+            double t[U], c[U];
 #pragma unroll
-                for (int j = 0; j < N2; ++j) { t_sum = add_rn(t_sum, v2); r = add_rn(r, rd); }
-                t_sum = add_rn(t_sum, rc.v[3]);
-                r = add_rn(r, rd);
-            } else {
-                if (n0) { t_sum = add_rn(t_sum, rc.v[0]); r = add_rn(r, rd); }
-                if (n1) {
-                    const double v1 = rc.v[1];
-                    for (uint32_t j = 0; j < n1; ++j) { t_sum = add_rn(t_sum, v1); r = add_rn(r, rd); }
-                }
-                const double v2 = rc.v[2];
-                for (uint32_t j = 0; j < n2; ++j) { t_sum = add_rn(t_sum, v2); r = add_rn(r, rd); }
-                if (n3) { t_sum = add_rn(t_sum, rc.v[3]); r = add_rn(r, rd); }
-            }
-            t_max = dmax(t_max, rc.tmax);
-            const double t_pp = add_rn(t_sum, mul_rn(nb, t_max));
-            const double t_iter = add_rn(add_rn(t_pp, dmax(it.sy, rc.sync)), dmax(it.up, rc.upd));
-            const double cost = add_rn(mul_rn(r, t_iter), c_comm);
-            bool good = (om >> dd) & 1u;
-            if (CONSTR) {
-                if (budget > 0.0) good &= !(cost > budget);
-                if (pp.min_rate > 0.0) good &= !(1.0 / t_iter < pp.min_rate);
-            }
-            const double score = OBJ == SAILOR_OBJ_MAX_THROUGHPUT ? t_iter
-                               : OBJ == SAILOR_OBJ_MIN_COST ? cost : mul_rn(t_iter, cost);
-            if (OFFER) {
-                const bool want = good && score <= top.thr_score;
-                if (__any_sync(FULL, want)) top.offer(want, score, item_flat + d, pp.k, lane);
-            } else {
-                if (CONSTR) feas += good;
-                min_cost = (good && cost < min_cost) ? cost : min_cost;
-                best = (good && score < best) ? score : best;
+            for (uint32_t u = 0; u < U; ++u) eval_candidate<NSEG, N2>(cs, it, Z, R, d + u, nb, t[u], c[u]);
+#pragma unroll
+            for (uint32_t u = 0; u < U; ++u) {
+                const bool g = ((om >> (dd + u)) & 1u) && within<CONSTR>(pp, budget, t[u], c[u]);
+                const double sc = score_of<OBJ>(t[u], c[u]);
+                if (CONSTR) feas += (uint32_t)g;
+                min_cost = (g && c[u] < min_cost) ? c[u] : min_cost;
+                best = (g && sc < best) ? sc : best;
             }
         }
+    }
+}
+
+// Rare second pass over an item: the same arithmetic, one digit at a time, and every candidate that
+// may enter the warp's top-k list is offered to it (warp-synchronous).  Nothing is counted.
+template <int NSEG, int OBJ, bool CONSTR, int N2>
+__device__ __forceinline__ void walk_offer(const PlanParams& pp, const CfgShared& cs, const ItemState& it,
+                                           uint32_t Z, uint32_t R, double budget, uint64_t item_flat,
+                                           WarpTopK& top, uint32_t lane) {
+    const double nb = (double)cs.n_b;
+    for (uint32_t d = 0; d < R; ++d) {
+        if (!((it.walk >> d) & 1ull)) continue;               // warp-uniform
+        double t, c;
+        eval_candidate<NSEG, N2>(cs, it, Z, R, d, nb, t, c);
+        const bool good = ((it.ok >> d) & 1ull) && within<CONSTR>(pp, budget, t, c);
+        const double score = score_of<OBJ>(t, c);
+        const bool want = good && score <= top.thr_score;
+        if (__any_sync(FULL, want)) top.offer(want, score, item_flat + d, pp.k, lane);
     }
 }
 
@@ -522,14 +561,14 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     // fast pass: no votes, no list updates; each lane keeps its item's best score
     double best = make_inf();
     uint32_t feas = 0;
-    walk_candidates<NSEG, OBJ, CONSTR, N2, false>(pp, cs, it, Z, R, budget, item_flat, best, feas, cnt.min_cost, top, lane);
+    walk_fast<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, best, feas, cnt.min_cost);
     if (CONSTR) {
         cnt.feasible += feas;
         cnt.over_constr += n_ok - feas;
     }
     // rare: some lane's item holds a candidate that may enter the warp's list; walk again and offer
     if (__any_sync(FULL, best < make_inf() && best <= top.thr_score))     // best == inf: the item has no feasible candidate
-        walk_candidates<NSEG, OBJ, CONSTR, N2, true>(pp, cs, it, Z, R, budget, item_flat, best, feas, cnt.min_cost, top, lane);
+        walk_offer<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, item_flat, top, lane);
 }
 
 template <int OBJ, bool CONSTR>
@@ -557,6 +596,11 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
 
     if (tid == 0) cs.cur_config = 0xffffffffu;
     if (tid < 6) cs.stat[tid] = 0;
+    // the padding digit of the tables is read (and masked out) by the two-digit steps: keep it finite
+    for (uint32_t x = tid; x < PLAN_PAD * sizeof(SegRec) / 8; x += PLAN_THREADS)
+        reinterpret_cast<double*>(a.rec + (size_t)SAILOR_SEG_MAX * R)[x] = 0.0;
+    for (uint32_t x = tid; x < PLAN_PAD * R; x += PLAN_THREADS) a.c2x[(size_t)R * R + x] = 0.0;
+    for (uint32_t x = tid; x < PLAN_PAD * Z; x += PLAN_THREADS) a.commx[(size_t)R * Z + x] = 0.0;
     WarpTopK top;
     top.init();
     Counters cnt = {0, 0, 0, 0, 0, 0, make_inf()};
