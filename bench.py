@@ -31,6 +31,8 @@ K_TOP = 32
 # divisions, maxima, compares, table reads of the stage-by-stage evaluation)
 OPS_PLAN, OPS_STAGE = 40, 35
 SM_COUNT, ISSUE_PER_SM, LANES = 148, 4, 32
+# ncu counters per plan_kernel launch (smsp__inst_executed.sum; dram__bytes_read.sum + dram__bytes_write.sum)
+NCU_PER_LAUNCH = {"cfg5-stress-96layer": {"warp_inst": 11847158504, "dram_bytes": 2910000}}
 
 
 def mean_ops_per_candidate(w: W.Workload) -> float:
@@ -62,7 +64,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             pass
@@ -249,8 +251,18 @@ def run_ours(args) -> None:
         sm_max = float(peaks.get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0)
         peak = SM_COUNT * ISSUE_PER_SM * LANES * sm_max * 1e6 / 1e12
         achieved = ops * n / k_s / 1e12
+        # counters of one plan_kernel launch on this workload, from the ncu capture summarised in
+        # profiles/plan_kernel_cfg5.md (valid for the kernel as committed with that file)
+        captured = NCU_PER_LAUNCH.get(w.name)
+        issued = None
+        if captured:
+            rate = captured["warp_inst"] / k_s
+            issued = {"warp_inst_per_launch": captured["warp_inst"], "warp_inst_per_s": rate,
+                      "frac_of_issue_peak": rate / (SM_COUNT * ISSUE_PER_SM * sm_max * 1e6),
+                      "lane_inst_per_candidate": captured["warp_inst"] * LANES / n}
         roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tlane-op/s",
-                    "frac": achieved / peak, "traffic": None,
+                    "frac": achieved / peak, "traffic": captured["dram_bytes"] if captured else None,
+                    "issued": issued,
                     "note": "algorithmic lane-ops (40 + 35 P per candidate) / kernel time; peak = 148 SMs x 4 issue "
                             "slots x 32 lanes x max SM clock; prefix reuse executes fewer instructions than the "
                             "algorithmic count, see profiles/ for issued-instruction utilisation",
@@ -267,6 +279,17 @@ def run_ours(args) -> None:
             cpu = {"value": counts["n_total"] / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
                    "sample": f"every {stride}-th flat index of {w.name}: {counts['n_total']} candidates in {dt:.1f} s"}
         aux = aux_measurements(B, torch, local) if (world == 1 and not args.no_aux) else None
+        if aux is not None:
+            # the same workload the way a planner would call it: memory/availability pruning on
+            ob = B.make_objective(w)
+            ts = []
+            for _ in range(5):
+                t0 = time.perf_counter()
+                B.sailor_set_availability(ctx, avail)
+                _, stp = B.sailor_plan(ctx, space, ob, K_TOP)
+                ts.append(time.perf_counter() - t0)
+            aux[args.workload + "_default_mode"] = {"candidates": int(stp.n_total), "search_s": statistics.median(ts),
+                                                    "kernel_ms": stp.kernel_ms, "feasible": int(stp.n_feasible)}
         line = {"metric": METRIC, "value": total / dev_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": 1e3 * dev_s / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",

@@ -15,6 +15,7 @@ using namespace sailor;
 namespace {
 
 constexpr int SIM_THREADS = 256;
+constexpr int PLAN_SMEM_CEILING = 200 * 1024;    // dynamic shared memory any search may ask for
 
 // ---- kernels of the explicit-batch path -----------------------------------------------------
 
@@ -261,7 +262,7 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
     }
     cs[n_config] = (uint32_t)chunks;
     const size_t smem = plan_smem_bytes(ctx->hdr.static_bytes, p_max, ctx->hdr.T, ctx->hdr.Z);
-    if (smem > 200 * 1024) return SAILOR_E_RANGE;
+    if (smem > (size_t)PLAN_SMEM_CEILING) return SAILOR_E_RANGE;
 
     sc.valid = false;
     cudaFree(sc.d_chunk_start);
@@ -309,6 +310,19 @@ PlanKernel pick_kernel(uint32_t obj, bool constr) {
     }
 }
 
+// The dynamic shared-memory opt-in belongs to the kernel (per device), not to a context: raise it
+// once per (device, variant) to the ceiling every space is checked against, so that contexts
+// with different table sizes cannot lower it under one another.
+bool g_optin_done[64][6] = {};
+
+int smem_optin(sailor_ctx* ctx, PlanKernel kern, uint32_t variant) {
+    const bool tracked = ctx->device >= 0 && ctx->device < 64;
+    if (tracked && g_optin_done[ctx->device][variant]) return SAILOR_OK;
+    CU(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PLAN_SMEM_CEILING));
+    if (tracked) g_optin_done[ctx->device][variant] = true;
+    return SAILOR_OK;
+}
+
 // Enqueue one search pass (clear, search, merge) on the context's stream.
 int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_ctrl, double min_rate,
                  uint32_t flags, uint64_t lo, uint64_t hi, uint32_t k, double next_budget_factor,
@@ -344,8 +358,9 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
         const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
         PlanKernel kern = pick_kernel(obj, constr);
         uint32_t& resident = ctx->grid_of[obj * 2 + (constr ? 1 : 0)];
-        if (resident == 0) {       // once per (space, kernel variant): opt in to the shared memory, size the grid
-            CU(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sc.smem));
+        if (resident == 0) {       // once per (space, kernel variant): size the grid
+            int rc_opt = smem_optin(ctx, kern, obj * 2 + (constr ? 1 : 0));
+            if (rc_opt) return rc_opt;
             int per_sm = 0;
             CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, sc.smem));
             if (per_sm < 1) return SAILOR_E_RANGE;
@@ -764,9 +779,10 @@ int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& d
     const uint32_t n_chunks = chunk_hi - chunk_lo;
     const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
     PlanKernel kern = pick_kernel(obj, constr);
-    // the opt-in is per kernel, not per call site: ask for the library-wide ceiling so that it also
-    // covers whatever another context's search set it to
-    CU(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    {
+        const int rc_opt = smem_optin(ctx, kern, obj * 2 + (constr ? 1 : 0));
+        if (rc_opt) return rc_opt;
+    }
     int per_sm = 0;
     CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, smem));
     if (per_sm < 1) return SAILOR_E_RANGE;

@@ -355,44 +355,53 @@ struct ItemState {
     const double* comm_col;              // commx[.][z_prev]
 };
 
-// Time and cost of the candidate that extends item `it` with last digit d.
-template <int NSEG, int N2>
-__device__ __forceinline__ void eval_candidate(const CfgShared& cs, const ItemState& it, uint32_t Z, uint32_t R,
-                                               uint32_t d, double nb, double& t_iter, double& cost) {
+// Time and cost of the W candidates that extend item `it` with last digits d .. d+W-1, evaluated
+// side by side (W independent dependency chains; the stage loops run once for all of them).
+template <int NSEG, int N2, int W>
+__device__ __forceinline__ void eval_candidates(const CfgShared& cs, const ItemState& it, uint32_t Z, uint32_t R,
+                                                uint32_t d, double nb, double (&t_iter)[W], double (&cost)[W]) {
     constexpr uint32_t last = NSEG - 1;
-    const SegRec& rc = it.recs[d];
-    double t_sum = it.acc, t_max = it.mx, c_comm = it.cc;
-    if (NSEG > 1) {                                   // last stage of the prefix sends to digit d
-        const double tb = add_rn(it.fb_b, it.c2x_col[d * R]);
-        t_sum = add_rn(t_sum, tb);
-        t_max = dmax(t_max, tb);
-        c_comm = add_rn(c_comm, it.comm_col[d * Z]);
+    const SegRec* rc = it.recs + d;
+    double t_sum[W], t_max[W], c_comm[W], r[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+        t_sum[w] = it.acc; t_max[w] = it.mx; c_comm[w] = it.cc; r[w] = it.rate;
+        if (NSEG > 1) {                                   // last stage of the prefix sends to digit d + w
+            const double tb = add_rn(it.fb_b, it.c2x_col[(d + w) * R]);
+            t_sum[w] = add_rn(t_sum[w], tb);
+            t_max[w] = dmax(t_max[w], tb);
+            c_comm[w] = add_rn(c_comm[w], it.comm_col[(d + w) * Z]);
+        }
     }
     // the segment's stages in order: [stage 0] [stages with an extra block] [plain stages] [final stage];
     // the price-rate sum takes one term per stage alongside
-    double r = it.rate;
-    const double rd = rc.rate;
+#define SAILOR_STAGE(RUN)                                                          \
+    _Pragma("unroll") for (int w = 0; w < W; ++w) {                                \
+        t_sum[w] = add_rn(t_sum[w], rc[w].v[RUN]);                                 \
+        r[w] = add_rn(r[w], rc[w].rate);                                           \
+    }
     if (N2 >= 0) {
-        const double v2 = rc.v[2];
 #pragma unroll
-        for (int j = 0; j < N2; ++j) { t_sum = add_rn(t_sum, v2); r = add_rn(r, rd); }
-        t_sum = add_rn(t_sum, rc.v[3]);
-        r = add_rn(r, rd);
+        for (int j = 0; j < N2; ++j) { SAILOR_STAGE(2) }
+        SAILOR_STAGE(3)
     } else {
         const uint32_t n0 = cs.n_run[last][0], n1 = cs.n_run[last][1], n2 = cs.n_run[last][2], n3 = cs.n_run[last][3];
-        if (n0) { t_sum = add_rn(t_sum, rc.v[0]); r = add_rn(r, rd); }
-        if (n1) {
-            const double v1 = rc.v[1];
-            for (uint32_t j = 0; j < n1; ++j) { t_sum = add_rn(t_sum, v1); r = add_rn(r, rd); }
-        }
-        const double v2 = rc.v[2];
-        for (uint32_t j = 0; j < n2; ++j) { t_sum = add_rn(t_sum, v2); r = add_rn(r, rd); }
-        if (n3) { t_sum = add_rn(t_sum, rc.v[3]); r = add_rn(r, rd); }
+        if (n0) { SAILOR_STAGE(0) }
+        for (uint32_t j = 0; j < n1; ++j) { SAILOR_STAGE(1) }
+        uint32_t j = n2;
+        for (; j >= 4; j -= 4) { SAILOR_STAGE(2) SAILOR_STAGE(2) SAILOR_STAGE(2) SAILOR_STAGE(2) }
+        if (j & 2) { SAILOR_STAGE(2) SAILOR_STAGE(2) }
+        if (j & 1) { SAILOR_STAGE(2) }
+        if (n3) { SAILOR_STAGE(3) }
     }
-    t_max = dmax(t_max, rc.tmax);
-    const double t_pp = add_rn(t_sum, mul_rn(nb, t_max));
-    t_iter = add_rn(add_rn(t_pp, dmax(it.sy, rc.sync)), dmax(it.up, rc.upd));
-    cost = add_rn(mul_rn(r, t_iter), c_comm);
+#undef SAILOR_STAGE
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+        t_max[w] = dmax(t_max[w], rc[w].tmax);
+        const double t_pp = add_rn(t_sum[w], mul_rn(nb, t_max[w]));
+        t_iter[w] = add_rn(add_rn(t_pp, dmax(it.sy, rc[w].sync)), dmax(it.up, rc[w].upd));
+        cost[w] = add_rn(mul_rn(r[w], t_iter[w]), c_comm[w]);
+    }
 }
 
 template <int OBJ>
@@ -426,8 +435,7 @@ __device__ __forceinline__ void walk_fast(const PlanParams& pp, const CfgShared&
             if (!((wm >> dd) & ((1u << U) - 1u))) continue;   // warp-uniform
             const uint32_t d = 32 * half + dd;
             double t[U], c[U];
-#pragma unroll
-            for (uint32_t u = 0; u < U; ++u) eval_candidate<NSEG, N2>(cs, it, Z, R, d + u, nb, t[u], c[u]);
+            eval_candidates<NSEG, N2, (int)U>(cs, it, Z, R, d, nb, t, c);
 #pragma unroll
             for (uint32_t u = 0; u < U; ++u) {
                 const bool g = ((om >> (dd + u)) & 1u) && within<CONSTR>(pp, budget, t[u], c[u]);
@@ -449,8 +457,9 @@ __device__ __forceinline__ void walk_offer(const PlanParams& pp, const CfgShared
     const double nb = (double)cs.n_b;
     for (uint32_t d = 0; d < R; ++d) {
         if (!((it.walk >> d) & 1ull)) continue;               // warp-uniform
-        double t, c;
-        eval_candidate<NSEG, N2>(cs, it, Z, R, d, nb, t, c);
+        double t1[1], c1[1];
+        eval_candidates<NSEG, N2, 1>(cs, it, Z, R, d, nb, t1, c1);
+        const double t = t1[0], c = c1[0];
         const bool good = ((it.ok >> d) & 1ull) && within<CONSTR>(pp, budget, t, c);
         const double score = score_of<OBJ>(t, c);
         const bool want = good && score <= top.thr_score;

@@ -270,6 +270,21 @@ def test_plan_range_split_merges_to_full(make_ctx):
     assert sorted(merged)[:16] == [(r.score, r.flat) for r in full]
 
 
+def test_plan_contexts_with_different_table_sizes_alternate(make_ctx):
+    """Two live contexts whose searches need different amounts of shared memory, used in turn."""
+    big, small = W.config3(), W.tiny(seed=9, n_types=1, n_zones=1)
+    cb, cs = make_ctx(big), make_ctx(small)
+    ob = Oracle(small)
+    hits, counts = ob.search(small.objective, 4)
+    lo, hi = 1000, 200_000
+    want, wc = Oracle(big).search(big.objective, 4, lo=lo, hi=hi)
+    for _ in range(2):
+        res, st = B.sailor_plan_range(cb.ctx, cb.space, B.make_objective(big), lo, hi, 4)
+        assert_plan_equal(res, st, want, wc, Oracle(big), "big")
+        res, st = B.sailor_plan(cs.ctx, cs.space, B.make_objective(small), 4)
+        assert_plan_equal(res, st, hits, counts, ob, "small")
+
+
 def test_plan_config1_full(make_ctx):
     w = W.config1()
     cx = make_ctx(w)
