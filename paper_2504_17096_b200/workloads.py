@@ -323,17 +323,21 @@ def config5() -> Workload:
 
 
 def tiny(seed: int = 7, *, n_types: int = 2, n_zones: int = 2, L: int = 4, alpha: float = 2e-5,
-         rc_values=(0, 1), objective: int = OBJ_MAX_THROUGHPUT, seg_max: int = 4) -> Workload:
-    """A cluster small enough to enumerate by brute force; alpha > 0, scarce GPUs, both rc values."""
-    mem = [24, 12, 8][:n_types]
-    base = [5.0e-4, 9.0e-4, 1.7e-3][:n_types]
-    price = [3.0, 1.9, 1.1][:n_types]
+         rc_values=(0, 1), objective: int = OBJ_MAX_THROUGHPUT, seg_max: int = 4, p_values=None,
+         d_values=(1, 2, 3, 4, 8), tp_values=(1, 2, 4), mbs_values=(1, 2, 4), gbs: int = 32) -> Workload:
+    """A cluster small enough to enumerate by brute force; alpha > 0, scarce GPUs, both rc values.
+    Up to 8 GPU types and 8 zones (the table limits)."""
+    mem = [24, 12, 8, 20, 16, 10, 32, 6][:n_types]
+    base = [5.0e-4, 9.0e-4, 1.7e-3, 6.0e-4, 7.5e-4, 1.2e-3, 4.0e-4, 2.2e-3][:n_types]
+    price = [3.0, 1.9, 1.1, 2.6, 2.2, 1.5, 3.8, 0.9][:n_types]
+    if p_values is None:
+        p_values = [p for p in (1, 2, 3, 4) if p <= L]
     return make_workload(
-        f"tiny-{seed}", seed=seed, L=L, h=512, a=8, s=512, V=8192, gbs=32,
+        f"tiny-{seed}", seed=seed, L=L, h=512, a=8, s=512, V=8192, gbs=gbs,
         type_mem_gib=mem, type_base=base, type_price=price, n_zones=n_zones, gpus_per_node=4,
         intra_gbs=100.0, inter_gbs=10.0, zone_bw_fn=lambda r: 0.5 + 2.0 * r.uniform(),
-        avail_fn=lambda r, z, g: r.randint(2, 12), tp_values=[1, 2, 4], mbs_values=[1, 2, 4],
-        p_values=[p for p in (1, 2, 3, 4) if p <= L], d_values=[1, 2, 3, 4, 8],
+        avail_fn=lambda r, z, g: r.randint(2, 12), tp_values=list(tp_values), mbs_values=list(mbs_values),
+        p_values=list(p_values), d_values=list(d_values),
         rc_values=list(rc_values), objective=objective, seg_max=seg_max, alpha=alpha,
         egress_usd_per_byte=2e-11)
 

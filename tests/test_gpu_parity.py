@@ -205,6 +205,42 @@ def test_plan_tiny_spaces_match_exhaustive_oracle(seed, T, Z, seg_max, objective
             assert_plan_equal(res, st, hits, counts, o, f"k={k} flags={flags}")
 
 
+def test_plan_table_limits_64_digits(make_ctx):
+    """8 types x 8 zones: 64 digits, the widest mask; two and three segments."""
+    for seg_max, p_values, d_values in ((2, [1, 2, 4], (1, 2, 4)), (3, [3, 4], (1, 2))):
+        w = W.tiny(seed=20 + seg_max, n_types=8, n_zones=8, seg_max=seg_max, p_values=p_values, d_values=d_values,
+                   tp_values=(1, 2), mbs_values=(1, 4), objective=W.OBJ_MAX_THROUGHPUT_PER_USD)
+        cx = make_ctx(w)
+        o = Oracle(w)
+        hits, counts = o.search(w.objective, 32)
+        assert counts["n_feasible"] > 32
+        for flags in (0, B.FLAG_EVAL_ALL):
+            res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=flags), 32)
+            assert_plan_equal(res, st, hits, counts, o, f"seg_max={seg_max} flags={flags}")
+        n = o.space_size()
+        a, b = n // 3 + 5, 2 * n // 3 + 17                       # a range that cuts items in the middle
+        hits, counts = o.search(w.objective, 7, lo=a, hi=b)
+        res, st = B.sailor_plan_range(cx.ctx, cx.space, B.make_objective(w), a, b, 7)
+        assert_plan_equal(res, st, hits, counts, o, "range")
+
+
+def test_plan_deep_pipelines_up_to_96_stages(make_ctx):
+    """The stage limit (96), long runs inside a segment, pipeline depths that do not divide the layer count."""
+    w = W.tiny(seed=31, n_types=2, n_zones=2, L=96, p_values=[96, 64, 48, 36, 7], d_values=(1, 2), tp_values=(1, 2),
+               mbs_values=(1, 2), gbs=64)
+    w.capacity[...] = w.capacity * 8                       # room for 96 layers' worth of state
+    w.avail[...] = 400
+    cx = make_ctx(w)
+    o = Oracle(w)
+    for objective in (W.OBJ_MAX_THROUGHPUT, W.OBJ_MIN_COST):
+        hits, counts = o.search(objective, 16)
+        assert counts["n_feasible"] > 16
+        res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, kind=objective, flags=B.FLAG_EVAL_ALL), 16)
+        assert_plan_equal(res, st, hits, counts, o, f"objective {objective}")
+    recs = W.random_plans(w, 3000, seed=3, hetero_tp=True)
+    assert_sim_equal(B.sailor_simulate(cx.ctx, B.pack_records(recs)), o.simulate_records(recs), "deep")
+
+
 def test_plan_constraints_and_empty_results(make_ctx):
     w = W.tiny(seed=8, n_types=2, n_zones=2)
     cx = make_ctx(w)
