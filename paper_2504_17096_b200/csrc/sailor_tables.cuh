@@ -105,7 +105,20 @@ __device__ __forceinline__ StageTimes stage_times(const TabView& v, uint32_t g, 
     return s;
 }
 
-__host__ __device__ __forceinline__ uint64_t ceil_div64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
+// ceil(a / b) for b >= 1; tensor-parallel degrees are powers of two in practice, which avoids the
+// 64-bit division routine.
+__host__ __device__ __forceinline__ uint64_t ceil_div64(uint64_t a, uint32_t b) {
+    if ((b & (b - 1u)) == 0u) {
+#ifdef __CUDA_ARCH__
+        return (a + b - 1u) >> (31 - __clz((int)b));
+#else
+        uint32_t sh = 0;
+        while ((1u << sh) < b) ++sh;
+        return (a + b - 1u) >> sh;
+#endif
+    }
+    return (a + b - 1u) / b;
+}
 
 // Parameters of stage i and its per-worker peak memory without the reserved bytes
 // (Sec. 4.3: M_peak = M_model + M_activation; stage i keeps min(P - i, N_b) microbatches).
@@ -225,28 +238,50 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
         const sailor_run a = r.run[q];
         const uint32_t g = a.type, z = a.zone, tpi = a.tp_idx, tp = h->tp_values[tpi];
         const double gpu_rate = mul_rn((double)(D * tp), v.price_s[z * h->T + g]);
+        const uint64_t cap = h->capacity[g], resv = h->reserved[g];
+        // a run's stages differ only by layer composition (embedding / extra block / plain / head):
+        // the composition-dependent values are formed when the composition changes, not per stage
+        uint32_t cur_nb = 0xffffffffu;
+        bool cur_e = false, cur_hd = false;
+        double fb = 0.0, upd = 0.0, sync = 0.0, t_self = 0.0;
+        uint64_t m_fixed = 0, m_keep = 0;
+        const double c2_self = mul_rn(2.0, boundary_time(v, g, z, tp, g, z, tp, D, msg));
         for (uint32_t j = 0; j < a.n_stages; ++j, ++i) {
             const uint32_t nb = base + (i < extra ? 1u : 0u);
             const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
+            if (nb != cur_nb || e != cur_e || hd != cur_hd) {
+                cur_nb = nb; cur_e = e; cur_hd = hd;
+                const StageTimes st = stage_times(v, g, tpi, mi, nb, e, hd);
+                const double b = rc ? add_rn(st.b, st.f) : st.b;
+                fb = add_rn(st.f, b);
+                upd = st.u;
+                const StageMem one = stage_memory(v, tpi, mi, rc, nb, e, hd, 1);     // model + 1 * kept + work
+                const StageMem zero = stage_memory(v, tpi, mi, rc, nb, e, hd, 0);    // model + work
+                m_keep = one.mem - zero.mem;
+                m_fixed = zero.mem + resv;
+                sync = sync_time(v, g, z, tp, D, one.params);
+                t_self = add_rn(fb, c2_self);
+            }
             const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
-            const StageMem sm = stage_memory(v, tpi, mi, rc, nb, e, hd, inflight);
-            const uint64_t m = sm.mem + h->reserved[g];
-            if (m > h->capacity[g]) status |= SAILOR_ST_OOM;
+            const uint64_t m = m_fixed + inflight * m_keep;
+            if (m > cap) status |= SAILOR_ST_OOM;
             peak = m > peak ? m : peak;
 
-            const StageTimes st = stage_times(v, g, tpi, mi, nb, e, hd);
-            const double b = rc ? add_rn(st.b, st.f) : st.b;
-            double c = 0.0;
+            double t = fb;                                   // the final stage sends nothing: fb + 2*0
             if (i + 1 < P) {
-                const sailor_run nx = (j + 1 < a.n_stages) ? a : r.run[q + 1];
-                c = boundary_time(v, g, z, tp, nx.type, nx.zone, h->tp_values[nx.tp_idx], D, msg);
-                if (nx.zone != z) c_comm = add_rn(c_comm, mul_rn((double)xbytes, v.egress[z * h->Z + nx.zone]));
+                if (j + 1 < a.n_stages) {
+                    t = t_self;
+                } else {
+                    const sailor_run nx = r.run[q + 1];
+                    const double c = boundary_time(v, g, z, tp, nx.type, nx.zone, h->tp_values[nx.tp_idx], D, msg);
+                    if (nx.zone != z) c_comm = add_rn(c_comm, mul_rn((double)xbytes, v.egress[z * h->Z + nx.zone]));
+                    t = add_rn(fb, mul_rn(2.0, c));
+                }
             }
-            const double t = add_rn(add_rn(st.f, b), mul_rn(2.0, c));
             sum_t = add_rn(sum_t, t);
             max_t = dmax(max_t, t);
-            max_u = dmax(max_u, st.u);
-            max_sync = dmax(max_sync, sync_time(v, g, z, tp, D, sm.params));
+            max_u = dmax(max_u, upd);
+            max_sync = dmax(max_sync, sync);
             rate = add_rn(rate, gpu_rate);
         }
     }
