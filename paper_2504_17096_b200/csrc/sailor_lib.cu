@@ -387,7 +387,7 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
     mp.k = k;
     mp.obj = obj;
     mp.budget_factor = next_budget_factor;
-    merge_kernel<<<1, MERGE_THREADS, 0, ctx->stream>>>(mp);
+    merge_kernel<<<1, MERGE_THREADS, ctx->hdr.static_bytes, ctx->stream>>>(mp);
     CU(ctx, cudaGetLastError());
     ++*n_launches;
     return SAILOR_OK;
@@ -545,8 +545,9 @@ int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_c
         CUF(cudaGetLastError());
     }
     CUF(cudaStreamSynchronize(ctx->stream));           // `blob` is pageable host memory
-    if (h.static_bytes > 24 * 1024)
-        CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)h.static_bytes));
+    // both kernels stage the static tables in dynamic shared memory; the create-time limit is 96 KB
+    CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
+    CUF(cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
 #undef CUF
     *out = ctx;
     return SAILOR_OK;
@@ -807,7 +808,7 @@ int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& d
     mp.k = k;
     mp.obj = obj;
     mp.budget_factor = next_budget_factor;
-    merge_kernel<<<1, MERGE_THREADS, 0, ctx->stream>>>(mp);
+    merge_kernel<<<1, MERGE_THREADS, ctx->hdr.static_bytes, ctx->stream>>>(mp);
     CU(ctx, cudaGetLastError());
     ++*n_launches;
     return SAILOR_OK;

@@ -106,8 +106,9 @@ struct WarpTopK {
         flat = thr_flat = ~0ull;
     }
     // Insert one candidate known to every lane.  (score, flat) pairs are unique.
-    __device__ __forceinline__ void insert(double s, uint64_t f, uint32_t k, uint32_t lane) {
-        if (!(s < thr_score || (s == thr_score && f < thr_flat))) return;   // warp-uniform
+    // Returns false when the candidate is not better than the current k-th (warp-uniform).
+    __device__ __forceinline__ bool insert(double s, uint64_t f, uint32_t k, uint32_t lane) {
+        if (!(s < thr_score || (s == thr_score && f < thr_flat))) return false;   // warp-uniform
         const bool before = (score < s) || (score == s && flat < f);
         const uint32_t pos = __popc(__ballot_sync(FULL, before));           // sorted: a prefix of lanes
         const double ps = __shfl_up_sync(FULL, score, 1);
@@ -116,6 +117,7 @@ struct WarpTopK {
         else if (lane == pos) { score = s; flat = f; }
         thr_score = __shfl_sync(FULL, score, k - 1);
         thr_flat = __shfl_sync(FULL, flat, k - 1);
+        return true;
     }
     // Offer per-lane candidates: `want` marks lanes whose candidate may qualify.
     __device__ __forceinline__ void offer(bool want, double s, uint64_t f, uint32_t k, uint32_t lane) {
@@ -705,7 +707,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             for (uint32_t j = 0; j < pp.k; ++j) {
                 const Hit hj = s_hits[w][j];
                 if (hj.flat == ~0ull) break;             // lists are sorted; the rest is empty
-                top.insert(hj.score, hj.flat, pp.k, lane);
+                if (!top.insert(hj.score, hj.flat, pp.k, lane)) break;   // ... and the rest is no better
             }
         const uint32_t n = __popc(__ballot_sync(FULL, top.flat != ~0ull && lane < pp.k));
         if (lane < pp.k) {
@@ -729,54 +731,77 @@ struct MergeParams {
     double budget_factor;              // > 0: write ctrl->budget = factor * best cost for the next pass
 };
 
-constexpr int MERGE_THREADS = 256;
+constexpr int MERGE_THREADS = 512;
 
 __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const __grid_constant__ MergeParams mp) {
+    extern __shared__ __align__(16) unsigned char dyn[];      // the static tables
     __shared__ Hit s_hits[MERGE_THREADS / 32][SAILOR_K_MAX];
+    __shared__ uint64_t mbar;
+    __shared__ uint32_t s_n;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = MERGE_THREADS / 32;
+    const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(mp.blob)->static_bytes;
+    if (!bulk_load(dyn, mp.blob, static_bytes, &mbar)) {
+        if (tid == 0) atomicExch(&mp.ctrl->error, 1u);
+        for (uint32_t x = tid; x < static_bytes / 16; x += MERGE_THREADS)
+            reinterpret_cast<uint4*>(dyn)[x] = reinterpret_cast<const uint4*>(mp.blob)[x];
+        __syncthreads();
+    }
     WarpTopK top;
     top.init();
     for (uint32_t b = warp; b < mp.n_partial; b += nw) {
         const uint32_t n = mp.partial_n[b];
-        for (uint32_t j = 0; j < n; ++j) {
-            const Hit hj = mp.partial[(size_t)b * SAILOR_K_MAX + j];
-            top.insert(hj.score, hj.flat, mp.k, lane);
+        Hit mine = {make_inf(), ~0ull};                  // one coalesced read of the block's list
+        if (lane < n) mine = mp.partial[(size_t)b * SAILOR_K_MAX + lane];
+        for (uint32_t j = 0; j < n; ++j) {               // the list is sorted: stop at the first reject
+            const double sj = __shfl_sync(FULL, mine.score, j);
+            const uint64_t fj = __shfl_sync(FULL, mine.flat, j);
+            if (!top.insert(sj, fj, mp.k, lane)) break;
         }
     }
     s_hits[warp][lane].score = top.score;
     s_hits[warp][lane].flat = top.flat;
     __syncthreads();
-    if (warp != 0) return;
-    for (uint32_t w = 1; w < nw; ++w)
-        for (uint32_t j = 0; j < mp.k; ++j) {
-            const Hit hj = s_hits[w][j];
-            if (hj.flat == ~0ull) break;
-            top.insert(hj.score, hj.flat, mp.k, lane);
-        }
-    const bool have = lane < mp.k && top.flat != ~0ull;
-    const uint32_t n = __popc(__ballot_sync(FULL, have));
-    TabView v;
-    v.bind(mp.blob, mp.blob);
-    double best_cost = 0.0;
-    if (have) {
-        sailor_result r;
-        r.flat = top.flat;
-        r.score = top.score;
-        r._pad = 0;
-        decode_flat(mp.sp, v.h->T, v.h->Z, top.flat, &r.plan);
-        const SimOut o = simulate_record(v, mp.avail, r.plan);
-        r.t_iter = o.t_iter;
-        r.cost = o.cost;
-        r.peak_mem = o.peak_mem;
-        r.status = o.status;
-        mp.results[lane] = r;
-        best_cost = o.cost;
+    if (warp == 0) {
+        for (uint32_t w = 1; w < nw; ++w)
+            for (uint32_t j = 0; j < mp.k; ++j) {
+                const Hit hj = s_hits[w][j];
+                if (hj.flat == ~0ull) break;
+                if (!top.insert(hj.score, hj.flat, mp.k, lane)) break;
+            }
+        const bool have = lane < mp.k && top.flat != ~0ull;
+        const uint32_t n = __popc(__ballot_sync(FULL, have));
+        s_hits[0][lane].score = top.score;
+        s_hits[0][lane].flat = top.flat;
+        if (lane == 0) s_n = n;
     }
-    best_cost = __shfl_sync(FULL, best_cost, 0);
-    if (lane == 0) {
-        mp.ctrl->n_found = n;
-        if (mp.budget_factor > 0.0)
-            mp.ctrl->budget = n ? mul_rn(mp.budget_factor, best_cost) : make_inf();
+    __syncthreads();
+    // the winners are simulated in full for the result records, one per warp at a time (each is a
+    // long single-thread dependency chain; different plans would diverge inside one warp)
+    const uint32_t n = s_n;
+    TabView v;
+    v.bind(dyn, mp.blob);
+    for (uint32_t j = warp; j < n; j += nw) {
+        if (lane == 0) {
+            sailor_result r;
+            r.flat = s_hits[0][j].flat;
+            r.score = s_hits[0][j].score;
+            r._pad = 0;
+            decode_flat(mp.sp, v.h->T, v.h->Z, r.flat, &r.plan);
+            const SimOut o = simulate_record(v, mp.avail, r.plan);
+            r.t_iter = o.t_iter;
+            r.cost = o.cost;
+            r.peak_mem = o.peak_mem;
+            r.status = o.status;
+            mp.results[j] = r;
+            if (j == 0) {
+                mp.ctrl->n_found = n;
+                if (mp.budget_factor > 0.0) mp.ctrl->budget = mul_rn(mp.budget_factor, o.cost);
+            }
+        }
+    }
+    if (n == 0 && tid == 0) {
+        mp.ctrl->n_found = 0;
+        if (mp.budget_factor > 0.0) mp.ctrl->budget = make_inf();
     }
 }
 
