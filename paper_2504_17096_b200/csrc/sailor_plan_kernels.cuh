@@ -489,25 +489,11 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
             x = y;
         }
     }
-    double acc = 0.0, mx = 0.0, sy = 0.0, up = 0.0, rate = 0.0, cc = 0.0;
+    // ---- status of the prefix: node validity, memory, availability (integer work only) ------------
     bool p_inv = false, p_oom = false, p_over = false;
 #pragma unroll
     for (int s = 0; s < NSEG - 1; ++s) {
         const uint32_t d = dg[s];
-        const SegRec& rc = a.rec[s * R + d];
-#pragma unroll
-        for (int r = 0; r < N_RUNS - 1; ++r) acc = add_n(acc, rc.v[r], cs.n_run[s][r]);   // run 3 is the final stage
-        mx = dmax(mx, rc.tmax);
-        sy = dmax(sy, rc.sync);
-        up = dmax(up, rc.upd);
-        rate = add_n(rate, rc.rate, cs.seg_a[s + 1] - cs.seg_a[s]);
-        if (s < NSEG - 2) {                               // the segment's last stage sends to the next prefix digit
-            const uint32_t dn = dg[s + 1];
-            const double tb = add_rn(a.fb_last[s * T + (a.tz[d] & 0xff)], a.c2x[dn * R + d]);
-            acc = add_rn(acc, tb);
-            mx = dmax(mx, tb);
-            cc = add_rn(cc, a.commx[dn * Z + (a.tz[d] >> 8)]);
-        }
         p_inv |= (cs.invalid_mask >> d) & 1;
         p_oom |= (cs.oom_mask[s] >> d) & 1;
         uint32_t tot = 0;                                 // demand of this digit over the prefix
@@ -554,10 +540,34 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     if (!CONSTR) cnt.feasible += n_ok;
 
     // ---- the candidates -----------------------------------------------------------------------
+    const uint64_t walk = pp.eval_all ? warp_or64(range) : warp_or64(ok);   // warp-uniform: skip dead digits
+    if (walk == 0) {                                      // nothing to evaluate for any lane of the warp
+        return;
+    }
+    // ---- running sums of the prefix, in stage order ---------------------------------------------
+    double acc = 0.0, mx = 0.0, sy = 0.0, up = 0.0, rate = 0.0, cc = 0.0;
+#pragma unroll
+    for (int s = 0; s < NSEG - 1; ++s) {
+        const uint32_t d = dg[s];
+        const SegRec& rc = a.rec[s * R + d];
+#pragma unroll
+        for (int r = 0; r < N_RUNS - 1; ++r) acc = add_n(acc, rc.v[r], cs.n_run[s][r]);   // run 3 is the final stage
+        mx = dmax(mx, rc.tmax);
+        sy = dmax(sy, rc.sync);
+        up = dmax(up, rc.upd);
+        rate = add_n(rate, rc.rate, cs.seg_a[s + 1] - cs.seg_a[s]);
+        if (s < NSEG - 2) {                               // the segment's last stage sends to the next prefix digit
+            const uint32_t dn = dg[s + 1];
+            const double tb = add_rn(a.fb_last[s * T + (a.tz[d] & 0xff)], a.c2x[dn * R + d]);
+            acc = add_rn(acc, tb);
+            mx = dmax(mx, tb);
+            cc = add_rn(cc, a.commx[dn * Z + (a.tz[d] >> 8)]);
+        }
+    }
     ItemState it;
     it.acc = acc; it.mx = mx; it.sy = sy; it.up = up; it.rate = rate; it.cc = cc;
     it.ok = ok;
-    it.walk = pp.eval_all ? warp_or64(range) : warp_or64(ok);   // warp-uniform: skip dead digits
+    it.walk = walk;
     it.fb_b = 0.0;
     uint32_t d_prev = 0, z_prev = 0;
     if (NSEG > 1) {
