@@ -153,6 +153,7 @@ struct CfgShared {
     // scalars (written by thread 0 / the build, read by all)
     Config cfg;
     uint32_t valid;              // gbs % (D*mbs) == 0 and heads % tp == 0
+    uint32_t dead;               // some segment has no digit that is valid and fits in memory
     uint32_t seg_a[SAILOR_SEG_MAX + 1];   // first stage of each segment; seg_a[nseg] = P
     uint32_t need[SAILOR_SEG_MAX];        // GPUs a segment takes of its digit: D * tp * stages
     uint32_t n_run[SAILOR_SEG_MAX][N_RUNS];   // stages in each run (without a non-final segment's last stage)
@@ -307,11 +308,17 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         a.rec[x] = r;
         if (oom) atomicOr(reinterpret_cast<unsigned long long*>(&cs.oom_mask[s]), 1ull << d);
     }
+    __syncthreads();                   // the memory masks are complete
     if (tid == 0) {
         uint64_t m = 0;
         for (uint32_t d = 0; d < R; ++d)
             if (cs.need[k.nseg - 1] <= a.availv[d]) m |= 1ull << d;
         cs.avail_last = m;
+        const uint64_t full = R == 64 ? ~0ull : ((1ull << R) - 1);
+        uint32_t dead = 0;
+        for (uint32_t s = 0; s < k.nseg; ++s)
+            if ((full & ~cs.invalid_mask & ~cs.oom_mask[s]) == 0) dead = 1;
+        cs.dead = dead;
     }
     __syncthreads();
 }
@@ -676,6 +683,20 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             const int fixed = (cs.n_run[3][0] == 0 && cs.n_run[3][1] == 0 && cs.n_run[3][3] == 1 && cs.n_run[3][2] <= 3)
                                   ? (int)cs.n_run[3][2] : -1;
 #define SAILOR_RUN(NS, NF) run_items<NS, OBJ, CONSTR, NF>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane)
+            if (cs.dead && !pp.eval_all && pp.cfg_flat_base[c] >= pp.flat_lo &&
+                pp.cfg_flat_base[c] + cs.n_items * R <= pp.flat_hi) {
+                // no candidate of this configuration can be valid and fit in memory: classes in closed
+                // form, added once (by whoever holds the configuration's first chunk), nothing evaluated
+                if (ch == pp.cfg_chunk_start[c] && tid == 0) {
+                    const uint64_t full = R == 64 ? ~0ull : ((1ull << R) - 1);
+                    const uint64_t n_all = cs.n_items * R;
+                    const uint64_t n_valid = ipow64(__popcll(full & ~cs.invalid_mask), cs.cfg.nseg);
+                    atomicAdd(&cs.stat[0], (unsigned long long)n_all);
+                    atomicAdd(&cs.stat[1], (unsigned long long)(n_all - n_valid));
+                    atomicAdd(&cs.stat[2], (unsigned long long)n_valid);
+                }
+                continue;
+            }
             switch (cs.cfg.nseg) {
                 case 1: SAILOR_RUN(1, -1); break;
                 case 2: SAILOR_RUN(2, -1); break;
