@@ -322,6 +322,21 @@ def config5() -> Workload:
     return w
 
 
+def config6() -> Workload:
+    """Shape of the paper's constrained scenario 1 (Sec. 5.2.4): two zones of one region, each with
+    128 GPUs of a 40 GiB and of a 16 GiB type; minimise cost per iteration subject to a minimum
+    throughput.  GPT-Neo-2.7B-shaped model, global batch 2048 (the paper's evaluation batch size)."""
+    w = make_workload(
+        "cfg6-min-cost-under-throughput", seed=SEED_BASE + 6, L=32, h=2560, a=20, s=2048, V=50257, gbs=2048,
+        type_mem_gib=[40, 16], type_base=[1.6e-3 / 0.55, 1.6e-3 / 0.25], type_price=[2.9, 2.5],
+        n_zones=2, gpus_per_node=4, intra_gbs=300.0, inter_gbs=25.0,
+        zone_bw_fn=lambda r: 20.0 + 5.0 * r.uniform(), avail_fn=lambda r, z, g: 128,
+        tp_values=[1, 2, 4], mbs_values=[1, 2, 4, 8], p_values=[1, 2, 4, 8, 16, 32],
+        d_values=[1, 2, 4, 8, 16, 32, 64, 128], rc_values=[0], objective=OBJ_MIN_COST)
+    w.min_iters_per_s = 0.2
+    return w
+
+
 def tiny(seed: int = 7, *, n_types: int = 2, n_zones: int = 2, L: int = 4, alpha: float = 2e-5,
          rc_values=(0, 1), objective: int = OBJ_MAX_THROUGHPUT, seg_max: int = 4, p_values=None,
          d_values=(1, 2, 3, 4, 8), tp_values=(1, 2, 4), mbs_values=(1, 2, 4), gbs: int = 32) -> Workload:
@@ -342,7 +357,7 @@ def tiny(seed: int = 7, *, n_types: int = 2, n_zones: int = 2, L: int = 4, alpha
         egress_usd_per_byte=2e-11)
 
 
-CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5}
+CONFIGS = {1: config1, 2: config2, 3: config3, 4: config4, 5: config5, 6: config6}
 
 
 def random_plans(w: Workload, n: int, seed: int, *, max_runs: int = 16, hetero_tp: bool = True):

@@ -241,6 +241,43 @@ def test_plan_deep_pipelines_up_to_96_stages(make_ctx):
     assert_sim_equal(B.sailor_simulate(cx.ctx, B.pack_records(recs)), o.simulate_records(recs), "deep")
 
 
+def test_plan_random_shapes_sweep(make_ctx):
+    """Seeded sweep over cluster shapes, layer counts, segment limits, objectives, constraints, k and
+    sub-ranges: every search must equal the exhaustive oracle."""
+    rng = W.SplitMix64(2024)
+    for case in range(24):
+        T, Z = rng.randint(1, 4), rng.randint(1, 3)
+        L = rng.randint(2, 9)
+        seg_max = rng.randint(1, 4)
+        objective = rng.randint(0, 2)
+        p_values = sorted({rng.randint(1, L) for _ in range(3)})
+        w = W.tiny(seed=100 + case, n_types=T, n_zones=Z, L=L, seg_max=seg_max, objective=objective,
+                   p_values=p_values, alpha=rng.uniform() * 1e-4)
+        if rng.uniform() < 0.3:
+            w.has_embed = 0
+        if rng.uniform() < 0.3:
+            w.has_head = 0
+        cx = make_ctx(w)
+        o = Oracle(w)
+        n = o.space_size()
+        k = rng.randint(1, 32)
+        kw = {}
+        probe, _ = o.search(objective, 32)
+        if probe and rng.uniform() < 0.5:
+            kw["budget"] = sorted(h["cost"] for h in probe)[len(probe) // 2]
+        if probe and rng.uniform() < 0.3:
+            kw["min_rate"] = 1.0 / sorted(h["t_iter"] for h in probe)[len(probe) // 2]
+        lo, hi = 0, n
+        if rng.uniform() < 0.5:
+            lo = rng.randint(0, n - 1)
+            hi = rng.randint(lo, n)
+        flags = B.FLAG_EVAL_ALL if rng.uniform() < 0.5 else 0
+        hits, counts = o.search(objective, k, lo=lo, hi=hi, **kw)
+        res, st = B.sailor_plan_range(cx.ctx, cx.space, B.make_objective(w, flags=flags, **kw), lo, hi, k)
+        assert_plan_equal(res, st, hits, counts, o, f"case {case}: T={T} Z={Z} L={L} seg_max={seg_max} obj={objective} "
+                                                    f"P={p_values} k={k} [{lo},{hi}) {kw} flags={flags}")
+
+
 def test_plan_constraints_and_empty_results(make_ctx):
     w = W.tiny(seed=8, n_types=2, n_zones=2)
     cx = make_ctx(w)
@@ -339,6 +376,19 @@ def test_plan_config2_budget_factor_two_pass(make_ctx):
     res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w), 16)
     assert st.budget_used == budget
     assert_plan_equal(res, st, hits, counts, o)
+
+
+def test_plan_config6_min_cost_under_throughput(make_ctx):
+    """Minimise cost subject to a minimum throughput (the paper's constrained scenario 1 shape)."""
+    w = W.config6()
+    cx = make_ctx(w)
+    o = Oracle(w)
+    hits, counts, _ = o.plan(16)
+    assert counts["n_over_constraint"] > 0 and counts["n_feasible"] > 16
+    for flags in (0, B.FLAG_EVAL_ALL):
+        res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=flags), 16)
+        assert_plan_equal(res, st, hits, counts, o, f"flags={flags}")
+    assert all(1.0 / r.t_iter >= w.min_iters_per_s for r in res)
 
 
 def test_plan_config4_snapshots_replan(make_ctx):
