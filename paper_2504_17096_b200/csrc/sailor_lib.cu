@@ -63,6 +63,8 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
     __shared__ uint64_t mbar;
     constexpr uint32_t W = sizeof(sailor_plan_rec) / 8;      // 9 words per record
     __shared__ uint64_t recs[SIM_THREADS * W];
+    __shared__ uint32_t hist[128];
+    __shared__ uint16_t perm[SIM_THREADS];
     const uint32_t tid = threadIdx.x;
     const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(blob)->static_bytes;
     if (!bulk_load(dyn, blob, static_bytes, &mbar)) {
@@ -74,20 +76,47 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
     TabView v;
     v.bind(dyn, blob);
     const uint64_t* src = reinterpret_cast<const uint64_t*>(plans);
+    uint32_t* counters = reinterpret_cast<uint32_t*>(dyn + static_bytes);      // [digit][thread]
     for (uint64_t tile = (uint64_t)blockIdx.x * SIM_THREADS; tile < n; tile += (uint64_t)gridDim.x * SIM_THREADS) {
-        const uint64_t cnt = n - tile < SIM_THREADS ? n - tile : SIM_THREADS;
+        const uint32_t cnt = (uint32_t)(n - tile < SIM_THREADS ? n - tile : SIM_THREADS);
         __syncthreads();
         for (uint32_t x = tid; x < cnt * W; x += SIM_THREADS) recs[x] = src[tile * W + x];
+        if (tid < 128) hist[tid] = 0;
+        __syncthreads();
+        // the work of a record grows with its stage count: order the tile by stage count so that the
+        // lanes of a warp run loops of similar length (counting sort; any order gives the same results)
+        uint32_t key = 0, rank = 0;
+        if (tid < cnt) {
+            key = (uint32_t)(recs[tid * W] & 0xff);            // byte 0 of a record is P
+            key = key > 127u ? 127u : key;
+            rank = atomicAdd(&hist[key], 1u);
+        }
+        __syncthreads();
+        if (tid < 32) {                                        // exclusive scan of the 128 bins by one warp
+            uint32_t h4[4], sum = 0;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { h4[q] = hist[tid * 4 + q]; sum += h4[q]; }
+            uint32_t incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t up = __shfl_up_sync(FULL, incl, o);
+                if (tid >= (uint32_t)o) incl += up;
+            }
+            uint32_t base = incl - sum;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) { hist[tid * 4 + q] = base; base += h4[q]; }
+        }
+        __syncthreads();
+        if (tid < cnt) perm[hist[key] + rank] = (uint16_t)tid;
         __syncthreads();
         if (tid < cnt) {
-            union { sailor_plan_rec r; uint64_t w[W]; } u;      // 8-byte aligned copy of the record
-#pragma unroll
-            for (uint32_t w = 0; w < W; ++w) u.w[w] = recs[tid * W + w];
-            const SimOut o = simulate_record(v, avail, u.r);
-            if (t_iter) t_iter[tile + tid] = o.t_iter;
-            if (peak_mem) peak_mem[tile + tid] = o.peak_mem;
-            if (cost) cost[tile + tid] = o.cost;
-            if (status) status[tile + tid] = o.status;
+            const uint32_t mine = perm[tid];
+            const sailor_plan_rec& rec = *reinterpret_cast<const sailor_plan_rec*>(&recs[mine * W]);   // in shared memory
+            const SimOut o = simulate_record(v, avail, rec, counters + tid, SIM_THREADS);
+            if (t_iter) t_iter[tile + mine] = o.t_iter;
+            if (peak_mem) peak_mem[tile + mine] = o.peak_mem;
+            if (cost) cost[tile + mine] = o.cost;
+            if (status) status[tile + mine] = o.status;
         }
     }
 }
@@ -546,7 +575,7 @@ int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_c
     }
     CUF(cudaStreamSynchronize(ctx->stream));           // `blob` is pageable host memory
     // both kernels stage the static tables in dynamic shared memory; the create-time limit is 96 KB
-    CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
+    CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
     CUF(cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
 #undef CUF
     *out = ctx;
@@ -622,7 +651,8 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
     const uint64_t tiles = (n + SIM_THREADS - 1) / SIM_THREADS;
     const uint64_t cap = (uint64_t)ctx->sm_count * 16;
     const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
-    simulate_kernel<<<grid, SIM_THREADS, ctx->hdr.static_bytes, ctx->stream>>>(
+    const size_t sim_smem = ctx->hdr.static_bytes + sizeof(uint32_t) * SIM_THREADS * ctx->hdr.R;   // tables + per-thread counters
+    simulate_kernel<<<grid, SIM_THREADS, sim_smem, ctx->stream>>>(
         ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s, &ctx->d_ctrl->error);
     CU(ctx, cudaGetLastError());
     if (!on_device) {

@@ -769,6 +769,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const __grid_const
     __shared__ Hit s_hits[MERGE_THREADS / 32][SAILOR_K_MAX];
     __shared__ uint64_t mbar;
     __shared__ uint32_t s_n;
+    __shared__ uint32_t s_cnt[R_MAX][MERGE_THREADS / 32];   // per-digit GPU counters of each warp's record
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = MERGE_THREADS / 32;
     const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(mp.blob)->static_bytes;
     if (!bulk_load(dyn, mp.blob, static_bytes, &mbar)) {
@@ -818,7 +819,7 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const __grid_const
             r.score = s_hits[0][j].score;
             r._pad = 0;
             decode_flat(mp.sp, v.h->T, v.h->Z, r.flat, &r.plan);
-            const SimOut o = simulate_record(v, mp.avail, r.plan);
+            const SimOut o = simulate_record(v, mp.avail, r.plan, &s_cnt[0][warp], MERGE_THREADS / 32);
             r.t_iter = o.t_iter;
             r.cost = o.cost;
             r.peak_mem = o.peak_mem;

@@ -191,8 +191,13 @@ __device__ __forceinline__ double make_inf() { return __longlong_as_double(0x7ff
 
 // Simulate one run-length encoded plan (Sec. 4.3).  Every index is checked before use; a
 // record that fails gets SAILOR_ST_BAD_RECORD and nothing is read through it.
+//
+// The stages are walked in one flat loop (no loop nest over runs), so that the lanes of a warp,
+// each with its own record, stay on the same instructions; values that depend only on the
+// stage's layer composition and run are refreshed when either changes.  `cnt` points to this
+// thread's per-digit GPU counters (digit d at cnt[d * cnt_stride], any initial contents).
 __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __restrict__ avail,
-                                         const sailor_plan_rec& r) {
+                                         const sailor_plan_rec& r, uint32_t* cnt, uint32_t cnt_stride) {
     const TabHdr* h = v.h;
     SimOut o;
     o.t_iter = o.cost = make_nan();
@@ -202,7 +207,7 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
     if (P < 1 || P > SAILOR_P_MAX || n_runs < 1 || n_runs > SAILOR_RUN_MAX || D < 1 || mi >= h->n_mbs) return o;
     uint32_t tot = 0;
     for (uint32_t q = 0; q < n_runs; ++q) {
-        const sailor_run& rr = r.run[q];
+        const sailor_run rr = r.run[q];
         if (rr.type >= h->T || rr.zone >= h->Z || rr.tp_idx >= h->n_tp || rr.n_stages < 1) return o;
         tot += rr.n_stages;
     }
@@ -214,76 +219,94 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
     if (h->gbs % dm != 0) status |= SAILOR_ST_INVALID;
     const uint64_t n_b = h->gbs / dm;
 
-    // resources: total demand of every (zone, type) a run touches
+    // resources: GPUs taken of every (zone, type), saturating at 2^32 - 1 (availability is 16 bits)
+    for (uint32_t d = 0; d < h->R; ++d) cnt[d * cnt_stride] = 0;
     for (uint32_t q = 0; q < n_runs; ++q) {
-        const sailor_run& a = r.run[q];
+        const sailor_run a = r.run[q];
         const uint32_t tp = h->tp_values[a.tp_idx];
         if (tp > h->gpn[a.type] || h->heads % tp != 0) status |= SAILOR_ST_INVALID;
-        uint64_t need = 0;
-        for (uint32_t q2 = 0; q2 < n_runs; ++q2) {
-            const sailor_run& b = r.run[q2];
-            if (b.type == a.type && b.zone == a.zone)
-                need += (uint64_t)D * h->tp_values[b.tp_idx] * b.n_stages;
-        }
-        if (need > avail[a.zone * h->T + a.type]) status |= SAILOR_ST_OVER_AVAIL;
+        uint32_t* c = cnt + (a.zone * h->T + a.type) * cnt_stride;
+        const uint64_t sum = (uint64_t)*c + (uint64_t)D * tp * a.n_stages;
+        *c = sum > 0xffffffffull ? 0xffffffffu : (uint32_t)sum;
+    }
+    for (uint32_t q = 0; q < n_runs; ++q) {
+        const uint32_t d = r.run[q].zone * h->T + r.run[q].type;
+        if (cnt[d * cnt_stride] > avail[d]) status |= SAILOR_ST_OVER_AVAIL;
     }
 
     const uint32_t base = h->n_blocks / P, extra = h->n_blocks % P;
     const double msg = (double)v.p2p[mi];
     const uint64_t xbytes = 2 * n_b * (uint64_t)D * v.p2p[mi];
+    const double steps = (double)(2 * (uint64_t)(D - 1));
+    const double coef = steps / (double)D;                 // ring all-reduce: 2(D-1)/D
     double sum_t = 0.0, max_t = 0.0, max_sync = 0.0, max_u = 0.0, rate = 0.0, c_comm = 0.0;
     uint64_t peak = 0;
-    uint32_t i = 0;
-    for (uint32_t q = 0; q < n_runs; ++q) {
-        const sailor_run a = r.run[q];
-        const uint32_t g = a.type, z = a.zone, tpi = a.tp_idx, tp = h->tp_values[tpi];
-        const double gpu_rate = mul_rn((double)(D * tp), v.price_s[z * h->T + g]);
-        const uint64_t cap = h->capacity[g], resv = h->reserved[g];
-        // a run's stages differ only by layer composition (embedding / extra block / plain / head):
-        // the composition-dependent values are formed when the composition changes, not per stage
-        uint32_t cur_nb = 0xffffffffu;
-        bool cur_e = false, cur_hd = false;
-        double fb = 0.0, upd = 0.0, sync = 0.0, t_self = 0.0;
-        uint64_t m_fixed = 0, m_keep = 0;
-        const double c2_self = mul_rn(2.0, boundary_time(v, g, z, tp, g, z, tp, D, msg));
-        for (uint32_t j = 0; j < a.n_stages; ++j, ++i) {
-            const uint32_t nb = base + (i < extra ? 1u : 0u);
-            const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
-            if (nb != cur_nb || e != cur_e || hd != cur_hd) {
-                cur_nb = nb; cur_e = e; cur_hd = hd;
-                const StageTimes st = stage_times(v, g, tpi, mi, nb, e, hd);
-                const double b = rc ? add_rn(st.b, st.f) : st.b;
-                fb = add_rn(st.f, b);
-                upd = st.u;
-                const StageMem one = stage_memory(v, tpi, mi, rc, nb, e, hd, 1);     // model + 1 * kept + work
-                const StageMem zero = stage_memory(v, tpi, mi, rc, nb, e, hd, 0);    // model + work
-                m_keep = one.mem - zero.mem;
-                m_fixed = zero.mem + resv;
-                sync = sync_time(v, g, z, tp, D, one.params);
-                t_self = add_rn(fb, c2_self);
-            }
-            const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
-            const uint64_t m = m_fixed + inflight * m_keep;
-            if (m > cap) status |= SAILOR_ST_OOM;
-            peak = m > peak ? m : peak;
 
-            double t = fb;                                   // the final stage sends nothing: fb + 2*0
-            if (i + 1 < P) {
-                if (j + 1 < a.n_stages) {
-                    t = t_self;
-                } else {
-                    const sailor_run nx = r.run[q + 1];
-                    const double c = boundary_time(v, g, z, tp, nx.type, nx.zone, h->tp_values[nx.tp_idx], D, msg);
-                    if (nx.zone != z) c_comm = add_rn(c_comm, mul_rn((double)xbytes, v.egress[z * h->Z + nx.zone]));
-                    t = add_rn(fb, mul_rn(2.0, c));
-                }
-            }
-            sum_t = add_rn(sum_t, t);
-            max_t = dmax(max_t, t);
-            max_u = dmax(max_u, upd);
-            max_sync = dmax(max_sync, sync);
-            rate = add_rn(rate, gpu_rate);
+    // current run
+    uint32_t q = 0, left = 0, g = 0, z = 0, tpi = 0, tp = 1;
+    double gpu_rate = 0.0, c2_self = 0.0, dp_alpha = 0.0, dp_inv = 0.0;
+    uint64_t cap = 0, resv = 0;
+    // current layer composition
+    uint32_t cur_nb = 0xffffffffu;
+    bool cur_e = false, cur_hd = false;
+    double fb = 0.0, upd = 0.0, sync = 0.0, t_self = 0.0;
+    uint64_t m_fixed = 0, m_keep = 0;
+
+    for (uint32_t i = 0; i < P; ++i) {
+        bool refresh = false;
+        if (left == 0) {                                   // enter run q
+            const sailor_run a = r.run[q];
+            g = a.type; z = a.zone; tpi = a.tp_idx; tp = h->tp_values[tpi]; left = a.n_stages;
+            const uint32_t d = z * h->T + g;
+            gpu_rate = mul_rn((double)(D * tp), v.price_s[d]);
+            cap = h->capacity[g];
+            resv = h->reserved[g];
+            c2_self = mul_rn(2.0, boundary_time(v, g, z, tp, g, z, tp, D, msg));
+            const bool intra = (uint64_t)D * tp <= h->gpn[g];
+            dp_alpha = intra ? v.intra_a[d] : v.inter_a[d];
+            dp_inv = intra ? v.intra_i[d] : v.inter_i[d];
+            refresh = true;
         }
+        const uint32_t nb = base + (i < extra ? 1u : 0u);
+        const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
+        if (refresh || nb != cur_nb || e != cur_e || hd != cur_hd) {
+            cur_nb = nb; cur_e = e; cur_hd = hd;
+            const StageTimes st = stage_times(v, g, tpi, mi, nb, e, hd);
+            const double b = rc ? add_rn(st.b, st.f) : st.b;
+            fb = add_rn(st.f, b);
+            upd = st.u;
+            const StageMem one = stage_memory(v, tpi, mi, rc, nb, e, hd, 1);     // model + 1 * kept + work
+            const StageMem zero = stage_memory(v, tpi, mi, rc, nb, e, hd, 0);    // model + work
+            m_keep = one.mem - zero.mem;
+            m_fixed = zero.mem + resv;
+            sync = 0.0;
+            if (D > 1) {
+                const double gradbytes = (double)(ceil_div64(one.params, tp) * h->grad_bytes);
+                sync = add_rn(mul_rn(mul_rn(coef, gradbytes), dp_inv), mul_rn(steps, dp_alpha));
+            }
+            t_self = add_rn(fb, c2_self);
+        }
+        const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
+        const uint64_t m = m_fixed + inflight * m_keep;
+        if (m > cap) status |= SAILOR_ST_OOM;
+        peak = m > peak ? m : peak;
+
+        double t = fb;                                       // the final stage sends nothing: fb + 2*0
+        if (i + 1 < P) {
+            t = t_self;                                      // next stage in the same run
+            if (left == 1) {                                 // next stage opens run q + 1
+                const sailor_run nx = r.run[q + 1];
+                const double c = boundary_time(v, g, z, tp, nx.type, nx.zone, h->tp_values[nx.tp_idx], D, msg);
+                if (nx.zone != z) c_comm = add_rn(c_comm, mul_rn((double)xbytes, v.egress[z * h->Z + nx.zone]));
+                t = add_rn(fb, mul_rn(2.0, c));
+            }
+        }
+        sum_t = add_rn(sum_t, t);
+        max_t = dmax(max_t, t);
+        max_u = dmax(max_u, upd);
+        max_sync = dmax(max_sync, sync);
+        rate = add_rn(rate, gpu_rate);
+        if (--left == 0) ++q;
     }
     o.peak_mem = peak;
     o.status = status;
