@@ -52,8 +52,12 @@ __global__ void chain_kernel(unsigned char* blob) {
     }
 }
 
-// One thread per explicit plan record (Sec. 4.3).  Records are staged through shared memory
-// with coalesced 8-byte loads; results leave as four structure-of-arrays streams.
+// One thread per explicit plan record (Sec. 4.3).  A block stages a pool of records in shared
+// memory with coalesced 8-byte loads, orders it by stage count (the work of a record grows with
+// its stages; any order gives the same results), and its warps take groups of 32 similar records
+// from the pool, longest first, until it is empty.  Results leave as four structure-of-arrays streams.
+constexpr uint32_t SIM_POOL = 512;
+
 __global__ void __launch_bounds__(SIM_THREADS)
 simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
                 const sailor_plan_rec* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
@@ -62,10 +66,11 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ uint64_t mbar;
     constexpr uint32_t W = sizeof(sailor_plan_rec) / 8;      // 9 words per record
-    __shared__ uint64_t recs[SIM_THREADS * W];
+    __shared__ uint64_t recs[SIM_POOL * W];
     __shared__ uint32_t hist[128];
-    __shared__ uint16_t perm[SIM_THREADS];
-    const uint32_t tid = threadIdx.x;
+    __shared__ uint16_t perm[SIM_POOL];
+    __shared__ uint32_t next_group;
+    const uint32_t tid = threadIdx.x, lane = tid & 31;
     const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(blob)->static_bytes;
     if (!bulk_load(dyn, blob, static_bytes, &mbar)) {
         if (tid == 0) atomicExch(error, 1u);
@@ -76,20 +81,25 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
     TabView v;
     v.bind(dyn, blob);
     const uint64_t* src = reinterpret_cast<const uint64_t*>(plans);
-    uint32_t* counters = reinterpret_cast<uint32_t*>(dyn + static_bytes);      // [digit][thread]
-    for (uint64_t tile = (uint64_t)blockIdx.x * SIM_THREADS; tile < n; tile += (uint64_t)gridDim.x * SIM_THREADS) {
-        const uint32_t cnt = (uint32_t)(n - tile < SIM_THREADS ? n - tile : SIM_THREADS);
+    uint32_t* counters = reinterpret_cast<uint32_t*>(dyn + static_bytes) + tid;      // [digit][thread]
+    for (uint64_t pool = (uint64_t)blockIdx.x * SIM_POOL; pool < n; pool += (uint64_t)gridDim.x * SIM_POOL) {
+        const uint32_t cnt = (uint32_t)(n - pool < SIM_POOL ? n - pool : SIM_POOL);
         __syncthreads();
-        for (uint32_t x = tid; x < cnt * W; x += SIM_THREADS) recs[x] = src[tile * W + x];
+        for (uint32_t x = tid; x < cnt * W; x += SIM_THREADS) recs[x] = src[pool * W + x];
         if (tid < 128) hist[tid] = 0;
+        if (tid == 0) next_group = 0;
         __syncthreads();
-        // the work of a record grows with its stage count: order the tile by stage count so that the
-        // lanes of a warp run loops of similar length (counting sort; any order gives the same results)
-        uint32_t key = 0, rank = 0;
-        if (tid < cnt) {
-            key = (uint32_t)(recs[tid * W] & 0xff);            // byte 0 of a record is P
-            key = key > 127u ? 127u : key;
-            rank = atomicAdd(&hist[key], 1u);
+        // counting sort by descending stage count (byte 0 of a record is P)
+        uint32_t key[SIM_POOL / SIM_THREADS], rank[SIM_POOL / SIM_THREADS];
+#pragma unroll
+        for (uint32_t u = 0; u < SIM_POOL / SIM_THREADS; ++u) {
+            const uint32_t x = tid + u * SIM_THREADS;
+            key[u] = rank[u] = 0;
+            if (x < cnt) {
+                const uint32_t P = (uint32_t)(recs[x * W] & 0xff);
+                key[u] = 127u - (P > 127u ? 127u : P);
+                rank[u] = atomicAdd(&hist[key[u]], 1u);
+            }
         }
         __syncthreads();
         if (tid < 32) {                                        // exclusive scan of the 128 bins by one warp
@@ -107,16 +117,29 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
             for (int q = 0; q < 4; ++q) { hist[tid * 4 + q] = base; base += h4[q]; }
         }
         __syncthreads();
-        if (tid < cnt) perm[hist[key] + rank] = (uint16_t)tid;
+#pragma unroll
+        for (uint32_t u = 0; u < SIM_POOL / SIM_THREADS; ++u) {
+            const uint32_t x = tid + u * SIM_THREADS;
+            if (x < cnt) perm[hist[key[u]] + rank[u]] = (uint16_t)x;
+        }
         __syncthreads();
-        if (tid < cnt) {
-            const uint32_t mine = perm[tid];
-            const sailor_plan_rec& rec = *reinterpret_cast<const sailor_plan_rec*>(&recs[mine * W]);   // in shared memory
-            const SimOut o = simulate_record(v, avail, rec, counters + tid, SIM_THREADS);
-            if (t_iter) t_iter[tile + mine] = o.t_iter;
-            if (peak_mem) peak_mem[tile + mine] = o.peak_mem;
-            if (cost) cost[tile + mine] = o.cost;
-            if (status) status[tile + mine] = o.status;
+        const uint32_t n_groups = (cnt + 31) / 32;
+        for (;;) {                                             // warps drain the pool, longest records first
+            uint32_t grp = 0;
+            if (lane == 0) grp = atomicAdd(&next_group, 1u);
+            grp = __shfl_sync(FULL, grp, 0);
+            if (grp >= n_groups) break;
+            const uint32_t slot = grp * 32 + lane;
+            if (slot < cnt) {
+                const uint32_t mine = perm[slot];
+                const sailor_plan_rec& rec = *reinterpret_cast<const sailor_plan_rec*>(&recs[mine * W]);
+                const SimOut o = simulate_record(v, avail, rec, counters, SIM_THREADS);
+                if (t_iter) t_iter[pool + mine] = o.t_iter;
+                if (peak_mem) peak_mem[pool + mine] = o.peak_mem;
+                if (cost) cost[pool + mine] = o.cost;
+                if (status) status[pool + mine] = o.status;
+            }
+            __syncwarp();
         }
     }
 }
@@ -648,7 +671,7 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
         CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_plan_rec), cudaMemcpyHostToDevice, ctx->stream));
         d_plans = dp;
     }
-    const uint64_t tiles = (n + SIM_THREADS - 1) / SIM_THREADS;
+    const uint64_t tiles = (n + SIM_POOL - 1) / SIM_POOL;
     const uint64_t cap = (uint64_t)ctx->sm_count * 16;
     const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
     const size_t sim_smem = ctx->hdr.static_bytes + sizeof(uint32_t) * SIM_THREADS * ctx->hdr.R;   // tables + per-thread counters
