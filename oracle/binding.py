@@ -53,6 +53,7 @@ class OrcInputs(C.Structure):
         ("capacity", _u64p), ("reserved", _u64p), ("gpus_per_node", _u32p),
         ("price_per_hour", _dp), ("intra_alpha", _dp), ("intra_inv_bw", _dp), ("inter_alpha", _dp),
         ("inter_inv_bw", _dp), ("zone_alpha", _dp), ("zone_inv_bw", _dp), ("egress", _dp),
+        ("intra_bw_poly", _dp), ("inter_bw_poly", _dp), ("zone_bw_poly", _dp),
         ("avail", _u16p),
     ]
 
@@ -153,6 +154,9 @@ class Oracle:
         for name in ("params", "act_saved", "act_ckpt", "act_work", "p2p_bytes", "capacity", "reserved"):
             put(name, getattr(w, name), np.uint64, _u64p)
         put("gpus_per_node", w.gpus_per_node, np.uint32, _u32p)
+        for name in ("intra_bw_poly", "inter_bw_poly", "zone_bw_poly"):
+            if getattr(w, name, None) is not None:
+                put(name, getattr(w, name), np.float64, _dp)
         self._avail = put("avail", np.array(w.avail if avail is None else avail, dtype=np.uint16, copy=True),
                           np.uint16, _u16p)
         self.inputs = i

@@ -38,9 +38,19 @@ static uint32_t stage_layers(const orc_inputs* in, uint32_t P, uint32_t i, uint8
     return n;
 }
 
-/* time of one message of `bytes` over a link: degree-1 fit of Sec. 4.1's bandwidth profile */
-static double link_time(double alpha, double inv_bw, uint64_t bytes) {
-    return alpha + (double)bytes * inv_bw;
+/* bandwidth of a link for a message of m bytes from its fitted polynomial (Sec. 4.1), Horner form */
+static double poly_bw(const double* poly, double m) {
+    return ((poly[3] * m + poly[2]) * m + poly[1]) * m + poly[0];
+}
+static const double* poly_at(const double* table, uint32_t idx) { return table ? table + 4 * idx : 0; }
+
+/* time of one message of `bytes` over a link (Sec. 4.1: bandwidth depends on the message size).
+ * With a fitted polynomial the time is alpha + m / bandwidth(m); without one it is the degree-1
+ * time model alpha + m * inv_bw. */
+static double link_time(double alpha, double inv_bw, const double* poly, uint64_t bytes) {
+    double m = (double)bytes;
+    if (poly) return alpha + m / poly_bw(poly, m);
+    return alpha + m * inv_bw;
 }
 
 void orc_simulate(const orc_inputs* in, const orc_plan* pl, orc_out* out) {
@@ -123,12 +133,16 @@ void orc_simulate(const orc_inputs* in, const orc_plan* pl, orc_out* out) {
             uint32_t g2 = pl->type[i + 1], z2 = pl->zone[i + 1];
             uint32_t tp2 = in->tp_values[pl->tp_idx[i + 1]];
             if (z != z2) {
-                c = link_time(in->zone_alpha[z * Z + z2], in->zone_inv_bw[z * Z + z2], msg);
+                c = link_time(in->zone_alpha[z * Z + z2], in->zone_inv_bw[z * Z + z2],
+                              poly_at(in->zone_bw_poly, z * Z + z2), msg);
             } else if (g == g2 && (uint64_t)D * (tp + tp2) <= in->gpus_per_node[g]) {
-                c = link_time(in->intra_alpha[z * T + g], in->intra_inv_bw[z * T + g], msg);
+                c = link_time(in->intra_alpha[z * T + g], in->intra_inv_bw[z * T + g],
+                              poly_at(in->intra_bw_poly, z * T + g), msg);
             } else {
-                double c1 = link_time(in->inter_alpha[z * T + g], in->inter_inv_bw[z * T + g], msg);
-                double c2 = link_time(in->inter_alpha[z * T + g2], in->inter_inv_bw[z * T + g2], msg);
+                double c1 = link_time(in->inter_alpha[z * T + g], in->inter_inv_bw[z * T + g],
+                                      poly_at(in->inter_bw_poly, z * T + g), msg);
+                double c2 = link_time(in->inter_alpha[z * T + g2], in->inter_inv_bw[z * T + g2],
+                                      poly_at(in->inter_bw_poly, z * T + g2), msg);
                 c = max_f64(c1, c2);
             }
         }
@@ -144,16 +158,24 @@ void orc_simulate(const orc_inputs* in, const orc_plan* pl, orc_out* out) {
         if (D > 1) {
             uint64_t gradbytes = ceil_div_u64(params_stage[i], tp) * in->grad_dtype_size;
             double alpha, inv;
+            const double* poly;
             if ((uint64_t)D * tp <= in->gpus_per_node[g]) {
                 alpha = in->intra_alpha[z * T + g];
                 inv = in->intra_inv_bw[z * T + g];
+                poly = poly_at(in->intra_bw_poly, z * T + g);
             } else {
                 alpha = in->inter_alpha[z * T + g];
                 inv = in->inter_inv_bw[z * T + g];
+                poly = poly_at(in->inter_bw_poly, z * T + g);
             }
-            double steps = (double)(2 * (uint64_t)(D - 1));
+            double steps = (double)(2 * (uint64_t)(D - 1));      /* ring: 2(D-1) messages of gradbytes/D */
             double coef = steps / (double)D;
-            sync = (coef * (double)gradbytes) * inv + steps * alpha;
+            if (poly) {
+                double chunk = (double)gradbytes / (double)D;
+                sync = (coef * (double)gradbytes) / poly_bw(poly, chunk) + steps * alpha;
+            } else {
+                sync = (coef * (double)gradbytes) * inv + steps * alpha;
+            }
         }
         out->stage_sync[i] = sync;
         max_sync = max_f64(max_sync, sync);

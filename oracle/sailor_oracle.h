@@ -67,6 +67,11 @@ typedef struct orc_inputs {
     const double* zone_alpha;      /* [zone][zone] */
     const double* zone_inv_bw;
     const double* egress;          /* [zone][zone] dollars per byte */
+    /* optional fitted bandwidth polynomials, Sec. 4.1: bandwidth(m) = p0 + p1 m + p2 m^2 + p3 m^3 bytes/s
+     * for a message of m bytes; NULL = the link uses inv_bw */
+    const double* intra_bw_poly;   /* [zone][type][4] or NULL */
+    const double* inter_bw_poly;   /* [zone][type][4] or NULL */
+    const double* zone_bw_poly;    /* [zone][zone][4] or NULL */
     const uint16_t* avail;         /* [zone][type] */
 } orc_inputs;
 

@@ -124,6 +124,10 @@ class Workload:
     budget_usd_per_iter: float = 0.0
     min_iters_per_s: float = 0.0
     budget_factor_over_cheapest: float = 0.0
+    # optional fitted bandwidth polynomials (bytes/s as a cubic in the message size); None = inv_bw is used
+    intra_bw_poly: Optional[np.ndarray] = None   # f64 [zone][type][4]
+    inter_bw_poly: Optional[np.ndarray] = None   # f64 [zone][type][4]
+    zone_bw_poly: Optional[np.ndarray] = None    # f64 [zone][zone][4]
     # dynamic availability (workload 4): [snapshot][zone][type]
     snapshots: Optional[np.ndarray] = None
     notes: Dict[str, float] = field(default_factory=dict)
@@ -237,6 +241,24 @@ def make_workload(name: str, *, seed: int, L: int, h: int, a: int, s: int, V: in
         p_values=list(p_values), mbs_idx=list(range(n_mbs)), tp_idx=list(range(n_tp)),
         rc_values=list(rc_values), d_values=list(d_values), seg_max=seg_max,
         objective=objective, budget_factor_over_cheapest=budget_factor)
+
+
+def with_bandwidth_polynomials(w: Workload, seed: int) -> Workload:
+    """Give every link a fitted bandwidth curve that rises with the message size (Sec. 4.1):
+    bandwidth(m) = bw * (0.25 + a1 * m + a2 * m^2) with small positive a1, a2 drawn from `seed`,
+    bw being the link's constant bandwidth.  The constant-bandwidth fields stay but are ignored."""
+    rng = SplitMix64(seed)
+
+    def curve(inv_bw: float):
+        bw = 1.0 / inv_bw if inv_bw > 0 else 1e9
+        return [0.25 * bw, bw * (2e-8 + 4e-8 * rng.uniform()), bw * 1e-16 * rng.uniform(), 0.0]
+
+    Z, T = w.n_zones, w.n_types
+    w.intra_bw_poly = np.array([[curve(w.intra_inv_bw[z, g]) for g in range(T)] for z in range(Z)])
+    w.inter_bw_poly = np.array([[curve(w.inter_inv_bw[z, g]) for g in range(T)] for z in range(Z)])
+    w.zone_bw_poly = np.array([[curve(w.zone_inv_bw[z0, z1]) for z1 in range(Z)] for z0 in range(Z)])
+    w.name += "-bwpoly"
+    return w
 
 
 def _cap_total(avail: np.ndarray, cap: int) -> np.ndarray:

@@ -23,8 +23,9 @@ def workload_from_tables(t: dict, name: str = "fixture") -> W.Workload:
     """A Workload from a fixture's written-out tables, with a one-point search space."""
     f64 = lambda k: np.array(t[k], dtype=np.float64)
     u64 = lambda k: np.array(t[k], dtype=np.uint64)
+    poly = {k: np.array(t[k], dtype=np.float64) for k in ("intra_bw_poly", "inter_bw_poly", "zone_bw_poly") if k in t}
     return W.Workload(
-        name=name, n_blocks=t["n_blocks"], has_embed=t["has_embed"], has_head=t["has_head"],
+        **poly, name=name, n_blocks=t["n_blocks"], has_embed=t["has_embed"], has_head=t["has_head"],
         heads=t["heads"], gbs=t["gbs"], mul_factor=t["mul_factor"], dtype_size=t["dtype_size"],
         grad_dtype_size=t["grad_dtype_size"], tp_values=list(t["tp_values"]),
         mbs_values=list(t["mbs_values"]), fwd=f64("fwd"), bwd=f64("bwd"), upd=f64("upd"),

@@ -218,6 +218,36 @@ def test_memory_mask_independent_of_availability(tiny_w):
     assert np.all((st1 & ST_OVER_AVAIL) != 0)
 
 
+def test_bandwidth_polynomials(tiny_w):
+    """Sec. 4.1: bandwidth as a fitted polynomial of the message size.  A constant polynomial equals
+    the constant-bandwidth model (up to the rounding of 1/x), and more bandwidth never costs time."""
+    base = Oracle(tiny_w)
+    plans = _random_feasible_plans(tiny_w, base, 200, seed=17)
+    ref = [base.simulate(p) for p in plans]
+    w2 = copy.deepcopy(tiny_w)
+    const = lambda inv: np.stack([1.0 / inv, 0 * inv, 0 * inv, 0 * inv], axis=-1)
+    w2.intra_bw_poly, w2.inter_bw_poly = const(w2.intra_inv_bw), const(w2.inter_inv_bw)
+    zi = np.where(w2.zone_inv_bw > 0, w2.zone_inv_bw, 1.0)
+    w2.zone_bw_poly = const(zi)
+    for name in ("intra_inv_bw", "inter_inv_bw", "zone_inv_bw"):
+        getattr(w2, name)[...] = 123.0                      # must be ignored now
+    o2 = Oracle(w2)
+    for p, r in zip(plans, ref):
+        s = o2.simulate(p)
+        assert s.t_iter == pytest.approx(r.t_iter, rel=1e-13) and s.cost == pytest.approx(r.cost, rel=1e-13)
+        assert s.status == r.status and s.peak_mem == r.peak_mem
+    w3 = W.with_bandwidth_polynomials(copy.deepcopy(tiny_w), seed=5)
+    o3 = Oracle(w3)
+    t3 = [o3.simulate(p).t_iter for p in plans]
+    w4 = copy.deepcopy(w3)
+    for name in ("intra_bw_poly", "inter_bw_poly", "zone_bw_poly"):
+        getattr(w4, name)[...] *= 2.0
+    o4 = Oracle(w4)
+    t4 = [o4.simulate(p).t_iter for p in plans]
+    assert all(b <= a for a, b in zip(t3, t4)) and any(b < a for a, b in zip(t3, t4))
+    assert any(abs(a - r.t_iter) > 1e-9 for a, r in zip(t3, ref))      # the curves do change the times
+
+
 # ---- enumeration -------------------------------------------------------------------------------
 
 def test_space_size_closed_form():
