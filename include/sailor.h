@@ -22,9 +22,11 @@
  *   b_i   = same over bwd, then + f_i when recomputation is on
  *   u_i   = same over upd[kind][g_i][tp_i]
  *   c_i   = alpha(link_i) + (double)p2p_bytes[mbs] * inv_bw(link_i), 0 for the last stage
+ *           (with a bandwidth polynomial: alpha + m / (((p3*m + p2)*m + p1)*m + p0))
  *   t_i   = (f_i + b_i) + 2 * c_i
  *   T_pp  = (t_0 + t_1 + ... left to right) + (double)N_b * max_i t_i
  *   sync_i= D == 1 ? 0 : ((2(D-1))/D * (double)gradbytes_i) * inv_bw_dp(i) + (2(D-1)) * alpha_dp(i)
+ *           (with a polynomial: "* inv_bw" becomes "/ bandwidth((double)gradbytes_i / D)")
  *   T_iter= (T_pp + max_i sync_i) + max_i u_i                          (Sec. 4.3, Sec. 4.2.2)
  *   rate  = sum_i (double)(D * tp_i) * (price_per_hour[z_i][g_i] / 3600)   left to right
  *   C_comm= sum over stage boundaries that cross zones of
@@ -120,6 +122,14 @@ typedef struct sailor_cluster {
     const double*   zone_alpha;      /* [zone][zone] link between zones (diagonal unused)    */
     const double*   zone_inv_bw;     /* [zone][zone]                                         */
     const double*   egress;          /* [zone][zone] USD per byte sent from row to column    */
+    /* Optional message-size-dependent bandwidth (Sec. 4.1: a polynomial fitted to measured
+     * bandwidth per link).  Four coefficients per link: bandwidth(m) = p0 + p1 m + p2 m^2 + p3 m^3
+     * bytes/s for a message of m bytes (Horner, binary64), all >= 0 and p0 > 0.  A link with a
+     * polynomial takes  alpha + m / bandwidth(m)  and ignores its inv_bw; the ring all-reduce
+     * evaluates the bandwidth at its chunk size gradbytes / D.  NULL = constant bandwidth. */
+    const double*   intra_bw_poly;   /* [zone][type][4] or NULL                               */
+    const double*   inter_bw_poly;   /* [zone][type][4] or NULL                               */
+    const double*   zone_bw_poly;    /* [zone][zone][4] or NULL                               */
 } sailor_cluster;
 
 /* One plan, stages run-length encoded: run r covers n_stages consecutive stages that share

@@ -42,7 +42,7 @@ class Cluster(C.Structure):
     _fields_ = [("n_types", C.c_uint32), ("n_zones", C.c_uint32), ("capacity", _u64p), ("reserved", _u64p),
                 ("gpus_per_node", _u32p), ("price_per_hour", _dp), ("intra_alpha", _dp), ("intra_inv_bw", _dp),
                 ("inter_alpha", _dp), ("inter_inv_bw", _dp), ("zone_alpha", _dp), ("zone_inv_bw", _dp),
-                ("egress", _dp)]
+                ("egress", _dp), ("intra_bw_poly", _dp), ("inter_bw_poly", _dp), ("zone_bw_poly", _dp)]
 
 
 class Run(C.Structure):
@@ -203,6 +203,9 @@ def sailor_create(w, device: int = 0, stream: int = 0) -> C.c_void_p:
     for name in ("price_per_hour", "intra_alpha", "intra_inv_bw", "inter_alpha", "inter_inv_bw", "zone_alpha",
                  "zone_inv_bw", "egress"):
         setattr(c, name, ptr(getattr(w, name), np.float64, _dp))
+    for name in ("intra_bw_poly", "inter_bw_poly", "zone_bw_poly"):       # optional: NULL when absent
+        if getattr(w, name, None) is not None:
+            setattr(c, name, ptr(getattr(w, name), np.float64, _dp))
     ctx = C.c_void_p()
     _check(load().sailor_create(C.byref(m), C.byref(p), C.byref(c), device, C.c_void_p(stream), C.byref(ctx)),
            "sailor_create")

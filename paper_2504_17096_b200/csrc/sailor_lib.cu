@@ -508,6 +508,16 @@ int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_c
         !finite_nonneg(c->inter_inv_bw, R) || !finite_nonneg(c->zone_alpha, (size_t)Z * Z) ||
         !finite_nonneg(c->zone_inv_bw, (size_t)Z * Z) || !finite_nonneg(c->egress, (size_t)Z * Z))
         return SAILOR_E_ARG;
+    {   // bandwidth polynomials: coefficients finite and >= 0, constant term > 0 (bandwidth stays positive)
+        const double* polys[3] = {c->intra_bw_poly, c->inter_bw_poly, c->zone_bw_poly};
+        const size_t counts[3] = {R, R, (size_t)Z * Z};
+        for (int q = 0; q < 3; ++q) {
+            if (!polys[q]) continue;
+            if (!finite_nonneg(polys[q], 4 * counts[q])) return SAILOR_E_ARG;
+            for (size_t j = 0; j < counts[q]; ++j)
+                if (!(polys[q][4 * j] > 0.0)) return SAILOR_E_ARG;
+        }
+    }
 
     sailor_ctx* ctx = new (std::nothrow) sailor_ctx();
     if (!ctx) return SAILOR_E_NOMEM;
@@ -550,6 +560,9 @@ int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_c
     h.off_zone_a = put(blob, c->zone_alpha, (size_t)Z * Z);
     h.off_zone_i = put(blob, c->zone_inv_bw, (size_t)Z * Z);
     h.off_egress = put(blob, c->egress, (size_t)Z * Z);
+    h.off_intra_p = c->intra_bw_poly ? put(blob, c->intra_bw_poly, 4 * R) : 0;
+    h.off_inter_p = c->inter_bw_poly ? put(blob, c->inter_bw_poly, 4 * R) : 0;
+    h.off_zone_p = c->zone_bw_poly ? put(blob, c->zone_bw_poly, 4 * (size_t)Z * Z) : 0;
     h.static_bytes = align16((uint32_t)blob.size());
     blob.resize(h.static_bytes);
     const size_t c4 = (size_t)2 * T * n_tp * n_mbs * h.chain_len, c3 = (size_t)2 * T * n_tp * h.chain_len;

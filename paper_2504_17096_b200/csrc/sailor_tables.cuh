@@ -37,6 +37,7 @@ struct alignas(16) TabHdr {
     uint32_t off_price_s;                         // f64 [digit]  price_per_hour / 3600
     uint32_t off_intra_a, off_intra_i, off_inter_a, off_inter_i;   // f64 [digit]
     uint32_t off_zone_a, off_zone_i, off_egress;  // f64 [zone][zone]
+    uint32_t off_intra_p, off_inter_p, off_zone_p; // f64 [..][4] bandwidth polynomials, 0 = none
     uint32_t static_bytes;                        // multiple of 16
     uint32_t off_chain_f, off_chain_b;            // f64 [start][type][tp][mbs][chain_len]
     uint32_t off_chain_u;                         // f64 [start][type][tp][chain_len]
@@ -51,6 +52,7 @@ struct TabView {
     const double *fwd, *bwd, *upd;
     const uint64_t *saved, *ckpt, *work, *p2p;
     const double *price_s, *intra_a, *intra_i, *inter_a, *inter_i, *zone_a, *zone_i, *egress;
+    const double *intra_p, *inter_p, *zone_p;      // nullptr when the link class has no polynomial
     const double *chain_f, *chain_b, *chain_u;
 
     __host__ __device__ void bind(const unsigned char* stat, const unsigned char* glob) {
@@ -70,6 +72,9 @@ struct TabView {
         zone_a = reinterpret_cast<const double*>(stat + h->off_zone_a);
         zone_i = reinterpret_cast<const double*>(stat + h->off_zone_i);
         egress = reinterpret_cast<const double*>(stat + h->off_egress);
+        intra_p = h->off_intra_p ? reinterpret_cast<const double*>(stat + h->off_intra_p) : nullptr;
+        inter_p = h->off_inter_p ? reinterpret_cast<const double*>(stat + h->off_inter_p) : nullptr;
+        zone_p = h->off_zone_p ? reinterpret_cast<const double*>(stat + h->off_zone_p) : nullptr;
         chain_f = reinterpret_cast<const double*>(glob + h->off_chain_f);
         chain_b = reinterpret_cast<const double*>(glob + h->off_chain_b);
         chain_u = reinterpret_cast<const double*>(glob + h->off_chain_u);
@@ -152,32 +157,50 @@ __device__ __forceinline__ StageMem stage_memory(const TabView& v, uint32_t tpi,
     return m;
 }
 
+// Bandwidth of a link for a message of m bytes from its fitted polynomial (Sec. 4.1), Horner form.
+__device__ __forceinline__ double poly_bw(const double* p, double m) {
+    return add_rn(mul_rn(add_rn(mul_rn(add_rn(mul_rn(p[3], m), p[2]), m), p[1]), m), p[0]);
+}
+// Time of a message of m bytes: alpha + m / bandwidth(m) with a polynomial, else alpha + m * inv_bw.
+__device__ __forceinline__ double link_time(double alpha, double inv_bw, const double* table, uint32_t idx, double m) {
+    if (table) return add_rn(alpha, m / poly_bw(table + 4 * idx, m));
+    return add_rn(alpha, mul_rn(m, inv_bw));
+}
+
 // Time of one message over the link between neighbouring stages (one direction).
 __device__ __forceinline__ double boundary_time(const TabView& v, uint32_t g, uint32_t z, uint32_t tp,
                                                 uint32_t g2, uint32_t z2, uint32_t tp2, uint32_t D, double msg) {
     const TabHdr* h = v.h;
-    if (z != z2) return add_rn(v.zone_a[z * h->Z + z2], mul_rn(msg, v.zone_i[z * h->Z + z2]));
+    if (z != z2) return link_time(v.zone_a[z * h->Z + z2], v.zone_i[z * h->Z + z2], v.zone_p, z * h->Z + z2, msg);
     const uint32_t d = z * h->T + g;
-    if (g == g2 && (uint64_t)D * (tp + tp2) <= h->gpn[g]) return add_rn(v.intra_a[d], mul_rn(msg, v.intra_i[d]));
+    if (g == g2 && (uint64_t)D * (tp + tp2) <= h->gpn[g]) return link_time(v.intra_a[d], v.intra_i[d], v.intra_p, d, msg);
     const uint32_t d2 = z * h->T + g2;
-    const double c1 = add_rn(v.inter_a[d], mul_rn(msg, v.inter_i[d]));
-    const double c2 = add_rn(v.inter_a[d2], mul_rn(msg, v.inter_i[d2]));
+    const double c1 = link_time(v.inter_a[d], v.inter_i[d], v.inter_p, d, msg);
+    const double c2 = link_time(v.inter_a[d2], v.inter_i[d2], v.inter_p, d2, msg);
     return dmax(c1, c2);
 }
 
-// Ring all-reduce of a stage's gradients among its D replicas (H5: inside one zone).
+// Ring all-reduce of `params` parameters' gradients (split over tp) among D replicas on the link of
+// digit d (H5: inside one zone): 2(D-1) messages of gradbytes / D.
+__device__ __forceinline__ double allreduce_time(const TabView& v, uint32_t g, uint32_t d, uint32_t tp, uint32_t D,
+                                                 uint64_t params, double steps, double coef) {
+    const TabHdr* h = v.h;
+    const bool intra = (uint64_t)D * tp <= h->gpn[g];
+    const double alpha = intra ? v.intra_a[d] : v.inter_a[d];
+    const double* poly = intra ? v.intra_p : v.inter_p;
+    const double gradbytes = (double)(ceil_div64(params, tp) * h->grad_bytes);
+    const double volume = mul_rn(coef, gradbytes);
+    double t;
+    if (poly) t = volume / poly_bw(poly + 4 * d, gradbytes / (double)D);
+    else t = mul_rn(volume, intra ? v.intra_i[d] : v.inter_i[d]);
+    return add_rn(t, mul_rn(steps, alpha));
+}
+
 __device__ __forceinline__ double sync_time(const TabView& v, uint32_t g, uint32_t z, uint32_t tp, uint32_t D,
                                             uint64_t params) {
     if (D <= 1) return 0.0;
-    const TabHdr* h = v.h;
-    const uint32_t d = z * h->T + g;
-    const bool intra = (uint64_t)D * tp <= h->gpn[g];
-    const double alpha = intra ? v.intra_a[d] : v.inter_a[d];
-    const double inv = intra ? v.intra_i[d] : v.inter_i[d];
-    const double gradbytes = (double)(ceil_div64(params, tp) * h->grad_bytes);
     const double steps = (double)(2 * (uint64_t)(D - 1));
-    const double coef = steps / (double)D;
-    return add_rn(mul_rn(mul_rn(coef, gradbytes), inv), mul_rn(steps, alpha));
+    return allreduce_time(v, g, z * v.h->T + g, tp, D, params, steps, steps / (double)D);
 }
 
 struct SimOut {
@@ -244,7 +267,7 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
 
     // current run
     uint32_t q = 0, left = 0, g = 0, z = 0, tpi = 0, tp = 1;
-    double gpu_rate = 0.0, c2_self = 0.0, dp_alpha = 0.0, dp_inv = 0.0;
+    double gpu_rate = 0.0, c2_self = 0.0;
     uint64_t cap = 0, resv = 0;
     // current layer composition
     uint32_t cur_nb = 0xffffffffu;
@@ -262,9 +285,6 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
             cap = h->capacity[g];
             resv = h->reserved[g];
             c2_self = mul_rn(2.0, boundary_time(v, g, z, tp, g, z, tp, D, msg));
-            const bool intra = (uint64_t)D * tp <= h->gpn[g];
-            dp_alpha = intra ? v.intra_a[d] : v.inter_a[d];
-            dp_inv = intra ? v.intra_i[d] : v.inter_i[d];
             refresh = true;
         }
         const uint32_t nb = base + (i < extra ? 1u : 0u);
@@ -279,11 +299,7 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
             const StageMem zero = stage_memory(v, tpi, mi, rc, nb, e, hd, 0);    // model + work
             m_keep = one.mem - zero.mem;
             m_fixed = zero.mem + resv;
-            sync = 0.0;
-            if (D > 1) {
-                const double gradbytes = (double)(ceil_div64(one.params, tp) * h->grad_bytes);
-                sync = add_rn(mul_rn(mul_rn(coef, gradbytes), dp_inv), mul_rn(steps, dp_alpha));
-            }
+            sync = D > 1 ? allreduce_time(v, g, z * h->T + g, tp, D, one.params, steps, coef) : 0.0;
             t_self = add_rn(fb, c2_self);
         }
         const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;

@@ -278,6 +278,33 @@ def test_plan_random_shapes_sweep(make_ctx):
                                                     f"P={p_values} k={k} [{lo},{hi}) {kw} flags={flags}")
 
 
+def test_bandwidth_polynomials_match_oracle(make_ctx):
+    """Message-size-dependent bandwidth (Sec. 4.1) in both entry points."""
+    for w in (W.with_bandwidth_polynomials(W.tiny(seed=41, n_types=3, n_zones=2), seed=1),
+              W.with_bandwidth_polynomials(W.config2(), seed=2)):
+        cx = make_ctx(w)
+        o = Oracle(w)
+        recs = W.random_plans(w, 4000, seed=6, hetero_tp=True)
+        assert_sim_equal(B.sailor_simulate(cx.ctx, B.pack_records(recs)), o.simulate_records(recs), w.name)
+        hits, counts, budget = o.plan(12)
+        res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w), 12)
+        assert_plan_equal(res, st, hits, counts, o, w.name)
+    # only some link classes carry a polynomial
+    w = W.with_bandwidth_polynomials(W.tiny(seed=42), seed=3)
+    w.inter_bw_poly = None
+    cx = make_ctx(w)
+    o = Oracle(w)
+    hits, counts = o.search(w.objective, 8)
+    res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w), 8)
+    assert_plan_equal(res, st, hits, counts, o, "partial")
+    # a polynomial whose constant term is not positive is rejected at create
+    w = W.with_bandwidth_polynomials(W.tiny(seed=43), seed=4)
+    w.zone_bw_poly[0, 1, 0] = 0.0
+    with pytest.raises(B.SailorError) as e:
+        B.sailor_create(w, 0, 0)
+    assert e.value.code == B.E_ARG
+
+
 def test_plan_constraints_and_empty_results(make_ctx):
     w = W.tiny(seed=8, n_types=2, n_zones=2)
     cx = make_ctx(w)
