@@ -282,7 +282,7 @@ def run_ours(args) -> None:
         peak = SM_COUNT * ISSUE_PER_SM * LANES * sm_max * 1e6 / 1e12
         achieved = ops * n / k_s / 1e12
         # counters of one plan_kernel launch on this workload, from the ncu capture summarised in
-        # profiles/plan_kernel_cfg5.md (valid for the kernel as committed with that file)
+        # profiles folder (valid for the kernel as committed with that summary)
         captured = NCU_PER_LAUNCH.get(w.name)
         issued = None
         if captured:
