@@ -157,6 +157,10 @@ struct SpaceCache {
     uint32_t* d_chunk_start = nullptr;
     uint64_t* d_flat_base = nullptr;
     size_t smem = 0;
+    // chunks of live prefixes only (see survey_kernel), for whole-space searches with pruning on
+    uint32_t* d_live_start = nullptr;      // [n_config + 1]
+    uint32_t live_chunks = 0;
+    unsigned long long closed[3] = {0, 0, 0};   // candidates counted in closed form: total, invalid, oom
 };
 
 struct OutBlock {                          // device -> pinned host
@@ -326,6 +330,31 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
     CU(ctx, cudaMemcpyAsync(sc.d_chunk_start, cs.data(), cs.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
     CU(ctx, cudaMemcpyAsync(sc.d_flat_base, fb.data(), fb.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, ctx->stream));
     CU(ctx, cudaStreamSynchronize(ctx->stream));       // the vectors are pageable
+    {   // survey the space once: live chunks per configuration and the closed-form class counts
+        cudaFree(sc.d_live_start);
+        sc.d_live_start = nullptr;
+        unsigned long long* d_closed = nullptr;
+        CU(ctx, cudaMalloc(&sc.d_live_start, (n_config + 1) * sizeof(uint32_t)));
+        CU(ctx, cudaMalloc(&d_closed, 3 * sizeof(unsigned long long)));
+        cudaError_t e = cudaMemsetAsync(d_closed, 0, 3 * sizeof(unsigned long long), ctx->stream);
+        const uint32_t grid = (uint32_t)(n_config < 2048 ? n_config : 2048);
+        if (e == cudaSuccess) {
+            survey_kernel<<<grid, SURVEY_THREADS, 0, ctx->stream>>>(ctx->d_blob, d, (uint32_t)n_config, sc.d_live_start, d_closed);
+            e = cudaGetLastError();
+        }
+        std::vector<uint32_t> live(n_config + 1, 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(live.data(), sc.d_live_start, n_config * sizeof(uint32_t), cudaMemcpyDeviceToHost, ctx->stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(sc.closed, d_closed, sizeof(sc.closed), cudaMemcpyDeviceToHost, ctx->stream);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+        cudaFree(d_closed);
+        if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_CUDA; }
+        uint64_t run = 0;                              // exclusive scan on the host: once per space
+        for (uint64_t j = 0; j < n_config; ++j) { const uint32_t v = live[j]; live[j] = (uint32_t)run; run += v; }
+        live[n_config] = (uint32_t)run;
+        sc.live_chunks = (uint32_t)run;
+        CU(ctx, cudaMemcpyAsync(sc.d_live_start, live.data(), (n_config + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
+        CU(ctx, cudaStreamSynchronize(ctx->stream));
+    }
     sc.key = *s;
     sc.desc = d;
     sc.n_config = (uint32_t)n_config;
@@ -377,7 +406,7 @@ int smem_optin(sailor_ctx* ctx, PlanKernel kern, uint32_t variant) {
 
 // Enqueue one search pass (clear, search, merge) on the context's stream.
 int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_ctrl, double min_rate,
-                 uint32_t flags, uint64_t lo, uint64_t hi, uint32_t k, double next_budget_factor,
+                 uint32_t flags, uint64_t lo, uint64_t hi, bool live, uint32_t k, double next_budget_factor,
                  uint32_t* n_launches) {
     SpaceCache& sc = ctx->space;
     // clear the counters; ctrl->budget (the previous pass may have written it) and the sticky error stay
@@ -403,9 +432,16 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
     pp.budget = budget;
     pp.min_rate = min_rate;
     uint32_t grid = 0;
-    if (hi > lo) {
+    if (live) {                    // whole space, pruning on: only chunks of live prefixes exist
+        pp.cfg_chunk_start = sc.d_live_start;
+        pp.live_mode = 1;
+        pp.chunk_lo = 0;
+        pp.chunk_hi = sc.live_chunks;
+    } else if (hi > lo) {
         pp.chunk_lo = chunk_of(ctx, lo);
         pp.chunk_hi = chunk_of(ctx, hi - 1) + 1;
+    }
+    if (pp.chunk_hi > pp.chunk_lo) {
         const uint32_t n_chunks = pp.chunk_hi - pp.chunk_lo;
         const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
         PlanKernel kern = pick_kernel(obj, constr);
@@ -632,6 +668,7 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->d_partial_n);
     cudaFree(ctx->space.d_chunk_start);
     cudaFree(ctx->space.d_flat_base);
+    cudaFree(ctx->space.d_live_start);
     cudaFree(ctx->d_stage);
     if (ctx->ev0) cudaEventDestroy(ctx->ev0);
     if (ctx->ev1) cudaEventDestroy(ctx->ev1);
@@ -732,14 +769,16 @@ int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objec
     uint32_t launches = 0;
     CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
     const bool two_pass = o->budget_factor_over_cheapest > 0.0;
+    // a whole-space search with pruning on walks only the prefixes the survey found live
+    const bool live = !(o->flags & SAILOR_FLAG_EVAL_ALL) && flat_lo == 0 && flat_hi == total;
     if (two_pass) {
         // cheapest feasible plan first; its merge step leaves factor * cost in ctrl->budget
-        rc = enqueue_pass(ctx, SAILOR_OBJ_MIN_COST, 0.0, false, 0.0, o->flags, flat_lo, flat_hi, 1,
+        rc = enqueue_pass(ctx, SAILOR_OBJ_MIN_COST, 0.0, false, 0.0, o->flags, flat_lo, flat_hi, live, 1,
                           o->budget_factor_over_cheapest, &launches);
         if (rc) return rc;
     }
     rc = enqueue_pass(ctx, o->kind, o->budget_usd_per_iter, two_pass, o->min_iters_per_s, o->flags, flat_lo,
-                      flat_hi, k, 0.0, &launches);
+                      flat_hi, live, k, 0.0, &launches);
     if (rc) return rc;
     CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
     CU(ctx, cudaMemcpyAsync(ctx->h_out->results, ctx->d_results, sizeof(sailor_result) * k, cudaMemcpyDeviceToHost,
@@ -751,9 +790,11 @@ int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objec
     *n_found = cr.n_found;
     memcpy(topk, ctx->h_out->results, sizeof(sailor_result) * cr.n_found);
     if (stats) {
-        stats->n_total = cr.stats[0];
-        stats->n_invalid = cr.stats[1];
-        stats->n_oom = cr.stats[2];
+        // in live mode the kernels count the evaluated candidates only; the rest is the survey's closed form
+        const SpaceCache& sc = ctx->space;
+        stats->n_total = live ? sc.closed[0] : cr.stats[0];
+        stats->n_invalid = live ? sc.closed[1] : cr.stats[1];
+        stats->n_oom = live ? sc.closed[2] : cr.stats[2];
         stats->n_over_avail = cr.stats[3];
         stats->n_over_constraint = cr.stats[4];
         stats->n_feasible = cr.stats[5];

@@ -58,6 +58,7 @@ struct PlanParams {
     uint32_t eval_all;
     uint32_t budget_from_ctrl;         // read the budget from ctrl->budget
     uint32_t p_max;                    // largest P of the space (sizes the stage tables)
+    uint32_t live_mode;                // cfg_chunk_start counts only chunks of prefixes made of usable digits
     double budget;                     // <= 0: none
     double min_rate;                   // <= 0: none
 };
@@ -153,7 +154,11 @@ struct CfgShared {
     // scalars (written by thread 0 / the build, read by all)
     Config cfg;
     uint32_t valid;              // gbs % (D*mbs) == 0 and heads % tp == 0
-    uint32_t dead;               // some segment has no digit that is valid and fits in memory
+    uint32_t packed;             // prefixes are enumerated over the usable digits of each segment only
+    uint32_t g_cnt[SAILOR_SEG_MAX];       // usable digits (valid type, fits in memory) per segment
+    uint32_t g_magic[SAILOR_SEG_MAX];     // floor(2^32 / g_cnt) + 1, for division by g_cnt
+    uint64_t live_items;         // product of g_cnt over the prefix segments
+    uint8_t good_list[SAILOR_SEG_MAX][R_MAX];   // the usable digits of each segment, ascending
     uint32_t seg_a[SAILOR_SEG_MAX + 1];   // first stage of each segment; seg_a[nseg] = P
     uint32_t need[SAILOR_SEG_MAX];        // GPUs a segment takes of its digit: D * tp * stages
     uint32_t n_run[SAILOR_SEG_MAX][N_RUNS];   // stages in each run (without a non-final segment's last stage)
@@ -231,6 +236,7 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
             for (uint32_t i = cs.seg_a[s]; i < t_end; ++i) cs.n_run[s][run_of(h, k.P, i)]++;
         }
         cs.n_items = ipow64(R, k.nseg - 1);
+        cs.packed = 0;                 // decided at the end of the build, and only for valid configurations
         cs.magic = (uint32_t)(0x100000000ull / R) + 1u;
         uint64_t inv = 0;
         for (uint32_t d = 0; d < R; ++d)
@@ -314,11 +320,21 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         for (uint32_t d = 0; d < R; ++d)
             if (cs.need[k.nseg - 1] <= a.availv[d]) m |= 1ull << d;
         cs.avail_last = m;
+        // usable digits per segment.  When the whole configuration is searched with pruning on, only
+        // prefixes made of usable digits are enumerated; everything else is counted in closed form.
         const uint64_t full = R == 64 ? ~0ull : ((1ull << R) - 1);
-        uint32_t dead = 0;
-        for (uint32_t s = 0; s < k.nseg; ++s)
-            if ((full & ~cs.invalid_mask & ~cs.oom_mask[s]) == 0) dead = 1;
-        cs.dead = dead;
+        uint64_t live = 1;
+        for (uint32_t s = 0; s < k.nseg; ++s) {
+            const uint64_t good = full & ~cs.invalid_mask & ~cs.oom_mask[s];
+            uint32_t n = 0;
+            for (uint32_t d = 0; d < R; ++d)
+                if ((good >> d) & 1) cs.good_list[s][n++] = (uint8_t)d;
+            cs.g_cnt[s] = n;
+            cs.g_magic[s] = n > 1 ? (uint32_t)(0x100000000ull / n) + 1u : 0u;
+            if (s + 1 < k.nseg) live *= n;
+        }
+        cs.live_items = live;
+        cs.packed = pp.live_mode;
     }
     __syncthreads();
 }
@@ -489,12 +505,28 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     uint32_t dg[NSEG > 1 ? NSEG - 1 : 1];
     {
         uint32_t x = active ? q : 0;
+        if (cs.packed) {                                   // mixed radix over the usable digits of each segment
 #pragma unroll
-        for (int s = NSEG - 2; s >= 0; --s) {
-            const uint32_t y = R == 1 ? x : __umulhi(x, cs.magic);     // x / R
-            dg[s] = x - y * R;
-            x = y;
+            for (int s = NSEG - 2; s >= 0; --s) {
+                const uint32_t n = cs.g_cnt[s];
+                const uint32_t y = n > 1 ? __umulhi(x, cs.g_magic[s]) : x;   // x / n
+                dg[s] = active ? cs.good_list[s][x - y * n] : 0u;
+                x = y;
+            }
+        } else {
+#pragma unroll
+            for (int s = NSEG - 2; s >= 0; --s) {
+                const uint32_t y = R == 1 ? x : __umulhi(x, cs.magic);     // x / R
+                dg[s] = x - y * R;
+                x = y;
+            }
         }
+    }
+    if (cs.packed) {                                       // the item's flat index follows from its digits
+        uint64_t pf = 0;
+#pragma unroll
+        for (int s = 0; s < NSEG - 1; ++s) pf = pf * R + dg[s];
+        item_flat = pp.cfg_flat_base[cs.cur_config] + pf * R;
     }
     // ---- status of the prefix: node validity, memory, availability (integer work only) ------------
     bool p_inv = false, p_oom = false, p_over = false;
@@ -532,9 +564,12 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     }
     // exactly one class per candidate: invalid, then oom, then over availability
     const uint32_t n_range = __popcll(range);
-    cnt.total += n_range;
-    if (p_inv) { cnt.invalid += n_range; ok = 0; }
+    if (cs.packed) {                                      // total, invalid and oom were added in closed form
+        if (p_over) { cnt.over_avail += __popcll(good_l); ok = 0; }
+        else cnt.over_avail += __popcll(good_l) - __popcll(ok);
+    } else if (p_inv) { cnt.total += n_range; cnt.invalid += n_range; ok = 0; }
     else {
+        cnt.total += n_range;
         cnt.invalid += n_range - __popcll(valid_l);
         if (p_oom) { cnt.oom += __popcll(valid_l); ok = 0; }
         else {
@@ -666,7 +701,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
                 build_config(pp, v, cs, a, c);
             }
             const uint32_t q = (ch - pp.cfg_chunk_start[c]) * PLAN_THREADS + tid;    // < R^3 + 256 <= 2^18 + 256
-            const bool active = q < cs.n_items;
+            const bool active = q < (cs.packed ? cs.live_items : cs.n_items);
             const uint64_t item_flat = pp.cfg_flat_base[c] + (uint64_t)q * R;
             if (!cs.valid) {
                 // every candidate of the configuration is invalid; count those in range
@@ -683,20 +718,6 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             const int fixed = (cs.n_run[3][0] == 0 && cs.n_run[3][1] == 0 && cs.n_run[3][3] == 1 && cs.n_run[3][2] <= 3)
                                   ? (int)cs.n_run[3][2] : -1;
 #define SAILOR_RUN(NS, NF) run_items<NS, OBJ, CONSTR, NF>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane)
-            if (cs.dead && !pp.eval_all && pp.cfg_flat_base[c] >= pp.flat_lo &&
-                pp.cfg_flat_base[c] + cs.n_items * R <= pp.flat_hi) {
-                // no candidate of this configuration can be valid and fit in memory: classes in closed
-                // form, added once (by whoever holds the configuration's first chunk), nothing evaluated
-                if (ch == pp.cfg_chunk_start[c] && tid == 0) {
-                    const uint64_t full = R == 64 ? ~0ull : ((1ull << R) - 1);
-                    const uint64_t n_all = cs.n_items * R;
-                    const uint64_t n_valid = ipow64(__popcll(full & ~cs.invalid_mask), cs.cfg.nseg);
-                    atomicAdd(&cs.stat[0], (unsigned long long)n_all);
-                    atomicAdd(&cs.stat[1], (unsigned long long)(n_all - n_valid));
-                    atomicAdd(&cs.stat[2], (unsigned long long)n_valid);
-                }
-                continue;
-            }
             switch (cs.cfg.nseg) {
                 case 1: SAILOR_RUN(1, -1); break;
                 case 2: SAILOR_RUN(2, -1); break;
@@ -746,6 +767,79 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             pp.partial[(size_t)blockIdx.x * SAILOR_K_MAX + lane].flat = top.flat;
         }
         if (lane == 0) pp.partial_n[blockIdx.x] = n;
+    }
+}
+
+// Which prefixes can matter at all?  Per configuration: the digits of every segment whose type can
+// host tp and whose stages fit in memory (H2: independent of availability), hence the number of
+// chunks of prefixes made of such digits only, and -- in closed form -- how many candidates are
+// invalid or out of memory.  Runs once per (context, space); the plan search then enumerates only
+// the live prefixes.  One block per configuration at a time.
+constexpr int SURVEY_THREADS = 128;
+
+__global__ void __launch_bounds__(SURVEY_THREADS)
+survey_kernel(const unsigned char* __restrict__ blob, SpaceDesc sp, uint32_t n_config, uint32_t* __restrict__ live_chunks,
+              unsigned long long* __restrict__ closed /* total, invalid, oom */) {
+    __shared__ uint32_t oom_stage[SAILOR_P_MAX];
+    __shared__ Config k;
+    __shared__ uint32_t valid;
+    __shared__ uint64_t n_b;
+    TabView v;
+    v.bind(blob, blob);
+    const TabHdr* h = v.h;
+    const uint32_t T = h->T, R = h->R, tid = threadIdx.x;
+    for (uint32_t c = blockIdx.x; c < n_config; c += gridDim.x) {
+        __syncthreads();
+        if (tid == 0) {
+            k = config_of(sp, c);
+            const uint32_t tp = h->tp_values[k.tpi];
+            const uint64_t dm = (uint64_t)k.D * h->mbs_values[k.mi];
+            valid = (k.D >= 1 && h->gbs % dm == 0 && h->heads % tp == 0) ? 1u : 0u;
+            n_b = k.D >= 1 ? h->gbs / dm : 0;
+        }
+        for (uint32_t i = tid; i < SAILOR_P_MAX; i += SURVEY_THREADS) oom_stage[i] = 0;
+        __syncthreads();
+        const uint32_t P = k.P;
+        if (valid) {
+            const uint32_t base = h->n_blocks / P, extra = h->n_blocks % P;
+            for (uint32_t x = tid; x < P * T; x += SURVEY_THREADS) {
+                const uint32_t i = x / T, g = x % T;
+                const uint32_t nb = base + (i < extra ? 1u : 0u);
+                const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
+                const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
+                const StageMem sm = stage_memory(v, k.tpi, k.mi, k.rc, nb, e, hd, inflight);
+                if (sm.mem + h->reserved[g] > h->capacity[g]) atomicOr(&oom_stage[i], 1u << g);
+            }
+        }
+        __syncthreads();
+        if (tid == 0) {
+            const uint64_t n_all = ipow64(R, k.nseg);
+            uint32_t chunks = 0;
+            if (!valid) {
+                atomicAdd(&closed[0], (unsigned long long)n_all);
+                atomicAdd(&closed[1], (unsigned long long)n_all);
+            } else {
+                const uint32_t tp = h->tp_values[k.tpi];
+                uint32_t type_ok = 0;                      // types whose nodes can host tp
+                for (uint32_t g = 0; g < T; ++g)
+                    if (tp <= h->gpn[g]) type_ok |= 1u << g;
+                const uint64_t n_valid = ipow64((uint64_t)__popc(type_ok) * h->Z, k.nseg);
+                uint64_t live = 1, fit = 1;
+                for (uint32_t s = 0; s < k.nseg; ++s) {
+                    const uint32_t sa = (s * P + k.nseg - 1) / k.nseg, se = ((s + 1) * P + k.nseg - 1) / k.nseg;
+                    uint32_t oom = 0;
+                    for (uint32_t i = sa; i < se; ++i) oom |= oom_stage[i];
+                    const uint64_t g_cnt = (uint64_t)__popc(type_ok & ~oom) * h->Z;     // usable digits of the segment
+                    fit *= g_cnt;
+                    if (s + 1 < k.nseg) live *= g_cnt;
+                }
+                if (fit) chunks = (uint32_t)((live + PLAN_THREADS - 1) / PLAN_THREADS);
+                atomicAdd(&closed[0], (unsigned long long)n_all);
+                atomicAdd(&closed[1], (unsigned long long)(n_all - n_valid));
+                atomicAdd(&closed[2], (unsigned long long)(n_valid - fit));
+            }
+            live_chunks[c] = chunks;
+        }
     }
 }
 
