@@ -305,6 +305,27 @@ def test_bandwidth_polynomials_match_oracle(make_ctx):
     assert e.value.code == B.E_ARG
 
 
+def test_plan_more_stages_than_blocks_and_empty_ranges(make_ctx):
+    """Pipelines deeper than the layer count (stages without a block) and empty flat ranges."""
+    w = W.tiny(seed=51, n_types=2, n_zones=2, L=2, p_values=[2, 3, 4, 6])
+    cx = make_ctx(w)
+    o = Oracle(w)
+    hits, counts = o.search(w.objective, 10)
+    assert counts["n_feasible"] > 0
+    for flags in (0, B.FLAG_EVAL_ALL):
+        res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=flags), 10)
+        assert_plan_equal(res, st, hits, counts, o, f"flags={flags}")
+    recs = W.random_plans(w, 2000, seed=8, hetero_tp=True)
+    recs["P"][:50] = 6                                   # force some deep ones (keep run lengths consistent)
+    recs["n_runs"][:50] = 1
+    recs["n_stages"][:50, 0] = 6
+    assert_sim_equal(B.sailor_simulate(cx.ctx, B.pack_records(recs)), o.simulate_records(recs), "deep-short")
+    n = o.space_size()
+    for lo, hi in ((5, 5), (n, n + 10), (n + 3, n + 1), (7, 3)):
+        res, st = B.sailor_plan_range(cx.ctx, cx.space, B.make_objective(w), lo, hi, 4)
+        assert res == [] and st.n_total == 0 and st.n_feasible == 0
+
+
 def test_plan_constraints_and_empty_results(make_ctx):
     w = W.tiny(seed=8, n_types=2, n_zones=2)
     cx = make_ctx(w)
