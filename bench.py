@@ -205,11 +205,20 @@ def run_ours(args) -> None:
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    # one rank per GPU over NCCL; for a dry run of the multi-rank control flow on fewer GPUs than
+    # ranks (the searches are independent, no rank waits for another rank's kernel) the environment
+    # may select the gloo backend and let ranks share devices
+    backend = os.environ.get("SAILOR_BENCH_BACKEND", "nccl")
+    if os.environ.get("SAILOR_BENCH_SHARE_GPUS"):
+        local %= torch.cuda.device_count()
     torch.cuda.set_device(local)
     dist = None
     if world > 1:
         import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
 
     w = workload_by_name(args.workload, args.only_p)
     # independent problems: every rank searches the whole space for its own availability snapshot
@@ -263,7 +272,7 @@ def run_ours(args) -> None:
     h2d = int(avail.size * 2)
     d2h = int(K_TOP * 120 + 80)
 
-    times = torch.tensor([dev_s, e2e_s], dtype=torch.float64, device="cuda")
+    times = torch.tensor([dev_s, e2e_s], dtype=torch.float64, device="cuda" if backend == "nccl" else "cpu")
     if dist is not None:
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
     dev_s, e2e_s = (float(x) for x in times.cpu())
