@@ -10,7 +10,8 @@
  *
  * Pins (see tests, all run without a GPU): three hand-computed two-stage cases and one
  * hand-computed three-stage case with embedding/head layers, recomputation, alpha > 0 and
- * mixed tensor parallelism; the homogeneous closed form (P + N_b) * t; monotonicity and
+ * mixed tensor parallelism; two hand-computed cases with fitted bandwidth polynomials (boundary
+ * link and all-reduce); the homogeneous closed form (P + N_b) * t; monotonicity and
  * scaling invariants; an independent nested-loop enumeration and brute-force minimum on
  * tiny clusters.
  * Parity unpinned: the absolute realism of the outputs against real clusters (Sec. 5.1
