@@ -163,6 +163,7 @@ struct CfgShared {
     uint32_t need[SAILOR_SEG_MAX];        // GPUs a segment takes of its digit: D * tp * stages
     uint32_t n_run[SAILOR_SEG_MAX][N_RUNS];   // stages in each run (without a non-final segment's last stage)
     uint32_t magic;              // floor(2^32 / R) + 1: x / R == umulhi(x, magic) for x < 2^26
+    double ar_steps, ar_coef;    // 2(D-1) and 2(D-1)/D of the ring all-reduce
     uint64_t n_b;
     uint64_t n_items;            // R^(nseg-1)
     uint64_t invalid_mask;       // digit d: tp > gpus_per_node[type(d)]
@@ -210,10 +211,10 @@ __device__ __forceinline__ void carve(unsigned char* dyn, uint32_t static_bytes,
 }
 
 // Run of stage i: 0 = stage 0 with the embedding, 1 = one extra block, 2 = plain, 3 = final stage.
-__device__ __forceinline__ uint32_t run_of(const TabHdr* h, uint32_t P, uint32_t i) {
+__device__ __forceinline__ uint32_t run_of(const TabHdr* h, uint32_t P, uint32_t extra, uint32_t i) {
     if (i == P - 1) return 3;
     if (i == 0 && h->has_embed) return 0;
-    return i < h->n_blocks % P ? 1 : 2;
+    return i < extra ? 1 : 2;                              // extra = n_blocks % P
 }
 
 // Build the tables of configuration `c`.  Called by the whole block; ends synchronised.
@@ -228,19 +229,23 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         cs.valid = (k.D >= 1 && h->gbs % dm == 0 && h->heads % tp == 0) ? 1u : 0u;
         cs.n_b = k.D >= 1 ? h->gbs / dm : 0;
         for (uint32_t s = 0; s <= k.nseg; ++s) cs.seg_a[s] = (s * k.P + k.nseg - 1) / k.nseg;
+        const uint32_t extra0 = h->n_blocks % k.P;
+        cs.ar_steps = (double)(2 * (uint64_t)(k.D > 0 ? k.D - 1 : 0));     // ring all-reduce: 2(D-1) messages
+        cs.ar_coef = k.D > 0 ? cs.ar_steps / (double)k.D : 0.0;
         for (uint32_t s = 0; s < k.nseg; ++s) {
             cs.need[s] = k.D * tp * (cs.seg_a[s + 1] - cs.seg_a[s]);
             cs.oom_mask[s] = 0;
             for (int r = 0; r < N_RUNS; ++r) cs.n_run[s][r] = 0;
             const uint32_t t_end = (s + 1 < k.nseg) ? cs.seg_a[s + 1] - 1 : cs.seg_a[s + 1];
-            for (uint32_t i = cs.seg_a[s]; i < t_end; ++i) cs.n_run[s][run_of(h, k.P, i)]++;
+            for (uint32_t i = cs.seg_a[s]; i < t_end; ++i) cs.n_run[s][run_of(h, k.P, extra0, i)]++;
         }
         cs.n_items = ipow64(R, k.nseg - 1);
         cs.packed = 0;                 // decided at the end of the build, and only for valid configurations
         cs.magic = (uint32_t)(0x100000000ull / R) + 1u;
         uint64_t inv = 0;
-        for (uint32_t d = 0; d < R; ++d)
-            if (tp > h->gpn[d % T]) inv |= 1ull << d;
+        for (uint32_t g = 0; g < T; ++g)
+            if (tp > h->gpn[g])
+                for (uint32_t z = 0; z < Z; ++z) inv |= 1ull << (z * T + g);
         cs.invalid_mask = inv;
         cs.cur_config = c;
     }
@@ -300,10 +305,10 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
             if (i < t_end) {
                 const double fbi = a.fb[i * T + g];
                 const double t = (i + 1 < P) ? add_rn(fbi, c2self) : fbi;
-                r.v[run_of(h, P, i)] = t;
+                r.v[run_of(h, P, extra, i)] = t;
                 tm = dmax(tm, t);
             }
-            sy = dmax(sy, sync_time(v, g, z, tp, k.D, cs.params[i]));
+            if (k.D > 1) sy = dmax(sy, allreduce_time(v, g, d, tp, k.D, cs.params[i], cs.ar_steps, cs.ar_coef));
             up = dmax(up, a.uu[i * T + g]);
             oom |= (cs.oom_stage[i] >> g) & 1u;
         }
@@ -324,7 +329,7 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         // prefixes made of usable digits are enumerated; everything else is counted in closed form.
         const uint64_t full = R == 64 ? ~0ull : ((1ull << R) - 1);
         uint64_t live = 1;
-        for (uint32_t s = 0; s < k.nseg; ++s) {
+        for (uint32_t s = 0; pp.live_mode && s < k.nseg; ++s) {
             const uint64_t good = full & ~cs.invalid_mask & ~cs.oom_mask[s];
             uint32_t n = 0;
             for (uint32_t d = 0; d < R; ++d)
