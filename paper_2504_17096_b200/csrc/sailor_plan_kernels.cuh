@@ -120,6 +120,24 @@ struct WarpTopK {
         thr_flat = __shfl_sync(FULL, flat, k - 1);
         return true;
     }
+    // Merge another ascending list of 32 (lane j passes its j-th element; empty slots are
+    // (+inf, ~0)) into this one, keeping the 32 smallest of the union: min(a[j], b[31-j]) is a
+    // bitonic sequence holding exactly those, and five compare-exchange stages sort it.
+    __device__ __forceinline__ void merge_sorted(double bs, uint64_t bf, uint32_t k, uint32_t lane) {
+        const double rs = __shfl_sync(FULL, bs, 31 - lane);
+        const uint64_t rf = __shfl_sync(FULL, bf, 31 - lane);
+        if (rs < score || (rs == score && rf < flat)) { score = rs; flat = rf; }
+#pragma unroll
+        for (int stride = 16; stride; stride >>= 1) {
+            const double os = __shfl_xor_sync(FULL, score, stride);
+            const uint64_t of = __shfl_xor_sync(FULL, flat, stride);
+            const bool other_less = os < score || (os == score && of < flat);
+            const bool upper = lane & stride;
+            if (other_less != upper) { score = os; flat = of; }     // lower lane keeps the smaller, upper the larger
+        }
+        thr_score = __shfl_sync(FULL, score, k - 1);
+        thr_flat = __shfl_sync(FULL, flat, k - 1);
+    }
     // Offer per-lane candidates: `want` marks lanes whose candidate may qualify.
     __device__ __forceinline__ void offer(bool want, double s, uint64_t f, uint32_t k, uint32_t lane) {
         unsigned m = __ballot_sync(FULL, want);
@@ -760,12 +778,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
     __syncthreads();
     if (tid < 6 && cs.stat[tid]) atomicAdd(&pp.ctrl->stats[tid], cs.stat[tid]);
     if (warp == 0) {
-        for (uint32_t w = 1; w < PLAN_WARPS; ++w)
-            for (uint32_t j = 0; j < pp.k; ++j) {
-                const Hit hj = s_hits[w][j];
-                if (hj.flat == ~0ull) break;             // lists are sorted; the rest is empty
-                if (!top.insert(hj.score, hj.flat, pp.k, lane)) break;   // ... and the rest is no better
-            }
+        for (uint32_t w = 1; w < PLAN_WARPS; ++w) {
+            if (s_hits[w][0].flat == ~0ull) continue;    // an empty list
+            top.merge_sorted(s_hits[w][lane].score, s_hits[w][lane].flat, pp.k, lane);
+        }
         const uint32_t n = __popc(__ballot_sync(FULL, top.flat != ~0ull && lane < pp.k));
         if (lane < pp.k) {
             pp.partial[(size_t)blockIdx.x * SAILOR_K_MAX + lane].score = top.score;
@@ -883,22 +899,16 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const __grid_const
         const uint32_t n = mp.partial_n[b];
         Hit mine = {make_inf(), ~0ull};                  // one coalesced read of the block's list
         if (lane < n) mine = mp.partial[(size_t)b * SAILOR_K_MAX + lane];
-        for (uint32_t j = 0; j < n; ++j) {               // the list is sorted: stop at the first reject
-            const double sj = __shfl_sync(FULL, mine.score, j);
-            const uint64_t fj = __shfl_sync(FULL, mine.flat, j);
-            if (!top.insert(sj, fj, mp.k, lane)) break;
-        }
+        if (n) top.merge_sorted(mine.score, mine.flat, mp.k, lane);
     }
     s_hits[warp][lane].score = top.score;
     s_hits[warp][lane].flat = top.flat;
     __syncthreads();
     if (warp == 0) {
-        for (uint32_t w = 1; w < nw; ++w)
-            for (uint32_t j = 0; j < mp.k; ++j) {
-                const Hit hj = s_hits[w][j];
-                if (hj.flat == ~0ull) break;
-                if (!top.insert(hj.score, hj.flat, mp.k, lane)) break;
-            }
+        for (uint32_t w = 1; w < nw; ++w) {
+            if (s_hits[w][0].flat == ~0ull) continue;
+            top.merge_sorted(s_hits[w][lane].score, s_hits[w][lane].flat, mp.k, lane);
+        }
         const bool have = lane < mp.k && top.flat != ~0ull;
         const uint32_t n = __popc(__ballot_sync(FULL, have));
         s_hits[0][lane].score = top.score;
