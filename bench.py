@@ -199,6 +199,9 @@ def aux_measurements(B, torch, dev) -> dict:
 def run_ours(args) -> None:
     import torch
     from paper_2504_17096_b200 import binding as B
+    from paper_2504_17096_b200 import build as cuda_build
+    if cuda_build.is_stale() and int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        cuda_build.build()                       # compile the CUDA library if it is missing or out of date
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
