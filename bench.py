@@ -200,8 +200,13 @@ def run_ours(args) -> None:
     import torch
     from paper_2504_17096_b200 import binding as B
     from paper_2504_17096_b200 import build as cuda_build
-    if cuda_build.is_stale() and int(os.environ.get("LOCAL_RANK", "0")) == 0:
-        cuda_build.build()                       # compile the CUDA library if it is missing or out of date
+    if cuda_build.is_stale():                    # compile the CUDA library if it is missing or out of date
+        if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+            cuda_build.build()
+        else:                                    # one rank per node builds, the others wait for the file
+            deadline = time.time() + 300
+            while cuda_build.is_stale() and time.time() < deadline:
+                time.sleep(0.5)
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
