@@ -151,29 +151,38 @@ def aux_measurements(B, torch, dev) -> dict:
     ctx = B.sailor_create(w, dev, torch.cuda.current_stream().cuda_stream)
     try:
         B.sailor_set_availability(ctx, w.avail)
-        base = B.pack_records(W.random_plans(w, 1 << 15, seed=11, hetero_tp=True))
-        reps = 128
-        n = base.size * reps                                           # 4.2e6 records, 302 MB: larger than L2
-        d_plans = torch.from_numpy(base.view(np.uint8).reshape(-1, 72).copy()).cuda().repeat(reps, 1).contiguous()
-        t = torch.empty(n, dtype=torch.float64, device="cuda")
-        c = torch.empty(n, dtype=torch.float64, device="cuda")
-        m = torch.empty(n, dtype=torch.int64, device="cuda")
-        st = torch.empty(n, dtype=torch.int32, device="cuda")
-        call = lambda: B.sailor_simulate_device(ctx, d_plans.data_ptr(), n, t.data_ptr(), m.data_ptr(), c.data_ptr(),
-                                                st.data_ptr())
-        for _ in range(3):
-            call()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(5):
-            call()
-        e1.record()
-        torch.cuda.synchronize()
-        ms = e0.elapsed_time(e1) / 5
-        mean_p = float(base["P"].astype(np.float64).mean())
-        out["simulate_cfg5_records"] = {"plans": n, "mean_stages": mean_p, "kernel_ms": ms, "plans_per_s": n / ms * 1e3,
-                                        "hbm_gb_per_s": n * 100 / ms / 1e6}
-        del d_plans, t, c, m, st
+        sp5 = B.make_space(w)
+        n5 = B.sailor_space_size(ctx, sp5)
+        rng = W.SplitMix64(12)
+        enumerated = np.zeros(1 << 15, dtype=B.REC_DTYPE)              # records of the search space itself
+        for j in range(enumerated.size):
+            rec = B.sailor_decode(ctx, sp5, rng.next_u64() % n5)
+            enumerated[j] = np.frombuffer(bytes(rec), dtype=B.REC_DTYPE)[0]
+        batches = {"simulate_cfg5_records": B.pack_records(W.random_plans(w, 1 << 15, seed=11, hetero_tp=True)),
+                   "simulate_cfg5_enumerated": enumerated}
+        for key, base in batches.items():
+            reps = 128
+            n = base.size * reps                                       # 4.2e6 records, 302 MB: larger than L2
+            d_plans = torch.from_numpy(base.view(np.uint8).reshape(-1, 72).copy()).cuda().repeat(reps, 1).contiguous()
+            t = torch.empty(n, dtype=torch.float64, device="cuda")
+            c = torch.empty(n, dtype=torch.float64, device="cuda")
+            m = torch.empty(n, dtype=torch.int64, device="cuda")
+            st = torch.empty(n, dtype=torch.int32, device="cuda")
+            call = lambda: B.sailor_simulate_device(ctx, d_plans.data_ptr(), n, t.data_ptr(), m.data_ptr(),
+                                                    c.data_ptr(), st.data_ptr())
+            for _ in range(3):
+                call()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(5):
+                call()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / 5
+            mean_p = float(base["P"].astype(np.float64).mean())
+            out[key] = {"plans": n, "mean_stages": mean_p, "kernel_ms": ms, "plans_per_s": n / ms * 1e3,
+                        "hbm_gb_per_s": n * 100 / ms / 1e6}
+            del d_plans, t, c, m, st
     finally:
         B.sailor_destroy(ctx)
     w = W.config4()
