@@ -239,33 +239,50 @@ __device__ __forceinline__ uint32_t run_of(const TabHdr* h, uint32_t P, uint32_t
 __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& cs, CfgArrays& a, uint32_t c) {
     const TabHdr* h = v.h;
     const uint32_t T = h->T, Z = h->Z, R = h->R, tid = threadIdx.x;
-    if (tid == 0) {
-        Config k = config_of(pp.sp, c);
-        cs.cfg = k;
-        const uint32_t tp = h->tp_values[k.tpi];
-        const uint64_t dm = (uint64_t)k.D * h->mbs_values[k.mi];
-        cs.valid = (k.D >= 1 && h->gbs % dm == 0 && h->heads % tp == 0) ? 1u : 0u;
-        cs.n_b = k.D >= 1 ? h->gbs / dm : 0;
-        for (uint32_t s = 0; s <= k.nseg; ++s) cs.seg_a[s] = (s * k.P + k.nseg - 1) / k.nseg;
-        const uint32_t extra0 = h->n_blocks % k.P;
-        cs.ar_steps = (double)(2 * (uint64_t)(k.D > 0 ? k.D - 1 : 0));     // ring all-reduce: 2(D-1) messages
-        cs.ar_coef = k.D > 0 ? cs.ar_steps / (double)k.D : 0.0;
-        for (uint32_t s = 0; s < k.nseg; ++s) {
-            cs.need[s] = k.D * tp * (cs.seg_a[s + 1] - cs.seg_a[s]);
-            cs.oom_mask[s] = 0;
-            for (int r = 0; r < N_RUNS; ++r) cs.n_run[s][r] = 0;
-            const uint32_t t_end = (s + 1 < k.nseg) ? cs.seg_a[s + 1] - 1 : cs.seg_a[s + 1];
-            for (uint32_t i = cs.seg_a[s]; i < t_end; ++i) cs.n_run[s][run_of(h, k.P, extra0, i)]++;
+    if (tid < 32) {                    // the first warp sets the configuration up, one segment per lane
+        Config k;
+        uint32_t valid = 0;
+        if (tid == 0) {
+            k = config_of(pp.sp, c);
+            cs.cfg = k;
+            const uint32_t tp0 = h->tp_values[k.tpi];
+            const uint64_t dm = (uint64_t)k.D * h->mbs_values[k.mi];
+            valid = (k.D >= 1 && h->gbs % dm == 0 && h->heads % tp0 == 0) ? 1u : 0u;
+            cs.valid = valid;
+            cs.n_b = k.D >= 1 ? h->gbs / dm : 0;
+            cs.ar_steps = (double)(2 * (uint64_t)(k.D > 0 ? k.D - 1 : 0));     // ring all-reduce: 2(D-1) messages
+            cs.ar_coef = k.D > 0 ? cs.ar_steps / (double)k.D : 0.0;
+            cs.n_items = ipow64(R, k.nseg - 1);
+            cs.packed = 0;             // decided at the end of the build, and only for valid configurations
+            cs.cur_config = c;
         }
-        cs.n_items = ipow64(R, k.nseg - 1);
-        cs.packed = 0;                 // decided at the end of the build, and only for valid configurations
-        cs.magic = (uint32_t)(0x100000000ull / R) + 1u;
-        uint64_t inv = 0;
-        for (uint32_t g = 0; g < T; ++g)
-            if (tp > h->gpn[g])
-                for (uint32_t z = 0; z < Z; ++z) inv |= 1ull << (z * T + g);
-        cs.invalid_mask = inv;
-        cs.cur_config = c;
+        const uint32_t P = __shfl_sync(FULL, k.P, 0), nseg = __shfl_sync(FULL, k.nseg, 0);
+        const uint32_t D = __shfl_sync(FULL, k.D, 0), tp = h->tp_values[__shfl_sync(FULL, k.tpi, 0)];
+        if (tid <= nseg) cs.seg_a[tid] = (tid * P + nseg - 1) / nseg;
+        if (tid < nseg) {              // stages [lo, hi) of segment `tid`, counted per run in closed form
+            const uint32_t lo = (tid * P + nseg - 1) / nseg, end = ((tid + 1) * P + nseg - 1) / nseg;
+            const uint32_t extra = h->n_blocks % P;
+            cs.need[tid] = D * tp * (end - lo);
+            cs.oom_mask[tid] = 0;
+            uint32_t hi = (tid + 1 < nseg) ? end - 1 : end;      // a non-final segment's last stage is kept apart
+            const uint32_t c3 = (hi == P && hi > lo) ? 1u : 0u;   // the final stage
+            hi -= c3;
+            const uint32_t c0 = (lo == 0 && h->has_embed && hi > lo) ? 1u : 0u;
+            const uint32_t lo1 = lo + c0;
+            const uint32_t top = hi < extra ? hi : extra;
+            const uint32_t c1 = top > lo1 ? top - lo1 : 0u;
+            cs.n_run[tid][0] = c0;
+            cs.n_run[tid][1] = c1;
+            cs.n_run[tid][2] = hi > lo1 ? (hi - lo1) - c1 : 0u;
+            cs.n_run[tid][3] = c3;
+        }
+        uint32_t inv_lo = 0, inv_hi = 0;                          // digits whose type cannot host tp
+        {
+            const uint32_t d0 = tid, d1 = tid + 32;
+            inv_lo = __ballot_sync(FULL, d0 < R && tp > h->gpn[d0 % T]);
+            inv_hi = __ballot_sync(FULL, d1 < R && tp > h->gpn[d1 % T]);
+        }
+        if (tid == 0) cs.invalid_mask = ((uint64_t)inv_hi << 32) | inv_lo;
     }
     for (uint32_t i = tid; i < SAILOR_P_MAX; i += PLAN_THREADS) cs.oom_stage[i] = 0;
     __syncthreads();
@@ -338,26 +355,33 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         if (oom) atomicOr(reinterpret_cast<unsigned long long*>(&cs.oom_mask[s]), 1ull << d);
     }
     __syncthreads();                   // the memory masks are complete
-    if (tid == 0) {
-        uint64_t m = 0;
-        for (uint32_t d = 0; d < R; ++d)
-            if (cs.need[k.nseg - 1] <= a.availv[d]) m |= 1ull << d;
-        cs.avail_last = m;
-        // usable digits per segment.  When the whole configuration is searched with pruning on, only
-        // prefixes made of usable digits are enumerated; everything else is counted in closed form.
-        const uint64_t full = R == 64 ? ~0ull : ((1ull << R) - 1);
-        uint64_t live = 1;
-        for (uint32_t s = 0; pp.live_mode && s < k.nseg; ++s) {
-            const uint64_t good = full & ~cs.invalid_mask & ~cs.oom_mask[s];
-            uint32_t n = 0;
-            for (uint32_t d = 0; d < R; ++d)
-                if ((good >> d) & 1) cs.good_list[s][n++] = (uint8_t)d;
-            cs.g_cnt[s] = n;
-            cs.g_magic[s] = n > 1 ? (uint32_t)(0x100000000ull / n) + 1u : 0u;
-            if (s + 1 < k.nseg) live *= n;
+    if (tid < 32) {
+        const uint32_t last = k.nseg - 1;
+        const uint32_t need_last = cs.need[last];
+        const uint32_t a_lo = __ballot_sync(FULL, tid < R && need_last <= a.availv[tid < R ? tid : 0]);
+        const uint32_t a_hi = __ballot_sync(FULL, tid + 32 < R && need_last <= a.availv[tid + 32 < R ? tid + 32 : 0]);
+        if (tid == 0) cs.avail_last = ((uint64_t)a_hi << 32) | a_lo;
+        if (pp.live_mode) {
+            // usable digits per segment (valid type, fits in memory): only prefixes made of them are
+            // enumerated; lane d places digit d (and d + 32) at its rank among the set bits
+            const uint64_t full = R == 64 ? ~0ull : ((1ull << R) - 1);
+            uint64_t live = 1;
+            for (uint32_t sgm = 0; sgm < k.nseg; ++sgm) {
+                const uint64_t good = full & ~cs.invalid_mask & ~cs.oom_mask[sgm];
+                const uint32_t g_lo = (uint32_t)good, g_hi = (uint32_t)(good >> 32);
+                const uint32_t below = (1u << tid) - 1u;
+                if ((g_lo >> tid) & 1u) cs.good_list[sgm][__popc(g_lo & below)] = (uint8_t)tid;
+                if ((g_hi >> tid) & 1u) cs.good_list[sgm][__popc(g_lo) + __popc(g_hi & below)] = (uint8_t)(tid + 32);
+                const uint32_t n = __popcll(good);
+                if (tid == 0) {
+                    cs.g_cnt[sgm] = n;
+                    cs.g_magic[sgm] = n > 1 ? (uint32_t)(0x100000000ull / n) + 1u : 0u;
+                }
+                if (sgm + 1 < k.nseg) live *= n;
+            }
+            if (tid == 0) cs.live_items = live;
         }
-        cs.live_items = live;
-        cs.packed = pp.live_mode;
+        if (tid == 0) cs.packed = pp.live_mode;
     }
     __syncthreads();
 }
@@ -680,7 +704,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
     CfgArrays a;
     carve(dyn, static_bytes, pp.p_max, T, Z, a);
 
-    if (tid == 0) cs.cur_config = 0xffffffffu;
+    if (tid == 0) {
+        cs.cur_config = 0xffffffffu;
+        cs.magic = (uint32_t)(0x100000000ull / (gh->R ? gh->R : 1u)) + 1u;      // for x / R, see CfgShared
+    }
     if (tid < 6) cs.stat[tid] = 0;
     // the padding digit of the tables is read (and masked out) by the two-digit steps: keep it finite
     for (uint32_t x = tid; x < PLAN_PAD * sizeof(SegRec) / 8; x += PLAN_THREADS)
@@ -895,24 +922,42 @@ __global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const __grid_const
     }
     WarpTopK top;
     top.init();
-    for (uint32_t b = warp; b < mp.n_partial; b += nw) {
-        const uint32_t n = mp.partial_n[b];
-        Hit mine = {make_inf(), ~0ull};                  // one coalesced read of the block's list
-        if (lane < n) mine = mp.partial[(size_t)b * SAILOR_K_MAX + lane];
-        if (n) top.merge_sorted(mine.score, mine.flat, mp.k, lane);
+    // every warp takes every nw-th block's list; four lists are fetched before they are merged, so
+    // that the loads overlap instead of queueing behind one another
+    for (uint32_t b0 = warp; b0 < mp.n_partial; b0 += 4 * nw) {
+        Hit mine[4];
+        uint32_t cnt[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t b = b0 + u * nw;
+            cnt[u] = b < mp.n_partial ? mp.partial_n[b] : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const uint32_t b = b0 + u * nw;
+            mine[u].score = make_inf();
+            mine[u].flat = ~0ull;
+            if (lane < cnt[u]) mine[u] = mp.partial[(size_t)b * SAILOR_K_MAX + lane];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (cnt[u]) top.merge_sorted(mine[u].score, mine[u].flat, mp.k, lane);
     }
+    // tree merge of the warps' lists through shared memory
     s_hits[warp][lane].score = top.score;
     s_hits[warp][lane].flat = top.flat;
     __syncthreads();
-    if (warp == 0) {
-        for (uint32_t w = 1; w < nw; ++w) {
-            if (s_hits[w][0].flat == ~0ull) continue;
-            top.merge_sorted(s_hits[w][lane].score, s_hits[w][lane].flat, mp.k, lane);
+    for (uint32_t step = 1; step < nw; step <<= 1) {
+        if ((warp & (2 * step - 1)) == 0 && warp + step < nw) {
+            top.merge_sorted(s_hits[warp + step][lane].score, s_hits[warp + step][lane].flat, mp.k, lane);
+            s_hits[warp][lane].score = top.score;
+            s_hits[warp][lane].flat = top.flat;
         }
+        __syncthreads();
+    }
+    if (warp == 0) {
         const bool have = lane < mp.k && top.flat != ~0ull;
         const uint32_t n = __popc(__ballot_sync(FULL, have));
-        s_hits[0][lane].score = top.score;
-        s_hits[0][lane].flat = top.flat;
         if (lane == 0) s_n = n;
     }
     __syncthreads();
