@@ -94,6 +94,13 @@ class OrcCounts(C.Structure):
                                           "n_over_constraint", "n_feasible")] + [("min_cost", C.c_double)]
 
 
+class OrcPrunedCounts(C.Structure):
+    _fields_ = [("looked_at", OrcCounts), ("n_pruned_tp", C.c_uint64), ("n_skipped", C.c_uint64),
+                ("n_configs", C.c_uint64), ("n_configs_evaluated", C.c_uint64)]
+
+
+PRUNE_D_ORDER, PRUNE_MIN_TP = 1, 2
+
 _lib = None
 
 
@@ -117,6 +124,9 @@ def lib():
         L.orc_simulate_batch.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcPlan), C.c_uint64,
                                          _u32p, _dp, _dp, _u64p]
         L.orc_simulate_batch.restype = None
+        L.orc_search_pruned.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcSpace), C.POINTER(OrcObjective),
+                                        C.c_uint32, C.c_uint32, C.POINTER(OrcHit), C.POINTER(OrcPrunedCounts)]
+        L.orc_search_pruned.restype = C.c_int32
         _lib = L
     return _lib
 
@@ -240,6 +250,24 @@ class Oracle:
         out = [dict(flat=int(h.flat), score=h.score, t_iter=h.t_iter, cost=h.cost, peak_mem=int(h.peak_mem))
                for h in hits[:n]]
         return out, {f: (getattr(cnt, f) if f == "min_cost" else int(getattr(cnt, f))) for f, _ in OrcCounts._fields_}
+
+    def search_pruned(self, kind: int, k: int, modes: int, *, budget: float = 0.0, min_rate: float = 0.0):
+        """Whole-space search with the planner's pruning heuristics as modes (PRUNE_D_ORDER: H3/H4,
+        PRUNE_MIN_TP: H2 extended): returns (hits, counts dict)."""
+        obj = OrcObjective(kind, 0, budget, min_rate)
+        hits = (OrcHit * max(k, 1))()
+        cnt = OrcPrunedCounts()
+        n = lib().orc_search_pruned(C.byref(self.inputs), C.byref(self.space), C.byref(obj), modes, k, hits,
+                                    C.byref(cnt))
+        if n < 0:
+            raise ValueError("the pruning mode is not defined for this objective")
+        out = [dict(flat=int(h.flat), score=h.score, t_iter=h.t_iter, cost=h.cost, peak_mem=int(h.peak_mem))
+               for h in hits[:n]]
+        counts = {f: (getattr(cnt.looked_at, f) if f == "min_cost" else int(getattr(cnt.looked_at, f)))
+                  for f, _ in OrcCounts._fields_}
+        for f in ("n_pruned_tp", "n_skipped", "n_configs", "n_configs_evaluated"):
+            counts[f] = int(getattr(cnt, f))
+        return out, counts
 
     def plan(self, k: int, *, lo: int = 0, hi: Optional[int] = None):
         """The workload's own objective, with the cheapest-feasible budget rule when it has one:

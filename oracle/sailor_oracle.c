@@ -258,6 +258,23 @@ static int hit_before(const orc_hit* a, double score, uint64_t flat) {
     return a->score < score || (a->score == score && a->flat < flat);
 }
 
+/* sorted insertion: (score, flat) ascending, keep k (Sec. 4.2: sort by objective); returns the new length */
+static uint32_t offer_hit(orc_hit* hits, uint32_t n_hits, uint32_t k, uint64_t flat, double score, const orc_out* o) {
+    if (k == 0) return n_hits;
+    if (n_hits == k && hit_before(&hits[k - 1], score, flat)) return n_hits;
+    uint32_t pos = n_hits < k ? n_hits : k - 1;
+    while (pos > 0 && !hit_before(&hits[pos - 1], score, flat)) {
+        hits[pos] = hits[pos - 1];
+        pos--;
+    }
+    hits[pos].flat = flat;
+    hits[pos].score = score;
+    hits[pos].t_iter = o->t_iter;
+    hits[pos].cost = o->cost;
+    hits[pos].peak_mem = o->peak_mem;
+    return n_hits < k ? n_hits + 1 : n_hits;
+}
+
 uint32_t orc_search(const orc_inputs* in, const orc_space* sp, const orc_objective* obj,
                     uint64_t lo, uint64_t hi, uint64_t stride, uint32_t k, orc_hit* hits,
                     orc_counts* counts) {
@@ -284,20 +301,7 @@ uint32_t orc_search(const orc_inputs* in, const orc_space* sp, const orc_objecti
         double score = obj->kind == ORC_OBJ_TIME ? o.t_iter
                      : obj->kind == ORC_OBJ_COST ? o.cost
                                                  : o.t_iter * o.cost;
-        /* sorted insertion: (score, flat) ascending, keep k (Sec. 4.2: sort by objective) */
-        if (k == 0) continue;
-        if (n_hits == k && hit_before(&hits[k - 1], score, flat)) continue;
-        uint32_t pos = n_hits < k ? n_hits : k - 1;
-        while (pos > 0 && !hit_before(&hits[pos - 1], score, flat)) {
-            hits[pos] = hits[pos - 1];
-            pos--;
-        }
-        hits[pos].flat = flat;
-        hits[pos].score = score;
-        hits[pos].t_iter = o.t_iter;
-        hits[pos].cost = o.cost;
-        hits[pos].peak_mem = o.peak_mem;
-        if (n_hits < k) n_hits++;
+        n_hits = offer_hit(hits, n_hits, k, flat, score, &o);
     }
     if (counts) *counts = c;
     return n_hits;
@@ -327,4 +331,107 @@ void orc_simulate_batch(const orc_inputs* in, const orc_plan* plans, uint64_t n,
         cost[j] = o.cost;
         peak_mem[j] = o.peak_mem;
     }
+}
+
+/* ---- the planner's pruning heuristics as search modes (Sec. 4.2.1) ------------------------------- */
+
+static double score_of(const orc_objective* obj, const orc_out* o) {
+    return obj->kind == ORC_OBJ_TIME ? o->t_iter : obj->kind == ORC_OBJ_COST ? o->cost : o->t_iter * o->cost;
+}
+
+/* H2, taken one step further than the paper's wording (which only drops tensor-parallel degrees that do
+ * not fit): is there a smaller degree in the space's list at which this very plan is valid and every
+ * stage fits in memory?  Then the plan is not the minimum-degree one and the mode drops it. */
+static int fits_with_smaller_tp(const orc_inputs* in, const orc_space* sp, const orc_plan* pl, uint32_t ti) {
+    const uint32_t tp = in->tp_values[sp->tp_idx[ti]];
+    for (uint32_t tj = 0; tj < sp->n_tp; ++tj) {
+        if (in->tp_values[sp->tp_idx[tj]] >= tp) continue;
+        orc_plan q = *pl;
+        for (uint32_t i = 0; i < q.P; ++i) q.tp_idx[i] = sp->tp_idx[tj];
+        orc_out o;
+        orc_simulate(in, &q, &o);
+        if (!(o.status & (ORC_INVALID | ORC_OOM))) return 1;
+    }
+    return 0;
+}
+
+int32_t orc_search_pruned(const orc_inputs* in, const orc_space* sp, const orc_objective* obj, uint32_t modes,
+                          uint32_t k, orc_hit* hits, orc_pruned_counts* counts) {
+    orc_pruned_counts c;
+    memset(&c, 0, sizeof(c));
+    if ((modes & ORC_PRUNE_D_ORDER) && obj->kind != ORC_OBJ_TIME && obj->kind != ORC_OBJ_COST) return -1;
+    const uint64_t radix = (uint64_t)in->n_types * in->n_zones;
+    const uint64_t base = (uint64_t)sp->n_mbs * sp->n_tp * sp->n_rc * sp->n_d;
+
+    /* the order in which a group's data-parallel degrees are tried: largest first when throughput is
+     * maximised (H3), smallest first when cost is minimised (H4); without the mode, as listed */
+    uint32_t order[256];
+    if (sp->n_d > 256) return -1;
+    for (uint32_t j = 0; j < sp->n_d; ++j) order[j] = j;
+    if (modes & ORC_PRUNE_D_ORDER) {
+        const int descending = obj->kind == ORC_OBJ_TIME;
+        for (uint32_t a = 1; a < sp->n_d; ++a) {             /* insertion sort, stable */
+            uint32_t x = order[a], b = a;
+            while (b > 0 && (descending ? sp->d_values[order[b - 1]] < sp->d_values[x]
+                                        : sp->d_values[order[b - 1]] > sp->d_values[x])) {
+                order[b] = order[b - 1];
+                b--;
+            }
+            order[b] = x;
+        }
+    }
+
+    uint32_t n_hits = 0;
+    uint64_t p_base = 0;                                     /* flat index of the sub-space of this P */
+    orc_plan pl;
+    orc_out o;
+    for (uint32_t jp = 0; jp < sp->n_p; ++jp) {
+        const uint32_t P = sp->p_values[jp];
+        const uint64_t per_cfg = ipow_u64(radix, nseg_of(sp, P));
+        for (uint32_t mi = 0; mi < sp->n_mbs; ++mi)
+        for (uint32_t ti = 0; ti < sp->n_tp; ++ti)
+        for (uint32_t ri = 0; ri < sp->n_rc; ++ri) {
+            /* one group: everything fixed but the data-parallel degree */
+            int have_prev = 0, stopped = 0;
+            double prev_best = 0.0;
+            for (uint32_t step = 0; step < sp->n_d; ++step) {
+                const uint32_t di = order[step];
+                c.n_configs++;
+                if (stopped) { c.n_skipped += per_cfg; continue; }
+                c.n_configs_evaluated++;
+                const uint64_t first = p_base + ((((uint64_t)mi * sp->n_tp + ti) * sp->n_rc + ri) * sp->n_d + di) * per_cfg;
+                int have_best = 0;
+                double best = 0.0;
+                for (uint64_t flat = first; flat < first + per_cfg; ++flat) {
+                    if (orc_decode(in, sp, flat, &pl) != 0) return -1;
+                    orc_simulate(in, &pl, &o);
+                    c.looked_at.n_total++;
+                    if (o.status & ORC_INVALID) { c.looked_at.n_invalid++; continue; }
+                    if (o.status & ORC_OOM) { c.looked_at.n_oom++; continue; }
+                    if ((modes & ORC_PRUNE_MIN_TP) && fits_with_smaller_tp(in, sp, &pl, ti)) { c.n_pruned_tp++; continue; }
+                    if (o.status & ORC_OVER_AVAIL) { c.looked_at.n_over_avail++; continue; }
+                    int over = 0;
+                    if (obj->budget > 0.0 && o.cost > obj->budget) over = 1;
+                    if (obj->min_rate > 0.0 && 1.0 / o.t_iter < obj->min_rate) over = 1;
+                    if (over) { c.looked_at.n_over_constraint++; continue; }
+                    c.looked_at.n_feasible++;
+                    if (c.looked_at.n_feasible == 1 || o.cost < c.looked_at.min_cost) c.looked_at.min_cost = o.cost;
+                    const double score = score_of(obj, &o);
+                    if (!have_best || score < best) { best = score; have_best = 1; }
+                    n_hits = offer_hit(hits, n_hits, k, flat, score, &o);
+                }
+                if (!(modes & ORC_PRUNE_D_ORDER)) continue;
+                /* H3 / H4: degrees without a feasible plan are passed over until the first feasible one is
+                 * found; from then on the next degree is tried only while the group's best objective
+                 * improved strictly */
+                if (!have_best) { if (have_prev) stopped = 1; continue; }
+                if (have_prev && !(best < prev_best)) { stopped = 1; continue; }
+                prev_best = best;
+                have_prev = 1;
+            }
+        }
+        p_base += base * per_cfg;
+    }
+    if (counts) *counts = c;
+    return (int32_t)n_hits;
 }

@@ -13,7 +13,9 @@
  * mixed tensor parallelism; two hand-computed cases with fitted bandwidth polynomials (boundary
  * link and all-reduce); the homogeneous closed form (P + N_b) * t; monotonicity and
  * scaling invariants; an independent nested-loop enumeration and brute-force minimum on
- * tiny clusters.
+ * tiny clusters.  The pruned search modes (H2-H4): three hand-worked searches, equality with the
+ * exhaustive search when no mode is on, and a brute-force restatement over per-candidate results
+ * on tiny clusters (group minimum over tensor-parallel degrees, per-configuration bests).
  * Parity unpinned: the absolute realism of the outputs against real clusters (Sec. 5.1
  * reports 4-6 % error on hardware this repository cannot reach).
  */
@@ -140,5 +142,39 @@ void orc_simulate_flat(const orc_inputs* in, const orc_space* sp, const uint64_t
 /* simulate n written-out plans */
 void orc_simulate_batch(const orc_inputs* in, const orc_plan* plans, uint64_t n,
                         uint32_t* status, double* t_iter, double* cost, uint64_t* peak_mem);
+
+/* ---- pruning heuristics of the planner as search modes (Sec. 4.2.1) ----------------------------
+ *
+ * ORC_PRUNE_D_ORDER (H3, H4).  A group is everything of a configuration but its data-parallel degree:
+ * (P, mbs, tp, recomputation).  Inside a group the degrees of the space are tried from the largest
+ * down when throughput is maximised (H3) and from the smallest up when cost is minimised (H4).
+ * Degrees that have no feasible plan are passed over until the first feasible one (H3 starts from the
+ * largest degree the available GPUs allow, H4 raises the degree until the constraint is met); after that
+ * the next degree is tried only while the best objective value of the group's last degree was strictly better
+ * than that of the degree before it.  The degree at which the improvement stops has been evaluated
+ * and its plans compete for the top-k like all others; the remaining degrees are never looked at.
+ * The paper states the rule for the two objectives only: any other objective is an error (-1).
+ *
+ * ORC_PRUNE_MIN_TP (H2, extended).  H2 as printed drops tensor-parallel degrees below the minimum that
+ * fits in memory, which the memory check already does.  The mode goes one step further and keeps,
+ * of the plans that differ only in the (plan-wide) tensor-parallel degree, only the one with the
+ * smallest degree that is valid and fits: a plan is dropped when some smaller degree of the space's
+ * list gives a valid plan in which every stage fits.  Dropped plans are counted in n_pruned_tp, after
+ * the invalid and out-of-memory classes and before the availability check.
+ */
+#define ORC_PRUNE_D_ORDER 1u
+#define ORC_PRUNE_MIN_TP 2u
+
+typedef struct orc_pruned_counts {
+    orc_counts looked_at;        /* classes over the candidates of the evaluated configurations;
+                                    n_total also contains n_pruned_tp */
+    uint64_t n_pruned_tp;
+    uint64_t n_skipped;          /* candidates of configurations that early termination never reached */
+    uint64_t n_configs, n_configs_evaluated;
+} orc_pruned_counts;
+
+/* whole space; returns the number of hits kept (<= k) or -1 for an unsupported request */
+int32_t orc_search_pruned(const orc_inputs* in, const orc_space* sp, const orc_objective* obj, uint32_t modes,
+                          uint32_t k, orc_hit* hits, orc_pruned_counts* counts);
 
 #endif
