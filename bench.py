@@ -126,6 +126,34 @@ def run_reference(args) -> None:
     print(json.dumps(line), flush=True)
 
 
+def pruning_modes(B, ctx, w, sp) -> dict:
+    """The planner's pruning heuristics as search modes (degree order with early termination, smallest
+    fitting tensor-parallel degree): search seconds, how much was left out, and whether the best plan
+    is still the exhaustive search's."""
+    full, _ = B.sailor_plan(ctx, sp, B.make_objective(w), 1)
+    modes = {"min_tp_only": B.FLAG_MIN_TP_ONLY}
+    if w.objective in (W.OBJ_MAX_THROUGHPUT, W.OBJ_MIN_COST):
+        modes["degree_order"] = B.FLAG_DEGREE_ORDER
+        modes["degree_order+min_tp_only"] = B.FLAG_DEGREE_ORDER | B.FLAG_MIN_TP_ONLY
+    out = {}
+    for name, flags in modes.items():
+        ob = B.make_objective(w, flags=flags)
+        B.sailor_plan(ctx, sp, ob, K_TOP)
+        ts = []
+        for _ in range(5):
+            t0 = time.perf_counter()
+            B.sailor_set_availability(ctx, w.avail)
+            res, st = B.sailor_plan(ctx, sp, ob, K_TOP)
+            ts.append(time.perf_counter() - t0)
+        out[name] = {"search_s": statistics.median(ts), "kernel_ms": st.kernel_ms, "launches": int(st.n_launches),
+                     "looked_at": int(st.n_total), "skipped": int(st.n_skipped), "pruned_tp": int(st.n_pruned_tp),
+                     "configs_evaluated": int(st.n_configs_evaluated), "configs": int(st.n_configs),
+                     "feasible": int(st.n_feasible),
+                     "same_best_as_exhaustive": bool(res and full and res[0].flat == full[0].flat),
+                     "score_over_exhaustive": (res[0].score / full[0].score) if (res and full) else None}
+    return out
+
+
 def aux_measurements(B, torch, dev) -> dict:
     """Search seconds of the other workloads through the public call (host buffers), default mode."""
     out = {}
@@ -144,6 +172,7 @@ def aux_measurements(B, torch, dev) -> dict:
                 ts.append(time.perf_counter() - t0)
             out[f"cfg{cfg}"] = {"candidates": int(st.n_total), "search_s": statistics.median(ts),
                                 "kernel_ms": st.kernel_ms, "passes": 2 if w.budget_factor_over_cheapest > 0 else 1}
+            out[f"cfg{cfg}"]["pruning_modes"] = pruning_modes(B, ctx, w, sp)
         finally:
             B.sailor_destroy(ctx)
     # explicit batches (sailor_simulate) with records resident in HBM: 72 B in + 28 B out per plan
@@ -345,7 +374,8 @@ def run_ours(args) -> None:
                 _, stp = B.sailor_plan(ctx, space, ob, K_TOP)
                 ts.append(time.perf_counter() - t0)
             aux[args.workload + "_default_mode"] = {"candidates": int(stp.n_total), "search_s": statistics.median(ts),
-                                                    "kernel_ms": stp.kernel_ms, "feasible": int(stp.n_feasible)}
+                                                    "kernel_ms": stp.kernel_ms, "feasible": int(stp.n_feasible),
+                                                    "pruning_modes": pruning_modes(B, ctx, w, space)}
         line = {"metric": METRIC, "value": total / dev_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": 1e3 * dev_s / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",

@@ -170,6 +170,29 @@ typedef struct sailor_space {
 #define SAILOR_FLAG_EVAL_ALL 1u  /* compute time and cost of every candidate, skipping nothing;
                                     results are identical with or without it                */
 
+/* The planner's pruning heuristics as search modes (Sec. 4.2.1).  They change what is searched, so
+ * the result may differ from the exhaustive search; sailor_stats says how much was left out.
+ *
+ * SAILOR_FLAG_DEGREE_ORDER (H3, H4).  A group is a configuration without its data-parallel degree:
+ * (P, mbs, tp, rc).  Inside every group the degrees of d_values are tried from the largest down
+ * when kind is MAX_THROUGHPUT (H3) and from the smallest up when it is MIN_COST (H4).  Degrees
+ * with no feasible plan are passed over until the first feasible one; from then on the next degree
+ * is tried only while the group's best score at the last degree was strictly better than at the
+ * degree before.  The degree at which improvement stops has been evaluated and its plans compete
+ * for the top-k; the group's remaining degrees are never looked at (n_skipped).  Whole-space
+ * searches only; E_ARG with MAX_THROUGHPUT_PER_USD, with SAILOR_FLAG_EVAL_ALL, with a sub-range,
+ * and in sailor_plan_noalloc.  With budget_factor_over_cheapest each of the two passes applies the
+ * order of its own objective.  On the device the groups advance together: one launch per
+ * position in the degree order evaluates that degree of every group still going.
+ *
+ * SAILOR_FLAG_MIN_TP_ONLY (H2, taken one step further).  The memory check already drops
+ * tensor-parallel degrees that do not fit, which is H2 as printed.  This mode also drops a plan
+ * when some smaller degree of tp_idx gives a valid plan in which every stage fits, so that of the
+ * plans that differ only in tp the one with the smallest fitting degree remains.  Dropped plans
+ * are counted in n_pruned_tp: after invalid and out of memory, before availability. */
+#define SAILOR_FLAG_DEGREE_ORDER 2u
+#define SAILOR_FLAG_MIN_TP_ONLY  4u
+
 typedef struct sailor_objective {
     uint32_t kind;
     uint32_t flags;
@@ -191,14 +214,19 @@ typedef struct sailor_result {
     sailor_plan_rec plan;
 } sailor_result;
 
-/* Every candidate falls in exactly one class: the first of invalid, oom, over_avail,
- * over_constraint (budget or throughput) that applies, else feasible. */
+/* Every candidate that was looked at falls in exactly one class: the first of invalid, oom,
+ * pruned_tp (SAILOR_FLAG_MIN_TP_ONLY), over_avail, over_constraint (budget or throughput) that
+ * applies, else feasible.  n_total is their sum; n_total + n_skipped is the size of the space. */
 typedef struct sailor_stats {
     uint64_t n_total, n_invalid, n_oom, n_over_avail, n_over_constraint, n_feasible;
     double   budget_used;       /* the budget the (last) pass ran with; <= 0 if none         */
     double   min_feasible_cost; /* smallest C_iter among the feasible candidates; 0 if none */
     float    kernel_ms;         /* device time of the search kernels (CUDA events)          */
     uint32_t n_launches;        /* kernels launched by this call                            */
+    uint64_t n_pruned_tp;       /* dropped because a smaller tensor-parallel degree fits     */
+    uint64_t n_skipped;         /* candidates of configurations early termination never reached */
+    uint32_t n_configs;         /* configurations (P, mbs, tp, rc, D) of the space           */
+    uint32_t n_configs_evaluated;   /* of which looked at (all of them without DEGREE_ORDER) */
 } sailor_stats;
 
 typedef struct sailor_ctx sailor_ctx;     /* opaque; owns device copies of the tables       */

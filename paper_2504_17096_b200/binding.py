@@ -16,7 +16,7 @@ KINDS, T_MAX, Z_MAX, TP_MAX, MBS_MAX, P_MAX, RUN_MAX, SEG_MAX, K_MAX, NP_MAX, ND
 OK, E_ARG, E_RANGE, E_CUDA, E_NOMEM, E_DEVICE = 0, -1, -2, -3, -4, -5
 ST_INVALID, ST_OVER_AVAIL, ST_OOM, ST_OVER_BUDGET, ST_UNDER_THROUGHPUT, ST_BAD_RECORD = 1, 2, 4, 8, 16, 32
 OBJ_MAX_THROUGHPUT, OBJ_MIN_COST, OBJ_MAX_THROUGHPUT_PER_USD = 0, 1, 2
-FLAG_EVAL_ALL = 1
+FLAG_EVAL_ALL, FLAG_DEGREE_ORDER, FLAG_MIN_TP_ONLY = 1, 2, 4
 
 EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
            "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_plan_noalloc",
@@ -75,11 +75,12 @@ class Stats(C.Structure):
     _fields_ = [("n_total", C.c_uint64), ("n_invalid", C.c_uint64), ("n_oom", C.c_uint64),
                 ("n_over_avail", C.c_uint64), ("n_over_constraint", C.c_uint64), ("n_feasible", C.c_uint64),
                 ("budget_used", C.c_double), ("min_feasible_cost", C.c_double), ("kernel_ms", C.c_float),
-                ("n_launches", C.c_uint32)]
+                ("n_launches", C.c_uint32), ("n_pruned_tp", C.c_uint64), ("n_skipped", C.c_uint64),
+                ("n_configs", C.c_uint32), ("n_configs_evaluated", C.c_uint32)]
 
 
 assert C.sizeof(PlanRec) == 72 and C.sizeof(Result) == 120 and C.sizeof(Space) == 152
-assert C.sizeof(Objective) == 32 and C.sizeof(Stats) == 72
+assert C.sizeof(Objective) == 32 and C.sizeof(Stats) == 96
 
 # numpy view of an array of plan records (same 72-byte layout)
 RUN_DTYPE = np.dtype([("type", "u1"), ("zone", "u1"), ("tp_idx", "u1"), ("n_stages", "u1")])

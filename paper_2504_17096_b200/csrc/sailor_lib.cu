@@ -161,7 +161,14 @@ struct SpaceCache {
     uint32_t* d_live_start = nullptr;      // [n_config + 1]
     uint32_t live_chunks = 0;
     unsigned long long closed[3] = {0, 0, 0};   // candidates counted in closed form: total, invalid, oom
+    // searches in degree order (spaces of at most WAVE_CONFIG_MAX configurations)
+    unsigned long long* d_cfg_closed = nullptr;   // [n_config][3] the closed-form counts per configuration
+    uint32_t* d_wave_start = nullptr;             // [n_config + 1] chunk offsets of the current wave
+    unsigned long long* d_cfg_best = nullptr;     // [n_config] best feasible score per configuration
+    GroupState* d_groups = nullptr;               // [n_config / n_d]
 };
+
+constexpr uint64_t WAVE_CONFIG_MAX = 1u << 16;
 
 struct OutBlock {                          // device -> pinned host
     sailor_result results[SAILOR_K_MAX];
@@ -332,14 +339,29 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
     CU(ctx, cudaStreamSynchronize(ctx->stream));       // the vectors are pageable
     {   // survey the space once: live chunks per configuration and the closed-form class counts
         cudaFree(sc.d_live_start);
+        cudaFree(sc.d_cfg_closed);
+        cudaFree(sc.d_wave_start);
+        cudaFree(sc.d_cfg_best);
+        cudaFree(sc.d_groups);
         sc.d_live_start = nullptr;
+        sc.d_cfg_closed = nullptr;
+        sc.d_wave_start = nullptr;
+        sc.d_cfg_best = nullptr;
+        sc.d_groups = nullptr;
         unsigned long long* d_closed = nullptr;
         CU(ctx, cudaMalloc(&sc.d_live_start, (n_config + 1) * sizeof(uint32_t)));
+        if (n_config <= WAVE_CONFIG_MAX) {
+            CU(ctx, cudaMalloc(&sc.d_cfg_closed, n_config * 3 * sizeof(unsigned long long)));
+            CU(ctx, cudaMalloc(&sc.d_wave_start, (n_config + 1) * sizeof(uint32_t)));
+            CU(ctx, cudaMalloc(&sc.d_cfg_best, n_config * sizeof(unsigned long long)));
+            CU(ctx, cudaMalloc(&sc.d_groups, (n_config / d.n_d) * sizeof(GroupState)));
+        }
         CU(ctx, cudaMalloc(&d_closed, 3 * sizeof(unsigned long long)));
         cudaError_t e = cudaMemsetAsync(d_closed, 0, 3 * sizeof(unsigned long long), ctx->stream);
         const uint32_t grid = (uint32_t)(n_config < 2048 ? n_config : 2048);
         if (e == cudaSuccess) {
-            survey_kernel<<<grid, SURVEY_THREADS, 0, ctx->stream>>>(ctx->d_blob, d, (uint32_t)n_config, sc.d_live_start, d_closed);
+            survey_kernel<<<grid, SURVEY_THREADS, 0, ctx->stream>>>(ctx->d_blob, d, (uint32_t)n_config, sc.d_live_start, d_closed,
+                                                                    sc.d_cfg_closed);
             e = cudaGetLastError();
         }
         std::vector<uint32_t> live(n_config + 1, 0);
@@ -405,10 +427,16 @@ int smem_optin(sailor_ctx* ctx, PlanKernel kern, uint32_t variant) {
 }
 
 // Enqueue one search pass (clear, search, merge) on the context's stream.
+//
+// With SAILOR_FLAG_DEGREE_ORDER (whole space, live layout) the search runs as n_d waves: a one-block
+// step kernel applies the H3/H4 rule to the previous wave's per-configuration bests and lays out the
+// next wave's chunks, then the search kernel evaluates them; every block carries its list from wave
+// to wave, so one merge at the end suffices.
 int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_ctrl, double min_rate,
                  uint32_t flags, uint64_t lo, uint64_t hi, bool live, uint32_t k, double next_budget_factor,
                  uint32_t* n_launches) {
     SpaceCache& sc = ctx->space;
+    const bool waves = (flags & SAILOR_FLAG_DEGREE_ORDER) != 0;
     // clear the counters; ctrl->budget (the previous pass may have written it) and the sticky error stay
     CU(ctx, cudaMemsetAsync(ctx->d_ctrl, 0, offsetof(Ctrl, min_cost_bits), ctx->stream));
     CU(ctx, cudaMemsetAsync(&ctx->d_ctrl->min_cost_bits, 0x7f, sizeof(unsigned long long), ctx->stream));
@@ -427,12 +455,20 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
     pp.flat_hi = hi;
     pp.k = k;
     pp.eval_all = (flags & SAILOR_FLAG_EVAL_ALL) ? 1u : 0u;
+    pp.min_tp_only = (flags & SAILOR_FLAG_MIN_TP_ONLY) ? 1u : 0u;
     pp.budget_from_ctrl = budget_from_ctrl ? 1u : 0u;
     pp.p_max = sc.p_max;
     pp.budget = budget;
     pp.min_rate = min_rate;
     uint32_t grid = 0;
-    if (live) {                    // whole space, pruning on: only chunks of live prefixes exist
+    if (waves) {                   // the chunk table and the chunk count of each wave are written on the device
+        pp.cfg_chunk_start = sc.d_wave_start;
+        pp.live_mode = 1;
+        pp.chunk_lo = 0;
+        pp.chunk_hi = 1;                           // the waves always run: they also gather the class counts
+        pp.chunk_hi_dev = &ctx->d_ctrl->wave_chunks;
+        pp.cfg_best = sc.d_cfg_best;
+    } else if (live) {                    // whole space, pruning on: only chunks of live prefixes exist
         pp.cfg_chunk_start = sc.d_live_start;
         pp.live_mode = 1;
         pp.chunk_lo = 0;
@@ -458,9 +494,45 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
         grid = n_chunks < resident ? n_chunks : resident;
         const uint32_t batch = n_chunks / (grid * 32u);
         pp.batch = batch < 1 ? 1 : (batch > 16 ? 16 : batch);
-        kern<<<grid, PLAN_THREADS, sc.smem, ctx->stream>>>(pp);
-        CU(ctx, cudaGetLastError());
-        ++*n_launches;
+        if (!waves) {
+            kern<<<grid, PLAN_THREADS, sc.smem, ctx->stream>>>(pp);
+            CU(ctx, cudaGetLastError());
+            ++*n_launches;
+        } else {
+            grid = resident < sc.live_chunks ? resident : (sc.live_chunks ? sc.live_chunks : 1u);   // the same blocks in every wave
+            WaveParams wp;
+            memset(&wp, 0, sizeof(wp));
+            wp.live_start = sc.d_live_start;
+            wp.cfg_closed = sc.d_cfg_closed;
+            wp.wave_start = sc.d_wave_start;
+            wp.cfg_best = sc.d_cfg_best;
+            wp.groups = sc.d_groups;
+            wp.ctrl = ctx->d_ctrl;
+            wp.n_config = sc.n_config;
+            wp.n_d = sc.desc.n_d;
+            // H3: largest degree first when throughput is maximised; H4: smallest first when cost is minimised
+            const bool descending = obj == SAILOR_OBJ_MAX_THROUGHPUT;
+            for (uint32_t j = 0; j < wp.n_d; ++j) wp.order[j] = (uint8_t)j;
+            for (uint32_t a = 1; a < wp.n_d; ++a) {        // stable insertion sort by degree
+                const uint8_t x = wp.order[a];
+                uint32_t b = a;
+                while (b > 0 && (descending ? sc.desc.d_values[wp.order[b - 1]] < sc.desc.d_values[x]
+                                            : sc.desc.d_values[wp.order[b - 1]] > sc.desc.d_values[x])) {
+                    wp.order[b] = wp.order[b - 1];
+                    --b;
+                }
+                wp.order[b] = x;
+            }
+            for (uint32_t w = 0; w < wp.n_d; ++w) {
+                wp.wave = w;
+                wave_step_kernel<<<1, WAVE_THREADS, 0, ctx->stream>>>(wp);
+                CU(ctx, cudaGetLastError());
+                pp.carry_lists = w ? 1u : 0u;
+                kern<<<grid, PLAN_THREADS, sc.smem, ctx->stream>>>(pp);
+                CU(ctx, cudaGetLastError());
+                *n_launches += 2;
+            }
+        }
     }
     MergeParams mp;
     memset(&mp, 0, sizeof(mp));
@@ -669,6 +741,10 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->space.d_chunk_start);
     cudaFree(ctx->space.d_flat_base);
     cudaFree(ctx->space.d_live_start);
+    cudaFree(ctx->space.d_cfg_closed);
+    cudaFree(ctx->space.d_wave_start);
+    cudaFree(ctx->space.d_cfg_best);
+    cudaFree(ctx->space.d_groups);
     cudaFree(ctx->d_stage);
     if (ctx->ev0) cudaEventDestroy(ctx->ev0);
     if (ctx->ev1) cudaEventDestroy(ctx->ev1);
@@ -765,6 +841,13 @@ int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objec
     const uint64_t total = ctx->space.n_total;
     if (flat_hi > total) flat_hi = total;
     if (flat_lo > flat_hi) flat_lo = flat_hi;
+    const bool waves = (o->flags & SAILOR_FLAG_DEGREE_ORDER) != 0;
+    if (waves) {
+        if (o->kind == SAILOR_OBJ_MAX_THROUGHPUT_PER_USD || (o->flags & SAILOR_FLAG_EVAL_ALL) || flat_lo != 0 ||
+            flat_hi != total)
+            return SAILOR_E_ARG;
+        if (!ctx->space.d_cfg_closed) return SAILOR_E_RANGE;     // more configurations than the wave tables hold
+    }
 
     uint32_t launches = 0;
     CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
@@ -791,10 +874,16 @@ int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objec
     memcpy(topk, ctx->h_out->results, sizeof(sailor_result) * cr.n_found);
     if (stats) {
         // in live mode the kernels count the evaluated candidates only; the rest is the survey's closed form
+        // (in degree order: of the configurations the waves selected, summed on the device)
         const SpaceCache& sc = ctx->space;
-        stats->n_total = live ? sc.closed[0] : cr.stats[0];
-        stats->n_invalid = live ? sc.closed[1] : cr.stats[1];
-        stats->n_oom = live ? sc.closed[2] : cr.stats[2];
+        const bool closed_form = live && !waves;
+        stats->n_total = closed_form ? sc.closed[0] : cr.stats[0];
+        stats->n_invalid = closed_form ? sc.closed[1] : cr.stats[1];
+        stats->n_oom = closed_form ? sc.closed[2] : cr.stats[2];
+        stats->n_pruned_tp = cr.stats[6];
+        stats->n_skipped = waves ? sc.closed[0] - cr.stats[0] : 0;
+        stats->n_configs = sc.n_config;
+        stats->n_configs_evaluated = waves ? cr.n_cfg_evaluated : sc.n_config;
         stats->n_over_avail = cr.stats[3];
         stats->n_over_constraint = cr.stats[4];
         stats->n_feasible = cr.stats[5];
@@ -878,6 +967,7 @@ int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& d
     pp.flat_hi = total;
     pp.k = k;
     pp.eval_all = (flags & SAILOR_FLAG_EVAL_ALL) ? 1u : 0u;
+    pp.min_tp_only = (flags & SAILOR_FLAG_MIN_TP_ONLY) ? 1u : 0u;
     pp.budget_from_ctrl = budget_from_ctrl ? 1u : 0u;
     pp.p_max = p_max;
     pp.budget = budget;
@@ -930,6 +1020,7 @@ extern "C" int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const
     if (std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) ||
         std::isnan(o->budget_factor_over_cheapest))
         return SAILOR_E_ARG;
+    if (o->flags & SAILOR_FLAG_DEGREE_ORDER) return SAILOR_E_ARG;           // needs tables this variant has no room for
     int rc = check_space(ctx, s);
     if (rc) return rc;
     const SpaceDesc d = to_desc(s);
@@ -1004,6 +1095,9 @@ extern "C" int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const
         stats->n_over_avail = cr.stats[3];
         stats->n_over_constraint = cr.stats[4];
         stats->n_feasible = cr.stats[5];
+        stats->n_pruned_tp = cr.stats[6];
+        stats->n_skipped = 0;
+        stats->n_configs = stats->n_configs_evaluated = (uint32_t)n_config;
         stats->budget_used = two_pass ? cr.budget : o->budget_usd_per_iter;
         double mc;
         memcpy(&mc, &cr.min_cost_bits, sizeof(mc));

@@ -33,9 +33,11 @@ struct Hit {
 };
 
 struct Ctrl {                       // one per context, device memory
-    unsigned int work_counter;      // next chunk to hand out (cleared per pass)
+    unsigned int work_counter;      // next chunk to hand out (cleared per pass, and per wave of a pass)
     unsigned int n_found;
-    unsigned long long stats[6];    // total, invalid, oom, over_avail, over_constraint, feasible
+    unsigned long long stats[7];    // total, invalid, oom, over_avail, over_constraint, feasible, pruned_tp
+    unsigned int wave_chunks;       // chunks of the current wave (searches in degree order)
+    unsigned int n_cfg_evaluated;   // configurations selected by the waves so far
     unsigned long long min_cost_bits;   // min C_iter over feasible candidates, as ordered bits
     double budget;                  // written by the cheapest-plan pass for the next pass
     unsigned int error;             // non-zero: a kernel gave up (bounded wait ran out); sticky
@@ -59,6 +61,10 @@ struct PlanParams {
     uint32_t budget_from_ctrl;         // read the budget from ctrl->budget
     uint32_t p_max;                    // largest P of the space (sizes the stage tables)
     uint32_t live_mode;                // cfg_chunk_start counts only chunks of prefixes made of usable digits
+    uint32_t min_tp_only;              // drop plans that also fit with a smaller tensor-parallel degree (H2)
+    uint32_t carry_lists;              // a block starts from the list it left in `partial` (waves of one search)
+    const uint32_t* chunk_hi_dev;      // non-null: chunks [0, *chunk_hi_dev) instead of [chunk_lo, chunk_hi)
+    unsigned long long* cfg_best;      // non-null: [n_config] best feasible score per configuration (ordered bits)
     double budget;                     // <= 0: none
     double min_rate;                   // <= 0: none
 };
@@ -186,12 +192,16 @@ struct CfgShared {
     uint64_t n_items;            // R^(nseg-1)
     uint64_t invalid_mask;       // digit d: tp > gpus_per_node[type(d)]
     uint64_t oom_mask[SAILOR_SEG_MAX];    // digit d: some stage of the segment does not fit type(d)
+    uint32_t n_lower;            // smaller tensor-parallel degrees of the space that the model accepts (min_tp_only)
+    uint32_t lower_tpi[SAILOR_TP_MAX];    // their tp indices
+    uint64_t lower_fit[SAILOR_TP_MAX][SAILOR_SEG_MAX];   // digit d: every stage of the segment fits at that degree
     uint64_t avail_last;         // digit d: need[last] <= avail[d]
     uint32_t cur_config;
     uint32_t next_chunk, batch_len;
-    uint32_t oom_stage[SAILOR_P_MAX];     // per stage: bit g set when the stage does not fit type g
+    unsigned long long oom_stage[SAILOR_P_MAX];   // per stage: bit 8 j + g set when the stage does not fit type g
+                                                  // at this configuration's degree (j = 0) or at lower_tpi[j - 1]
     uint64_t params[SAILOR_P_MAX];
-    unsigned long long stat[6];
+    unsigned long long stat[7];
     uint64_t mbar;
 };
 
@@ -255,6 +265,13 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
             cs.n_items = ipow64(R, k.nseg - 1);
             cs.packed = 0;             // decided at the end of the build, and only for valid configurations
             cs.cur_config = c;
+            uint32_t n_lower = 0;
+            if (pp.min_tp_only)
+                for (uint32_t j = 0; j < pp.sp.n_tp; ++j) {
+                    const uint32_t tj = pp.sp.tp_idx[j], tv = h->tp_values[tj];
+                    if (tv < tp0 && h->heads % tv == 0 && n_lower < SAILOR_TP_MAX - 1) cs.lower_tpi[n_lower++] = tj;
+                }
+            cs.n_lower = n_lower;
         }
         const uint32_t P = __shfl_sync(FULL, k.P, 0), nseg = __shfl_sync(FULL, k.nseg, 0);
         const uint32_t D = __shfl_sync(FULL, k.D, 0), tp = h->tp_values[__shfl_sync(FULL, k.tpi, 0)];
@@ -264,6 +281,7 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
             const uint32_t extra = h->n_blocks % P;
             cs.need[tid] = D * tp * (end - lo);
             cs.oom_mask[tid] = 0;
+            for (uint32_t j = 0; j < SAILOR_TP_MAX; ++j) cs.lower_fit[j][tid] = 0;
             uint32_t hi = (tid + 1 < nseg) ? end - 1 : end;      // a non-final segment's last stage is kept apart
             const uint32_t c3 = (hi == P && hi > lo) ? 1u : 0u;   // the final stage
             hi -= c3;
@@ -302,8 +320,16 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         a.uu[x] = st.u;
         const uint64_t inflight = (uint64_t)(P - i) < cs.n_b ? (uint64_t)(P - i) : cs.n_b;
         const StageMem sm = stage_memory(v, k.tpi, k.mi, k.rc, nb, e, hd, inflight);
-        if (sm.mem + h->reserved[g] > h->capacity[g]) atomicOr(&cs.oom_stage[i], 1u << g);
+        if (sm.mem + h->reserved[g] > h->capacity[g]) atomicOr(&cs.oom_stage[i], 1ull << g);
         if (g == 0) cs.params[i] = sm.params;
+    }
+    for (uint32_t x = tid; x < cs.n_lower * P * T; x += PLAN_THREADS) {      // the same stages at the smaller degrees
+        const uint32_t j = x / (P * T), i = (x / T) % P, g = x % T;
+        const uint32_t nb = base + (i < extra ? 1u : 0u);
+        const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
+        const uint64_t inflight = (uint64_t)(P - i) < cs.n_b ? (uint64_t)(P - i) : cs.n_b;
+        const StageMem sm = stage_memory(v, cs.lower_tpi[j], k.mi, k.rc, nb, e, hd, inflight);
+        if (sm.mem + h->reserved[g] > h->capacity[g]) atomicOr(&cs.oom_stage[i], 1ull << (8 * (j + 1) + g));
     }
     for (uint32_t d = tid; d < R; d += PLAN_THREADS) {
         a.availv[d] = pp.avail[d];
@@ -336,7 +362,9 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         for (int q = 0; q < N_RUNS; ++q) r.v[q] = 0.0;
         double tm = 0.0, sy = 0.0, up = 0.0;
         bool oom = false;
+        unsigned long long oom_bits = 0;
         for (uint32_t i = sa; i < se; ++i) {
+            oom_bits |= cs.oom_stage[i];
             if (i < t_end) {
                 const double fbi = a.fb[i * T + g];
                 const double t = (i + 1 < P) ? add_rn(fbi, c2self) : fbi;
@@ -353,6 +381,9 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
         r.rate = mul_rn((double)(k.D * tp), v.price_s[d]);
         a.rec[x] = r;
         if (oom) atomicOr(reinterpret_cast<unsigned long long*>(&cs.oom_mask[s]), 1ull << d);
+        for (uint32_t j = 0; j < cs.n_lower; ++j)
+            if (!((oom_bits >> (8 * (j + 1) + g)) & 1ull))
+                atomicOr(reinterpret_cast<unsigned long long*>(&cs.lower_fit[j][s]), 1ull << d);
     }
     __syncthreads();                   // the memory masks are complete
     if (tid < 32) {
@@ -393,15 +424,30 @@ __device__ __forceinline__ uint64_t warp_or64(uint64_t x) {
 }
 
 struct Counters {
-    uint32_t invalid, oom, over_avail, over_constr, feasible, total;
+    uint32_t invalid, oom, over_avail, over_constr, feasible, total, pruned;
     double min_cost;
+    double cfg_best;     // best feasible score seen in the current configuration
 };
+
+// Hand the block's best feasible score of configuration `c` to the per-configuration table (positive
+// doubles order like their bit patterns) and start over.
+__device__ __forceinline__ void flush_cfg_best(const PlanParams& pp, Counters& cnt, uint32_t c, uint32_t lane) {
+    unsigned long long b = (unsigned long long)__double_as_longlong(cnt.cfg_best);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(FULL, b, o);
+        b = other < b ? other : b;
+    }
+    if (lane == 0 && b < (unsigned long long)__double_as_longlong(make_inf())) atomicMin(&pp.cfg_best[c], b);
+    cnt.cfg_best = make_inf();
+}
 
 // Add a warp's per-thread counters to the block's 64-bit sums and clear them.
 __device__ __forceinline__ void flush_counters(CfgShared& cs, Counters& cnt, uint32_t lane) {
-    uint32_t* vals[6] = {&cnt.total, &cnt.invalid, &cnt.oom, &cnt.over_avail, &cnt.over_constr, &cnt.feasible};
+    uint32_t* vals[7] = {&cnt.total, &cnt.invalid, &cnt.oom, &cnt.over_avail, &cnt.over_constr, &cnt.feasible,
+                         &cnt.pruned};
 #pragma unroll
-    for (int j = 0; j < 6; ++j) {
+    for (int j = 0; j < 7; ++j) {
         unsigned long long s = *vals[j];
 #pragma unroll
         for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(FULL, s, o);
@@ -599,7 +645,16 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     }
     if (!active) range = 0;
     const uint64_t valid_l = range & ~cs.invalid_mask;
-    const uint64_t good_l = valid_l & ~cs.oom_mask[last];
+    const uint64_t fit_l = valid_l & ~cs.oom_mask[last];
+    uint64_t drop = 0;            // last digits at which the whole plan also fits with a smaller degree
+    if (pp.min_tp_only)
+        for (uint32_t j = 0; j < cs.n_lower; ++j) {
+            bool pf = true;
+#pragma unroll
+            for (int s = 0; s < NSEG - 1; ++s) pf &= (cs.lower_fit[j][s] >> dg[s]) & 1;
+            if (pf) drop |= cs.lower_fit[j][last];
+        }
+    const uint64_t good_l = fit_l & ~drop;
     uint64_t ok = good_l & cs.avail_last;
 #pragma unroll
     for (int s = 0; s < NSEG - 1; ++s) {                  // a last digit equal to a prefix digit adds up
@@ -612,6 +667,7 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     // exactly one class per candidate: invalid, then oom, then over availability
     const uint32_t n_range = __popcll(range);
     if (cs.packed) {                                      // total, invalid and oom were added in closed form
+        cnt.pruned += __popcll(fit_l) - __popcll(good_l);
         if (p_over) { cnt.over_avail += __popcll(good_l); ok = 0; }
         else cnt.over_avail += __popcll(good_l) - __popcll(ok);
     } else if (p_inv) { cnt.total += n_range; cnt.invalid += n_range; ok = 0; }
@@ -620,7 +676,8 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
         cnt.invalid += n_range - __popcll(valid_l);
         if (p_oom) { cnt.oom += __popcll(valid_l); ok = 0; }
         else {
-            cnt.oom += __popcll(valid_l) - __popcll(good_l);
+            cnt.oom += __popcll(valid_l) - __popcll(fit_l);
+            cnt.pruned += __popcll(fit_l) - __popcll(good_l);
             if (p_over) { cnt.over_avail += __popcll(good_l); ok = 0; }
             else cnt.over_avail += __popcll(good_l) - __popcll(ok);
         }
@@ -672,6 +729,7 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     double best = make_inf();
     uint32_t feas = 0;
     walk_fast<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, best, feas, cnt.min_cost);
+    cnt.cfg_best = best < cnt.cfg_best ? best : cnt.cfg_best;
     if (CONSTR) {
         cnt.feasible += feas;
         cnt.over_constr += n_ok - feas;
@@ -708,7 +766,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
         cs.cur_config = 0xffffffffu;
         cs.magic = (uint32_t)(0x100000000ull / (gh->R ? gh->R : 1u)) + 1u;      // for x / R, see CfgShared
     }
-    if (tid < 6) cs.stat[tid] = 0;
+    if (tid < 7) cs.stat[tid] = 0;
     // the padding digit of the tables is read (and masked out) by the two-digit steps: keep it finite
     for (uint32_t x = tid; x < PLAN_PAD * sizeof(SegRec) / 8; x += PLAN_THREADS)
         reinterpret_cast<double*>(a.rec + (size_t)SAILOR_SEG_MAX * R)[x] = 0.0;
@@ -716,8 +774,18 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
     for (uint32_t x = tid; x < PLAN_PAD * Z; x += PLAN_THREADS) a.commx[(size_t)R * Z + x] = 0.0;
     WarpTopK top;
     top.init();
-    Counters cnt = {0, 0, 0, 0, 0, 0, make_inf()};
+    if (pp.carry_lists && warp == 0) {     // a later wave of one search: go on from the list this block left behind
+        if (lane < pp.partial_n[blockIdx.x]) {
+            top.score = pp.partial[(size_t)blockIdx.x * SAILOR_K_MAX + lane].score;
+            top.flat = pp.partial[(size_t)blockIdx.x * SAILOR_K_MAX + lane].flat;
+        }
+        top.thr_score = __shfl_sync(FULL, top.score, pp.k - 1);
+        top.thr_flat = __shfl_sync(FULL, top.flat, pp.k - 1);
+    }
+    Counters cnt = {0, 0, 0, 0, 0, 0, 0, make_inf(), make_inf()};
     const double budget = pp.budget_from_ctrl ? pp.ctrl->budget : pp.budget;
+    const uint32_t chunk_lo = pp.chunk_hi_dev ? 0u : pp.chunk_lo;
+    const uint32_t chunk_hi = pp.chunk_hi_dev ? *pp.chunk_hi_dev : pp.chunk_hi;
     __syncthreads();
 
     uint32_t c = 0;     // configuration of the current chunk (monotone within a batch)
@@ -725,17 +793,17 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
         if (tid == 0) {
             // guided self-scheduling: long runs of consecutive chunks first (a block then stays inside
             // one configuration and rebuilds its tables rarely), single chunks at the end (even finish)
-            const uint32_t n_chunks = pp.chunk_hi - pp.chunk_lo;
+            const uint32_t n_chunks = chunk_hi - chunk_lo;
             const uint32_t seen = *reinterpret_cast<volatile unsigned int*>(&pp.ctrl->work_counter);
             const uint32_t left = seen < n_chunks ? n_chunks - seen : 0u;
             const uint32_t len = max(1u, left / (gridDim.x * 4u));
-            cs.next_chunk = pp.chunk_lo + atomicAdd(&pp.ctrl->work_counter, len);
+            cs.next_chunk = chunk_lo + atomicAdd(&pp.ctrl->work_counter, len);
             cs.batch_len = len;
         }
         __syncthreads();
         const uint32_t first = cs.next_chunk;
-        if (first >= pp.chunk_hi) break;
-        const uint32_t end = min(first + cs.batch_len, pp.chunk_hi);
+        if (first >= chunk_hi) break;
+        const uint32_t end = min(first + cs.batch_len, chunk_hi);
         {   // configuration of the first chunk: binary search (uniform)
             uint32_t lo = 0, hi = pp.n_config;
             while (hi - lo > 1) {
@@ -747,6 +815,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
         for (uint32_t ch = first; ch < end; ++ch) {
             while (ch >= pp.cfg_chunk_start[c + 1]) ++c;
             if (cs.cur_config != c) {
+                if (pp.cfg_best && cs.cur_config != 0xffffffffu) flush_cfg_best(pp, cnt, cs.cur_config, lane);
                 __syncthreads();
                 build_config(pp, v, cs, a, c);
             }
@@ -790,6 +859,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
     }
 
     // ---- block reduction: counters, then the warps' lists ---------------------------------------
+    if (pp.cfg_best && cs.cur_config != 0xffffffffu) flush_cfg_best(pp, cnt, cs.cur_config, lane);
     flush_counters(cs, cnt, lane);
     {
         unsigned long long mc = (unsigned long long)__double_as_longlong(cnt.min_cost);   // positive: bits order
@@ -803,7 +873,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
     s_hits[warp][lane].score = top.score;
     s_hits[warp][lane].flat = top.flat;
     __syncthreads();
-    if (tid < 6 && cs.stat[tid]) atomicAdd(&pp.ctrl->stats[tid], cs.stat[tid]);
+    if (tid < 7 && cs.stat[tid]) atomicAdd(&pp.ctrl->stats[tid], cs.stat[tid]);
     if (warp == 0) {
         for (uint32_t w = 1; w < PLAN_WARPS; ++w) {
             if (s_hits[w][0].flat == ~0ull) continue;    // an empty list
@@ -827,7 +897,8 @@ constexpr int SURVEY_THREADS = 128;
 
 __global__ void __launch_bounds__(SURVEY_THREADS)
 survey_kernel(const unsigned char* __restrict__ blob, SpaceDesc sp, uint32_t n_config, uint32_t* __restrict__ live_chunks,
-              unsigned long long* __restrict__ closed /* total, invalid, oom */) {
+              unsigned long long* __restrict__ closed /* total, invalid, oom */,
+              unsigned long long* __restrict__ cfg_closed /* [n_config][3], the same per configuration; may be null */) {
     __shared__ uint32_t oom_stage[SAILOR_P_MAX];
     __shared__ Config k;
     __shared__ uint32_t valid;
@@ -863,10 +934,8 @@ survey_kernel(const unsigned char* __restrict__ blob, SpaceDesc sp, uint32_t n_c
         if (tid == 0) {
             const uint64_t n_all = ipow64(R, k.nseg);
             uint32_t chunks = 0;
-            if (!valid) {
-                atomicAdd(&closed[0], (unsigned long long)n_all);
-                atomicAdd(&closed[1], (unsigned long long)n_all);
-            } else {
+            unsigned long long mine[3] = {n_all, n_all, 0};     // total, invalid, oom of this configuration
+            if (valid) {
                 const uint32_t tp = h->tp_values[k.tpi];
                 uint32_t type_ok = 0;                      // types whose nodes can host tp
                 for (uint32_t g = 0; g < T; ++g)
@@ -882,13 +951,114 @@ survey_kernel(const unsigned char* __restrict__ blob, SpaceDesc sp, uint32_t n_c
                     if (s + 1 < k.nseg) live *= g_cnt;
                 }
                 if (fit) chunks = (uint32_t)((live + PLAN_THREADS - 1) / PLAN_THREADS);
-                atomicAdd(&closed[0], (unsigned long long)n_all);
-                atomicAdd(&closed[1], (unsigned long long)(n_all - n_valid));
-                atomicAdd(&closed[2], (unsigned long long)(n_valid - fit));
+                mine[1] = n_all - n_valid;
+                mine[2] = n_valid - fit;
+            }
+            for (int j = 0; j < 3; ++j) {
+                if (mine[j]) atomicAdd(&closed[j], mine[j]);
+                if (cfg_closed) cfg_closed[3 * (size_t)c + j] = mine[j];
             }
             live_chunks[c] = chunks;
         }
     }
+}
+
+// ---- searches in degree order (H3 / H4) -----------------------------------------------------------
+//
+// A group is a configuration without its data-parallel degree; its degrees sit next to each other in
+// the configuration index (c = group * n_d + position in d_values).  The rule of a group is
+// sequential (try the next degree only while the last one improved), but the groups are independent,
+// so they advance together: wave w evaluates, for every group still going, the w-th degree of the
+// order.  Between two waves one small block applies the rule to what the last wave found and lays
+// out the chunk table of the next one; nothing returns to the host in between.
+struct GroupState {
+    unsigned long long prev_bits;      // best score at the last degree that had a feasible plan
+    uint32_t state;                    // 0: no feasible degree yet, 1: going, 2: stopped
+    uint32_t _pad;
+};
+
+struct WaveParams {
+    const uint32_t* live_start;        // [n_config + 1] chunk offsets when every configuration is searched
+    const unsigned long long* cfg_closed;   // [n_config][3] total, invalid, oom per configuration
+    uint32_t* wave_start;              // [n_config + 1] out: chunk offsets of this wave
+    unsigned long long* cfg_best;      // [n_config]
+    GroupState* groups;                // [n_config / n_d]
+    Ctrl* ctrl;
+    uint32_t n_config, n_d, wave;
+    uint8_t order[SAILOR_ND_MAX];      // positions in d_values, in the order they are tried
+};
+
+constexpr int WAVE_THREADS = 1024;
+
+__global__ void __launch_bounds__(WAVE_THREADS) wave_step_kernel(const __grid_constant__ WaveParams wp) {
+    __shared__ uint32_t warp_sum[WAVE_THREADS / 32];
+    __shared__ unsigned long long s_closed[3];
+    __shared__ uint32_t s_eval;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t n_groups = wp.n_config / wp.n_d;
+    const unsigned long long inf_bits = (unsigned long long)__double_as_longlong(make_inf());
+    if (tid < 3) s_closed[tid] = 0;
+    if (tid == 0) s_eval = 0;
+    // the rule, applied to what the previous wave found
+    for (uint32_t g = tid; g < n_groups; g += WAVE_THREADS) {
+        GroupState gs = wp.groups[g];
+        if (wp.wave == 0) { gs.prev_bits = inf_bits; gs.state = 0; gs._pad = 0; }
+        else if (gs.state != 2) {
+            const unsigned long long best = wp.cfg_best[(size_t)g * wp.n_d + wp.order[wp.wave - 1]];
+            if (best == inf_bits) { if (gs.state == 1) gs.state = 2; }         // nothing feasible at that degree
+            else if (gs.state == 1 && !(best < gs.prev_bits)) gs.state = 2;     // no strict improvement
+            else { gs.prev_bits = best; gs.state = 1; }
+        }
+        wp.groups[g] = gs;
+    }
+    __syncthreads();
+    // chunk table of this wave: the configuration (group, order[wave]) of every group still going
+    const uint32_t per = (wp.n_config + WAVE_THREADS - 1) / WAVE_THREADS;
+    const uint32_t c0 = min(tid * per, wp.n_config), c1 = min(c0 + per, wp.n_config);
+    const uint32_t pick = wp.order[wp.wave];
+    uint32_t mine = 0, n_eval = 0;
+    unsigned long long closed[3] = {0, 0, 0};
+    for (uint32_t c = c0; c < c1; ++c) {
+        if (c % wp.n_d != pick || wp.groups[c / wp.n_d].state == 2) continue;
+        mine += wp.live_start[c + 1] - wp.live_start[c];
+        wp.cfg_best[c] = inf_bits;
+        ++n_eval;
+        for (int j = 0; j < 3; ++j) closed[j] += wp.cfg_closed[3 * (size_t)c + j];
+    }
+    uint32_t incl = mine;                                   // exclusive scan of `mine` over the block
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t up = __shfl_up_sync(FULL, incl, o);
+        if (lane >= (uint32_t)o) incl += up;
+    }
+    if (lane == 31) warp_sum[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        uint32_t w = warp_sum[lane], wi = w;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t up = __shfl_up_sync(FULL, wi, o);
+            if (lane >= (uint32_t)o) wi += up;
+        }
+        warp_sum[lane] = wi - w;
+        if (lane == 31) {
+            wp.wave_start[wp.n_config] = wi;
+            wp.ctrl->wave_chunks = wi;
+            wp.ctrl->work_counter = 0;
+        }
+    }
+    __syncthreads();
+    uint32_t at = warp_sum[warp] + incl - mine;
+    for (uint32_t c = c0; c < c1; ++c) {
+        wp.wave_start[c] = at;
+        if (c % wp.n_d == pick && wp.groups[c / wp.n_d].state != 2) at += wp.live_start[c + 1] - wp.live_start[c];
+    }
+    for (int j = 0; j < 3; ++j)
+        if (closed[j]) atomicAdd(&s_closed[j], closed[j]);
+    if (n_eval) atomicAdd(&s_eval, n_eval);
+    __syncthreads();
+    if (tid < 3 && s_closed[tid]) atomicAdd(&wp.ctrl->stats[tid], s_closed[tid]);
+    if (tid == 0) wp.ctrl->n_cfg_evaluated += s_eval;
 }
 
 // Merge the blocks' lists, then simulate the winners in full for the result records.

@@ -28,7 +28,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_sizes_match_the_header(lib):
     assert C.sizeof(B.PlanRec) == 72 and C.sizeof(B.Run) == 4
-    assert C.sizeof(B.Result) == 120 and C.sizeof(B.Stats) == 72
+    assert C.sizeof(B.Result) == 120 and C.sizeof(B.Stats) == 96
     assert C.sizeof(B.Space) == 152 and C.sizeof(B.Objective) == 32
 
 
