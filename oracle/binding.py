@@ -101,6 +101,16 @@ class OrcPrunedCounts(C.Structure):
 
 PRUNE_D_ORDER, PRUNE_MIN_TP = 1, 2
 
+
+class OrcDpProblem(C.Structure):
+    _fields_ = [("P", C.c_uint32), ("mbs_idx", C.c_uint32), ("tp_idx", C.c_uint32), ("rc", C.c_uint32),
+                ("D", C.c_uint32), ("n_zones_used", C.c_uint32), ("zone_list", C.c_uint32 * 16)]
+
+
+class OrcDpResult(C.Structure):
+    _fields_ = [("found", C.c_int32), ("_pad", C.c_uint32), ("value", C.c_double), ("n_states", C.c_uint64),
+                ("plan", OrcPlan)]
+
 _lib = None
 
 
@@ -127,6 +137,8 @@ def lib():
         L.orc_search_pruned.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcSpace), C.POINTER(OrcObjective),
                                         C.c_uint32, C.c_uint32, C.POINTER(OrcHit), C.POINTER(OrcPrunedCounts)]
         L.orc_search_pruned.restype = C.c_int32
+        L.orc_solve_dp.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcDpProblem), C.c_int, C.POINTER(OrcDpResult)]
+        L.orc_solve_dp.restype = C.c_int
         _lib = L
     return _lib
 
@@ -268,6 +280,24 @@ class Oracle:
         for f in ("n_pruned_tp", "n_skipped", "n_configs", "n_configs_evaluated"):
             counts[f] = int(getattr(cnt, f))
         return out, counts
+
+    def solve_dp(self, P: int, mbs_idx: int, tp_idx: int, rc: int, D: int, zone_list: Sequence[int], *,
+                 use_memo: bool = True) -> Optional[dict]:
+        """Per-stage GPU types by the dynamic-programming recursion (Sec. 4.2.2) for one configuration and
+        one zone order; None when no plan fits.  Returns value, types, zones, the written-out plan and the
+        number of states solved."""
+        pb = OrcDpProblem()
+        pb.P, pb.mbs_idx, pb.tp_idx, pb.rc, pb.D, pb.n_zones_used = P, mbs_idx, tp_idx, rc, D, len(zone_list)
+        for j, z in enumerate(zone_list):
+            pb.zone_list[j] = int(z)
+        out = OrcDpResult()
+        if lib().orc_solve_dp(C.byref(self.inputs), C.byref(pb), 1 if use_memo else 0, C.byref(out)) != 0:
+            raise ValueError("problem beyond the oracle's limits")
+        if not out.found:
+            return None
+        plan = OrcPlan.from_buffer_copy(out.plan)
+        return {"value": out.value, "types": list(plan.type[:P]), "zones": list(plan.zone[:P]), "plan": plan,
+                "n_states": int(out.n_states)}
 
     def plan(self, k: int, *, lo: int = 0, hi: Optional[int] = None):
         """The workload's own objective, with the cheapest-feasible budget rule when it has one:

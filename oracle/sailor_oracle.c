@@ -8,6 +8,7 @@
 #include "sailor_oracle.h"
 
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 static uint64_t ceil_div_u64(uint64_t a, uint64_t b) { return (a + b - 1) / b; }
@@ -434,4 +435,246 @@ int32_t orc_search_pruned(const orc_inputs* in, const orc_space* sp, const orc_o
     }
     if (counts) *counts = c;
     return (int32_t)n_hits;
+}
+
+/* ---- per-stage resource assignment by dynamic programming (Sec. 4.2.2, Eq. 1 and the listing) ------
+ *
+ * Everything of a plan is fixed but the GPU type of each stage: P, mbs, tp, recomputation, D, and the
+ * order in which the zones are filled.  Stage i takes D replicas of tp GPUs of one type g_i and is placed
+ * by first fit: the first zone, at or after the zone of stage i-1 in the given order, that still has
+ * D*tp GPUs of that type free.  The recursion gives stage i its resources, solves stages i+1.. on what
+ * is left, and combines the two by T_total (straggler * N_b + slowest synchronisation + sum of the stage
+ * times, and the slowest update as in Sec. 4.3); it keeps the best and remembers it per state.  As in the
+ * paper the rest of the pipeline is solved on its own, so the result is the best plan among those whose
+ * every suffix is the best one for its state: an approximation of the optimum, not the optimum.
+ */
+
+/* the quantities of one stage that the simulator adds up, computed the same way (layer by layer) */
+static void dp_stage(const orc_inputs* in, uint32_t P, uint32_t i, uint32_t g, uint32_t tpi, uint32_t mbs_idx,
+                     uint32_t rc, uint64_t n_b, double* fb, double* upd, uint64_t* params, int* fits) {
+    uint8_t kinds[1024 + 2];
+    const uint32_t nl = stage_layers(in, P, i, kinds);
+    const uint64_t tp = in->tp_values[tpi];
+    double f = 0.0, b = 0.0, u = 0.0;
+    uint64_t par = 0, A = 0, W = 0;
+    for (uint32_t l = 0; l < nl; ++l) {
+        const uint32_t k = kinds[l];
+        f = f + tab4(in, in->fwd, k, g, tpi, mbs_idx);
+        b = b + tab4(in, in->bwd, k, g, tpi, mbs_idx);
+        u = u + tab_upd(in, k, g, tpi);
+        par += in->params[k];
+        A += rc ? tab_act(in, in->act_ckpt, k, tpi, mbs_idx) : tab_act(in, in->act_saved, k, tpi, mbs_idx);
+        const uint64_t w = rc ? tab_act(in, in->act_saved, k, tpi, mbs_idx) : tab_act(in, in->act_work, k, tpi, mbs_idx);
+        if (w > W) W = w;
+    }
+    if (rc) b = b + f;
+    *fb = f + b;
+    *upd = u;
+    *params = par;
+    const uint64_t m = ceil_div_u64(par, tp) * in->mul_factor * in->dtype_size + min_u64((uint64_t)(P - i), n_b) * A + W +
+                       in->reserved[g];
+    *fits = m <= in->capacity[g] && tp <= in->gpus_per_node[g];
+}
+
+/* one message from a stage on (g, z) to the next stage on (g2, z2), both with degree tp */
+static double dp_p2p(const orc_inputs* in, uint32_t g, uint32_t z, uint32_t g2, uint32_t z2, uint32_t tp, uint32_t D,
+                     uint64_t msg) {
+    const uint32_t T = in->n_types, Z = in->n_zones;
+    if (z != z2)
+        return link_time(in->zone_alpha[z * Z + z2], in->zone_inv_bw[z * Z + z2], poly_at(in->zone_bw_poly, z * Z + z2), msg);
+    if (g == g2 && (uint64_t)D * (tp + tp) <= in->gpus_per_node[g])
+        return link_time(in->intra_alpha[z * T + g], in->intra_inv_bw[z * T + g], poly_at(in->intra_bw_poly, z * T + g), msg);
+    const double c1 = link_time(in->inter_alpha[z * T + g], in->inter_inv_bw[z * T + g], poly_at(in->inter_bw_poly, z * T + g), msg);
+    const double c2 = link_time(in->inter_alpha[z * T + g2], in->inter_inv_bw[z * T + g2], poly_at(in->inter_bw_poly, z * T + g2), msg);
+    return max_f64(c1, c2);
+}
+
+/* ring all-reduce of a stage's gradients among its D replicas on (g, z) */
+static double dp_sync(const orc_inputs* in, uint32_t g, uint32_t z, uint32_t tp, uint32_t D, uint64_t params) {
+    if (D <= 1) return 0.0;
+    const uint32_t T = in->n_types, d = z * T + g;
+    const uint64_t gradbytes = ceil_div_u64(params, tp) * in->grad_dtype_size;
+    const int intra = (uint64_t)D * tp <= in->gpus_per_node[g];
+    const double alpha = intra ? in->intra_alpha[d] : in->inter_alpha[d];
+    const double inv = intra ? in->intra_inv_bw[d] : in->inter_inv_bw[d];
+    const double* poly = intra ? poly_at(in->intra_bw_poly, d) : poly_at(in->inter_bw_poly, d);
+    const double steps = (double)(2 * (uint64_t)(D - 1));
+    const double coef = steps / (double)D;
+    if (poly) return (coef * (double)gradbytes) / poly_bw(poly, (double)gradbytes / (double)D) + steps * alpha;
+    return (coef * (double)gradbytes) * inv + steps * alpha;
+}
+
+typedef struct dp_val {
+    int state;                 /* 0 not computed, 1 no plan, 2 plan */
+    int next_g;                /* type of the next stage in the kept plan */
+    double sum, mx, sy, up;    /* sum of stage times, straggler, slowest synchronisation, slowest update */
+} dp_val;
+
+typedef struct dp_key { uint64_t used; uint32_t igz; } dp_key;       /* used: one byte per type; igz: stage, type, zone position */
+
+typedef struct dp_ctx {
+    const orc_inputs* in;
+    const orc_dp_problem* pb;
+    uint32_t T, need, tp;
+    uint64_t n_b, msg;
+    int use_memo;
+    /* per (stage, type) */
+    double fb[ORC_STAGES_MAX][ORC_DP_T_MAX], upd[ORC_STAGES_MAX][ORC_DP_T_MAX];
+    uint64_t params[ORC_STAGES_MAX];
+    int fits[ORC_STAGES_MAX][ORC_DP_T_MAX];
+    /* memo: open addressing */
+    dp_key* keys; dp_val* vals; uint8_t* full; uint64_t cap, count;
+    uint64_t n_states;
+} dp_ctx;
+
+static double dp_value(const dp_ctx* c, const dp_val* v) {
+    return ((v->sum + (double)c->n_b * v->mx) + v->sy) + v->up;
+}
+
+static uint64_t dp_hash(dp_key k) {
+    uint64_t x = k.used * 0x9E3779B97F4A7C15ull ^ ((uint64_t)k.igz * 0xBF58476D1CE4E5B9ull);
+    x ^= x >> 29;
+    return x * 0x94D049BB133111EBull;
+}
+
+static dp_val* memo_slot(dp_ctx* c, dp_key k) {
+    if ((c->count + 1) * 2 > c->cap) {                       /* grow and reinsert */
+        const uint64_t ncap = c->cap ? c->cap * 2 : 1024;
+        dp_key* nk = (dp_key*)calloc(ncap, sizeof(dp_key));
+        dp_val* nv = (dp_val*)calloc(ncap, sizeof(dp_val));
+        uint8_t* nf = (uint8_t*)calloc(ncap, 1);
+        for (uint64_t j = 0; j < c->cap; ++j) {
+            if (!c->full[j]) continue;
+            uint64_t h = dp_hash(c->keys[j]) & (ncap - 1);
+            while (nf[h]) h = (h + 1) & (ncap - 1);
+            nk[h] = c->keys[j]; nv[h] = c->vals[j]; nf[h] = 1;
+        }
+        free(c->keys); free(c->vals); free(c->full);
+        c->keys = nk; c->vals = nv; c->full = nf; c->cap = ncap;
+    }
+    uint64_t h = dp_hash(k) & (c->cap - 1);
+    while (c->full[h]) {
+        if (c->keys[h].used == k.used && c->keys[h].igz == k.igz) return &c->vals[h];
+        h = (h + 1) & (c->cap - 1);
+    }
+    c->full[h] = 1;
+    c->keys[h] = k;
+    memset(&c->vals[h], 0, sizeof(dp_val));
+    c->count++;
+    return &c->vals[h];
+}
+
+/* first zone position at or after `zp` with D*tp GPUs of type g free; `used` counts the stages already
+ * placed in zone position zp, per type (later zones are untouched, earlier ones are not revisited) */
+static int first_fit(const dp_ctx* c, uint32_t zp, const uint8_t* used, uint32_t g) {
+    for (uint32_t p = zp; p < c->pb->n_zones_used; ++p) {
+        const uint64_t have = c->in->avail[c->pb->zone_list[p] * c->T + g];
+        const uint64_t taken = (p == zp) ? (uint64_t)used[g] * c->need : 0;
+        if (have >= taken + c->need) return (int)p;
+    }
+    return -1;
+}
+
+/* best plan for stages i.. given that stage i runs on type g in zone position zp and `used` (which
+ * includes stage i) describes that zone */
+static dp_val solve_suffix(dp_ctx* c, uint32_t i, uint32_t g, uint32_t zp, const uint8_t* used) {
+    const uint32_t P = c->pb->P, z = c->pb->zone_list[zp];
+    dp_val none; memset(&none, 0, sizeof(none)); none.state = 1; none.next_g = -1;
+    if (!c->fits[i][g]) return none;
+    dp_key key; key.used = 0; key.igz = (i << 8) | (g << 4) | zp;
+    for (uint32_t t = 0; t < c->T; ++t) key.used |= (uint64_t)used[t] << (8 * t);
+    if (c->use_memo) {
+        dp_val* slot = memo_slot(c, key);
+        if (slot->state) return *slot;
+    }
+    c->n_states++;
+    dp_val best = none;
+    const double sync = dp_sync(c->in, g, z, c->tp, c->pb->D, c->params[i]);
+    if (i == P - 1) {
+        best.state = 2;
+        best.sum = c->fb[i][g];                  /* the last stage sends nothing */
+        best.mx = c->fb[i][g];
+        best.sy = sync;
+        best.up = c->upd[i][g];
+    } else {
+        for (uint32_t g2 = 0; g2 < c->T; ++g2) {
+            if (!c->fits[i + 1][g2]) continue;
+            const int zp2 = first_fit(c, zp, used, g2);
+            if (zp2 < 0) continue;
+            uint8_t used2[ORC_DP_T_MAX];
+            for (uint32_t t = 0; t < c->T; ++t) used2[t] = ((uint32_t)zp2 == zp) ? used[t] : 0;
+            used2[g2]++;
+            const dp_val nxt = solve_suffix(c, i + 1, g2, (uint32_t)zp2, used2);
+            if (nxt.state != 2) continue;
+            const double cmsg = dp_p2p(c->in, g, z, g2, c->pb->zone_list[zp2], c->tp, c->pb->D, c->msg);
+            const double t = c->fb[i][g] + 2.0 * cmsg;
+            dp_val cand;
+            cand.state = 2;
+            cand.next_g = (int)g2;
+            cand.sum = t + nxt.sum;
+            cand.mx = max_f64(t, nxt.mx);
+            cand.sy = max_f64(sync, nxt.sy);
+            cand.up = max_f64(c->upd[i][g], nxt.up);
+            if (best.state != 2 || dp_value(c, &cand) < dp_value(c, &best)) best = cand;
+        }
+    }
+    if (c->use_memo) *memo_slot(c, key) = best;
+    return best;
+}
+
+int orc_solve_dp(const orc_inputs* in, const orc_dp_problem* pb, int use_memo, orc_dp_result* out) {
+    memset(out, 0, sizeof(*out));
+    const uint32_t P = pb->P, T = in->n_types;
+    if (P < 1 || P > ORC_STAGES_MAX || T > ORC_DP_T_MAX || pb->n_zones_used < 1 || pb->n_zones_used > 16 || pb->D < 1) return -1;
+    const uint64_t mbs = in->mbs_values[pb->mbs_idx];
+    const uint32_t tp = in->tp_values[pb->tp_idx];
+    if (in->gbs % ((uint64_t)pb->D * mbs) != 0 || in->heads % tp != 0) return 0;      /* no valid plan in this problem */
+    dp_ctx* c = (dp_ctx*)calloc(1, sizeof(dp_ctx));
+    c->in = in; c->pb = pb; c->T = T; c->tp = tp; c->need = pb->D * tp;
+    c->n_b = in->gbs / ((uint64_t)pb->D * mbs);
+    c->msg = in->p2p_bytes[pb->mbs_idx];
+    c->use_memo = use_memo;
+    for (uint32_t i = 0; i < P; ++i)
+        for (uint32_t g = 0; g < T; ++g) {
+            uint64_t par;
+            dp_stage(in, P, i, g, pb->tp_idx, pb->mbs_idx, pb->rc, c->n_b, &c->fb[i][g], &c->upd[i][g], &par, &c->fits[i][g]);
+            c->params[i] = par;
+        }
+    /* stage 0: every type, placed by first fit from the first zone of the order */
+    dp_val best; memset(&best, 0, sizeof(best)); best.state = 1;
+    int best_g = -1, best_zp = -1;
+    const uint8_t nothing[ORC_DP_T_MAX] = {0};
+    for (uint32_t g = 0; g < T; ++g) {
+        const int zp = first_fit(c, 0, nothing, g);
+        if (zp < 0) continue;
+        uint8_t used[ORC_DP_T_MAX] = {0};
+        used[g] = 1;
+        const dp_val v = solve_suffix(c, 0, g, (uint32_t)zp, used);
+        if (v.state != 2) continue;
+        if (best.state != 2 || dp_value(c, &v) < dp_value(c, &best)) { best = v; best_g = (int)g; best_zp = zp; }
+    }
+    out->n_states = c->n_states;
+    if (best.state == 2) {
+        out->found = 1;
+        out->value = dp_value(c, &best);
+        /* walk the kept choices to write the plan out */
+        orc_plan* pl = &out->plan;
+        pl->P = P; pl->mbs_idx = pb->mbs_idx; pl->rc = pb->rc; pl->D = pb->D;
+        uint8_t used[ORC_DP_T_MAX] = {0};
+        uint32_t g = (uint32_t)best_g, zp = (uint32_t)best_zp;
+        used[g] = 1;
+        dp_val v = best;
+        for (uint32_t i = 0; i < P; ++i) {
+            pl->type[i] = g; pl->zone[i] = pb->zone_list[zp]; pl->tp_idx[i] = pb->tp_idx;
+            if (i + 1 == P) break;
+            const uint32_t g2 = (uint32_t)v.next_g;
+            const int zp2 = first_fit(c, zp, used, g2);
+            if ((uint32_t)zp2 != zp) memset(used, 0, sizeof(used));
+            used[g2]++;
+            g = g2; zp = (uint32_t)zp2;
+            v = solve_suffix(c, i + 1, g, zp, used);
+        }
+    }
+    free(c->keys); free(c->vals); free(c->full); free(c);
+    return 0;
 }

@@ -177,4 +177,42 @@ typedef struct orc_pruned_counts {
 int32_t orc_search_pruned(const orc_inputs* in, const orc_space* sp, const orc_objective* obj, uint32_t modes,
                           uint32_t k, orc_hit* hits, orc_pruned_counts* counts);
 
+
+/* ---- per-stage resource assignment by dynamic programming (Sec. 4.2.2: Eq. 1, T_total, the listing) ----
+ *
+ * A problem fixes P, mbs, tp, recomputation, D and the order in which zones are filled (the paper's
+ * planner loops over region combinations outside the recursion).  The recursion chooses the GPU type of
+ * each stage (all D replicas of a stage alike); a stage goes to the first zone, at or after the
+ * previous stage's zone in the order, with D*tp GPUs of its type free.  For stage i on type g it tries
+ * every type g' for stage i+1 in ascending order, solves stages i+1.. for what is left (remembered per
+ * state: stage, type, zone position, stages per type already placed in that zone), and combines:
+ *     t     = (f_i + b_i) + 2 * c(i -> i+1)            [the last stage: f + b]
+ *     sum   = t + sum_rest        mx = max(t, mx_rest)
+ *     sy    = max(sync_i, sy_rest)        up = max(u_i, up_rest)
+ *     value = ((sum + N_b * mx) + sy) + up              [T_total of Sec. 4.2.2 plus the update of Sec. 4.3]
+ * keeping the smallest value (the first found among equals).  The rest of the pipeline is always the best
+ * one for its own state, as in Eq. 1, so the result can be worse than the true optimum over all type
+ * sequences.  Pins: equality with a plain recursion without the memory; a hand-worked case in which the
+ * recursion provably misses the optimum by a known amount; brute force over all type sequences (never
+ * better than the optimum, equal for P <= 2, the plan obeys first fit and availability, and the
+ * simulator reproduces the value from the plan).  The budget loop of Sec. 4.2.3 is not part of it. */
+#define ORC_DP_T_MAX 8
+
+typedef struct orc_dp_problem {
+    uint32_t P, mbs_idx, tp_idx, rc, D;
+    uint32_t n_zones_used;
+    uint32_t zone_list[16];      /* zones in the order they are filled */
+} orc_dp_problem;
+
+typedef struct orc_dp_result {
+    int32_t found;               /* 0: no plan fits */
+    uint32_t _pad;
+    double value;                /* the recursion's own value of the kept plan (sums run from the last stage) */
+    uint64_t n_states;           /* states solved (not counting remembered ones) */
+    orc_plan plan;
+} orc_dp_result;
+
+/* returns 0, or -1 for sizes beyond the limits; use_memo = 0 is the plain recursion */
+int orc_solve_dp(const orc_inputs* in, const orc_dp_problem* pb, int use_memo, orc_dp_result* out);
+
 #endif
