@@ -315,6 +315,76 @@ int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objec
 int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint32_t k,
                         sailor_result* topk, uint32_t* n_found, sailor_stats* stats);
 
+/* ---- per-stage GPU types by dynamic programming (Sec. 4.2.2: Eq. 1, T_total, the listing) --------
+ *
+ * sailor_plan varies the GPU type and zone of at most SAILOR_SEG_MAX segments of a pipeline.  This
+ * entry point gives every stage its own GPU type, the way the paper's planner does: by a recursion
+ * over the stages that hands stage i its resources, solves stages i+1.. on what is left, and combines
+ * the two by T_total.
+ *
+ * A problem is one configuration (P, mbs, tp, rc, D) of the space (seg_max is ignored) together
+ * with one zone order, the order in which zones are filled (the paper's planner loops over region
+ * combinations outside the recursion; H5 keeps a stage inside one zone).  All D replicas of a stage
+ * use the same GPU type and tp.  A stage goes to the first zone, at or after the previous stage's
+ * zone in the order, that still has D*tp GPUs of its type free.  For stage i on type g the
+ * recursion tries every type g' for stage i+1 in ascending order, takes the best plan of stages
+ * i+1.. for the state that results, and combines (binary64, this order, no fused multiply-add):
+ *     t     = (f_i + b_i) + 2 * c(i -> i+1)                 the last stage: f + b
+ *     sum   = t + sum_rest          mx = max(t, mx_rest)
+ *     sy    = max(sync_i, sy_rest)  up = max(u_i, up_rest)
+ *     value = ((sum + N_b * mx) + sy) + up
+ * keeping the smallest value (the first among equals).  As in Eq. 1 the rest of the pipeline is
+ * the best one for its own state, so the plan found can be worse than the best of all type
+ * sequences.  `value` sums the stage times from the last stage backwards; t_iter, cost and
+ * peak_mem of a result are the simulator's figures for the written-out plan (stage order), equal
+ * to value up to rounding.  The budget loop of Sec. 4.2.3 is not implemented: the objective is
+ * iteration time (maximum throughput) without a constraint.
+ *
+ * On the device every problem is a dense table over its states (stage, type, zone position,
+ * stages per type already placed in that zone; a type with room for all P stages in a zone is not
+ * counted there), filled from the last stage to the first, one launch per stage for all problems
+ * of a batch together; batches are cut so that the tables fit `workspace_bytes`. */
+typedef struct sailor_zone_order {
+    uint8_t n;                          /* 1 .. SAILOR_Z_MAX zones, each at most once                */
+    uint8_t zone[SAILOR_Z_MAX];
+    uint8_t _pad[3];
+} sailor_zone_order;
+
+typedef struct sailor_dp_result {
+    uint32_t config;                    /* configuration index: (((p * n_mbs + mbs) * n_tp + tp) * n_rc + rc) * n_d + d,
+                                           positions in the space's lists                             */
+    uint32_t order;                     /* index into `orders`                                        */
+    double   value;                     /* the recursion's value of the plan                          */
+    double   t_iter, cost;              /* the simulator's figures for the plan (Sec. 4.3)            */
+    uint64_t peak_mem;
+    uint32_t status;                    /* the simulator's status of the plan: 0                      */
+    uint8_t  P, mbs_idx, tp_idx, rc;
+    uint16_t D;
+    uint16_t _pad;
+    uint8_t  type[SAILOR_P_MAX];        /* GPU type of every stage                                    */
+    uint8_t  zone[SAILOR_P_MAX];        /* zone of every stage                                        */
+} sailor_dp_result;
+
+typedef struct sailor_dp_stats {
+    uint64_t n_problems;                /* configurations x zone orders                               */
+    uint64_t n_solved;                  /* problems that have a plan                                  */
+    uint64_t n_states;                  /* table entries filled (all problems, all stages)            */
+    uint64_t workspace_used;            /* bytes of the largest batch                                 */
+    float    kernel_ms;
+    uint32_t n_launches, n_batches, _pad;
+} sailor_dp_stats;
+
+/* Solve every problem of `s` x `orders` and return the k best plans by (value, problem index =
+ * config * n_orders + order) ascending; *n_found <= k.  `topk` is a HOST array of k records;
+ * `stats` may be NULL.  Uses the availability last set.  `workspace_bytes` bounds the device memory
+ * of the tables (0 = 8 GiB); it is allocated on first use and kept by the context (grow-only).
+ * Errors: E_ARG (null, k == 0, n_orders == 0, a zone twice or out of range), E_RANGE (k >
+ * SAILOR_K_MAX, space limits as sailor_plan, a single problem whose tables exceed the workspace or
+ * 2^31 entries per stage), E_NOMEM, E_CUDA. */
+int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders, uint32_t n_orders,
+                   uint64_t workspace_bytes, uint32_t k, sailor_dp_result* topk, uint32_t* n_found,
+                   sailor_dp_stats* stats);
+
 const char* sailor_strerror(int code);
 int sailor_last_cuda_error(const sailor_ctx* ctx);   /* cudaError_t of the last E_CUDA      */
 

@@ -20,7 +20,7 @@ FLAG_EVAL_ALL, FLAG_DEGREE_ORDER, FLAG_MIN_TP_ONLY = 1, 2, 4
 
 EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
            "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_plan_noalloc",
-           "sailor_strerror", "sailor_last_cuda_error")
+           "sailor_plan_dp", "sailor_strerror", "sailor_last_cuda_error")
 
 _dp, _u64p, _u32p, _u16p = C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.POINTER(C.c_uint16)
 
@@ -79,7 +79,25 @@ class Stats(C.Structure):
                 ("n_configs", C.c_uint32), ("n_configs_evaluated", C.c_uint32)]
 
 
+class ZoneOrder(C.Structure):
+    _fields_ = [("n", C.c_uint8), ("zone", C.c_uint8 * Z_MAX), ("_pad", C.c_uint8 * 3)]
+
+
+class DpResult(C.Structure):
+    _fields_ = [("config", C.c_uint32), ("order", C.c_uint32), ("value", C.c_double), ("t_iter", C.c_double),
+                ("cost", C.c_double), ("peak_mem", C.c_uint64), ("status", C.c_uint32), ("P", C.c_uint8),
+                ("mbs_idx", C.c_uint8), ("tp_idx", C.c_uint8), ("rc", C.c_uint8), ("D", C.c_uint16),
+                ("_pad", C.c_uint16), ("type", C.c_uint8 * P_MAX), ("zone", C.c_uint8 * P_MAX)]
+
+
+class DpStats(C.Structure):
+    _fields_ = [("n_problems", C.c_uint64), ("n_solved", C.c_uint64), ("n_states", C.c_uint64),
+                ("workspace_used", C.c_uint64), ("kernel_ms", C.c_float), ("n_launches", C.c_uint32),
+                ("n_batches", C.c_uint32), ("_pad", C.c_uint32)]
+
+
 assert C.sizeof(PlanRec) == 72 and C.sizeof(Result) == 120 and C.sizeof(Space) == 152
+assert C.sizeof(ZoneOrder) == 12 and C.sizeof(DpResult) == 248 and C.sizeof(DpStats) == 48
 assert C.sizeof(Objective) == 32 and C.sizeof(Stats) == 96
 
 # numpy view of an array of plan records (same 72-byte layout)
@@ -122,6 +140,8 @@ def load() -> C.CDLL:
     L.sailor_plan_range.argtypes = [vp, C.POINTER(Space), C.POINTER(Objective), C.c_uint64, C.c_uint64, C.c_uint32,
                                     C.POINTER(Result), _u32p, C.POINTER(Stats)]
     L.sailor_plan_noalloc.argtypes = L.sailor_plan.argtypes
+    L.sailor_plan_dp.argtypes = [vp, C.POINTER(Space), C.POINTER(ZoneOrder), C.c_uint32, C.c_uint64, C.c_uint32,
+                                 C.POINTER(DpResult), _u32p, C.POINTER(DpStats)]
     L.sailor_strerror.argtypes = [C.c_int]
     L.sailor_strerror.restype = C.c_char_p
     L.sailor_last_cuda_error.argtypes = [vp]
@@ -278,6 +298,24 @@ def sailor_plan_noalloc(ctx, space: Space, obj: Objective, k: int):
     st = Stats()
     _check(load().sailor_plan_noalloc(ctx, C.byref(space), C.byref(obj), k, res, C.byref(n), C.byref(st)),
            "sailor_plan_noalloc", ctx)
+    return list(res[: n.value]), st
+
+
+def sailor_plan_dp(ctx, space: Space, zone_orders, k: int, workspace_bytes: int = 0):
+    """Per-stage GPU types by dynamic programming for every configuration of the space and every zone
+    order (a list of zone lists): the k best plans by the recursion's value, and the statistics."""
+    orders = (ZoneOrder * len(zone_orders))()
+    for j, zl in enumerate(zone_orders):
+        if len(zl) > Z_MAX:
+            raise ValueError("a zone order holds at most %d zones" % Z_MAX)
+        orders[j].n = len(zl)
+        for q, z in enumerate(zl):
+            orders[j].zone[q] = int(z)
+    res = (DpResult * k)()
+    n = C.c_uint32()
+    st = DpStats()
+    _check(load().sailor_plan_dp(ctx, C.byref(space), orders, len(zone_orders), workspace_bytes, k, res, C.byref(n),
+                                 C.byref(st)), "sailor_plan_dp", ctx)
     return list(res[: n.value]), st
 
 

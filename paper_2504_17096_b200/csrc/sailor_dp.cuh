@@ -1,0 +1,344 @@
+// Per-stage GPU types by dynamic programming (Sailor Sec. 4.2.2: Eq. 1 and T_total).
+//
+// A problem is one configuration (P, mbs, tp, rc, D) with one zone order.  Its states are
+// (stage i, type g of stage i, zone position zp of stage i, u = stages per type already placed in
+// that zone, stage i included).  Zones before zp are never revisited and zones after it are
+// untouched (first fit), so nothing else of the past matters.  A type that a zone could give to all
+// P stages is not counted in u.  States are laid out densely: for every zone position and type a
+// slice of S[zp] entries indexed by u in mixed radix.  The value of a state is the best plan of
+// stages i.. from it: (sum of stage times, straggler, slowest synchronisation, slowest update).
+//
+// The tables are filled from the last stage to the first.  One launch handles one stage distance
+// from the end for every problem of a batch (problems are sorted by depth, so the launch for
+// distance s covers a prefix of the block list); a thread owns one state and tries every type for
+// the next stage.  Per-configuration quantities (stage times per type, synchronisation per digit,
+// message times per digit pair) are formed once per configuration by dp_tables_kernel.
+#pragma once
+
+#include "sailor_plan_kernels.cuh"
+
+namespace sailor {
+
+constexpr int DP_THREADS = 256;
+constexpr uint8_t DP_NONE = 255;
+
+struct DpVal {                       // best plan of stages i.. from a state; sum = +inf: there is none
+    double sum, mx, sy, up;
+};
+
+struct DpProblem {
+    uint64_t val_off;                // first entry of this problem in the two level buffers of its batch
+    uint64_t choice_off;             // first byte of its choices: [stage][entry]
+    uint32_t config, order, index;   // index = config * n_orders + order
+    uint32_t n_lvl;                  // entries per stage
+    uint32_t P, nz, need;            // need = D * tp GPUs per stage
+    uint8_t zone[SAILOR_Z_MAX];      // zone of each position of the order
+    uint8_t cap[SAILOR_Z_MAX][SAILOR_T_MAX];       // stages a (position, type) can host, saturated at 255
+    uint8_t first_later[SAILOR_Z_MAX][SAILOR_T_MAX];   // first position after zp that can host a stage of the type
+    uint32_t stride[SAILOR_Z_MAX][SAILOR_T_MAX];   // mixed-radix stride of a counted type; 0: not counted
+    uint32_t S[SAILOR_Z_MAX];        // entries of one (position, type) slice
+    uint32_t zp_base[SAILOR_Z_MAX + 1];            // first entry of each position's T slices
+};
+
+struct DpResult {                    // per problem, written by dp_finish_kernel
+    double value;                    // +inf: no plan
+    uint8_t type[SAILOR_P_MAX];
+    uint8_t zone[SAILOR_P_MAX];
+};
+
+// Per-configuration tables in global memory, one block of `stride` doubles per configuration:
+//   fb[p_max][T], upd[p_max][T], sync[p_max][R], c2x[R][R] (2 * message time, [next digit][this digit]),
+//   then ok[p_max] (u32 bit g: stage fits type g and tp fits its node), n_b (u64), valid (u32).
+struct DpTabLayout {
+    uint32_t p_max, T, R;
+    __host__ __device__ size_t off_fb() const { return 0; }
+    __host__ __device__ size_t off_upd() const { return (size_t)p_max * T; }
+    __host__ __device__ size_t off_sync() const { return 2 * (size_t)p_max * T; }
+    __host__ __device__ size_t off_c2x() const { return 2 * (size_t)p_max * T + (size_t)p_max * R; }
+    __host__ __device__ size_t off_ok() const { return off_c2x() + (size_t)R * R; }               // in doubles
+    __host__ __device__ size_t off_nb() const { return off_ok() + (p_max + 1) / 2; }
+    __host__ __device__ size_t stride() const { return off_nb() + 2; }
+};
+
+__global__ void __launch_bounds__(DP_THREADS)
+dp_tables_kernel(const unsigned char* __restrict__ blob, SpaceDesc sp, uint32_t n_config, DpTabLayout lay,
+                 double* __restrict__ tabs) {
+    __shared__ uint64_t s_params[SAILOR_P_MAX];
+    __shared__ uint32_t s_ok[SAILOR_P_MAX];
+    TabView v;
+    v.bind(blob, blob);
+    const TabHdr* h = v.h;
+    const uint32_t T = h->T, R = h->R, tid = threadIdx.x;
+    for (uint32_t c = blockIdx.x; c < n_config; c += gridDim.x) {
+        __syncthreads();
+        const Config k = config_of(sp, c);
+        double* tab = tabs + (size_t)c * lay.stride();
+        const uint32_t tp = h->tp_values[k.tpi];
+        const uint64_t dm = (uint64_t)k.D * h->mbs_values[k.mi];
+        const bool valid = k.D >= 1 && h->gbs % dm == 0 && h->heads % tp == 0;
+        const uint64_t n_b = valid ? h->gbs / dm : 0;
+        if (tid == 0) {
+            *reinterpret_cast<uint64_t*>(tab + lay.off_nb()) = n_b;
+            *reinterpret_cast<uint32_t*>(tab + lay.off_nb() + 1) = valid ? 1u : 0u;
+        }
+        for (uint32_t i = tid; i < SAILOR_P_MAX; i += DP_THREADS) s_ok[i] = 0;
+        __syncthreads();
+        if (!valid) continue;
+        const uint32_t P = k.P, base = h->n_blocks / P, extra = h->n_blocks % P;
+        for (uint32_t x = tid; x < P * T; x += DP_THREADS) {
+            const uint32_t i = x / T, g = x % T;
+            const uint32_t nb = base + (i < extra ? 1u : 0u);
+            const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
+            const StageTimes st = stage_times(v, g, k.tpi, k.mi, nb, e, hd);
+            const double b = k.rc ? add_rn(st.b, st.f) : st.b;
+            tab[lay.off_fb() + x] = add_rn(st.f, b);
+            tab[lay.off_upd() + x] = st.u;
+            const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
+            const StageMem sm = stage_memory(v, k.tpi, k.mi, k.rc, nb, e, hd, inflight);
+            if (sm.mem + h->reserved[g] <= h->capacity[g] && tp <= h->gpn[g]) atomicOr(&s_ok[i], 1u << g);
+            if (g == 0) s_params[i] = sm.params;
+        }
+        __syncthreads();
+        const double steps = (double)(2 * (uint64_t)(k.D - 1)), coef = steps / (double)k.D;
+        for (uint32_t x = tid; x < P * R; x += DP_THREADS) {
+            const uint32_t i = x / R, d = x % R;
+            tab[lay.off_sync() + x] = k.D > 1 ? allreduce_time(v, d % T, d, tp, k.D, s_params[i], steps, coef) : 0.0;
+        }
+        const double msg = (double)v.p2p[k.mi];
+        for (uint32_t x = tid; x < R * R; x += DP_THREADS) {
+            const uint32_t dn = x / R, d = x % R;          // [next][this]
+            tab[lay.off_c2x() + x] = mul_rn(2.0, boundary_time(v, d % T, d / T, tp, dn % T, dn / T, tp, k.D, msg));
+        }
+        for (uint32_t i = tid; i < P; i += DP_THREADS) reinterpret_cast<uint32_t*>(tab + lay.off_ok())[i] = s_ok[i];
+    }
+}
+
+// Where does a stage of type g2 go when the previous stage sits at position zp with counts u?
+// Returns the position (DP_NONE: nowhere) and the entry index of the state that results.
+struct DpMove { uint32_t zp, entry; };
+
+__device__ __forceinline__ DpMove dp_move(const DpProblem& pb, uint32_t zp, uint32_t ui, uint32_t g2) {
+    DpMove m;
+    const uint32_t st = pb.stride[zp][g2], cap = pb.cap[zp][g2];
+    bool here;
+    if (st == 0) here = cap >= 1;                                  // not counted: room for every stage, or none at all
+    else here = (ui / st) % (cap + 1u) < cap;
+    if (here) {
+        m.zp = zp;
+        m.entry = pb.zp_base[zp] + g2 * pb.S[zp] + ui + st;
+        return m;
+    }
+    const uint32_t p = pb.first_later[zp][g2];
+    m.zp = p;
+    m.entry = p == DP_NONE ? 0u : pb.zp_base[p] + g2 * pb.S[p] + pb.stride[p][g2];      // the new zone holds this stage only
+    return m;
+}
+
+struct DpLevelParams {
+    const DpProblem* problems;
+    const uint32_t* blk_problem;     // block -> problem of the batch
+    const uint32_t* blk_first;       // block -> first entry it covers
+    const double* tabs;
+    DpVal* val[2];                   // level buffers; stage i lives in val[(P - 1 - i) & 1]
+    uint8_t* choice;
+    DpTabLayout lay;
+    uint32_t T;
+    uint32_t dist;                   // stage i = P - 1 - dist
+};
+
+__global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_constant__ DpLevelParams lp) {
+    __shared__ DpProblem pb;
+    const uint32_t tid = threadIdx.x;
+    {
+        const DpProblem* src = lp.problems + lp.blk_problem[blockIdx.x];
+        for (uint32_t x = tid; x < sizeof(DpProblem) / 4; x += DP_THREADS)
+            reinterpret_cast<uint32_t*>(&pb)[x] = reinterpret_cast<const uint32_t*>(src)[x];
+    }
+    __syncthreads();
+    const uint32_t e = lp.blk_first[blockIdx.x] + tid;
+    if (e >= pb.n_lvl) return;
+    const uint32_t T = lp.T, P = pb.P, i = P - 1 - lp.dist;
+    const double* tab = lp.tabs + (size_t)pb.config * lp.lay.stride();
+    const uint32_t* okv = reinterpret_cast<const uint32_t*>(tab + lp.lay.off_ok());
+    const double nb = (double)*reinterpret_cast<const uint64_t*>(tab + lp.lay.off_nb());
+    // entry -> (zone position, type, counts)
+    uint32_t zp = 0;
+    while (zp + 1 < pb.nz && e >= pb.zp_base[zp + 1]) ++zp;
+    const uint32_t g = (e - pb.zp_base[zp]) / pb.S[zp], ui = (e - pb.zp_base[zp]) % pb.S[zp];
+    DpVal* cur = lp.val[lp.dist & 1] + pb.val_off;
+    const DpVal* nxt = lp.val[(lp.dist & 1) ^ 1] + pb.val_off;
+    uint8_t* choice = lp.choice + pb.choice_off + (size_t)i * pb.n_lvl;
+    DpVal best;
+    best.sum = make_inf(); best.mx = best.sy = best.up = 0.0;
+    uint8_t pick = DP_NONE;
+    // a state holds stage i itself: its type must be usable there and, when counted, counted at least once
+    const uint32_t st_g = pb.stride[zp][g];
+    const bool self = ((okv[i] >> g) & 1u) && pb.cap[zp][g] >= 1 && (st_g == 0 || (ui / st_g) % (pb.cap[zp][g] + 1u) >= 1);
+    if (self) {
+        const uint32_t d = pb.zone[zp] * T + g;
+        const double fb = tab[lp.lay.off_fb() + i * T + g], upd = tab[lp.lay.off_upd() + i * T + g];
+        const double sync = tab[lp.lay.off_sync() + (size_t)i * lp.lay.R + d];
+        if (lp.dist == 0) {                                      // the last stage sends nothing
+            best.sum = fb; best.mx = fb; best.sy = sync; best.up = upd;
+        } else {
+            double best_v = make_inf();
+            const uint32_t ok_next = okv[i + 1];
+            for (uint32_t g2 = 0; g2 < T; ++g2) {
+                if (!((ok_next >> g2) & 1u)) continue;
+                const DpMove mv = dp_move(pb, zp, ui, g2);
+                if (mv.zp == DP_NONE) continue;
+                const DpVal n = nxt[mv.entry];
+                if (!(n.sum < make_inf())) continue;
+                const uint32_t d2 = pb.zone[mv.zp] * T + g2;
+                const double t = add_rn(fb, tab[lp.lay.off_c2x() + (size_t)d2 * lp.lay.R + d]);
+                DpVal c;
+                c.sum = add_rn(t, n.sum);
+                c.mx = dmax(t, n.mx);
+                c.sy = dmax(sync, n.sy);
+                c.up = dmax(upd, n.up);
+                const double val = add_rn(add_rn(add_rn(c.sum, mul_rn(nb, c.mx)), c.sy), c.up);
+                if (pick == DP_NONE || val < best_v) { best = c; best_v = val; pick = (uint8_t)g2; }
+            }
+        }
+    }
+    cur[e] = best;
+    choice[e] = pick;
+}
+
+// Stage 0 and the walk through the kept choices: one thread per problem.
+struct DpFinishParams {
+    const DpProblem* problems;
+    const double* tabs;
+    const DpVal* val[2];
+    const uint8_t* choice;
+    DpResult* results;               // indexed by problem index
+    DpTabLayout lay;
+    uint32_t n_problems, T;
+};
+
+__global__ void __launch_bounds__(128) dp_finish_kernel(const __grid_constant__ DpFinishParams fp) {
+    const uint32_t x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= fp.n_problems) return;
+    const DpProblem& pb = fp.problems[x];
+    DpResult& out = fp.results[pb.index];
+    const uint32_t T = fp.T, P = pb.P;
+    const double* tab = fp.tabs + (size_t)pb.config * fp.lay.stride();
+    const uint32_t* okv = reinterpret_cast<const uint32_t*>(tab + fp.lay.off_ok());
+    const double nb = (double)*reinterpret_cast<const uint64_t*>(tab + fp.lay.off_nb());
+    const DpVal* lvl0 = fp.val[(P - 1) & 1] + pb.val_off;
+    double best_v = make_inf();
+    uint32_t g = DP_NONE, zp = 0, entry = 0;
+    for (uint32_t g0 = 0; g0 < T; ++g0) {                    // stage 0 by first fit from the first zone of the order
+        if (!((okv[0] >> g0) & 1u)) continue;
+        const uint32_t p = pb.cap[0][g0] >= 1 ? 0u : pb.first_later[0][g0];
+        if (p == DP_NONE) continue;
+        const uint32_t e = pb.zp_base[p] + g0 * pb.S[p] + pb.stride[p][g0];
+        const DpVal v = lvl0[e];
+        if (!(v.sum < make_inf())) continue;
+        const double val = add_rn(add_rn(add_rn(v.sum, mul_rn(nb, v.mx)), v.sy), v.up);
+        if (g == DP_NONE || val < best_v) { best_v = val; g = g0; zp = p; entry = e; }
+    }
+    out.value = best_v;
+    if (g == DP_NONE) return;
+    for (uint32_t i = 0; i < P; ++i) {
+        out.type[i] = (uint8_t)g;
+        out.zone[i] = pb.zone[zp];
+        if (i + 1 == P) break;
+        const uint8_t g2 = fp.choice[pb.choice_off + (size_t)i * pb.n_lvl + entry];
+        const uint32_t ui = (entry - pb.zp_base[zp]) % pb.S[zp];
+        const DpMove mv = dp_move(pb, zp, ui, g2);
+        g = g2; zp = mv.zp; entry = mv.entry;
+    }
+}
+
+// The k best problems by (value, problem index), then the simulator's figures for their plans.
+struct DpSelectParams {
+    const unsigned char* blob;
+    const uint16_t* avail;
+    const DpResult* results;
+    sailor_dp_result* out;           // [k] device
+    unsigned long long* counters;    // [0] problems with a plan, [1] number written to out
+    SpaceDesc sp;
+    uint32_t n_problems, n_orders, k;
+};
+
+constexpr int DP_SELECT_THREADS = 512;
+
+__global__ void __launch_bounds__(DP_SELECT_THREADS) dp_select_kernel(const __grid_constant__ DpSelectParams sp) {
+    __shared__ Hit s_hits[DP_SELECT_THREADS / 32][SAILOR_K_MAX];
+    __shared__ uint32_t s_cnt[R_MAX][DP_SELECT_THREADS / 32];
+    __shared__ uint32_t s_n;
+    __shared__ unsigned long long s_solved;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = DP_SELECT_THREADS / 32;
+    if (tid == 0) s_solved = 0;
+    __syncthreads();
+    WarpTopK top;
+    top.init();
+    uint32_t solved = 0;
+    for (uint32_t base = warp * 32; base < sp.n_problems; base += nw * 32) {
+        const uint32_t j = base + lane;
+        const double v = j < sp.n_problems ? sp.results[j].value : make_inf();
+        const bool have = v < make_inf();
+        solved += have;
+        const bool want = have && v <= top.thr_score;
+        if (__any_sync(FULL, want)) top.offer(want, v, j, sp.k, lane);
+    }
+#pragma unroll
+    for (int o = 16; o; o >>= 1) solved += __shfl_xor_sync(FULL, solved, o);
+    if (lane == 0 && solved) atomicAdd(&s_solved, (unsigned long long)solved);
+    s_hits[warp][lane].score = top.score;
+    s_hits[warp][lane].flat = top.flat;
+    __syncthreads();
+    for (uint32_t step = 1; step < nw; step <<= 1) {
+        if ((warp & (2 * step - 1)) == 0 && warp + step < nw) {
+            top.merge_sorted(s_hits[warp + step][lane].score, s_hits[warp + step][lane].flat, sp.k, lane);
+            s_hits[warp][lane].score = top.score;
+            s_hits[warp][lane].flat = top.flat;
+        }
+        __syncthreads();
+    }
+    if (warp == 0) {
+        const uint32_t n = __popc(__ballot_sync(FULL, lane < sp.k && top.flat != ~0ull));
+        if (lane == 0) {
+            s_n = n;
+            sp.counters[0] = s_solved;
+            sp.counters[1] = n;
+        }
+    }
+    __syncthreads();
+    TabView v;
+    v.bind(sp.blob, sp.blob);
+    for (uint32_t j = warp; j < s_n; j += nw) {
+        if (lane != 0) continue;
+        const uint32_t idx = (uint32_t)s_hits[0][j].flat;
+        const DpResult& r = sp.results[idx];
+        const uint32_t c = idx / sp.n_orders;
+        const Config k = config_of(sp.sp, c);
+        sailor_dp_result o;
+        for (int q = 0; q < (int)sizeof(o); ++q) reinterpret_cast<unsigned char*>(&o)[q] = 0;
+        o.config = c;
+        o.order = idx % sp.n_orders;
+        o.value = r.value;
+        o.P = (uint8_t)k.P; o.mbs_idx = (uint8_t)k.mi; o.tp_idx = (uint8_t)k.tpi; o.rc = (uint8_t)k.rc; o.D = (uint16_t)k.D;
+        sailor_run runs[SAILOR_P_MAX];
+        uint32_t n_runs = 0;
+        for (uint32_t i = 0; i < k.P; ++i) {
+            o.type[i] = r.type[i];
+            o.zone[i] = r.zone[i];
+            if (n_runs && runs[n_runs - 1].type == r.type[i] && runs[n_runs - 1].zone == r.zone[i]) runs[n_runs - 1].n_stages++;
+            else {
+                runs[n_runs].type = r.type[i]; runs[n_runs].zone = r.zone[i];
+                runs[n_runs].tp_idx = (uint8_t)k.tpi; runs[n_runs].n_stages = 1;
+                ++n_runs;
+            }
+        }
+        const SimOut so = simulate_runs(v, sp.avail, k.P, n_runs, k.D, k.mi, k.rc, runs, SAILOR_P_MAX, &s_cnt[0][warp], nw);
+        o.t_iter = so.t_iter;
+        o.cost = so.cost;
+        o.peak_mem = so.peak_mem;
+        o.status = so.status;
+        sp.out[j] = o;
+    }
+}
+
+}  // namespace sailor

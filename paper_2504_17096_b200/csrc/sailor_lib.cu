@@ -8,7 +8,9 @@
 #include <new>
 #include <vector>
 
-#include "sailor_plan_kernels.cuh"
+#include <algorithm>
+
+#include "sailor_dp.cuh"
 
 using namespace sailor;
 
@@ -198,6 +200,9 @@ struct sailor_ctx {
     // explicit-batch staging (grow-only)
     unsigned char* d_stage = nullptr;
     size_t stage_bytes = 0;
+    // tables of the dynamic-programming search (grow-only)
+    unsigned char* d_dp = nullptr;
+    size_t dp_bytes = 0;
 };
 
 namespace {
@@ -746,6 +751,7 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->space.d_cfg_best);
     cudaFree(ctx->space.d_groups);
     cudaFree(ctx->d_stage);
+    cudaFree(ctx->d_dp);
     if (ctx->ev0) cudaEventDestroy(ctx->ev0);
     if (ctx->ev1) cudaEventDestroy(ctx->ev1);
     delete ctx;
@@ -1106,6 +1112,260 @@ extern "C" int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const
         CU(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
         stats->kernel_ms = ms;
         stats->n_launches = launches;
+    }
+    return SAILOR_OK;
+}
+
+// ---- per-stage GPU types by dynamic programming ---------------------------------------------------
+
+namespace {
+
+struct Bump {                       // carves 256-byte aligned pieces out of one device buffer
+    unsigned char* base;
+    size_t at = 0;
+    template <typename T>
+    T* take(size_t n) {
+        T* p = reinterpret_cast<T*>(base + at);
+        at += (n * sizeof(T) + 255) & ~(size_t)255;
+        return p;
+    }
+};
+
+size_t padded(size_t bytes) { return (bytes + 255) & ~(size_t)255; }
+
+}  // namespace
+
+extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders,
+                              uint32_t n_orders, uint64_t workspace_bytes, uint32_t k, sailor_dp_result* topk,
+                              uint32_t* n_found, sailor_dp_stats* stats) {
+    if (!ctx || !s || !orders || !topk || !n_found || k == 0 || n_orders == 0) return SAILOR_E_ARG;
+    if (k > SAILOR_K_MAX) return SAILOR_E_RANGE;
+    int rc = check_space(ctx, s);
+    if (rc) return rc;
+    const TabHdr& h = ctx->hdr;
+    const uint32_t T = h.T, Z = h.Z;
+    for (uint32_t o = 0; o < n_orders; ++o) {
+        if (orders[o].n < 1 || orders[o].n > Z) return SAILOR_E_ARG;
+        uint32_t seen = 0;
+        for (uint32_t j = 0; j < orders[o].n; ++j) {
+            if (orders[o].zone[j] >= Z || ((seen >> orders[o].zone[j]) & 1u)) return SAILOR_E_ARG;
+            seen |= 1u << orders[o].zone[j];
+        }
+    }
+    const SpaceDesc d = to_desc(s);
+    const uint64_t n_config = (uint64_t)d.n_p * d.n_mbs * d.n_tp * d.n_rc * d.n_d;
+    if (n_config * n_orders > (1u << 22)) return SAILOR_E_RANGE;
+    if (workspace_bytes == 0) workspace_bytes = 8ull << 30;
+    uint32_t p_max = 0;
+    for (uint32_t j = 0; j < d.n_p; ++j) p_max = d.p_values[j] > p_max ? d.p_values[j] : p_max;
+
+    // every problem's table layout, from the availability last set (host copy)
+    const uint64_t n_problems = n_config * n_orders;
+    std::vector<DpProblem> prob(n_problems);
+    uint64_t n_states = 0;
+    for (uint64_t c = 0; c < n_config; ++c) {
+        const Config cf = config_of(d, (uint32_t)c);
+        const uint32_t tp = h.tp_values[cf.tpi];
+        const uint64_t dm = (uint64_t)cf.D * h.mbs_values[cf.mi];
+        const bool valid = h.gbs % dm == 0 && h.heads % tp == 0;
+        const uint64_t need = (uint64_t)cf.D * tp;
+        for (uint32_t o = 0; o < n_orders; ++o) {
+            DpProblem& pb = prob[c * n_orders + o];
+            memset(&pb, 0, sizeof(pb));
+            pb.config = (uint32_t)c; pb.order = o; pb.index = (uint32_t)(c * n_orders + o);
+            pb.P = cf.P; pb.nz = orders[o].n; pb.need = (uint32_t)(need > 0xffffffffull ? 0xffffffffull : need);
+            memset(pb.first_later, DP_NONE, sizeof(pb.first_later));
+            if (!valid) continue;                           // no entries: the finish step finds no plan
+            uint64_t n_lvl = 0;
+            for (uint32_t zp = 0; zp < pb.nz; ++zp) {
+                pb.zone[zp] = orders[o].zone[zp];
+                uint64_t S = 1;
+                for (uint32_t g = 0; g < T; ++g) {
+                    const uint64_t cap = ctx->h_avail[pb.zone[zp] * T + g] / need;
+                    pb.cap[zp][g] = (uint8_t)(cap > 255 ? 255 : cap);
+                    if (cap >= 1 && cap < cf.P) {           // counted: the zone cannot host every stage
+                        pb.stride[zp][g] = (uint32_t)S;
+                        S *= cap + 1;
+                        if (S > (1ull << 31)) return SAILOR_E_RANGE;
+                    }
+                }
+                pb.S[zp] = (uint32_t)S;
+                pb.zp_base[zp] = (uint32_t)n_lvl;
+                n_lvl += (uint64_t)T * S;
+                if (n_lvl > (1ull << 31)) return SAILOR_E_RANGE;
+            }
+            pb.zp_base[pb.nz] = (uint32_t)n_lvl;
+            for (uint32_t zp = 0; zp < pb.nz; ++zp)
+                for (uint32_t g = 0; g < T; ++g)
+                    for (uint32_t q = zp + 1; q < pb.nz; ++q)
+                        if (pb.cap[q][g] >= 1) { pb.first_later[zp][g] = (uint8_t)q; break; }
+            pb.n_lvl = (uint32_t)n_lvl;
+            n_states += n_lvl * cf.P;
+        }
+    }
+    // deepest pipelines first, so that the launch for a distance from the last stage covers a prefix
+    std::vector<uint32_t> by_depth;
+    by_depth.reserve(n_problems);
+    for (uint64_t j = 0; j < n_problems; ++j)
+        if (prob[j].n_lvl) by_depth.push_back((uint32_t)j);
+    std::stable_sort(by_depth.begin(), by_depth.end(), [&](uint32_t a, uint32_t b) { return prob[a].P > prob[b].P; });
+    auto work_bytes = [](const DpProblem& pb) { return (uint64_t)pb.n_lvl * (2 * sizeof(DpVal) + pb.P); };
+    struct Batch { size_t first, count; uint64_t entries, choice_bytes, blocks; };
+    std::vector<Batch> batches;
+    uint64_t largest = 0;
+    for (size_t j = 0; j < by_depth.size();) {
+        Batch b = {j, 0, 0, 0, 0};
+        uint64_t bytes = 0;
+        while (j < by_depth.size()) {
+            const DpProblem& pb = prob[by_depth[j]];
+            const uint64_t wb = work_bytes(pb) + 512;
+            if (b.count && bytes + wb > workspace_bytes) break;
+            if (wb > workspace_bytes) return SAILOR_E_RANGE;      // one problem alone does not fit
+            bytes += wb;
+            b.entries += pb.n_lvl;
+            b.choice_bytes += (uint64_t)pb.n_lvl * pb.P;
+            b.blocks += (pb.n_lvl + DP_THREADS - 1) / DP_THREADS;
+            ++b.count; ++j;
+        }
+        largest = bytes > largest ? bytes : largest;
+        batches.push_back(b);
+    }
+    uint64_t max_entries = 0, max_choice = 0, max_blocks = 0, max_count = 0;
+    for (const Batch& b : batches) {
+        max_entries = std::max(max_entries, b.entries);
+        max_choice = std::max(max_choice, b.choice_bytes);
+        max_blocks = std::max(max_blocks, b.blocks);
+        max_count = std::max<uint64_t>(max_count, b.count);
+    }
+    if (max_blocks > 0x7fffffffull) return SAILOR_E_RANGE;
+
+    DeviceGuard guard(ctx->device);
+    DpTabLayout lay;
+    lay.p_max = p_max; lay.T = T; lay.R = h.R;
+    const size_t tab_bytes = (size_t)n_config * lay.stride() * sizeof(double);
+    const size_t total = padded(tab_bytes) + padded(n_problems * sizeof(DpResult)) + padded(n_problems * sizeof(DpProblem)) +
+                         2 * padded(max_blocks * sizeof(uint32_t)) + 2 * padded(max_entries * sizeof(DpVal)) +
+                         padded(max_choice) + padded(sizeof(sailor_dp_result) * SAILOR_K_MAX) + padded(16) + 4096;
+    if (total > ctx->dp_bytes) {
+        CU(ctx, cudaStreamSynchronize(ctx->stream));
+        cudaFree(ctx->d_dp);
+        ctx->d_dp = nullptr;
+        ctx->dp_bytes = 0;
+        cudaError_t e = cudaMalloc(&ctx->d_dp, total);
+        if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
+        ctx->dp_bytes = total;
+    }
+    Bump bump{ctx->d_dp};
+    double* d_tabs = bump.take<double>(tab_bytes / sizeof(double));
+    DpResult* d_results = bump.take<DpResult>(n_problems);
+    DpProblem* d_problems = bump.take<DpProblem>(n_problems);
+    uint32_t* d_blk_problem = bump.take<uint32_t>(max_blocks);
+    uint32_t* d_blk_first = bump.take<uint32_t>(max_blocks);
+    DpVal* d_val0 = bump.take<DpVal>(max_entries);
+    DpVal* d_val1 = bump.take<DpVal>(max_entries);
+    uint8_t* d_choice = bump.take<uint8_t>(max_choice);
+    sailor_dp_result* d_out = bump.take<sailor_dp_result>(SAILOR_K_MAX);
+    unsigned long long* d_counters = bump.take<unsigned long long>(2);
+
+    uint32_t launches = 0;
+    CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
+    CU(ctx, cudaMemsetAsync(d_tabs, 0, tab_bytes, ctx->stream));
+    CU(ctx, cudaMemsetAsync(d_counters, 0, 16, ctx->stream));
+    {
+        const uint32_t grid = (uint32_t)(n_config < 4096 ? n_config : 4096);
+        dp_tables_kernel<<<grid, DP_THREADS, 0, ctx->stream>>>(ctx->d_blob, d, (uint32_t)n_config, lay, d_tabs);
+        CU(ctx, cudaGetLastError());
+        ++launches;
+    }
+    // problems that have no entries still get their "no plan" result from the finish step
+    std::vector<DpProblem> stage_buf;
+    std::vector<uint32_t> blk_problem, blk_first;
+    {
+        stage_buf.clear();
+        for (uint64_t j = 0; j < n_problems; ++j)
+            if (!prob[j].n_lvl) stage_buf.push_back(prob[j]);
+        if (!stage_buf.empty()) {
+            CU(ctx, cudaMemcpyAsync(d_problems, stage_buf.data(), stage_buf.size() * sizeof(DpProblem), cudaMemcpyHostToDevice,
+                                    ctx->stream));
+            DpFinishParams fp;
+            memset(&fp, 0, sizeof(fp));
+            fp.problems = d_problems; fp.tabs = d_tabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
+            fp.results = d_results; fp.lay = lay; fp.n_problems = (uint32_t)stage_buf.size(); fp.T = T;
+            dp_finish_kernel<<<(fp.n_problems + 127) / 128, 128, 0, ctx->stream>>>(fp);
+            CU(ctx, cudaGetLastError());
+            ++launches;
+            CU(ctx, cudaStreamSynchronize(ctx->stream));       // the staging vector is reused below
+        }
+    }
+    for (const Batch& b : batches) {
+        stage_buf.resize(b.count);
+        blk_problem.clear();
+        blk_first.clear();
+        uint64_t val_off = 0, choice_off = 0;
+        uint32_t max_p = 0;
+        std::vector<uint64_t> blocks_upto(p_max + 2, 0);       // blocks of problems deeper than a distance
+        for (size_t j = 0; j < b.count; ++j) {
+            DpProblem pb = prob[by_depth[b.first + j]];
+            pb.val_off = val_off;
+            pb.choice_off = choice_off;
+            val_off += pb.n_lvl;
+            choice_off += (uint64_t)pb.n_lvl * pb.P;
+            stage_buf[j] = pb;
+            max_p = pb.P > max_p ? pb.P : max_p;
+            const uint32_t nb = (pb.n_lvl + DP_THREADS - 1) / DP_THREADS;
+            for (uint32_t q = 0; q < nb; ++q) { blk_problem.push_back((uint32_t)j); blk_first.push_back(q * DP_THREADS); }
+            for (uint32_t dist = 0; dist < pb.P; ++dist) blocks_upto[dist] += nb;
+        }
+        CU(ctx, cudaMemcpyAsync(d_problems, stage_buf.data(), b.count * sizeof(DpProblem), cudaMemcpyHostToDevice, ctx->stream));
+        CU(ctx, cudaMemcpyAsync(d_blk_problem, blk_problem.data(), blk_problem.size() * sizeof(uint32_t), cudaMemcpyHostToDevice,
+                                ctx->stream));
+        CU(ctx, cudaMemcpyAsync(d_blk_first, blk_first.data(), blk_first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice,
+                                ctx->stream));
+        DpLevelParams lp;
+        memset(&lp, 0, sizeof(lp));
+        lp.problems = d_problems; lp.blk_problem = d_blk_problem; lp.blk_first = d_blk_first; lp.tabs = d_tabs;
+        lp.val[0] = d_val0; lp.val[1] = d_val1; lp.choice = d_choice; lp.lay = lay; lp.T = T;
+        for (uint32_t dist = 0; dist < max_p; ++dist) {
+            lp.dist = dist;
+            dp_level_kernel<<<(uint32_t)blocks_upto[dist], DP_THREADS, 0, ctx->stream>>>(lp);
+            CU(ctx, cudaGetLastError());
+            ++launches;
+        }
+        DpFinishParams fp;
+        memset(&fp, 0, sizeof(fp));
+        fp.problems = d_problems; fp.tabs = d_tabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
+        fp.results = d_results; fp.lay = lay; fp.n_problems = (uint32_t)b.count; fp.T = T;
+        dp_finish_kernel<<<(fp.n_problems + 127) / 128, 128, 0, ctx->stream>>>(fp);
+        CU(ctx, cudaGetLastError());
+        ++launches;
+        CU(ctx, cudaStreamSynchronize(ctx->stream));           // the host vectors are reused by the next batch
+    }
+    DpSelectParams sel;
+    memset(&sel, 0, sizeof(sel));
+    sel.blob = ctx->d_blob; sel.avail = ctx->d_avail; sel.results = d_results; sel.out = d_out; sel.counters = d_counters;
+    sel.sp = d; sel.n_problems = (uint32_t)n_problems; sel.n_orders = n_orders; sel.k = k;
+    dp_select_kernel<<<1, DP_SELECT_THREADS, 0, ctx->stream>>>(sel);
+    CU(ctx, cudaGetLastError());
+    ++launches;
+    CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
+    unsigned long long counters[2] = {0, 0};
+    std::vector<sailor_dp_result> host_out(k);
+    CU(ctx, cudaMemcpyAsync(counters, d_counters, sizeof(counters), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(host_out.data(), d_out, sizeof(sailor_dp_result) * k, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, cudaStreamSynchronize(ctx->stream));
+    *n_found = (uint32_t)counters[1];
+    memcpy(topk, host_out.data(), sizeof(sailor_dp_result) * counters[1]);
+    if (stats) {
+        stats->n_problems = n_problems;
+        stats->n_solved = counters[0];
+        stats->n_states = n_states;
+        stats->workspace_used = largest;
+        float ms = 0.f;
+        CU(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
+        stats->kernel_ms = ms;
+        stats->n_launches = launches;
+        stats->n_batches = (uint32_t)batches.size();
+        stats->_pad = 0;
     }
     return SAILOR_OK;
 }

@@ -212,25 +212,27 @@ struct SimOut {
 __device__ __forceinline__ double make_nan() { return __longlong_as_double(0x7ff8000000000000LL); }
 __device__ __forceinline__ double make_inf() { return __longlong_as_double(0x7ff0000000000000LL); }
 
-// Simulate one run-length encoded plan (Sec. 4.3).  Every index is checked before use; a
-// record that fails gets SAILOR_ST_BAD_RECORD and nothing is read through it.
+// Simulate one run-length encoded plan (Sec. 4.3), given as its header values and `n_runs` runs
+// (at most `max_runs`).  Every index is checked before use; a plan that fails gets
+// SAILOR_ST_BAD_RECORD and nothing is read through it.
 //
 // The stages are walked in one flat loop (no loop nest over runs), so that the lanes of a warp,
 // each with its own record, stay on the same instructions; values that depend only on the
 // stage's layer composition and run are refreshed when either changes.  `cnt` points to this
 // thread's per-digit GPU counters (digit d at cnt[d * cnt_stride], any initial contents).
-__device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __restrict__ avail,
-                                         const sailor_plan_rec& r, uint32_t* cnt, uint32_t cnt_stride) {
+__device__ __forceinline__ SimOut simulate_runs(const TabView& v, const uint16_t* __restrict__ avail, uint32_t P,
+                                                uint32_t n_runs, uint32_t D, uint32_t mi, uint32_t rc,
+                                                const sailor_run* runs, uint32_t max_runs, uint32_t* cnt,
+                                                uint32_t cnt_stride) {
     const TabHdr* h = v.h;
     SimOut o;
     o.t_iter = o.cost = make_nan();
     o.peak_mem = 0;
     o.status = SAILOR_ST_BAD_RECORD;
-    const uint32_t P = r.P, n_runs = r.n_runs, D = r.D, mi = r.mbs_idx, rc = r.rc ? 1u : 0u;
-    if (P < 1 || P > SAILOR_P_MAX || n_runs < 1 || n_runs > SAILOR_RUN_MAX || D < 1 || mi >= h->n_mbs) return o;
+    if (P < 1 || P > SAILOR_P_MAX || n_runs < 1 || n_runs > max_runs || D < 1 || mi >= h->n_mbs) return o;
     uint32_t tot = 0;
     for (uint32_t q = 0; q < n_runs; ++q) {
-        const sailor_run rr = r.run[q];
+        const sailor_run rr = runs[q];
         if (rr.type >= h->T || rr.zone >= h->Z || rr.tp_idx >= h->n_tp || rr.n_stages < 1) return o;
         tot += rr.n_stages;
     }
@@ -245,7 +247,7 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
     // resources: GPUs taken of every (zone, type), saturating at 2^32 - 1 (availability is 16 bits)
     for (uint32_t d = 0; d < h->R; ++d) cnt[d * cnt_stride] = 0;
     for (uint32_t q = 0; q < n_runs; ++q) {
-        const sailor_run a = r.run[q];
+        const sailor_run a = runs[q];
         const uint32_t tp = h->tp_values[a.tp_idx];
         if (tp > h->gpn[a.type] || h->heads % tp != 0) status |= SAILOR_ST_INVALID;
         uint32_t* c = cnt + (a.zone * h->T + a.type) * cnt_stride;
@@ -253,7 +255,7 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
         *c = sum > 0xffffffffull ? 0xffffffffu : (uint32_t)sum;
     }
     for (uint32_t q = 0; q < n_runs; ++q) {
-        const uint32_t d = r.run[q].zone * h->T + r.run[q].type;
+        const uint32_t d = runs[q].zone * h->T + runs[q].type;
         if (cnt[d * cnt_stride] > avail[d]) status |= SAILOR_ST_OVER_AVAIL;
     }
 
@@ -278,7 +280,7 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
     for (uint32_t i = 0; i < P; ++i) {
         bool refresh = false;
         if (left == 0) {                                   // enter run q
-            const sailor_run a = r.run[q];
+            const sailor_run a = runs[q];
             g = a.type; z = a.zone; tpi = a.tp_idx; tp = h->tp_values[tpi]; left = a.n_stages;
             const uint32_t d = z * h->T + g;
             gpu_rate = mul_rn((double)(D * tp), v.price_s[d]);
@@ -311,7 +313,7 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
         if (i + 1 < P) {
             t = t_self;                                      // next stage in the same run
             if (left == 1) {                                 // next stage opens run q + 1
-                const sailor_run nx = r.run[q + 1];
+                const sailor_run nx = runs[q + 1];
                 const double c = boundary_time(v, g, z, tp, nx.type, nx.zone, h->tp_values[nx.tp_idx], D, msg);
                 if (nx.zone != z) c_comm = add_rn(c_comm, mul_rn((double)xbytes, v.egress[z * h->Z + nx.zone]));
                 t = add_rn(fb, mul_rn(2.0, c));
@@ -331,6 +333,11 @@ __device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __res
     o.t_iter = add_rn(add_rn(t_pp, max_sync), max_u);
     o.cost = add_rn(mul_rn(rate, o.t_iter), c_comm);
     return o;
+}
+
+__device__ inline SimOut simulate_record(const TabView& v, const uint16_t* __restrict__ avail,
+                                         const sailor_plan_rec& r, uint32_t* cnt, uint32_t cnt_stride) {
+    return simulate_runs(v, avail, r.P, r.n_runs, r.D, r.mbs_idx, r.rc ? 1u : 0u, r.run, SAILOR_RUN_MAX, cnt, cnt_stride);
 }
 
 // ---- search space -------------------------------------------------------------------------
