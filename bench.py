@@ -154,6 +154,28 @@ def pruning_modes(B, ctx, w, sp) -> dict:
     return out
 
 
+def dp_search(B, ctx, w, sp) -> dict:
+    """Per-stage GPU types by the dynamic-programming recursion (one zone order: zones as numbered),
+    next to the best iteration time the segment search finds in its own space."""
+    orders = [list(range(w.n_zones))]
+    B.sailor_plan_dp(ctx, sp, orders, K_TOP)
+    ts = []
+    for _ in range(3):
+        t0 = time.perf_counter()
+        B.sailor_set_availability(ctx, w.avail)
+        res, st = B.sailor_plan_dp(ctx, sp, orders, K_TOP)
+        ts.append(time.perf_counter() - t0)
+    seg, _ = B.sailor_plan(ctx, sp, B.make_objective(w, kind=W.OBJ_MAX_THROUGHPUT, budget=0.0, min_rate=0.0, factor=0.0), 1)
+    # bytes the level kernel must move per table entry: its value (32 B) and choice (1 B) written once
+    return {"search_s": statistics.median(ts), "kernel_ms": st.kernel_ms, "problems": int(st.n_problems),
+            "solved": int(st.n_solved), "table_entries": int(st.n_states), "batches": int(st.n_batches),
+            "launches": int(st.n_launches), "workspace_bytes": int(st.workspace_used),
+            "entries_per_s": st.n_states / (st.kernel_ms / 1e3) if st.kernel_ms > 0 else None,
+            "write_gb_per_s": st.n_states * 33 / (st.kernel_ms / 1e3) / 1e9 if st.kernel_ms > 0 else None,
+            "best_t_iter": res[0].t_iter if res else None, "best_stages": int(res[0].P) if res else None,
+            "segment_search_best_t_iter": seg[0].t_iter if seg else None}
+
+
 def aux_measurements(B, torch, dev) -> dict:
     """Search seconds of the other workloads through the public call (host buffers), default mode."""
     out = {}
@@ -173,6 +195,7 @@ def aux_measurements(B, torch, dev) -> dict:
             out[f"cfg{cfg}"] = {"candidates": int(st.n_total), "search_s": statistics.median(ts),
                                 "kernel_ms": st.kernel_ms, "passes": 2 if w.budget_factor_over_cheapest > 0 else 1}
             out[f"cfg{cfg}"]["pruning_modes"] = pruning_modes(B, ctx, w, sp)
+            out[f"cfg{cfg}"]["dp"] = dp_search(B, ctx, w, sp)
         finally:
             B.sailor_destroy(ctx)
     # explicit batches (sailor_simulate) with records resident in HBM: 72 B in + 28 B out per plan
@@ -375,7 +398,8 @@ def run_ours(args) -> None:
                 ts.append(time.perf_counter() - t0)
             aux[args.workload + "_default_mode"] = {"candidates": int(stp.n_total), "search_s": statistics.median(ts),
                                                     "kernel_ms": stp.kernel_ms, "feasible": int(stp.n_feasible),
-                                                    "pruning_modes": pruning_modes(B, ctx, w, space)}
+                                                    "pruning_modes": pruning_modes(B, ctx, w, space),
+                                                    "dp": dp_search(B, ctx, w, space)}
         line = {"metric": METRIC, "value": total / dev_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": 1e3 * dev_s / args.steps, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",

@@ -337,8 +337,12 @@ int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const sailor_obj
  * the best one for its own state, so the plan found can be worse than the best of all type
  * sequences.  `value` sums the stage times from the last stage backwards; t_iter, cost and
  * peak_mem of a result are the simulator's figures for the written-out plan (stage order), equal
- * to value up to rounding.  The budget loop of Sec. 4.2.3 is not implemented: the objective is
- * iteration time (maximum throughput) without a constraint.
+ * to value up to rounding.  The objective is iteration time (o->kind must be MAX_THROUGHPUT, no
+ * flags, no budget factor).  A budget or a minimum throughput in `o` is checked on the plan the
+ * recursion returns for a problem, by the simulator's cost and time (Sec. 4.2: a configuration
+ * counts only when it is within the constraint); a problem whose plan fails it drops out.  The
+ * straggler-guessing budget loop of Sec. 4.2.3, which steers the recursion itself by the remaining
+ * budget, is not implemented.
  *
  * On the device every problem is a dense table over its states (stage, type, zone position,
  * stages per type already placed in that zone; a type with room for all P stages in a zone is not
@@ -368,22 +372,24 @@ typedef struct sailor_dp_result {
 typedef struct sailor_dp_stats {
     uint64_t n_problems;                /* configurations x zone orders                               */
     uint64_t n_solved;                  /* problems that have a plan                                  */
+    uint64_t n_over_constraint;         /* of which the plan is over the budget or under the throughput */
     uint64_t n_states;                  /* table entries filled (all problems, all stages)            */
     uint64_t workspace_used;            /* bytes of the largest batch                                 */
     float    kernel_ms;
     uint32_t n_launches, n_batches, _pad;
 } sailor_dp_stats;
 
-/* Solve every problem of `s` x `orders` and return the k best plans by (value, problem index =
- * config * n_orders + order) ascending; *n_found <= k.  `topk` is a HOST array of k records;
+/* Solve every problem of `s` x `orders` and return the k best plans within the constraint by
+ * (value, problem index = config * n_orders + order) ascending; *n_found <= k.  `topk` is a HOST array of k records;
  * `stats` may be NULL.  Uses the availability last set.  `workspace_bytes` bounds the device memory
  * of the tables (0 = 8 GiB); it is allocated on first use and kept by the context (grow-only).
- * Errors: E_ARG (null, k == 0, n_orders == 0, a zone twice or out of range), E_RANGE (k >
+ * Errors: E_ARG (null, k == 0, n_orders == 0, a zone twice or out of range, an objective other
+ * than plain MAX_THROUGHPUT), E_RANGE (k >
  * SAILOR_K_MAX, space limits as sailor_plan, a single problem whose tables exceed the workspace or
  * 2^31 entries per stage), E_NOMEM, E_CUDA. */
 int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders, uint32_t n_orders,
-                   uint64_t workspace_bytes, uint32_t k, sailor_dp_result* topk, uint32_t* n_found,
-                   sailor_dp_stats* stats);
+                   const sailor_objective* o, uint64_t workspace_bytes, uint32_t k, sailor_dp_result* topk,
+                   uint32_t* n_found, sailor_dp_stats* stats);
 
 const char* sailor_strerror(int code);
 int sailor_last_cuda_error(const sailor_ctx* ctx);   /* cudaError_t of the last E_CUDA      */

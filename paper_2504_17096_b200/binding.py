@@ -91,13 +91,14 @@ class DpResult(C.Structure):
 
 
 class DpStats(C.Structure):
-    _fields_ = [("n_problems", C.c_uint64), ("n_solved", C.c_uint64), ("n_states", C.c_uint64),
+    _fields_ = [("n_problems", C.c_uint64), ("n_solved", C.c_uint64), ("n_over_constraint", C.c_uint64),
+                ("n_states", C.c_uint64),
                 ("workspace_used", C.c_uint64), ("kernel_ms", C.c_float), ("n_launches", C.c_uint32),
                 ("n_batches", C.c_uint32), ("_pad", C.c_uint32)]
 
 
 assert C.sizeof(PlanRec) == 72 and C.sizeof(Result) == 120 and C.sizeof(Space) == 152
-assert C.sizeof(ZoneOrder) == 12 and C.sizeof(DpResult) == 248 and C.sizeof(DpStats) == 48
+assert C.sizeof(ZoneOrder) == 12 and C.sizeof(DpResult) == 248 and C.sizeof(DpStats) == 56
 assert C.sizeof(Objective) == 32 and C.sizeof(Stats) == 96
 
 # numpy view of an array of plan records (same 72-byte layout)
@@ -140,8 +141,8 @@ def load() -> C.CDLL:
     L.sailor_plan_range.argtypes = [vp, C.POINTER(Space), C.POINTER(Objective), C.c_uint64, C.c_uint64, C.c_uint32,
                                     C.POINTER(Result), _u32p, C.POINTER(Stats)]
     L.sailor_plan_noalloc.argtypes = L.sailor_plan.argtypes
-    L.sailor_plan_dp.argtypes = [vp, C.POINTER(Space), C.POINTER(ZoneOrder), C.c_uint32, C.c_uint64, C.c_uint32,
-                                 C.POINTER(DpResult), _u32p, C.POINTER(DpStats)]
+    L.sailor_plan_dp.argtypes = [vp, C.POINTER(Space), C.POINTER(ZoneOrder), C.c_uint32, C.POINTER(Objective),
+                                 C.c_uint64, C.c_uint32, C.POINTER(DpResult), _u32p, C.POINTER(DpStats)]
     L.sailor_strerror.argtypes = [C.c_int]
     L.sailor_strerror.restype = C.c_char_p
     L.sailor_last_cuda_error.argtypes = [vp]
@@ -301,9 +302,13 @@ def sailor_plan_noalloc(ctx, space: Space, obj: Objective, k: int):
     return list(res[: n.value]), st
 
 
-def sailor_plan_dp(ctx, space: Space, zone_orders, k: int, workspace_bytes: int = 0):
+def sailor_plan_dp(ctx, space: Space, zone_orders, k: int, workspace_bytes: int = 0, *, budget: float = 0.0,
+                   min_rate: float = 0.0, obj: Optional[Objective] = None):
     """Per-stage GPU types by dynamic programming for every configuration of the space and every zone
-    order (a list of zone lists): the k best plans by the recursion's value, and the statistics."""
+    order (a list of zone lists): the k best plans by the recursion's value among those within the
+    budget / minimum throughput, and the statistics."""
+    if obj is None:
+        obj = Objective(OBJ_MAX_THROUGHPUT, 0, budget, min_rate, 0.0)
     orders = (ZoneOrder * len(zone_orders))()
     for j, zl in enumerate(zone_orders):
         if len(zl) > Z_MAX:
@@ -314,8 +319,8 @@ def sailor_plan_dp(ctx, space: Space, zone_orders, k: int, workspace_bytes: int 
     res = (DpResult * k)()
     n = C.c_uint32()
     st = DpStats()
-    _check(load().sailor_plan_dp(ctx, C.byref(space), orders, len(zone_orders), workspace_bytes, k, res, C.byref(n),
-                                 C.byref(st)), "sailor_plan_dp", ctx)
+    _check(load().sailor_plan_dp(ctx, C.byref(space), orders, len(zone_orders), C.byref(obj), workspace_bytes, k, res,
+                                 C.byref(n), C.byref(st)), "sailor_plan_dp", ctx)
     return list(res[: n.value]), st
 
 

@@ -42,6 +42,9 @@ struct DpProblem {
 
 struct DpResult {                    // per problem, written by dp_finish_kernel
     double value;                    // +inf: no plan
+    double t_iter, cost;             // the simulator's figures for the plan (stage order)
+    uint64_t peak_mem;
+    uint32_t status, _pad;
     uint8_t type[SAILOR_P_MAX];
     uint8_t zone[SAILOR_P_MAX];
 };
@@ -165,6 +168,14 @@ __global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_const
     uint32_t zp = 0;
     while (zp + 1 < pb.nz && e >= pb.zp_base[zp + 1]) ++zp;
     const uint32_t g = (e - pb.zp_base[zp]) / pb.S[zp], ui = (e - pb.zp_base[zp]) % pb.S[zp];
+    // stage i is at most the (i+1)-th stage of its zone: entries that count more are never reached, and
+    // since a move raises the count by one per stage, no entry that passes this test ever reads one that fails it
+    {
+        uint32_t placed = 0;
+        for (uint32_t t = 0; t < T; ++t)
+            if (pb.stride[zp][t]) placed += (ui / pb.stride[zp][t]) % (pb.cap[zp][t] + 1u);
+        if (placed > i + 1) return;
+    }
     DpVal* cur = lp.val[lp.dist & 1] + pb.val_off;
     const DpVal* nxt = lp.val[(lp.dist & 1) ^ 1] + pb.val_off;
     uint8_t* choice = lp.choice + pb.choice_off + (size_t)i * pb.n_lvl;
@@ -207,6 +218,9 @@ __global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_const
 
 // Stage 0 and the walk through the kept choices: one thread per problem.
 struct DpFinishParams {
+    const unsigned char* blob;
+    const uint16_t* avail;
+    SpaceDesc sp;
     const DpProblem* problems;
     const double* tabs;
     const DpVal* val[2];
@@ -240,52 +254,79 @@ __global__ void __launch_bounds__(128) dp_finish_kernel(const __grid_constant__ 
     }
     out.value = best_v;
     if (g == DP_NONE) return;
+    const Config k = config_of(fp.sp, pb.config);
+    sailor_run runs[SAILOR_P_MAX];
+    uint32_t n_runs = 0;
     for (uint32_t i = 0; i < P; ++i) {
+        const uint8_t z = pb.zone[zp];
         out.type[i] = (uint8_t)g;
-        out.zone[i] = pb.zone[zp];
+        out.zone[i] = z;
+        if (n_runs && runs[n_runs - 1].type == g && runs[n_runs - 1].zone == z) runs[n_runs - 1].n_stages++;
+        else {
+            runs[n_runs].type = (uint8_t)g; runs[n_runs].zone = z;
+            runs[n_runs].tp_idx = (uint8_t)k.tpi; runs[n_runs].n_stages = 1;
+            ++n_runs;
+        }
         if (i + 1 == P) break;
         const uint8_t g2 = fp.choice[pb.choice_off + (size_t)i * pb.n_lvl + entry];
         const uint32_t ui = (entry - pb.zp_base[zp]) % pb.S[zp];
         const DpMove mv = dp_move(pb, zp, ui, g2);
         g = g2; zp = mv.zp; entry = mv.entry;
     }
+    // the plan written out, through the simulator (Sec. 4.3): what a caller compares with a constraint
+    TabView v;
+    v.bind(fp.blob, fp.blob);
+    uint32_t cnt[R_MAX];
+    const SimOut so = simulate_runs(v, fp.avail, P, n_runs, k.D, k.mi, k.rc, runs, SAILOR_P_MAX, cnt, 1);
+    out.t_iter = so.t_iter;
+    out.cost = so.cost;
+    out.peak_mem = so.peak_mem;
+    out.status = so.status;
 }
 
 // The k best problems by (value, problem index), then the simulator's figures for their plans.
 struct DpSelectParams {
-    const unsigned char* blob;
-    const uint16_t* avail;
     const DpResult* results;
     sailor_dp_result* out;           // [k] device
-    unsigned long long* counters;    // [0] problems with a plan, [1] number written to out
+    unsigned long long* counters;    // [0] problems with a plan, [1] number written to out, [2] plans over the constraint
     SpaceDesc sp;
     uint32_t n_problems, n_orders, k;
+    double budget, min_rate;         // <= 0: none
 };
 
 constexpr int DP_SELECT_THREADS = 512;
 
 __global__ void __launch_bounds__(DP_SELECT_THREADS) dp_select_kernel(const __grid_constant__ DpSelectParams sp) {
     __shared__ Hit s_hits[DP_SELECT_THREADS / 32][SAILOR_K_MAX];
-    __shared__ uint32_t s_cnt[R_MAX][DP_SELECT_THREADS / 32];
     __shared__ uint32_t s_n;
-    __shared__ unsigned long long s_solved;
+    __shared__ unsigned long long s_solved, s_over;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = DP_SELECT_THREADS / 32;
-    if (tid == 0) s_solved = 0;
+    if (tid == 0) { s_solved = 0; s_over = 0; }
     __syncthreads();
     WarpTopK top;
     top.init();
-    uint32_t solved = 0;
+    uint32_t solved = 0, over = 0;
     for (uint32_t base = warp * 32; base < sp.n_problems; base += nw * 32) {
         const uint32_t j = base + lane;
         const double v = j < sp.n_problems ? sp.results[j].value : make_inf();
-        const bool have = v < make_inf();
+        bool have = v < make_inf();
         solved += have;
+        if (have) {                                           // the planner keeps a plan only within the constraint
+            const DpResult& r = sp.results[j];
+            const bool out_of = (sp.budget > 0.0 && r.cost > sp.budget) || (sp.min_rate > 0.0 && 1.0 / r.t_iter < sp.min_rate);
+            over += out_of;
+            have = !out_of;
+        }
         const bool want = have && v <= top.thr_score;
         if (__any_sync(FULL, want)) top.offer(want, v, j, sp.k, lane);
     }
 #pragma unroll
-    for (int o = 16; o; o >>= 1) solved += __shfl_xor_sync(FULL, solved, o);
+    for (int o = 16; o; o >>= 1) {
+        solved += __shfl_xor_sync(FULL, solved, o);
+        over += __shfl_xor_sync(FULL, over, o);
+    }
     if (lane == 0 && solved) atomicAdd(&s_solved, (unsigned long long)solved);
+    if (lane == 0 && over) atomicAdd(&s_over, (unsigned long long)over);
     s_hits[warp][lane].score = top.score;
     s_hits[warp][lane].flat = top.flat;
     __syncthreads();
@@ -303,11 +344,10 @@ __global__ void __launch_bounds__(DP_SELECT_THREADS) dp_select_kernel(const __gr
             s_n = n;
             sp.counters[0] = s_solved;
             sp.counters[1] = n;
+            sp.counters[2] = s_over;
         }
     }
     __syncthreads();
-    TabView v;
-    v.bind(sp.blob, sp.blob);
     for (uint32_t j = warp; j < s_n; j += nw) {
         if (lane != 0) continue;
         const uint32_t idx = (uint32_t)s_hits[0][j].flat;
@@ -320,23 +360,14 @@ __global__ void __launch_bounds__(DP_SELECT_THREADS) dp_select_kernel(const __gr
         o.order = idx % sp.n_orders;
         o.value = r.value;
         o.P = (uint8_t)k.P; o.mbs_idx = (uint8_t)k.mi; o.tp_idx = (uint8_t)k.tpi; o.rc = (uint8_t)k.rc; o.D = (uint16_t)k.D;
-        sailor_run runs[SAILOR_P_MAX];
-        uint32_t n_runs = 0;
         for (uint32_t i = 0; i < k.P; ++i) {
             o.type[i] = r.type[i];
             o.zone[i] = r.zone[i];
-            if (n_runs && runs[n_runs - 1].type == r.type[i] && runs[n_runs - 1].zone == r.zone[i]) runs[n_runs - 1].n_stages++;
-            else {
-                runs[n_runs].type = r.type[i]; runs[n_runs].zone = r.zone[i];
-                runs[n_runs].tp_idx = (uint8_t)k.tpi; runs[n_runs].n_stages = 1;
-                ++n_runs;
-            }
         }
-        const SimOut so = simulate_runs(v, sp.avail, k.P, n_runs, k.D, k.mi, k.rc, runs, SAILOR_P_MAX, &s_cnt[0][warp], nw);
-        o.t_iter = so.t_iter;
-        o.cost = so.cost;
-        o.peak_mem = so.peak_mem;
-        o.status = so.status;
+        o.t_iter = r.t_iter;
+        o.cost = r.cost;
+        o.peak_mem = r.peak_mem;
+        o.status = r.status;
         sp.out[j] = o;
     }
 }

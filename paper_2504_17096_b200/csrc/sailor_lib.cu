@@ -1136,20 +1136,24 @@ size_t padded(size_t bytes) { return (bytes + 255) & ~(size_t)255; }
 }  // namespace
 
 extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders,
-                              uint32_t n_orders, uint64_t workspace_bytes, uint32_t k, sailor_dp_result* topk,
-                              uint32_t* n_found, sailor_dp_stats* stats) {
-    if (!ctx || !s || !orders || !topk || !n_found || k == 0 || n_orders == 0) return SAILOR_E_ARG;
+                              uint32_t n_orders, const sailor_objective* o, uint64_t workspace_bytes, uint32_t k,
+                              sailor_dp_result* topk, uint32_t* n_found, sailor_dp_stats* stats) {
+    if (!ctx || !s || !orders || !o || !topk || !n_found || k == 0 || n_orders == 0) return SAILOR_E_ARG;
     if (k > SAILOR_K_MAX) return SAILOR_E_RANGE;
+    // the recursion minimises iteration time; a constraint is checked on the plan it returns per problem
+    if (o->kind != SAILOR_OBJ_MAX_THROUGHPUT || o->flags != 0 || o->budget_factor_over_cheapest > 0.0 ||
+        std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) || std::isnan(o->budget_factor_over_cheapest))
+        return SAILOR_E_ARG;
     int rc = check_space(ctx, s);
     if (rc) return rc;
     const TabHdr& h = ctx->hdr;
     const uint32_t T = h.T, Z = h.Z;
-    for (uint32_t o = 0; o < n_orders; ++o) {
-        if (orders[o].n < 1 || orders[o].n > Z) return SAILOR_E_ARG;
+    for (uint32_t q = 0; q < n_orders; ++q) {
+        if (orders[q].n < 1 || orders[q].n > Z) return SAILOR_E_ARG;
         uint32_t seen = 0;
-        for (uint32_t j = 0; j < orders[o].n; ++j) {
-            if (orders[o].zone[j] >= Z || ((seen >> orders[o].zone[j]) & 1u)) return SAILOR_E_ARG;
-            seen |= 1u << orders[o].zone[j];
+        for (uint32_t j = 0; j < orders[q].n; ++j) {
+            if (orders[q].zone[j] >= Z || ((seen >> orders[q].zone[j]) & 1u)) return SAILOR_E_ARG;
+            seen |= 1u << orders[q].zone[j];
         }
     }
     const SpaceDesc d = to_desc(s);
@@ -1169,16 +1173,16 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
         const uint64_t dm = (uint64_t)cf.D * h.mbs_values[cf.mi];
         const bool valid = h.gbs % dm == 0 && h.heads % tp == 0;
         const uint64_t need = (uint64_t)cf.D * tp;
-        for (uint32_t o = 0; o < n_orders; ++o) {
-            DpProblem& pb = prob[c * n_orders + o];
+        for (uint32_t q = 0; q < n_orders; ++q) {
+            DpProblem& pb = prob[c * n_orders + q];
             memset(&pb, 0, sizeof(pb));
-            pb.config = (uint32_t)c; pb.order = o; pb.index = (uint32_t)(c * n_orders + o);
-            pb.P = cf.P; pb.nz = orders[o].n; pb.need = (uint32_t)(need > 0xffffffffull ? 0xffffffffull : need);
+            pb.config = (uint32_t)c; pb.order = q; pb.index = (uint32_t)(c * n_orders + q);
+            pb.P = cf.P; pb.nz = orders[q].n; pb.need = (uint32_t)(need > 0xffffffffull ? 0xffffffffull : need);
             memset(pb.first_later, DP_NONE, sizeof(pb.first_later));
             if (!valid) continue;                           // no entries: the finish step finds no plan
             uint64_t n_lvl = 0;
             for (uint32_t zp = 0; zp < pb.nz; ++zp) {
-                pb.zone[zp] = orders[o].zone[zp];
+                pb.zone[zp] = orders[q].zone[zp];
                 uint64_t S = 1;
                 for (uint32_t g = 0; g < T; ++g) {
                     const uint64_t cap = ctx->h_avail[pb.zone[zp] * T + g] / need;
@@ -1245,7 +1249,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     const size_t tab_bytes = (size_t)n_config * lay.stride() * sizeof(double);
     const size_t total = padded(tab_bytes) + padded(n_problems * sizeof(DpResult)) + padded(n_problems * sizeof(DpProblem)) +
                          2 * padded(max_blocks * sizeof(uint32_t)) + 2 * padded(max_entries * sizeof(DpVal)) +
-                         padded(max_choice) + padded(sizeof(sailor_dp_result) * SAILOR_K_MAX) + padded(16) + 4096;
+                         padded(max_choice) + padded(sizeof(sailor_dp_result) * SAILOR_K_MAX) + padded(24) + 4096;
     if (total > ctx->dp_bytes) {
         CU(ctx, cudaStreamSynchronize(ctx->stream));
         cudaFree(ctx->d_dp);
@@ -1265,12 +1269,12 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     DpVal* d_val1 = bump.take<DpVal>(max_entries);
     uint8_t* d_choice = bump.take<uint8_t>(max_choice);
     sailor_dp_result* d_out = bump.take<sailor_dp_result>(SAILOR_K_MAX);
-    unsigned long long* d_counters = bump.take<unsigned long long>(2);
+    unsigned long long* d_counters = bump.take<unsigned long long>(3);
 
     uint32_t launches = 0;
     CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
     CU(ctx, cudaMemsetAsync(d_tabs, 0, tab_bytes, ctx->stream));
-    CU(ctx, cudaMemsetAsync(d_counters, 0, 16, ctx->stream));
+    CU(ctx, cudaMemsetAsync(d_counters, 0, 24, ctx->stream));
     {
         const uint32_t grid = (uint32_t)(n_config < 4096 ? n_config : 4096);
         dp_tables_kernel<<<grid, DP_THREADS, 0, ctx->stream>>>(ctx->d_blob, d, (uint32_t)n_config, lay, d_tabs);
@@ -1289,7 +1293,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
                                     ctx->stream));
             DpFinishParams fp;
             memset(&fp, 0, sizeof(fp));
-            fp.problems = d_problems; fp.tabs = d_tabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
+            fp.blob = ctx->d_blob; fp.avail = ctx->d_avail; fp.sp = d; fp.problems = d_problems; fp.tabs = d_tabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
             fp.results = d_results; fp.lay = lay; fp.n_problems = (uint32_t)stage_buf.size(); fp.T = T;
             dp_finish_kernel<<<(fp.n_problems + 127) / 128, 128, 0, ctx->stream>>>(fp);
             CU(ctx, cudaGetLastError());
@@ -1333,7 +1337,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
         }
         DpFinishParams fp;
         memset(&fp, 0, sizeof(fp));
-        fp.problems = d_problems; fp.tabs = d_tabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
+        fp.blob = ctx->d_blob; fp.avail = ctx->d_avail; fp.sp = d; fp.problems = d_problems; fp.tabs = d_tabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
         fp.results = d_results; fp.lay = lay; fp.n_problems = (uint32_t)b.count; fp.T = T;
         dp_finish_kernel<<<(fp.n_problems + 127) / 128, 128, 0, ctx->stream>>>(fp);
         CU(ctx, cudaGetLastError());
@@ -1342,13 +1346,14 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     }
     DpSelectParams sel;
     memset(&sel, 0, sizeof(sel));
-    sel.blob = ctx->d_blob; sel.avail = ctx->d_avail; sel.results = d_results; sel.out = d_out; sel.counters = d_counters;
+    sel.results = d_results; sel.out = d_out; sel.counters = d_counters;
     sel.sp = d; sel.n_problems = (uint32_t)n_problems; sel.n_orders = n_orders; sel.k = k;
+    sel.budget = o->budget_usd_per_iter; sel.min_rate = o->min_iters_per_s;
     dp_select_kernel<<<1, DP_SELECT_THREADS, 0, ctx->stream>>>(sel);
     CU(ctx, cudaGetLastError());
     ++launches;
     CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
-    unsigned long long counters[2] = {0, 0};
+    unsigned long long counters[3] = {0, 0, 0};
     std::vector<sailor_dp_result> host_out(k);
     CU(ctx, cudaMemcpyAsync(counters, d_counters, sizeof(counters), cudaMemcpyDeviceToHost, ctx->stream));
     CU(ctx, cudaMemcpyAsync(host_out.data(), d_out, sizeof(sailor_dp_result) * k, cudaMemcpyDeviceToHost, ctx->stream));
@@ -1358,6 +1363,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     if (stats) {
         stats->n_problems = n_problems;
         stats->n_solved = counters[0];
+        stats->n_over_constraint = counters[2];
         stats->n_states = n_states;
         stats->workspace_used = largest;
         float ms = 0.f;

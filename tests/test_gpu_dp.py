@@ -157,6 +157,26 @@ def test_dp_sampled_problems_of_the_large_workloads():
             assert (r.value, r.t_iter, r.cost, r.peak_mem, r.status) == (ref["value"], sim.t_iter, sim.cost, sim.peak_mem, 0)
 
 
+def test_dp_constraints_drop_plans_after_the_recursion():
+    """A budget or a throughput floor is checked on each problem's plan by the simulator's cost and time."""
+    w, orders = W.tiny(seed=3, n_types=3, n_zones=2, L=6, p_values=[1, 2, 3, 6]), [[0, 1], [1, 0]]
+    o = Oracle(w)
+    want = oracle_all(w, o, orders)
+    sims = [o.simulate(x[2]["plan"]) for x in want]
+    budget = float(np.median([s.cost for s in sims]))
+    min_rate = 1.0 / float(np.median([s.t_iter for s in sims]))
+    with Ctx(w) as cx:
+        for kw in ({"budget": budget}, {"min_rate": min_rate}, {"budget": budget, "min_rate": min_rate}):
+            keep = [x for x, s in zip(want, sims)
+                    if not (kw.get("budget", 0) > 0 and s.cost > kw["budget"])
+                    and not (kw.get("min_rate", 0) > 0 and 1.0 / s.t_iter < kw["min_rate"])]
+            assert 0 < len(keep) < len(want)
+            res, st = B.sailor_plan_dp(cx.ctx, cx.space, orders, 32, **kw)
+            assert st.n_solved == len(want) and st.n_over_constraint == len(want) - len(keep)
+            assert [(r.config * len(orders) + r.order) for r in res] == [x[1] for x in keep[:32]]
+            assert [r.value for r in res] == [x[0] for x in keep[:32]]
+
+
 def test_dp_argument_checks():
     w = W.tiny(seed=3)
     with Ctx(w) as cx:
@@ -167,6 +187,11 @@ def test_dp_argument_checks():
         with pytest.raises(B.SailorError) as e:
             B.sailor_plan_dp(cx.ctx, cx.space, [[0]], 33)
         assert e.value.code == B.E_RANGE
+        for obj in (B.Objective(B.OBJ_MIN_COST, 0, 0.0, 0.0, 0.0), B.Objective(B.OBJ_MAX_THROUGHPUT, B.FLAG_EVAL_ALL, 0.0, 0.0, 0.0),
+                    B.Objective(B.OBJ_MAX_THROUGHPUT, 0, 0.0, 0.0, 1.2)):
+            with pytest.raises(B.SailorError) as e:
+                B.sailor_plan_dp(cx.ctx, cx.space, [[0]], 4, obj=obj)
+            assert e.value.code == B.E_ARG
         with pytest.raises(B.SailorError) as e:
             B.sailor_plan_dp(cx.ctx, cx.space, [[0, 1]], 4, workspace_bytes=64)
         assert e.value.code == B.E_RANGE
