@@ -32,7 +32,7 @@ K_TOP = 32
 OPS_PLAN, OPS_STAGE = 40, 35
 SM_COUNT, ISSUE_PER_SM, LANES = 148, 4, 32
 # ncu counters per plan_kernel launch (smsp__inst_executed.sum; dram__bytes_read.sum + dram__bytes_write.sum)
-NCU_PER_LAUNCH = {"cfg5-stress-96layer": {"warp_inst": 11942834741, "dram_bytes": 2930768}}
+NCU_PER_LAUNCH = {"cfg5-stress-96layer": {"warp_inst": 11245134608, "dram_bytes": 841216}}
 
 
 def mean_ops_per_candidate(w: W.Workload) -> float:
