@@ -111,6 +111,22 @@ class OrcDpResult(C.Structure):
     _fields_ = [("found", C.c_int32), ("_pad", C.c_uint32), ("value", C.c_double), ("n_states", C.c_uint64),
                 ("plan", OrcPlan)]
 
+GROUPS_MAX = 4
+
+
+class OrcReplicaGroup(C.Structure):
+    _fields_ = [("type", C.c_uint32), ("tp_idx", C.c_uint32), ("count", C.c_uint32)]
+
+
+class OrcMixedStage(C.Structure):
+    _fields_ = [("zone", C.c_uint32), ("n_groups", C.c_uint32), ("group", OrcReplicaGroup * GROUPS_MAX)]
+
+
+class OrcMixedPlan(C.Structure):
+    _fields_ = [("P", C.c_uint32), ("mbs_idx", C.c_uint32), ("rc", C.c_uint32), ("D", C.c_uint32),
+                ("stage", OrcMixedStage * STAGES_MAX)]
+
+
 _lib = None
 
 
@@ -139,6 +155,11 @@ def lib():
         L.orc_search_pruned.restype = C.c_int32
         L.orc_solve_dp.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcDpProblem), C.c_int, C.POINTER(OrcDpResult)]
         L.orc_solve_dp.restype = C.c_int
+        L.orc_simulate_mixed.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedPlan), C.POINTER(OrcOut)]
+        L.orc_simulate_mixed.restype = None
+        L.orc_simulate_mixed_batch.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedPlan), C.c_uint64,
+                                               _u32p, _dp, _dp, _u64p]
+        L.orc_simulate_mixed_batch.restype = None
         _lib = L
     return _lib
 
@@ -209,6 +230,37 @@ class Oracle:
         out = OrcOut()
         lib().orc_simulate(C.byref(self.inputs), C.byref(plan), C.byref(out))
         return out
+
+    # -- plans whose stages mix GPU types among their replicas ---------------------------
+    @staticmethod
+    def make_mixed_plan(plan: dict) -> OrcMixedPlan:
+        """plan = {"P", "mbs_idx", "rc", "D", "stages": [{"zone", "groups": [(type, tp_idx, count), ...]}, ...]}"""
+        pl = OrcMixedPlan()
+        pl.P, pl.mbs_idx, pl.rc, pl.D = plan["P"], plan["mbs_idx"], plan["rc"], plan["D"]
+        for i, st in enumerate(plan["stages"]):
+            if len(st["groups"]) > GROUPS_MAX:
+                raise ValueError("too many groups in a stage")
+            pl.stage[i].zone = int(st["zone"])
+            pl.stage[i].n_groups = len(st["groups"])
+            for q, (g, tpi, count) in enumerate(st["groups"]):
+                pl.stage[i].group[q].type, pl.stage[i].group[q].tp_idx, pl.stage[i].group[q].count = int(g), int(tpi), int(count)
+        return pl
+
+    def simulate_mixed(self, plan: dict) -> OrcOut:
+        out = OrcOut()
+        pl = self.make_mixed_plan(plan)
+        lib().orc_simulate_mixed(C.byref(self.inputs), C.byref(pl), C.byref(out))
+        return out
+
+    def simulate_mixed_batch(self, plans):
+        n = len(plans)
+        arr = (OrcMixedPlan * n)()
+        for j, p in enumerate(plans):
+            arr[j] = self.make_mixed_plan(p)
+        st = np.zeros(n, np.uint32); t = np.zeros(n); c = np.zeros(n); m = np.zeros(n, np.uint64)
+        lib().orc_simulate_mixed_batch(C.byref(self.inputs), arr, n, st.ctypes.data_as(_u32p), t.ctypes.data_as(_dp),
+                                       c.ctypes.data_as(_dp), m.ctypes.data_as(_u64p))
+        return st, t, c, m
 
     def space_size(self) -> int:
         return int(lib().orc_space_size(C.byref(self.inputs), C.byref(self.space)))

@@ -678,3 +678,194 @@ int orc_solve_dp(const orc_inputs* in, const orc_dp_problem* pb, int use_memo, o
     free(c->keys); free(c->vals); free(c->full); free(c);
     return 0;
 }
+
+/* ---- plans whose stages mix GPU types among their replicas (Sec. 4.2, Sec. 4.3, Sec. 4.4) -----------
+ *
+ * Stage i has D replicas in one zone (H5), given as groups: `count` replicas on one GPU type with one
+ * tensor-parallel degree (H1).  Replicas are numbered group after group, and pipeline k runs on replica
+ * k of every stage, so the pipelines differ and T_iter takes the slowest one (Sec. 4.3).
+ */
+void orc_simulate_mixed(const orc_inputs* in, const orc_mixed_plan* pl, orc_out* out) {
+    static uint8_t kinds[ORC_STAGES_MAX][1024 + 2];
+    uint32_t nl[ORC_STAGES_MAX];
+    const uint32_t P = pl->P, T = in->n_types, Z = in->n_zones;
+    const uint32_t mbs_idx = pl->mbs_idx, D = pl->D, rc = pl->rc;
+    const uint64_t mbs = in->mbs_values[mbs_idx];
+    uint32_t status = 0;
+    memset(out, 0, sizeof(*out));
+
+    /* validity: the batch divides evenly, every stage has exactly D replicas, tensor parallelism stays in a node */
+    if (D == 0 || in->gbs % ((uint64_t)D * mbs) != 0) status |= ORC_INVALID;
+    for (uint32_t i = 0; i < P; ++i) {
+        uint64_t replicas = 0;
+        for (uint32_t q = 0; q < pl->stage[i].n_groups; ++q) {
+            const orc_replica_group* gr = &pl->stage[i].group[q];
+            const uint32_t tp = in->tp_values[gr->tp_idx];
+            replicas += gr->count;
+            if (gr->count == 0 || tp > in->gpus_per_node[gr->type] || in->heads % tp != 0) status |= ORC_INVALID;
+        }
+        if (replicas != D) status |= ORC_INVALID;
+    }
+    const uint64_t n_b = D ? in->gbs / ((uint64_t)D * mbs) : 0;
+    out->n_b = n_b;
+
+    /* resources */
+    uint64_t used[64 * 64];
+    memset(used, 0, sizeof(uint64_t) * Z * T);
+    for (uint32_t i = 0; i < P; ++i)
+        for (uint32_t q = 0; q < pl->stage[i].n_groups; ++q) {
+            const orc_replica_group* gr = &pl->stage[i].group[q];
+            used[pl->stage[i].zone * T + gr->type] += (uint64_t)gr->count * in->tp_values[gr->tp_idx];
+        }
+    for (uint32_t d = 0; d < Z * T; ++d)
+        if (used[d] > in->avail[d]) status |= ORC_OVER_AVAIL;
+
+    /* memory of every kind of worker: M_peak = M_model + M_activation */
+    uint64_t params_stage[ORC_STAGES_MAX];
+    uint64_t peak = 0;
+    for (uint32_t i = 0; i < P; ++i) {
+        nl[i] = stage_layers(in, P, i, kinds[i]);
+        uint64_t stage_peak = 0;
+        for (uint32_t q = 0; q < pl->stage[i].n_groups; ++q) {
+            const orc_replica_group* gr = &pl->stage[i].group[q];
+            const uint32_t tpi = gr->tp_idx;
+            const uint64_t tp = in->tp_values[tpi];
+            uint64_t params = 0, A = 0, W = 0;
+            for (uint32_t l = 0; l < nl[i]; ++l) {
+                const uint32_t k = kinds[i][l];
+                params += in->params[k];
+                A += rc ? tab_act(in, in->act_ckpt, k, tpi, mbs_idx) : tab_act(in, in->act_saved, k, tpi, mbs_idx);
+                const uint64_t w = rc ? tab_act(in, in->act_saved, k, tpi, mbs_idx) : tab_act(in, in->act_work, k, tpi, mbs_idx);
+                if (w > W) W = w;
+            }
+            params_stage[i] = params;
+            const uint64_t m = ceil_div_u64(params, tp) * in->mul_factor * in->dtype_size +
+                               min_u64((uint64_t)(P - i), n_b) * A + W + in->reserved[gr->type];
+            if (m > in->capacity[gr->type]) status |= ORC_OOM;
+            if (m > stage_peak) stage_peak = m;
+        }
+        out->stage_mem[i] = stage_peak;
+        if (stage_peak > peak) peak = stage_peak;
+    }
+    out->peak_mem = peak;
+    out->status = status;
+    if (status & ORC_INVALID) {
+        out->t_iter = NAN;
+        out->cost = NAN;
+        return;
+    }
+
+    /* the pipelines, one after the other: pipeline k uses, in stage i, the group that holds replica k */
+    const uint64_t msg = in->p2p_bytes[mbs_idx];
+    double max_pp = 0.0;
+    for (uint32_t k = 0; k < D; ++k) {
+        uint32_t grp[ORC_STAGES_MAX];
+        for (uint32_t i = 0; i < P; ++i) {
+            uint32_t q = 0, upto = pl->stage[i].group[0].count;
+            while (k >= upto) { ++q; upto += pl->stage[i].group[q].count; }
+            grp[i] = q;
+        }
+        double sum_t = 0.0, max_t = 0.0;
+        for (uint32_t i = 0; i < P; ++i) {
+            const orc_replica_group* gr = &pl->stage[i].group[grp[i]];
+            const uint32_t g = gr->type, z = pl->stage[i].zone, tpi = gr->tp_idx;
+            double f = 0.0, b = 0.0;
+            for (uint32_t l = 0; l < nl[i]; ++l) {
+                f = f + tab4(in, in->fwd, kinds[i][l], g, tpi, mbs_idx);
+                b = b + tab4(in, in->bwd, kinds[i][l], g, tpi, mbs_idx);
+            }
+            if (rc) b = b + f;
+            double c = 0.0;
+            if (i + 1 < P) {
+                const orc_replica_group* g2r = &pl->stage[i + 1].group[grp[i + 1]];
+                const uint32_t g2 = g2r->type, z2 = pl->stage[i + 1].zone;
+                if (z != z2) {
+                    c = link_time(in->zone_alpha[z * Z + z2], in->zone_inv_bw[z * Z + z2], poly_at(in->zone_bw_poly, z * Z + z2), msg);
+                } else if (g == g2 && (uint64_t)gr->count * in->tp_values[tpi] + (uint64_t)g2r->count * in->tp_values[g2r->tp_idx] <=
+                                          in->gpus_per_node[g]) {
+                    /* the two groups' GPUs all sit in one node */
+                    c = link_time(in->intra_alpha[z * T + g], in->intra_inv_bw[z * T + g], poly_at(in->intra_bw_poly, z * T + g), msg);
+                } else {
+                    const double c1 = link_time(in->inter_alpha[z * T + g], in->inter_inv_bw[z * T + g], poly_at(in->inter_bw_poly, z * T + g), msg);
+                    const double c2 = link_time(in->inter_alpha[z * T + g2], in->inter_inv_bw[z * T + g2], poly_at(in->inter_bw_poly, z * T + g2), msg);
+                    c = max_f64(c1, c2);
+                }
+            }
+            const double t = (f + b) + 2.0 * c;
+            sum_t = sum_t + t;
+            max_t = max_f64(max_t, t);
+        }
+        const double t_pp = sum_t + (double)n_b * max_t;
+        max_pp = max_f64(max_pp, t_pp);
+    }
+
+    /* synchronisation and update: the slowest over stages, and within a stage over its groups */
+    double max_sync = 0.0, max_u = 0.0;
+    for (uint32_t i = 0; i < P; ++i) {
+        const uint32_t z = pl->stage[i].zone, ng = pl->stage[i].n_groups;
+        /* the ring moves the largest shard (the group with the smallest tp sets the message size) */
+        uint64_t gradbytes = 0;
+        for (uint32_t q = 0; q < ng; ++q) {
+            const uint64_t gb = ceil_div_u64(params_stage[i], in->tp_values[pl->stage[i].group[q].tp_idx]) * in->grad_dtype_size;
+            if (gb > gradbytes) gradbytes = gb;
+        }
+        double sync = 0.0;
+        for (uint32_t q = 0; q < ng; ++q) {
+            const orc_replica_group* gr = &pl->stage[i].group[q];
+            const uint32_t g = gr->type, d = z * T + g;
+            double u = 0.0;
+            for (uint32_t l = 0; l < nl[i]; ++l) u = u + tab_upd(in, kinds[i][l], g, gr->tp_idx);
+            max_u = max_f64(max_u, u);
+            if (D > 1) {
+                /* one group whose GPUs fit a node talks inside the node; otherwise every group's inter-node
+                 * link carries the ring and the slowest of them sets the time */
+                const int intra = ng == 1 && (uint64_t)D * in->tp_values[gr->tp_idx] <= in->gpus_per_node[g];
+                const double alpha = intra ? in->intra_alpha[d] : in->inter_alpha[d];
+                const double inv = intra ? in->intra_inv_bw[d] : in->inter_inv_bw[d];
+                const double* poly = intra ? poly_at(in->intra_bw_poly, d) : poly_at(in->inter_bw_poly, d);
+                const double steps = (double)(2 * (uint64_t)(D - 1));
+                const double coef = steps / (double)D;
+                double s;
+                if (poly) s = (coef * (double)gradbytes) / poly_bw(poly, (double)gradbytes / (double)D) + steps * alpha;
+                else s = (coef * (double)gradbytes) * inv + steps * alpha;
+                sync = max_f64(sync, s);
+            }
+        }
+        out->stage_sync[i] = sync;
+        max_sync = max_f64(max_sync, sync);
+    }
+    const double t_iter = (max_pp + max_sync) + max_u;
+    out->t_pp = max_pp;
+    out->t_sync = max_sync;
+    out->t_update = max_u;
+    out->t_iter = t_iter;
+
+    /* cost: every replica's GPUs for the whole iteration, and the bytes that cross zones */
+    double rate = 0.0;
+    for (uint32_t i = 0; i < P; ++i)
+        for (uint32_t q = 0; q < pl->stage[i].n_groups; ++q) {
+            const orc_replica_group* gr = &pl->stage[i].group[q];
+            const uint32_t n_gpus = gr->count * in->tp_values[gr->tp_idx];
+            rate = rate + (double)n_gpus * (in->price_per_hour[pl->stage[i].zone * T + gr->type] / 3600.0);
+        }
+    double c_comm = 0.0;
+    for (uint32_t i = 0; i + 1 < P; ++i) {
+        const uint32_t z = pl->stage[i].zone, z2 = pl->stage[i + 1].zone;
+        if (z != z2) c_comm = c_comm + (double)(2 * n_b * (uint64_t)D * msg) * in->egress[z * Z + z2];
+    }
+    out->rate_per_s = rate;
+    out->c_comm = c_comm;
+    out->cost = rate * t_iter + c_comm;
+}
+
+void orc_simulate_mixed_batch(const orc_inputs* in, const orc_mixed_plan* plans, uint64_t n, uint32_t* status,
+                              double* t_iter, double* cost, uint64_t* peak_mem) {
+    orc_out o;
+    for (uint64_t j = 0; j < n; ++j) {
+        orc_simulate_mixed(in, &plans[j], &o);
+        status[j] = o.status;
+        t_iter[j] = o.t_iter;
+        cost[j] = o.cost;
+        peak_mem[j] = o.peak_mem;
+    }
+}

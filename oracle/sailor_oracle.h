@@ -215,4 +215,36 @@ typedef struct orc_dp_result {
 /* returns 0, or -1 for sizes beyond the limits; use_memo = 0 is the plain recursion */
 int orc_solve_dp(const orc_inputs* in, const orc_dp_problem* pb, int use_memo, orc_dp_result* out);
 
+
+/* ---- plans whose stages mix GPU types among their replicas ------------------------------------------
+ *
+ * The paper's plan gives every stage D replicas, each with its own (GPU type, tp), all in one zone
+ * (Sec. 4.2 problem statement, H1, H5), and its framework runs such plans (Sec. 4.4).  Here a stage lists
+ * its replicas as groups of `count` equal replicas.  What the paper leaves open is read as follows:
+ *   - replicas are numbered group after group; pipeline k is replica k of every stage; every pipeline
+ *     processes N_b = gbs / (D * mbs) microbatches; T_pp of a pipeline is sum_i t_i + N_b * max_i t_i over its
+ *     own stages, and T_iter = max_k T_pp(k) + T_sync + T_update (Sec. 4.3);
+ *   - the message between two neighbouring replicas stays inside a node only when they have the same GPU
+ *     type and the two groups they belong to fit one node together; across zones the zone link; otherwise
+ *     the slower of the two types' inter-node links (as for plans without mixing);
+ *   - a stage's all-reduce moves the largest gradient shard among its groups (smallest tp); a single group
+ *     that fits a node uses the intra-node link, otherwise the ring is as slow as the slowest group's
+ *     inter-node link;
+ *   - memory is checked per group (stage, tp, GPU type); T_update and the price rate run over all groups.
+ * A plan whose stages all have one group is the plan of orc_simulate and gives bit-identical results
+ * (pinned), and a plan whose stages all split D the same way has exactly the slower of its two
+ * homogeneous pipelines (pinned against orc_simulate); one case is worked by hand. */
+#define ORC_GROUPS_MAX 4
+
+typedef struct orc_replica_group { uint32_t type, tp_idx, count; } orc_replica_group;
+typedef struct orc_mixed_stage { uint32_t zone, n_groups; orc_replica_group group[ORC_GROUPS_MAX]; } orc_mixed_stage;
+typedef struct orc_mixed_plan {
+    uint32_t P, mbs_idx, rc, D;
+    orc_mixed_stage stage[ORC_STAGES_MAX];
+} orc_mixed_plan;
+
+void orc_simulate_mixed(const orc_inputs* in, const orc_mixed_plan* plan, orc_out* out);
+void orc_simulate_mixed_batch(const orc_inputs* in, const orc_mixed_plan* plans, uint64_t n, uint32_t* status,
+                              double* t_iter, double* cost, uint64_t* peak_mem);
+
 #endif

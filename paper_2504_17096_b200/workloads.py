@@ -412,3 +412,30 @@ def random_plans(w: Workload, n: int, seed: int, *, max_runs: int = 16, hetero_t
             out["tp_idx"][j, r] = rng.randint(0, len(w.tp_values) - 1) if hetero_tp else tp0
             out["n_stages"][j, r] = ln
     return out
+
+
+def random_mixed_plans(w: Workload, n: int, seed: int, *, p_max: int = 32, groups_max: int = 4):
+    """n random plans whose stages split their D replicas into groups of different (type, tp), as a list of
+    dicts {"P", "mbs_idx", "rc", "D", "stages": [{"zone", "groups": [(type, tp_idx, count), ...]}]}.
+    About a quarter of the plans have one group in every stage (no mixing)."""
+    rng = SplitMix64(seed)
+    plans = []
+    for _ in range(n):
+        P = w.p_values[rng.randint(0, len(w.p_values) - 1)] if rng.uniform() < 0.7 else rng.randint(1, min(w.n_blocks, p_max))
+        P = min(P, p_max)
+        D = w.d_values[rng.randint(0, len(w.d_values) - 1)]
+        plain = rng.uniform() < 0.25
+        zone = rng.randint(0, w.n_zones - 1)
+        stages = []
+        for i in range(P):
+            if rng.uniform() < 0.3:
+                zone = rng.randint(0, w.n_zones - 1)
+            ng = 1 if plain else rng.randint(1, min(groups_max, D))
+            cuts = sorted({rng.randint(1, D - 1) for _ in range(ng - 1)}) if D > 1 else []
+            bounds = [0] + cuts + [D]
+            groups = [(rng.randint(0, w.n_types - 1), rng.randint(0, len(w.tp_values) - 1), bounds[q + 1] - bounds[q])
+                      for q in range(len(bounds) - 1)]
+            stages.append({"zone": zone, "groups": groups})
+        plans.append({"P": P, "mbs_idx": rng.randint(0, len(w.mbs_values) - 1),
+                      "rc": w.rc_values[rng.randint(0, len(w.rc_values) - 1)], "D": D, "stages": stages})
+    return plans
