@@ -315,6 +315,51 @@ int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objec
 int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint32_t k,
                         sailor_result* topk, uint32_t* n_found, sailor_stats* stats);
 
+/* ---- plans whose stages mix GPU types among their replicas (Sec. 4.2 problem statement, Sec. 4.3) ----
+ *
+ * In the paper a stage has D replicas, each with its own (GPU type, tp), all in one zone (H1, H5).
+ * A stage lists its replicas as up to SAILOR_MIX_GROUPS_MAX groups of `count` equal replicas; the
+ * counts of a stage add up to D.  Readings where the paper is silent:
+ *   - replicas are numbered group after group and pipeline k is replica k of every stage; every
+ *     pipeline processes N_b = gbs / (D * mbs) microbatches; T_pp(k) = sum_i t_i + N_b * max_i t_i over
+ *     pipeline k's own stages; T_iter = (max_k T_pp(k) + max_i sync_i) + max update;
+ *   - a message between neighbouring replicas stays inside a node only when both have the same GPU
+ *     type and their two groups fit one node together (count*tp + count'*tp' <= gpus_per_node);
+ *     across zones it takes the zone link, otherwise the slower of the two types' inter-node times;
+ *   - a stage's all-reduce moves the largest gradient shard among its groups (the smallest tp); one
+ *     group that fits a node (D*tp <= gpus_per_node) uses the intra-node link, otherwise every
+ *     group's inter-node link carries the ring and the slowest sets the time;
+ *   - memory is checked per group; the update time is the largest over stages and groups; the price
+ *     rate adds (double)(count*tp) * price per second group after group, stage after stage.
+ * A plan with one group in every stage gives bit-identical results to sailor_simulate. */
+#define SAILOR_MIX_P_MAX       32
+#define SAILOR_MIX_GROUPS_MAX  4
+
+typedef struct sailor_replica_group {
+    uint8_t  type, tp_idx;
+    uint16_t count;                     /* replicas in the group, >= 1                               */
+} sailor_replica_group;
+
+typedef struct sailor_mixed_stage {
+    uint8_t  zone, n_groups;            /* 1 .. SAILOR_MIX_GROUPS_MAX                                 */
+    uint16_t _pad;
+    sailor_replica_group group[SAILOR_MIX_GROUPS_MAX];
+} sailor_mixed_stage;
+
+typedef struct sailor_mixed_plan {      /* 648 bytes; arrays must be 8-byte aligned                  */
+    uint8_t  P;                         /* 1 .. SAILOR_MIX_P_MAX                                      */
+    uint8_t  mbs_idx, rc, _pad;
+    uint16_t D;                         /* >= 1                                                       */
+    uint16_t _pad2;
+    sailor_mixed_stage stage[SAILOR_MIX_P_MAX];
+} sailor_mixed_plan;
+
+/* Simulate n such plans.  Pointers, outputs, NULLs, on_device and errors as sailor_simulate.
+ * SAILOR_ST_INVALID also covers a stage whose counts do not add up to D or a group with count 0;
+ * SAILOR_ST_BAD_RECORD an index outside its table or n_groups / P outside their limits. */
+int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint64_t n, int on_device,
+                          double* t_iter, uint64_t* peak_mem, double* cost, uint32_t* status);
+
 /* ---- per-stage GPU types by dynamic programming (Sec. 4.2.2: Eq. 1, T_total, the listing) --------
  *
  * sailor_plan varies the GPU type and zone of at most SAILOR_SEG_MAX segments of a pipeline.  This

@@ -20,7 +20,7 @@ FLAG_EVAL_ALL, FLAG_DEGREE_ORDER, FLAG_MIN_TP_ONLY = 1, 2, 4
 
 EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
            "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_plan_noalloc",
-           "sailor_plan_dp", "sailor_strerror", "sailor_last_cuda_error")
+           "sailor_plan_dp", "sailor_simulate_mixed", "sailor_strerror", "sailor_last_cuda_error")
 
 _dp, _u64p, _u32p, _u16p = C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.POINTER(C.c_uint16)
 
@@ -108,6 +108,34 @@ REC_DTYPE = np.dtype([("P", "u1"), ("mbs_idx", "u1"), ("rc", "u1"), ("n_runs", "
 assert REC_DTYPE.itemsize == 72
 
 
+MIX_P_MAX, MIX_GROUPS_MAX = 32, 4
+MIX_GROUP_DTYPE = np.dtype([("type", "u1"), ("tp_idx", "u1"), ("count", "<u2")])
+MIX_STAGE_DTYPE = np.dtype([("zone", "u1"), ("n_groups", "u1"), ("_pad", "<u2"), ("group", MIX_GROUP_DTYPE, (MIX_GROUPS_MAX,))])
+MIX_DTYPE = np.dtype([("P", "u1"), ("mbs_idx", "u1"), ("rc", "u1"), ("_pad", "u1"), ("D", "<u2"), ("_pad2", "<u2"),
+                      ("stage", MIX_STAGE_DTYPE, (MIX_P_MAX,))])
+assert MIX_DTYPE.itemsize == 648
+
+
+def pack_mixed_plans(plans) -> np.ndarray:
+    """List of dicts {"P", "mbs_idx", "rc", "D", "stages": [{"zone", "groups": [(type, tp_idx, count), ...]}]}
+    -> array of 648-byte records."""
+    out = np.zeros(len(plans), dtype=MIX_DTYPE)
+    for j, p in enumerate(plans):
+        if p["P"] > MIX_P_MAX:
+            raise ValueError("at most %d stages" % MIX_P_MAX)
+        out["P"][j], out["mbs_idx"][j], out["rc"][j], out["D"][j] = p["P"], p["mbs_idx"], p["rc"], p["D"]
+        for i, st in enumerate(p["stages"]):
+            if len(st["groups"]) > MIX_GROUPS_MAX:
+                raise ValueError("at most %d groups per stage" % MIX_GROUPS_MAX)
+            out["stage"]["zone"][j, i] = st["zone"]
+            out["stage"]["n_groups"][j, i] = len(st["groups"])
+            for q, (g, tpi, count) in enumerate(st["groups"]):
+                out["stage"]["group"]["type"][j, i, q] = g
+                out["stage"]["group"]["tp_idx"][j, i, q] = tpi
+                out["stage"]["group"]["count"][j, i, q] = count
+    return out
+
+
 class SailorError(RuntimeError):
     def __init__(self, code: int, where: str, cuda: int = 0):
         self.code = code
@@ -134,6 +162,7 @@ def load() -> C.CDLL:
     L.sailor_destroy.argtypes = [vp]
     L.sailor_set_availability.argtypes = [vp, _u16p]
     L.sailor_simulate.argtypes = [vp, vp, C.c_uint64, C.c_int, vp, vp, vp, vp]
+    L.sailor_simulate_mixed.argtypes = [vp, vp, C.c_uint64, C.c_int, vp, vp, vp, vp]
     L.sailor_space_size.argtypes = [vp, C.POINTER(Space), _u64p]
     L.sailor_decode.argtypes = [vp, C.POINTER(Space), C.c_uint64, C.POINTER(PlanRec)]
     L.sailor_plan.argtypes = [vp, C.POINTER(Space), C.POINTER(Objective), C.c_uint32, C.POINTER(Result), _u32p,
@@ -259,6 +288,24 @@ def sailor_simulate_device(ctx, plans_ptr: int, n: int, t_iter_ptr: int, peak_me
     """Device path: raw device pointers (e.g. torch tensors' data_ptr()); only enqueues work."""
     _check(load().sailor_simulate(ctx, plans_ptr, n, 1, t_iter_ptr or None, peak_mem_ptr or None, cost_ptr or None,
                                   status_ptr or None), "sailor_simulate", ctx)
+
+
+def sailor_simulate_mixed(ctx, plans: np.ndarray):
+    """Plans with mixed replicas (MIX_DTYPE array, see pack_mixed_plans) in, (t_iter, peak_mem, cost, status) out."""
+    plans = np.ascontiguousarray(plans, dtype=MIX_DTYPE)
+    n = plans.size
+    t, c = np.empty(n, np.float64), np.empty(n, np.float64)
+    m, s = np.empty(n, np.uint64), np.empty(n, np.uint32)
+    _check(load().sailor_simulate_mixed(ctx, plans.ctypes.data, n, 0, t.ctypes.data, m.ctypes.data, c.ctypes.data,
+                                        s.ctypes.data), "sailor_simulate_mixed", ctx)
+    return t, m, c, s
+
+
+def sailor_simulate_mixed_device(ctx, plans_ptr: int, n: int, t_iter_ptr: int, peak_mem_ptr: int, cost_ptr: int,
+                                 status_ptr: int) -> None:
+    """Device path of sailor_simulate_mixed: raw device pointers; only enqueues work."""
+    _check(load().sailor_simulate_mixed(ctx, plans_ptr, n, 1, t_iter_ptr or None, peak_mem_ptr or None, cost_ptr or None,
+                                        status_ptr or None), "sailor_simulate_mixed", ctx)
 
 
 def sailor_space_size(ctx, space: Space) -> int:

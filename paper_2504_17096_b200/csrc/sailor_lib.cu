@@ -11,6 +11,7 @@
 #include <algorithm>
 
 #include "sailor_dp.cuh"
+#include "sailor_mixed.cuh"
 
 using namespace sailor;
 
@@ -143,6 +144,36 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
             }
             __syncwarp();
         }
+    }
+}
+
+// One thread per plan with mixed replicas (648-byte records, read in place: a thread walks its own
+// record several times, the second time from L1/L2).  Tables in shared memory, per-thread GPU counters
+// in shared memory as [digit][thread].
+__global__ void __launch_bounds__(SIM_THREADS)
+simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
+                      const sailor_mixed_plan* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
+                      uint64_t* __restrict__ peak_mem, double* __restrict__ cost, uint32_t* __restrict__ status,
+                      unsigned int* error) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ uint64_t mbar;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(blob)->static_bytes;
+    if (!bulk_load(dyn, blob, static_bytes, &mbar)) {
+        if (tid == 0) atomicExch(error, 1u);
+        for (uint32_t x = tid; x < static_bytes / 16; x += SIM_THREADS)
+            reinterpret_cast<uint4*>(dyn)[x] = reinterpret_cast<const uint4*>(blob)[x];
+        __syncthreads();
+    }
+    TabView v;
+    v.bind(dyn, blob);
+    uint32_t* counters = reinterpret_cast<uint32_t*>(dyn + static_bytes) + tid;
+    for (uint64_t j = (uint64_t)blockIdx.x * SIM_THREADS + tid; j < n; j += (uint64_t)gridDim.x * SIM_THREADS) {
+        const SimOut o = simulate_mixed_record(v, avail, plans[j], counters, SIM_THREADS);
+        if (t_iter) t_iter[j] = o.t_iter;
+        if (peak_mem) peak_mem[j] = o.peak_mem;
+        if (cost) cost[j] = o.cost;
+        if (status) status[j] = o.status;
     }
 }
 
@@ -725,6 +756,7 @@ int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_c
     CUF(cudaStreamSynchronize(ctx->stream));           // `blob` is pageable host memory
     // both kernels stage the static tables in dynamic shared memory; the create-time limit is 96 KB
     CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
+    CUF(cudaFuncSetAttribute(simulate_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
     CUF(cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
 #undef CUF
     *out = ctx;
@@ -809,6 +841,64 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
     const size_t sim_smem = ctx->hdr.static_bytes + sizeof(uint32_t) * SIM_THREADS * ctx->hdr.R;   // tables + per-thread counters
     simulate_kernel<<<grid, SIM_THREADS, sim_smem, ctx->stream>>>(
         ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s, &ctx->d_ctrl->error);
+    CU(ctx, cudaGetLastError());
+    if (!on_device) {
+        if (t_iter) CU(ctx, cudaMemcpyAsync(t_iter, d_t, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
+        if (cost) CU(ctx, cudaMemcpyAsync(cost, d_c, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
+        if (peak_mem) CU(ctx, cudaMemcpyAsync(peak_mem, d_m, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
+        if (status) CU(ctx, cudaMemcpyAsync(status, d_s, 4 * n, cudaMemcpyDeviceToHost, ctx->stream));
+        CU(ctx, cudaStreamSynchronize(ctx->stream));
+    }
+    return SAILOR_OK;
+}
+
+int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint64_t n, int on_device, double* t_iter,
+                          uint64_t* peak_mem, double* cost, uint32_t* status) {
+    if (!ctx || (!plans && n)) return SAILOR_E_ARG;
+    if (n == 0) return SAILOR_OK;
+    if ((uintptr_t)plans % 8 != 0) return SAILOR_E_ARG;
+    DeviceGuard guard(ctx->device);
+    const sailor_mixed_plan* d_plans = plans;
+    double *d_t = t_iter, *d_c = cost;
+    uint64_t* d_m = peak_mem;
+    uint32_t* d_s = status;
+    if (!on_device) {
+        const TabHdr& h = ctx->hdr;
+        for (uint64_t j = 0; j < n; ++j) {
+            const sailor_mixed_plan& r = plans[j];
+            if (r.P < 1 || r.P > SAILOR_MIX_P_MAX || r.D < 1 || r.mbs_idx >= h.n_mbs) return SAILOR_E_RANGE;
+            for (uint32_t i = 0; i < r.P; ++i) {
+                const sailor_mixed_stage& st = r.stage[i];
+                if (st.zone >= h.Z || st.n_groups < 1 || st.n_groups > SAILOR_MIX_GROUPS_MAX) return SAILOR_E_RANGE;
+                for (uint32_t q = 0; q < st.n_groups; ++q)
+                    if (st.group[q].type >= h.T || st.group[q].tp_idx >= h.n_tp) return SAILOR_E_RANGE;
+            }
+        }
+        const size_t need = n * (sizeof(sailor_mixed_plan) + 32);
+        if (need > ctx->stage_bytes) {
+            CU(ctx, cudaStreamSynchronize(ctx->stream));
+            cudaFree(ctx->d_stage);
+            ctx->d_stage = nullptr;
+            ctx->stage_bytes = 0;
+            cudaError_t e = cudaMalloc(&ctx->d_stage, need);
+            if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
+            ctx->stage_bytes = need;
+        }
+        unsigned char* base = ctx->d_stage;
+        d_t = reinterpret_cast<double*>(base);
+        d_c = reinterpret_cast<double*>(base + 8 * n);
+        d_m = reinterpret_cast<uint64_t*>(base + 16 * n);
+        d_s = reinterpret_cast<uint32_t*>(base + 24 * n);
+        sailor_mixed_plan* dp = reinterpret_cast<sailor_mixed_plan*>(base + 32 * n);
+        CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_mixed_plan), cudaMemcpyHostToDevice, ctx->stream));
+        d_plans = dp;
+    }
+    const uint64_t tiles = (n + SIM_THREADS - 1) / SIM_THREADS;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 16;
+    const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
+    const size_t smem = ctx->hdr.static_bytes + sizeof(uint32_t) * SIM_THREADS * ctx->hdr.R;
+    simulate_mixed_kernel<<<grid, SIM_THREADS, smem, ctx->stream>>>(ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s,
+                                                                     &ctx->d_ctrl->error);
     CU(ctx, cudaGetLastError());
     if (!on_device) {
         if (t_iter) CU(ctx, cudaMemcpyAsync(t_iter, d_t, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
