@@ -38,7 +38,11 @@ struct DpProblem {
     uint32_t stride[SAILOR_Z_MAX][SAILOR_T_MAX];   // mixed-radix stride of a counted type; 0: not counted
     uint32_t S[SAILOR_Z_MAX];        // entries of one (position, type) slice
     uint32_t zp_base[SAILOR_Z_MAX + 1];            // first entry of each position's T slices
+    uint32_t _pad;
+    uint64_t magic[SAILOR_Z_MAX][SAILOR_T_MAX];    // ceil(2^64 / (cap + 1)) of a counted type: for 32-bit x,
+                                                   // x / (cap + 1) == high 64 bits of x * magic
 };
+static_assert(sizeof(DpProblem) % 8 == 0, "copied word by word");
 
 struct DpResult {                    // per problem, written by dp_finish_kernel
     double value;                    // +inf: no plan
@@ -164,18 +168,31 @@ __global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_const
     const double* tab = lp.tabs + (size_t)pb.config * lp.lay.stride();
     const uint32_t* okv = reinterpret_cast<const uint32_t*>(tab + lp.lay.off_ok());
     const double nb = (double)*reinterpret_cast<const uint64_t*>(tab + lp.lay.off_nb());
-    // entry -> (zone position, type, counts)
+    // entry -> (zone position, type, counts); no division by run-time values: the slices of a position are
+    // stepped through, and the counts come off by multiplication with the precomputed reciprocals
     uint32_t zp = 0;
     while (zp + 1 < pb.nz && e >= pb.zp_base[zp + 1]) ++zp;
-    const uint32_t g = (e - pb.zp_base[zp]) / pb.S[zp], ui = (e - pb.zp_base[zp]) % pb.S[zp];
+    uint32_t g = 0, ui = e - pb.zp_base[zp];
+    const uint32_t S = pb.S[zp];
+    while (ui >= S) { ui -= S; ++g; }
+    uint32_t u[SAILOR_T_MAX];
+    uint32_t placed = 0;
+    {
+        uint32_t rem = ui;
+#pragma unroll
+        for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
+            u[t] = 0;
+            if (t < T && pb.stride[zp][t]) {
+                const uint32_t q = (uint32_t)__umul64hi((uint64_t)rem, pb.magic[zp][t]);
+                u[t] = rem - q * (pb.cap[zp][t] + 1u);
+                rem = q;
+                placed += u[t];
+            }
+        }
+    }
     // stage i is at most the (i+1)-th stage of its zone: entries that count more are never reached, and
     // since a move raises the count by one per stage, no entry that passes this test ever reads one that fails it
-    {
-        uint32_t placed = 0;
-        for (uint32_t t = 0; t < T; ++t)
-            if (pb.stride[zp][t]) placed += (ui / pb.stride[zp][t]) % (pb.cap[zp][t] + 1u);
-        if (placed > i + 1) return;
-    }
+    if (placed > i + 1) return;
     DpVal* cur = lp.val[lp.dist & 1] + pb.val_off;
     const DpVal* nxt = lp.val[(lp.dist & 1) ^ 1] + pb.val_off;
     uint8_t* choice = lp.choice + pb.choice_off + (size_t)i * pb.n_lvl;
@@ -183,8 +200,10 @@ __global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_const
     best.sum = make_inf(); best.mx = best.sy = best.up = 0.0;
     uint8_t pick = DP_NONE;
     // a state holds stage i itself: its type must be usable there and, when counted, counted at least once
-    const uint32_t st_g = pb.stride[zp][g];
-    const bool self = ((okv[i] >> g) & 1u) && pb.cap[zp][g] >= 1 && (st_g == 0 || (ui / st_g) % (pb.cap[zp][g] + 1u) >= 1);
+    uint32_t u_g = 0;
+#pragma unroll
+    for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) u_g = t == g ? u[t] : u_g;
+    const bool self = ((okv[i] >> g) & 1u) && pb.cap[zp][g] >= 1 && (pb.stride[zp][g] == 0 || u_g >= 1);
     if (self) {
         const uint32_t d = pb.zone[zp] * T + g;
         const double fb = tab[lp.lay.off_fb() + i * T + g], upd = tab[lp.lay.off_upd() + i * T + g];
@@ -194,13 +213,26 @@ __global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_const
         } else {
             double best_v = make_inf();
             const uint32_t ok_next = okv[i + 1];
-            for (uint32_t g2 = 0; g2 < T; ++g2) {
+            const uint32_t here_base = pb.zp_base[zp] + ui;
+#pragma unroll
+            for (uint32_t g2 = 0; g2 < SAILOR_T_MAX; ++g2) {
+                if (g2 >= T) break;
                 if (!((ok_next >> g2) & 1u)) continue;
-                const DpMove mv = dp_move(pb, zp, ui, g2);
-                if (mv.zp == DP_NONE) continue;
-                const DpVal n = nxt[mv.entry];
+                // first fit: this zone while it has room for one more stage of the type, else the next zone that has
+                const uint32_t st2 = pb.stride[zp][g2], cap2 = pb.cap[zp][g2];
+                const bool here = st2 == 0 ? cap2 >= 1 : u[g2] < cap2;
+                uint32_t zp2, entry;
+                if (here) {
+                    zp2 = zp;
+                    entry = here_base + g2 * S + st2;
+                } else {
+                    zp2 = pb.first_later[zp][g2];
+                    if (zp2 == DP_NONE) continue;
+                    entry = pb.zp_base[zp2] + g2 * pb.S[zp2] + pb.stride[zp2][g2];
+                }
+                const DpVal n = nxt[entry];
                 if (!(n.sum < make_inf())) continue;
-                const uint32_t d2 = pb.zone[mv.zp] * T + g2;
+                const uint32_t d2 = pb.zone[zp2] * T + g2;
                 const double t = add_rn(fb, tab[lp.lay.off_c2x() + (size_t)d2 * lp.lay.R + d]);
                 DpVal c;
                 c.sum = add_rn(t, n.sum);

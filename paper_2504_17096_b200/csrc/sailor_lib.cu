@@ -1278,6 +1278,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
                     const uint64_t cap = ctx->h_avail[pb.zone[zp] * T + g] / need;
                     pb.cap[zp][g] = (uint8_t)(cap > 255 ? 255 : cap);
                     if (cap >= 1 && cap < cf.P) {           // counted: the zone cannot host every stage
+                        pb.magic[zp][g] = ~0ull / (cap + 1) + 1;                // ceil(2^64 / (cap + 1)), cap + 1 >= 2
                         pb.stride[zp][g] = (uint32_t)S;
                         S *= cap + 1;
                         if (S > (1ull << 31)) return SAILOR_E_RANGE;
