@@ -15,7 +15,9 @@
  * scaling invariants; an independent nested-loop enumeration and brute-force minimum on
  * tiny clusters.  The pruned search modes (H2-H4): three hand-worked searches, equality with the
  * exhaustive search when no mode is on, and a brute-force restatement over per-candidate results
- * on tiny clusters (group minimum over tensor-parallel degrees, per-configuration bests).
+ * on tiny clusters (group minimum over tensor-parallel degrees, per-configuration bests).  The
+ * dynamic-programming recursion and the simulator for plans that mix GPU types inside a stage: see the
+ * comments above their declarations below.
  * Parity unpinned: the absolute realism of the outputs against real clusters (Sec. 5.1
  * reports 4-6 % error on hardware this repository cannot reach).
  */

@@ -98,6 +98,23 @@ def _tiny():
     yield w, [[0, 1], [1, 0]]
 
 
+def test_dp_deepest_pipelines_and_bandwidth_polynomials():
+    """96 stages (the limit), pipelines that do not divide the layer count, and message-size-dependent links."""
+    w = W.tiny(seed=31, n_types=2, n_zones=2, L=96, p_values=[96, 64, 7], d_values=(1, 2), tp_values=(1, 2),
+               mbs_values=(1, 2), gbs=64)
+    w.capacity[...] = w.capacity * 8
+    w.avail[...] = np.array([[70, 40], [90, 200]], dtype=np.uint16)      # scarce enough that plans change zone and type
+    for wl in (w, W.with_bandwidth_polynomials(W.tiny(seed=41, n_types=3, n_zones=2, L=6, p_values=[2, 3, 6]), seed=1)):
+        orders = [[0, 1], [1, 0]]
+        o = Oracle(wl)
+        want = oracle_all(wl, o, orders)
+        assert len(want) >= 4
+        with Ctx(wl) as cx:
+            res, st = B.sailor_plan_dp(cx.ctx, cx.space, orders, 32)
+        assert_dp_equal(res, st, want, wl, o, orders, 32, wl.name)
+        assert any(len(set(x[2]["types"])) > 1 for x in want), "no plan ever mixes types across stages"
+
+
 @pytest.mark.parametrize("w,orders", list(_tiny()), ids=lambda x: getattr(x, "name", None))
 def test_dp_matches_oracle_on_tiny_clusters(w, orders):
     o = Oracle(w)

@@ -122,6 +122,23 @@ def test_modes_match_oracle_on_tiny_spaces(w, modes):
             assert_same(res, st, hits, counts, f"{w.name} eval-all")
 
 
+def test_modes_with_deep_pipelines_and_bandwidth_polynomials():
+    """Up to 96 stages, non-divisor depths, four segments, message-size-dependent links."""
+    deep = W.tiny(seed=31, n_types=2, n_zones=2, L=96, p_values=[96, 48, 7], d_values=(4, 1, 2), tp_values=(1, 2, 4),
+                  mbs_values=(1, 2), gbs=64)
+    deep.capacity[...] = deep.capacity * 4
+    deep.avail[...] = 300
+    for w in (deep, W.with_bandwidth_polynomials(W.tiny(seed=41, n_types=3, n_zones=2), seed=1)):
+        o = Oracle(w)
+        with Ctx(w) as cx:
+            for modes in (PRUNE_D_ORDER, PRUNE_MIN_TP, PRUNE_D_ORDER | PRUNE_MIN_TP):
+                for kind in (0, 1):
+                    hits, counts = o.search_pruned(kind, 16, modes)
+                    res, st = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, kind=kind, flags=gpu_flags(modes), factor=0.0,
+                                                                               budget=0.0, min_rate=0.0), 16)
+                    assert_same(res, st, hits, counts, f"{w.name} modes={modes} kind={kind}")
+
+
 @pytest.mark.parametrize("cfg", [1, 2, 6])
 @pytest.mark.parametrize("modes", [PRUNE_D_ORDER, PRUNE_D_ORDER | PRUNE_MIN_TP, PRUNE_MIN_TP])
 def test_modes_match_oracle_on_workloads(cfg, modes):
