@@ -4,9 +4,12 @@
 // (stage i, type g of stage i, zone position zp of stage i, u = stages per type already placed in
 // that zone, stage i included).  Zones before zp are never revisited and zones after it are
 // untouched (first fit), so nothing else of the past matters.  A type that a zone could give to all
-// P stages is not counted in u.  States are laid out densely: for every zone position and type a
-// slice of S[zp] entries indexed by u in mixed radix.  The value of a state is the best plan of
-// stages i.. from it: (sum of stage times, straggler, slowest synchronisation, slowest update).
+// P stages is not counted in u.  For every zone position and type there is a slice of S[zp] entries
+// indexed by u, in one of two ways chosen per zone position: densely in mixed radix (radix cap + 1 per
+// counted type), or compactly by the rank of u among the count vectors that respect the caps and add
+// up to at most P (a zone never holds more than P stages); the compact index is much smaller when
+// many types are scarce at once.  The value of a state is the best plan of stages i.. from it:
+// (sum of stage times, straggler, slowest synchronisation, slowest update).
 //
 // The tables are filled from the last stage to the first.  One launch handles one stage distance
 // from the end for every problem of a batch (problems are sorted by depth, so the launch for
@@ -21,6 +24,7 @@ namespace sailor {
 
 constexpr int DP_THREADS = 256;
 constexpr uint8_t DP_NONE = 255;
+constexpr uint32_t DP_DENSE = 0xffffffffu;
 
 struct DpVal {                       // best plan of stages i.. from a state; sum = +inf: there is none
     double sum, mx, sy, up;
@@ -39,6 +43,8 @@ struct DpProblem {
     uint32_t S[SAILOR_Z_MAX];        // entries of one (position, type) slice
     uint32_t zp_base[SAILOR_Z_MAX + 1];            // first entry of each position's T slices
     uint32_t _pad;
+    uint32_t first_idx[SAILOR_Z_MAX][SAILOR_T_MAX];    // index of "one stage, of this type" inside a slice
+    uint32_t vt_off[SAILOR_Z_MAX];   // compact index: offset of the position's rank table in `vtabs`; DP_DENSE: mixed radix
     uint64_t magic[SAILOR_Z_MAX][SAILOR_T_MAX];    // ceil(2^64 / (cap + 1)) of a counted type: for 32-bit x,
                                                    // x / (cap + 1) == high 64 bits of x * magic
 };
@@ -120,24 +126,103 @@ dp_tables_kernel(const unsigned char* __restrict__ blob, SpaceDesc sp, uint32_t 
     }
 }
 
-// Where does a stage of type g2 go when the previous stage sits at position zp with counts u?
+// ---- the index of a count vector inside a slice -------------------------------------------------------
+//
+// Compact index of zone position zp: the counted types j = 0 .. m-1 (ascending type) have caps c_j.  With
+// W[j][s] = number of (u_j .. u_{m-1}) within the caps that add up to at most s, and V[j][s] = W[j][0] + .. +
+// W[j][s], the rank of u in lexicographic order is sum_j (V[j+1][s_j] - V[j+1][s_j - u_j]), s_0 = P,
+// s_{j+1} = s_j - u_j.  The table holds V[j][s] for j = 0 .. m, s = 0 .. P, row after row.
+
+// counts of a slice index: u[t] for counted types, 0 for the others
+__device__ __forceinline__ void dp_counts(const DpProblem& pb, const uint32_t* __restrict__ vtabs, uint32_t zp, uint32_t T,
+                                          uint32_t ui, uint32_t (&u)[SAILOR_T_MAX]) {
+    if (pb.vt_off[zp] == DP_DENSE) {
+        uint32_t rem = ui;
+#pragma unroll
+        for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
+            u[t] = 0;
+            if (t < T && pb.stride[zp][t]) {
+                const uint32_t q = (uint32_t)__umul64hi((uint64_t)rem, pb.magic[zp][t]);
+                u[t] = rem - q * (pb.cap[zp][t] + 1u);
+                rem = q;
+            }
+        }
+    } else {
+        const uint32_t* vt = vtabs + pb.vt_off[zp];
+        const uint32_t w = pb.P + 1;
+        uint32_t r = ui, s = pb.P, j = 0;
+#pragma unroll
+        for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
+            u[t] = 0;
+            if (t < T && pb.stride[zp][t]) {
+                const uint32_t* row = vt + (j + 1) * w;
+                const uint32_t top = row[s], lim = min((uint32_t)pb.cap[zp][t], s);
+                uint32_t x = 0, below = 0;                       // `below`: vectors that start with a count smaller than x
+                while (x < lim) {
+                    const uint32_t nxt = top - row[s - x - 1];              // x < lim <= s
+                    if (nxt > r) break;
+                    below = nxt;
+                    ++x;
+                }
+                u[t] = x;
+                r -= below;
+                s -= x;
+                ++j;
+            }
+        }
+    }
+}
+
+// slice index of the count vector u with one more stage of type `plus_one` (compact index only)
+__device__ __forceinline__ uint32_t dp_rank(const DpProblem& pb, const uint32_t* __restrict__ vtabs, uint32_t zp, uint32_t T,
+                                            const uint32_t (&u)[SAILOR_T_MAX], uint32_t plus_one) {
+    const uint32_t* vt = vtabs + pb.vt_off[zp];
+    const uint32_t w = pb.P + 1;
+    uint32_t r = 0, s = pb.P, j = 0;
+#pragma unroll
+    for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
+        if (t < T && pb.stride[zp][t]) {
+            const uint32_t x = u[t] + (t == plus_one ? 1u : 0u);
+            const uint32_t* row = vt + (j + 1) * w;
+            if (x) r += row[s] - row[s - x];                     // the caller keeps the counts within P in total
+            s -= x;
+            ++j;
+        }
+    }
+    return r;
+}
+
+// Where does a stage of type g2 go when the previous stage sits at position zp with counts u (slice index ui)?
 // Returns the position (DP_NONE: nowhere) and the entry index of the state that results.
 struct DpMove { uint32_t zp, entry; };
 
-__device__ __forceinline__ DpMove dp_move(const DpProblem& pb, uint32_t zp, uint32_t ui, uint32_t g2) {
+__device__ __forceinline__ DpMove dp_move(const DpProblem& pb, const uint32_t* __restrict__ vtabs, uint32_t T, uint32_t zp,
+                                          uint32_t ui, const uint32_t (&u)[SAILOR_T_MAX], uint32_t g2) {
     DpMove m;
-    const uint32_t st = pb.stride[zp][g2], cap = pb.cap[zp][g2];
-    bool here;
-    if (st == 0) here = cap >= 1;                                  // not counted: room for every stage, or none at all
-    else here = (ui / st) % (cap + 1u) < cap;
+    const uint32_t cap = pb.cap[zp][g2];
+    uint32_t u_g2 = 0, placed = 0;
+#pragma unroll
+    for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
+        u_g2 = t == g2 ? u[t] : u_g2;
+        placed += u[t];
+    }
+    // first fit: this zone while it has room for one more stage of the type, else the next zone that has
+    const bool counted = pb.stride[zp][g2] != 0;
+    const bool here = counted ? u_g2 < cap : cap >= 1;           // not counted: room for every stage, or none at all
     if (here) {
         m.zp = zp;
-        m.entry = pb.zp_base[zp] + g2 * pb.S[zp] + ui + st;
+        uint32_t idx = ui;
+        if (counted) {
+            if (pb.vt_off[zp] == DP_DENSE) idx = ui + pb.stride[zp][g2];
+            else if (placed >= pb.P) { m.zp = DP_NONE; m.entry = 0; return m; }      // more than P stages: no such state
+            else idx = dp_rank(pb, vtabs, zp, T, u, g2);
+        }
+        m.entry = pb.zp_base[zp] + g2 * pb.S[zp] + idx;
         return m;
     }
     const uint32_t p = pb.first_later[zp][g2];
     m.zp = p;
-    m.entry = p == DP_NONE ? 0u : pb.zp_base[p] + g2 * pb.S[p] + pb.stride[p][g2];      // the new zone holds this stage only
+    m.entry = p == DP_NONE ? 0u : pb.zp_base[p] + g2 * pb.S[p] + pb.first_idx[p][g2];      // the new zone holds this stage only
     return m;
 }
 
@@ -146,6 +231,7 @@ struct DpLevelParams {
     const uint32_t* blk_problem;     // block -> problem of the batch
     const uint32_t* blk_first;       // block -> first entry it covers
     const double* tabs;
+    const uint32_t* vtabs;           // rank tables of the compactly indexed zone positions
     DpVal* val[2];                   // level buffers; stage i lives in val[(P - 1 - i) & 1]
     uint8_t* choice;
     DpTabLayout lay;
@@ -153,7 +239,7 @@ struct DpLevelParams {
     uint32_t dist;                   // stage i = P - 1 - dist
 };
 
-__global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_constant__ DpLevelParams lp) {
+__global__ void __launch_bounds__(DP_THREADS, 4) dp_level_kernel(const __grid_constant__ DpLevelParams lp) {
     __shared__ DpProblem pb;
     const uint32_t tid = threadIdx.x;
     {
@@ -169,27 +255,17 @@ __global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_const
     const uint32_t* okv = reinterpret_cast<const uint32_t*>(tab + lp.lay.off_ok());
     const double nb = (double)*reinterpret_cast<const uint64_t*>(tab + lp.lay.off_nb());
     // entry -> (zone position, type, counts); no division by run-time values: the slices of a position are
-    // stepped through, and the counts come off by multiplication with the precomputed reciprocals
+    // stepped through, and the counts come off by reciprocal multiplication or by a walk through the rank table
     uint32_t zp = 0;
     while (zp + 1 < pb.nz && e >= pb.zp_base[zp + 1]) ++zp;
     uint32_t g = 0, ui = e - pb.zp_base[zp];
     const uint32_t S = pb.S[zp];
     while (ui >= S) { ui -= S; ++g; }
     uint32_t u[SAILOR_T_MAX];
+    dp_counts(pb, lp.vtabs, zp, T, ui, u);
     uint32_t placed = 0;
-    {
-        uint32_t rem = ui;
 #pragma unroll
-        for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
-            u[t] = 0;
-            if (t < T && pb.stride[zp][t]) {
-                const uint32_t q = (uint32_t)__umul64hi((uint64_t)rem, pb.magic[zp][t]);
-                u[t] = rem - q * (pb.cap[zp][t] + 1u);
-                rem = q;
-                placed += u[t];
-            }
-        }
-    }
+    for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) placed += u[t];
     // stage i is at most the (i+1)-th stage of its zone: entries that count more are never reached, and
     // since a move raises the count by one per stage, no entry that passes this test ever reads one that fails it
     if (placed > i + 1) return;
@@ -213,23 +289,13 @@ __global__ void __launch_bounds__(DP_THREADS) dp_level_kernel(const __grid_const
         } else {
             double best_v = make_inf();
             const uint32_t ok_next = okv[i + 1];
-            const uint32_t here_base = pb.zp_base[zp] + ui;
 #pragma unroll
             for (uint32_t g2 = 0; g2 < SAILOR_T_MAX; ++g2) {
                 if (g2 >= T) break;
                 if (!((ok_next >> g2) & 1u)) continue;
-                // first fit: this zone while it has room for one more stage of the type, else the next zone that has
-                const uint32_t st2 = pb.stride[zp][g2], cap2 = pb.cap[zp][g2];
-                const bool here = st2 == 0 ? cap2 >= 1 : u[g2] < cap2;
-                uint32_t zp2, entry;
-                if (here) {
-                    zp2 = zp;
-                    entry = here_base + g2 * S + st2;
-                } else {
-                    zp2 = pb.first_later[zp][g2];
-                    if (zp2 == DP_NONE) continue;
-                    entry = pb.zp_base[zp2] + g2 * pb.S[zp2] + pb.stride[zp2][g2];
-                }
+                const DpMove mv = dp_move(pb, lp.vtabs, T, zp, ui, u, g2);
+                if (mv.zp == DP_NONE) continue;
+                const uint32_t zp2 = mv.zp, entry = mv.entry;
                 const DpVal n = nxt[entry];
                 if (!(n.sum < make_inf())) continue;
                 const uint32_t d2 = pb.zone[zp2] * T + g2;
@@ -255,6 +321,7 @@ struct DpFinishParams {
     SpaceDesc sp;
     const DpProblem* problems;
     const double* tabs;
+    const uint32_t* vtabs;
     const DpVal* val[2];
     const uint8_t* choice;
     DpResult* results;               // indexed by problem index
@@ -278,7 +345,7 @@ __global__ void __launch_bounds__(128) dp_finish_kernel(const __grid_constant__ 
         if (!((okv[0] >> g0) & 1u)) continue;
         const uint32_t p = pb.cap[0][g0] >= 1 ? 0u : pb.first_later[0][g0];
         if (p == DP_NONE) continue;
-        const uint32_t e = pb.zp_base[p] + g0 * pb.S[p] + pb.stride[p][g0];
+        const uint32_t e = pb.zp_base[p] + g0 * pb.S[p] + pb.first_idx[p][g0];
         const DpVal v = lvl0[e];
         if (!(v.sum < make_inf())) continue;
         const double val = add_rn(add_rn(add_rn(v.sum, mul_rn(nb, v.mx)), v.sy), v.up);
@@ -302,7 +369,9 @@ __global__ void __launch_bounds__(128) dp_finish_kernel(const __grid_constant__ 
         if (i + 1 == P) break;
         const uint8_t g2 = fp.choice[pb.choice_off + (size_t)i * pb.n_lvl + entry];
         const uint32_t ui = (entry - pb.zp_base[zp]) % pb.S[zp];
-        const DpMove mv = dp_move(pb, zp, ui, g2);
+        uint32_t u[SAILOR_T_MAX];
+        dp_counts(pb, fp.vtabs, zp, T, ui, u);
+        const DpMove mv = dp_move(pb, fp.vtabs, T, zp, ui, u, g2);
         g = g2; zp = mv.zp; entry = mv.entry;
     }
     // the plan written out, through the simulator (Sec. 4.3): what a caller compares with a constraint

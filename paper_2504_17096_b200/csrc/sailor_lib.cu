@@ -1256,6 +1256,11 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     // every problem's table layout, from the availability last set (host copy)
     const uint64_t n_problems = n_config * n_orders;
     std::vector<DpProblem> prob(n_problems);
+    std::vector<uint32_t> vtabs;        // rank tables of the compactly indexed zone positions, all problems
+    // how a zone position's count vectors are indexed: 0 = the smaller of the two ways, 1 = mixed radix whenever it
+    // fits, 2 = by rank whenever it fits (the environment variable exists for tests that exercise each way)
+    int index_mode = 0;
+    if (const char* env = getenv("SAILOR_DP_INDEX")) index_mode = !strcmp(env, "dense") ? 1 : !strcmp(env, "compact") ? 2 : 0;
     uint64_t n_states = 0;
     for (uint64_t c = 0; c < n_config; ++c) {
         const Config cf = config_of(d, (uint32_t)c);
@@ -1273,15 +1278,59 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
             uint64_t n_lvl = 0;
             for (uint32_t zp = 0; zp < pb.nz; ++zp) {
                 pb.zone[zp] = orders[q].zone[zp];
-                uint64_t S = 1;
+                // counted types: the zone can host some but not all P stages of them
+                uint32_t counted[SAILOR_T_MAX], m = 0;
+                uint64_t dense = 1;
+                bool dense_ok = true;
                 for (uint32_t g = 0; g < T; ++g) {
                     const uint64_t cap = ctx->h_avail[pb.zone[zp] * T + g] / need;
                     pb.cap[zp][g] = (uint8_t)(cap > 255 ? 255 : cap);
-                    if (cap >= 1 && cap < cf.P) {           // counted: the zone cannot host every stage
-                        pb.magic[zp][g] = ~0ull / (cap + 1) + 1;                // ceil(2^64 / (cap + 1)), cap + 1 >= 2
+                    if (cap >= 1 && cap < cf.P) {
+                        counted[m++] = g;
+                        if (dense_ok) dense *= cap + 1;
+                        if (dense > (1ull << 31)) dense_ok = false;
+                    }
+                }
+                // compact index: count vectors within the caps that add up to at most P (rank tables V[j][s])
+                const uint32_t w = cf.P + 1;
+                std::vector<uint64_t> V((size_t)(m + 1) * w);
+                for (uint32_t sgm = 0; sgm < w; ++sgm) V[(size_t)m * w + sgm] = sgm + 1;           // W = 1 each
+                bool compact_ok = true;
+                for (uint32_t j = m; j-- > 0;) {
+                    const uint64_t cj = pb.cap[zp][counted[j]];
+                    uint64_t run = 0;
+                    for (uint32_t sgm = 0; sgm < w; ++sgm) {
+                        const uint64_t lo = sgm > cj ? V[(size_t)(j + 1) * w + (sgm - cj - 1)] : 0;
+                        run += V[(size_t)(j + 1) * w + sgm] - lo;                                  // W[j][s]
+                        V[(size_t)j * w + sgm] = run;
+                        if (run > (1ull << 31)) compact_ok = false;
+                    }
+                }
+                const uint64_t compact = m ? V[cf.P] - (cf.P ? V[cf.P - 1] : 0) : 1;                // W[0][P]
+                if (!dense_ok && !compact_ok) return SAILOR_E_RANGE;
+                const bool use_compact = index_mode == 2 ? compact_ok && m > 0
+                                         : index_mode == 1 ? !dense_ok
+                                                           : (m > 0 && compact_ok && (!dense_ok || dense > 4 * compact));
+                uint64_t S = 1;
+                if (use_compact) {
+                    S = compact;
+                    pb.vt_off[zp] = (uint32_t)vtabs.size();
+                    for (uint64_t x : V) vtabs.push_back((uint32_t)x);
+                    for (uint32_t j = 0; j < m; ++j) {
+                        // rank of "one stage of type counted[j]": every vector that has a zero there and is zero before it
+                        // comes first: V[j+1][P] - V[j+1][P-1] ... summed by the rank formula with u = e_j
+                        pb.stride[zp][counted[j]] = 1;                                         // marks the type as counted
+                        pb.first_idx[zp][counted[j]] = (uint32_t)(V[(size_t)(j + 1) * w + cf.P] - V[(size_t)(j + 1) * w + cf.P - 1]);
+                    }
+                    if (vtabs.size() > (1ull << 30)) return SAILOR_E_RANGE;
+                } else {
+                    pb.vt_off[zp] = DP_DENSE;
+                    for (uint32_t j = 0; j < m; ++j) {
+                        const uint32_t g = counted[j];
+                        pb.magic[zp][g] = ~0ull / (pb.cap[zp][g] + 1ull) + 1;                  // ceil(2^64 / (cap + 1)), cap + 1 >= 2
                         pb.stride[zp][g] = (uint32_t)S;
-                        S *= cap + 1;
-                        if (S > (1ull << 31)) return SAILOR_E_RANGE;
+                        pb.first_idx[zp][g] = (uint32_t)S;
+                        S *= pb.cap[zp][g] + 1ull;
                     }
                 }
                 pb.S[zp] = (uint32_t)S;
@@ -1338,7 +1387,8 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     DpTabLayout lay;
     lay.p_max = p_max; lay.T = T; lay.R = h.R;
     const size_t tab_bytes = (size_t)n_config * lay.stride() * sizeof(double);
-    const size_t total = padded(tab_bytes) + padded(n_problems * sizeof(DpResult)) + padded(n_problems * sizeof(DpProblem)) +
+    const size_t total = padded(tab_bytes) + padded(vtabs.size() * sizeof(uint32_t) + 4) + padded(n_problems * sizeof(DpResult)) +
+                         padded(n_problems * sizeof(DpProblem)) +
                          2 * padded(max_blocks * sizeof(uint32_t)) + 2 * padded(max_entries * sizeof(DpVal)) +
                          padded(max_choice) + padded(sizeof(sailor_dp_result) * SAILOR_K_MAX) + padded(24) + 4096;
     if (total > ctx->dp_bytes) {
@@ -1352,6 +1402,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     }
     Bump bump{ctx->d_dp};
     double* d_tabs = bump.take<double>(tab_bytes / sizeof(double));
+    uint32_t* d_vtabs = bump.take<uint32_t>(vtabs.size() + 1);
     DpResult* d_results = bump.take<DpResult>(n_problems);
     DpProblem* d_problems = bump.take<DpProblem>(n_problems);
     uint32_t* d_blk_problem = bump.take<uint32_t>(max_blocks);
@@ -1366,6 +1417,8 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
     CU(ctx, cudaMemsetAsync(d_tabs, 0, tab_bytes, ctx->stream));
     CU(ctx, cudaMemsetAsync(d_counters, 0, 24, ctx->stream));
+    if (!vtabs.empty())
+        CU(ctx, cudaMemcpyAsync(d_vtabs, vtabs.data(), vtabs.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
     {
         const uint32_t grid = (uint32_t)(n_config < 4096 ? n_config : 4096);
         dp_tables_kernel<<<grid, DP_THREADS, 0, ctx->stream>>>(ctx->d_blob, d, (uint32_t)n_config, lay, d_tabs);
@@ -1384,7 +1437,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
                                     ctx->stream));
             DpFinishParams fp;
             memset(&fp, 0, sizeof(fp));
-            fp.blob = ctx->d_blob; fp.avail = ctx->d_avail; fp.sp = d; fp.problems = d_problems; fp.tabs = d_tabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
+            fp.blob = ctx->d_blob; fp.avail = ctx->d_avail; fp.sp = d; fp.problems = d_problems; fp.tabs = d_tabs; fp.vtabs = d_vtabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
             fp.results = d_results; fp.lay = lay; fp.n_problems = (uint32_t)stage_buf.size(); fp.T = T;
             dp_finish_kernel<<<(fp.n_problems + 127) / 128, 128, 0, ctx->stream>>>(fp);
             CU(ctx, cudaGetLastError());
@@ -1419,6 +1472,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
         DpLevelParams lp;
         memset(&lp, 0, sizeof(lp));
         lp.problems = d_problems; lp.blk_problem = d_blk_problem; lp.blk_first = d_blk_first; lp.tabs = d_tabs;
+        lp.vtabs = d_vtabs;
         lp.val[0] = d_val0; lp.val[1] = d_val1; lp.choice = d_choice; lp.lay = lay; lp.T = T;
         for (uint32_t dist = 0; dist < max_p; ++dist) {
             lp.dist = dist;
@@ -1428,7 +1482,7 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
         }
         DpFinishParams fp;
         memset(&fp, 0, sizeof(fp));
-        fp.blob = ctx->d_blob; fp.avail = ctx->d_avail; fp.sp = d; fp.problems = d_problems; fp.tabs = d_tabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
+        fp.blob = ctx->d_blob; fp.avail = ctx->d_avail; fp.sp = d; fp.problems = d_problems; fp.tabs = d_tabs; fp.vtabs = d_vtabs; fp.val[0] = d_val0; fp.val[1] = d_val1; fp.choice = d_choice;
         fp.results = d_results; fp.lay = lay; fp.n_problems = (uint32_t)b.count; fp.T = T;
         dp_finish_kernel<<<(fp.n_problems + 127) / 128, 128, 0, ctx->stream>>>(fp);
         CU(ctx, cudaGetLastError());

@@ -24,6 +24,16 @@ def _needs_cuda():
         pytest.fail("the gpu tests need a CUDA device")
 
 
+@pytest.fixture(params=["auto", "dense", "compact"], autouse=True)
+def _index_mode(request, monkeypatch):
+    """Every test runs with each way of indexing the tables' count vectors (mixed radix, by rank, the smaller)."""
+    if request.param == "auto":
+        monkeypatch.delenv("SAILOR_DP_INDEX", raising=False)
+    else:
+        monkeypatch.setenv("SAILOR_DP_INDEX", request.param)
+    return request.param
+
+
 class Ctx:
     def __init__(self, w):
         self.ctx = B.sailor_create(w, 0, 0)
