@@ -125,6 +125,24 @@ def test_dp_deepest_pipelines_and_bandwidth_polynomials():
         assert any(len(set(x[2]["types"])) > 1 for x in want), "no plan ever mixes types across stages"
 
 
+def test_dp_eight_types_eight_zones(_index_mode):
+    """Eight scarce types in eight zones: one problem's mixed-radix tables need 24 GB, beyond the default
+    workspace of 8 GiB; indexed by rank they fit with room to spare."""
+    w = W.tiny(seed=14, n_types=8, n_zones=8, L=12, p_values=[12, 5], d_values=(1, 2), tp_values=(1, 2), mbs_values=(1, 4))
+    orders = [[7, 6, 5, 4, 3, 2, 1, 0], [2, 5]]
+    with Ctx(w) as cx:
+        if _index_mode == "dense":
+            with pytest.raises(B.SailorError) as e:
+                B.sailor_plan_dp(cx.ctx, cx.space, orders, 8)
+            assert e.value.code == B.E_RANGE
+            return
+        o = Oracle(w)
+        want = oracle_all(w, o, orders)
+        assert len(want) >= 8
+        res, st = B.sailor_plan_dp(cx.ctx, cx.space, orders, 32)
+        assert_dp_equal(res, st, want, w, o, orders, 32, w.name)
+
+
 @pytest.mark.parametrize("w,orders", list(_tiny()), ids=lambda x: getattr(x, "name", None))
 def test_dp_matches_oracle_on_tiny_clusters(w, orders):
     o = Oracle(w)
