@@ -622,8 +622,8 @@ const char* sailor_strerror(int code) {
 
 int sailor_last_cuda_error(const sailor_ctx* ctx) { return ctx ? ctx->last_cuda : 0; }
 
-int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_cluster* c, int cuda_device,
-                  void* cuda_stream, sailor_ctx** out) {
+static int create_impl(const sailor_model* m, const sailor_profile* p, const sailor_cluster* c, int cuda_device,
+                       void* cuda_stream, sailor_ctx** out) {
     if (!m || !p || !c || !out) return SAILOR_E_ARG;
     *out = nullptr;
     if (!p->fwd || !p->bwd || !p->upd || !p->params || !p->act_saved || !p->act_ckpt || !p->act_work ||
@@ -924,8 +924,8 @@ int sailor_decode(const sailor_ctx* ctx, const sailor_space* s, uint64_t flat, s
     return decode_flat(to_desc(s), ctx->hdr.T, ctx->hdr.Z, flat, out) ? SAILOR_OK : SAILOR_E_RANGE;
 }
 
-int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint64_t flat_lo,
-                      uint64_t flat_hi, uint32_t k, sailor_result* topk, uint32_t* n_found, sailor_stats* stats) {
+static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint64_t flat_lo,
+                           uint64_t flat_hi, uint32_t k, sailor_result* topk, uint32_t* n_found, sailor_stats* stats) {
     if (!ctx || !s || !o || !topk || !n_found || k == 0) return SAILOR_E_ARG;
     if (k > SAILOR_K_MAX || o->kind > SAILOR_OBJ_MAX_THROUGHPUT_PER_USD) return SAILOR_E_RANGE;
     if (std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) ||
@@ -1225,9 +1225,9 @@ size_t padded(size_t bytes) { return (bytes + 255) & ~(size_t)255; }
 
 }  // namespace
 
-extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders,
-                              uint32_t n_orders, const sailor_objective* o, uint64_t workspace_bytes, uint32_t k,
-                              sailor_dp_result* topk, uint32_t* n_found, sailor_dp_stats* stats) {
+static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders,
+                        uint32_t n_orders, const sailor_objective* o, uint64_t workspace_bytes, uint32_t k,
+                        sailor_dp_result* topk, uint32_t* n_found, sailor_dp_stats* stats) {
     if (!ctx || !s || !orders || !o || !topk || !n_found || k == 0 || n_orders == 0) return SAILOR_E_ARG;
     if (k > SAILOR_K_MAX) return SAILOR_E_RANGE;
     // the recursion minimises iteration time; a constraint is checked on the plan it returns per problem
@@ -1520,3 +1520,34 @@ extern "C" int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sail
     }
     return SAILOR_OK;
 }
+
+// ---- entry points that build host-side tables: no exception may cross the C boundary -------------------
+
+#define SAILOR_NO_THROW(call)                              \
+    try {                                                  \
+        return call;                                       \
+    } catch (const std::bad_alloc&) {                      \
+        return SAILOR_E_NOMEM;                             \
+    } catch (...) {                                        \
+        return SAILOR_E_ARG;                               \
+    }
+
+extern "C" {
+
+int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_cluster* c, int cuda_device,
+                  void* cuda_stream, sailor_ctx** out) {
+    SAILOR_NO_THROW(create_impl(m, p, c, cuda_device, cuda_stream, out))
+}
+
+int sailor_plan_range(sailor_ctx* ctx, const sailor_space* s, const sailor_objective* o, uint64_t flat_lo,
+                      uint64_t flat_hi, uint32_t k, sailor_result* topk, uint32_t* n_found, sailor_stats* stats) {
+    SAILOR_NO_THROW(plan_range_impl(ctx, s, o, flat_lo, flat_hi, k, topk, n_found, stats))
+}
+
+int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders, uint32_t n_orders,
+                   const sailor_objective* o, uint64_t workspace_bytes, uint32_t k, sailor_dp_result* topk,
+                   uint32_t* n_found, sailor_dp_stats* stats) {
+    SAILOR_NO_THROW(plan_dp_impl(ctx, s, orders, n_orders, o, workspace_bytes, k, topk, n_found, stats))
+}
+
+}  // extern "C"

@@ -56,7 +56,7 @@ __device__ inline SimOut simulate_mixed_record(const TabView& v, const uint16_t*
         const uint32_t nb = base + (i < extra ? 1u : 0u), ng = s.n_groups;
         const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
         const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
-        uint64_t replicas = 0, gradbytes = 0, params = 0;
+        uint64_t replicas = 0, gradbytes = 0;
         for (uint32_t q = 0; q < ng; ++q) {
             const sailor_replica_group gr = s.group[q];
             const uint32_t tp = h->tp_values[gr.tp_idx];
@@ -69,12 +69,10 @@ __device__ inline SimOut simulate_mixed_record(const TabView& v, const uint16_t*
             const uint64_t m = sm.mem + h->reserved[gr.type];
             if (m > h->capacity[gr.type]) status |= SAILOR_ST_OOM;
             peak = m > peak ? m : peak;
-            params = sm.params;
             const uint64_t gb = ceil_div64(sm.params, tp) * h->grad_bytes;
             gradbytes = gb > gradbytes ? gb : gradbytes;          // the ring moves the largest shard
         }
         if (replicas != D) status |= SAILOR_ST_INVALID;
-        (void)params;
         double sync = 0.0;
         for (uint32_t q = 0; q < ng; ++q) {
             const sailor_replica_group gr = s.group[q];
