@@ -55,6 +55,43 @@ __global__ void chain_kernel(unsigned char* blob) {
     }
 }
 
+// What a stage needs, per stage composition (embedding?, head?, number of blocks): parameters, gradient bytes per
+// worker, memory without and per in-flight microbatch, f + b, update time.  Formed with the same functions and
+// the same operation order as a stage-by-stage evaluation; one thread per (composition, type, tp, mbs, rc).
+__global__ void compose_kernel(unsigned char* blob) {
+    TabView v;
+    v.bind(blob, blob);
+    const TabHdr* h = v.h;
+    const size_t n_comp = (size_t)4 * h->chain_len;
+    const size_t total = n_comp * h->T * h->n_tp * h->n_mbs * 2;
+    for (size_t x = (size_t)blockIdx.x * blockDim.x + threadIdx.x; x < total; x += (size_t)gridDim.x * blockDim.x) {
+        size_t y = x;
+        const uint32_t rc = y % 2; y /= 2;
+        const uint32_t mi = y % h->n_mbs; y /= h->n_mbs;
+        const uint32_t tpi = y % h->n_tp; y /= h->n_tp;
+        const uint32_t g = y % h->T; y /= h->T;
+        const size_t comp = y;
+        const uint32_t nb = (uint32_t)(comp % h->chain_len), eh = (uint32_t)(comp / h->chain_len);
+        const bool e = eh & 2u, hd = eh & 1u;
+        const StageTimes st = stage_times(v, g, tpi, mi, nb, e, hd);
+        const double b = rc ? add_rn(st.b, st.f) : st.b;
+        reinterpret_cast<double*>(blob + h->off_cmp_fb)[x] = add_rn(st.f, b);
+        if (mi == 0 && rc == 0) reinterpret_cast<double*>(blob + h->off_cmp_upd)[(comp * h->T + g) * h->n_tp + tpi] = st.u;
+        if (g == 0) {
+            const StageMem one = stage_memory(v, tpi, mi, rc, nb, e, hd, 1);     // model + 1 * kept + work
+            const StageMem zero = stage_memory(v, tpi, mi, rc, nb, e, hd, 0);    // model + work
+            uint64_t* mm = reinterpret_cast<uint64_t*>(blob + h->off_cmp_mem) + (((comp * h->n_tp + tpi) * h->n_mbs + mi) * 2 + rc) * 2;
+            mm[0] = zero.mem;
+            mm[1] = one.mem - zero.mem;
+            if (mi == 0 && rc == 0) {
+                reinterpret_cast<double*>(blob + h->off_cmp_grad)[comp * h->n_tp + tpi] =
+                    (double)(ceil_div64(one.params, h->tp_values[tpi]) * h->grad_bytes);
+                if (tpi == 0) reinterpret_cast<uint64_t*>(blob + h->off_cmp_params)[comp] = one.params;
+            }
+        }
+    }
+}
+
 // One thread per explicit plan record (Sec. 4.3).  A block stages a pool of records in shared
 // memory with coalesced 8-byte loads, orders it by stage count (the work of a record grows with
 // its stages; any order gives the same results), and its warps take groups of 32 similar records
@@ -710,13 +747,22 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     h.static_bytes = align16((uint32_t)blob.size());
     blob.resize(h.static_bytes);
     const size_t c4 = (size_t)2 * T * n_tp * n_mbs * h.chain_len, c3 = (size_t)2 * T * n_tp * h.chain_len;
-    if (h.static_bytes + (2 * c4 + c3) * sizeof(double) > (1ull << 30) || h.static_bytes > 96 * 1024) {
+    const size_t n_comp = (size_t)4 * h.chain_len;
+    const size_t cmp_fb = n_comp * T * n_tp * n_mbs * 2, cmp_upd = n_comp * T * n_tp, cmp_mem = n_comp * n_tp * n_mbs * 2 * 2,
+                 cmp_grad = n_comp * n_tp;
+    if (h.static_bytes + (2 * c4 + c3 + cmp_fb + cmp_upd + cmp_mem + cmp_grad + n_comp) * sizeof(double) + 256 > (1ull << 30) ||
+        h.static_bytes > 96 * 1024) {
         delete ctx;
         return SAILOR_E_RANGE;
     }
     h.off_chain_f = put<double>(blob, nullptr, c4);
     h.off_chain_b = put<double>(blob, nullptr, c4);
     h.off_chain_u = put<double>(blob, nullptr, c3);
+    h.off_cmp_params = put<uint64_t>(blob, nullptr, n_comp);
+    h.off_cmp_grad = put<double>(blob, nullptr, cmp_grad);
+    h.off_cmp_mem = put<uint64_t>(blob, nullptr, cmp_mem);
+    h.off_cmp_fb = put<double>(blob, nullptr, cmp_fb);
+    h.off_cmp_upd = put<double>(blob, nullptr, cmp_upd);
     h.total_bytes = align16((uint32_t)blob.size());
     blob.resize(h.total_bytes);
     memcpy(blob.data(), &h, sizeof(h));
@@ -751,6 +797,10 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     {
         const uint32_t n_threads = 4 * T * n_tp * n_mbs + 2 * T * n_tp;
         chain_kernel<<<(n_threads + 127) / 128, 128, 0, ctx->stream>>>(ctx->d_blob);
+        CUF(cudaGetLastError());
+        const size_t n_cmp = cmp_fb;
+        const uint32_t grid = (uint32_t)((n_cmp + 127) / 128 < 65536 ? (n_cmp + 127) / 128 : 65536);
+        compose_kernel<<<grid, 128, 0, ctx->stream>>>(ctx->d_blob);
         CUF(cudaGetLastError());
     }
     CUF(cudaStreamSynchronize(ctx->stream));           // `blob` is pageable host memory

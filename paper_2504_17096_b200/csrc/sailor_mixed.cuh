@@ -11,18 +11,6 @@
 
 namespace sailor {
 
-// Ring all-reduce of `gradbytes` among D replicas over the intra- or inter-node link of digit d.
-__device__ __forceinline__ double allreduce_bytes_time(const TabView& v, uint32_t d, bool intra, double gradbytes, uint32_t D,
-                                                       double steps, double coef) {
-    const double alpha = intra ? v.intra_a[d] : v.inter_a[d];
-    const double* poly = intra ? v.intra_p : v.inter_p;
-    const double volume = mul_rn(coef, gradbytes);
-    double t;
-    if (poly) t = volume / poly_bw(poly + 4 * d, gradbytes / (double)D);
-    else t = mul_rn(volume, intra ? v.intra_i[d] : v.inter_i[d]);
-    return add_rn(t, mul_rn(steps, alpha));
-}
-
 // `cnt` points to this thread's per-digit GPU counters (digit d at cnt[d * cnt_stride]).
 __device__ inline SimOut simulate_mixed_record(const TabView& v, const uint16_t* __restrict__ avail,
                                                const sailor_mixed_plan& r, uint32_t* cnt, uint32_t cnt_stride) {

@@ -42,6 +42,14 @@ struct alignas(16) TabHdr {
     uint32_t off_chain_f, off_chain_b;            // f64 [start][type][tp][mbs][chain_len]
     uint32_t off_chain_u;                         // f64 [start][type][tp][chain_len]
     uint32_t total_bytes;
+    // per stage composition c = (embedding * 2 + head) * chain_len + blocks: what a stage of that make-up needs,
+    // formed once per context so that a simulated stage is a handful of loads
+    uint32_t off_cmp_params;                      // u64 [c]                        parameters
+    uint32_t off_cmp_grad;                        // f64 [c][tp]                    gradient bytes of one worker, as a double
+    uint32_t off_cmp_mem;                         // u64 [c][tp][mbs][rc][2]        model + working bytes, bytes kept per in-flight microbatch
+    uint32_t off_cmp_fb;                          // f64 [c][type][tp][mbs][rc]     f + b (+ f with recomputation)
+    uint32_t off_cmp_upd;                         // f64 [c][type][tp]              update time
+    uint32_t _pad[3];
 };
 static_assert(sizeof(TabHdr) % 16 == 0, "header must keep the arrays 16-byte aligned");
 
@@ -54,6 +62,8 @@ struct TabView {
     const double *price_s, *intra_a, *intra_i, *inter_a, *inter_i, *zone_a, *zone_i, *egress;
     const double *intra_p, *inter_p, *zone_p;      // nullptr when the link class has no polynomial
     const double *chain_f, *chain_b, *chain_u;
+    const uint64_t *cmp_params, *cmp_mem;
+    const double *cmp_grad, *cmp_fb, *cmp_upd;
 
     __host__ __device__ void bind(const unsigned char* stat, const unsigned char* glob) {
         h = reinterpret_cast<const TabHdr*>(stat);
@@ -78,6 +88,11 @@ struct TabView {
         chain_f = reinterpret_cast<const double*>(glob + h->off_chain_f);
         chain_b = reinterpret_cast<const double*>(glob + h->off_chain_b);
         chain_u = reinterpret_cast<const double*>(glob + h->off_chain_u);
+        cmp_params = reinterpret_cast<const uint64_t*>(glob + h->off_cmp_params);
+        cmp_grad = reinterpret_cast<const double*>(glob + h->off_cmp_grad);
+        cmp_mem = reinterpret_cast<const uint64_t*>(glob + h->off_cmp_mem);
+        cmp_fb = reinterpret_cast<const double*>(glob + h->off_cmp_fb);
+        cmp_upd = reinterpret_cast<const double*>(glob + h->off_cmp_upd);
     }
 };
 
@@ -196,6 +211,18 @@ __device__ __forceinline__ double allreduce_time(const TabView& v, uint32_t g, u
     return add_rn(t, mul_rn(steps, alpha));
 }
 
+// The same ring with the gradient bytes of one worker given (as a double) and the link class decided by the caller.
+__device__ __forceinline__ double allreduce_bytes_time(const TabView& v, uint32_t d, bool intra, double gradbytes, uint32_t D,
+                                                       double steps, double coef) {
+    const double alpha = intra ? v.intra_a[d] : v.inter_a[d];
+    const double* poly = intra ? v.intra_p : v.inter_p;
+    const double volume = mul_rn(coef, gradbytes);
+    double t;
+    if (poly) t = volume / poly_bw(poly + 4 * d, gradbytes / (double)D);
+    else t = mul_rn(volume, intra ? v.intra_i[d] : v.inter_i[d]);
+    return add_rn(t, mul_rn(steps, alpha));
+}
+
 __device__ __forceinline__ double sync_time(const TabView& v, uint32_t g, uint32_t z, uint32_t tp, uint32_t D,
                                             uint64_t params) {
     if (D <= 1) return 0.0;
@@ -241,11 +268,18 @@ __device__ __forceinline__ SimOut simulate_runs(const TabView& v, const uint16_t
     uint32_t status = 0;
     const uint64_t mbs = h->mbs_values[mi];
     const uint64_t dm = (uint64_t)D * mbs;
-    if (h->gbs % dm != 0) status |= SAILOR_ST_INVALID;
-    const uint64_t n_b = h->gbs / dm;
+    uint64_t n_b;
+    if (((h->gbs | dm) >> 32) == 0) {                      // the usual case: a 32-bit division
+        const uint32_t q32 = (uint32_t)h->gbs / (uint32_t)dm;
+        n_b = q32;
+        if (q32 * (uint32_t)dm != (uint32_t)h->gbs) status |= SAILOR_ST_INVALID;
+    } else {
+        n_b = h->gbs / dm;
+        if (n_b * dm != h->gbs) status |= SAILOR_ST_INVALID;
+    }
 
-    // resources: GPUs taken of every (zone, type), saturating at 2^32 - 1 (availability is 16 bits)
-    for (uint32_t d = 0; d < h->R; ++d) cnt[d * cnt_stride] = 0;
+    // resources: GPUs taken of every (zone, type) the plan uses, saturating at 2^32 - 1 (availability is 16 bits)
+    for (uint32_t q = 0; q < n_runs; ++q) cnt[(runs[q].zone * h->T + runs[q].type) * cnt_stride] = 0;
     for (uint32_t q = 0; q < n_runs; ++q) {
         const sailor_run a = runs[q];
         const uint32_t tp = h->tp_values[a.tp_idx];
@@ -293,15 +327,15 @@ __device__ __forceinline__ SimOut simulate_runs(const TabView& v, const uint16_t
         const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
         if (refresh || nb != cur_nb || e != cur_e || hd != cur_hd) {
             cur_nb = nb; cur_e = e; cur_hd = hd;
-            const StageTimes st = stage_times(v, g, tpi, mi, nb, e, hd);
-            const double b = rc ? add_rn(st.b, st.f) : st.b;
-            fb = add_rn(st.f, b);
-            upd = st.u;
-            const StageMem one = stage_memory(v, tpi, mi, rc, nb, e, hd, 1);     // model + 1 * kept + work
-            const StageMem zero = stage_memory(v, tpi, mi, rc, nb, e, hd, 0);    // model + work
-            m_keep = one.mem - zero.mem;
-            m_fixed = zero.mem + resv;
-            sync = D > 1 ? allreduce_time(v, g, z * h->T + g, tp, D, one.params, steps, coef) : 0.0;
+            // everything a stage of this make-up needs was formed once per context (compose_kernel)
+            const size_t comp = (size_t)((e ? 2u : 0u) + (hd ? 1u : 0u)) * h->chain_len + nb;
+            const size_t ct = comp * h->n_tp + tpi;
+            fb = v.cmp_fb[(((comp * h->T + g) * h->n_tp + tpi) * h->n_mbs + mi) * 2 + rc];
+            upd = v.cmp_upd[(comp * h->T + g) * h->n_tp + tpi];
+            const uint64_t* mm = v.cmp_mem + ((ct * h->n_mbs + mi) * 2 + rc) * 2;
+            m_fixed = mm[0] + resv;
+            m_keep = mm[1];
+            sync = D > 1 ? allreduce_bytes_time(v, z * h->T + g, (uint64_t)D * tp <= h->gpn[g], v.cmp_grad[ct], D, steps, coef) : 0.0;
             t_self = add_rn(fb, c2_self);
         }
         const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
