@@ -349,6 +349,14 @@ def sailor_plan_noalloc(ctx, space: Space, obj: Objective, k: int):
     return list(res[: n.value]), st
 
 
+def all_zone_orders(n_zones: int, max_len: Optional[int] = None):
+    """Every ordered selection of 1 .. max_len distinct zones (the region combinations a planner would loop over):
+    n_zones = 3 gives 15 orders, 4 gives 64, 5 gives 325."""
+    import itertools
+    max_len = n_zones if max_len is None else min(max_len, n_zones)
+    return [list(p) for n in range(1, max_len + 1) for p in itertools.permutations(range(n_zones), n)]
+
+
 def sailor_plan_dp(ctx, space: Space, zone_orders, k: int, workspace_bytes: int = 0, *, budget: float = 0.0,
                    min_rate: float = 0.0, obj: Optional[Objective] = None):
     """Per-stage GPU types by dynamic programming for every configuration of the space and every zone

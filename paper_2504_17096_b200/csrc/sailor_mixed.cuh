@@ -44,7 +44,10 @@ __device__ inline SimOut simulate_mixed_record(const TabView& v, const uint16_t*
         const uint32_t nb = base + (i < extra ? 1u : 0u), ng = s.n_groups;
         const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
         const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
-        uint64_t replicas = 0, gradbytes = 0;
+        // what a stage of this make-up needs was formed once per context (per-composition tables)
+        const size_t comp = (size_t)((e ? 2u : 0u) + (hd ? 1u : 0u)) * h->chain_len + nb;
+        uint64_t replicas = 0;
+        double gradbytes = 0.0;
         for (uint32_t q = 0; q < ng; ++q) {
             const sailor_replica_group gr = s.group[q];
             const uint32_t tp = h->tp_values[gr.tp_idx];
@@ -53,23 +56,22 @@ __device__ inline SimOut simulate_mixed_record(const TabView& v, const uint16_t*
             uint32_t* c = cnt + (s.zone * T + gr.type) * cnt_stride;
             const uint64_t sum = (uint64_t)*c + (uint64_t)gr.count * tp;
             *c = sum > 0xffffffffull ? 0xffffffffu : (uint32_t)sum;
-            const StageMem sm = stage_memory(v, gr.tp_idx, mi, rc, nb, e, hd, inflight);
-            const uint64_t m = sm.mem + h->reserved[gr.type];
+            const size_t ct = comp * h->n_tp + gr.tp_idx;
+            const uint64_t* mm = v.cmp_mem + ((ct * h->n_mbs + mi) * 2 + rc) * 2;
+            const uint64_t m = mm[0] + inflight * mm[1] + h->reserved[gr.type];
             if (m > h->capacity[gr.type]) status |= SAILOR_ST_OOM;
             peak = m > peak ? m : peak;
-            const uint64_t gb = ceil_div64(sm.params, tp) * h->grad_bytes;
-            gradbytes = gb > gradbytes ? gb : gradbytes;          // the ring moves the largest shard
+            gradbytes = dmax(gradbytes, v.cmp_grad[ct]);          // the ring moves the largest shard (smallest tp)
         }
         if (replicas != D) status |= SAILOR_ST_INVALID;
         double sync = 0.0;
         for (uint32_t q = 0; q < ng; ++q) {
             const sailor_replica_group gr = s.group[q];
             const uint32_t d = s.zone * T + gr.type, tp = h->tp_values[gr.tp_idx];
-            const StageTimes st = stage_times(v, gr.type, gr.tp_idx, mi, nb, e, hd);
-            max_u = dmax(max_u, st.u);
+            max_u = dmax(max_u, v.cmp_upd[(comp * T + gr.type) * h->n_tp + gr.tp_idx]);
             if (D > 1) {
                 const bool intra = ng == 1 && (uint64_t)D * tp <= h->gpn[gr.type];
-                sync = dmax(sync, allreduce_bytes_time(v, d, intra, (double)gradbytes, D, steps, coef));
+                sync = dmax(sync, allreduce_bytes_time(v, d, intra, gradbytes, D, steps, coef));
             }
             rate = add_rn(rate, mul_rn((double)((uint32_t)gr.count * tp), v.price_s[d]));
         }
@@ -103,9 +105,8 @@ __device__ inline SimOut simulate_mixed_record(const TabView& v, const uint16_t*
             const sailor_replica_group gr = s.group[q_cur];
             const uint32_t nb = base + (i < extra ? 1u : 0u);
             const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
-            const StageTimes st = stage_times(v, gr.type, gr.tp_idx, mi, nb, e, hd);
-            const double b = rc ? add_rn(st.b, st.f) : st.b;
-            const double fb = add_rn(st.f, b);
+            const size_t comp = (size_t)((e ? 2u : 0u) + (hd ? 1u : 0u)) * h->chain_len + nb;
+            const double fb = v.cmp_fb[(((comp * T + gr.type) * h->n_tp + gr.tp_idx) * h->n_mbs + mi) * 2 + rc];
             double c = 0.0;
             if (i + 1 < P) {
                 const sailor_mixed_stage& s2 = r.stage[i + 1];

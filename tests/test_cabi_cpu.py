@@ -55,3 +55,10 @@ def test_product_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower(), f
+
+
+def test_zone_order_helper():
+    from paper_2504_17096_b200 import binding as B
+    assert len(B.all_zone_orders(3)) == 15 and len(B.all_zone_orders(4)) == 64 and len(B.all_zone_orders(5)) == 325
+    assert B.all_zone_orders(3, 1) == [[0], [1], [2]]
+    assert all(len(set(o)) == len(o) for o in B.all_zone_orders(4))
