@@ -280,6 +280,31 @@ def aux_measurements(B, torch, dev) -> dict:
     return out
 
 
+def run_dp_only(args) -> None:
+    """Only the dynamic-programming search of the workload (one zone order), a few times: a small command for
+    profiling its kernels.  Prints one JSON line of its own (not the benchmark line)."""
+    import torch
+    from paper_2504_17096_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    w = workload_by_name(args.workload, args.only_p)
+    ctx = B.sailor_create(w, 0, torch.cuda.current_stream().cuda_stream)
+    try:
+        B.sailor_set_availability(ctx, w.avail)
+        sp = B.make_space(w)
+        orders = [list(range(w.n_zones))]
+        for _ in range(max(1, args.steps)):
+            t0 = time.perf_counter()
+            res, st = B.sailor_plan_dp(ctx, sp, orders, K_TOP, workspace_bytes=int(args.dp_workspace_gib * (1 << 30)))
+            dt = time.perf_counter() - t0
+        print(json.dumps({"dp_only": w.name, "search_s": dt, "kernel_ms": st.kernel_ms, "problems": int(st.n_problems),
+                          "solved": int(st.n_solved), "table_entries": int(st.n_states), "batches": int(st.n_batches),
+                          "launches": int(st.n_launches), "workspace_bytes": int(st.workspace_used),
+                          "best_t_iter": res[0].t_iter if res else None}), flush=True)
+    finally:
+        B.sailor_destroy(ctx)
+
+
 def run_ours(args) -> None:
     import torch
     from paper_2504_17096_b200 import binding as B
@@ -451,12 +476,16 @@ def main() -> None:
     ap.add_argument("--cpu-sample", type=int, default=20_000_000, help="candidates the CPU baseline evaluates")
     ap.add_argument("--ref-sample", type=int, default=4_000_000, help="candidates per reference step")
     ap.add_argument("--only-p", type=int, nargs="*", default=None, help="keep only these pipeline depths")
+    ap.add_argument("--dp-only", action="store_true", help="run only the dynamic-programming search (for profiling)")
+    ap.add_argument("--dp-workspace-gib", type=float, default=8.0, help="table workspace of --dp-only")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-aux", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     if args.impl == "reference":
         run_reference(args)
+    elif args.dp_only:
+        run_dp_only(args)
     else:
         run_ours(args)
 
