@@ -2,7 +2,11 @@
 
 Candidates are independent, so a space is cut into contiguous flat-index ranges, each rank runs
 `sailor_plan_range` on its own GPU, and the per-rank top-k lists are merged by (score, flat).
-The only exchange is k small records per rank; there is no data-path collective."""
+The only exchange is k small records per rank; there is no data-path collective.
+
+The dynamic-programming search shards by zone order: its problems (configuration x zone order) are
+independent, a rank solves every configuration for its slice of the order list with `sailor_plan_dp`,
+and the per-rank lists are merged by (value, problem index) with the order index made global."""
 from __future__ import annotations
 
 from typing import List, Sequence, Tuple
@@ -44,3 +48,17 @@ def gather_and_merge(local: Sequence[Tuple[float, int]], local_counts: dict, k: 
     dist.all_gather_object(lists, list(local), group=group)
     dist.all_gather_object(counts, dict(local_counts), group=group)
     return merge_topk(lists, k), sum_counts(counts)
+
+
+def split_zone_orders(orders: Sequence[Sequence[int]], world: int, rank: int):
+    """The slice of the zone-order list that rank `rank` solves: (index of its first order, its orders)."""
+    lo, hi = split_range(len(orders), world, rank)
+    return lo, [list(o) for o in orders[lo:hi]]
+
+
+def merge_dp(lists: Sequence[Sequence[Tuple[float, int, int]]], n_orders_total: int, k: int) -> List[Tuple[float, int, int]]:
+    """Merge per-rank lists of (value, configuration, global order index): ascending by value, ties to the
+    lowest problem index = configuration * n_orders_total + order, as one call over all orders would rank them."""
+    allp = [tuple(p) for l in lists for p in l]
+    allp.sort(key=lambda p: (p[0], p[1] * n_orders_total + p[2]))
+    return allp[:k]

@@ -78,3 +78,65 @@ def test_two_ranks_merge_to_the_full_search():
         assert merged == want
         assert total["n_total"] == counts["n_total"] and total["n_feasible"] == counts["n_feasible"]
         assert total["min_feasible_cost"] == counts["min_cost"]
+
+
+def _dp_worker(rank, world, port, q):
+    import itertools
+    import torch.distributed as dist
+    from oracle.binding import Oracle
+    from paper_2504_17096_b200 import binding as B
+    from paper_2504_17096_b200 import workloads as W
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        w = W.tiny(seed=7, n_types=2, n_zones=3, L=5, p_values=[2, 4, 5], d_values=(1, 2, 4))
+        orders = B.all_zone_orders(w.n_zones)
+        lo, mine = sharding.split_zone_orders(orders, world, rank)
+        o = Oracle(w)
+        local = []
+        cfgs = list(itertools.product(w.p_values, w.mbs_idx, w.tp_idx, w.rc_values, w.d_values))
+        for c, (P, mi, ti, rc, D) in enumerate(cfgs):          # the oracle stands in for this rank's GPU
+            for j, zl in enumerate(mine):
+                r = o.solve_dp(P, mi, ti, rc, D, zl)
+                if r is not None:
+                    local.append((r["value"], c, lo + j))
+        local.sort(key=lambda p: (p[0], p[1] * len(orders) + p[2]))
+        lists = [None] * world
+        dist.all_gather_object(lists, local[:8])
+        q.put((rank, sharding.merge_dp(lists, len(orders), 8)))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_split_the_zone_orders_of_the_dp_search():
+    import itertools
+    from oracle.binding import Oracle
+    from paper_2504_17096_b200 import binding as B
+    from paper_2504_17096_b200 import workloads as W
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_dp_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    got = [q.get(timeout=120) for _ in range(world)]
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    w = W.tiny(seed=7, n_types=2, n_zones=3, L=5, p_values=[2, 4, 5], d_values=(1, 2, 4))
+    orders = B.all_zone_orders(w.n_zones)
+    o = Oracle(w)
+    full = []
+    for c, (P, mi, ti, rc, D) in enumerate(itertools.product(w.p_values, w.mbs_idx, w.tp_idx, w.rc_values, w.d_values)):
+        for j, zl in enumerate(orders):
+            r = o.solve_dp(P, mi, ti, rc, D, zl)
+            if r is not None:
+                full.append((r["value"], c, j))
+    full.sort(key=lambda p: (p[0], p[1] * len(orders) + p[2]))
+    assert len(full) > 8
+    for rank, merged in got:
+        assert merged == full[:8]
+    lo0, a = sharding.split_zone_orders(orders, 2, 0)
+    lo1, b = sharding.split_zone_orders(orders, 2, 1)
+    assert lo0 == 0 and lo1 == len(a) and a + b == orders
