@@ -92,6 +92,12 @@ def test_hand_worked_recursion():
         assert list(res[0].type[: p["P"]]) == e["types"] and list(res[0].zone[: p["P"]]) == e["zones"]
         assert res[0].value == pytest.approx(e["value"], rel=1e-12)
         assert res[0].t_iter == pytest.approx(e["value"], rel=1e-12)
+        if "cost" in e:
+            assert res[0].cost == pytest.approx(e["cost"], rel=1e-12)
+        for zl in e.get("no_plan_zone_lists", []):
+            with Ctx(w) as cx:
+                none, st = B.sailor_plan_dp(cx.ctx, cx.space, [zl], 4)
+            assert none == [] and st.n_solved == 0
 
 
 def _tiny():

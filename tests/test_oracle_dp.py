@@ -73,6 +73,10 @@ def test_hand_worked_recursion(case):
     assert o.simulate(r["plan"]).t_iter == pytest.approx(e["value"], rel=1e-12)
     opt = brute_force(w, o, p["P"], p["mbs_idx"], p["tp_idx"], p["rc"], p["D"], p["zone_list"])
     assert opt[1] == e["optimum_types"] and opt[0] == pytest.approx(e["optimum"], rel=1e-12)
+    if "cost" in e:
+        assert o.simulate(r["plan"]).cost == pytest.approx(e["cost"], rel=1e-12)
+    for zl in e.get("no_plan_zone_lists", []):
+        assert o.solve_dp(p["P"], p["mbs_idx"], p["tp_idx"], p["rc"], p["D"], zl) is None
 
 
 def _problems(w):
