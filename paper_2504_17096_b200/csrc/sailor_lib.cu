@@ -236,7 +236,12 @@ struct SpaceCache {
     uint32_t* d_wave_start = nullptr;             // [n_config + 1] chunk offsets of the current wave
     unsigned long long* d_cfg_best = nullptr;     // [n_config] best feasible score per configuration
     GroupState* d_groups = nullptr;               // [n_config / n_d]
+    // the per-configuration tables, built once per space (spaces whose records fit CFG_CACHE_MAX_BYTES)
+    uint4* d_cfg_cache = nullptr;
+    uint32_t cache_head16 = 0, cache_arr16 = 0;
 };
+
+constexpr size_t CFG_CACHE_MAX_BYTES = 512ull << 20;
 
 constexpr uint64_t WAVE_CONFIG_MAX = 1u << 16;
 
@@ -416,6 +421,8 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
         cudaFree(sc.d_wave_start);
         cudaFree(sc.d_cfg_best);
         cudaFree(sc.d_groups);
+        cudaFree(sc.d_cfg_cache);
+        sc.d_cfg_cache = nullptr;
         sc.d_live_start = nullptr;
         sc.d_cfg_closed = nullptr;
         sc.d_wave_start = nullptr;
@@ -449,6 +456,38 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
         sc.live_chunks = (uint32_t)run;
         CU(ctx, cudaMemcpyAsync(sc.d_live_start, live.data(), (n_config + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
         CU(ctx, cudaStreamSynchronize(ctx->stream));
+    }
+    {   // the tables of every configuration, once: later searches copy them instead of building them
+        sc.cache_head16 = cache_head16();
+        sc.cache_arr16 = cache_arr16(ctx->hdr.T, ctx->hdr.Z);
+        const size_t rec_bytes = 16 * ((size_t)sc.cache_head16 + sc.cache_arr16);
+        if (n_config * rec_bytes <= CFG_CACHE_MAX_BYTES && cudaMalloc(&sc.d_cfg_cache, n_config * rec_bytes) == cudaSuccess) {
+            static bool optin_done[64] = {};
+            const bool tracked = ctx->device >= 0 && ctx->device < 64;
+            if (!tracked || !optin_done[ctx->device]) {
+                CU(ctx, cudaFuncSetAttribute(cfg_cache_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PLAN_SMEM_CEILING));
+                if (tracked) optin_done[ctx->device] = true;
+            }
+            PlanParams pp;
+            memset(&pp, 0, sizeof(pp));
+            pp.blob = ctx->d_blob;
+            pp.avail = ctx->d_avail;
+            pp.ctrl = ctx->d_ctrl;
+            pp.sp = d;
+            pp.n_config = (uint32_t)n_config;
+            pp.p_max = p_max;
+            pp.live_mode = 1;                  // the lists of usable digits are part of a record
+            pp.min_tp_only = 1;                // and so are the masks of the smaller tensor-parallel degrees
+            pp.cache_head16 = sc.cache_head16;
+            pp.cache_arr16 = sc.cache_arr16;
+            const uint32_t grid = (uint32_t)(n_config < (uint64_t)ctx->sm_count * 2 ? n_config : (uint64_t)ctx->sm_count * 2);
+            cfg_cache_kernel<<<grid, PLAN_THREADS, smem, ctx->stream>>>(pp, sc.d_cfg_cache);
+            CU(ctx, cudaGetLastError());
+            CU(ctx, cudaStreamSynchronize(ctx->stream));
+        } else {
+            sc.d_cfg_cache = nullptr;          // too large (or no memory): searches build the tables themselves
+            (void)cudaGetLastError();
+        }
     }
     sc.key = *s;
     sc.desc = d;
@@ -529,6 +568,9 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
     pp.k = k;
     pp.eval_all = (flags & SAILOR_FLAG_EVAL_ALL) ? 1u : 0u;
     pp.min_tp_only = (flags & SAILOR_FLAG_MIN_TP_ONLY) ? 1u : 0u;
+    pp.cfg_cache = sc.d_cfg_cache;
+    pp.cache_head16 = sc.cache_head16;
+    pp.cache_arr16 = sc.cache_arr16;
     pp.budget_from_ctrl = budget_from_ctrl ? 1u : 0u;
     pp.p_max = sc.p_max;
     pp.budget = budget;
@@ -832,6 +874,7 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->space.d_wave_start);
     cudaFree(ctx->space.d_cfg_best);
     cudaFree(ctx->space.d_groups);
+    cudaFree(ctx->space.d_cfg_cache);
     cudaFree(ctx->d_stage);
     cudaFree(ctx->d_dp);
     if (ctx->ev0) cudaEventDestroy(ctx->ev0);

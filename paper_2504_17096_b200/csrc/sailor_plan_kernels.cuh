@@ -65,6 +65,8 @@ struct PlanParams {
     uint32_t carry_lists;              // a block starts from the list it left in `partial` (waves of one search)
     const uint32_t* chunk_hi_dev;      // non-null: chunks [0, *chunk_hi_dev) instead of [chunk_lo, chunk_hi)
     unsigned long long* cfg_best;      // non-null: [n_config] best feasible score per configuration (ordered bits)
+    const uint4* cfg_cache;            // non-null: the per-configuration tables, built once per space (cfg_cache_kernel)
+    uint32_t cache_head16, cache_arr16;    // 16-byte words of a cached record: CfgShared head, then the arrays
     double budget;                     // <= 0: none
     double min_rate;                   // <= 0: none
 };
@@ -174,7 +176,7 @@ struct alignas(16) SegRec {                  // one per (segment, digit); 64 byt
     double rate;                 // D * tp * price per second of one stage
 };
 
-struct CfgShared {
+struct alignas(16) CfgShared {
     // scalars (written by thread 0 / the build, read by all)
     Config cfg;
     uint32_t valid;              // gbs % (D*mbs) == 0 and heads % tp == 0
@@ -186,7 +188,6 @@ struct CfgShared {
     uint32_t seg_a[SAILOR_SEG_MAX + 1];   // first stage of each segment; seg_a[nseg] = P
     uint32_t need[SAILOR_SEG_MAX];        // GPUs a segment takes of its digit: D * tp * stages
     uint32_t n_run[SAILOR_SEG_MAX][N_RUNS];   // stages in each run (without a non-final segment's last stage)
-    uint32_t magic;              // floor(2^32 / R) + 1: x / R == umulhi(x, magic) for x < 2^26
     double ar_steps, ar_coef;    // 2(D-1) and 2(D-1)/D of the ring all-reduce
     uint64_t n_b;
     uint64_t n_items;            // R^(nseg-1)
@@ -195,7 +196,10 @@ struct CfgShared {
     uint32_t n_lower;            // smaller tensor-parallel degrees of the space that the model accepts (min_tp_only)
     uint32_t lower_tpi[SAILOR_TP_MAX];    // their tp indices
     uint64_t lower_fit[SAILOR_TP_MAX][SAILOR_SEG_MAX];   // digit d: every stage of the segment fits at that degree
-    uint64_t avail_last;         // digit d: need[last] <= avail[d]
+    // ---- everything above depends on the configuration and the context only, not on availability: it is what a
+    // ---- cached record holds (with the arrays rec .. fb_last); everything below belongs to the block or the snapshot
+    alignas(16) uint64_t avail_last;     // digit d: need[last] <= avail[d]
+    uint32_t magic;              // floor(2^32 / R) + 1: x / R == umulhi(x, magic) for x < 2^26
     uint32_t cur_config;
     uint32_t next_chunk, batch_len;
     unsigned long long oom_stage[SAILOR_P_MAX];   // per stage: bit 8 j + g set when the stage does not fit type g
@@ -222,6 +226,16 @@ __host__ __device__ inline size_t plan_smem_bytes(uint32_t static_bytes, uint32_
     n += sizeof(double) * ((R + PLAN_PAD) * R + (R + PLAN_PAD) * Z + (size_t)SAILOR_SEG_MAX * T + 2 * (size_t)p_max * T);
     n += sizeof(uint32_t) * 2 * R;
     return (n + 15) & ~(size_t)15;
+}
+
+// A cached configuration record: the head of CfgShared up to avail_last, then the arrays rec, c2x, commx, fb_last
+// (with their padding entries), both in 16-byte words.
+__host__ __device__ inline uint32_t cache_head16() { return (uint32_t)(offsetof(CfgShared, avail_last) / 16); }
+__host__ __device__ inline uint32_t cache_arr16(uint32_t T, uint32_t Z) {
+    const size_t R = (size_t)T * Z;
+    const size_t bytes = sizeof(SegRec) * (SAILOR_SEG_MAX * R + PLAN_PAD) +
+                         sizeof(double) * ((R + PLAN_PAD) * R + (R + PLAN_PAD) * Z + (size_t)SAILOR_SEG_MAX * T);
+    return (uint32_t)((bytes + 15) / 16);
 }
 
 __device__ __forceinline__ void carve(unsigned char* dyn, uint32_t static_bytes, uint32_t p_max, uint32_t T,
@@ -413,6 +427,28 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
             if (tid == 0) cs.live_items = live;
         }
         if (tid == 0) cs.packed = pp.live_mode;
+    }
+    __syncthreads();
+}
+
+// The tables of configuration `c` from the cache instead of building them: two straight copies, then the
+// availability mask of the last segment, which is the only part that follows the snapshot.  Called by the
+// whole block (after a barrier); ends synchronised.  `a.availv` holds the snapshot already.
+__device__ void load_config(const PlanParams& pp, CfgShared& cs, CfgArrays& a, uint32_t R, uint32_t c) {
+    const uint32_t tid = threadIdx.x;
+    const uint4* src = pp.cfg_cache + (size_t)c * (pp.cache_head16 + pp.cache_arr16);
+    for (uint32_t x = tid; x < pp.cache_head16; x += PLAN_THREADS) reinterpret_cast<uint4*>(&cs)[x] = src[x];
+    for (uint32_t x = tid; x < pp.cache_arr16; x += PLAN_THREADS) reinterpret_cast<uint4*>(a.rec)[x] = src[pp.cache_head16 + x];
+    __syncthreads();
+    if (tid < 32) {
+        const uint32_t need_last = cs.need[cs.cfg.nseg - 1];
+        const uint32_t a_lo = __ballot_sync(FULL, tid < R && need_last <= a.availv[tid < R ? tid : 0]);
+        const uint32_t a_hi = __ballot_sync(FULL, tid + 32 < R && need_last <= a.availv[tid + 32 < R ? tid + 32 : 0]);
+        if (tid == 0) {
+            cs.avail_last = ((uint64_t)a_hi << 32) | a_lo;
+            cs.packed = cs.valid ? pp.live_mode : 0u;
+            cs.cur_config = c;
+        }
     }
     __syncthreads();
 }
@@ -772,6 +808,10 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
         reinterpret_cast<double*>(a.rec + (size_t)SAILOR_SEG_MAX * R)[x] = 0.0;
     for (uint32_t x = tid; x < PLAN_PAD * R; x += PLAN_THREADS) a.c2x[(size_t)R * R + x] = 0.0;
     for (uint32_t x = tid; x < PLAN_PAD * Z; x += PLAN_THREADS) a.commx[(size_t)R * Z + x] = 0.0;
+    for (uint32_t d = tid; d < R; d += PLAN_THREADS) {      // what does not depend on the configuration
+        a.availv[d] = pp.avail[d];
+        a.tz[d] = (d % T) | ((d / T) << 8);
+    }
     WarpTopK top;
     top.init();
     if (pp.carry_lists && warp == 0) {     // a later wave of one search: go on from the list this block left behind
@@ -817,7 +857,8 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             if (cs.cur_config != c) {
                 if (pp.cfg_best && cs.cur_config != 0xffffffffu) flush_cfg_best(pp, cnt, cs.cur_config, lane);
                 __syncthreads();
-                build_config(pp, v, cs, a, c);
+                if (pp.cfg_cache) load_config(pp, cs, a, R, c);
+                else build_config(pp, v, cs, a, c);
             }
             const uint32_t q = (ch - pp.cfg_chunk_start[c]) * PLAN_THREADS + tid;    // < R^3 + 256 <= 2^18 + 256
             const bool active = q < (cs.packed ? cs.live_items : cs.n_items);
@@ -885,6 +926,40 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             pp.partial[(size_t)blockIdx.x * SAILOR_K_MAX + lane].flat = top.flat;
         }
         if (lane == 0) pp.partial_n[blockIdx.x] = n;
+    }
+}
+
+// The tables of every configuration, built once per (context, space) and kept in global memory: all of them but
+// the availability mask of the last segment depend on the context and the configuration only, so a search after
+// a new snapshot copies them instead of rebuilding them.  One block per configuration at a time.
+__global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) cfg_cache_kernel(const __grid_constant__ PlanParams pp, uint4* cache) {
+    extern __shared__ __align__(16) unsigned char dyn[];
+    __shared__ CfgShared cs;
+    const uint32_t tid = threadIdx.x;
+    const TabHdr* gh = reinterpret_cast<const TabHdr*>(pp.blob);
+    const uint32_t static_bytes = gh->static_bytes;
+    if (!bulk_load(dyn, pp.blob, static_bytes, &cs.mbar)) {
+        if (tid == 0) atomicExch(&pp.ctrl->error, 1u);
+        for (uint32_t x = tid; x < static_bytes / 16; x += PLAN_THREADS)
+            reinterpret_cast<uint4*>(dyn)[x] = reinterpret_cast<const uint4*>(pp.blob)[x];
+        __syncthreads();
+    }
+    TabView v;
+    v.bind(dyn, pp.blob);
+    const uint32_t T = v.h->T, Z = v.h->Z;
+    CfgArrays a;
+    carve(dyn, static_bytes, pp.p_max, T, Z, a);
+    // the whole cached region starts from zero, so that records do not depend on what the block did before
+    for (uint32_t x = tid; x < pp.cache_arr16; x += PLAN_THREADS) reinterpret_cast<uint4*>(a.rec)[x] = make_uint4(0, 0, 0, 0);
+    for (uint32_t x = tid; x < pp.cache_head16; x += PLAN_THREADS) reinterpret_cast<uint4*>(&cs)[x] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    for (uint32_t c = blockIdx.x; c < pp.n_config; c += gridDim.x) {
+        __syncthreads();
+        build_config(pp, v, cs, a, c);
+        __syncthreads();
+        uint4* dst = cache + (size_t)c * (pp.cache_head16 + pp.cache_arr16);
+        for (uint32_t x = tid; x < pp.cache_head16; x += PLAN_THREADS) dst[x] = reinterpret_cast<const uint4*>(&cs)[x];
+        for (uint32_t x = tid; x < pp.cache_arr16; x += PLAN_THREADS) dst[pp.cache_head16 + x] = reinterpret_cast<const uint4*>(a.rec)[x];
     }
 }
 
