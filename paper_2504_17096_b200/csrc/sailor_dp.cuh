@@ -133,9 +133,11 @@ dp_tables_kernel(const unsigned char* __restrict__ blob, SpaceDesc sp, uint32_t 
 // W[j][s], the rank of u in lexicographic order is sum_j (V[j+1][s_j] - V[j+1][s_j - u_j]), s_0 = P,
 // s_{j+1} = s_j - u_j.  The table holds V[j][s] for j = 0 .. m, s = 0 .. P, row after row.
 
-// counts of a slice index: u[t] for counted types, 0 for the others
-__device__ __forceinline__ void dp_counts(const DpProblem& pb, const uint32_t* __restrict__ vtabs, uint32_t zp, uint32_t T,
-                                          uint32_t ui, uint32_t (&u)[SAILOR_T_MAX]) {
+// counts of a slice index: u[t] for counted types, 0 for the others.  Returns false, possibly before all counts
+// are known, as soon as they add up to more than `limit`.
+__device__ __forceinline__ bool dp_counts(const DpProblem& pb, const uint32_t* __restrict__ vtabs, uint32_t zp, uint32_t T,
+                                          uint32_t ui, uint32_t (&u)[SAILOR_T_MAX], uint32_t limit) {
+    uint32_t total = 0;
     if (pb.vt_off[zp] == DP_DENSE) {
         uint32_t rem = ui;
 #pragma unroll
@@ -145,8 +147,10 @@ __device__ __forceinline__ void dp_counts(const DpProblem& pb, const uint32_t* _
                 const uint32_t q = (uint32_t)__umul64hi((uint64_t)rem, pb.magic[zp][t]);
                 u[t] = rem - q * (pb.cap[zp][t] + 1u);
                 rem = q;
+                total += u[t];
             }
         }
+        return total <= limit;
     } else {
         const uint32_t* vt = vtabs + pb.vt_off[zp];
         const uint32_t w = pb.P + 1;
@@ -165,11 +169,14 @@ __device__ __forceinline__ void dp_counts(const DpProblem& pb, const uint32_t* _
                     ++x;
                 }
                 u[t] = x;
+                total += x;
+                if (total > limit) return false;                 // the walks of the remaining types are not needed
                 r -= below;
                 s -= x;
                 ++j;
             }
         }
+        return true;
     }
 }
 
@@ -262,13 +269,9 @@ __global__ void __launch_bounds__(DP_THREADS, 4) dp_level_kernel(const __grid_co
     const uint32_t S = pb.S[zp];
     while (ui >= S) { ui -= S; ++g; }
     uint32_t u[SAILOR_T_MAX];
-    dp_counts(pb, lp.vtabs, zp, T, ui, u);
-    uint32_t placed = 0;
-#pragma unroll
-    for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) placed += u[t];
     // stage i is at most the (i+1)-th stage of its zone: entries that count more are never reached, and
     // since a move raises the count by one per stage, no entry that passes this test ever reads one that fails it
-    if (placed > i + 1) return;
+    if (!dp_counts(pb, lp.vtabs, zp, T, ui, u, i + 1)) return;
     DpVal* cur = lp.val[lp.dist & 1] + pb.val_off;
     const DpVal* nxt = lp.val[(lp.dist & 1) ^ 1] + pb.val_off;
     uint8_t* choice = lp.choice + pb.choice_off + (size_t)i * pb.n_lvl;
@@ -370,7 +373,7 @@ __global__ void __launch_bounds__(128) dp_finish_kernel(const __grid_constant__ 
         const uint8_t g2 = fp.choice[pb.choice_off + (size_t)i * pb.n_lvl + entry];
         const uint32_t ui = (entry - pb.zp_base[zp]) % pb.S[zp];
         uint32_t u[SAILOR_T_MAX];
-        dp_counts(pb, fp.vtabs, zp, T, ui, u);
+        dp_counts(pb, fp.vtabs, zp, T, ui, u, P);
         const DpMove mv = dp_move(pb, fp.vtabs, T, zp, ui, u, g2);
         g = g2; zp = mv.zp; entry = mv.entry;
     }
