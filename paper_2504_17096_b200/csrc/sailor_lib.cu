@@ -825,6 +825,7 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     CUF(cudaMalloc(&ctx->d_blob, h.total_bytes));
     CUF(cudaMalloc(&ctx->d_avail, R_MAX * sizeof(uint16_t)));
     CUF(cudaMallocHost(&ctx->h_avail, R_MAX * sizeof(uint16_t)));
+    memset(ctx->h_avail, 0, R_MAX * sizeof(uint16_t));       // availability starts at zero on both sides
     CUF(cudaMalloc(&ctx->d_ctrl, sizeof(Ctrl)));
     CUF(cudaMalloc(&ctx->d_results, sizeof(sailor_result) * SAILOR_K_MAX));
     CUF(cudaMallocHost(&ctx->h_out, sizeof(OutBlock)));

@@ -228,6 +228,17 @@ def test_dp_constraints_drop_plans_after_the_recursion():
             assert [r.value for r in res] == [x[0] for x in keep[:32]]
 
 
+def test_dp_before_any_availability_is_set():
+    """A fresh context has no GPUs available on either side: no problem has a plan."""
+    w = W.tiny(seed=3)
+    ctx = B.sailor_create(w, 0, 0)
+    try:
+        res, st = B.sailor_plan_dp(ctx, B.make_space(w), [[0, 1]], 4)
+        assert res == [] and st.n_solved == 0
+    finally:
+        B.sailor_destroy(ctx)
+
+
 def test_dp_argument_checks():
     w = W.tiny(seed=3)
     with Ctx(w) as cx:
