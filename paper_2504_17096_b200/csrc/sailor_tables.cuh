@@ -301,64 +301,68 @@ __device__ __forceinline__ SimOut simulate_runs(const TabView& v, const uint16_t
     double sum_t = 0.0, max_t = 0.0, max_sync = 0.0, max_u = 0.0, rate = 0.0, c_comm = 0.0;
     uint64_t peak = 0;
 
-    // current run
-    uint32_t q = 0, left = 0, g = 0, z = 0, tpi = 0, tp = 1;
-    double gpu_rate = 0.0, c2_self = 0.0;
-    uint64_t cap = 0, resv = 0;
-    // current layer composition
-    uint32_t cur_nb = 0xffffffffu;
-    bool cur_e = false, cur_hd = false;
-    double fb = 0.0, upd = 0.0, sync = 0.0, t_self = 0.0;
-    uint64_t m_fixed = 0, m_keep = 0;
-
-    for (uint32_t i = 0; i < P; ++i) {
-        bool refresh = false;
-        if (left == 0) {                                   // enter run q
-            const sailor_run a = runs[q];
-            g = a.type; z = a.zone; tpi = a.tp_idx; tp = h->tp_values[tpi]; left = a.n_stages;
-            const uint32_t d = z * h->T + g;
-            gpu_rate = mul_rn((double)(D * tp), v.price_s[d]);
-            cap = h->capacity[g];
-            resv = h->reserved[g];
-            c2_self = mul_rn(2.0, boundary_time(v, g, z, tp, g, z, tp, D, msg));
-            refresh = true;
-        }
-        const uint32_t nb = base + (i < extra ? 1u : 0u);
-        const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
-        if (refresh || nb != cur_nb || e != cur_e || hd != cur_hd) {
-            cur_nb = nb; cur_e = e; cur_hd = hd;
+    // The stages are walked piece by piece: a piece is a stretch of one run with one layer make-up, so all its
+    // stages have the same f + b, memory terms and synchronisation; only the stage that closes a run (it sends to
+    // the next run) and the final stage (it sends nothing) have a time of their own.  Within a piece the sums take
+    // one addition per stage, in stage order, exactly as a stage-by-stage walk would add them; memory is largest at
+    // the piece's first stage (the in-flight microbatches never grow with the stage index), so that one is checked.
+    uint32_t i = 0;
+    for (uint32_t q = 0; q < n_runs; ++q) {
+        const sailor_run a = runs[q];
+        const uint32_t g = a.type, z = a.zone, tpi = a.tp_idx, tp = h->tp_values[tpi];
+        const uint32_t d = z * h->T + g, run_end = i + a.n_stages;
+        const double gpu_rate = mul_rn((double)(D * tp), v.price_s[d]);
+        const uint64_t cap = h->capacity[g], resv = h->reserved[g];
+        const double c2_self = mul_rn(2.0, boundary_time(v, g, z, tp, g, z, tp, D, msg));
+        const bool intra_dp = (uint64_t)D * tp <= h->gpn[g];
+        while (i < run_end) {
+            const uint32_t nb = base + (i < extra ? 1u : 0u);
+            const bool e = (i == 0) && h->has_embed, hd = (i == P - 1) && h->has_head;
+            // the piece ends with the run, after the embedding stage, where the extra blocks run out, before the head stage
+            uint32_t piece_end = run_end;
+            if (e) piece_end = 1;
+            else {
+                if (i < extra && extra < piece_end) piece_end = extra;
+                if (h->has_head && i < P - 1 && P - 1 < piece_end) piece_end = P - 1;
+            }
             // everything a stage of this make-up needs was formed once per context (compose_kernel)
             const size_t comp = (size_t)((e ? 2u : 0u) + (hd ? 1u : 0u)) * h->chain_len + nb;
             const size_t ct = comp * h->n_tp + tpi;
-            fb = v.cmp_fb[(((comp * h->T + g) * h->n_tp + tpi) * h->n_mbs + mi) * 2 + rc];
-            upd = v.cmp_upd[(comp * h->T + g) * h->n_tp + tpi];
+            const double fb = v.cmp_fb[(((comp * h->T + g) * h->n_tp + tpi) * h->n_mbs + mi) * 2 + rc];
+            const double upd = v.cmp_upd[(comp * h->T + g) * h->n_tp + tpi];
             const uint64_t* mm = v.cmp_mem + ((ct * h->n_mbs + mi) * 2 + rc) * 2;
-            m_fixed = mm[0] + resv;
-            m_keep = mm[1];
-            sync = D > 1 ? allreduce_bytes_time(v, z * h->T + g, (uint64_t)D * tp <= h->gpn[g], v.cmp_grad[ct], D, steps, coef) : 0.0;
-            t_self = add_rn(fb, c2_self);
-        }
-        const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
-        const uint64_t m = m_fixed + inflight * m_keep;
-        if (m > cap) status |= SAILOR_ST_OOM;
-        peak = m > peak ? m : peak;
-
-        double t = fb;                                       // the final stage sends nothing: fb + 2*0
-        if (i + 1 < P) {
-            t = t_self;                                      // next stage in the same run
-            if (left == 1) {                                 // next stage opens run q + 1
-                const sailor_run nx = runs[q + 1];
-                const double c = boundary_time(v, g, z, tp, nx.type, nx.zone, h->tp_values[nx.tp_idx], D, msg);
-                if (nx.zone != z) c_comm = add_rn(c_comm, mul_rn((double)xbytes, v.egress[z * h->Z + nx.zone]));
-                t = add_rn(fb, mul_rn(2.0, c));
+            const double sync = D > 1 ? allreduce_bytes_time(v, d, intra_dp, v.cmp_grad[ct], D, steps, coef) : 0.0;
+            const uint64_t inflight = (uint64_t)(P - i) < n_b ? (uint64_t)(P - i) : n_b;
+            const uint64_t m = mm[0] + resv + inflight * mm[1];
+            if (m > cap) status |= SAILOR_ST_OOM;
+            peak = m > peak ? m : peak;
+            max_u = dmax(max_u, upd);
+            max_sync = dmax(max_sync, sync);
+            // stages of the piece whose receiver sits in the same run
+            const bool closes = piece_end == run_end || piece_end == P;      // its last stage has a time of its own
+            const uint32_t n_plain = piece_end - i - (closes ? 1u : 0u);
+            if (n_plain) {
+                const double t_self = add_rn(fb, c2_self);
+                max_t = dmax(max_t, t_self);
+                for (uint32_t n = 0; n < n_plain; ++n) {
+                    sum_t = add_rn(sum_t, t_self);
+                    rate = add_rn(rate, gpu_rate);
+                }
             }
+            if (closes) {
+                double t = fb;                                       // the final stage sends nothing: fb + 2*0
+                if (piece_end < P) {                                 // the next stage opens run q + 1
+                    const sailor_run nx = runs[q + 1];
+                    const double c = boundary_time(v, g, z, tp, nx.type, nx.zone, h->tp_values[nx.tp_idx], D, msg);
+                    if (nx.zone != z) c_comm = add_rn(c_comm, mul_rn((double)xbytes, v.egress[z * h->Z + nx.zone]));
+                    t = add_rn(fb, mul_rn(2.0, c));
+                }
+                sum_t = add_rn(sum_t, t);
+                max_t = dmax(max_t, t);
+                rate = add_rn(rate, gpu_rate);
+            }
+            i = piece_end;
         }
-        sum_t = add_rn(sum_t, t);
-        max_t = dmax(max_t, t);
-        max_u = dmax(max_u, upd);
-        max_sync = dmax(max_sync, sync);
-        rate = add_rn(rate, gpu_rate);
-        if (--left == 0) ++q;
     }
     o.peak_mem = peak;
     o.status = status;
