@@ -45,6 +45,8 @@ struct DpProblem {
     uint32_t _pad;
     uint32_t first_idx[SAILOR_Z_MAX][SAILOR_T_MAX];    // index of "one stage, of this type" inside a slice
     uint32_t vt_off[SAILOR_Z_MAX];   // compact index: offset of the position's rank table in `vtabs`; DP_DENSE: mixed radix
+    uint32_t rank_off[SAILOR_Z_MAX]; // the position's rank table whatever its index (DP_DENSE: no counted type, or
+                                     // none built): lets a launch enumerate only the count vectors a stage can reach
     uint64_t magic[SAILOR_Z_MAX][SAILOR_T_MAX];    // ceil(2^64 / (cap + 1)) of a counted type: for 32-bit x,
                                                    // x / (cap + 1) == high 64 bits of x * magic
 };
@@ -180,6 +182,32 @@ __device__ __forceinline__ bool dp_counts(const DpProblem& pb, const uint32_t* _
     }
 }
 
+// The r-th count vector (lexicographic) among those within the caps that add up to at most `budget`.
+__device__ __forceinline__ void dp_unrank(const DpProblem& pb, const uint32_t* __restrict__ vt, uint32_t zp, uint32_t T,
+                                          uint32_t r, uint32_t budget, uint32_t (&u)[SAILOR_T_MAX]) {
+    const uint32_t w = pb.P + 1;
+    uint32_t s = budget, j = 0;
+#pragma unroll
+    for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
+        u[t] = 0;
+        if (t < T && pb.stride[zp][t]) {
+            const uint32_t* row = vt + (j + 1) * w;
+            const uint32_t top = row[s], lim = min((uint32_t)pb.cap[zp][t], s);
+            uint32_t x = 0, below = 0;
+            while (x < lim) {
+                const uint32_t nxt = top - row[s - x - 1];
+                if (nxt > r) break;
+                below = nxt;
+                ++x;
+            }
+            u[t] = x;
+            r -= below;
+            s -= x;
+            ++j;
+        }
+    }
+}
+
 // slice index of the count vector u with one more stage of type `plus_one` (compact index only)
 __device__ __forceinline__ uint32_t dp_rank(const DpProblem& pb, const uint32_t* __restrict__ vtabs, uint32_t zp, uint32_t T,
                                             const uint32_t (&u)[SAILOR_T_MAX], uint32_t plus_one) {
@@ -235,8 +263,10 @@ __device__ __forceinline__ DpMove dp_move(const DpProblem& pb, const uint32_t* _
 
 struct DpLevelParams {
     const DpProblem* problems;
-    const uint32_t* blk_problem;     // block -> problem of the batch
-    const uint32_t* blk_first;       // block -> first entry it covers
+    const uint32_t* blk_problem;     // entries mode: block -> problem of the batch
+    const uint32_t* blk_first;       // entries mode: block -> first entry it covers
+    const uint32_t* blk_prefix;      // live mode: [n_active + 1] blocks before each problem of this launch
+    uint32_t n_active;               // live mode: problems of this launch (a prefix of the batch)
     const double* tabs;
     const uint32_t* vtabs;           // rank tables of the compactly indexed zone positions
     DpVal* val[2];                   // level buffers; stage i lives in val[(P - 1 - i) & 1]
@@ -246,32 +276,81 @@ struct DpLevelParams {
     uint32_t dist;                   // stage i = P - 1 - dist
 };
 
+// LIVE = false: a thread per table entry (block map over entries); entries no stage sequence can reach at this
+// stage leave early.  LIVE = true: a thread per count vector that stage i can have reached (at most i + 1 stages
+// in the zone), enumerated by rank with that budget through the positions' rank tables (block map over those).
+template <bool LIVE>
 __global__ void __launch_bounds__(DP_THREADS, 4) dp_level_kernel(const __grid_constant__ DpLevelParams lp) {
     __shared__ DpProblem pb;
     const uint32_t tid = threadIdx.x;
+    uint32_t which, first;
+    if (LIVE) {                                              // the problem whose blocks include this one (all threads alike)
+        uint32_t lo = 0, hi = lp.n_active;
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (lp.blk_prefix[mid] <= blockIdx.x) lo = mid; else hi = mid;
+        }
+        which = lo;
+        first = (blockIdx.x - lp.blk_prefix[lo]) * DP_THREADS;
+    } else {
+        which = lp.blk_problem[blockIdx.x];
+        first = lp.blk_first[blockIdx.x];
+    }
     {
-        const DpProblem* src = lp.problems + lp.blk_problem[blockIdx.x];
+        const DpProblem* src = lp.problems + which;
         for (uint32_t x = tid; x < sizeof(DpProblem) / 4; x += DP_THREADS)
             reinterpret_cast<uint32_t*>(&pb)[x] = reinterpret_cast<const uint32_t*>(src)[x];
     }
     __syncthreads();
-    const uint32_t e = lp.blk_first[blockIdx.x] + tid;
-    if (e >= pb.n_lvl) return;
     const uint32_t T = lp.T, P = pb.P, i = P - 1 - lp.dist;
     const double* tab = lp.tabs + (size_t)pb.config * lp.lay.stride();
     const uint32_t* okv = reinterpret_cast<const uint32_t*>(tab + lp.lay.off_ok());
     const double nb = (double)*reinterpret_cast<const uint64_t*>(tab + lp.lay.off_nb());
-    // entry -> (zone position, type, counts); no division by run-time values: the slices of a position are
-    // stepped through, and the counts come off by reciprocal multiplication or by a walk through the rank table
-    uint32_t zp = 0;
-    while (zp + 1 < pb.nz && e >= pb.zp_base[zp + 1]) ++zp;
-    uint32_t g = 0, ui = e - pb.zp_base[zp];
-    const uint32_t S = pb.S[zp];
-    while (ui >= S) { ui -= S; ++g; }
+    uint32_t zp = 0, g = 0, ui, e;
     uint32_t u[SAILOR_T_MAX];
-    // stage i is at most the (i+1)-th stage of its zone: entries that count more are never reached, and
-    // since a move raises the count by one per stage, no entry that passes this test ever reads one that fails it
-    if (!dp_counts(pb, lp.vtabs, zp, T, ui, u, i + 1)) return;
+    uint32_t S;
+    if (LIVE) {
+        // live index -> (zone position, type, r-th count vector with at most i + 1 stages) -> its table entry
+        uint32_t l = first + tid;
+        const uint32_t budget = i + 1;                       // <= P
+        uint32_t wz = 0;
+        for (;; ++zp) {
+            if (zp == pb.nz) return;                             // past the last live vector of this stage
+            wz = 1;
+            if (pb.rank_off[zp] != DP_DENSE) {
+                const uint32_t* row0 = lp.vtabs + pb.rank_off[zp];   // V[0][s]: vectors of all counted types up to sum s
+                wz = row0[budget] - row0[budget - 1];
+            }
+            if (l < T * wz) break;
+            l -= T * wz;
+        }
+        while (l >= wz) { l -= wz; ++g; }
+        S = pb.S[zp];
+        if (pb.rank_off[zp] != DP_DENSE) dp_unrank(pb, lp.vtabs + pb.rank_off[zp], zp, T, l, budget, u);
+        else {
+#pragma unroll
+            for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) u[t] = 0;
+        }
+        if (pb.vt_off[zp] != DP_DENSE) ui = dp_rank(pb, lp.vtabs, zp, T, u, 0xffffffffu);
+        else {
+            ui = 0;
+#pragma unroll
+            for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) ui += (t < T) ? u[t] * pb.stride[zp][t] : 0u;
+        }
+        e = pb.zp_base[zp] + g * S + ui;
+    } else {
+        e = first + tid;
+        if (e >= pb.n_lvl) return;
+        // entry -> (zone position, type, counts); no division by run-time values: the slices of a position are
+        // stepped through, and the counts come off by reciprocal multiplication or by a walk through the rank table
+        while (zp + 1 < pb.nz && e >= pb.zp_base[zp + 1]) ++zp;
+        ui = e - pb.zp_base[zp];
+        S = pb.S[zp];
+        while (ui >= S) { ui -= S; ++g; }
+        // stage i is at most the (i+1)-th stage of its zone: entries that count more are never reached, and
+        // since a move raises the count by one per stage, no entry that passes this test ever reads one that fails it
+        if (!dp_counts(pb, lp.vtabs, zp, T, ui, u, i + 1)) return;
+    }
     DpVal* cur = lp.val[lp.dist & 1] + pb.val_off;
     const DpVal* nxt = lp.val[(lp.dist & 1) ^ 1] + pb.val_off;
     uint8_t* choice = lp.choice + pb.choice_off + (size_t)i * pb.n_lvl;

@@ -1355,6 +1355,13 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     // fits, 2 = by rank whenever it fits (the environment variable exists for tests that exercise each way)
     int index_mode = 0;
     if (const char* env = getenv("SAILOR_DP_INDEX")) index_mode = !strcmp(env, "dense") ? 1 : !strcmp(env, "compact") ? 2 : 0;
+    // which threads a stage's launch has: one per count vector the stage can have reached ("live", whenever every
+    // zone position has its rank table), or one per table entry (SAILOR_DP_ENUM=entries, for tests)
+    bool all_live = true;
+    if (const char* env = getenv("SAILOR_DP_ENUM")) all_live = strcmp(env, "entries") != 0;
+    std::vector<uint64_t> V, live_stage;                     // scratch of the loop below
+    std::vector<uint64_t> live_off(n_problems + 1, 0);      // per problem: where its per-stage live counts start
+    std::vector<uint32_t> live_cnt;                          // live count vectors (x types) of stage i, all positions
     uint64_t n_states = 0;
     for (uint64_t c = 0; c < n_config; ++c) {
         const Config cf = config_of(d, (uint32_t)c);
@@ -1368,8 +1375,10 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
             pb.config = (uint32_t)c; pb.order = q; pb.index = (uint32_t)(c * n_orders + q);
             pb.P = cf.P; pb.nz = orders[q].n; pb.need = (uint32_t)(need > 0xffffffffull ? 0xffffffffull : need);
             memset(pb.first_later, DP_NONE, sizeof(pb.first_later));
+            live_off[c * n_orders + q] = live_cnt.size();
             if (!valid) continue;                           // no entries: the finish step finds no plan
             uint64_t n_lvl = 0;
+            live_stage.assign(cf.P, 0);
             for (uint32_t zp = 0; zp < pb.nz; ++zp) {
                 pb.zone[zp] = orders[q].zone[zp];
                 // counted types: the zone can host some but not all P stages of them
@@ -1387,7 +1396,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                 }
                 // compact index: count vectors within the caps that add up to at most P (rank tables V[j][s])
                 const uint32_t w = cf.P + 1;
-                std::vector<uint64_t> V((size_t)(m + 1) * w);
+                V.assign((size_t)(m + 1) * w, 0);
                 for (uint32_t sgm = 0; sgm < w; ++sgm) V[(size_t)m * w + sgm] = sgm + 1;           // W = 1 each
                 bool compact_ok = true;
                 for (uint32_t j = m; j-- > 0;) {
@@ -1406,17 +1415,27 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                                          : index_mode == 1 ? !dense_ok
                                                            : (m > 0 && compact_ok && (!dense_ok || dense > 4 * compact));
                 uint64_t S = 1;
+                pb.rank_off[zp] = DP_DENSE;
+                if (m > 0 && compact_ok) {                   // the rank table serves the live enumeration in any case
+                    pb.rank_off[zp] = (uint32_t)vtabs.size();
+                    for (uint64_t x : V) vtabs.push_back((uint32_t)x);
+                    if (vtabs.size() > (1ull << 30)) return SAILOR_E_RANGE;
+                } else if (m > 0) {
+                    all_live = false;
+                }
+                for (uint32_t st = 0; st < cf.P; ++st) {     // count vectors with at most st + 1 stages, times the types
+                    const uint32_t bud = st + 1;
+                    live_stage[st] += (uint64_t)T * (m > 0 && compact_ok ? V[bud] - V[bud - 1] : 1);
+                }
                 if (use_compact) {
                     S = compact;
-                    pb.vt_off[zp] = (uint32_t)vtabs.size();
-                    for (uint64_t x : V) vtabs.push_back((uint32_t)x);
+                    pb.vt_off[zp] = pb.rank_off[zp];
                     for (uint32_t j = 0; j < m; ++j) {
                         // rank of "one stage of type counted[j]": every vector that has a zero there and is zero before it
                         // comes first: V[j+1][P] - V[j+1][P-1] ... summed by the rank formula with u = e_j
                         pb.stride[zp][counted[j]] = 1;                                         // marks the type as counted
                         pb.first_idx[zp][counted[j]] = (uint32_t)(V[(size_t)(j + 1) * w + cf.P] - V[(size_t)(j + 1) * w + cf.P - 1]);
                     }
-                    if (vtabs.size() > (1ull << 30)) return SAILOR_E_RANGE;
                 } else {
                     pb.vt_off[zp] = DP_DENSE;
                     for (uint32_t j = 0; j < m; ++j) {
@@ -1439,6 +1458,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                         if (pb.cap[q][g] >= 1) { pb.first_later[zp][g] = (uint8_t)q; break; }
             pb.n_lvl = (uint32_t)n_lvl;
             n_states += n_lvl * cf.P;
+            for (uint32_t st = 0; st < cf.P; ++st) live_cnt.push_back((uint32_t)(live_stage[st] > n_lvl ? n_lvl : live_stage[st]));
         }
     }
     // deepest pipelines first, so that the launch for a distance from the last stage covers a prefix
@@ -1462,7 +1482,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
             bytes += wb;
             b.entries += pb.n_lvl;
             b.choice_bytes += (uint64_t)pb.n_lvl * pb.P;
-            b.blocks += (pb.n_lvl + DP_THREADS - 1) / DP_THREADS;
+            b.blocks += all_live ? (uint64_t)pb.P + 1 : (pb.n_lvl + DP_THREADS - 1) / DP_THREADS;   // words of the block lists
             ++b.count; ++j;
         }
         largest = bytes > largest ? bytes : largest;
@@ -1476,6 +1496,10 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
         max_count = std::max<uint64_t>(max_count, b.count);
     }
     if (max_blocks > 0x7fffffffull) return SAILOR_E_RANGE;
+    if (all_live) {                                        // what the launches visit: live count vectors only
+        n_states = 0;
+        for (uint32_t x : live_cnt) n_states += x;
+    }
 
     DeviceGuard guard(ctx->device);
     DpTabLayout lay;
@@ -1483,7 +1507,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     const size_t tab_bytes = (size_t)n_config * lay.stride() * sizeof(double);
     const size_t total = padded(tab_bytes) + padded(vtabs.size() * sizeof(uint32_t) + 4) + padded(n_problems * sizeof(DpResult)) +
                          padded(n_problems * sizeof(DpProblem)) +
-                         2 * padded(max_blocks * sizeof(uint32_t)) + 2 * padded(max_entries * sizeof(DpVal)) +
+                         2 * padded((max_blocks + p_max + 16) * sizeof(uint32_t)) + 2 * padded(max_entries * sizeof(DpVal)) +
                          padded(max_choice) + padded(sizeof(sailor_dp_result) * SAILOR_K_MAX) + padded(24) + 4096;
     if (total > ctx->dp_bytes) {
         CU(ctx, cudaStreamSynchronize(ctx->stream));
@@ -1499,8 +1523,8 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     uint32_t* d_vtabs = bump.take<uint32_t>(vtabs.size() + 1);
     DpResult* d_results = bump.take<DpResult>(n_problems);
     DpProblem* d_problems = bump.take<DpProblem>(n_problems);
-    uint32_t* d_blk_problem = bump.take<uint32_t>(max_blocks);
-    uint32_t* d_blk_first = bump.take<uint32_t>(max_blocks);
+    uint32_t* d_blk_problem = bump.take<uint32_t>(max_blocks + p_max + 16);
+    uint32_t* d_blk_first = bump.take<uint32_t>(max_blocks + p_max + 16);
     DpVal* d_val0 = bump.take<DpVal>(max_entries);
     DpVal* d_val1 = bump.take<DpVal>(max_entries);
     uint8_t* d_choice = bump.take<uint8_t>(max_choice);
@@ -1545,7 +1569,8 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
         blk_first.clear();
         uint64_t val_off = 0, choice_off = 0;
         uint32_t max_p = 0;
-        std::vector<uint64_t> blocks_upto(p_max + 2, 0);       // blocks of problems deeper than a distance
+        std::vector<uint64_t> blocks_upto(p_max + 2, 0);       // entries mode: blocks of problems deeper than a distance
+        std::vector<uint64_t> dist_off(p_max + 2, 0);          // live mode: where the block list of a distance starts
         for (size_t j = 0; j < b.count; ++j) {
             DpProblem pb = prob[by_depth[b.first + j]];
             pb.val_off = val_off;
@@ -1554,9 +1579,29 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
             choice_off += (uint64_t)pb.n_lvl * pb.P;
             stage_buf[j] = pb;
             max_p = pb.P > max_p ? pb.P : max_p;
-            const uint32_t nb = (pb.n_lvl + DP_THREADS - 1) / DP_THREADS;
-            for (uint32_t q = 0; q < nb; ++q) { blk_problem.push_back((uint32_t)j); blk_first.push_back(q * DP_THREADS); }
-            for (uint32_t dist = 0; dist < pb.P; ++dist) blocks_upto[dist] += nb;
+            if (!all_live) {
+                const uint32_t nb = (pb.n_lvl + DP_THREADS - 1) / DP_THREADS;
+                for (uint32_t q = 0; q < nb; ++q) { blk_problem.push_back((uint32_t)j); blk_first.push_back(q * DP_THREADS); }
+                for (uint32_t dist = 0; dist < pb.P; ++dist) blocks_upto[dist] += nb;
+            }
+        }
+        std::vector<uint32_t> n_active(p_max + 1, 0);
+        if (all_live) {                                        // per distance from the last stage: blocks before each problem
+            for (uint32_t dist = 0; dist < max_p; ++dist) {
+                dist_off[dist] = blk_problem.size();
+                uint32_t blocks = 0;
+                for (size_t j = 0; j < b.count; ++j) {
+                    const uint32_t pj = by_depth[b.first + j];
+                    const DpProblem& pb = prob[pj];
+                    if (pb.P <= dist) break;                   // sorted by depth
+                    blk_problem.push_back(blocks);
+                    blocks += (live_cnt[live_off[pj] + (pb.P - 1 - dist)] + DP_THREADS - 1) / DP_THREADS;
+                    ++n_active[dist];
+                }
+                blk_problem.push_back(blocks);
+            }
+            dist_off[max_p] = blk_problem.size();
+            blk_first.assign(1, 0);                            // unused in this mode
         }
         CU(ctx, cudaMemcpyAsync(d_problems, stage_buf.data(), b.count * sizeof(DpProblem), cudaMemcpyHostToDevice, ctx->stream));
         CU(ctx, cudaMemcpyAsync(d_blk_problem, blk_problem.data(), blk_problem.size() * sizeof(uint32_t), cudaMemcpyHostToDevice,
@@ -1570,7 +1615,15 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
         lp.val[0] = d_val0; lp.val[1] = d_val1; lp.choice = d_choice; lp.lay = lay; lp.T = T;
         for (uint32_t dist = 0; dist < max_p; ++dist) {
             lp.dist = dist;
-            dp_level_kernel<<<(uint32_t)blocks_upto[dist], DP_THREADS, 0, ctx->stream>>>(lp);
+            if (all_live) {
+                const uint32_t n_blk = blk_problem[dist_off[dist] + n_active[dist]];
+                if (n_blk == 0) continue;
+                lp.blk_prefix = d_blk_problem + dist_off[dist];
+                lp.n_active = n_active[dist];
+                dp_level_kernel<true><<<n_blk, DP_THREADS, 0, ctx->stream>>>(lp);
+            } else {
+                dp_level_kernel<false><<<(uint32_t)blocks_upto[dist], DP_THREADS, 0, ctx->stream>>>(lp);
+            }
             CU(ctx, cudaGetLastError());
             ++launches;
         }

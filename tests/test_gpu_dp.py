@@ -24,14 +24,20 @@ def _needs_cuda():
         pytest.fail("the gpu tests need a CUDA device")
 
 
-@pytest.fixture(params=["auto", "dense", "compact"], autouse=True)
+@pytest.fixture(params=["auto", "dense", "compact", "auto-entries", "compact-entries"], autouse=True)
 def _index_mode(request, monkeypatch):
-    """Every test runs with each way of indexing the tables' count vectors (mixed radix, by rank, the smaller)."""
-    if request.param == "auto":
+    """Every test runs with each way of indexing the tables' count vectors (mixed radix, by rank, the smaller) and
+    with both ways of enumerating a stage's work (reachable count vectors only, or every table entry)."""
+    index, _, enum = request.param.partition("-")
+    if index == "auto":
         monkeypatch.delenv("SAILOR_DP_INDEX", raising=False)
     else:
-        monkeypatch.setenv("SAILOR_DP_INDEX", request.param)
-    return request.param
+        monkeypatch.setenv("SAILOR_DP_INDEX", index)
+    if enum:
+        monkeypatch.setenv("SAILOR_DP_ENUM", enum)
+    else:
+        monkeypatch.delenv("SAILOR_DP_ENUM", raising=False)
+    return index
 
 
 class Ctx:
