@@ -280,7 +280,7 @@ struct DpLevelParams {
 // stage leave early.  LIVE = true: a thread per count vector that stage i can have reached (at most i + 1 stages
 // in the zone), enumerated by rank with that budget through the positions' rank tables (block map over those).
 template <bool LIVE>
-__global__ void __launch_bounds__(DP_THREADS, 4) dp_level_kernel(const __grid_constant__ DpLevelParams lp) {
+__global__ void __launch_bounds__(DP_THREADS, 5) dp_level_kernel(const __grid_constant__ DpLevelParams lp) {
     __shared__ DpProblem pb;
     const uint32_t tid = threadIdx.x;
     uint32_t which, first;
