@@ -42,11 +42,12 @@ struct DpProblem {
     uint32_t stride[SAILOR_Z_MAX][SAILOR_T_MAX];   // mixed-radix stride of a counted type; 0: not counted
     uint32_t S[SAILOR_Z_MAX];        // entries of one (position, type) slice
     uint32_t zp_base[SAILOR_Z_MAX + 1];            // first entry of each position's T slices
-    uint32_t _pad;
+    uint32_t vt_lo;                  // the problem's rank tables are vtabs[vt_lo .. vt_lo + vt_len)
     uint32_t first_idx[SAILOR_Z_MAX][SAILOR_T_MAX];    // index of "one stage, of this type" inside a slice
     uint32_t vt_off[SAILOR_Z_MAX];   // compact index: offset of the position's rank table in `vtabs`; DP_DENSE: mixed radix
     uint32_t rank_off[SAILOR_Z_MAX]; // the position's rank table whatever its index (DP_DENSE: no counted type, or
                                      // none built): lets a launch enumerate only the count vectors a stage can reach
+    uint32_t vt_len, _pad;
     uint64_t magic[SAILOR_Z_MAX][SAILOR_T_MAX];    // ceil(2^64 / (cap + 1)) of a counted type: for 32-bit x,
                                                    // x / (cap + 1) == high 64 bits of x * magic
 };
@@ -267,6 +268,7 @@ struct DpLevelParams {
     const uint32_t* blk_first;       // entries mode: block -> first entry it covers
     const uint32_t* blk_prefix;      // live mode: [n_active + 1] blocks before each problem of this launch
     uint32_t n_active;               // live mode: problems of this launch (a prefix of the batch)
+    uint32_t per_thread;             // vector kernel: count vectors a thread takes, a block's width apart
     const double* tabs;
     const uint32_t* vtabs;           // rank tables of the compactly indexed zone positions
     DpVal* val[2];                   // level buffers; stage i lives in val[(P - 1 - i) & 1]
@@ -394,6 +396,139 @@ __global__ void __launch_bounds__(DP_THREADS, 5) dp_level_kernel(const __grid_co
     }
     cur[e] = best;
     choice[e] = pick;
+}
+
+// A thread per reachable count vector, all types of stage i at once (TM >= T types).  The T entries that share a
+// count vector share its unranking, its table index and, for every type of the next stage, the moved vector's entry:
+// those are formed once, the next stage's values are gathered together, and only the T x T combinations remain per
+// type.  Same arithmetic per (type, next type) pair and the same order of the next types as dp_level_kernel.
+
+constexpr uint32_t DP_VEC_PER_THREAD = 4;       // in launches large enough to fill the GPU several times over
+
+template <uint32_t TM>
+__global__ void __launch_bounds__(DP_THREADS, TM <= 4 ? 3 : 2) dp_level_vec_kernel(const __grid_constant__ DpLevelParams lp) {
+    extern __shared__ uint32_t s_vt[];                       // the problem's rank tables
+    __shared__ DpProblem pb;
+    __shared__ uint32_t s_lo;
+    const uint32_t tid = threadIdx.x;
+    uint32_t which = 0;
+    // the problem whose blocks include this one: a search with DP_THREADS probes per round instead of two, so that
+    // a block waits for one or two loads, not for a chain of them
+    {
+        uint32_t lo = 0, n = lp.n_active;                    // invariant: prefix[lo] <= block < prefix[lo + n]
+        while (n > 1) {
+            const uint32_t step = (n + DP_THREADS - 1) / DP_THREADS;
+            const uint32_t a = lo + tid * step, b = a + step < lo + n ? a + step : lo + n;
+            if (a < lo + n && lp.blk_prefix[a] <= blockIdx.x && blockIdx.x < lp.blk_prefix[b]) s_lo = a;
+            __syncthreads();
+            const uint32_t got = s_lo;
+            __syncthreads();
+            n = got + step < lo + n ? step : lo + n - got;
+            lo = got;
+        }
+        which = lo;
+    }
+    const uint32_t first = (blockIdx.x - lp.blk_prefix[which]) * (DP_THREADS * lp.per_thread);
+    {
+        const DpProblem* src = lp.problems + which;
+        for (uint32_t x = tid; x < sizeof(DpProblem) / 4; x += DP_THREADS)
+            reinterpret_cast<uint32_t*>(&pb)[x] = reinterpret_cast<const uint32_t*>(src)[x];
+    }
+    __syncthreads();
+    for (uint32_t x = tid; x < pb.vt_len; x += DP_THREADS) s_vt[x] = lp.vtabs[pb.vt_lo + x];
+    __syncthreads();
+    // offsets into the rank tables count from the start of all tables: the staged copy is addressed the same way
+    const uint32_t* const vtabs = s_vt - pb.vt_lo;
+    const uint32_t T = lp.T, P = pb.P, i = P - 1 - lp.dist;
+    const double* tab = lp.tabs + (size_t)pb.config * lp.lay.stride();
+    const uint32_t* okv = reinterpret_cast<const uint32_t*>(tab + lp.lay.off_ok());
+    const double nb = (double)*reinterpret_cast<const uint64_t*>(tab + lp.lay.off_nb());
+    DpVal* cur = lp.val[lp.dist & 1] + pb.val_off;
+    const DpVal* nxt = lp.val[(lp.dist & 1) ^ 1] + pb.val_off;
+    uint8_t* choice = lp.choice + pb.choice_off + (size_t)i * pb.n_lvl;
+    const uint32_t budget = i + 1;                           // <= P
+    const uint32_t ok_here = okv[i];
+    // several vectors per thread, a block's width apart: the block's set-up (its problem, the rank tables) is paid once
+    for (uint32_t round = 0; round < lp.per_thread; ++round) {
+        uint32_t zp = 0, ui;
+        uint32_t u[SAILOR_T_MAX];
+        uint32_t l = first + round * DP_THREADS + tid;
+        for (;; ++zp) {
+            if (zp == pb.nz) return;                             // past the last reachable vector (later rounds too)
+            uint32_t wz = 1;
+            if (pb.rank_off[zp] != DP_DENSE) {
+                const uint32_t* row0 = vtabs + pb.rank_off[zp];
+                wz = row0[budget] - row0[budget - 1];
+            }
+            if (l < wz) break;
+            l -= wz;
+        }
+        const uint32_t S = pb.S[zp];
+        if (pb.rank_off[zp] != DP_DENSE) dp_unrank(pb, vtabs + pb.rank_off[zp], zp, T, l, budget, u);
+        else {
+#pragma unroll
+            for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) u[t] = 0;
+        }
+        if (pb.vt_off[zp] != DP_DENSE) ui = dp_rank(pb, vtabs, zp, T, u, 0xffffffffu);
+        else {
+            ui = 0;
+#pragma unroll
+            for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) ui += (t < T) ? u[t] * pb.stride[zp][t] : 0u;
+        }
+        const uint32_t e0 = pb.zp_base[zp] + ui;
+        // what follows a stage of each type g2: the entry it leads to (the same for every type of stage i) and its value
+        DpVal n[TM];
+        uint32_t d2v[TM];
+#pragma unroll
+        for (uint32_t g2 = 0; g2 < TM; ++g2) {
+            d2v[g2] = DP_NONE;
+            n[g2].sum = make_inf(); n[g2].mx = n[g2].sy = n[g2].up = 0.0;
+        }
+        if (lp.dist != 0) {
+            const uint32_t ok_next = okv[i + 1];
+#pragma unroll
+            for (uint32_t g2 = 0; g2 < TM; ++g2) {
+                if (g2 >= T || !((ok_next >> g2) & 1u)) continue;
+                const DpMove mv = dp_move(pb, vtabs, T, zp, ui, u, g2);
+                if (mv.zp == DP_NONE) continue;
+                n[g2] = nxt[mv.entry];
+                d2v[g2] = pb.zone[mv.zp] * T + g2;
+            }
+        }
+#pragma unroll
+        for (uint32_t g = 0; g < TM; ++g) {
+            if (g >= T) break;
+            DpVal best;
+            best.sum = make_inf(); best.mx = best.sy = best.up = 0.0;
+            uint8_t pick = DP_NONE;
+            // a state holds stage i itself: its type must be usable there and, when counted, counted at least once
+            const bool self = ((ok_here >> g) & 1u) && pb.cap[zp][g] >= 1 && (pb.stride[zp][g] == 0 || u[g] >= 1);
+            if (self) {
+                const uint32_t d = pb.zone[zp] * T + g;
+                const double fb = tab[lp.lay.off_fb() + i * T + g], upd = tab[lp.lay.off_upd() + i * T + g];
+                const double sync = tab[lp.lay.off_sync() + (size_t)i * lp.lay.R + d];
+                if (lp.dist == 0) {                                  // the last stage sends nothing
+                    best.sum = fb; best.mx = fb; best.sy = sync; best.up = upd;
+                } else {
+                    double best_v = make_inf();
+#pragma unroll
+                    for (uint32_t g2 = 0; g2 < TM; ++g2) {
+                        if (d2v[g2] == DP_NONE || !(n[g2].sum < make_inf())) continue;
+                        const double t = add_rn(fb, tab[lp.lay.off_c2x() + (size_t)d2v[g2] * lp.lay.R + d]);
+                        DpVal c;
+                        c.sum = add_rn(t, n[g2].sum);
+                        c.mx = dmax(t, n[g2].mx);
+                        c.sy = dmax(sync, n[g2].sy);
+                        c.up = dmax(upd, n[g2].up);
+                        const double val = add_rn(add_rn(add_rn(c.sum, mul_rn(nb, c.mx)), c.sy), c.up);
+                        if (pick == DP_NONE || val < best_v) { best = c; best_v = val; pick = (uint8_t)g2; }
+                    }
+                }
+            }
+            cur[e0 + g * S] = best;
+            choice[e0 + g * S] = pick;
+        }
+    }
 }
 
 // Stage 0 and the walk through the kept choices: one thread per problem.

@@ -1361,8 +1361,9 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     if (const char* env = getenv("SAILOR_DP_ENUM")) all_live = strcmp(env, "entries") != 0;
     std::vector<uint64_t> V, live_stage;                     // scratch of the loop below
     std::vector<uint64_t> live_off(n_problems + 1, 0);      // per problem: where its per-stage live counts start
-    std::vector<uint32_t> live_cnt;                          // live count vectors (x types) of stage i, all positions
+    std::vector<uint32_t> live_cnt;                          // count vectors stage i can have reached, all positions
     uint64_t n_states = 0;
+    uint32_t vt_len_max = 0;                                 // words of the largest problem's rank tables
     for (uint64_t c = 0; c < n_config; ++c) {
         const Config cf = config_of(d, (uint32_t)c);
         const uint32_t tp = h.tp_values[cf.tpi];
@@ -1378,6 +1379,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
             live_off[c * n_orders + q] = live_cnt.size();
             if (!valid) continue;                           // no entries: the finish step finds no plan
             uint64_t n_lvl = 0;
+            pb.vt_lo = (uint32_t)vtabs.size();
             live_stage.assign(cf.P, 0);
             for (uint32_t zp = 0; zp < pb.nz; ++zp) {
                 pb.zone[zp] = orders[q].zone[zp];
@@ -1423,9 +1425,9 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                 } else if (m > 0) {
                     all_live = false;
                 }
-                for (uint32_t st = 0; st < cf.P; ++st) {     // count vectors with at most st + 1 stages, times the types
+                for (uint32_t st = 0; st < cf.P; ++st) {     // count vectors with at most st + 1 stages
                     const uint32_t bud = st + 1;
-                    live_stage[st] += (uint64_t)T * (m > 0 && compact_ok ? V[bud] - V[bud - 1] : 1);
+                    live_stage[st] += m > 0 && compact_ok ? V[bud] - V[bud - 1] : 1;
                 }
                 if (use_compact) {
                     S = compact;
@@ -1457,8 +1459,10 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                     for (uint32_t q = zp + 1; q < pb.nz; ++q)
                         if (pb.cap[q][g] >= 1) { pb.first_later[zp][g] = (uint8_t)q; break; }
             pb.n_lvl = (uint32_t)n_lvl;
+            pb.vt_len = (uint32_t)(vtabs.size() - pb.vt_lo);
+            vt_len_max = pb.vt_len > vt_len_max ? pb.vt_len : vt_len_max;
             n_states += n_lvl * cf.P;
-            for (uint32_t st = 0; st < cf.P; ++st) live_cnt.push_back((uint32_t)(live_stage[st] > n_lvl ? n_lvl : live_stage[st]));
+            for (uint32_t st = 0; st < cf.P; ++st) live_cnt.push_back((uint32_t)(live_stage[st] > n_lvl ? n_lvl : live_stage[st]));   // <= n_lvl / T
         }
     }
     // deepest pipelines first, so that the launch for a distance from the last stage covers a prefix
@@ -1498,8 +1502,13 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     if (max_blocks > 0x7fffffffull) return SAILOR_E_RANGE;
     if (all_live) {                                        // what the launches visit: live count vectors only
         n_states = 0;
-        for (uint32_t x : live_cnt) n_states += x;
+        for (uint32_t x : live_cnt) n_states += (uint64_t)x * T;
     }
+    // a thread per count vector for all its types at once, or a thread per (count vector, type)
+    // (its blocks stage their problem's rank tables in shared memory: at most Z * (T + 1) * (P + 1) words)
+    bool by_vector = all_live && vt_len_max * 4 <= 40 * 1024;
+    if (const char* env = getenv("SAILOR_DP_ENUM")) by_vector = by_vector && strcmp(env, "types") != 0;
+    const uint32_t live_mult = by_vector ? 1u : T;
 
     DeviceGuard guard(ctx->device);
     DpTabLayout lay;
@@ -1585,17 +1594,26 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                 for (uint32_t dist = 0; dist < pb.P; ++dist) blocks_upto[dist] += nb;
             }
         }
-        std::vector<uint32_t> n_active(p_max + 1, 0);
+        std::vector<uint32_t> n_active(p_max + 1, 0), per_thread(p_max + 1, 1);
         if (all_live) {                                        // per distance from the last stage: blocks before each problem
             for (uint32_t dist = 0; dist < max_p; ++dist) {
                 dist_off[dist] = blk_problem.size();
                 uint32_t blocks = 0;
+                if (by_vector) {                               // small launches keep one vector per thread: more blocks
+                    uint64_t vectors = 0;
+                    for (size_t j = 0; j < b.count && prob[by_depth[b.first + j]].P > dist; ++j) {
+                        const uint32_t pj = by_depth[b.first + j];
+                        vectors += live_cnt[live_off[pj] + (prob[pj].P - 1 - dist)];
+                    }
+                    if (vectors >= 16ull * ctx->sm_count * DP_THREADS * DP_VEC_PER_THREAD) per_thread[dist] = DP_VEC_PER_THREAD;
+                }
+                const uint32_t per_block = DP_THREADS * per_thread[dist];
                 for (size_t j = 0; j < b.count; ++j) {
                     const uint32_t pj = by_depth[b.first + j];
                     const DpProblem& pb = prob[pj];
                     if (pb.P <= dist) break;                   // sorted by depth
                     blk_problem.push_back(blocks);
-                    blocks += (live_cnt[live_off[pj] + (pb.P - 1 - dist)] + DP_THREADS - 1) / DP_THREADS;
+                    blocks += (uint32_t)(((uint64_t)live_cnt[live_off[pj] + (pb.P - 1 - dist)] * live_mult + per_block - 1) / per_block);
                     ++n_active[dist];
                 }
                 blk_problem.push_back(blocks);
@@ -1620,7 +1638,10 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                 if (n_blk == 0) continue;
                 lp.blk_prefix = d_blk_problem + dist_off[dist];
                 lp.n_active = n_active[dist];
-                dp_level_kernel<true><<<n_blk, DP_THREADS, 0, ctx->stream>>>(lp);
+                lp.per_thread = per_thread[dist];
+                if (by_vector && T <= 4) dp_level_vec_kernel<4><<<n_blk, DP_THREADS, vt_len_max * 4, ctx->stream>>>(lp);
+                else if (by_vector) dp_level_vec_kernel<SAILOR_T_MAX><<<n_blk, DP_THREADS, vt_len_max * 4, ctx->stream>>>(lp);
+                else dp_level_kernel<true><<<n_blk, DP_THREADS, 0, ctx->stream>>>(lp);
             } else {
                 dp_level_kernel<false><<<(uint32_t)blocks_upto[dist], DP_THREADS, 0, ctx->stream>>>(lp);
             }

@@ -24,10 +24,11 @@ def _needs_cuda():
         pytest.fail("the gpu tests need a CUDA device")
 
 
-@pytest.fixture(params=["auto", "dense", "compact", "auto-entries", "compact-entries"], autouse=True)
+@pytest.fixture(params=["auto", "dense", "compact", "auto-types", "compact-types", "auto-entries", "compact-entries"], autouse=True)
 def _index_mode(request, monkeypatch):
     """Every test runs with each way of indexing the tables' count vectors (mixed radix, by rank, the smaller) and
-    with both ways of enumerating a stage's work (reachable count vectors only, or every table entry)."""
+    with each way of enumerating a stage's work (a thread per reachable count vector for all its types, which is the
+    default up to four GPU types; a thread per reachable count vector and type; a thread per table entry)."""
     index, _, enum = request.param.partition("-")
     if index == "auto":
         monkeypatch.delenv("SAILOR_DP_INDEX", raising=False)
