@@ -26,7 +26,8 @@ constexpr int DP_THREADS = 256;
 constexpr uint8_t DP_NONE = 255;
 constexpr uint32_t DP_DENSE = 0xffffffffu;
 
-struct DpVal {                       // best plan of stages i.. from a state; sum = +inf: there is none
+struct alignas(32) DpVal {           // best plan of stages i.. from a state; sum = +inf: there is none.  Aligned to its
+                                     // size: a value then moves in one load or store
     double sum, mx, sy, up;
 };
 
