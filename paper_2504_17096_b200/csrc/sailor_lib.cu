@@ -9,6 +9,8 @@
 #include <vector>
 
 #include <algorithm>
+#include <array>
+#include <map>
 
 #include "sailor_dp.cuh"
 #include "sailor_mixed.cuh"
@@ -1364,6 +1366,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     std::vector<uint32_t> live_cnt;                          // count vectors stage i can have reached, all positions
     uint64_t n_states = 0;
     uint32_t vt_len_max = 0;                                 // words of the largest problem's rank tables
+    std::map<std::array<uint64_t, 3>, uint64_t> same_states;
     for (uint64_t c = 0; c < n_config; ++c) {
         const Config cf = config_of(d, (uint32_t)c);
         const uint32_t tp = h.tp_values[cf.tpi];
@@ -1378,6 +1381,20 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
             memset(pb.first_later, DP_NONE, sizeof(pb.first_later));
             live_off[c * n_orders + q] = live_cnt.size();
             if (!valid) continue;                           // no entries: the finish step finds no plan
+            // the states, their index and the rank tables depend on (P, D * tp, zone order) only: configurations
+            // that differ in the microbatch size or in recomputation take them from the first such problem
+            const std::array<uint64_t, 3> key = {cf.P, need, q};
+            const auto seen = same_states.find(key);
+            if (seen != same_states.end()) {
+                const DpProblem& first = prob[seen->second];
+                const uint32_t config = pb.config, index = pb.index;
+                pb = first;
+                pb.config = config; pb.index = index;
+                live_off[c * n_orders + q] = live_off[seen->second];
+                n_states += (uint64_t)pb.n_lvl * cf.P;
+                continue;
+            }
+            same_states.emplace(key, c * n_orders + q);
             uint64_t n_lvl = 0;
             pb.vt_lo = (uint32_t)vtabs.size();
             live_stage.assign(cf.P, 0);
@@ -1502,7 +1519,8 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     if (max_blocks > 0x7fffffffull) return SAILOR_E_RANGE;
     if (all_live) {                                        // what the launches visit: live count vectors only
         n_states = 0;
-        for (uint32_t x : live_cnt) n_states += (uint64_t)x * T;
+        for (uint64_t j = 0; j < n_problems; ++j)
+            for (uint32_t st = 0; prob[j].n_lvl && st < prob[j].P; ++st) n_states += (uint64_t)live_cnt[live_off[j] + st] * T;
     }
     // a thread per count vector for all its types at once, or a thread per (count vector, type)
     // (its blocks stage their problem's rank tables in shared memory: at most Z * (T + 1) * (P + 1) words)
