@@ -49,6 +49,7 @@ struct DpProblem {
     uint32_t rank_off[SAILOR_Z_MAX]; // the position's rank table whatever its index (DP_DENSE: no counted type, or
                                      // none built): lets a launch enumerate only the count vectors a stage can reach
     uint32_t vt_len, _pad;
+    uint8_t n_counted[SAILOR_Z_MAX]; // counted types of each position
     uint64_t magic[SAILOR_Z_MAX][SAILOR_T_MAX];    // ceil(2^64 / (cap + 1)) of a counted type: for 32-bit x,
                                                    // x / (cap + 1) == high 64 bits of x * magic
 };
@@ -137,6 +138,28 @@ dp_tables_kernel(const unsigned char* __restrict__ blob, SpaceDesc sp, uint32_t 
 // W[j][s], the rank of u in lexicographic order is sum_j (V[j+1][s_j] - V[j+1][s_j - u_j]), s_0 = P,
 // s_{j+1} = s_j - u_j.  The table holds V[j][s] for j = 0 .. m, s = 0 .. P, row after row.
 
+// One digit of an unranking: the count x of a type, given the rank r among the vectors that agree on the types
+// before it and have s stages left for this type and the later ones.  `row` = V[j + 1][.] of the type's successor:
+// below(x) = row[s] - row[s - x] vectors start with a smaller count, and x is the largest count <= lim with
+// below(x) <= r.  After the last counted type nothing varies (V = s + 1), so below(x) = x there; elsewhere below is
+// non-decreasing in x and a bisection finds x.
+__device__ __forceinline__ void dp_digit(const uint32_t* __restrict__ row, uint32_t s, uint32_t lim, uint32_t r, bool last,
+                                         uint32_t& x, uint32_t& below) {
+    if (last) {
+        x = min(lim, r);
+        below = x;
+        return;
+    }
+    const uint32_t top = row[s];
+    uint32_t lo = 0, hi = lim;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi + 1) >> 1;                 // 1 <= mid <= lim <= s
+        if (top - row[s - mid] <= r) lo = mid; else hi = mid - 1;
+    }
+    x = lo;
+    below = lo ? top - row[s - lo] : 0u;
+}
+
 // counts of a slice index: u[t] for counted types, 0 for the others.  Returns false, possibly before all counts
 // are known, as soon as they add up to more than `limit`.
 __device__ __forceinline__ bool dp_counts(const DpProblem& pb, const uint32_t* __restrict__ vtabs, uint32_t zp, uint32_t T,
@@ -163,15 +186,9 @@ __device__ __forceinline__ bool dp_counts(const DpProblem& pb, const uint32_t* _
         for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
             u[t] = 0;
             if (t < T && pb.stride[zp][t]) {
-                const uint32_t* row = vt + (j + 1) * w;
-                const uint32_t top = row[s], lim = min((uint32_t)pb.cap[zp][t], s);
-                uint32_t x = 0, below = 0;                       // `below`: vectors that start with a count smaller than x
-                while (x < lim) {
-                    const uint32_t nxt = top - row[s - x - 1];              // x < lim <= s
-                    if (nxt > r) break;
-                    below = nxt;
-                    ++x;
-                }
+                const uint32_t lim = min((uint32_t)pb.cap[zp][t], s);
+                uint32_t x, below;                               // `below`: vectors that start with a count smaller than x
+                dp_digit(vt + (j + 1) * w, s, lim, r, j + 1 == pb.n_counted[zp], x, below);
                 u[t] = x;
                 total += x;
                 if (total > limit) return false;                 // the walks of the remaining types are not needed
@@ -193,15 +210,9 @@ __device__ __forceinline__ void dp_unrank(const DpProblem& pb, const uint32_t* _
     for (uint32_t t = 0; t < SAILOR_T_MAX; ++t) {
         u[t] = 0;
         if (t < T && pb.stride[zp][t]) {
-            const uint32_t* row = vt + (j + 1) * w;
-            const uint32_t top = row[s], lim = min((uint32_t)pb.cap[zp][t], s);
-            uint32_t x = 0, below = 0;
-            while (x < lim) {
-                const uint32_t nxt = top - row[s - x - 1];
-                if (nxt > r) break;
-                below = nxt;
-                ++x;
-            }
+            const uint32_t lim = min((uint32_t)pb.cap[zp][t], s);
+            uint32_t x, below;
+            dp_digit(vt + (j + 1) * w, s, lim, r, j + 1 == pb.n_counted[zp], x, below);
             u[t] = x;
             r -= below;
             s -= x;

@@ -1413,6 +1413,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                         if (dense > (1ull << 31)) dense_ok = false;
                     }
                 }
+                pb.n_counted[zp] = (uint8_t)m;
                 // compact index: count vectors within the caps that add up to at most P (rank tables V[j][s])
                 const uint32_t w = cf.P + 1;
                 V.assign((size_t)(m + 1) * w, 0);
