@@ -186,9 +186,8 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
     }
 }
 
-// One thread per plan with mixed replicas (648-byte records, read in place: a thread walks its own
-// record several times, the second time from L1/L2).  Tables in shared memory, per-thread GPU counters
-// in shared memory as [digit][thread].
+// One warp per plan with mixed replicas (648-byte records, read in place, lane i reading stage i).  Tables in
+// shared memory, then R 64-bit GPU counters per warp.
 __global__ void __launch_bounds__(SIM_THREADS)
 simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
                       const sailor_mixed_plan* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
@@ -196,7 +195,8 @@ simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __
                       unsigned int* error) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ uint64_t mbar;
-    const uint32_t tid = threadIdx.x;
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    constexpr uint32_t WARPS = SIM_THREADS / 32;
     const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(blob)->static_bytes;
     if (!bulk_load(dyn, blob, static_bytes, &mbar)) {
         if (tid == 0) atomicExch(error, 1u);
@@ -206,13 +206,16 @@ simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __
     }
     TabView v;
     v.bind(dyn, blob);
-    uint32_t* counters = reinterpret_cast<uint32_t*>(dyn + static_bytes) + tid;
-    for (uint64_t j = (uint64_t)blockIdx.x * SIM_THREADS + tid; j < n; j += (uint64_t)gridDim.x * SIM_THREADS) {
-        const SimOut o = simulate_mixed_record(v, avail, plans[j], counters, SIM_THREADS);
-        if (t_iter) t_iter[j] = o.t_iter;
-        if (peak_mem) peak_mem[j] = o.peak_mem;
-        if (cost) cost[j] = o.cost;
-        if (status) status[j] = o.status;
+    unsigned long long* counters = reinterpret_cast<unsigned long long*>(dyn + static_bytes) + (size_t)warp * v.h->R;
+    for (uint64_t j = (uint64_t)blockIdx.x * WARPS + warp; j < n; j += (uint64_t)gridDim.x * WARPS) {
+        const SimOut o = simulate_mixed_warp(v, avail, plans[j], counters, lane);
+        if (lane == 0) {
+            if (t_iter) t_iter[j] = o.t_iter;
+            if (peak_mem) peak_mem[j] = o.peak_mem;
+            if (cost) cost[j] = o.cost;
+            if (status) status[j] = o.status;
+        }
+        __syncwarp();
     }
 }
 
@@ -989,10 +992,10 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
         CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_mixed_plan), cudaMemcpyHostToDevice, ctx->stream));
         d_plans = dp;
     }
-    const uint64_t tiles = (n + SIM_THREADS - 1) / SIM_THREADS;
-    const uint64_t cap = (uint64_t)ctx->sm_count * 16;
+    const uint64_t tiles = (n + SIM_THREADS / 32 - 1) / (SIM_THREADS / 32);     // a warp per plan
+    const uint64_t cap = (uint64_t)ctx->sm_count * 32;
     const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
-    const size_t smem = ctx->hdr.static_bytes + sizeof(uint32_t) * SIM_THREADS * ctx->hdr.R;
+    const size_t smem = ctx->hdr.static_bytes + sizeof(unsigned long long) * (SIM_THREADS / 32) * ctx->hdr.R;
     simulate_mixed_kernel<<<grid, SIM_THREADS, smem, ctx->stream>>>(ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s,
                                                                      &ctx->d_ctrl->error);
     CU(ctx, cudaGetLastError());
