@@ -417,51 +417,24 @@ __global__ void __launch_bounds__(DP_THREADS, 5) dp_level_kernel(const __grid_co
 
 constexpr uint32_t DP_VEC_PER_THREAD = 4;       // in launches large enough to fill the GPU several times over
 
+// The work of one stage (distance `dist` from the last) of the problem `pb` for the count vectors first + tid,
+// first + DP_THREADS + tid, ... (`rounds` of them): see dp_level_vec_kernel.  `vtabs` addresses the problem's rank
+// tables by their offsets from the start of all tables.
 template <uint32_t TM>
-__global__ void __launch_bounds__(DP_THREADS, TM <= 4 ? 3 : 2) dp_level_vec_kernel(const __grid_constant__ DpLevelParams lp) {
-    extern __shared__ uint32_t s_vt[];                       // the problem's rank tables
-    __shared__ DpProblem pb;
-    __shared__ uint32_t s_lo;
+__device__ __forceinline__ void dp_vec_level(const DpLevelParams& lp, const DpProblem& pb, const uint32_t* vtabs, uint32_t dist,
+                                             uint32_t first, uint32_t rounds) {
     const uint32_t tid = threadIdx.x;
-    uint32_t which = 0;
-    // the problem whose blocks include this one: a search with DP_THREADS probes per round instead of two, so that
-    // a block waits for one or two loads, not for a chain of them
-    {
-        uint32_t lo = 0, n = lp.n_active;                    // invariant: prefix[lo] <= block < prefix[lo + n]
-        while (n > 1) {
-            const uint32_t step = (n + DP_THREADS - 1) / DP_THREADS;
-            const uint32_t a = lo + tid * step, b = a + step < lo + n ? a + step : lo + n;
-            if (a < lo + n && lp.blk_prefix[a] <= blockIdx.x && blockIdx.x < lp.blk_prefix[b]) s_lo = a;
-            __syncthreads();
-            const uint32_t got = s_lo;
-            __syncthreads();
-            n = got + step < lo + n ? step : lo + n - got;
-            lo = got;
-        }
-        which = lo;
-    }
-    const uint32_t first = (blockIdx.x - lp.blk_prefix[which]) * (DP_THREADS * lp.per_thread);
-    {
-        const DpProblem* src = lp.problems + which;
-        for (uint32_t x = tid; x < sizeof(DpProblem) / 4; x += DP_THREADS)
-            reinterpret_cast<uint32_t*>(&pb)[x] = reinterpret_cast<const uint32_t*>(src)[x];
-    }
-    __syncthreads();
-    for (uint32_t x = tid; x < pb.vt_len; x += DP_THREADS) s_vt[x] = lp.vtabs[pb.vt_lo + x];
-    __syncthreads();
-    // offsets into the rank tables count from the start of all tables: the staged copy is addressed the same way
-    const uint32_t* const vtabs = s_vt - pb.vt_lo;
-    const uint32_t T = lp.T, P = pb.P, i = P - 1 - lp.dist;
+    const uint32_t T = lp.T, P = pb.P, i = P - 1 - dist;
     const double* tab = lp.tabs + (size_t)pb.config * lp.lay.stride();
     const uint32_t* okv = reinterpret_cast<const uint32_t*>(tab + lp.lay.off_ok());
     const double nb = (double)*reinterpret_cast<const uint64_t*>(tab + lp.lay.off_nb());
-    DpVal* cur = lp.val[lp.dist & 1] + pb.val_off;
-    const DpVal* nxt = lp.val[(lp.dist & 1) ^ 1] + pb.val_off;
+    DpVal* cur = lp.val[dist & 1] + pb.val_off;
+    const DpVal* nxt = lp.val[(dist & 1) ^ 1] + pb.val_off;
     uint8_t* choice = lp.choice + pb.choice_off + (size_t)i * pb.n_lvl;
     const uint32_t budget = i + 1;                           // <= P
     const uint32_t ok_here = okv[i];
     // several vectors per thread, a block's width apart: the block's set-up (its problem, the rank tables) is paid once
-    for (uint32_t round = 0; round < lp.per_thread; ++round) {
+    for (uint32_t round = 0; round < rounds; ++round) {
         uint32_t zp = 0, ui;
         uint32_t u[SAILOR_T_MAX];
         uint32_t l = first + round * DP_THREADS + tid;
@@ -496,7 +469,7 @@ __global__ void __launch_bounds__(DP_THREADS, TM <= 4 ? 3 : 2) dp_level_vec_kern
             d2v[g2] = DP_NONE;
             n[g2].sum = make_inf(); n[g2].mx = n[g2].sy = n[g2].up = 0.0;
         }
-        if (lp.dist != 0) {
+        if (dist != 0) {
             const uint32_t ok_next = okv[i + 1];
 #pragma unroll
             for (uint32_t g2 = 0; g2 < TM; ++g2) {
@@ -519,7 +492,7 @@ __global__ void __launch_bounds__(DP_THREADS, TM <= 4 ? 3 : 2) dp_level_vec_kern
                 const uint32_t d = pb.zone[zp] * T + g;
                 const double fb = tab[lp.lay.off_fb() + i * T + g], upd = tab[lp.lay.off_upd() + i * T + g];
                 const double sync = tab[lp.lay.off_sync() + (size_t)i * lp.lay.R + d];
-                if (lp.dist == 0) {                                  // the last stage sends nothing
+                if (dist == 0) {                                  // the last stage sends nothing
                     best.sum = fb; best.mx = fb; best.sy = sync; best.up = upd;
                 } else {
                     double best_v = make_inf();
@@ -540,6 +513,76 @@ __global__ void __launch_bounds__(DP_THREADS, TM <= 4 ? 3 : 2) dp_level_vec_kern
             cur[e0 + g * S] = best;
             choice[e0 + g * S] = pick;
         }
+    }
+}
+
+template <uint32_t TM>
+__global__ void __launch_bounds__(DP_THREADS, TM <= 4 ? 3 : 2) dp_level_vec_kernel(const __grid_constant__ DpLevelParams lp) {
+    extern __shared__ uint32_t s_vt[];                       // the problem's rank tables
+    __shared__ DpProblem pb;
+    __shared__ uint32_t s_lo;
+    const uint32_t tid = threadIdx.x;
+    uint32_t which = 0;
+    // the problem whose blocks include this one: a search with DP_THREADS probes per round instead of two, so that
+    // a block waits for one or two loads, not for a chain of them
+    {
+        uint32_t lo = 0, n = lp.n_active;                    // invariant: prefix[lo] <= block < prefix[lo + n]
+        while (n > 1) {
+            const uint32_t step = (n + DP_THREADS - 1) / DP_THREADS;
+            const uint32_t a = lo + tid * step, b = a + step < lo + n ? a + step : lo + n;
+            if (a < lo + n && lp.blk_prefix[a] <= blockIdx.x && blockIdx.x < lp.blk_prefix[b]) s_lo = a;
+            __syncthreads();
+            const uint32_t got = s_lo;
+            __syncthreads();
+            n = got + step < lo + n ? step : lo + n - got;
+            lo = got;
+        }
+        which = lo;
+    }
+    const uint32_t first = (blockIdx.x - lp.blk_prefix[which]) * (DP_THREADS * lp.per_thread);
+    {
+        const DpProblem* src = lp.problems + which;
+        for (uint32_t x = tid; x < sizeof(DpProblem) / 4; x += DP_THREADS)
+            reinterpret_cast<uint32_t*>(&pb)[x] = reinterpret_cast<const uint32_t*>(src)[x];
+    }
+    __syncthreads();
+    for (uint32_t x = tid; x < pb.vt_len; x += DP_THREADS) s_vt[x] = lp.vtabs[pb.vt_lo + x];
+    __syncthreads();
+    // offsets into the rank tables count from the start of all tables: the staged copy is addressed the same way
+    const uint32_t* const vtabs = s_vt - pb.vt_lo;
+    dp_vec_level<TM>(lp, pb, vtabs, lp.dist, first, lp.per_thread);
+}
+
+// Small problems: a block takes one problem through all its stages, from the last to the first, with a barrier
+// between stages (a stage reads only what the same block wrote for the stage after it): one launch per batch
+// instead of one per stage.
+template <uint32_t TM>
+__global__ void __launch_bounds__(DP_THREADS, TM <= 4 ? 3 : 2) dp_problem_kernel(const __grid_constant__ DpLevelParams lp) {
+    extern __shared__ uint32_t s_vt[];                       // the problem's rank tables
+    __shared__ DpProblem pb;
+    const uint32_t tid = threadIdx.x;
+    {
+        const DpProblem* src = lp.problems + blockIdx.x;
+        for (uint32_t x = tid; x < sizeof(DpProblem) / 4; x += DP_THREADS)
+            reinterpret_cast<uint32_t*>(&pb)[x] = reinterpret_cast<const uint32_t*>(src)[x];
+    }
+    __syncthreads();
+    for (uint32_t x = tid; x < pb.vt_len; x += DP_THREADS) s_vt[x] = lp.vtabs[pb.vt_lo + x];
+    __syncthreads();
+    const uint32_t* const vtabs = s_vt - pb.vt_lo;
+    for (uint32_t dist = 0; dist < pb.P; ++dist) {
+        const uint32_t budget = pb.P - dist;                 // stage i = P - 1 - dist has at most i + 1 stages behind it
+        uint32_t vectors = 0;
+        for (uint32_t zp = 0; zp < pb.nz; ++zp) {
+            uint32_t wz = 1;
+            if (pb.rank_off[zp] != DP_DENSE) {
+                const uint32_t* row0 = vtabs + pb.rank_off[zp];
+                wz = row0[budget] - row0[budget - 1];
+            }
+            vectors += wz;
+        }
+        dp_vec_level<TM>(lp, pb, vtabs, dist, 0, (vectors + DP_THREADS - 1) / DP_THREADS);
+        __syncthreads();
     }
 }
 

@@ -1617,7 +1617,15 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
             }
         }
         std::vector<uint32_t> n_active(p_max + 1, 0), per_thread(p_max + 1, 1);
-        if (all_live) {                                        // per distance from the last stage: blocks before each problem
+        // small problems only (no stage of any problem has more than a few blocks' worth of count vectors): a block
+        // per problem runs all its stages in one launch
+        bool block_per_problem = by_vector;
+        for (size_t j = 0; block_per_problem && j < b.count; ++j) {
+            const uint32_t pj = by_depth[b.first + j];
+            for (uint32_t st = 0; st < prob[pj].P; ++st)
+                if (live_cnt[live_off[pj] + st] > 8u * DP_THREADS) { block_per_problem = false; break; }
+        }
+        if (all_live && !block_per_problem) {                                        // per distance from the last stage: blocks before each problem
             for (uint32_t dist = 0; dist < max_p; ++dist) {
                 dist_off[dist] = blk_problem.size();
                 uint32_t blocks = 0;
@@ -1644,16 +1652,24 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
             blk_first.assign(1, 0);                            // unused in this mode
         }
         CU(ctx, cudaMemcpyAsync(d_problems, stage_buf.data(), b.count * sizeof(DpProblem), cudaMemcpyHostToDevice, ctx->stream));
-        CU(ctx, cudaMemcpyAsync(d_blk_problem, blk_problem.data(), blk_problem.size() * sizeof(uint32_t), cudaMemcpyHostToDevice,
-                                ctx->stream));
-        CU(ctx, cudaMemcpyAsync(d_blk_first, blk_first.data(), blk_first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice,
-                                ctx->stream));
+        if (!blk_problem.empty())
+            CU(ctx, cudaMemcpyAsync(d_blk_problem, blk_problem.data(), blk_problem.size() * sizeof(uint32_t), cudaMemcpyHostToDevice,
+                                    ctx->stream));
+        if (!blk_first.empty())
+            CU(ctx, cudaMemcpyAsync(d_blk_first, blk_first.data(), blk_first.size() * sizeof(uint32_t), cudaMemcpyHostToDevice,
+                                    ctx->stream));
         DpLevelParams lp;
         memset(&lp, 0, sizeof(lp));
         lp.problems = d_problems; lp.blk_problem = d_blk_problem; lp.blk_first = d_blk_first; lp.tabs = d_tabs;
         lp.vtabs = d_vtabs;
         lp.val[0] = d_val0; lp.val[1] = d_val1; lp.choice = d_choice; lp.lay = lay; lp.T = T;
-        for (uint32_t dist = 0; dist < max_p; ++dist) {
+        if (block_per_problem) {
+            if (T <= 4) dp_problem_kernel<4><<<(uint32_t)b.count, DP_THREADS, vt_len_max * 4, ctx->stream>>>(lp);
+            else dp_problem_kernel<SAILOR_T_MAX><<<(uint32_t)b.count, DP_THREADS, vt_len_max * 4, ctx->stream>>>(lp);
+            CU(ctx, cudaGetLastError());
+            ++launches;
+        }
+        for (uint32_t dist = 0; dist < max_p && !block_per_problem; ++dist) {
             lp.dist = dist;
             if (all_live) {
                 const uint32_t n_blk = blk_problem[dist_off[dist] + n_active[dist]];
