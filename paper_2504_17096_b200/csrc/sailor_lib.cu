@@ -188,7 +188,7 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
 
 // One warp per plan with mixed replicas (648-byte records, read in place, lane i reading stage i).  Tables in
 // shared memory, then R 64-bit GPU counters per warp.
-__global__ void __launch_bounds__(SIM_THREADS)
+__global__ void __launch_bounds__(SIM_THREADS, 4)
 simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
                       const sailor_mixed_plan* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
                       uint64_t* __restrict__ peak_mem, double* __restrict__ cost, uint32_t* __restrict__ status,
