@@ -406,3 +406,25 @@ def parallel_search(w, kind: int, k: int, *, budget: float = 0.0, min_rate: floa
     costs = [c["min_cost"] for _, c in parts if c["n_feasible"]]
     counts["min_cost"] = min(costs) if costs else 0.0
     return hits, counts
+
+
+def _plan_snapshot(args):
+    w, snap, k = args
+    o = Oracle(w, snap)
+    return o.plan(k)
+
+
+def plan_snapshots(w, snapshots, k: int, *, procs: int = 0, pool=None):
+    """Oracle.plan for each availability snapshot of one workload, the snapshots spread over worker
+    processes (spawned).  Returns a list of (hits, counts, budget), one per snapshot, in order."""
+    import multiprocessing as mp
+    tasks = [(w, np.array(s, dtype=np.uint16, copy=True), k) for s in snapshots]
+    own = pool is None
+    if own:
+        pool = mp.get_context("spawn").Pool(procs or os.cpu_count() or 1)
+    try:
+        return pool.map(_plan_snapshot, tasks, chunksize=1)
+    finally:
+        if own:
+            pool.close()
+            pool.join()

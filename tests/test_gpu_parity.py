@@ -9,7 +9,7 @@ import numpy as np
 import pytest
 
 from helpers import REL_TOL_F64, golden_cases, rel_close, stages_to_records, workload_from_tables
-from oracle.binding import Oracle, parallel_search
+from oracle.binding import Oracle, parallel_search, plan_snapshots
 from paper_2504_17096_b200 import binding as B
 from paper_2504_17096_b200 import workloads as W
 
@@ -440,25 +440,27 @@ def test_plan_config6_min_cost_under_throughput(make_ctx):
 
 
 def test_plan_config4_snapshots_replan(make_ctx):
-    """Dynamic availability: re-plan per snapshot on one context; only the counts are uploaded."""
+    """Dynamic availability: re-plan per snapshot on one context (only the counts are uploaded); every one
+    of the 200 snapshots is compared with the oracle's two-pass plan, and the best plans must all agree."""
     w = W.config4(n_snapshots=200)
+    expected = plan_snapshots(w, w.snapshots, 4)         # the oracle, snapshots spread over the host cores
     cx = make_ctx(w)
     o = Oracle(w)
     obj = B.make_objective(w)
-    checked = 0
-    for t in range(0, 200, 8):                       # 25 of the 200 snapshots
-        snap = w.snapshots[t]
-        o.set_availability(snap)
+    agree = with_plan = 0
+    for t, snap in enumerate(w.snapshots):
+        hits, counts, budget = expected[t]
         B.sailor_set_availability(cx.ctx, snap)
-        hits, counts, budget = o.plan(4)
         res, st = B.sailor_plan(cx.ctx, cx.space, obj, 4)
         if hits:
+            with_plan += 1
             assert st.budget_used == budget
             assert_plan_equal(res, st, hits, counts, o, f"snapshot {t}")
+            agree += int(res[0].flat == hits[0]["flat"])
         else:
             assert res == []
-        checked += 1
-    assert checked == 25
+            agree += 1
+    assert agree == 200 and with_plan > 150
 
 
 def test_plan_config3_full_space(make_ctx):
@@ -508,3 +510,27 @@ def test_plan_config5_windows_and_sampled_winner(make_ctx):
     kept = {r.flat for r in res}
     for f, t in zip(sample[feas], ts[feas]):
         assert (t, int(f)) >= worst or int(f) in kept
+
+
+def test_config5_sampled_candidates_match_oracle_one_by_one(make_ctx):
+    """The seeded uniform subsample of 1e6 flat indices of workload 5, candidate by candidate: the library's
+    decoder gives the record, the batch simulator its status, peak bytes, time and cost, and each must equal
+    what the oracle computes for the same flat index (integers exact, times and costs identical in their bits)."""
+    w = W.config5()
+    cx = make_ctx(w)
+    o = Oracle(w)
+    n = o.space_size()
+    rng = W.SplitMix64(55)
+    sample = np.array(sorted({rng.next_u64() % n for _ in range(1_000_000)}), dtype=np.uint64)
+    recs = (B.PlanRec * sample.size)()
+    decode, space = B.load().sailor_decode, C.byref(cx.space)
+    for j, f in enumerate(sample.tolist()):
+        assert decode(cx.ctx, space, f, C.byref(recs[j])) == 0
+    packed = np.frombuffer(recs, dtype=B.REC_DTYPE)
+    gpu = B.sailor_simulate(cx.ctx, packed)
+    orc = o.simulate_flat(sample)
+    assert_sim_equal(gpu, orc, "cfg5 sample")
+    # the sample covers every class and every pipeline depth of the space
+    assert set(np.unique(packed["P"]).tolist()) == set(w.p_values)
+    s = orc[0]
+    assert (s == 0).any() and (s & B.ST_OOM).any() and (s & B.ST_OVER_AVAIL).any() and (s & B.ST_INVALID).any()

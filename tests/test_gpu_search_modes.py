@@ -189,6 +189,26 @@ def test_degree_order_on_the_large_workloads_is_consistent():
             assert sorted((r.score, r.flat) for r in res) == [(r.score, r.flat) for r in res]
 
 
+def test_degree_order_on_a_four_segment_part_of_workload_3():
+    """Workload 3's model and cluster (5 zones x 4 types: 20 digits, four segments) with two pipeline depths and
+    a thinned configuration list, so that the oracle's pruned search finishes in seconds: degree order for both
+    objectives that have one, alone and with the tensor-parallel rule."""
+    w = W.config3()
+    w.p_values = [4, 8]
+    w.mbs_idx = [w.mbs_idx[0], w.mbs_idx[2]]
+    w.tp_idx = [w.tp_idx[1], w.tp_idx[3]]
+    w.budget_factor_over_cheapest = 0.0
+    o = Oracle(w)
+    assert w.radix == 20 and w.space_size() == 2 * (2 * 2 * len(w.rc_values) * len(w.d_values)) * 20 ** 4
+    with Ctx(w) as cx:
+        for kind, modes in ((W.OBJ_MAX_THROUGHPUT, PRUNE_D_ORDER), (W.OBJ_MIN_COST, PRUNE_D_ORDER | PRUNE_MIN_TP)):
+            hits, counts = o.search_pruned(kind, 16, modes)
+            obj = B.make_objective(w, kind=kind, flags=gpu_flags(modes), factor=0.0, budget=0.0, min_rate=0.0)
+            res, st = B.sailor_plan(cx.ctx, cx.space, obj, 16)
+            assert_same(res, st, hits, counts, f"cfg3 part kind={kind} modes={modes}")
+            assert counts["n_feasible"] > 16 and 0 < counts["n_configs_evaluated"] <= counts["n_configs"]
+
+
 def test_mode_argument_checks():
     w = W.tiny(seed=3)
     with Ctx(w) as cx:
