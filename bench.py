@@ -5,6 +5,19 @@
 A step is one whole search (`sailor_plan`: decode, simulate, select) over the workload's
 candidate space with every candidate's time and cost evaluated (no pruning).  Rank 0 prints one
 JSON line.  With --impl reference the CPU oracle is timed instead, on bounded samples.
+
+With N > 1 ranks (one per GPU) the one space is split into contiguous flat-index ranges of equal
+estimated cost, each rank searches its range with `sailor_plan_range`, and the per-rank lists are
+merged by (score, flat) after one gather of k records per rank ("scaling": "strong");
+`--replicas` instead gives every rank the whole space and its own availability snapshot ("weak").
+
+Hooks for the profiling commands quoted under profiles/ (they change what is run, not how it is
+timed): `--only-p P ...` keeps only those pipeline depths of the workload (a small case for ncu),
+`--dp-only` runs just the dynamic-programming search, `--dp-workspace-gib` bounds its tables, `--sim-only`
+runs just the explicit-batch kernels,
+`--no-cpu` / `--no-aux` drop the oracle leg / the secondary measurements, and
+`--write-counters LOG.csv` turns an ncu `--csv` log of one plan_kernel launch into the counter file
+the roofline figure reads (stamped with a hash of the kernel sources it was captured on).
 """
 from __future__ import annotations
 
@@ -30,9 +43,68 @@ K_TOP = 32
 # algorithmic work of one candidate with P stages, in lane operations (adds, multiplies,
 # divisions, maxima, compares, table reads of the stage-by-stage evaluation)
 OPS_PLAN, OPS_STAGE = 40, 35
-SM_COUNT, ISSUE_PER_SM, LANES = 148, 4, 32
-# ncu counters per plan_kernel launch (smsp__inst_executed.sum; dram__bytes_read.sum + dram__bytes_write.sum)
-NCU_PER_LAUNCH = {"cfg5-stress-96layer": {"warp_inst": 11245134608, "dram_bytes": 841216}}
+ISSUE_PER_SM, LANES = 4, 32
+# counters of one plan_kernel launch (ncu, one pass), kept with a hash of the sources they were captured on
+COUNTER_FILE = os.path.join(ROOT, "profiles", "plan_kernel_cfg5_counters.txt")
+COUNTER_METRICS = ("smsp__inst_executed.sum", "smsp__inst_executed_pipe_fp64.sum", "smsp__inst_executed_pipe_alu.sum",
+                   "smsp__inst_executed_pipe_fma.sum", "smsp__inst_executed_pipe_lsu.sum", "dram__bytes_read.sum",
+                   "dram__bytes_write.sum")
+KERNEL_SOURCES = ("sailor_plan_kernels.cuh", "sailor_tables.cuh")
+
+
+def kernel_source_hash() -> str:
+    """Hash of the files that define plan_kernel and of the compiler flags: a counter file is only valid for
+    the kernel it was captured on."""
+    import hashlib
+    from paper_2504_17096_b200 import build as cuda_build
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(cuda_build.CSRC, name), "rb") as f:
+            h.update(f.read())
+    h.update(" ".join(cuda_build.NVCC_FLAGS).encode())
+    return h.hexdigest()[:16]
+
+
+def read_counters(workload: str):
+    """The stored counters of one plan_kernel launch on `workload`, or (None, why)."""
+    try:
+        with open(COUNTER_FILE) as f:
+            rows = dict(line.split(None, 1) for line in f if line.strip() and not line.startswith("#"))
+    except OSError:
+        return None, "no counter file"
+    rows = {k: v.strip() for k, v in rows.items()}
+    if rows.get("workload") != workload:
+        return None, f"counters are of {rows.get('workload')}"
+    if rows.get("source_sha256_16") != kernel_source_hash():
+        return None, "the kernel sources changed after the counters were captured"
+    return {k: int(float(rows[k])) for k in COUNTER_METRICS if k in rows}, None
+
+
+def write_counters(args) -> None:
+    """ncu --csv log (one plan_kernel launch, the metrics of COUNTER_METRICS) -> the counter file."""
+    import csv
+    w = workload_by_name(args.workload, args.only_p)
+    found = {}
+    with open(args.write_counters, newline="") as f:
+        rows = [r for r in csv.reader(f) if len(r) > 3]
+    head = next(r for r in rows if "Metric Name" in r)
+    i_name, i_val, i_kernel = head.index("Metric Name"), head.index("Metric Value"), head.index("Kernel Name")
+    for r in rows:
+        if len(r) > max(i_name, i_val) and r[i_name] in COUNTER_METRICS and "plan_kernel" in r[i_kernel]:
+            found.setdefault(r[i_name], int(float(r[i_val].replace(",", ""))))
+    missing = [m for m in COUNTER_METRICS if m not in found]
+    if missing:
+        raise SystemExit(f"the log lacks {missing}")
+    with open(COUNTER_FILE, "w") as f:
+        f.write("# Counters of ONE plan_kernel launch (every candidate evaluated), from one ncu pass set:\n")
+        f.write("#   ncu --metrics " + ",".join(COUNTER_METRICS) + " --clock-control none -k regex:plan_kernel -c 1 \\\n")
+        f.write("#       --csv --log-file LOG.csv python bench.py --steps 1 --warmup 1 --no-cpu --no-aux\n")
+        f.write("#   python bench.py --write-counters LOG.csv\n")
+        f.write("# bench.py uses them only while source_sha256_16 equals the hash of the kernel sources in the tree.\n")
+        f.write(f"workload {w.name}\nsource_sha256_16 {kernel_source_hash()}\n")
+        for m in COUNTER_METRICS:
+            f.write(f"{m} {found[m]}\n")
+    print(open(COUNTER_FILE).read())
 
 
 def mean_ops_per_candidate(w: W.Workload) -> float:
@@ -64,7 +136,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20"],
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "10"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             pass
@@ -91,9 +163,9 @@ class ClockSampler:
             for name, v in zip(names, f[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        top = sorted(sm)[len(sm) // 2:] if sm else []        # the upper half: samples under load
-        return {"sm_mhz": statistics.median(top) if top else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        # the sampler runs only while the timed regions run, so every sample is under load
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
 def run_reference(args) -> None:
@@ -176,28 +248,24 @@ def dp_search(B, ctx, w, sp) -> dict:
             "segment_search_best_t_iter": seg[0].t_iter if seg else None}
 
 
-def aux_measurements(B, torch, dev) -> dict:
-    """Search seconds of the other workloads through the public call (host buffers), default mode."""
+def cold_search(B, torch, dev, w, flags: int = 0) -> dict:
+    """What a planner invoked once per job pays: a fresh context (tables uploaded, per-composition sums formed)
+    and its first search of the space (index arrays, survey, per-configuration table cache), wall clock."""
+    t0 = time.perf_counter()
+    ctx = B.sailor_create(w, dev, torch.cuda.current_stream().cuda_stream)
+    try:
+        B.sailor_set_availability(ctx, w.avail)
+        t1 = time.perf_counter()
+        res, _ = B.sailor_plan(ctx, B.make_space(w), B.make_objective(w, flags=flags), K_TOP)
+        t2 = time.perf_counter()
+    finally:
+        B.sailor_destroy(ctx)
+    return {"create_s": t1 - t0, "first_search_s": t2 - t1, "cold_search_s": t2 - t0, "found": len(res)}
+
+
+def explicit_batches(B, torch, dev) -> dict:
+    """sailor_simulate / sailor_simulate_mixed on batches resident in HBM (larger than L2), CUDA events."""
     out = {}
-    for cfg in (1, 2, 3, 6):
-        w = W.CONFIGS[cfg]()
-        ctx = B.sailor_create(w, dev, torch.cuda.current_stream().cuda_stream)
-        try:
-            sp, ob = B.make_space(w), B.make_objective(w)
-            B.sailor_set_availability(ctx, w.avail)
-            B.sailor_plan(ctx, sp, ob, K_TOP)
-            ts = []
-            for _ in range(5):
-                t0 = time.perf_counter()
-                B.sailor_set_availability(ctx, w.avail)
-                _, st = B.sailor_plan(ctx, sp, ob, K_TOP)
-                ts.append(time.perf_counter() - t0)
-            out[f"cfg{cfg}"] = {"candidates": int(st.n_total), "search_s": statistics.median(ts),
-                                "kernel_ms": st.kernel_ms, "passes": 2 if w.budget_factor_over_cheapest > 0 else 1}
-            out[f"cfg{cfg}"]["pruning_modes"] = pruning_modes(B, ctx, w, sp)
-            out[f"cfg{cfg}"]["dp"] = dp_search(B, ctx, w, sp)
-        finally:
-            B.sailor_destroy(ctx)
     # explicit batches (sailor_simulate) with records resident in HBM: 72 B in + 28 B out per plan
     w = W.config5()
     ctx = B.sailor_create(w, dev, torch.cuda.current_stream().cuda_stream)
@@ -260,24 +328,69 @@ def aux_measurements(B, torch, dev) -> dict:
         del d_plans, t, c, m, st
     finally:
         B.sailor_destroy(ctx)
+    return out
+
+
+def aux_measurements(B, torch, dev, oracle_cfg4=None) -> dict:
+    """Search seconds of the other workloads through the public call (host buffers), default mode."""
+    out = {}
+    for cfg in (1, 2, 3, 6):
+        w = W.CONFIGS[cfg]()
+        cold = cold_search(B, torch, dev, w)
+        ctx = B.sailor_create(w, dev, torch.cuda.current_stream().cuda_stream)
+        try:
+            sp, ob = B.make_space(w), B.make_objective(w)
+            B.sailor_set_availability(ctx, w.avail)
+            B.sailor_plan(ctx, sp, ob, K_TOP)
+            ts = []
+            for _ in range(5):
+                t0 = time.perf_counter()
+                B.sailor_set_availability(ctx, w.avail)
+                _, st = B.sailor_plan(ctx, sp, ob, K_TOP)
+                ts.append(time.perf_counter() - t0)
+            out[f"cfg{cfg}"] = {"candidates": int(st.n_total), "search_s": statistics.median(ts),
+                                "kernel_ms": st.kernel_ms, "h2d_ms": st.h2d_ms, "d2h_ms": st.d2h_ms,
+                                "launches": int(st.n_launches), "passes": 2 if w.budget_factor_over_cheapest > 0 else 1,
+                                "cold_search_s": cold["cold_search_s"], "cold": cold}
+            out[f"cfg{cfg}"]["pruning_modes"] = pruning_modes(B, ctx, w, sp)
+            out[f"cfg{cfg}"]["dp"] = dp_search(B, ctx, w, sp)
+        finally:
+            B.sailor_destroy(ctx)
+    out.update(explicit_batches(B, torch, dev))
     w = W.config4()
     ctx = B.sailor_create(w, dev, torch.cuda.current_stream().cuda_stream)
     try:
         sp, ob = B.make_space(w), B.make_objective(w)
         B.sailor_set_availability(ctx, w.snapshots[0])
         B.sailor_plan(ctx, sp, ob, 4)
-        lat = []
+        lat, best = [], []
         for snap in w.snapshots:
             t0 = time.perf_counter()
             B.sailor_set_availability(ctx, snap)
-            B.sailor_plan(ctx, sp, ob, 4)
+            res, _ = B.sailor_plan(ctx, sp, ob, 4)
             lat.append(time.perf_counter() - t0)
+            best.append(int(res[0].flat) if res else None)
         lat.sort()
         out["cfg4"] = {"snapshots": len(lat), "replan_p50_s": lat[len(lat) // 2], "replan_p99_s": lat[int(len(lat) * 0.99)],
                        "replan_max_s": lat[-1]}
+        if oracle_cfg4 is not None:        # best-plan agreement with the oracle's two-pass plan of every snapshot
+            want = [(h[0]["flat"] if h else None) for h, _, _ in oracle_cfg4["plans"]]
+            out["cfg4"]["agree"] = f"{sum(int(a == b) for a, b in zip(best, want))}/{len(want)}"
+            out["cfg4"]["oracle_s_per_snapshot"] = oracle_cfg4["core_s"] / len(want)
+            out["cfg4"]["oracle_cores"] = oracle_cfg4["cores"]
     finally:
         B.sailor_destroy(ctx)
     return out
+
+
+def run_sim_only(args) -> None:
+    """Only the explicit-batch kernels (a few hundred MB on the device): a small command for profiling them.
+    Prints one JSON line of its own (not the benchmark line)."""
+    import torch
+    from paper_2504_17096_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    print(json.dumps({"sim_only": explicit_batches(B, torch, 0)}), flush=True)
 
 
 def run_dp_only(args) -> None:
@@ -305,10 +418,23 @@ def run_dp_only(args) -> None:
         B.sailor_destroy(ctx)
 
 
+def oracle_cfg4_plans() -> dict:
+    """The oracle's two-pass plan of each of workload 4's 200 snapshots, spread over the host cores (spawned
+    workers), for the best-plan agreement count."""
+    from oracle.binding import plan_snapshots
+    w = W.config4()
+    cores = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    plans = plan_snapshots(w, w.snapshots, 1, procs=cores)
+    dt = time.perf_counter() - t0
+    return {"plans": plans, "cores": cores, "wall_s": dt, "core_s": dt * min(cores, len(plans))}
+
+
 def run_ours(args) -> None:
     import torch
     from paper_2504_17096_b200 import binding as B
     from paper_2504_17096_b200 import build as cuda_build
+    from paper_2504_17096_b200 import sharding
     if cuda_build.is_stale():                    # compile the CUDA library if it is missing or out of date
         if int(os.environ.get("LOCAL_RANK", "0")) == 0:
             cuda_build.build()
@@ -338,9 +464,11 @@ def run_ours(args) -> None:
             dist.init_process_group(backend)
 
     w = workload_by_name(args.workload, args.only_p)
-    # independent problems: every rank searches the whole space for its own availability snapshot
+    # one space split over the ranks by flat-index range, unless asked for replicas (or the workload's budget
+    # rule needs the cheapest plan of the whole space first)
+    split = world > 1 and not args.replicas and not w.budget_factor_over_cheapest > 0
     avail = w.avail.copy()
-    if rank:
+    if rank and not split:               # replicas: every rank searches the whole space for its own snapshot
         rng = W.SplitMix64(0xA7A11 + rank)
         for idx in np.ndindex(avail.shape):
             avail[idx] = min(65535, max(0, int(avail[idx]) + rng.randint(0, 8) - 4))
@@ -349,6 +477,7 @@ def run_ours(args) -> None:
     space = B.make_space(w)
     obj = B.make_objective(w, flags=B.FLAG_EVAL_ALL)
     n = B.sailor_space_size(ctx, space)
+    lo, hi = (sharding.split_by_cost(sharding.subspace_costs(w), world, rank) if split else (0, n))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than the 126 MB L2
 
     def barrier():
@@ -356,44 +485,75 @@ def run_ours(args) -> None:
             dist.barrier()
         torch.cuda.synchronize()
 
+    def search():
+        return B.sailor_plan_range(ctx, space, obj, lo, hi, K_TOP) if split else B.sailor_plan(ctx, space, obj, K_TOP)
+
+    def merged(res, st):
+        """The job's result: this rank's list, or the lists of all ranges merged by (score, flat)."""
+        if not split:
+            return [(r.score, int(r.flat)) for r in res], int(st.n_total)
+        counts = {"n_total": int(st.n_total), "n_feasible": int(st.n_feasible), "min_feasible_cost": st.min_feasible_cost}
+        top, tot = sharding.gather_and_merge([(r.score, int(r.flat)) for r in res], counts, K_TOP)
+        return top, tot["n_total"]
+
+    split_check = None
+    if split:      # the split must reproduce a single search: checked on a small workload before anything is timed
+        small = W.config1()
+        c1 = B.sailor_create(small, local, stream.cuda_stream)
+        try:
+            B.sailor_set_availability(c1, small.avail)
+            sp1, ob1 = B.make_space(small), B.make_objective(small)
+            a, b = sharding.split_range(B.sailor_space_size(c1, sp1), world, rank)
+            part, pst = B.sailor_plan_range(c1, sp1, ob1, a, b, K_TOP)
+            top, _ = sharding.gather_and_merge([(r.score, int(r.flat)) for r in part], {"n_total": int(pst.n_total)}, K_TOP)
+            whole, _ = B.sailor_plan(c1, sp1, ob1, K_TOP)
+            split_check = top == [(r.score, int(r.flat)) for r in whole]
+            assert split_check, "the merged per-range lists differ from the single search"
+        finally:
+            B.sailor_destroy(c1)
+
     B.sailor_set_availability(ctx, avail)
     for _ in range(args.warmup):
-        B.sailor_plan(ctx, space, obj, K_TOP)
+        search()
 
     # ---- device-timed region: inputs resident, CUDA events on the launching stream ------------
     barrier()
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(local).uuid)) if rank == 0 else None
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    kernel_ms, launches, best = [], 0, None
+    kernel_ms, launches, res, st = [], 0, [], None
     for a, b in ev:
         flush.fill_(1)                                   # L2 flush between timed iterations
         a.record(stream)
-        res, st = B.sailor_plan(ctx, space, obj, K_TOP)
+        res, st = search()
         b.record(stream)
         kernel_ms.append(st.kernel_ms)
         launches += st.n_launches
-        best = res[0] if res else None
     barrier()
-    clocks = sampler.stop() if sampler else None
     step_ms = [a.elapsed_time(b) for a, b in ev]
     dev_s = sum(step_ms) / 1e3
+    top, n_seen = merged(res, st)
 
-    # ---- end to end: the public call with host buffers (availability up, results down) ----------
+    # ---- end to end: the public call with host buffers (availability up, results down; with several ranks
+    # ---- also the exchange and merge of the per-range lists) -----------------------------------------
     barrier()
     t0 = time.perf_counter()
     for _ in range(args.steps):
         B.sailor_set_availability(ctx, avail)
-        res, st = B.sailor_plan(ctx, space, obj, K_TOP)
+        res, st = search()
+        merged(res, st)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
+    clocks = sampler.stop() if sampler else None          # samples of both timed regions
     h2d = int(avail.size * 2)
-    d2h = int(K_TOP * 120 + 80)
+    d2h = int(K_TOP * 120 + 96)
 
     times = torch.tensor([dev_s, e2e_s], dtype=torch.float64, device="cuda" if backend == "nccl" else "cpu")
     if dist is not None:
         dist.all_reduce(times, op=dist.ReduceOp.MAX)
     dev_s, e2e_s = (float(x) for x in times.cpu())
-    total = n * args.steps * world
+    total = n * args.steps * (1 if split else world)
+    if split:
+        assert n_seen == n, "the ranges do not add up to the space"
 
     if rank == 0:
         ops = mean_ops_per_candidate(w)
@@ -404,26 +564,39 @@ def run_ours(args) -> None:
                 peaks = json.load(f)
         except OSError:
             pass
+        # the ceiling: what the device really issues, measured now with three instruction streams
+        rates = B.sailor_measure_issue_rates(local, stream.cuda_stream, 5)
         sm_max = float(peaks.get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0)
-        peak = SM_COUNT * ISSUE_PER_SM * LANES * sm_max * 1e6 / 1e12
-        achieved = ops * n / k_s / 1e12
-        # counters of one plan_kernel launch on this workload, from the ncu capture summarised in
-        # profiles folder (valid for the kernel as committed with that summary)
-        captured = NCU_PER_LAUNCH.get(w.name)
-        issued = None
-        if captured:
-            rate = captured["warp_inst"] / k_s
-            issued = {"warp_inst_per_launch": captured["warp_inst"], "warp_inst_per_s": rate,
-                      "frac_of_issue_peak": rate / (SM_COUNT * ISSUE_PER_SM * sm_max * 1e6),
-                      "lane_inst_per_candidate": captured["warp_inst"] * LANES / n}
-        roofline = {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "Tlane-op/s",
-                    "frac": achieved / peak, "traffic": captured["dram_bytes"] if captured else None,
-                    "issued": issued,
-                    "note": "algorithmic lane-ops (40 + 35 P per candidate) / kernel time; peak = 148 SMs x 4 issue "
-                            "slots x 32 lanes x max SM clock; prefix reuse executes fewer instructions than the "
-                            "algorithmic count, see profiles/ for issued-instruction utilisation",
-                    "kernel_ms": 1e3 * k_s, "ops_per_candidate": ops}
-        cpu = None
+        units_x_clock = rates.sm_count * ISSUE_PER_SM * sm_max * 1e6                 # warp-instructions/s
+        counters, why_not = (read_counters(w.name) if world == 1 else (None, "counters are of a whole-space launch"))
+        roofline = {"bound": "alu", "unit": "warp-inst/s", "achieved": None, "peak": rates.ffma_warp_inst_per_s,
+                    "frac": None, "traffic": None,
+                    "peak_kind": "measured: FP32 multiply-add stream, 8 chains per thread, 4 x 256 threads per SM",
+                    "peak_units_x_clock": units_x_clock, "frac_of_units_x_clock": None,
+                    "issue_peak_measured": {"ffma": rates.ffma_warp_inst_per_s, "imad": rates.imad_warp_inst_per_s,
+                                            "dadd": rates.dadd_warp_inst_per_s,
+                                            "per_sm_per_cycle_at_max_clock": {
+                                                k: v / (rates.sm_count * sm_max * 1e6) for k, v in
+                                                (("ffma", rates.ffma_warp_inst_per_s), ("imad", rates.imad_warp_inst_per_s),
+                                                 ("dadd", rates.dadd_warp_inst_per_s))}},
+                    "fp64_achieved": None, "fp64_peak": rates.dadd_warp_inst_per_s, "fp64_frac": None,
+                    "lane_inst_per_candidate": None, "counters": why_not or os.path.relpath(COUNTER_FILE, ROOT),
+                    "algorithmic_over_peak": ops * n / k_s / (units_x_clock * LANES),
+                    "ops_per_candidate_model": ops, "kernel_ms": 1e3 * k_s,
+                    "note": "achieved = warp-instructions one plan_kernel launch executes (ncu smsp__inst_executed.sum, "
+                            "stored with a hash of the kernel sources) / this run's kernel time; fp64_* = the same for the "
+                            "FP64 pipe against the FP64-add stream; algorithmic_over_peak = (40 + 35 P lane-ops per "
+                            "candidate) / kernel time over units x clock: above 1 because prefix sums and run-length "
+                            "segments remove most of the stage-by-stage work"}
+        if counters:
+            inst, fp64 = counters["smsp__inst_executed.sum"], counters["smsp__inst_executed_pipe_fp64.sum"]
+            roofline.update(achieved=inst / k_s, frac=inst / k_s / rates.ffma_warp_inst_per_s,
+                            frac_of_units_x_clock=inst / k_s / units_x_clock,
+                            traffic=counters["dram__bytes_read.sum"] + counters["dram__bytes_write.sum"],
+                            fp64_achieved=fp64 / k_s, fp64_frac=fp64 / k_s / rates.dadd_warp_inst_per_s,
+                            lane_inst_per_candidate=inst * LANES / n,
+                            pipe_share={k.split("pipe_")[1].split(".")[0]: counters[k] / inst for k in counters if "pipe_" in k})
+        cpu, oracle4 = None, None
         if world == 1 and not args.no_cpu:
             from oracle.binding import Oracle
             o = Oracle(w)
@@ -434,7 +607,9 @@ def run_ours(args) -> None:
             dt = time.perf_counter() - t0
             cpu = {"value": counts["n_total"] / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
                    "sample": f"every {stride}-th flat index of {w.name}: {counts['n_total']} candidates in {dt:.1f} s"}
-        aux = aux_measurements(B, torch, local) if (world == 1 and not args.no_aux) else None
+            if not args.no_aux:
+                oracle4 = oracle_cfg4_plans()
+        aux = aux_measurements(B, torch, local, oracle4) if (world == 1 and not args.no_aux) else None
         if aux is not None:
             # the same workload the way a planner would call it: memory/availability pruning on
             ob = B.make_objective(w)
@@ -446,18 +621,23 @@ def run_ours(args) -> None:
                 ts.append(time.perf_counter() - t0)
             aux[args.workload + "_default_mode"] = {"candidates": int(stp.n_total), "search_s": statistics.median(ts),
                                                     "kernel_ms": stp.kernel_ms, "feasible": int(stp.n_feasible),
+                                                    "cold": cold_search(B, torch, local, w),
                                                     "pruning_modes": pruning_modes(B, ctx, w, space),
                                                     "dp": dp_search(B, ctx, w, space)}
+            aux[args.workload + "_every_candidate"] = {"cold": cold_search(B, torch, local, w, B.FLAG_EVAL_ALL)}
         line = {"metric": METRIC, "value": total / dev_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": 1e3 * dev_s / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                "scaling": "strong" if split else "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
                 "config": {"workload": w.name, "candidates": n, "top_k": K_TOP, "mode": "every candidate evaluated",
                            "objective": w.objective, "l2": "flushed between timed iterations (256 MiB write)",
-                           "parallelism": f"{world} independent searches" if world > 1 else "1 gpu"},
+                           "parallelism": ("1 gpu" if world == 1 else
+                                           f"one space split into {world} flat-index ranges of equal estimated cost, "
+                                           f"top-{K_TOP} lists merged" if split else f"{world} independent searches"),
+                           "split_check": split_check},
                 "e2e": {"value": total / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                        "search_s": e2e_s / args.steps},
+                        "search_s": e2e_s / args.steps, "h2d_ms": st.h2d_ms, "d2h_ms": st.d2h_ms},
                 "gpu_launches": launches, "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu,
-                "best": None if best is None else {"flat": int(best.flat), "t_iter": best.t_iter, "cost": best.cost},
+                "best": None if not top else {"flat": top[0][1], "score": top[0][0]},
                 "aux": aux}
         print(json.dumps(line), flush=True)
     B.sailor_destroy(ctx)
@@ -469,7 +649,7 @@ def run_ours(args) -> None:
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="cfg5")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
@@ -477,15 +657,22 @@ def main() -> None:
     ap.add_argument("--ref-sample", type=int, default=4_000_000, help="candidates per reference step")
     ap.add_argument("--only-p", type=int, nargs="*", default=None, help="keep only these pipeline depths")
     ap.add_argument("--dp-only", action="store_true", help="run only the dynamic-programming search (for profiling)")
+    ap.add_argument("--sim-only", action="store_true", help="run only the explicit-batch kernels (for profiling)")
     ap.add_argument("--dp-workspace-gib", type=float, default=8.0, help="table workspace of --dp-only")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-aux", action="store_true")
+    ap.add_argument("--replicas", action="store_true", help="N > 1: every rank searches the whole space (weak scaling)")
+    ap.add_argument("--write-counters", default=None, metavar="NCU_CSV", help="write the counter file from an ncu --csv log")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
-    if args.impl == "reference":
+    if args.write_counters:
+        write_counters(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.dp_only:
         run_dp_only(args)
+    elif args.sim_only:
+        run_sim_only(args)
     else:
         run_ours(args)
 

@@ -33,7 +33,9 @@
  *           (double)(2 * N_b * D * p2p_bytes[mbs]) * egress[z_i][z_{i+1}]  left to right
  *   C_iter= rate * T_iter + C_comm                                      (Sec. 4.3, Sec. 4.2.3)
  *
- * Threading.  A context is not thread-safe; use one context per host thread.
+ * Threading.  A context is not thread-safe; use one context per host thread.  Different
+ * contexts may be used from different threads at the same time (the library's few process-wide
+ * flags are atomic).  The library reads no environment variable and keeps no other global state.
  */
 #ifndef SAILOR_H
 #define SAILOR_H
@@ -63,15 +65,17 @@ extern "C" {
 #define SAILOR_E_RANGE    (-2)  /* an index or a size is outside a table or a limit above    */
 #define SAILOR_E_CUDA     (-3)  /* a CUDA call failed; see sailor_last_cuda_error            */
 #define SAILOR_E_NOMEM    (-4)  /* host or device allocation failed                          */
-#define SAILOR_E_DEVICE   (-5)  /* a kernel reported an internal fault (bounded wait ran out) */
+#define SAILOR_E_DEVICE   (-5)  /* a kernel reported an internal fault (bounded wait ran out)
+                                   during THIS call; the flag is cleared with the call, the
+                                   context stays usable and the next call starts clean        */
 
 /* ---- status bits of one simulated plan ------------------------------------------------- */
 #define SAILOR_ST_INVALID          1u   /* gbs % (D*mbs) != 0, tp > gpus_per_node, heads % tp != 0 (H1) */
 #define SAILOR_ST_OVER_AVAIL       2u   /* needs more GPUs of some (zone, type) than available           */
 #define SAILOR_ST_OOM              4u   /* some stage's peak memory exceeds its GPU's capacity (H2)     */
-#define SAILOR_ST_OVER_BUDGET      8u   /* C_iter > budget                                              */
-#define SAILOR_ST_UNDER_THROUGHPUT 16u  /* 1 / T_iter < min_iters_per_s                                 */
 #define SAILOR_ST_BAD_RECORD       32u  /* device-side record failed its bounds checks; nothing read    */
+/* A budget or a throughput floor belongs to a search, not to a plan: sailor_simulate knows neither, so
+ * no status bit exists for them; a search counts such candidates in sailor_stats.n_over_constraint. */
 
 /* ---- inputs --------------------------------------------------------------------------- */
 
@@ -227,6 +231,9 @@ typedef struct sailor_stats {
     uint64_t n_skipped;         /* candidates of configurations early termination never reached */
     uint32_t n_configs;         /* configurations (P, mbs, tp, rc, D) of the space           */
     uint32_t n_configs_evaluated;   /* of which looked at (all of them without DEGREE_ORDER) */
+    float    h2d_ms;            /* device time of the last availability upload (CUDA events
+                                   around the copy in sailor_set_availability)               */
+    float    d2h_ms;            /* device time of this call's result read-back               */
 } sailor_stats;
 
 typedef struct sailor_ctx sailor_ctx;     /* opaque; owns device copies of the tables       */
@@ -383,7 +390,7 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
  * sequences.  `value` sums the stage times from the last stage backwards; t_iter, cost and
  * peak_mem of a result are the simulator's figures for the written-out plan (stage order), equal
  * to value up to rounding.  The objective is iteration time (o->kind must be MAX_THROUGHPUT, no
- * flags, no budget factor).  A budget or a minimum throughput in `o` is checked on the plan the
+ * flags other than SAILOR_DP_FLAG_*, no budget factor).  A budget or a minimum throughput in `o` is checked on the plan the
  * recursion returns for a problem, by the simulator's cost and time (Sec. 4.2: a configuration
  * counts only when it is within the constraint); a problem whose plan fails it drops out.  The
  * straggler-guessing budget loop of Sec. 4.2.3, which steers the recursion itself by the remaining
@@ -393,6 +400,17 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
  * stages per type already placed in that zone; a type with room for all P stages in a zone is not
  * counted there), filled from the last stage to the first, one launch per stage for all problems
  * of a batch together; batches are cut so that the tables fit `workspace_bytes`. */
+/* How sailor_plan_dp lays out and walks its tables, in sailor_objective.flags.  The results do not
+ * depend on them; they exist so that every code path can be selected (and tested) through this
+ * interface.  Index of a zone position's count vectors: the smaller of the two ways (default), mixed
+ * radix whenever it fits (DENSE), by rank whenever it fits (COMPACT).  Threads of a stage's launch: one
+ * per reachable count vector for all its types (default), one per reachable count vector and type
+ * (BY_TYPE), one per table entry (BY_ENTRY). */
+#define SAILOR_DP_FLAG_INDEX_DENSE    0x100u
+#define SAILOR_DP_FLAG_INDEX_COMPACT  0x200u
+#define SAILOR_DP_FLAG_ENUM_BY_TYPE   0x400u
+#define SAILOR_DP_FLAG_ENUM_BY_ENTRY  0x800u
+
 typedef struct sailor_zone_order {
     uint8_t n;                          /* 1 .. SAILOR_Z_MAX zones, each at most once                */
     uint8_t zone[SAILOR_Z_MAX];
@@ -435,6 +453,26 @@ typedef struct sailor_dp_stats {
 int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders, uint32_t n_orders,
                    const sailor_objective* o, uint64_t workspace_bytes, uint32_t k, sailor_dp_result* topk,
                    uint32_t* n_found, sailor_dp_stats* stats);
+
+/* ---- sustained issue rates of the device (a measurement, not part of the method) -------------------
+ *
+ * The search is bound by instruction issue, so its throughput is judged against the rate at which
+ * the device really issues instructions.  This call times three instruction streams (FP32 fused
+ * multiply-add, 32-bit integer multiply-add, FP64 add; eight independent chains per thread, four
+ * blocks of 256 threads per SM, about a millisecond each, best of `repeats` runs) with CUDA events on
+ * `cuda_stream` and reports warp-instructions per second for each.  It allocates and frees 8 bytes of
+ * device memory and synchronises the stream.  Errors: E_ARG (null, repeats == 0), E_CUDA (no context
+ * to record the code in: the return value is all there is). */
+typedef struct sailor_issue_rates {
+    double   ffma_warp_inst_per_s;      /* FP32 pipe stream: what the four schedulers of an SM sustain  */
+    double   imad_warp_inst_per_s;      /* integer multiply-add stream                                   */
+    double   dadd_warp_inst_per_s;      /* FP64 pipe stream                                              */
+    float    ffma_ms, imad_ms, dadd_ms; /* duration of the best run of each stream                       */
+    uint32_t sm_count;
+    uint64_t warp_inst_per_run;         /* stream instructions one run of a kernel executes              */
+} sailor_issue_rates;
+
+int sailor_measure_issue_rates(int cuda_device, void* cuda_stream, uint32_t repeats, sailor_issue_rates* out);
 
 const char* sailor_strerror(int code);
 int sailor_last_cuda_error(const sailor_ctx* ctx);   /* cudaError_t of the last E_CUDA      */

@@ -20,7 +20,7 @@ _HDR = os.path.join(_HERE, "sailor_oracle.h")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
 STAGES_MAX = 128
-ST_INVALID, ST_OVER_AVAIL, ST_OOM, ST_OVER_BUDGET, ST_UNDER_THROUGHPUT = 1, 2, 4, 8, 16
+ST_INVALID, ST_OVER_AVAIL, ST_OOM = 1, 2, 4
 
 
 def build(force: bool = False) -> str:
@@ -111,6 +111,12 @@ class OrcDpResult(C.Structure):
     _fields_ = [("found", C.c_int32), ("_pad", C.c_uint32), ("value", C.c_double), ("n_states", C.c_uint64),
                 ("plan", OrcPlan)]
 
+
+class OrcDpBudgetResult(C.Structure):
+    _fields_ = [("found", C.c_int32), ("_pad", C.c_uint32), ("value", C.c_double), ("charged_cost", C.c_double),
+                ("n_states", C.c_uint64), ("plan", OrcPlan)]
+
+
 GROUPS_MAX = 4
 
 
@@ -155,6 +161,9 @@ def lib():
         L.orc_search_pruned.restype = C.c_int32
         L.orc_solve_dp.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcDpProblem), C.c_int, C.POINTER(OrcDpResult)]
         L.orc_solve_dp.restype = C.c_int
+        L.orc_solve_dp_budget.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcDpProblem), C.c_double,
+                                          C.POINTER(OrcDpBudgetResult)]
+        L.orc_solve_dp_budget.restype = C.c_int
         L.orc_simulate_mixed.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedPlan), C.POINTER(OrcOut)]
         L.orc_simulate_mixed.restype = None
         L.orc_simulate_mixed_batch.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedPlan), C.c_uint64,
@@ -350,6 +359,23 @@ class Oracle:
         plan = OrcPlan.from_buffer_copy(out.plan)
         return {"value": out.value, "types": list(plan.type[:P]), "zones": list(plan.zone[:P]), "plan": plan,
                 "n_states": int(out.n_states)}
+
+    def solve_dp_budget(self, P: int, mbs_idx: int, tp_idx: int, rc: int, D: int, zone_list: Sequence[int],
+                        limit: float) -> Optional[dict]:
+        """The recursion under a cost limit (Sec. 4.2.3: stages charged by the assumed straggler, re-solved when
+        the straggler turns out different); None when no plan is within the limit."""
+        pb = OrcDpProblem()
+        pb.P, pb.mbs_idx, pb.tp_idx, pb.rc, pb.D, pb.n_zones_used = P, mbs_idx, tp_idx, rc, D, len(zone_list)
+        for j, z in enumerate(zone_list):
+            pb.zone_list[j] = int(z)
+        out = OrcDpBudgetResult()
+        if lib().orc_solve_dp_budget(C.byref(self.inputs), C.byref(pb), float(limit), C.byref(out)) != 0:
+            raise ValueError("problem beyond the oracle's limits")
+        if not out.found:
+            return None
+        plan = OrcPlan.from_buffer_copy(out.plan)
+        return {"value": out.value, "charged_cost": out.charged_cost, "types": list(plan.type[:P]),
+                "zones": list(plan.zone[:P]), "plan": plan, "n_states": int(out.n_states)}
 
     def plan(self, k: int, *, lo: int = 0, hi: Optional[int] = None):
         """The workload's own objective, with the cheapest-feasible budget rule when it has one:

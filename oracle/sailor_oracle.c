@@ -679,6 +679,129 @@ int orc_solve_dp(const orc_inputs* in, const orc_dp_problem* pb, int use_memo, o
     return 0;
 }
 
+/* ---- the recursion under a cost limit (Sec. 4.2.3) ---------------------------------------------------- */
+
+typedef struct dpb_val {
+    int found;
+    double sum, mx, sy, up;              /* as dp_val */
+    double cost;                         /* what stages i.. were charged */
+    uint8_t type[ORC_STAGES_MAX];        /* types of stages i.. of the kept plan, at their own positions */
+} dpb_val;
+
+static double dpb_value(const dp_ctx* c, const dpb_val* v) {
+    return ((v->sum + (double)c->n_b * v->mx) + v->sy) + v->up;
+}
+
+/* best plan within `limit` for stages i.. given that stage i runs on type g in zone position zp and `used`
+ * (which includes stage i) describes that zone */
+static dpb_val solve_suffix_budget(dp_ctx* c, uint32_t i, uint32_t g, uint32_t zp, const uint8_t* used, double limit) {
+    const orc_inputs* in = c->in;
+    const uint32_t P = c->pb->P, z = c->pb->zone_list[zp], D = c->pb->D;
+    dpb_val best; memset(&best, 0, sizeof(best));
+    if (!c->fits[i][g]) return best;
+    c->n_states++;
+    const double sync = dp_sync(in, g, z, c->tp, D, c->params[i]);
+    const double rate = (double)(D * c->tp) * (in->price_per_hour[z * c->T + g] / 3600.0);
+    if (i == P - 1) {
+        const double t = c->fb[i][g];                        /* the last stage sends nothing and is its own straggler */
+        const double charge = rate * ((double)c->n_b * t);
+        if (charge <= limit) {
+            best.found = 1;
+            best.sum = t; best.mx = t; best.sy = sync; best.up = c->upd[i][g];
+            best.cost = charge;
+            best.type[i] = (uint8_t)g;
+        }
+        return best;
+    }
+    for (uint32_t g2 = 0; g2 < c->T; ++g2) {
+        if (!c->fits[i + 1][g2]) continue;
+        const int zp2 = first_fit(c, zp, used, g2);
+        if (zp2 < 0) continue;
+        uint8_t used2[ORC_DP_T_MAX];
+        for (uint32_t t = 0; t < c->T; ++t) used2[t] = ((uint32_t)zp2 == zp) ? used[t] : 0;
+        used2[g2]++;
+        const uint32_t z2 = c->pb->zone_list[zp2];
+        const double cmsg = dp_p2p(in, g, z, g2, z2, c->tp, D, c->msg);
+        const double t = c->fb[i][g] + 2.0 * cmsg;
+        const double comm = (z2 != z) ? (double)(2 * c->n_b * (uint64_t)D * c->msg) * in->egress[z * in->n_zones + z2] : 0.0;
+        double assumed = t;                                  /* first: this stage is the straggler */
+        for (;;) {
+            const double charge = rate * ((double)c->n_b * assumed) + comm;
+            const double rest = limit - charge;
+            if (!(rest > 0.0)) break;
+            const dpb_val nxt = solve_suffix_budget(c, i + 1, g2, (uint32_t)zp2, used2, rest);
+            if (!nxt.found) break;
+            if (nxt.mx <= assumed) {                         /* the assumption holds */
+                const double all = charge + nxt.cost;
+                if (all <= limit) {
+                    dpb_val cand = nxt;                      /* keeps the types of the later stages */
+                    cand.found = 1;
+                    cand.sum = t + nxt.sum;
+                    cand.mx = max_f64(t, nxt.mx);
+                    cand.sy = max_f64(sync, nxt.sy);
+                    cand.up = max_f64(c->upd[i][g], nxt.up);
+                    cand.cost = all;
+                    cand.type[i] = (uint8_t)g;
+                    if (!best.found || dpb_value(c, &cand) < dpb_value(c, &best)) best = cand;
+                }
+                break;
+            }
+            assumed = nxt.mx;                                /* charge again with the straggler that was found */
+        }
+    }
+    return best;
+}
+
+int orc_solve_dp_budget(const orc_inputs* in, const orc_dp_problem* pb, double limit, orc_dp_budget_result* out) {
+    memset(out, 0, sizeof(*out));
+    const uint32_t P = pb->P, T = in->n_types;
+    if (P < 1 || P > ORC_STAGES_MAX || T > ORC_DP_T_MAX || pb->n_zones_used < 1 || pb->n_zones_used > 16 || pb->D < 1) return -1;
+    const uint64_t mbs = in->mbs_values[pb->mbs_idx];
+    const uint32_t tp = in->tp_values[pb->tp_idx];
+    if (in->gbs % ((uint64_t)pb->D * mbs) != 0 || in->heads % tp != 0) return 0;      /* no valid plan in this problem */
+    dp_ctx* c = (dp_ctx*)calloc(1, sizeof(dp_ctx));
+    c->in = in; c->pb = pb; c->T = T; c->tp = tp; c->need = pb->D * tp;
+    c->n_b = in->gbs / ((uint64_t)pb->D * mbs);
+    c->msg = in->p2p_bytes[pb->mbs_idx];
+    for (uint32_t i = 0; i < P; ++i)
+        for (uint32_t g = 0; g < T; ++g) {
+            uint64_t par;
+            dp_stage(in, P, i, g, pb->tp_idx, pb->mbs_idx, pb->rc, c->n_b, &c->fb[i][g], &c->upd[i][g], &par, &c->fits[i][g]);
+            c->params[i] = par;
+        }
+    dpb_val best; memset(&best, 0, sizeof(best));
+    const uint8_t nothing[ORC_DP_T_MAX] = {0};
+    for (uint32_t g = 0; g < T; ++g) {                       /* stage 0: every type, first fit from the first zone */
+        const int zp = first_fit(c, 0, nothing, g);
+        if (zp < 0) continue;
+        uint8_t used[ORC_DP_T_MAX] = {0};
+        used[g] = 1;
+        const dpb_val v = solve_suffix_budget(c, 0, g, (uint32_t)zp, used, limit);
+        if (!v.found) continue;
+        if (!best.found || dpb_value(c, &v) < dpb_value(c, &best)) best = v;
+    }
+    out->n_states = c->n_states;
+    if (best.found) {
+        out->found = 1;
+        out->value = dpb_value(c, &best);
+        out->charged_cost = best.cost;
+        orc_plan* pl = &out->plan;
+        pl->P = P; pl->mbs_idx = pb->mbs_idx; pl->rc = pb->rc; pl->D = pb->D;
+        uint8_t used[ORC_DP_T_MAX] = {0};
+        uint32_t zp = 0;
+        for (uint32_t i = 0; i < P; ++i) {                   /* zones by first fit, as the recursion placed them */
+            const uint32_t g = best.type[i];
+            const int zp2 = first_fit(c, zp, used, g);
+            if ((uint32_t)zp2 != zp) memset(used, 0, sizeof(used));
+            used[g]++;
+            zp = (uint32_t)zp2;
+            pl->type[i] = g; pl->zone[i] = pb->zone_list[zp]; pl->tp_idx[i] = pb->tp_idx;
+        }
+    }
+    free(c);
+    return 0;
+}
+
 /* ---- plans whose stages mix GPU types among their replicas (Sec. 4.2, Sec. 4.3, Sec. 4.4) -----------
  *
  * Stage i has D replicas in one zone (H5), given as groups: `count` replicas on one GPU type with one

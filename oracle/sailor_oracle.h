@@ -34,8 +34,6 @@
 #define ORC_INVALID 1u
 #define ORC_OVER_AVAIL 2u
 #define ORC_OOM 4u
-#define ORC_OVER_BUDGET 8u
-#define ORC_UNDER_THROUGHPUT 16u
 
 /* objective kinds: what is minimised */
 #define ORC_OBJ_TIME 0           /* maximise throughput            */
@@ -216,6 +214,31 @@ typedef struct orc_dp_result {
 
 /* returns 0, or -1 for sizes beyond the limits; use_memo = 0 is the plain recursion */
 int orc_solve_dp(const orc_inputs* in, const orc_dp_problem* pb, int use_memo, orc_dp_result* out);
+
+/* The same recursion under a cost limit (Sec. 4.2.3, "Adding a monetary cost constraint", and the second half of
+ * the listing).  A stage is charged by the simplified cost of that section:
+ *     C_i = rate_i * (N_b * t_straggler) + C_comm_i
+ * rate_i = (double)(D * tp) * (price_per_hour / 3600) of its GPUs, C_comm_i = the transfer cost of its message
+ * to the next stage when that crosses zones ((double)(2 * N_b * D * p2p_bytes) * egress), and t_straggler the
+ * ASSUMED straggler: first the stage's own time; the stages after it are solved with what is left of the limit,
+ * C_rem = C_cur - C_i; when their straggler turns out slower than the assumed one, the stage is charged again
+ * with that straggler and they are solved again with the smaller remainder, until the assumption holds
+ * (their straggler <= the assumed one: then the plan counts if C_i + their cost <= C_cur), nothing is left
+ * (C_rem <= 0) or they have no plan.  The last stage is its own straggler and counts if its charge is within
+ * its limit.  Candidates combine and compare exactly as in orc_solve_dp.  The remaining limit is an argument of
+ * the recursion, so nothing is remembered between calls here (a state reached with two different remainders is
+ * solved twice); with limit = +infinity the result is orc_solve_dp's bit for bit.
+ * charged_cost is the sum of the charges of the kept plan; n_states counts the calls of the recursion. */
+typedef struct orc_dp_budget_result {
+    int32_t found;
+    uint32_t _pad;
+    double value;
+    double charged_cost;
+    uint64_t n_states;
+    orc_plan plan;
+} orc_dp_budget_result;
+
+int orc_solve_dp_budget(const orc_inputs* in, const orc_dp_problem* pb, double limit, orc_dp_budget_result* out);
 
 
 /* ---- plans whose stages mix GPU types among their replicas ------------------------------------------

@@ -14,13 +14,15 @@ LIB_PATH = os.path.join(HERE, "libsailor_b200.so")
 
 KINDS, T_MAX, Z_MAX, TP_MAX, MBS_MAX, P_MAX, RUN_MAX, SEG_MAX, K_MAX, NP_MAX, ND_MAX = 3, 8, 8, 8, 16, 96, 16, 4, 32, 32, 32
 OK, E_ARG, E_RANGE, E_CUDA, E_NOMEM, E_DEVICE = 0, -1, -2, -3, -4, -5
-ST_INVALID, ST_OVER_AVAIL, ST_OOM, ST_OVER_BUDGET, ST_UNDER_THROUGHPUT, ST_BAD_RECORD = 1, 2, 4, 8, 16, 32
+ST_INVALID, ST_OVER_AVAIL, ST_OOM, ST_BAD_RECORD = 1, 2, 4, 32
 OBJ_MAX_THROUGHPUT, OBJ_MIN_COST, OBJ_MAX_THROUGHPUT_PER_USD = 0, 1, 2
 FLAG_EVAL_ALL, FLAG_DEGREE_ORDER, FLAG_MIN_TP_ONLY = 1, 2, 4
+DP_FLAG_INDEX_DENSE, DP_FLAG_INDEX_COMPACT, DP_FLAG_ENUM_BY_TYPE, DP_FLAG_ENUM_BY_ENTRY = 0x100, 0x200, 0x400, 0x800
 
 EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
            "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_plan_noalloc",
-           "sailor_plan_dp", "sailor_simulate_mixed", "sailor_strerror", "sailor_last_cuda_error")
+           "sailor_plan_dp", "sailor_simulate_mixed", "sailor_measure_issue_rates", "sailor_strerror",
+           "sailor_last_cuda_error")
 
 _dp, _u64p, _u32p, _u16p = C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.POINTER(C.c_uint16)
 
@@ -76,7 +78,14 @@ class Stats(C.Structure):
                 ("n_over_avail", C.c_uint64), ("n_over_constraint", C.c_uint64), ("n_feasible", C.c_uint64),
                 ("budget_used", C.c_double), ("min_feasible_cost", C.c_double), ("kernel_ms", C.c_float),
                 ("n_launches", C.c_uint32), ("n_pruned_tp", C.c_uint64), ("n_skipped", C.c_uint64),
-                ("n_configs", C.c_uint32), ("n_configs_evaluated", C.c_uint32)]
+                ("n_configs", C.c_uint32), ("n_configs_evaluated", C.c_uint32), ("h2d_ms", C.c_float),
+                ("d2h_ms", C.c_float)]
+
+
+class IssueRates(C.Structure):
+    _fields_ = [("ffma_warp_inst_per_s", C.c_double), ("imad_warp_inst_per_s", C.c_double),
+                ("dadd_warp_inst_per_s", C.c_double), ("ffma_ms", C.c_float), ("imad_ms", C.c_float),
+                ("dadd_ms", C.c_float), ("sm_count", C.c_uint32), ("warp_inst_per_run", C.c_uint64)]
 
 
 class ZoneOrder(C.Structure):
@@ -99,7 +108,7 @@ class DpStats(C.Structure):
 
 assert C.sizeof(PlanRec) == 72 and C.sizeof(Result) == 120 and C.sizeof(Space) == 152
 assert C.sizeof(ZoneOrder) == 12 and C.sizeof(DpResult) == 248 and C.sizeof(DpStats) == 56
-assert C.sizeof(Objective) == 32 and C.sizeof(Stats) == 96
+assert C.sizeof(Objective) == 32 and C.sizeof(Stats) == 104
 
 # numpy view of an array of plan records (same 72-byte layout)
 RUN_DTYPE = np.dtype([("type", "u1"), ("zone", "u1"), ("tp_idx", "u1"), ("n_stages", "u1")])
@@ -172,6 +181,7 @@ def load() -> C.CDLL:
     L.sailor_plan_noalloc.argtypes = L.sailor_plan.argtypes
     L.sailor_plan_dp.argtypes = [vp, C.POINTER(Space), C.POINTER(ZoneOrder), C.c_uint32, C.POINTER(Objective),
                                  C.c_uint64, C.c_uint32, C.POINTER(DpResult), _u32p, C.POINTER(DpStats)]
+    L.sailor_measure_issue_rates.argtypes = [C.c_int, vp, C.c_uint32, C.POINTER(IssueRates)]
     L.sailor_strerror.argtypes = [C.c_int]
     L.sailor_strerror.restype = C.c_char_p
     L.sailor_last_cuda_error.argtypes = [vp]
@@ -357,13 +367,24 @@ def all_zone_orders(n_zones: int, max_len: Optional[int] = None):
     return [list(p) for n in range(1, max_len + 1) for p in itertools.permutations(range(n_zones), n)]
 
 
+def sailor_measure_issue_rates(device: int = 0, stream: int = 0, repeats: int = 5) -> IssueRates:
+    """Sustained warp-instructions per second of an FP32 multiply-add, an integer multiply-add and an FP64 add
+    stream on the device (CUDA events, best of `repeats`)."""
+    r = IssueRates()
+    _check(load().sailor_measure_issue_rates(device, C.c_void_p(stream), repeats, C.byref(r)), "sailor_measure_issue_rates")
+    return r
+
+
+dp_default_flags = 0      # SAILOR_DP_FLAG_* that sailor_plan_dp passes when the caller gives no objective
+
+
 def sailor_plan_dp(ctx, space: Space, zone_orders, k: int, workspace_bytes: int = 0, *, budget: float = 0.0,
                    min_rate: float = 0.0, obj: Optional[Objective] = None):
     """Per-stage GPU types by dynamic programming for every configuration of the space and every zone
     order (a list of zone lists): the k best plans by the recursion's value among those within the
     budget / minimum throughput, and the statistics."""
     if obj is None:
-        obj = Objective(OBJ_MAX_THROUGHPUT, 0, budget, min_rate, 0.0)
+        obj = Objective(OBJ_MAX_THROUGHPUT, dp_default_flags, budget, min_rate, 0.0)
     orders = (ZoneOrder * len(zone_orders))()
     for j, zl in enumerate(zone_orders):
         if len(zl) > Z_MAX:

@@ -1,6 +1,7 @@
 // C ABI of the library (see include/sailor.h): context management, argument checks, launches.
 // Every simulation step runs in the kernels; the host only validates, packs tables and
 // enqueues work on the caller's stream.
+#include <atomic>
 #include <cmath>
 #include <cstddef>
 #include <cstdlib>
@@ -12,8 +13,10 @@
 #include <array>
 #include <map>
 
+#include "sailor_batch.cuh"
 #include "sailor_dp.cuh"
 #include "sailor_mixed.cuh"
+#include "sailor_peaks.cuh"
 
 using namespace sailor;
 
@@ -94,98 +97,6 @@ __global__ void compose_kernel(unsigned char* blob) {
     }
 }
 
-// One thread per explicit plan record (Sec. 4.3).  A block stages a pool of records in shared
-// memory with coalesced 8-byte loads, orders it by stage count (the work of a record grows with
-// its stages; any order gives the same results), and its warps take groups of 32 similar records
-// from the pool, longest first, until it is empty.  Results leave as four structure-of-arrays streams.
-constexpr uint32_t SIM_POOL = 512;
-
-__global__ void __launch_bounds__(SIM_THREADS)
-simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
-                const sailor_plan_rec* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
-                uint64_t* __restrict__ peak_mem, double* __restrict__ cost, uint32_t* __restrict__ status,
-                unsigned int* error) {
-    extern __shared__ __align__(16) unsigned char dyn[];
-    __shared__ uint64_t mbar;
-    constexpr uint32_t W = sizeof(sailor_plan_rec) / 8;      // 9 words per record
-    __shared__ uint64_t recs[SIM_POOL * W];
-    __shared__ uint32_t hist[128];
-    __shared__ uint16_t perm[SIM_POOL];
-    __shared__ uint32_t next_group;
-    const uint32_t tid = threadIdx.x, lane = tid & 31;
-    const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(blob)->static_bytes;
-    if (!bulk_load(dyn, blob, static_bytes, &mbar)) {
-        if (tid == 0) atomicExch(error, 1u);
-        for (uint32_t x = tid; x < static_bytes / 16; x += SIM_THREADS)
-            reinterpret_cast<uint4*>(dyn)[x] = reinterpret_cast<const uint4*>(blob)[x];
-        __syncthreads();
-    }
-    TabView v;
-    v.bind(dyn, blob);
-    const uint64_t* src = reinterpret_cast<const uint64_t*>(plans);
-    uint32_t* counters = reinterpret_cast<uint32_t*>(dyn + static_bytes) + tid;      // [digit][thread]
-    for (uint64_t pool = (uint64_t)blockIdx.x * SIM_POOL; pool < n; pool += (uint64_t)gridDim.x * SIM_POOL) {
-        const uint32_t cnt = (uint32_t)(n - pool < SIM_POOL ? n - pool : SIM_POOL);
-        __syncthreads();
-        for (uint32_t x = tid; x < cnt * W; x += SIM_THREADS) recs[x] = src[pool * W + x];
-        if (tid < 128) hist[tid] = 0;
-        if (tid == 0) next_group = 0;
-        __syncthreads();
-        // counting sort by descending stage count (byte 0 of a record is P)
-        uint32_t key[SIM_POOL / SIM_THREADS], rank[SIM_POOL / SIM_THREADS];
-#pragma unroll
-        for (uint32_t u = 0; u < SIM_POOL / SIM_THREADS; ++u) {
-            const uint32_t x = tid + u * SIM_THREADS;
-            key[u] = rank[u] = 0;
-            if (x < cnt) {
-                const uint32_t P = (uint32_t)(recs[x * W] & 0xff);
-                key[u] = 127u - (P > 127u ? 127u : P);
-                rank[u] = atomicAdd(&hist[key[u]], 1u);
-            }
-        }
-        __syncthreads();
-        if (tid < 32) {                                        // exclusive scan of the 128 bins by one warp
-            uint32_t h4[4], sum = 0;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) { h4[q] = hist[tid * 4 + q]; sum += h4[q]; }
-            uint32_t incl = sum;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t up = __shfl_up_sync(FULL, incl, o);
-                if (tid >= (uint32_t)o) incl += up;
-            }
-            uint32_t base = incl - sum;
-#pragma unroll
-            for (int q = 0; q < 4; ++q) { hist[tid * 4 + q] = base; base += h4[q]; }
-        }
-        __syncthreads();
-#pragma unroll
-        for (uint32_t u = 0; u < SIM_POOL / SIM_THREADS; ++u) {
-            const uint32_t x = tid + u * SIM_THREADS;
-            if (x < cnt) perm[hist[key[u]] + rank[u]] = (uint16_t)x;
-        }
-        __syncthreads();
-        const uint32_t n_groups = (cnt + 31) / 32;
-        for (;;) {                                             // warps drain the pool, longest records first
-            uint32_t grp = 0;
-            if (lane == 0) grp = atomicAdd(&next_group, 1u);
-            grp = __shfl_sync(FULL, grp, 0);
-            if (grp >= n_groups) break;
-            const uint32_t slot = grp * 32 + lane;
-            if (slot < cnt) {
-                const uint32_t mine = perm[slot];
-                const sailor_plan_rec& rec = *reinterpret_cast<const sailor_plan_rec*>(&recs[mine * W]);
-                const SimOut o = simulate_record(v, avail, rec, counters, SIM_THREADS);
-                if (t_iter) t_iter[pool + mine] = o.t_iter;
-                if (peak_mem) peak_mem[pool + mine] = o.peak_mem;
-                if (cost) cost[pool + mine] = o.cost;
-                if (status) status[pool + mine] = o.status;
-            }
-            __syncwarp();
-        }
-    }
-}
-
 // One warp per plan with mixed replicas (648-byte records, read in place, lane i reading stage i).  Tables in
 // shared memory, then R 64-bit GPU counters per warp.
 __global__ void __launch_bounds__(SIM_THREADS, 4)
@@ -250,11 +161,6 @@ constexpr size_t CFG_CACHE_MAX_BYTES = 512ull << 20;
 
 constexpr uint64_t WAVE_CONFIG_MAX = 1u << 16;
 
-struct OutBlock {                          // device -> pinned host
-    sailor_result results[SAILOR_K_MAX];
-    Ctrl ctrl;
-};
-
 }  // namespace
 
 struct sailor_ctx {
@@ -267,14 +173,20 @@ struct sailor_ctx {
     uint16_t* d_avail = nullptr;
     uint16_t* h_avail = nullptr;           // pinned
     Ctrl* d_ctrl = nullptr;
-    sailor_result* d_results = nullptr;
-    OutBlock* h_out = nullptr;             // pinned
+    unsigned int* d_sim_error = nullptr;   // error word of the explicit-batch kernels
+    PlanOut* d_out = nullptr;
+    PlanOut* h_out = nullptr;              // pinned
+    bool ctrl_dirty = true;                // the counters must be cleared from the host (first call, or after a failed one)
+    uint64_t sync_epoch = 1;               // stream synchronisations by this context so far
+    uint64_t avail_epoch = 0;              // sync_epoch when the pinned availability buffer was last handed to a copy
+    bool h2d_fresh = false;                // an availability upload has been timed and not yet read
+    float h2d_ms = 0.f;
     Hit* d_partial = nullptr;
     uint32_t* d_partial_n = nullptr;
     uint32_t max_grid = 0;                 // capacity of the partial-result buffers
     uint32_t grid_of[6] = {0, 0, 0, 0, 0, 0};   // resident blocks per kernel variant, for the cached space
     SpaceCache space;
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr, evh0 = nullptr, evh1 = nullptr;
     // explicit-batch staging (grow-only)
     unsigned char* d_stage = nullptr;
     size_t stage_bytes = 0;
@@ -293,6 +205,13 @@ namespace {
             return SAILOR_E_CUDA;                      \
         }                                              \
     } while (0)
+
+// Synchronise the context's stream; everything enqueued before (the availability upload among it) is done after.
+cudaError_t stream_sync(sailor_ctx* ctx) {
+    const cudaError_t e = cudaStreamSynchronize(ctx->stream);
+    if (e == cudaSuccess) ++ctx->sync_epoch;
+    return e;
+}
 
 struct DeviceGuard {
     int prev = -1;
@@ -407,7 +326,7 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
         }
     }
     cs[n_config] = (uint32_t)chunks;
-    const size_t smem = plan_smem_bytes(ctx->hdr.static_bytes, p_max, ctx->hdr.T, ctx->hdr.Z);
+    const size_t smem = plan_smem_bytes(ctx->hdr.static_bytes, p_max, ctx->hdr.T, ctx->hdr.Z, (uint32_t)n_config);
     if (smem > (size_t)PLAN_SMEM_CEILING) return SAILOR_E_RANGE;
 
     sc.valid = false;
@@ -419,7 +338,7 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
     CU(ctx, cudaMalloc(&sc.d_flat_base, fb.size() * sizeof(uint64_t)));
     CU(ctx, cudaMemcpyAsync(sc.d_chunk_start, cs.data(), cs.size() * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
     CU(ctx, cudaMemcpyAsync(sc.d_flat_base, fb.data(), fb.size() * sizeof(uint64_t), cudaMemcpyHostToDevice, ctx->stream));
-    CU(ctx, cudaStreamSynchronize(ctx->stream));       // the vectors are pageable
+    CU(ctx, stream_sync(ctx));       // the vectors are pageable
     {   // survey the space once: live chunks per configuration and the closed-form class counts
         cudaFree(sc.d_live_start);
         cudaFree(sc.d_cfg_closed);
@@ -460,24 +379,26 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
         live[n_config] = (uint32_t)run;
         sc.live_chunks = (uint32_t)run;
         CU(ctx, cudaMemcpyAsync(sc.d_live_start, live.data(), (n_config + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->stream));
-        CU(ctx, cudaStreamSynchronize(ctx->stream));
+        CU(ctx, stream_sync(ctx));
     }
     {   // the tables of every configuration, once: later searches copy them instead of building them
         sc.cache_head16 = cache_head16();
         sc.cache_arr16 = cache_arr16(ctx->hdr.T, ctx->hdr.Z);
         const size_t rec_bytes = 16 * ((size_t)sc.cache_head16 + sc.cache_arr16);
         if (n_config * rec_bytes <= CFG_CACHE_MAX_BYTES && cudaMalloc(&sc.d_cfg_cache, n_config * rec_bytes) == cudaSuccess) {
-            static bool optin_done[64] = {};
+            // (setting the attribute twice from two threads is harmless: both set the same value)
+            static std::atomic<bool> optin_done[64];
             const bool tracked = ctx->device >= 0 && ctx->device < 64;
-            if (!tracked || !optin_done[ctx->device]) {
+            if (!tracked || !optin_done[ctx->device].load(std::memory_order_acquire)) {
                 CU(ctx, cudaFuncSetAttribute(cfg_cache_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PLAN_SMEM_CEILING));
-                if (tracked) optin_done[ctx->device] = true;
+                if (tracked) optin_done[ctx->device].store(true, std::memory_order_release);
             }
             PlanParams pp;
             memset(&pp, 0, sizeof(pp));
             pp.blob = ctx->d_blob;
             pp.avail = ctx->d_avail;
             pp.ctrl = ctx->d_ctrl;
+            pp.cfg_flat_base = sc.d_flat_base;
             pp.sp = d;
             pp.n_config = (uint32_t)n_config;
             pp.p_max = p_max;
@@ -488,7 +409,7 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
             const uint32_t grid = (uint32_t)(n_config < (uint64_t)ctx->sm_count * 2 ? n_config : (uint64_t)ctx->sm_count * 2);
             cfg_cache_kernel<<<grid, PLAN_THREADS, smem, ctx->stream>>>(pp, sc.d_cfg_cache);
             CU(ctx, cudaGetLastError());
-            CU(ctx, cudaStreamSynchronize(ctx->stream));
+            CU(ctx, stream_sync(ctx));
         } else {
             sc.d_cfg_cache = nullptr;          // too large (or no memory): searches build the tables themselves
             (void)cudaGetLastError();
@@ -533,30 +454,31 @@ PlanKernel pick_kernel(uint32_t obj, bool constr) {
 // The dynamic shared-memory opt-in belongs to the kernel (per device), not to a context: raise it
 // once per (device, variant) to the ceiling every space is checked against, so that contexts
 // with different table sizes cannot lower it under one another.
-bool g_optin_done[64][6] = {};
+// The flags are atomic: contexts on different host threads may get here together, and setting the
+// attribute twice to the same value is harmless.
+std::atomic<bool> g_optin_done[64][6];
 
 int smem_optin(sailor_ctx* ctx, PlanKernel kern, uint32_t variant) {
     const bool tracked = ctx->device >= 0 && ctx->device < 64;
-    if (tracked && g_optin_done[ctx->device][variant]) return SAILOR_OK;
+    if (tracked && g_optin_done[ctx->device][variant].load(std::memory_order_acquire)) return SAILOR_OK;
     CU(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, PLAN_SMEM_CEILING));
-    if (tracked) g_optin_done[ctx->device][variant] = true;
+    if (tracked) g_optin_done[ctx->device][variant].store(true, std::memory_order_release);
     return SAILOR_OK;
 }
 
-// Enqueue one search pass (clear, search, merge) on the context's stream.
+// Enqueue one search pass on the context's stream: the search kernel, whose last block also merges the
+// blocks' lists and writes the results (no separate merge launch, no clearing from the host).
 //
 // With SAILOR_FLAG_DEGREE_ORDER (whole space, live layout) the search runs as n_d waves: a one-block
 // step kernel applies the H3/H4 rule to the previous wave's per-configuration bests and lays out the
 // next wave's chunks, then the search kernel evaluates them; every block carries its list from wave
-// to wave, so one merge at the end suffices.
+// to wave, and the last wave's launch ends the pass.
 int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_ctrl, double min_rate,
                  uint32_t flags, uint64_t lo, uint64_t hi, bool live, uint32_t k, double next_budget_factor,
-                 uint32_t* n_launches) {
+                 uint32_t* n_launches, bool* launched) {
     SpaceCache& sc = ctx->space;
     const bool waves = (flags & SAILOR_FLAG_DEGREE_ORDER) != 0;
-    // clear the counters; ctrl->budget (the previous pass may have written it) and the sticky error stay
-    CU(ctx, cudaMemsetAsync(ctx->d_ctrl, 0, offsetof(Ctrl, min_cost_bits), ctx->stream));
-    CU(ctx, cudaMemsetAsync(&ctx->d_ctrl->min_cost_bits, 0x7f, sizeof(unsigned long long), ctx->stream));
+    // the counters start from the values the last finished pass (or the host, after a failure) left them at
     PlanParams pp;
     memset(&pp, 0, sizeof(pp));
     pp.blob = ctx->d_blob;
@@ -580,6 +502,10 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
     pp.p_max = sc.p_max;
     pp.budget = budget;
     pp.min_rate = min_rate;
+    pp.out = ctx->d_out;
+    pp.finish = 1;
+    pp.next_budget_factor = next_budget_factor;
+    pp.cost_only = next_budget_factor > 0.0 ? 1u : 0u;
     uint32_t grid = 0;
     if (waves) {                   // the chunk table and the chunk count of each wave are written on the device
         pp.cfg_chunk_start = sc.d_wave_start;
@@ -648,28 +574,28 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
                 wave_step_kernel<<<1, WAVE_THREADS, 0, ctx->stream>>>(wp);
                 CU(ctx, cudaGetLastError());
                 pp.carry_lists = w ? 1u : 0u;
+                pp.finish = (w + 1 == wp.n_d) ? 1u : 0u;       // the last wave's launch ends the pass
                 kern<<<grid, PLAN_THREADS, sc.smem, ctx->stream>>>(pp);
                 CU(ctx, cudaGetLastError());
                 *n_launches += 2;
             }
         }
     }
-    MergeParams mp;
-    memset(&mp, 0, sizeof(mp));
-    mp.blob = ctx->d_blob;
-    mp.avail = ctx->d_avail;
-    mp.partial = ctx->d_partial;
-    mp.partial_n = ctx->d_partial_n;
-    mp.ctrl = ctx->d_ctrl;
-    mp.results = ctx->d_results;
-    mp.sp = sc.desc;
-    mp.n_partial = grid;
-    mp.k = k;
-    mp.obj = obj;
-    mp.budget_factor = next_budget_factor;
-    merge_kernel<<<1, MERGE_THREADS, ctx->hdr.static_bytes, ctx->stream>>>(mp);
-    CU(ctx, cudaGetLastError());
-    ++*n_launches;
+    *launched = grid != 0;
+    return SAILOR_OK;
+}
+
+// End of a host-side batch call: read the batch kernels' error word with the results, wait, and report (and
+// clear) a fault.  Device-side batch calls only enqueue work; a fault in one of them is reported here as well,
+// by the next host-side call.
+int finish_host_batch(sailor_ctx* ctx) {
+    unsigned int* h_err = &ctx->h_out->ctrl.error;               // pinned; no search is in flight on this context
+    CU(ctx, cudaMemcpyAsync(h_err, ctx->d_sim_error, sizeof(unsigned int), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, stream_sync(ctx));
+    if (*h_err) {
+        CU(ctx, cudaMemsetAsync(ctx->d_sim_error, 0, sizeof(unsigned int), ctx->stream));
+        return SAILOR_E_DEVICE;
+    }
     return SAILOR_OK;
 }
 
@@ -769,6 +695,8 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
         h.reserved[g] = c->reserved[g];
     }
     for (int k = 0; k < SAILOR_KINDS; ++k) h.params[k] = p->params[k];
+    for (uint32_t i = 0; i < n_tp; ++i)
+        if (m->heads % p->tp_values[i] == 0) h.heads_ok |= 1u << i;
 
     std::vector<unsigned char> blob(sizeof(TabHdr));
     h.off_fwd = put(blob, p->fwd, n4);
@@ -797,7 +725,8 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     const size_t n_comp = (size_t)4 * h.chain_len;
     const size_t cmp_fb = n_comp * T * n_tp * n_mbs * 2, cmp_upd = n_comp * T * n_tp, cmp_mem = n_comp * n_tp * n_mbs * 2 * 2,
                  cmp_grad = n_comp * n_tp;
-    if (h.static_bytes + (2 * c4 + c3 + cmp_fb + cmp_upd + cmp_mem + cmp_grad + n_comp) * sizeof(double) + 256 > (1ull << 30) ||
+    if (h.static_bytes + (2 * c4 + c3 + cmp_fb + cmp_upd + cmp_mem + cmp_grad + n_comp) * sizeof(double) +
+                cmp_fb * sizeof(PieceRec) + (2 * R + (size_t)Z * Z) * n_mbs * sizeof(double) + 512 > (1ull << 30) ||
         h.static_bytes > 96 * 1024) {
         delete ctx;
         return SAILOR_E_RANGE;
@@ -810,6 +739,10 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     h.off_cmp_mem = put<uint64_t>(blob, nullptr, cmp_mem);
     h.off_cmp_fb = put<double>(blob, nullptr, cmp_fb);
     h.off_cmp_upd = put<double>(blob, nullptr, cmp_upd);
+    h.off_piece = put<PieceRec>(blob, nullptr, cmp_fb);
+    h.off_lnk_intra2 = put<double>(blob, nullptr, R * n_mbs);
+    h.off_lnk_inter2 = put<double>(blob, nullptr, R * n_mbs);
+    h.off_lnk_zone2 = put<double>(blob, nullptr, (size_t)Z * Z * n_mbs);
     h.total_bytes = align16((uint32_t)blob.size());
     blob.resize(h.total_bytes);
     memcpy(blob.data(), &h, sizeof(h));
@@ -832,16 +765,21 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     CUF(cudaMallocHost(&ctx->h_avail, R_MAX * sizeof(uint16_t)));
     memset(ctx->h_avail, 0, R_MAX * sizeof(uint16_t));       // availability starts at zero on both sides
     CUF(cudaMalloc(&ctx->d_ctrl, sizeof(Ctrl)));
-    CUF(cudaMalloc(&ctx->d_results, sizeof(sailor_result) * SAILOR_K_MAX));
-    CUF(cudaMallocHost(&ctx->h_out, sizeof(OutBlock)));
+    CUF(cudaMalloc(&ctx->d_sim_error, sizeof(unsigned int)));
+    CUF(cudaMalloc(&ctx->d_out, sizeof(PlanOut)));
+    CUF(cudaMallocHost(&ctx->h_out, sizeof(PlanOut)));
     CUF(cudaMalloc(&ctx->d_partial, sizeof(Hit) * SAILOR_K_MAX * ctx->max_grid));
     CUF(cudaMalloc(&ctx->d_partial_n, sizeof(uint32_t) * ctx->max_grid));
     CUF(cudaEventCreate(&ctx->ev0));
     CUF(cudaEventCreate(&ctx->ev1));
+    CUF(cudaEventCreate(&ctx->ev2));
+    CUF(cudaEventCreate(&ctx->evh0));
+    CUF(cudaEventCreate(&ctx->evh1));
     CUF(cudaMemcpyAsync(ctx->d_blob, blob.data(), h.total_bytes, cudaMemcpyHostToDevice, ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_avail, 0, R_MAX * sizeof(uint16_t), ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_ctrl, 0, sizeof(Ctrl), ctx->stream));
-    CUF(cudaMemsetAsync(ctx->d_results, 0, sizeof(sailor_result) * SAILOR_K_MAX, ctx->stream));
+    CUF(cudaMemsetAsync(ctx->d_sim_error, 0, sizeof(unsigned int), ctx->stream));
+    CUF(cudaMemsetAsync(ctx->d_out, 0, sizeof(PlanOut), ctx->stream));
     {
         const uint32_t n_threads = 4 * T * n_tp * n_mbs + 2 * T * n_tp;
         chain_kernel<<<(n_threads + 127) / 128, 128, 0, ctx->stream>>>(ctx->d_blob);
@@ -850,12 +788,13 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
         const uint32_t grid = (uint32_t)((n_cmp + 127) / 128 < 65536 ? (n_cmp + 127) / 128 : 65536);
         compose_kernel<<<grid, 128, 0, ctx->stream>>>(ctx->d_blob);
         CUF(cudaGetLastError());
+        batch_tables_kernel<<<grid, 128, 0, ctx->stream>>>(ctx->d_blob);
+        CUF(cudaGetLastError());
     }
     CUF(cudaStreamSynchronize(ctx->stream));           // `blob` is pageable host memory
     // both kernels stage the static tables in dynamic shared memory; the create-time limit is 96 KB
-    CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
+    CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)batch_smem_bytes(R_MAX)));
     CUF(cudaFuncSetAttribute(simulate_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
-    CUF(cudaFuncSetAttribute(merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024));
 #undef CUF
     *out = ctx;
     return SAILOR_OK;
@@ -869,7 +808,8 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->d_avail);
     cudaFreeHost(ctx->h_avail);
     cudaFree(ctx->d_ctrl);
-    cudaFree(ctx->d_results);
+    cudaFree(ctx->d_sim_error);
+    cudaFree(ctx->d_out);
     cudaFreeHost(ctx->h_out);
     cudaFree(ctx->d_partial);
     cudaFree(ctx->d_partial_n);
@@ -883,8 +823,8 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->space.d_cfg_cache);
     cudaFree(ctx->d_stage);
     cudaFree(ctx->d_dp);
-    if (ctx->ev0) cudaEventDestroy(ctx->ev0);
-    if (ctx->ev1) cudaEventDestroy(ctx->ev1);
+    for (cudaEvent_t e : {ctx->ev0, ctx->ev1, ctx->ev2, ctx->evh0, ctx->evh1})
+        if (e) cudaEventDestroy(e);
     delete ctx;
     return SAILOR_OK;
 }
@@ -892,11 +832,15 @@ int sailor_destroy(sailor_ctx* ctx) {
 int sailor_set_availability(sailor_ctx* ctx, const uint16_t* avail) {
     if (!ctx || !avail) return SAILOR_E_ARG;
     DeviceGuard guard(ctx->device);
-    // the pinned staging buffer may still feed the previous copy
-    CU(ctx, cudaStreamSynchronize(ctx->stream));
+    // the pinned staging buffer may still feed the previous copy, unless the stream has been synchronised since
+    if (ctx->avail_epoch == ctx->sync_epoch) CU(ctx, stream_sync(ctx));
     memcpy(ctx->h_avail, avail, ctx->hdr.R * sizeof(uint16_t));
+    CU(ctx, cudaEventRecord(ctx->evh0, ctx->stream));
     CU(ctx, cudaMemcpyAsync(ctx->d_avail, ctx->h_avail, ctx->hdr.R * sizeof(uint16_t), cudaMemcpyHostToDevice,
                             ctx->stream));
+    CU(ctx, cudaEventRecord(ctx->evh1, ctx->stream));
+    ctx->avail_epoch = ctx->sync_epoch;
+    ctx->h2d_fresh = true;
     return SAILOR_OK;
 }
 
@@ -917,7 +861,7 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
         }
         const size_t need = n * (sizeof(sailor_plan_rec) + 32);
         if (need > ctx->stage_bytes) {
-            CU(ctx, cudaStreamSynchronize(ctx->stream));
+            CU(ctx, stream_sync(ctx));
             cudaFree(ctx->d_stage);
             ctx->d_stage = nullptr;
             ctx->stage_bytes = 0;
@@ -934,19 +878,18 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
         CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_plan_rec), cudaMemcpyHostToDevice, ctx->stream));
         d_plans = dp;
     }
-    const uint64_t tiles = (n + SIM_POOL - 1) / SIM_POOL;
-    const uint64_t cap = (uint64_t)ctx->sm_count * 16;
+    const uint64_t tiles = (n + BATCH_POOL - 1) / BATCH_POOL;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 12;         // three resident blocks per SM, four pools each at least
     const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
-    const size_t sim_smem = ctx->hdr.static_bytes + sizeof(uint32_t) * SIM_THREADS * ctx->hdr.R;   // tables + per-thread counters
-    simulate_kernel<<<grid, SIM_THREADS, sim_smem, ctx->stream>>>(
-        ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s, &ctx->d_ctrl->error);
+    simulate_kernel<<<grid, BATCH_THREADS, batch_smem_bytes(ctx->hdr.R), ctx->stream>>>(
+        ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s);
     CU(ctx, cudaGetLastError());
     if (!on_device) {
         if (t_iter) CU(ctx, cudaMemcpyAsync(t_iter, d_t, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
         if (cost) CU(ctx, cudaMemcpyAsync(cost, d_c, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
         if (peak_mem) CU(ctx, cudaMemcpyAsync(peak_mem, d_m, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
         if (status) CU(ctx, cudaMemcpyAsync(status, d_s, 4 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        CU(ctx, cudaStreamSynchronize(ctx->stream));
+        return finish_host_batch(ctx);
     }
     return SAILOR_OK;
 }
@@ -975,7 +918,7 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
         }
         const size_t need = n * (sizeof(sailor_mixed_plan) + 32);
         if (need > ctx->stage_bytes) {
-            CU(ctx, cudaStreamSynchronize(ctx->stream));
+            CU(ctx, stream_sync(ctx));
             cudaFree(ctx->d_stage);
             ctx->d_stage = nullptr;
             ctx->stage_bytes = 0;
@@ -997,14 +940,14 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
     const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
     const size_t smem = ctx->hdr.static_bytes + sizeof(unsigned long long) * (SIM_THREADS / 32) * ctx->hdr.R;
     simulate_mixed_kernel<<<grid, SIM_THREADS, smem, ctx->stream>>>(ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s,
-                                                                     &ctx->d_ctrl->error);
+                                                                     ctx->d_sim_error);
     CU(ctx, cudaGetLastError());
     if (!on_device) {
         if (t_iter) CU(ctx, cudaMemcpyAsync(t_iter, d_t, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
         if (cost) CU(ctx, cudaMemcpyAsync(cost, d_c, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
         if (peak_mem) CU(ctx, cudaMemcpyAsync(peak_mem, d_m, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
         if (status) CU(ctx, cudaMemcpyAsync(status, d_s, 4 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        CU(ctx, cudaStreamSynchronize(ctx->stream));
+        return finish_host_batch(ctx);
     }
     return SAILOR_OK;
 }
@@ -1030,6 +973,7 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
     if (std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) ||
         std::isnan(o->budget_factor_over_cheapest))
         return SAILOR_E_ARG;
+    if (o->flags & ~(SAILOR_FLAG_EVAL_ALL | SAILOR_FLAG_DEGREE_ORDER | SAILOR_FLAG_MIN_TP_ONLY)) return SAILOR_E_ARG;
     DeviceGuard guard(ctx->device);
     int rc = prepare_space(ctx, s);
     if (rc) return rc;
@@ -1045,26 +989,38 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
     }
 
     uint32_t launches = 0;
+    if (ctx->ctrl_dirty) {             // first search of the context, or the last one failed half-way
+        CU(ctx, cudaMemsetAsync(ctx->d_ctrl, 0, sizeof(Ctrl), ctx->stream));
+        CU(ctx, cudaMemsetAsync(&ctx->d_ctrl->min_cost_bits, 0x7f, sizeof(unsigned long long), ctx->stream));
+    }
+    ctx->ctrl_dirty = true;            // until this call has gone through
     CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
     const bool two_pass = o->budget_factor_over_cheapest > 0.0;
     // a whole-space search with pruning on walks only the prefixes the survey found live
     const bool live = !(o->flags & SAILOR_FLAG_EVAL_ALL) && flat_lo == 0 && flat_hi == total;
+    bool launched = false;
     if (two_pass) {
-        // cheapest feasible plan first; its merge step leaves factor * cost in ctrl->budget
+        // cheapest feasible plan first; the block that ends that pass leaves factor * cost in ctrl->budget
         rc = enqueue_pass(ctx, SAILOR_OBJ_MIN_COST, 0.0, false, 0.0, o->flags, flat_lo, flat_hi, live, 1,
-                          o->budget_factor_over_cheapest, &launches);
+                          o->budget_factor_over_cheapest, &launches, &launched);
         if (rc) return rc;
     }
     rc = enqueue_pass(ctx, o->kind, o->budget_usd_per_iter, two_pass, o->min_iters_per_s, o->flags, flat_lo,
-                      flat_hi, live, k, 0.0, &launches);
+                      flat_hi, live, k, 0.0, &launches, &launched);
     if (rc) return rc;
     CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
-    CU(ctx, cudaMemcpyAsync(ctx->h_out->results, ctx->d_results, sizeof(sailor_result) * k, cudaMemcpyDeviceToHost,
-                            ctx->stream));
-    CU(ctx, cudaMemcpyAsync(&ctx->h_out->ctrl, ctx->d_ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, ctx->stream));
-    CU(ctx, cudaStreamSynchronize(ctx->stream));
+    if (launched) {
+        CU(ctx, cudaMemcpyAsync(ctx->h_out, ctx->d_out, sizeof(Ctrl) + sizeof(sailor_result) * k, cudaMemcpyDeviceToHost,
+                                ctx->stream));
+        if (stats) CU(ctx, cudaEventRecord(ctx->ev2, ctx->stream));
+    } else {
+        memset(&ctx->h_out->ctrl, 0, sizeof(Ctrl));           // an empty range: nothing ran, nothing was found
+    }
+    CU(ctx, stream_sync(ctx));
+    ctx->ctrl_dirty = false;
     const Ctrl& cr = ctx->h_out->ctrl;
     if (cr.error) return SAILOR_E_DEVICE;
+    if (cr.n_found > k) return SAILOR_E_DEVICE;               // cannot happen; never copy past the caller's k records
     *n_found = cr.n_found;
     memcpy(topk, ctx->h_out->results, sizeof(sailor_result) * cr.n_found);
     if (stats) {
@@ -1082,7 +1038,7 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
         stats->n_over_avail = cr.stats[3];
         stats->n_over_constraint = cr.stats[4];
         stats->n_feasible = cr.stats[5];
-        stats->budget_used = two_pass ? cr.budget : o->budget_usd_per_iter;
+        stats->budget_used = two_pass ? (launched ? cr.budget : 0.0) : o->budget_usd_per_iter;
         double mc;
         memcpy(&mc, &cr.min_cost_bits, sizeof(mc));
         stats->min_feasible_cost = cr.stats[5] ? mc : 0.0;
@@ -1090,6 +1046,13 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
         CU(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
         stats->kernel_ms = ms;
         stats->n_launches = launches;
+        stats->d2h_ms = 0.f;
+        if (launched) CU(ctx, cudaEventElapsedTime(&stats->d2h_ms, ctx->ev1, ctx->ev2));
+        if (ctx->h2d_fresh) {              // the upload was enqueued before this search and is complete by now
+            CU(ctx, cudaEventElapsedTime(&ctx->h2d_ms, ctx->evh0, ctx->evh1));
+            ctx->h2d_fresh = false;
+        }
+        stats->h2d_ms = ctx->h2d_ms;
     }
     return SAILOR_OK;
 }
@@ -1113,7 +1076,7 @@ constexpr uint32_t NOALLOC_GRID_MAX = 1024;     // blocks whose partial lists fi
 
 struct NoAllocScratch {                         // layout of the fixed scratch array
     Ctrl ctrl;
-    sailor_result results[SAILOR_K_MAX];
+    PlanOut out;
     uint32_t partial_n[NOALLOC_GRID_MAX];
     Hit partial[(size_t)NOALLOC_GRID_MAX * SAILOR_K_MAX];
     uint32_t cfg_chunk_start[SAILOR_NOALLOC_CONFIG_MAX + 1];
@@ -1123,23 +1086,30 @@ struct NoAllocScratch {                         // layout of the fixed scratch a
 // About 0.6 MB, held by every GPU that loads the library until the process exits.  In host code
 // this name is only a handle for cudaGetSymbolAddress; it is never passed to a kernel.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+static_assert(offsetof(NoAllocScratch, partial) % 16 == 0, "the lists are read 16 bytes at a time");
 
 constexpr int NOALLOC_DEVICES_MAX = 64;
-NoAllocScratch* g_noalloc_ptr[NOALLOC_DEVICES_MAX] = {};     // device address of the array, per device
+// device address of the array, per device (atomic: two threads resolving it together store the same address)
+std::atomic<NoAllocScratch*> g_noalloc_ptr[NOALLOC_DEVICES_MAX];
+// resident blocks per SM of each kernel variant at a given shared-memory size, per device (0 = not asked yet)
+struct OccupancyMemo { std::atomic<uint64_t> smem_and_blocks; };
+OccupancyMemo g_noalloc_occ[NOALLOC_DEVICES_MAX][6];
 
 // Device address of the scratch on the current device; resolved on first use per device.
 int noalloc_scratch(sailor_ctx* ctx, NoAllocScratch** out) {
     if (ctx->device < 0 || ctx->device >= NOALLOC_DEVICES_MAX) return SAILOR_E_RANGE;
-    if (!g_noalloc_ptr[ctx->device]) {
+    NoAllocScratch* known = g_noalloc_ptr[ctx->device].load(std::memory_order_acquire);
+    if (!known) {
         void* p = nullptr;
         CU(ctx, cudaGetSymbolAddress(&p, g_noalloc_scratch));
-        g_noalloc_ptr[ctx->device] = static_cast<NoAllocScratch*>(p);
+        known = static_cast<NoAllocScratch*>(p);
+        g_noalloc_ptr[ctx->device].store(known, std::memory_order_release);
     }
-    *out = g_noalloc_ptr[ctx->device];
+    *out = known;
     return SAILOR_OK;
 }
 
-// One pass (clear, search, merge) whose scratch all lies in `sc`.
+// One pass (clear, search with its merge) whose scratch all lies in `sc`.
 int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& desc, uint32_t n_config,
                          uint32_t p_max, size_t smem, uint32_t chunk_lo, uint32_t chunk_hi, uint64_t total,
                          uint32_t obj, double budget, bool budget_from_ctrl, double min_rate, uint32_t flags,
@@ -1169,15 +1139,27 @@ int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& d
     pp.min_rate = min_rate;
     pp.chunk_lo = chunk_lo;
     pp.chunk_hi = chunk_hi;
+    pp.out = &sc->out;
+    pp.finish = 1;
+    pp.next_budget_factor = next_budget_factor;
+    pp.cost_only = next_budget_factor > 0.0 ? 1u : 0u;
     const uint32_t n_chunks = chunk_hi - chunk_lo;
     const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
     PlanKernel kern = pick_kernel(obj, constr);
+    const uint32_t variant = obj * 2 + (constr ? 1 : 0);
     {
-        const int rc_opt = smem_optin(ctx, kern, obj * 2 + (constr ? 1 : 0));
+        const int rc_opt = smem_optin(ctx, kern, variant);
         if (rc_opt) return rc_opt;
     }
+    // the occupancy query costs host time on a path that exists for its latency: ask once per (device, variant, size)
     int per_sm = 0;
-    CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, smem));
+    std::atomic<uint64_t>& memo = g_noalloc_occ[ctx->device][variant].smem_and_blocks;
+    const uint64_t seen = memo.load(std::memory_order_acquire);
+    if (seen && (seen >> 8) == (uint64_t)smem) per_sm = (int)(seen & 0xff);
+    else {
+        CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, smem));
+        if (per_sm >= 1 && per_sm < 256) memo.store(((uint64_t)smem << 8) | (uint64_t)per_sm, std::memory_order_release);
+    }
     if (per_sm < 1) return SAILOR_E_RANGE;
     uint32_t grid = (uint32_t)per_sm * (uint32_t)ctx->sm_count;
     if (grid > NOALLOC_GRID_MAX) grid = NOALLOC_GRID_MAX;
@@ -1185,22 +1167,6 @@ int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& d
     const uint32_t batch = n_chunks / (grid * 32u);
     pp.batch = batch < 1 ? 1 : (batch > 16 ? 16 : batch);
     kern<<<grid, PLAN_THREADS, smem, ctx->stream>>>(pp);
-    CU(ctx, cudaGetLastError());
-    ++*n_launches;
-    MergeParams mp;
-    memset(&mp, 0, sizeof(mp));
-    mp.blob = ctx->d_blob;
-    mp.avail = ctx->d_avail;
-    mp.partial = sc->partial;
-    mp.partial_n = sc->partial_n;
-    mp.ctrl = &sc->ctrl;
-    mp.results = sc->results;
-    mp.sp = desc;
-    mp.n_partial = grid;
-    mp.k = k;
-    mp.obj = obj;
-    mp.budget_factor = next_budget_factor;
-    merge_kernel<<<1, MERGE_THREADS, ctx->hdr.static_bytes, ctx->stream>>>(mp);
     CU(ctx, cudaGetLastError());
     ++*n_launches;
     return SAILOR_OK;
@@ -1215,7 +1181,7 @@ extern "C" int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const
     if (std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) ||
         std::isnan(o->budget_factor_over_cheapest))
         return SAILOR_E_ARG;
-    if (o->flags & SAILOR_FLAG_DEGREE_ORDER) return SAILOR_E_ARG;           // needs tables this variant has no room for
+    if (o->flags & ~(SAILOR_FLAG_EVAL_ALL | SAILOR_FLAG_MIN_TP_ONLY)) return SAILOR_E_ARG;   // degree order needs tables this variant has no room for
     int rc = check_space(ctx, s);
     if (rc) return rc;
     const SpaceDesc d = to_desc(s);
@@ -1246,41 +1212,49 @@ extern "C" int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const
         }
     }
     h_chunk_start[n_config] = (uint32_t)chunks;
-    const size_t smem = plan_smem_bytes(ctx->hdr.static_bytes, p_max, ctx->hdr.T, ctx->hdr.Z);
+    const size_t smem = plan_smem_bytes(ctx->hdr.static_bytes, p_max, ctx->hdr.T, ctx->hdr.Z, (uint32_t)n_config);
     if (smem > 200 * 1024) return SAILOR_E_RANGE;
 
     DeviceGuard guard(ctx->device);
     NoAllocScratch* sc = nullptr;
     rc = noalloc_scratch(ctx, &sc);
     if (rc) return rc;
-    // the host arrays are reused by the next call on this thread: wait for the copies below at the end
-    CU(ctx, cudaMemcpyAsync(sc->cfg_chunk_start, h_chunk_start, (n_config + 1) * sizeof(uint32_t),
-                            cudaMemcpyHostToDevice, ctx->stream));
-    CU(ctx, cudaMemcpyAsync(sc->cfg_flat_base, h_flat_base, n_config * sizeof(uint64_t), cudaMemcpyHostToDevice,
-                            ctx->stream));
-    CU(ctx, cudaMemsetAsync(&sc->ctrl, 0, sizeof(Ctrl), ctx->stream));      // also the sticky error word
+    // the host arrays are reused by the next call on this thread: once a copy from them is enqueued, no path
+    // leaves this function without waiting for the stream
+    cudaError_t ce = cudaMemcpyAsync(sc->cfg_chunk_start, h_chunk_start, (n_config + 1) * sizeof(uint32_t),
+                                     cudaMemcpyHostToDevice, ctx->stream);
+    if (ce == cudaSuccess)
+        ce = cudaMemcpyAsync(sc->cfg_flat_base, h_flat_base, n_config * sizeof(uint64_t), cudaMemcpyHostToDevice, ctx->stream);
+    if (ce == cudaSuccess) ce = cudaMemsetAsync(&sc->ctrl, 0, sizeof(Ctrl), ctx->stream);      // also the error word
+    if (ce == cudaSuccess) ce = cudaMemsetAsync(&sc->out.ctrl, 0, sizeof(Ctrl), ctx->stream);  // read back even if nothing runs
 
     uint32_t launches = 0;
-    CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
+    if (ce == cudaSuccess) ce = cudaEventRecord(ctx->ev0, ctx->stream);
     const bool two_pass = o->budget_factor_over_cheapest > 0.0;
-    if (total > 0) {
-        if (two_pass) {
+    rc = SAILOR_OK;
+    if (ce == cudaSuccess && total > 0) {
+        if (two_pass)
             rc = enqueue_pass_noalloc(ctx, sc, d, (uint32_t)n_config, p_max, smem, 0, (uint32_t)chunks, total,
                                       SAILOR_OBJ_MIN_COST, 0.0, false, 0.0, o->flags, 1,
                                       o->budget_factor_over_cheapest, &launches);
-            if (rc) return rc;
-        }
-        rc = enqueue_pass_noalloc(ctx, sc, d, (uint32_t)n_config, p_max, smem, 0, (uint32_t)chunks, total, o->kind,
-                                  o->budget_usd_per_iter, two_pass, o->min_iters_per_s, o->flags, k, 0.0, &launches);
-        if (rc) return rc;
+        if (rc == SAILOR_OK)
+            rc = enqueue_pass_noalloc(ctx, sc, d, (uint32_t)n_config, p_max, smem, 0, (uint32_t)chunks, total, o->kind,
+                                      o->budget_usd_per_iter, two_pass, o->min_iters_per_s, o->flags, k, 0.0, &launches);
     }
-    CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
-    CU(ctx, cudaMemcpyAsync(ctx->h_out->results, sc->results, sizeof(sailor_result) * k, cudaMemcpyDeviceToHost,
-                            ctx->stream));
-    CU(ctx, cudaMemcpyAsync(&ctx->h_out->ctrl, &sc->ctrl, sizeof(Ctrl), cudaMemcpyDeviceToHost, ctx->stream));
-    CU(ctx, cudaStreamSynchronize(ctx->stream));
+    if (ce == cudaSuccess && rc == SAILOR_OK) ce = cudaEventRecord(ctx->ev1, ctx->stream);
+    if (ce == cudaSuccess && rc == SAILOR_OK)
+        ce = cudaMemcpyAsync(ctx->h_out, &sc->out, sizeof(Ctrl) + sizeof(sailor_result) * k, cudaMemcpyDeviceToHost, ctx->stream);
+    if (ce == cudaSuccess && rc == SAILOR_OK && stats) ce = cudaEventRecord(ctx->ev2, ctx->stream);
+    {
+        const cudaError_t se = stream_sync(ctx);               // on every path: the copies above read this thread's arrays
+        if (ce == cudaSuccess) ce = se;
+    }
+    if (ce != cudaSuccess) { ctx->last_cuda = (int)ce; return SAILOR_E_CUDA; }
+    if (rc) return rc;
     const Ctrl& cr = ctx->h_out->ctrl;
     if (cr.error) return SAILOR_E_DEVICE;
+    // overlapping calls race on the shared array (documented): whatever they left, never copy past k records
+    if (cr.n_found > k) return SAILOR_E_DEVICE;
     *n_found = cr.n_found;
     memcpy(topk, ctx->h_out->results, sizeof(sailor_result) * cr.n_found);
     if (stats) {
@@ -1301,6 +1275,13 @@ extern "C" int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const
         CU(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
         stats->kernel_ms = ms;
         stats->n_launches = launches;
+        stats->d2h_ms = 0.f;
+        CU(ctx, cudaEventElapsedTime(&stats->d2h_ms, ctx->ev1, ctx->ev2));
+        if (ctx->h2d_fresh) {
+            CU(ctx, cudaEventElapsedTime(&ctx->h2d_ms, ctx->evh0, ctx->evh1));
+            ctx->h2d_fresh = false;
+        }
+        stats->h2d_ms = ctx->h2d_ms;
     }
     return SAILOR_OK;
 }
@@ -1330,7 +1311,12 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     if (!ctx || !s || !orders || !o || !topk || !n_found || k == 0 || n_orders == 0) return SAILOR_E_ARG;
     if (k > SAILOR_K_MAX) return SAILOR_E_RANGE;
     // the recursion minimises iteration time; a constraint is checked on the plan it returns per problem
-    if (o->kind != SAILOR_OBJ_MAX_THROUGHPUT || o->flags != 0 || o->budget_factor_over_cheapest > 0.0 ||
+    constexpr uint32_t dp_flags = SAILOR_DP_FLAG_INDEX_DENSE | SAILOR_DP_FLAG_INDEX_COMPACT | SAILOR_DP_FLAG_ENUM_BY_TYPE |
+                                  SAILOR_DP_FLAG_ENUM_BY_ENTRY;
+    if (o->kind != SAILOR_OBJ_MAX_THROUGHPUT || (o->flags & ~dp_flags) != 0 ||
+        ((o->flags & SAILOR_DP_FLAG_INDEX_DENSE) && (o->flags & SAILOR_DP_FLAG_INDEX_COMPACT)) ||
+        ((o->flags & SAILOR_DP_FLAG_ENUM_BY_TYPE) && (o->flags & SAILOR_DP_FLAG_ENUM_BY_ENTRY)) ||
+        o->budget_factor_over_cheapest > 0.0 ||
         std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) || std::isnan(o->budget_factor_over_cheapest))
         return SAILOR_E_ARG;
     int rc = check_space(ctx, s);
@@ -1357,13 +1343,11 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     std::vector<DpProblem> prob(n_problems);
     std::vector<uint32_t> vtabs;        // rank tables of the compactly indexed zone positions, all problems
     // how a zone position's count vectors are indexed: 0 = the smaller of the two ways, 1 = mixed radix whenever it
-    // fits, 2 = by rank whenever it fits (the environment variable exists for tests that exercise each way)
-    int index_mode = 0;
-    if (const char* env = getenv("SAILOR_DP_INDEX")) index_mode = !strcmp(env, "dense") ? 1 : !strcmp(env, "compact") ? 2 : 0;
+    // fits, 2 = by rank whenever it fits (SAILOR_DP_FLAG_INDEX_*)
+    const int index_mode = (o->flags & SAILOR_DP_FLAG_INDEX_DENSE) ? 1 : (o->flags & SAILOR_DP_FLAG_INDEX_COMPACT) ? 2 : 0;
     // which threads a stage's launch has: one per count vector the stage can have reached ("live", whenever every
-    // zone position has its rank table), or one per table entry (SAILOR_DP_ENUM=entries, for tests)
-    bool all_live = true;
-    if (const char* env = getenv("SAILOR_DP_ENUM")) all_live = strcmp(env, "entries") != 0;
+    // zone position has its rank table), or one per table entry (SAILOR_DP_FLAG_ENUM_BY_ENTRY)
+    bool all_live = !(o->flags & SAILOR_DP_FLAG_ENUM_BY_ENTRY);
     std::vector<uint64_t> V, live_stage;                     // scratch of the loop below
     std::vector<uint64_t> live_off(n_problems + 1, 0);      // per problem: where its per-stage live counts start
     std::vector<uint32_t> live_cnt;                          // count vectors stage i can have reached, all positions
@@ -1528,8 +1512,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     }
     // a thread per count vector for all its types at once, or a thread per (count vector, type)
     // (its blocks stage their problem's rank tables in shared memory: at most Z * (T + 1) * (P + 1) words)
-    bool by_vector = all_live && vt_len_max * 4 <= 40 * 1024;
-    if (const char* env = getenv("SAILOR_DP_ENUM")) by_vector = by_vector && strcmp(env, "types") != 0;
+    const bool by_vector = all_live && vt_len_max * 4 <= 40 * 1024 && !(o->flags & SAILOR_DP_FLAG_ENUM_BY_TYPE);
     const uint32_t live_mult = by_vector ? 1u : T;
 
     DeviceGuard guard(ctx->device);
@@ -1541,7 +1524,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
                          2 * padded((max_blocks + p_max + 16) * sizeof(uint32_t)) + 2 * padded(max_entries * sizeof(DpVal)) +
                          padded(max_choice) + padded(sizeof(sailor_dp_result) * SAILOR_K_MAX) + padded(24) + 4096;
     if (total > ctx->dp_bytes) {
-        CU(ctx, cudaStreamSynchronize(ctx->stream));
+        CU(ctx, stream_sync(ctx));
         cudaFree(ctx->d_dp);
         ctx->d_dp = nullptr;
         ctx->dp_bytes = 0;
@@ -1591,7 +1574,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
             dp_finish_kernel<<<(fp.n_problems + 127) / 128, 128, 0, ctx->stream>>>(fp);
             CU(ctx, cudaGetLastError());
             ++launches;
-            CU(ctx, cudaStreamSynchronize(ctx->stream));       // the staging vector is reused below
+            CU(ctx, stream_sync(ctx));       // the staging vector is reused below
         }
     }
     for (const Batch& b : batches) {
@@ -1693,7 +1676,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
         dp_finish_kernel<<<(fp.n_problems + 127) / 128, 128, 0, ctx->stream>>>(fp);
         CU(ctx, cudaGetLastError());
         ++launches;
-        CU(ctx, cudaStreamSynchronize(ctx->stream));           // the host vectors are reused by the next batch
+        CU(ctx, stream_sync(ctx));           // the host vectors are reused by the next batch
     }
     DpSelectParams sel;
     memset(&sel, 0, sizeof(sel));
@@ -1708,7 +1691,8 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     std::vector<sailor_dp_result> host_out(k);
     CU(ctx, cudaMemcpyAsync(counters, d_counters, sizeof(counters), cudaMemcpyDeviceToHost, ctx->stream));
     CU(ctx, cudaMemcpyAsync(host_out.data(), d_out, sizeof(sailor_dp_result) * k, cudaMemcpyDeviceToHost, ctx->stream));
-    CU(ctx, cudaStreamSynchronize(ctx->stream));
+    CU(ctx, stream_sync(ctx));
+    if (counters[1] > k) return SAILOR_E_DEVICE;               // cannot happen; never copy past the caller's k records
     *n_found = (uint32_t)counters[1];
     memcpy(topk, host_out.data(), sizeof(sailor_dp_result) * counters[1]);
     if (stats) {
@@ -1724,6 +1708,51 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
         stats->n_batches = (uint32_t)batches.size();
         stats->_pad = 0;
     }
+    return SAILOR_OK;
+}
+
+// ---- sustained issue rates (measurement) ---------------------------------------------------------------
+
+extern "C" int sailor_measure_issue_rates(int cuda_device, void* cuda_stream, uint32_t repeats, sailor_issue_rates* out) {
+    if (!out || repeats == 0) return SAILOR_E_ARG;
+    memset(out, 0, sizeof(*out));
+    DeviceGuard guard(cuda_device);
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, cuda_device) != cudaSuccess) return SAILOR_E_CUDA;
+    double* sink = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaMalloc(&sink, sizeof(double)) != cudaSuccess) return SAILOR_E_CUDA;
+    int rc = SAILOR_OK;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) rc = SAILOR_E_CUDA;
+    const uint32_t grid = (uint32_t)prop.multiProcessorCount * 4, iters = 2048;
+    const uint64_t per_run = (uint64_t)grid * (PEAK_THREADS / 32) * iters * PEAK_CHAINS * PEAK_ROUNDS;
+    float best[3] = {0.f, 0.f, 0.f};
+    for (int kind = 0; kind < 3 && rc == SAILOR_OK; ++kind) {
+        for (uint32_t r = 0; r <= repeats && rc == SAILOR_OK; ++r) {        // run 0 warms up
+            cudaEventRecord(e0, stream);
+            // multipliers just below one and small addends keep every chain finite for any run length
+            if (kind == PEAK_FFMA) issue_stream_kernel<PEAK_FFMA><<<grid, PEAK_THREADS, 0, stream>>>(iters, 0.999f, 0.5f, 0, 0, 0.0, sink);
+            else if (kind == PEAK_IMAD) issue_stream_kernel<PEAK_IMAD><<<grid, PEAK_THREADS, 0, stream>>>(iters, 0.f, 0.f, 2654435761u, 12345u, 0.0, sink);
+            else issue_stream_kernel<PEAK_DADD><<<grid, PEAK_THREADS, 0, stream>>>(iters, 0.f, 0.f, 0, 0, 0.25, sink);
+            cudaEventRecord(e1, stream);
+            float ms = 0.f;
+            if (cudaGetLastError() != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess ||
+                cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess)
+                rc = SAILOR_E_CUDA;
+            else if (r > 0 && ms > 0.f && (best[kind] == 0.f || ms < best[kind])) best[kind] = ms;
+        }
+    }
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    cudaFree(sink);
+    if (rc) return rc;
+    out->ffma_ms = best[0]; out->imad_ms = best[1]; out->dadd_ms = best[2];
+    out->ffma_warp_inst_per_s = best[0] > 0.f ? (double)per_run / (best[0] * 1e-3) : 0.0;
+    out->imad_warp_inst_per_s = best[1] > 0.f ? (double)per_run / (best[1] * 1e-3) : 0.0;
+    out->dadd_warp_inst_per_s = best[2] > 0.f ? (double)per_run / (best[2] * 1e-3) : 0.0;
+    out->sm_count = (uint32_t)prop.multiProcessorCount;
+    out->warp_inst_per_run = per_run;
     return SAILOR_OK;
 }
 

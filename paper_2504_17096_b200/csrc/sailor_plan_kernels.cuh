@@ -27,22 +27,32 @@ constexpr int PLAN_WARPS = PLAN_THREADS / 32;
 constexpr unsigned FULL = 0xffffffffu;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;   // bound of every spin-wait in this file
 
-struct Hit {
+struct alignas(16) Hit {
     double score;
     uint64_t flat;
 };
 
 struct Ctrl {                       // one per context, device memory
-    unsigned int work_counter;      // next chunk to hand out (cleared per pass, and per wave of a pass)
-    unsigned int n_found;
+    unsigned int work_counter;      // next chunk to hand out (starts at zero in every launch)
+    unsigned int blocks_done;       // blocks of the running launch that have handed in their list
     unsigned long long stats[7];    // total, invalid, oom, over_avail, over_constraint, feasible, pruned_tp
     unsigned int wave_chunks;       // chunks of the current wave (searches in degree order)
     unsigned int n_cfg_evaluated;   // configurations selected by the waves so far
     unsigned long long min_cost_bits;   // min C_iter over feasible candidates, as ordered bits
     double budget;                  // written by the cheapest-plan pass for the next pass
-    unsigned int error;             // non-zero: a kernel gave up (bounded wait ran out); sticky
-    unsigned int _pad;
+    unsigned int error;             // non-zero: a kernel gave up during this call (bounded wait ran out)
+    unsigned int n_found;
 };
+
+// What a pass leaves for the host (one device-to-host copy: the counters, then the k records).  The block that
+// finishes a pass writes it and then puts the live counters back to their starting values, so that the next pass
+// or the next call needs no clearing from the host.
+struct PlanOut {
+    Ctrl ctrl;
+    sailor_result results[SAILOR_K_MAX];
+};
+
+constexpr unsigned long long COST_BITS_START = 0x7ff0000000000000ull;   // +inf: above every cost
 
 struct PlanParams {
     const unsigned char* blob;
@@ -65,6 +75,10 @@ struct PlanParams {
     uint32_t carry_lists;              // a block starts from the list it left in `partial` (waves of one search)
     const uint32_t* chunk_hi_dev;      // non-null: chunks [0, *chunk_hi_dev) instead of [chunk_lo, chunk_hi)
     unsigned long long* cfg_best;      // non-null: [n_config] best feasible score per configuration (ordered bits)
+    PlanOut* out;                      // where the block that finishes the pass leaves the results
+    uint32_t finish;                   // this launch ends a pass: its last block merges the lists and writes `out`
+    double next_budget_factor;         // > 0: the finishing block writes ctrl->budget = factor * best cost (next pass)
+    uint32_t cost_only;                // the pass only looks for the cheapest feasible cost (no lists, no result records)
     const uint4* cfg_cache;            // non-null: the per-configuration tables, built once per space (cfg_cache_kernel)
     uint32_t cache_head16, cache_arr16;    // 16-byte words of a cached record: CfgShared head, then the arrays
     double budget;                     // <= 0: none
@@ -196,6 +210,8 @@ struct alignas(16) CfgShared {
     uint32_t n_lower;            // smaller tensor-parallel degrees of the space that the model accepts (min_tp_only)
     uint32_t lower_tpi[SAILOR_TP_MAX];    // their tp indices
     uint64_t lower_fit[SAILOR_TP_MAX][SAILOR_SEG_MAX];   // digit d: every stage of the segment fits at that degree
+    uint64_t flat_base;          // flat index of the configuration's first candidate
+    uint64_t _pad_head;
     // ---- everything above depends on the configuration and the context only, not on availability: it is what a
     // ---- cached record holds (with the arrays rec .. fb_last); everything below belongs to the block or the snapshot
     alignas(16) uint64_t avail_last;     // digit d: need[last] <= avail[d]
@@ -217,11 +233,15 @@ struct CfgArrays {               // pointers into dynamic shared memory
     double *fb, *uu;             // [P][T]   build scratch: f+b (+f if rc), update
     uint32_t* availv;            // [R]
     uint32_t* tz;                // [R]      type | zone << 8 of a digit
+    uint32_t* chunk_tab;         // [n_config + 1] copy of the chunk offsets (spaces of fewer than PLAN_CFG_SMEM configurations)
 };
 
-__host__ __device__ inline size_t plan_smem_bytes(uint32_t static_bytes, uint32_t p_max, uint32_t T, uint32_t Z) {
+constexpr uint32_t PLAN_CFG_SMEM = 4096;
+
+__host__ __device__ inline size_t plan_smem_bytes(uint32_t static_bytes, uint32_t p_max, uint32_t T, uint32_t Z, uint32_t n_config) {
     const size_t R = (size_t)T * Z;
     size_t n = static_bytes;
+    if (n_config < 4096) n += sizeof(uint32_t) * ((size_t)n_config + 1);
     n += sizeof(SegRec) * (SAILOR_SEG_MAX * R + PLAN_PAD);               // padding digits, see walk_fast
     n += sizeof(double) * ((R + PLAN_PAD) * R + (R + PLAN_PAD) * Z + (size_t)SAILOR_SEG_MAX * T + 2 * (size_t)p_max * T);
     n += sizeof(uint32_t) * 2 * R;
@@ -250,6 +270,7 @@ __device__ __forceinline__ void carve(unsigned char* dyn, uint32_t static_bytes,
     a.uu = p;        p += (size_t)p_max * T;
     a.availv = reinterpret_cast<uint32_t*>(p);
     a.tz = a.availv + R;
+    a.chunk_tab = a.tz + R;
 }
 
 // Run of stage i: 0 = stage 0 with the embedding, 1 = one extra block, 2 = plain, 3 = final stage.
@@ -277,6 +298,8 @@ __device__ void build_config(const PlanParams& pp, const TabView& v, CfgShared& 
             cs.ar_steps = (double)(2 * (uint64_t)(k.D > 0 ? k.D - 1 : 0));     // ring all-reduce: 2(D-1) messages
             cs.ar_coef = k.D > 0 ? cs.ar_steps / (double)k.D : 0.0;
             cs.n_items = ipow64(R, k.nseg - 1);
+            cs.flat_base = pp.cfg_flat_base[c];
+            cs._pad_head = 0;
             cs.packed = 0;             // decided at the end of the build, and only for valid configurations
             cs.cur_config = c;
             uint32_t n_lower = 0;
@@ -655,7 +678,7 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
         uint64_t pf = 0;
 #pragma unroll
         for (int s = 0; s < NSEG - 1; ++s) pf = pf * R + dg[s];
-        item_flat = pp.cfg_flat_base[cs.cur_config] + pf * R;
+        item_flat = cs.flat_base + pf * R;
     }
     // ---- status of the prefix: node validity, memory, availability (integer work only) ------------
     bool p_inv = false, p_oom = false, p_over = false;
@@ -771,8 +794,149 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
         cnt.over_constr += n_ok - feas;
     }
     // rare: some lane's item holds a candidate that may enter the warp's list; walk again and offer
-    if (__any_sync(FULL, best < make_inf() && best <= top.thr_score))     // best == inf: the item has no feasible candidate
+    if (!pp.cost_only && __any_sync(FULL, best < make_inf() && best <= top.thr_score))     // best == inf: the item has no feasible candidate
         walk_offer<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, item_flat, top, lane);
+}
+
+// End of a pass, run by the one block that hands in its list last (no block waits for another: every block
+// adds one to Ctrl::blocks_done after its list is written, and the block that reads gridDim.x - 1 knows all the
+// lists are in memory).  Merges the blocks' lists, simulates the winners in full for the result records, copies
+// the counters next to them, hands `factor x best cost` to a following pass, and puts the counters back to
+// their starting values.  `v` is the block's own view of the static tables (already in shared memory); `s_hits`
+// (PLAN_WARPS lists) and `s_cnt` (R x SAILOR_K_MAX words) are scratch in shared memory.
+__device__ __noinline__ void finish_pass(const PlanParams& pp, const TabView& v, Hit (*s_hits)[SAILOR_K_MAX],
+                                         uint32_t* s_cnt, uint32_t* s_n) {
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = PLAN_WARPS;
+    const uint32_t n_partial = gridDim.x;
+    if (pp.cost_only) {
+        // the cheapest-plan pass of a budget-factor search: all the next pass needs is factor x the cheapest feasible
+        // cost, which every block has already folded into Ctrl::min_cost_bits (the same bits a full simulation of
+        // that plan gives: one operation order everywhere)
+        if (tid == 0) {
+            volatile Ctrl* live = pp.ctrl;
+            const bool any = live->stats[5] != 0;
+            const double cheapest = __longlong_as_double((long long)live->min_cost_bits);
+            pp.ctrl->budget = any ? mul_rn(pp.next_budget_factor, cheapest) : make_inf();
+            Ctrl* c = pp.ctrl;
+            c->work_counter = 0;
+            for (int q = 0; q < 7; ++q) c->stats[q] = 0;
+            c->wave_chunks = 0;
+            c->n_cfg_evaluated = 0;
+            c->min_cost_bits = COST_BITS_START;
+            c->n_found = 0;
+        }
+        return;
+    }
+    // The k best of all lists lie in the k lists with the best first elements: k elements (those heads) are at
+    // least as good as the k-th best head, and a list whose head is worse holds nothing better than its head.
+    // So: the k best heads first (one element per list, all loads in flight together), then only those lists.
+    // (Every block writes all k slots of its list, empty ones as (+inf, ~0); read them in L2, other SMs wrote them.)
+    auto load_hit = [&](uint32_t b, uint32_t slot, double& sc, uint64_t& fl) {
+        const double2 raw = __ldcg(reinterpret_cast<const double2*>(&pp.partial[(size_t)b * SAILOR_K_MAX + slot]));
+        sc = raw.x;
+        fl = (uint64_t)__double_as_longlong(raw.y);
+    };
+    WarpTopK top;
+    top.init();
+    const uint32_t rounds = (n_partial + PLAN_THREADS - 1) / PLAN_THREADS;
+    for (uint32_t r = 0; r < rounds; ++r) {
+        const uint32_t b = r * PLAN_THREADS + tid;
+        double hs = make_inf();
+        uint64_t hf = ~0ull;
+        if (b < n_partial) load_hit(b, 0, hs, hf);
+        top.offer(hf != ~0ull && (hs < top.thr_score || (hs == top.thr_score && hf < top.thr_flat)), hs, hf, pp.k, lane);
+    }
+    auto tree_merge = [&]() {          // the warps' lists into warp 0's, through shared memory
+        s_hits[warp][lane].score = top.score;
+        s_hits[warp][lane].flat = top.flat;
+        __syncthreads();
+        for (uint32_t step = 1; step < nw; step <<= 1) {
+            if ((warp & (2 * step - 1)) == 0 && warp + step < nw) {
+                top.merge_sorted(s_hits[warp + step][lane].score, s_hits[warp + step][lane].flat, pp.k, lane);
+                s_hits[warp][lane].score = top.score;
+                s_hits[warp][lane].flat = top.flat;
+            }
+            __syncthreads();
+        }
+    };
+    tree_merge();
+    const double cut_s = s_hits[0][pp.k - 1].score;          // the k-th best head (or (+inf, ~0): fewer than k lists hold anything)
+    const uint64_t cut_f = s_hits[0][pp.k - 1].flat;
+    uint32_t* sel = s_cnt;                                    // the chosen lists (at most k), then reused as counters
+    if (tid == 0) *s_n = 0;
+    __syncthreads();
+    for (uint32_t r = 0; r < rounds; ++r) {
+        const uint32_t b = r * PLAN_THREADS + tid;
+        double hs = make_inf();
+        uint64_t hf = ~0ull;
+        if (b < n_partial) load_hit(b, 0, hs, hf);
+        if (hf != ~0ull && (hs < cut_s || (hs == cut_s && hf <= cut_f))) sel[atomicAdd(s_n, 1u)] = b;
+    }
+    __syncthreads();
+    const uint32_t n_sel = *s_n;
+    top.init();
+    for (uint32_t q = warp; q < n_sel; q += nw) {
+        double ls = make_inf();
+        uint64_t lf = ~0ull;
+        if (lane < pp.k) load_hit(sel[q], lane, ls, lf);
+        top.merge_sorted(ls, lf, pp.k, lane);
+    }
+    __syncthreads();                                           // `sel` has been read by everyone
+    tree_merge();
+    if (warp == 0) {
+        const bool have = lane < pp.k && top.flat != ~0ull;
+        const uint32_t n = __popc(__ballot_sync(FULL, have));
+        if (lane == 0) *s_n = n;
+    }
+    __syncthreads();
+    // the winners are simulated in full for the result records, all at once: winner j by lane j / PLAN_WARPS of warp
+    // j % PLAN_WARPS (each is a long single-thread dependency chain of table look-ups; spread over the warps, at
+    // most four different plans share a warp's instruction stream)
+    const uint32_t n = *s_n;
+    {
+        const uint32_t j = lane * nw + warp;
+        if (lane < (SAILOR_K_MAX + nw - 1) / nw && j < n) {
+            sailor_result r;
+            r.flat = s_hits[0][j].flat;
+            r.score = s_hits[0][j].score;
+            r._pad = 0;
+            decode_flat(pp.sp, v.h->T, v.h->Z, r.flat, &r.plan);
+            const SimOut o = simulate_record(v, pp.avail, r.plan, s_cnt + j, SAILOR_K_MAX);
+            r.t_iter = o.t_iter;
+            r.cost = o.cost;
+            r.peak_mem = o.peak_mem;
+            r.status = o.status;
+            pp.out->results[j] = r;
+            if (j == 0 && pp.next_budget_factor > 0.0) pp.ctrl->budget = mul_rn(pp.next_budget_factor, o.cost);
+        }
+    }
+    if (tid == 0) {
+        if (n == 0 && pp.next_budget_factor > 0.0) pp.ctrl->budget = make_inf();
+        // the counters as they stand (every block's contribution is in: atomics, then its blocks_done increment)
+        volatile Ctrl* live = pp.ctrl;
+        Ctrl c;
+        c.work_counter = live->work_counter;
+        c.blocks_done = live->blocks_done;
+        for (int q = 0; q < 7; ++q) c.stats[q] = live->stats[q];
+        c.wave_chunks = live->wave_chunks;
+        c.n_cfg_evaluated = live->n_cfg_evaluated;
+        c.min_cost_bits = live->min_cost_bits;
+        c.error = live->error;
+        c.n_found = n;
+        pp.out->ctrl = c;
+    }
+    __syncthreads();                   // the budget of the next pass is written (thread 0 or warp 0's lane 0)
+    if (tid == 0) {
+        pp.out->ctrl.budget = *reinterpret_cast<volatile double*>(&pp.ctrl->budget);
+        Ctrl* live = pp.ctrl;          // back to the starting values; the budget stays for the next pass
+        live->work_counter = 0;
+        for (int q = 0; q < 7; ++q) live->stats[q] = 0;
+        live->wave_chunks = 0;
+        live->n_cfg_evaluated = 0;
+        live->min_cost_bits = COST_BITS_START;
+        if (!(pp.next_budget_factor > 0.0)) live->error = 0;   // a following pass of the same call keeps the flag
+        live->n_found = 0;
+    }
 }
 
 template <int OBJ, bool CONSTR>
@@ -812,6 +976,12 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
         a.availv[d] = pp.avail[d];
         a.tz[d] = (d % T) | ((d / T) << 8);
     }
+    // the chunk offsets are searched once per run of chunks and read once per chunk: keep a copy next to the tables
+    // (the waves of a degree-order search rewrite them between launches, so every launch copies them afresh)
+    const bool tab_local = pp.n_config < PLAN_CFG_SMEM;
+    if (tab_local)
+        for (uint32_t x = tid; x <= pp.n_config; x += PLAN_THREADS) a.chunk_tab[x] = pp.cfg_chunk_start[x];
+    const uint32_t* chunk_start = tab_local ? a.chunk_tab : pp.cfg_chunk_start;
     WarpTopK top;
     top.init();
     if (pp.carry_lists && warp == 0) {     // a later wave of one search: go on from the list this block left behind
@@ -829,17 +999,31 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
     __syncthreads();
 
     uint32_t c = 0;     // configuration of the current chunk (monotone within a batch)
+    bool first_round = true;
     for (;;) {
         if (tid == 0) {
-            // guided self-scheduling: long runs of consecutive chunks first (a block then stays inside
-            // one configuration and rebuilds its tables rarely), single chunks at the end (even finish)
+            // every block starts with the chunk of its own number (no counter involved: small searches are bound by
+            // such round trips); the rest is handed out by guided self-scheduling: long runs of consecutive chunks
+            // first (a block then stays inside one configuration and changes its tables rarely), single chunks at
+            // the end (even finish)
             const uint32_t n_chunks = chunk_hi - chunk_lo;
-            const uint32_t seen = *reinterpret_cast<volatile unsigned int*>(&pp.ctrl->work_counter);
-            const uint32_t left = seen < n_chunks ? n_chunks - seen : 0u;
-            const uint32_t len = max(1u, left / (gridDim.x * 4u));
-            cs.next_chunk = chunk_lo + atomicAdd(&pp.ctrl->work_counter, len);
-            cs.batch_len = len;
+            if (first_round) {
+                cs.next_chunk = chunk_lo + min(blockIdx.x, n_chunks);
+                cs.batch_len = 1;
+            } else if (n_chunks <= gridDim.x) {
+                cs.next_chunk = chunk_hi;                    // every chunk had a block of its own
+                cs.batch_len = 1;
+            } else {
+                const uint32_t rest = n_chunks - gridDim.x;
+                const uint32_t seen = *reinterpret_cast<volatile unsigned int*>(&pp.ctrl->work_counter);
+                const uint32_t left = seen < rest ? rest - seen : 0u;
+                const uint32_t len = max(1u, left / (gridDim.x * 4u));
+                const uint32_t got = atomicAdd(&pp.ctrl->work_counter, len);
+                cs.next_chunk = got < rest ? chunk_lo + gridDim.x + got : chunk_hi;
+                cs.batch_len = len;
+            }
         }
+        first_round = false;
         __syncthreads();
         const uint32_t first = cs.next_chunk;
         if (first >= chunk_hi) break;
@@ -848,21 +1032,21 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             uint32_t lo = 0, hi = pp.n_config;
             while (hi - lo > 1) {
                 const uint32_t mid = (lo + hi) >> 1;
-                if (pp.cfg_chunk_start[mid] <= first) lo = mid; else hi = mid;
+                if (chunk_start[mid] <= first) lo = mid; else hi = mid;
             }
             c = lo;
         }
         for (uint32_t ch = first; ch < end; ++ch) {
-            while (ch >= pp.cfg_chunk_start[c + 1]) ++c;
+            while (ch >= chunk_start[c + 1]) ++c;
             if (cs.cur_config != c) {
                 if (pp.cfg_best && cs.cur_config != 0xffffffffu) flush_cfg_best(pp, cnt, cs.cur_config, lane);
                 __syncthreads();
                 if (pp.cfg_cache) load_config(pp, cs, a, R, c);
                 else build_config(pp, v, cs, a, c);
             }
-            const uint32_t q = (ch - pp.cfg_chunk_start[c]) * PLAN_THREADS + tid;    // < R^3 + 256 <= 2^18 + 256
+            const uint32_t q = (ch - chunk_start[c]) * PLAN_THREADS + tid;    // < R^3 + 256 <= 2^18 + 256
             const bool active = q < (cs.packed ? cs.live_items : cs.n_items);
-            const uint64_t item_flat = pp.cfg_flat_base[c] + (uint64_t)q * R;
+            const uint64_t item_flat = cs.flat_base + (uint64_t)q * R;
             if (!cs.valid) {
                 // every candidate of the configuration is invalid; count those in range
                 if (active) {
@@ -926,6 +1110,22 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             pp.partial[(size_t)blockIdx.x * SAILOR_K_MAX + lane].flat = top.flat;
         }
         if (lane == 0) pp.partial_n[blockIdx.x] = n;
+    }
+    // hand the list in; the block that does so last ends the launch (and, in a pass's final launch, the pass)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int before = atomicAdd(&pp.ctrl->blocks_done, 1u);
+        cs.next_chunk = (before == gridDim.x - 1) ? 1u : 0u;
+        if (before == gridDim.x - 1) {
+            pp.ctrl->blocks_done = 0;                    // the next launch counts from zero
+            if (!pp.finish) pp.ctrl->work_counter = 0;   // (a finishing launch resets all counters below)
+        }
+    }
+    __syncthreads();
+    if (cs.next_chunk && pp.finish) {
+        __threadfence();
+        finish_pass(pp, v, s_hits, reinterpret_cast<uint32_t*>(a.rec), &cs.batch_len);
     }
 }
 
@@ -1134,106 +1334,6 @@ __global__ void __launch_bounds__(WAVE_THREADS) wave_step_kernel(const __grid_co
     __syncthreads();
     if (tid < 3 && s_closed[tid]) atomicAdd(&wp.ctrl->stats[tid], s_closed[tid]);
     if (tid == 0) wp.ctrl->n_cfg_evaluated += s_eval;
-}
-
-// Merge the blocks' lists, then simulate the winners in full for the result records.
-struct MergeParams {
-    const unsigned char* blob;
-    const uint16_t* avail;
-    const Hit* partial;
-    const uint32_t* partial_n;
-    Ctrl* ctrl;
-    sailor_result* results;            // [k] device
-    SpaceDesc sp;
-    uint32_t n_partial, k, obj;
-    double budget_factor;              // > 0: write ctrl->budget = factor * best cost for the next pass
-};
-
-constexpr int MERGE_THREADS = 512;
-
-__global__ void __launch_bounds__(MERGE_THREADS) merge_kernel(const __grid_constant__ MergeParams mp) {
-    extern __shared__ __align__(16) unsigned char dyn[];      // the static tables
-    __shared__ Hit s_hits[MERGE_THREADS / 32][SAILOR_K_MAX];
-    __shared__ uint64_t mbar;
-    __shared__ uint32_t s_n;
-    __shared__ uint32_t s_cnt[R_MAX][MERGE_THREADS / 32];   // per-digit GPU counters of each warp's record
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = MERGE_THREADS / 32;
-    const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(mp.blob)->static_bytes;
-    if (!bulk_load(dyn, mp.blob, static_bytes, &mbar)) {
-        if (tid == 0) atomicExch(&mp.ctrl->error, 1u);
-        for (uint32_t x = tid; x < static_bytes / 16; x += MERGE_THREADS)
-            reinterpret_cast<uint4*>(dyn)[x] = reinterpret_cast<const uint4*>(mp.blob)[x];
-        __syncthreads();
-    }
-    WarpTopK top;
-    top.init();
-    // every warp takes every nw-th block's list; four lists are fetched before they are merged, so
-    // that the loads overlap instead of queueing behind one another
-    for (uint32_t b0 = warp; b0 < mp.n_partial; b0 += 4 * nw) {
-        Hit mine[4];
-        uint32_t cnt[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t b = b0 + u * nw;
-            cnt[u] = b < mp.n_partial ? mp.partial_n[b] : 0u;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const uint32_t b = b0 + u * nw;
-            mine[u].score = make_inf();
-            mine[u].flat = ~0ull;
-            if (lane < cnt[u]) mine[u] = mp.partial[(size_t)b * SAILOR_K_MAX + lane];
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (cnt[u]) top.merge_sorted(mine[u].score, mine[u].flat, mp.k, lane);
-    }
-    // tree merge of the warps' lists through shared memory
-    s_hits[warp][lane].score = top.score;
-    s_hits[warp][lane].flat = top.flat;
-    __syncthreads();
-    for (uint32_t step = 1; step < nw; step <<= 1) {
-        if ((warp & (2 * step - 1)) == 0 && warp + step < nw) {
-            top.merge_sorted(s_hits[warp + step][lane].score, s_hits[warp + step][lane].flat, mp.k, lane);
-            s_hits[warp][lane].score = top.score;
-            s_hits[warp][lane].flat = top.flat;
-        }
-        __syncthreads();
-    }
-    if (warp == 0) {
-        const bool have = lane < mp.k && top.flat != ~0ull;
-        const uint32_t n = __popc(__ballot_sync(FULL, have));
-        if (lane == 0) s_n = n;
-    }
-    __syncthreads();
-    // the winners are simulated in full for the result records, one per warp at a time (each is a
-    // long single-thread dependency chain; different plans would diverge inside one warp)
-    const uint32_t n = s_n;
-    TabView v;
-    v.bind(dyn, mp.blob);
-    for (uint32_t j = warp; j < n; j += nw) {
-        if (lane == 0) {
-            sailor_result r;
-            r.flat = s_hits[0][j].flat;
-            r.score = s_hits[0][j].score;
-            r._pad = 0;
-            decode_flat(mp.sp, v.h->T, v.h->Z, r.flat, &r.plan);
-            const SimOut o = simulate_record(v, mp.avail, r.plan, &s_cnt[0][warp], MERGE_THREADS / 32);
-            r.t_iter = o.t_iter;
-            r.cost = o.cost;
-            r.peak_mem = o.peak_mem;
-            r.status = o.status;
-            mp.results[j] = r;
-            if (j == 0) {
-                mp.ctrl->n_found = n;
-                if (mp.budget_factor > 0.0) mp.ctrl->budget = mul_rn(mp.budget_factor, o.cost);
-            }
-        }
-    }
-    if (n == 0 && tid == 0) {
-        mp.ctrl->n_found = 0;
-        if (mp.budget_factor > 0.0) mp.ctrl->budget = make_inf();
-    }
 }
 
 }  // namespace sailor

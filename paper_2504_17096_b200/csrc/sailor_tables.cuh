@@ -49,7 +49,12 @@ struct alignas(16) TabHdr {
     uint32_t off_cmp_mem;                         // u64 [c][tp][mbs][rc][2]        model + working bytes, bytes kept per in-flight microbatch
     uint32_t off_cmp_fb;                          // f64 [c][type][tp][mbs][rc]     f + b (+ f with recomputation)
     uint32_t off_cmp_upd;                         // f64 [c][type][tp]              update time
-    uint32_t _pad[3];
+    // tables of the explicit-batch kernel (sailor_batch.cuh)
+    uint32_t off_piece;                           // PieceRec [c][type][tp][mbs][rc]
+    uint32_t off_lnk_intra2, off_lnk_inter2;      // f64 [digit][mbs]   2 x one-way message time of the link
+    uint32_t off_lnk_zone2;                       // f64 [zone][zone][mbs]
+    uint32_t heads_ok;                            // bit i: tp_values[i] divides the number of attention heads
+    uint32_t _pad[2];
 };
 static_assert(sizeof(TabHdr) % 16 == 0, "header must keep the arrays 16-byte aligned");
 

@@ -19,6 +19,47 @@ def split_range(n: int, world: int, rank: int) -> Tuple[int, int]:
     return n * rank // world, n * (rank + 1) // world
 
 
+def subspace_costs(w) -> List[Tuple[int, float]]:
+    """(candidates, relative cost of one candidate) of each pipeline depth's sub-space, in flat-index order.
+    A candidate costs its fixed part plus one step per stage of the last segment (the search keeps the running
+    sums of the other segments per prefix), which is how the measured per-depth times of the search scale."""
+    base = len(w.mbs_idx) * len(w.tp_idx) * len(w.rc_values) * len(w.d_values)
+    out = []
+    for p in w.p_values:
+        nseg = min(p, w.seg_max)
+        last = p - ((nseg - 1) * p + nseg - 1) // nseg          # stages of the last segment
+        out.append((base * w.radix ** nseg, COST_FIXED + COST_PER_STAGE * last))
+    return out
+
+
+COST_FIXED, COST_PER_STAGE = 9.0, 1.0
+
+
+def split_by_cost(parts: Sequence[Tuple[int, float]], world: int, rank: int) -> Tuple[int, int]:
+    """Contiguous [lo, hi) of rank `rank`: the flat range [0, sum of sizes) cut where the estimated cost
+    (size x weight, summed over consecutive parts) reaches rank / world and (rank + 1) / world of the total.
+    The ranges of all ranks tile the space exactly."""
+    if world < 1 or not 0 <= rank < world:
+        raise ValueError("bad world/rank")
+    total = sum(n * wgt for n, wgt in parts)
+    n_all = sum(n for n, _ in parts)
+
+    def cut(j: int) -> int:
+        if j <= 0:
+            return 0
+        if j >= world:
+            return n_all
+        want, flat, cost = total * j / world, 0, 0.0
+        for n, wgt in parts:
+            if cost + n * wgt >= want and wgt > 0:
+                return min(n_all, flat + int((want - cost) / wgt))
+            flat += n
+            cost += n * wgt
+        return n_all
+
+    return cut(rank), cut(rank + 1)
+
+
 def merge_topk(lists: Sequence[Sequence[Tuple[float, int]]], k: int) -> List[Tuple[float, int]]:
     """Merge per-range lists of (score, flat) pairs; ascending, ties to the lowest flat index."""
     allp = [tuple(p) for l in lists for p in l]

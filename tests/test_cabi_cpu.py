@@ -28,8 +28,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 def test_struct_sizes_match_the_header(lib):
     assert C.sizeof(B.PlanRec) == 72 and C.sizeof(B.Run) == 4
-    assert C.sizeof(B.Result) == 120 and C.sizeof(B.Stats) == 96
-    assert C.sizeof(B.Space) == 152 and C.sizeof(B.Objective) == 32
+    assert C.sizeof(B.Result) == 120 and C.sizeof(B.Stats) == 104
+    assert C.sizeof(B.Space) == 152 and C.sizeof(B.Objective) == 32 and C.sizeof(B.IssueRates) == 48
 
 
 def test_error_strings_and_null_arguments(lib):
@@ -46,6 +46,15 @@ def test_error_strings_and_null_arguments(lib):
     assert lib.sailor_space_size(None, None, C.byref(n)) == B.E_ARG
     assert lib.sailor_plan(None, None, None, 1, None, None, None) == B.E_ARG
     assert lib.sailor_last_cuda_error(None) == 0
+    assert lib.sailor_measure_issue_rates(0, None, 3, None) == B.E_ARG
+    assert lib.sailor_measure_issue_rates(0, None, 0, C.byref(B.IssueRates())) == B.E_ARG
+
+
+def test_library_reads_no_environment_variable():
+    """The interface is plain structs: nothing in the library's sources looks at the environment."""
+    csrc = os.path.join(ROOT, "paper_2504_17096_b200", "csrc")
+    for f in os.listdir(csrc):
+        assert "getenv" not in open(os.path.join(csrc, f)).read(), f
 
 
 def test_product_does_not_import_the_oracle():

@@ -30,14 +30,9 @@ def _index_mode(request, monkeypatch):
     with each way of enumerating a stage's work (a thread per reachable count vector for all its types, which is the
     default up to four GPU types; a thread per reachable count vector and type; a thread per table entry)."""
     index, _, enum = request.param.partition("-")
-    if index == "auto":
-        monkeypatch.delenv("SAILOR_DP_INDEX", raising=False)
-    else:
-        monkeypatch.setenv("SAILOR_DP_INDEX", index)
-    if enum:
-        monkeypatch.setenv("SAILOR_DP_ENUM", enum)
-    else:
-        monkeypatch.delenv("SAILOR_DP_ENUM", raising=False)
+    flags = {"auto": 0, "dense": B.DP_FLAG_INDEX_DENSE, "compact": B.DP_FLAG_INDEX_COMPACT}[index]
+    flags |= {"": 0, "types": B.DP_FLAG_ENUM_BY_TYPE, "entries": B.DP_FLAG_ENUM_BY_ENTRY}[enum]
+    monkeypatch.setattr(B, "dp_default_flags", flags)
     return index
 
 
@@ -257,7 +252,9 @@ def test_dp_argument_checks():
             B.sailor_plan_dp(cx.ctx, cx.space, [[0]], 33)
         assert e.value.code == B.E_RANGE
         for obj in (B.Objective(B.OBJ_MIN_COST, 0, 0.0, 0.0, 0.0), B.Objective(B.OBJ_MAX_THROUGHPUT, B.FLAG_EVAL_ALL, 0.0, 0.0, 0.0),
-                    B.Objective(B.OBJ_MAX_THROUGHPUT, 0, 0.0, 0.0, 1.2)):
+                    B.Objective(B.OBJ_MAX_THROUGHPUT, 0, 0.0, 0.0, 1.2),
+                    B.Objective(B.OBJ_MAX_THROUGHPUT, B.DP_FLAG_INDEX_DENSE | B.DP_FLAG_INDEX_COMPACT, 0.0, 0.0, 0.0),
+                    B.Objective(B.OBJ_MAX_THROUGHPUT, B.DP_FLAG_ENUM_BY_TYPE | B.DP_FLAG_ENUM_BY_ENTRY, 0.0, 0.0, 0.0)):
             with pytest.raises(B.SailorError) as e:
                 B.sailor_plan_dp(cx.ctx, cx.space, [[0]], 4, obj=obj)
             assert e.value.code == B.E_ARG

@@ -370,6 +370,38 @@ def test_plan_argument_errors(make_ctx):
     bad = B.make_space(w)
     bad.seg_max = 5
     assert L.sailor_plan(cx.ctx, C.byref(bad), C.byref(obj), 1, res, C.byref(n), None) == B.E_RANGE
+    for flags in (8, 0x100, 1 << 31):                    # flags this entry point does not know
+        odd = B.make_objective(w, flags=flags)
+        assert L.sailor_plan(cx.ctx, C.byref(cx.space), C.byref(odd), 1, res, C.byref(n), None) == B.E_ARG
+
+
+def test_stats_report_transfer_times_and_launches(make_ctx):
+    """One launch per pass (the search kernel's last block merges), and the device times of the availability
+    upload and of the result read-back beside the kernel time."""
+    w = W.config2()
+    cx = make_ctx(w)
+    obj = B.make_objective(w)
+    B.sailor_plan(cx.ctx, cx.space, obj, 4)
+    B.sailor_set_availability(cx.ctx, w.avail)
+    res, st = B.sailor_plan(cx.ctx, cx.space, obj, 4)
+    assert st.n_launches == 2 and len(res) == 4           # two passes: cheapest plan, then the budget
+    assert 0.0 < st.h2d_ms < 5.0 and 0.0 < st.d2h_ms < 5.0 and 0.0 < st.kernel_ms < 50.0
+    res1, st1 = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, factor=0.0), 4)
+    assert st1.n_launches == 1
+    assert st1.h2d_ms == st.h2d_ms                        # no new upload: the last one's time stays
+
+
+def test_issue_rate_measurement_is_plausible(torch_cuda):
+    """The instruction streams behind the roofline's ceiling: an SM cannot issue more than four warp-instructions
+    a cycle, the FP64 pipe runs at about half the FP32 rate, and the streams come close to those limits."""
+    r = B.sailor_measure_issue_rates(0, 0, 3)
+    props = torch_cuda.cuda.get_device_properties(0)
+    limit = props.multi_processor_count * 4 * props.clock_rate * 1e3      # schedulers x max clock
+    assert r.sm_count == props.multi_processor_count
+    assert 0.5 * limit < r.ffma_warp_inst_per_s <= 1.02 * limit
+    assert 0.2 * limit < r.imad_warp_inst_per_s <= 1.02 * limit
+    assert 0.2 * limit < r.dadd_warp_inst_per_s <= 0.55 * limit
+    assert r.warp_inst_per_run == r.sm_count * 4 * 8 * 2048 * 128
 
 
 def test_plan_range_split_merges_to_full(make_ctx):

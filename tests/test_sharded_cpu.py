@@ -21,6 +21,29 @@ def test_split_range_tiles_exactly():
         sharding.split_range(10, 2, 2)
 
 
+def test_split_by_cost_tiles_exactly_and_balances_the_estimate():
+    from paper_2504_17096_b200 import workloads as W
+    for w in (W.config5(), W.config3(), W.config1()):
+        parts = sharding.subspace_costs(w)
+        assert sum(n for n, _ in parts) == w.space_size()
+        total = sum(n * c for n, c in parts)
+        for world in (1, 2, 3, 8):
+            edges = [sharding.split_by_cost(parts, world, r) for r in range(world)]
+            assert edges[0][0] == 0 and edges[-1][1] == w.space_size()
+            assert all(a[1] == b[0] for a, b in zip(edges[:-1], edges[1:]))
+
+            def cost(lo, hi):          # estimated cost of [lo, hi)
+                out, at = 0.0, 0
+                for n, c in parts:
+                    out += max(0, min(hi, at + n) - max(lo, at)) * c
+                    at += n
+                return out
+            for lo, hi in edges:
+                assert abs(cost(lo, hi) - total / world) <= max(c for _, c in parts) * 2
+    with pytest.raises(ValueError):
+        sharding.split_by_cost([(10, 1.0)], 2, 2)
+
+
 def test_merge_topk_breaks_ties_by_flat_index():
     a = [(1.0, 9), (2.0, 3)]
     b = [(1.0, 4), (3.0, 1)]
