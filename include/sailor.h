@@ -392,9 +392,25 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
  * to value up to rounding.  The objective is iteration time (o->kind must be MAX_THROUGHPUT, no
  * flags other than SAILOR_DP_FLAG_*, no budget factor).  A budget or a minimum throughput in `o` is checked on the plan the
  * recursion returns for a problem, by the simulator's cost and time (Sec. 4.2: a configuration
- * counts only when it is within the constraint); a problem whose plan fails it drops out.  The
- * straggler-guessing budget loop of Sec. 4.2.3, which steers the recursion itself by the remaining
- * budget, is not implemented.
+ * counts only when it is within the constraint); a problem whose plan fails it drops out.
+ *
+ * With SAILOR_DP_FLAG_BUDGET_LOOP the budget also steers the recursion, the way Sec. 4.2.3 ("Adding a
+ * monetary cost constraint") and the second half of the listing describe.  A stage is charged
+ *     C_i = rate_i * (N_b * t_straggler) + C_comm_i
+ * (rate_i = (double)(D * tp) * price per second of its GPUs; C_comm_i = (double)(2 * N_b * D * p2p_bytes) * egress
+ * of its message to the next stage when that crosses zones) with an ASSUMED straggler: first the stage's own time t.
+ * The stages after it are solved with what is left, C_rem = C_cur - C_i (nothing is tried when C_rem <= 0).  If
+ * their straggler is not slower than the assumed one, the candidate counts when C_i + their charges <= C_cur; if it
+ * is slower, the stage is charged again with that straggler and they are solved again with the smaller remainder.
+ * The last stage is its own straggler and counts when its charge is within its limit.  Candidates combine and
+ * compare as above.  The remaining budget is an argument of the recursion (a state reached with two different
+ * remainders is solved twice), so the tables above do not apply: each problem is walked depth-first by one GPU
+ * thread, problems in parallel.  The work can grow as T^P: a branch is cut when what is left cannot pay the
+ * cheapest conceivable rest of the pipeline (this changes no result), and a problem that needs more than 2^24 calls
+ * of the recursion is given up and counted in n_unfinished.  The charge underestimates the simulator's cost (it
+ * leaves out warm-up, cool-down, synchronisation and update time, as the paper's simplification does), so the
+ * check of the simulator's cost against the budget still follows, as without the flag.  n_states then counts the
+ * calls of the recursion.
  *
  * On the device every problem is a dense table over its states (stage, type, zone position,
  * stages per type already placed in that zone; a type with room for all P stages in a zone is not
@@ -410,6 +426,10 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
 #define SAILOR_DP_FLAG_INDEX_COMPACT  0x200u
 #define SAILOR_DP_FLAG_ENUM_BY_TYPE   0x400u
 #define SAILOR_DP_FLAG_ENUM_BY_ENTRY  0x800u
+/* Steer the recursion by the budget (Sec. 4.2.3) instead of only checking it on the plan the recursion returns: see
+ * sailor_plan_dp.  Needs budget_usd_per_iter > 0; pipelines of at most SAILOR_DP_BUDGET_P_MAX stages. */
+#define SAILOR_DP_FLAG_BUDGET_LOOP    0x1000u
+#define SAILOR_DP_BUDGET_P_MAX        32
 
 typedef struct sailor_zone_order {
     uint8_t n;                          /* 1 .. SAILOR_Z_MAX zones, each at most once                */
@@ -439,7 +459,8 @@ typedef struct sailor_dp_stats {
     uint64_t n_states;                  /* table entries filled (all problems, all stages)            */
     uint64_t workspace_used;            /* bytes of the largest batch                                 */
     float    kernel_ms;
-    uint32_t n_launches, n_batches, _pad;
+    uint32_t n_launches, n_batches;
+    uint32_t n_unfinished;              /* SAILOR_DP_FLAG_BUDGET_LOOP: problems given up (too many calls)   */
 } sailor_dp_stats;
 
 /* Solve every problem of `s` x `orders` and return the k best plans within the constraint by
@@ -447,7 +468,7 @@ typedef struct sailor_dp_stats {
  * `stats` may be NULL.  Uses the availability last set.  `workspace_bytes` bounds the device memory
  * of the tables (0 = 8 GiB); it is allocated on first use and kept by the context (grow-only).
  * Errors: E_ARG (null, k == 0, n_orders == 0, a zone twice or out of range, an objective other
- * than plain MAX_THROUGHPUT), E_RANGE (k >
+ * than plain MAX_THROUGHPUT, the budget loop without a budget), E_RANGE (k >
  * SAILOR_K_MAX, space limits as sailor_plan, a single problem whose tables exceed the workspace or
  * 2^31 entries per stage), E_NOMEM, E_CUDA. */
 int sailor_plan_dp(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders, uint32_t n_orders,

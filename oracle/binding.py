@@ -133,6 +133,12 @@ class OrcMixedPlan(C.Structure):
                 ("stage", OrcMixedStage * STAGES_MAX)]
 
 
+class OrcMixedSpace(C.Structure):
+    _fields_ = [("n_p", C.c_uint32), ("n_mbs", C.c_uint32), ("n_rc", C.c_uint32), ("n_d", C.c_uint32),
+                ("seg_max", C.c_uint32), ("granularity", C.c_uint32), ("p_values", _u32p), ("mbs_idx", _u32p),
+                ("rc_values", _u32p), ("d_values", _u32p), ("tp_idx_of_type", _u32p)]
+
+
 _lib = None
 
 
@@ -169,6 +175,17 @@ def lib():
         L.orc_simulate_mixed_batch.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedPlan), C.c_uint64,
                                                _u32p, _dp, _dp, _u64p]
         L.orc_simulate_mixed_batch.restype = None
+        L.orc_mixed_n_comb.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedSpace), C.c_uint32]
+        L.orc_mixed_n_comb.restype = C.c_uint64
+        L.orc_mixed_comb.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedSpace), C.c_uint32, C.c_uint64, _u32p]
+        L.orc_mixed_comb.restype = C.c_int
+        L.orc_mixed_space_size.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedSpace)]
+        L.orc_mixed_space_size.restype = C.c_uint64
+        L.orc_mixed_decode.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedSpace), C.c_uint64, C.POINTER(OrcMixedPlan)]
+        L.orc_mixed_decode.restype = C.c_int
+        L.orc_search_mixed.argtypes = [C.POINTER(OrcInputs), C.POINTER(OrcMixedSpace), C.POINTER(OrcObjective),
+                                       C.c_uint64, C.c_uint64, C.c_uint32, C.POINTER(OrcHit), C.POINTER(OrcCounts)]
+        L.orc_search_mixed.restype = C.c_uint32
         _lib = L
     return _lib
 
@@ -376,6 +393,58 @@ class Oracle:
         plan = OrcPlan.from_buffer_copy(out.plan)
         return {"value": out.value, "charged_cost": out.charged_cost, "types": list(plan.type[:P]),
                 "zones": list(plan.zone[:P]), "plan": plan, "n_states": int(out.n_states)}
+
+    # -- search over plans with mixed replicas ----------------------------------------------
+    def mixed_space(self, granularity: int, tp_idx_of_type: Sequence[int], *, p_values=None, mbs_idx=None,
+                    rc_values=None, d_values=None, seg_max=None) -> OrcMixedSpace:
+        """The workload's radix lists (or the given ones) as a space of plans with mixed replicas."""
+        w = self.w
+        s = OrcMixedSpace()
+        lists = {"p_values": w.p_values if p_values is None else p_values,
+                 "mbs_idx": w.mbs_idx if mbs_idx is None else mbs_idx,
+                 "rc_values": w.rc_values if rc_values is None else rc_values,
+                 "d_values": w.d_values if d_values is None else d_values,
+                 "tp_idx_of_type": tp_idx_of_type}
+        for name, value in lists.items():
+            a, p = _arr(value, np.uint32, _u32p)
+            self._keep.append(a)
+            setattr(s, name, p)
+        s.n_p, s.n_mbs, s.n_rc, s.n_d = (len(lists[k]) for k in ("p_values", "mbs_idx", "rc_values", "d_values"))
+        s.seg_max = w.seg_max if seg_max is None else seg_max
+        s.granularity = granularity
+        return s
+
+    def mixed_n_comb(self, space: OrcMixedSpace, D: int) -> int:
+        return int(lib().orc_mixed_n_comb(C.byref(self.inputs), C.byref(space), D))
+
+    def mixed_comb(self, space: OrcMixedSpace, D: int, c: int):
+        u = (C.c_uint32 * 8)()
+        if lib().orc_mixed_comb(C.byref(self.inputs), C.byref(space), D, c, u) != 0:
+            raise IndexError(c)
+        return list(u[: self.w.n_types])
+
+    def mixed_space_size(self, space: OrcMixedSpace) -> int:
+        return int(lib().orc_mixed_space_size(C.byref(self.inputs), C.byref(space)))
+
+    def mixed_decode(self, space: OrcMixedSpace, flat: int) -> dict:
+        pl = OrcMixedPlan()
+        if lib().orc_mixed_decode(C.byref(self.inputs), C.byref(space), flat, C.byref(pl)) != 0:
+            raise IndexError(flat)
+        return {"P": pl.P, "mbs_idx": pl.mbs_idx, "rc": pl.rc, "D": pl.D,
+                "stages": [{"zone": pl.stage[i].zone,
+                            "groups": [(pl.stage[i].group[q].type, pl.stage[i].group[q].tp_idx, pl.stage[i].group[q].count)
+                                       for q in range(pl.stage[i].n_groups)]} for i in range(pl.P)]}
+
+    def search_mixed(self, space: OrcMixedSpace, kind: int, k: int, *, budget: float = 0.0, min_rate: float = 0.0,
+                     lo: int = 0, hi: Optional[int] = None):
+        hi = self.mixed_space_size(space) if hi is None else hi
+        obj = OrcObjective(kind, 0, budget, min_rate)
+        hits = (OrcHit * max(k, 1))()
+        cnt = OrcCounts()
+        n = lib().orc_search_mixed(C.byref(self.inputs), C.byref(space), C.byref(obj), lo, hi, k, hits, C.byref(cnt))
+        out = [dict(flat=int(h.flat), score=h.score, t_iter=h.t_iter, cost=h.cost, peak_mem=int(h.peak_mem))
+               for h in hits[:n]]
+        return out, {f: (getattr(cnt, f) if f == "min_cost" else int(getattr(cnt, f))) for f, _ in OrcCounts._fields_}
 
     def plan(self, k: int, *, lo: int = 0, hi: Optional[int] = None):
         """The workload's own objective, with the cheapest-feasible budget rule when it has one:

@@ -992,3 +992,126 @@ void orc_simulate_mixed_batch(const orc_inputs* in, const orc_mixed_plan* plans,
         peak_mem[j] = o.peak_mem;
     }
 }
+
+/* ---- searching over plans with mixed replicas (Sec. 4.2.2, "Implementation") ----------------------------- */
+
+static uint32_t mixed_units(const orc_mixed_space* sp, uint32_t D) {
+    return (sp->granularity >= 1 && D % sp->granularity == 0) ? sp->granularity : D;
+}
+
+/* Walks the combinations in DESCENDING lexicographic order (all replicas on type 0 comes first, so that with one unit
+ * combination c is "everything on type c"), plainly: type 0's units from the most down, inside that type 1's, and so
+ * on, the last type taking what is left; tuples with more than ORC_GROUPS_MAX non-zero entries are skipped.
+ * Returns how many there are; the tuple of index `want` is left in `u`. */
+static uint64_t walk_combs(uint32_t T, uint32_t units, uint64_t want, uint32_t* u, int* found) {
+    uint64_t n = 0;
+    uint32_t cur[ORC_DP_T_MAX];
+    for (uint32_t t = 0; t < ORC_DP_T_MAX; ++t) cur[t] = units;
+    for (;;) {
+        uint32_t used = 0, nonzero = 0;
+        for (uint32_t t = 0; t + 1 < T; ++t) { used += cur[t]; nonzero += cur[t] != 0; }
+        if (used <= units) {
+            const uint32_t last = units - used;
+            if (nonzero + (last != 0) <= ORC_GROUPS_MAX) {
+                if (n == want && u) {
+                    for (uint32_t t = 0; t + 1 < T; ++t) u[t] = cur[t];
+                    u[T - 1] = last;
+                    if (found) *found = 1;
+                }
+                n++;
+            }
+        }
+        /* previous tuple of the first T - 1 entries in lexicographic order: the last of them fastest */
+        int t = (int)T - 2;
+        while (t >= 0 && cur[t] == 0) { cur[t] = units; t--; }
+        if (t < 0) break;
+        cur[t]--;
+    }
+    return n;
+}
+
+uint64_t orc_mixed_n_comb(const orc_inputs* in, const orc_mixed_space* sp, uint32_t D) {
+    return walk_combs(in->n_types, mixed_units(sp, D), ~0ull, NULL, NULL);
+}
+
+int orc_mixed_comb(const orc_inputs* in, const orc_mixed_space* sp, uint32_t D, uint64_t c, uint32_t* units_per_type) {
+    int found = 0;
+    walk_combs(in->n_types, mixed_units(sp, D), c, units_per_type, &found);
+    return found ? 0 : -1;
+}
+
+static uint32_t mixed_nseg(const orc_mixed_space* sp, uint32_t P) { return P < sp->seg_max ? P : sp->seg_max; }
+
+uint64_t orc_mixed_space_size(const orc_inputs* in, const orc_mixed_space* sp) {
+    uint64_t n = 0;
+    for (uint32_t jp = 0; jp < sp->n_p; ++jp)
+        for (uint32_t jd = 0; jd < sp->n_d; ++jd) {
+            const uint64_t radix = (uint64_t)in->n_zones * orc_mixed_n_comb(in, sp, sp->d_values[jd]);
+            n += (uint64_t)sp->n_mbs * sp->n_rc * ipow_u64(radix, mixed_nseg(sp, sp->p_values[jp]));
+        }
+    return n;
+}
+
+int orc_mixed_decode(const orc_inputs* in, const orc_mixed_space* sp, uint64_t flat, orc_mixed_plan* out) {
+    memset(out, 0, sizeof(*out));
+    for (uint32_t jp = 0; jp < sp->n_p; ++jp) {
+        const uint32_t P = sp->p_values[jp], nseg = mixed_nseg(sp, P);
+        for (uint32_t mi = 0; mi < sp->n_mbs; ++mi)
+        for (uint32_t ri = 0; ri < sp->n_rc; ++ri)
+        for (uint32_t jd = 0; jd < sp->n_d; ++jd) {
+            const uint32_t D = sp->d_values[jd];
+            const uint64_t n_comb = orc_mixed_n_comb(in, sp, D), radix = (uint64_t)in->n_zones * n_comb;
+            const uint64_t block = ipow_u64(radix, nseg);
+            if (flat >= block) { flat -= block; continue; }
+            uint64_t digit[ORC_STAGES_MAX];
+            for (uint32_t s = nseg; s-- > 0;) { digit[s] = flat % radix; flat /= radix; }
+            out->P = P; out->mbs_idx = sp->mbs_idx[mi]; out->rc = sp->rc_values[ri]; out->D = D;
+            const uint32_t units = mixed_units(sp, D), per_unit = D / units;
+            uint32_t u[ORC_GROUPS_MAX][ORC_DP_T_MAX];        /* the combination of each segment (nseg <= seg_max <= 4) */
+            if (nseg > ORC_GROUPS_MAX) return -1;
+            for (uint32_t s = 0; s < nseg; ++s)
+                if (orc_mixed_comb(in, sp, D, digit[s] % n_comb, u[s]) != 0) return -1;
+            for (uint32_t i = 0; i < P; ++i) {
+                const uint32_t sg = (uint32_t)((uint64_t)i * nseg / P);
+                orc_mixed_stage* st = &out->stage[i];
+                st->zone = (uint32_t)(digit[sg] / n_comb);
+                st->n_groups = 0;
+                for (uint32_t g = 0; g < in->n_types; ++g) {
+                    if (!u[sg][g]) continue;
+                    st->group[st->n_groups].type = g;
+                    st->group[st->n_groups].tp_idx = sp->tp_idx_of_type[g];
+                    st->group[st->n_groups].count = u[sg][g] * per_unit;
+                    st->n_groups++;
+                }
+            }
+            return 0;
+        }
+    }
+    return -1;
+}
+
+uint32_t orc_search_mixed(const orc_inputs* in, const orc_mixed_space* sp, const orc_objective* obj, uint64_t lo,
+                          uint64_t hi, uint32_t k, orc_hit* hits, orc_counts* counts) {
+    static orc_mixed_plan pl;
+    orc_out o;
+    uint32_t n_hits = 0;
+    orc_counts c;
+    memset(&c, 0, sizeof(c));
+    for (uint64_t flat = lo; flat < hi; ++flat) {
+        if (orc_mixed_decode(in, sp, flat, &pl) != 0) break;
+        orc_simulate_mixed(in, &pl, &o);
+        c.n_total++;
+        if (o.status & ORC_INVALID) { c.n_invalid++; continue; }
+        if (o.status & ORC_OOM) { c.n_oom++; continue; }
+        if (o.status & ORC_OVER_AVAIL) { c.n_over_avail++; continue; }
+        int over = 0;
+        if (obj->budget > 0.0 && o.cost > obj->budget) over = 1;
+        if (obj->min_rate > 0.0 && 1.0 / o.t_iter < obj->min_rate) over = 1;
+        if (over) { c.n_over_constraint++; continue; }
+        c.n_feasible++;
+        if (c.n_feasible == 1 || o.cost < c.min_cost) c.min_cost = o.cost;
+        n_hits = offer_hit(hits, n_hits, k, flat, score_of(obj, &o), &o);
+    }
+    if (counts) *counts = c;
+    return n_hits;
+}

@@ -272,4 +272,39 @@ void orc_simulate_mixed(const orc_inputs* in, const orc_mixed_plan* plan, orc_ou
 void orc_simulate_mixed_batch(const orc_inputs* in, const orc_mixed_plan* plans, uint64_t n, uint32_t* status,
                               double* t_iter, double* cost, uint64_t* peak_mem);
 
+/* ---- searching over such plans (Sec. 4.2.2 "Implementation": the planner generates, per stage, the resource
+ * combinations of different GPU types that give the stage its D replicas) --------------------------------------
+ *
+ * A combination splits the D replicas of a stage over the GPU types: n_g replicas on type g, sum = D.  To keep
+ * the number of combinations bounded the split is made in `granularity` equal parts when granularity divides D
+ * (a part = D / granularity replicas), else replica by replica: units(D) = granularity or D, and a combination is a
+ * tuple (u_0 .. u_{T-1}) of non-negative units that add up to units(D), at most ORC_GROUPS_MAX of them non-zero;
+ * combinations are numbered in DESCENDING lexicographic order of the tuple (everything on type 0 first; with one
+ * unit, combination c is "everything on type c").  A stage built from a combination lists
+ * its non-empty types in ascending order (group q = the q-th such type, count = units * D / units(D), tensor
+ * parallel degree tp_idx_of_type[type]: the degree the planner fixed for that type, H2).
+ *
+ * Space: as orc_space, but without the tensor-parallel list (it is per type) and with a (zone, combination) per
+ * segment instead of a (zone, type): stage i belongs to segment floor(i * nseg / P), nseg = min(P, seg_max <= 4); the
+ * segment digit is zone * n_comb(D) + combination.  Flat index, low to high: seg[nseg-1] .. seg[0]; then the
+ * positions in d_values, rc_values, mbs_idx; the sub-spaces of p_values concatenated.  The radix of a segment digit
+ * depends on D. */
+typedef struct orc_mixed_space {
+    uint32_t n_p, n_mbs, n_rc, n_d, seg_max, granularity;
+    const uint32_t *p_values, *mbs_idx, *rc_values, *d_values;
+    const uint32_t* tp_idx_of_type;      /* [n_types] */
+} orc_mixed_space;
+
+/* number of combinations for a degree, and the c-th one (units per type); -1 if c is out of range */
+uint64_t orc_mixed_n_comb(const orc_inputs* in, const orc_mixed_space* sp, uint32_t D);
+int orc_mixed_comb(const orc_inputs* in, const orc_mixed_space* sp, uint32_t D, uint64_t c, uint32_t* units_per_type);
+
+uint64_t orc_mixed_space_size(const orc_inputs* in, const orc_mixed_space* sp);
+int orc_mixed_decode(const orc_inputs* in, const orc_mixed_space* sp, uint64_t flat, orc_mixed_plan* out);
+
+/* every candidate of [lo, hi) simulated, classified (first of invalid, oom, over availability, over the constraint
+ * that applies, else feasible) and the k best by (score, flat) kept: as orc_search */
+uint32_t orc_search_mixed(const orc_inputs* in, const orc_mixed_space* sp, const orc_objective* obj, uint64_t lo,
+                          uint64_t hi, uint32_t k, orc_hit* hits, orc_counts* counts);
+
 #endif

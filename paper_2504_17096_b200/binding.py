@@ -18,6 +18,7 @@ ST_INVALID, ST_OVER_AVAIL, ST_OOM, ST_BAD_RECORD = 1, 2, 4, 32
 OBJ_MAX_THROUGHPUT, OBJ_MIN_COST, OBJ_MAX_THROUGHPUT_PER_USD = 0, 1, 2
 FLAG_EVAL_ALL, FLAG_DEGREE_ORDER, FLAG_MIN_TP_ONLY = 1, 2, 4
 DP_FLAG_INDEX_DENSE, DP_FLAG_INDEX_COMPACT, DP_FLAG_ENUM_BY_TYPE, DP_FLAG_ENUM_BY_ENTRY = 0x100, 0x200, 0x400, 0x800
+DP_FLAG_BUDGET_LOOP, DP_BUDGET_P_MAX = 0x1000, 32
 
 EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
            "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_plan_noalloc",
@@ -103,7 +104,7 @@ class DpStats(C.Structure):
     _fields_ = [("n_problems", C.c_uint64), ("n_solved", C.c_uint64), ("n_over_constraint", C.c_uint64),
                 ("n_states", C.c_uint64),
                 ("workspace_used", C.c_uint64), ("kernel_ms", C.c_float), ("n_launches", C.c_uint32),
-                ("n_batches", C.c_uint32), ("_pad", C.c_uint32)]
+                ("n_batches", C.c_uint32), ("n_unfinished", C.c_uint32)]
 
 
 assert C.sizeof(PlanRec) == 72 and C.sizeof(Result) == 120 and C.sizeof(Space) == 152
@@ -379,12 +380,12 @@ dp_default_flags = 0      # SAILOR_DP_FLAG_* that sailor_plan_dp passes when the
 
 
 def sailor_plan_dp(ctx, space: Space, zone_orders, k: int, workspace_bytes: int = 0, *, budget: float = 0.0,
-                   min_rate: float = 0.0, obj: Optional[Objective] = None):
+                   min_rate: float = 0.0, obj: Optional[Objective] = None, budget_loop: bool = False):
     """Per-stage GPU types by dynamic programming for every configuration of the space and every zone
     order (a list of zone lists): the k best plans by the recursion's value among those within the
     budget / minimum throughput, and the statistics."""
     if obj is None:
-        obj = Objective(OBJ_MAX_THROUGHPUT, dp_default_flags, budget, min_rate, 0.0)
+        obj = Objective(OBJ_MAX_THROUGHPUT, DP_FLAG_BUDGET_LOOP if budget_loop else dp_default_flags, budget, min_rate, 0.0)
     orders = (ZoneOrder * len(zone_orders))()
     for j, zl in enumerate(zone_orders):
         if len(zl) > Z_MAX:

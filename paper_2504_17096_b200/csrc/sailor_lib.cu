@@ -15,6 +15,7 @@
 
 #include "sailor_batch.cuh"
 #include "sailor_dp.cuh"
+#include "sailor_dp_budget.cuh"
 #include "sailor_mixed.cuh"
 #include "sailor_peaks.cuh"
 
@@ -163,6 +164,8 @@ constexpr uint64_t WAVE_CONFIG_MAX = 1u << 16;
 
 }  // namespace
 
+static_assert(offsetof(Ctrl, thr_bits) == offsetof(Ctrl, min_cost_bits) + 8, "cleared together");
+
 struct sailor_ctx {
     int device = 0;
     cudaStream_t stream = nullptr;
@@ -184,7 +187,7 @@ struct sailor_ctx {
     Hit* d_partial = nullptr;
     uint32_t* d_partial_n = nullptr;
     uint32_t max_grid = 0;                 // capacity of the partial-result buffers
-    uint32_t grid_of[6] = {0, 0, 0, 0, 0, 0};   // resident blocks per kernel variant, for the cached space
+    uint32_t grid_of[12] = {0};            // resident blocks per kernel variant, for the cached space
     SpaceCache space;
     cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr, evh0 = nullptr, evh1 = nullptr;
     // explicit-batch staging (grow-only)
@@ -443,20 +446,33 @@ uint32_t chunk_of(const sailor_ctx* ctx, uint64_t f) {
 
 using PlanKernel = void (*)(const PlanParams);
 
-PlanKernel pick_kernel(uint32_t obj, bool constr) {
+constexpr int PLAN_VARIANTS = 12;      // objective x constraint x fused
+
+uint32_t variant_of(uint32_t obj, bool constr, bool fused) { return (obj * 2 + (constr ? 1 : 0)) * 2 + (fused ? 1 : 0); }
+
+template <bool FUSED>
+PlanKernel pick_kernel_of(uint32_t obj, bool constr) {
     switch (obj) {
-        case SAILOR_OBJ_MAX_THROUGHPUT: return constr ? plan_kernel<0, true> : plan_kernel<0, false>;
-        case SAILOR_OBJ_MIN_COST: return constr ? plan_kernel<1, true> : plan_kernel<1, false>;
-        default: return constr ? plan_kernel<2, true> : plan_kernel<2, false>;
+        case SAILOR_OBJ_MAX_THROUGHPUT: return constr ? plan_kernel<0, true, FUSED> : plan_kernel<0, false, FUSED>;
+        case SAILOR_OBJ_MIN_COST: return constr ? plan_kernel<1, true, FUSED> : plan_kernel<1, false, FUSED>;
+        default: return constr ? plan_kernel<2, true, FUSED> : plan_kernel<2, false, FUSED>;
     }
 }
+
+PlanKernel pick_kernel(uint32_t obj, bool constr, bool fused) {
+    return fused ? pick_kernel_of<true>(obj, constr) : pick_kernel_of<false>(obj, constr);
+}
+
+// Searches of up to this many chunks per resident block end their pass inside the search kernel; longer ones
+// launch finish_kernel after it.
+constexpr uint32_t FUSED_CHUNKS_PER_BLOCK = 256;
 
 // The dynamic shared-memory opt-in belongs to the kernel (per device), not to a context: raise it
 // once per (device, variant) to the ceiling every space is checked against, so that contexts
 // with different table sizes cannot lower it under one another.
 // The flags are atomic: contexts on different host threads may get here together, and setting the
 // attribute twice to the same value is harmless.
-std::atomic<bool> g_optin_done[64][6];
+std::atomic<bool> g_optin_done[64][PLAN_VARIANTS];
 
 int smem_optin(sailor_ctx* ctx, PlanKernel kern, uint32_t variant) {
     const bool tracked = ctx->device >= 0 && ctx->device < 64;
@@ -524,12 +540,14 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
         pp.chunk_hi = chunk_of(ctx, hi - 1) + 1;
     }
     if (pp.chunk_hi > pp.chunk_lo) {
-        const uint32_t n_chunks = pp.chunk_hi - pp.chunk_lo;
+        const uint32_t n_chunks = waves ? sc.live_chunks : pp.chunk_hi - pp.chunk_lo;
         const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
-        PlanKernel kern = pick_kernel(obj, constr);
-        uint32_t& resident = ctx->grid_of[obj * 2 + (constr ? 1 : 0)];
+        const bool fused = n_chunks <= FUSED_CHUNKS_PER_BLOCK * 2u * (uint32_t)ctx->sm_count;
+        PlanKernel kern = pick_kernel(obj, constr, fused);
+        const uint32_t variant = variant_of(obj, constr, fused);
+        uint32_t& resident = ctx->grid_of[variant];
         if (resident == 0) {       // once per (space, kernel variant): size the grid
-            int rc_opt = smem_optin(ctx, kern, obj * 2 + (constr ? 1 : 0));
+            int rc_opt = smem_optin(ctx, kern, variant);
             if (rc_opt) return rc_opt;
             int per_sm = 0;
             CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, sc.smem));
@@ -537,7 +555,7 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
             resident = (uint32_t)per_sm * (uint32_t)ctx->sm_count;
             if (resident > ctx->max_grid) resident = ctx->max_grid;
         }
-        grid = n_chunks < resident ? n_chunks : resident;
+        grid = n_chunks < resident ? (n_chunks ? n_chunks : 1u) : resident;
         const uint32_t batch = n_chunks / (grid * 32u);
         pp.batch = batch < 1 ? 1 : (batch > 16 ? 16 : batch);
         if (!waves) {
@@ -579,6 +597,11 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
                 CU(ctx, cudaGetLastError());
                 *n_launches += 2;
             }
+        }
+        if (!fused) {              // the end of the pass as a launch of its own
+            finish_kernel<<<1, PLAN_THREADS, ctx->hdr.static_bytes + sizeof(uint32_t) * SAILOR_K_MAX * ctx->hdr.R, ctx->stream>>>(pp, grid);
+            CU(ctx, cudaGetLastError());
+            ++*n_launches;
         }
     }
     *launched = grid != 0;
@@ -795,6 +818,7 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     // both kernels stage the static tables in dynamic shared memory; the create-time limit is 96 KB
     CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)batch_smem_bytes(R_MAX)));
     CUF(cudaFuncSetAttribute(simulate_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
+    CUF(cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 8) * 1024));
 #undef CUF
     *out = ctx;
     return SAILOR_OK;
@@ -991,7 +1015,7 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
     uint32_t launches = 0;
     if (ctx->ctrl_dirty) {             // first search of the context, or the last one failed half-way
         CU(ctx, cudaMemsetAsync(ctx->d_ctrl, 0, sizeof(Ctrl), ctx->stream));
-        CU(ctx, cudaMemsetAsync(&ctx->d_ctrl->min_cost_bits, 0x7f, sizeof(unsigned long long), ctx->stream));
+        CU(ctx, cudaMemsetAsync(&ctx->d_ctrl->min_cost_bits, 0x7f, 2 * sizeof(unsigned long long), ctx->stream));
     }
     ctx->ctrl_dirty = true;            // until this call has gone through
     CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
@@ -1093,7 +1117,7 @@ constexpr int NOALLOC_DEVICES_MAX = 64;
 std::atomic<NoAllocScratch*> g_noalloc_ptr[NOALLOC_DEVICES_MAX];
 // resident blocks per SM of each kernel variant at a given shared-memory size, per device (0 = not asked yet)
 struct OccupancyMemo { std::atomic<uint64_t> smem_and_blocks; };
-OccupancyMemo g_noalloc_occ[NOALLOC_DEVICES_MAX][6];
+OccupancyMemo g_noalloc_occ[NOALLOC_DEVICES_MAX][PLAN_VARIANTS];
 
 // Device address of the scratch on the current device; resolved on first use per device.
 int noalloc_scratch(sailor_ctx* ctx, NoAllocScratch** out) {
@@ -1116,7 +1140,7 @@ int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& d
                          uint32_t k, double next_budget_factor, uint32_t* n_launches) {
     // the array keeps the previous call's contents: counters and the work counter restart at zero
     CU(ctx, cudaMemsetAsync(&sc->ctrl, 0, offsetof(Ctrl, min_cost_bits), ctx->stream));
-    CU(ctx, cudaMemsetAsync(&sc->ctrl.min_cost_bits, 0x7f, sizeof(unsigned long long), ctx->stream));
+    CU(ctx, cudaMemsetAsync(&sc->ctrl.min_cost_bits, 0x7f, 2 * sizeof(unsigned long long), ctx->stream));
     PlanParams pp;
     memset(&pp, 0, sizeof(pp));
     pp.blob = ctx->d_blob;
@@ -1145,8 +1169,8 @@ int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& d
     pp.cost_only = next_budget_factor > 0.0 ? 1u : 0u;
     const uint32_t n_chunks = chunk_hi - chunk_lo;
     const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
-    PlanKernel kern = pick_kernel(obj, constr);
-    const uint32_t variant = obj * 2 + (constr ? 1 : 0);
+    PlanKernel kern = pick_kernel(obj, constr, true);
+    const uint32_t variant = variant_of(obj, constr, true);
     {
         const int rc_opt = smem_optin(ctx, kern, variant);
         if (rc_opt) return rc_opt;
@@ -1305,6 +1329,118 @@ size_t padded(size_t bytes) { return (bytes + 255) & ~(size_t)255; }
 
 }  // namespace
 
+// The recursion steered by the budget (Sec. 4.2.3): one thread per problem, depth first.
+static int plan_dp_budget_impl(sailor_ctx* ctx, const SpaceDesc& d, const sailor_zone_order* orders, uint32_t n_orders,
+                               const sailor_objective* o, uint64_t workspace_bytes, uint32_t k, sailor_dp_result* topk,
+                               uint32_t* n_found, sailor_dp_stats* stats) {
+    const TabHdr& h = ctx->hdr;
+    const uint32_t T = h.T;
+    const uint64_t n_config = (uint64_t)d.n_p * d.n_mbs * d.n_tp * d.n_rc * d.n_d, n_problems = n_config * n_orders;
+    uint32_t p_max = 0;
+    for (uint32_t j = 0; j < d.n_p; ++j) p_max = d.p_values[j] > p_max ? d.p_values[j] : p_max;
+    // what first fit needs of every problem, from the availability last set (host copy)
+    std::vector<DpProblem> prob(n_problems);
+    for (uint64_t c = 0; c < n_config; ++c) {
+        const Config cf = config_of(d, (uint32_t)c);
+        const uint64_t need = (uint64_t)cf.D * h.tp_values[cf.tpi];
+        for (uint32_t q = 0; q < n_orders; ++q) {
+            DpProblem& pb = prob[c * n_orders + q];
+            memset(&pb, 0, sizeof(pb));
+            pb.config = (uint32_t)c; pb.order = q; pb.index = (uint32_t)(c * n_orders + q);
+            pb.P = cf.P; pb.nz = orders[q].n; pb.need = (uint32_t)(need > 0xffffffffull ? 0xffffffffull : need);
+            memset(pb.first_later, DP_NONE, sizeof(pb.first_later));
+            for (uint32_t zp = 0; zp < pb.nz; ++zp) {
+                pb.zone[zp] = orders[q].zone[zp];
+                for (uint32_t g = 0; g < T; ++g) {
+                    const uint64_t cap = ctx->h_avail[pb.zone[zp] * T + g] / need;
+                    pb.cap[zp][g] = (uint8_t)(cap > 255 ? 255 : cap);
+                }
+            }
+            for (uint32_t zp = 0; zp < pb.nz; ++zp)
+                for (uint32_t g = 0; g < T; ++g)
+                    for (uint32_t later = zp + 1; later < pb.nz; ++later)
+                        if (pb.cap[later][g] >= 1) { pb.first_later[zp][g] = (uint8_t)later; break; }
+        }
+    }
+    DeviceGuard guard(ctx->device);
+    DpTabLayout lay;
+    lay.p_max = p_max; lay.T = T; lay.R = h.R;
+    const size_t tab_bytes = (size_t)n_config * lay.stride() * sizeof(double);
+    const size_t total = padded(tab_bytes) + padded(n_problems * sizeof(DpResult)) + padded(n_problems * sizeof(DpProblem)) +
+                         padded(n_problems * DP_BUDGET_P_MAX * sizeof(DpbFrame)) + padded(sizeof(sailor_dp_result) * SAILOR_K_MAX) +
+                         padded(40) + 4096;
+    if (total > workspace_bytes) return SAILOR_E_RANGE;
+    if (total > ctx->dp_bytes) {
+        CU(ctx, stream_sync(ctx));
+        cudaFree(ctx->d_dp);
+        ctx->d_dp = nullptr;
+        ctx->dp_bytes = 0;
+        cudaError_t e = cudaMalloc(&ctx->d_dp, total);
+        if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
+        ctx->dp_bytes = total;
+    }
+    Bump bump{ctx->d_dp};
+    double* d_tabs = bump.take<double>(tab_bytes / sizeof(double));
+    DpResult* d_results = bump.take<DpResult>(n_problems);
+    DpProblem* d_problems = bump.take<DpProblem>(n_problems);
+    DpbFrame* d_frames = bump.take<DpbFrame>(n_problems * DP_BUDGET_P_MAX);
+    sailor_dp_result* d_out = bump.take<sailor_dp_result>(SAILOR_K_MAX);
+    unsigned long long* d_counters = bump.take<unsigned long long>(5);
+
+    uint32_t launches = 0;
+    CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
+    CU(ctx, cudaMemsetAsync(d_tabs, 0, tab_bytes, ctx->stream));
+    CU(ctx, cudaMemsetAsync(d_counters, 0, 40, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(d_problems, prob.data(), n_problems * sizeof(DpProblem), cudaMemcpyHostToDevice, ctx->stream));
+    {
+        const uint32_t grid = (uint32_t)(n_config < 4096 ? n_config : 4096);
+        dp_tables_kernel<<<grid, DP_THREADS, 0, ctx->stream>>>(ctx->d_blob, d, (uint32_t)n_config, lay, d_tabs);
+        CU(ctx, cudaGetLastError());
+        ++launches;
+    }
+    DpBudgetParams bp;
+    memset(&bp, 0, sizeof(bp));
+    bp.blob = ctx->d_blob; bp.avail = ctx->d_avail; bp.sp = d; bp.problems = d_problems; bp.tabs = d_tabs;
+    bp.results = d_results; bp.frames = d_frames; bp.counters = d_counters; bp.lay = lay;
+    bp.n_problems = (uint32_t)n_problems; bp.T = T;
+    bp.limit = o->budget_usd_per_iter;
+    bp.node_limit = 1ull << 24;
+    dp_budget_kernel<<<(uint32_t)((n_problems + 63) / 64), 64, 0, ctx->stream>>>(bp);
+    CU(ctx, cudaGetLastError());
+    ++launches;
+    DpSelectParams sel;
+    memset(&sel, 0, sizeof(sel));
+    sel.results = d_results; sel.out = d_out; sel.counters = d_counters;
+    sel.sp = d; sel.n_problems = (uint32_t)n_problems; sel.n_orders = n_orders; sel.k = k;
+    sel.budget = o->budget_usd_per_iter; sel.min_rate = o->min_iters_per_s;
+    dp_select_kernel<<<1, DP_SELECT_THREADS, 0, ctx->stream>>>(sel);
+    CU(ctx, cudaGetLastError());
+    ++launches;
+    CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
+    unsigned long long counters[5] = {0, 0, 0, 0, 0};
+    std::vector<sailor_dp_result> host_out(k);
+    CU(ctx, cudaMemcpyAsync(counters, d_counters, sizeof(counters), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(host_out.data(), d_out, sizeof(sailor_dp_result) * k, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, stream_sync(ctx));                                 // also: `prob` is pageable
+    if (counters[1] > k) return SAILOR_E_DEVICE;
+    *n_found = (uint32_t)counters[1];
+    memcpy(topk, host_out.data(), sizeof(sailor_dp_result) * counters[1]);
+    if (stats) {
+        stats->n_problems = n_problems;
+        stats->n_solved = counters[0];
+        stats->n_over_constraint = counters[2];
+        stats->n_states = counters[4];
+        stats->workspace_used = total;
+        float ms = 0.f;
+        CU(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
+        stats->kernel_ms = ms;
+        stats->n_launches = launches;
+        stats->n_batches = 1;
+        stats->n_unfinished = (uint32_t)counters[3];
+    }
+    return SAILOR_OK;
+}
+
 static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zone_order* orders,
                         uint32_t n_orders, const sailor_objective* o, uint64_t workspace_bytes, uint32_t k,
                         sailor_dp_result* topk, uint32_t* n_found, sailor_dp_stats* stats) {
@@ -1312,7 +1448,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     if (k > SAILOR_K_MAX) return SAILOR_E_RANGE;
     // the recursion minimises iteration time; a constraint is checked on the plan it returns per problem
     constexpr uint32_t dp_flags = SAILOR_DP_FLAG_INDEX_DENSE | SAILOR_DP_FLAG_INDEX_COMPACT | SAILOR_DP_FLAG_ENUM_BY_TYPE |
-                                  SAILOR_DP_FLAG_ENUM_BY_ENTRY;
+                                  SAILOR_DP_FLAG_ENUM_BY_ENTRY | SAILOR_DP_FLAG_BUDGET_LOOP;
     if (o->kind != SAILOR_OBJ_MAX_THROUGHPUT || (o->flags & ~dp_flags) != 0 ||
         ((o->flags & SAILOR_DP_FLAG_INDEX_DENSE) && (o->flags & SAILOR_DP_FLAG_INDEX_COMPACT)) ||
         ((o->flags & SAILOR_DP_FLAG_ENUM_BY_TYPE) && (o->flags & SAILOR_DP_FLAG_ENUM_BY_ENTRY)) ||
@@ -1337,6 +1473,11 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     if (workspace_bytes == 0) workspace_bytes = 8ull << 30;
     uint32_t p_max = 0;
     for (uint32_t j = 0; j < d.n_p; ++j) p_max = d.p_values[j] > p_max ? d.p_values[j] : p_max;
+    if (o->flags & SAILOR_DP_FLAG_BUDGET_LOOP) {
+        if (!(o->budget_usd_per_iter > 0.0)) return SAILOR_E_ARG;
+        if (p_max > DP_BUDGET_P_MAX) return SAILOR_E_RANGE;
+        return plan_dp_budget_impl(ctx, d, orders, n_orders, o, workspace_bytes, k, topk, n_found, stats);
+    }
 
     // every problem's table layout, from the availability last set (host copy)
     const uint64_t n_problems = n_config * n_orders;
@@ -1706,7 +1847,7 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
         stats->kernel_ms = ms;
         stats->n_launches = launches;
         stats->n_batches = (uint32_t)batches.size();
-        stats->_pad = 0;
+        stats->n_unfinished = 0;
     }
     return SAILOR_OK;
 }

@@ -39,6 +39,8 @@ struct Ctrl {                       // one per context, device memory
     unsigned int wave_chunks;       // chunks of the current wave (searches in degree order)
     unsigned int n_cfg_evaluated;   // configurations selected by the waves so far
     unsigned long long min_cost_bits;   // min C_iter over feasible candidates, as ordered bits
+    unsigned long long thr_bits;    // a score no candidate of the final top-k exceeds (ordered bits): the best k-th
+                                    // best any warp has seen so far; lets all other warps skip what cannot matter
     double budget;                  // written by the cheapest-plan pass for the next pass
     unsigned int error;             // non-zero: a kernel gave up during this call (bounded wait ran out)
     unsigned int n_found;
@@ -222,6 +224,7 @@ struct alignas(16) CfgShared {
                                                   // at this configuration's degree (j = 0) or at lower_tpi[j - 1]
     uint64_t params[SAILOR_P_MAX];
     unsigned long long stat[7];
+    unsigned long long thr_bits;     // the block's copy of Ctrl::thr_bits, lowered by its own warps as their lists fill
     uint64_t mbar;
 };
 
@@ -630,7 +633,7 @@ __device__ __forceinline__ void walk_fast(const PlanParams& pp, const CfgShared&
 template <int NSEG, int OBJ, bool CONSTR, int N2>
 __device__ __forceinline__ void walk_offer(const PlanParams& pp, const CfgShared& cs, const ItemState& it,
                                            uint32_t Z, uint32_t R, double budget, uint64_t item_flat,
-                                           WarpTopK& top, uint32_t lane) {
+                                           WarpTopK& top, uint32_t lane, double outer_thr) {
     const double nb = (double)cs.n_b;
     for (uint32_t d = 0; d < R; ++d) {
         if (!((it.walk >> d) & 1ull)) continue;               // warp-uniform
@@ -639,7 +642,7 @@ __device__ __forceinline__ void walk_offer(const PlanParams& pp, const CfgShared
         const double t = t1[0], c = c1[0];
         const bool good = ((it.ok >> d) & 1ull) && within<CONSTR>(pp, budget, t, c);
         const double score = score_of<OBJ>(t, c);
-        const bool want = good && score <= top.thr_score;
+        const bool want = good && score <= top.thr_score && score <= outer_thr;
         if (__any_sync(FULL, want)) top.offer(want, score, item_flat + d, pp.k, lane);
     }
 }
@@ -794,8 +797,15 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
         cnt.over_constr += n_ok - feas;
     }
     // rare: some lane's item holds a candidate that may enter the warp's list; walk again and offer
-    if (!pp.cost_only && __any_sync(FULL, best < make_inf() && best <= top.thr_score))     // best == inf: the item has no feasible candidate
-        walk_offer<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, item_flat, top, lane);
+    // (a candidate worse than the k-th best of ANY warp's list cannot be among the k best overall: the block keeps
+    // the lowest such score its warps and the other blocks have reached; equal scores still pass, the list decides)
+    const double outer_thr = __longlong_as_double((long long)*reinterpret_cast<const volatile unsigned long long*>(&cs.thr_bits));
+    if (!pp.cost_only && __any_sync(FULL, best < make_inf() && best <= top.thr_score && best <= outer_thr)) {   // best == inf: no feasible candidate
+        const double before = top.thr_score;
+        walk_offer<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, item_flat, top, lane, outer_thr);
+        if (lane == 0 && top.thr_score < before)
+            atomicMin(const_cast<unsigned long long*>(&cs.thr_bits), (unsigned long long)__double_as_longlong(top.thr_score));
+    }
 }
 
 // End of a pass, run by the one block that hands in its list last (no block waits for another: every block
@@ -805,9 +815,8 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
 // their starting values.  `v` is the block's own view of the static tables (already in shared memory); `s_hits`
 // (PLAN_WARPS lists) and `s_cnt` (R x SAILOR_K_MAX words) are scratch in shared memory.
 __device__ __noinline__ void finish_pass(const PlanParams& pp, const TabView& v, Hit (*s_hits)[SAILOR_K_MAX],
-                                         uint32_t* s_cnt, uint32_t* s_n) {
+                                         uint32_t* s_cnt, uint32_t* s_n, uint32_t n_partial) {
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = PLAN_WARPS;
-    const uint32_t n_partial = gridDim.x;
     if (pp.cost_only) {
         // the cheapest-plan pass of a budget-factor search: all the next pass needs is factor x the cheapest feasible
         // cost, which every block has already folded into Ctrl::min_cost_bits (the same bits a full simulation of
@@ -823,6 +832,7 @@ __device__ __noinline__ void finish_pass(const PlanParams& pp, const TabView& v,
             c->wave_chunks = 0;
             c->n_cfg_evaluated = 0;
             c->min_cost_bits = COST_BITS_START;
+            c->thr_bits = COST_BITS_START;
             c->n_found = 0;
         }
         return;
@@ -921,6 +931,7 @@ __device__ __noinline__ void finish_pass(const PlanParams& pp, const TabView& v,
         c.wave_chunks = live->wave_chunks;
         c.n_cfg_evaluated = live->n_cfg_evaluated;
         c.min_cost_bits = live->min_cost_bits;
+        c.thr_bits = live->thr_bits;
         c.error = live->error;
         c.n_found = n;
         pp.out->ctrl = c;
@@ -934,12 +945,16 @@ __device__ __noinline__ void finish_pass(const PlanParams& pp, const TabView& v,
         live->wave_chunks = 0;
         live->n_cfg_evaluated = 0;
         live->min_cost_bits = COST_BITS_START;
+        live->thr_bits = COST_BITS_START;
         if (!(pp.next_budget_factor > 0.0)) live->error = 0;   // a following pass of the same call keeps the flag
         live->n_found = 0;
     }
 }
 
-template <int OBJ, bool CONSTR>
+// FUSED: the block that hands in its list last also ends the pass (one launch per pass: what small searches, bound
+// by launch and hand-over latencies, want).  Not FUSED: the lists are left for finish_kernel (the call inside the
+// kernel costs the candidate loop a few registers, which long searches would pay for in every iteration).
+template <int OBJ, bool CONSTR, bool FUSED>
 __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(const __grid_constant__ PlanParams pp) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ CfgShared cs;
@@ -967,6 +982,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
         cs.magic = (uint32_t)(0x100000000ull / (gh->R ? gh->R : 1u)) + 1u;      // for x / R, see CfgShared
     }
     if (tid < 7) cs.stat[tid] = 0;
+    if (tid == 7) cs.thr_bits = *reinterpret_cast<volatile unsigned long long*>(&pp.ctrl->thr_bits);
     // the padding digit of the tables is read (and masked out) by the two-digit steps: keep it finite
     for (uint32_t x = tid; x < PLAN_PAD * sizeof(SegRec) / 8; x += PLAN_THREADS)
         reinterpret_cast<double*>(a.rec + (size_t)SAILOR_SEG_MAX * R)[x] = 0.0;
@@ -1007,6 +1023,12 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             // first (a block then stays inside one configuration and changes its tables rarely), single chunks at
             // the end (even finish)
             const uint32_t n_chunks = chunk_hi - chunk_lo;
+            if (!first_round) {      // trade thresholds with the other blocks
+                const unsigned long long theirs = *reinterpret_cast<volatile unsigned long long*>(&pp.ctrl->thr_bits);
+                const unsigned long long ours = *reinterpret_cast<volatile unsigned long long*>(&cs.thr_bits);
+                if (ours < theirs) atomicMin(&pp.ctrl->thr_bits, ours);
+                else if (theirs < ours) atomicMin(&cs.thr_bits, theirs);
+            }
             if (first_round) {
                 cs.next_chunk = chunk_lo + min(blockIdx.x, n_chunks);
                 cs.batch_len = 1;
@@ -1111,22 +1133,43 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
         }
         if (lane == 0) pp.partial_n[blockIdx.x] = n;
     }
-    // hand the list in; the block that does so last ends the launch (and, in a pass's final launch, the pass)
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const unsigned int before = atomicAdd(&pp.ctrl->blocks_done, 1u);
-        cs.next_chunk = (before == gridDim.x - 1) ? 1u : 0u;
-        if (before == gridDim.x - 1) {
-            pp.ctrl->blocks_done = 0;                    // the next launch counts from zero
-            if (!pp.finish) pp.ctrl->work_counter = 0;   // (a finishing launch resets all counters below)
+    if (FUSED) {
+        // hand the list in; the block that does so last ends the launch (and, in a pass's final launch, the pass)
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            const unsigned int before = atomicAdd(&pp.ctrl->blocks_done, 1u);
+            cs.next_chunk = (before == gridDim.x - 1) ? 1u : 0u;
+            if (before == gridDim.x - 1) {
+                pp.ctrl->blocks_done = 0;                    // the next launch counts from zero
+                if (!pp.finish) pp.ctrl->work_counter = 0;   // (a finishing launch resets all counters below)
+            }
+        }
+        __syncthreads();
+        if (cs.next_chunk && pp.finish) {
+            __threadfence();
+            finish_pass(pp, v, s_hits, reinterpret_cast<uint32_t*>(a.rec), &cs.batch_len, gridDim.x);
         }
     }
-    __syncthreads();
-    if (cs.next_chunk && pp.finish) {
-        __threadfence();
-        finish_pass(pp, v, s_hits, reinterpret_cast<uint32_t*>(a.rec), &cs.batch_len);
+}
+
+// The end of a pass as a launch of its own (one block), after a search kernel that is not FUSED.
+__global__ void __launch_bounds__(PLAN_THREADS) finish_kernel(const __grid_constant__ PlanParams pp, uint32_t n_partial) {
+    extern __shared__ __align__(16) unsigned char dyn[];      // the static tables, then R x SAILOR_K_MAX counters
+    __shared__ Hit s_hits[PLAN_WARPS][SAILOR_K_MAX];
+    __shared__ uint64_t mbar;
+    __shared__ uint32_t s_n;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(pp.blob)->static_bytes;
+    if (!bulk_load(dyn, pp.blob, static_bytes, &mbar)) {
+        if (tid == 0) atomicExch(&pp.ctrl->error, 1u);
+        for (uint32_t x = tid; x < static_bytes / 16; x += PLAN_THREADS)
+            reinterpret_cast<uint4*>(dyn)[x] = reinterpret_cast<const uint4*>(pp.blob)[x];
+        __syncthreads();
     }
+    TabView v;
+    v.bind(dyn, pp.blob);
+    finish_pass(pp, v, s_hits, reinterpret_cast<uint32_t*>(dyn + static_bytes), &s_n, n_partial);
 }
 
 // The tables of every configuration, built once per (context, space) and kept in global memory: all of them but
