@@ -367,6 +367,64 @@ typedef struct sailor_mixed_plan {      /* 648 bytes; arrays must be 8-byte alig
 int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint64_t n, int on_device,
                           double* t_iter, uint64_t* peak_mem, double* cost, uint32_t* status);
 
+/* ---- searching over such plans (Sec. 4.2.2 "Implementation": per stage, the planner generates the resource
+ * combinations of different GPU types that give the stage its D replicas) ---------------------------------
+ *
+ * A combination splits the D replicas of a stage over the GPU types.  To keep their number bounded the split is made
+ * in `granularity` equal parts when granularity divides D (a part = D / granularity replicas), else replica by
+ * replica: units(D) = granularity or D (at most SAILOR_MIX_UNITS_MAX), and a combination is a tuple (u_0 .. u_{T-1})
+ * of units per type that add up to units(D), at most SAILOR_MIX_GROUPS_MAX of them non-zero.  Combinations are
+ * numbered in descending lexicographic order of the tuple (everything on type 0 first; with one unit, combination c
+ * is "everything on type c").  A stage built from a combination lists its non-empty types in ascending order: group
+ * q = the q-th such type, count = units * D / units(D), tensor-parallel degree tp_idx_of_type[type] (the degree the
+ * planner fixed for that type, H2).
+ *
+ * The space: every (P, mbs, rc, D) of the lists and one (zone, combination) per segment (stage i belongs to segment
+ * floor(i * nseg / P), nseg = min(P, seg_max)); the segment digit is zone * n_comb(D) + combination.  Flat index,
+ * digits from low to high: seg[nseg-1] .. seg[0], then the positions in d_values, rc_values, mbs_idx; the
+ * sub-spaces of the entries of p_values are concatenated.  With granularity 1 and one tensor-parallel degree for
+ * all types this is exactly the space of sailor_plan with that degree, index by index. */
+#define SAILOR_MIX_UNITS_MAX 16
+
+typedef struct sailor_mixed_space {
+    uint32_t n_p, n_mbs, n_rc, n_d, seg_max, granularity;
+    uint8_t  p_values[SAILOR_NP_MAX];       /* each 1 .. SAILOR_MIX_P_MAX                                */
+    uint8_t  mbs_idx[SAILOR_MBS_MAX];
+    uint8_t  rc_values[2];
+    uint8_t  tp_idx_of_type[SAILOR_T_MAX];  /* tensor-parallel degree (index) of every GPU type          */
+    uint8_t  _pad[6];
+    uint16_t d_values[SAILOR_ND_MAX];
+} sailor_mixed_space;
+
+typedef struct sailor_mixed_result {
+    uint64_t flat;
+    double   t_iter;
+    double   cost;
+    uint64_t peak_mem;
+    double   score;
+    uint32_t status;
+    uint32_t _pad;
+    sailor_mixed_plan plan;                 /* stages past P are zero                                    */
+} sailor_mixed_result;
+
+/* Number of candidates (host arithmetic).  E_RANGE: a limit above, units(D) beyond SAILOR_MIX_UNITS_MAX, more than
+ * 2^63 candidates. */
+int sailor_mixed_space_size(const sailor_ctx* ctx, const sailor_mixed_space* s, uint64_t* n_out);
+
+/* Flat index -> plan record (host arithmetic), the inverse of the enumeration order. */
+int sailor_mixed_decode(const sailor_ctx* ctx, const sailor_mixed_space* s, uint64_t flat, sailor_mixed_plan* out);
+
+/* Search the whole space: every candidate is built on the device from its flat index, simulated as
+ * sailor_simulate_mixed simulates it, classed (the first of invalid, out of memory, over availability, over the
+ * budget or under the throughput floor that applies, else feasible) and the k best feasible ones by (score, flat)
+ * returned, best first, with their records.  o->flags must be 0 and o->budget_factor_over_cheapest 0 (E_ARG).
+ * `topk` is a HOST array of k records; `stats` may be NULL (n_pruned_tp, n_skipped are 0; n_configs counts the
+ * (P, mbs, rc, D) tuples).  Uses the availability last set; allocates device memory on first use (grow-only, kept by
+ * the context); synchronises the stream.  Errors: E_ARG, E_RANGE (as sailor_mixed_space_size; k > SAILOR_K_MAX),
+ * E_NOMEM, E_CUDA, E_DEVICE. */
+int sailor_plan_mixed(sailor_ctx* ctx, const sailor_mixed_space* s, const sailor_objective* o, uint32_t k,
+                      sailor_mixed_result* topk, uint32_t* n_found, sailor_stats* stats);
+
 /* ---- per-stage GPU types by dynamic programming (Sec. 4.2.2: Eq. 1, T_total, the listing) --------
  *
  * sailor_plan varies the GPU type and zone of at most SAILOR_SEG_MAX segments of a pipeline.  This

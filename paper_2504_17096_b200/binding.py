@@ -22,7 +22,8 @@ DP_FLAG_BUDGET_LOOP, DP_BUDGET_P_MAX = 0x1000, 32
 
 EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
            "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_plan_noalloc",
-           "sailor_plan_dp", "sailor_simulate_mixed", "sailor_measure_issue_rates", "sailor_strerror",
+           "sailor_plan_dp", "sailor_simulate_mixed", "sailor_mixed_space_size", "sailor_mixed_decode",
+           "sailor_plan_mixed", "sailor_measure_issue_rates", "sailor_strerror",
            "sailor_last_cuda_error")
 
 _dp, _u64p, _u32p, _u16p = C.POINTER(C.c_double), C.POINTER(C.c_uint64), C.POINTER(C.c_uint32), C.POINTER(C.c_uint16)
@@ -146,6 +147,40 @@ def pack_mixed_plans(plans) -> np.ndarray:
     return out
 
 
+class MixedGroup(C.Structure):
+    _fields_ = [("type", C.c_uint8), ("tp_idx", C.c_uint8), ("count", C.c_uint16)]
+
+
+class MixedStage(C.Structure):
+    _fields_ = [("zone", C.c_uint8), ("n_groups", C.c_uint8), ("_pad", C.c_uint16), ("group", MixedGroup * MIX_GROUPS_MAX)]
+
+
+class MixedPlan(C.Structure):
+    _fields_ = [("P", C.c_uint8), ("mbs_idx", C.c_uint8), ("rc", C.c_uint8), ("_pad", C.c_uint8), ("D", C.c_uint16),
+                ("_pad2", C.c_uint16), ("stage", MixedStage * MIX_P_MAX)]
+
+    def as_dict(self) -> dict:
+        return {"P": self.P, "mbs_idx": self.mbs_idx, "rc": self.rc, "D": self.D,
+                "stages": [{"zone": self.stage[i].zone,
+                            "groups": [(self.stage[i].group[q].type, self.stage[i].group[q].tp_idx, self.stage[i].group[q].count)
+                                       for q in range(self.stage[i].n_groups)]} for i in range(self.P)]}
+
+
+class MixedSpace(C.Structure):
+    _fields_ = [("n_p", C.c_uint32), ("n_mbs", C.c_uint32), ("n_rc", C.c_uint32), ("n_d", C.c_uint32),
+                ("seg_max", C.c_uint32), ("granularity", C.c_uint32), ("p_values", C.c_uint8 * NP_MAX),
+                ("mbs_idx", C.c_uint8 * MBS_MAX), ("rc_values", C.c_uint8 * 2), ("tp_idx_of_type", C.c_uint8 * T_MAX),
+                ("_pad", C.c_uint8 * 6), ("d_values", C.c_uint16 * ND_MAX)]
+
+
+class MixedResult(C.Structure):
+    _fields_ = [("flat", C.c_uint64), ("t_iter", C.c_double), ("cost", C.c_double), ("peak_mem", C.c_uint64),
+                ("score", C.c_double), ("status", C.c_uint32), ("_pad", C.c_uint32), ("plan", MixedPlan)]
+
+
+assert C.sizeof(MixedPlan) == 648 and C.sizeof(MixedResult) == 696 and C.sizeof(MixedSpace) == 152
+
+
 class SailorError(RuntimeError):
     def __init__(self, code: int, where: str, cuda: int = 0):
         self.code = code
@@ -183,6 +218,10 @@ def load() -> C.CDLL:
     L.sailor_plan_dp.argtypes = [vp, C.POINTER(Space), C.POINTER(ZoneOrder), C.c_uint32, C.POINTER(Objective),
                                  C.c_uint64, C.c_uint32, C.POINTER(DpResult), _u32p, C.POINTER(DpStats)]
     L.sailor_measure_issue_rates.argtypes = [C.c_int, vp, C.c_uint32, C.POINTER(IssueRates)]
+    L.sailor_mixed_space_size.argtypes = [vp, C.POINTER(MixedSpace), _u64p]
+    L.sailor_mixed_decode.argtypes = [vp, C.POINTER(MixedSpace), C.c_uint64, C.POINTER(MixedPlan)]
+    L.sailor_plan_mixed.argtypes = [vp, C.POINTER(MixedSpace), C.POINTER(Objective), C.c_uint32, C.POINTER(MixedResult),
+                                    _u32p, C.POINTER(Stats)]
     L.sailor_strerror.argtypes = [C.c_int]
     L.sailor_strerror.restype = C.c_char_p
     L.sailor_last_cuda_error.argtypes = [vp]
@@ -366,6 +405,45 @@ def all_zone_orders(n_zones: int, max_len: Optional[int] = None):
     import itertools
     max_len = n_zones if max_len is None else min(max_len, n_zones)
     return [list(p) for n in range(1, max_len + 1) for p in itertools.permutations(range(n_zones), n)]
+
+
+def make_mixed_space(w, granularity: int, tp_idx_of_type, *, p_values=None, mbs_idx=None, rc_values=None,
+                     d_values=None, seg_max=None) -> MixedSpace:
+    """sailor_mixed_space from a workload's radix lists (or the given ones)."""
+    s = MixedSpace()
+    lists = {"p_values": w.p_values if p_values is None else p_values, "mbs_idx": w.mbs_idx if mbs_idx is None else mbs_idx,
+             "rc_values": w.rc_values if rc_values is None else rc_values, "d_values": w.d_values if d_values is None else d_values,
+             "tp_idx_of_type": tp_idx_of_type}
+    for name, values in lists.items():
+        arr = getattr(s, name)
+        for i, x in enumerate(values):
+            arr[i] = int(x)
+    s.n_p, s.n_mbs, s.n_rc, s.n_d = (len(lists[k]) for k in ("p_values", "mbs_idx", "rc_values", "d_values"))
+    s.seg_max = w.seg_max if seg_max is None else seg_max
+    s.granularity = granularity
+    return s
+
+
+def sailor_mixed_space_size(ctx, space: MixedSpace) -> int:
+    n = C.c_uint64()
+    _check(load().sailor_mixed_space_size(ctx, C.byref(space), C.byref(n)), "sailor_mixed_space_size")
+    return int(n.value)
+
+
+def sailor_mixed_decode(ctx, space: MixedSpace, flat: int) -> MixedPlan:
+    r = MixedPlan()
+    _check(load().sailor_mixed_decode(ctx, C.byref(space), flat, C.byref(r)), "sailor_mixed_decode")
+    return r
+
+
+def sailor_plan_mixed(ctx, space: MixedSpace, obj: Objective, k: int):
+    """Search over plans whose stages mix GPU types among their replicas: the k best and the statistics."""
+    res = (MixedResult * k)()
+    n = C.c_uint32()
+    st = Stats()
+    _check(load().sailor_plan_mixed(ctx, C.byref(space), C.byref(obj), k, res, C.byref(n), C.byref(st)),
+           "sailor_plan_mixed", ctx)
+    return list(res[: n.value]), st
 
 
 def sailor_measure_issue_rates(device: int = 0, stream: int = 0, repeats: int = 5) -> IssueRates:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsailor_b200.so")
 SOURCES = [os.path.join(CSRC, "sailor_lib.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("sailor_tables.cuh", "sailor_plan_kernels.cuh", "sailor_dp.cuh", "sailor_dp_budget.cuh", "sailor_batch.cuh", "sailor_mixed.cuh", "sailor_peaks.cuh")] + [
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("sailor_tables.cuh", "sailor_plan_kernels.cuh", "sailor_dp.cuh", "sailor_dp_budget.cuh", "sailor_batch.cuh", "sailor_mixed.cuh", "sailor_mixed_search.cuh", "sailor_peaks.cuh")] + [
     os.path.join(os.path.dirname(HERE), "include", "sailor.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -17,6 +17,7 @@
 #include "sailor_dp.cuh"
 #include "sailor_dp_budget.cuh"
 #include "sailor_mixed.cuh"
+#include "sailor_mixed_search.cuh"
 #include "sailor_peaks.cuh"
 
 using namespace sailor;
@@ -193,6 +194,9 @@ struct sailor_ctx {
     // explicit-batch staging (grow-only)
     unsigned char* d_stage = nullptr;
     size_t stage_bytes = 0;
+    // working memory of the search over plans with mixed replicas (grow-only)
+    unsigned char* d_mix = nullptr;
+    size_t mix_bytes = 0;
     // tables of the dynamic-programming search (grow-only)
     unsigned char* d_dp = nullptr;
     size_t dp_bytes = 0;
@@ -819,6 +823,8 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)batch_smem_bytes(R_MAX)));
     CUF(cudaFuncSetAttribute(simulate_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
     CUF(cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 8) * 1024));
+    CUF(cudaFuncSetAttribute(plan_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 16) * 1024));
+    CUF(cudaFuncSetAttribute(mixed_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 16) * 1024));
 #undef CUF
     *out = ctx;
     return SAILOR_OK;
@@ -846,6 +852,7 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->space.d_groups);
     cudaFree(ctx->space.d_cfg_cache);
     cudaFree(ctx->d_stage);
+    cudaFree(ctx->d_mix);
     cudaFree(ctx->d_dp);
     for (cudaEvent_t e : {ctx->ev0, ctx->ev1, ctx->ev2, ctx->evh0, ctx->evh1})
         if (e) cudaEventDestroy(e);
@@ -1850,6 +1857,211 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
         stats->n_unfinished = 0;
     }
     return SAILOR_OK;
+}
+
+// ---- search over plans with mixed replicas -------------------------------------------------------------
+
+namespace {
+
+// The combinations of `units` over T types with at most SAILOR_MIX_GROUPS_MAX non-empty types, in descending
+// lexicographic order, one 64-bit word each (byte g = units on type g).
+void list_combinations(uint32_t T, uint32_t units, std::vector<uint64_t>& out) {
+    struct Rec {
+        static void go(uint32_t T, uint32_t t, uint32_t left, uint32_t nonzero, uint64_t word, std::vector<uint64_t>& out) {
+            if (t + 1 == T) {                                  // the last type takes what is left
+                if (nonzero + (left ? 1u : 0u) <= SAILOR_MIX_GROUPS_MAX) out.push_back(word | ((uint64_t)left << (8 * t)));
+                return;
+            }
+            for (uint32_t u = left + 1; u-- > 0;) {            // most units first
+                const uint32_t nz = nonzero + (u ? 1u : 0u);
+                if (nz > SAILOR_MIX_GROUPS_MAX) continue;
+                go(T, t + 1, left - u, nz, word | ((uint64_t)u << (8 * t)), out);
+            }
+        }
+    };
+    Rec::go(T, 0, units, 0, 0, out);
+}
+
+struct MixedTables {
+    MixedSpaceDesc desc;
+    std::vector<uint64_t> combs;
+    std::vector<uint64_t> flat_base;           // [n_config + 1]
+    uint32_t n_config = 0;
+};
+
+int build_mixed_tables(const sailor_ctx* ctx, const sailor_mixed_space* s, MixedTables& mt) {
+    if (!ctx || !s) return SAILOR_E_ARG;
+    if (s->n_p == 0 || s->n_mbs == 0 || s->n_rc == 0 || s->n_d == 0 || s->granularity == 0) return SAILOR_E_ARG;
+    if (s->n_p > SAILOR_NP_MAX || s->n_mbs > SAILOR_MBS_MAX || s->n_rc > 2 || s->n_d > SAILOR_ND_MAX || s->seg_max < 1 ||
+        s->seg_max > SAILOR_SEG_MAX)
+        return SAILOR_E_RANGE;
+    const TabHdr& h = ctx->hdr;
+    for (uint32_t i = 0; i < s->n_p; ++i)
+        if (s->p_values[i] < 1 || s->p_values[i] > SAILOR_MIX_P_MAX) return SAILOR_E_RANGE;
+    for (uint32_t i = 0; i < s->n_mbs; ++i)
+        if (s->mbs_idx[i] >= h.n_mbs) return SAILOR_E_RANGE;
+    for (uint32_t i = 0; i < s->n_rc; ++i)
+        if (s->rc_values[i] > 1) return SAILOR_E_RANGE;
+    for (uint32_t g = 0; g < h.T; ++g)
+        if (s->tp_idx_of_type[g] >= h.n_tp) return SAILOR_E_RANGE;
+    MixedSpaceDesc& d = mt.desc;
+    memset(&d, 0, sizeof(d));
+    d.n_p = s->n_p; d.n_mbs = s->n_mbs; d.n_rc = s->n_rc; d.n_d = s->n_d; d.seg_max = s->seg_max; d.granularity = s->granularity;
+    memcpy(d.p_values, s->p_values, sizeof(d.p_values));
+    memcpy(d.mbs_idx, s->mbs_idx, sizeof(d.mbs_idx));
+    memcpy(d.rc_values, s->rc_values, sizeof(d.rc_values));
+    memcpy(d.tp_idx_of_type, s->tp_idx_of_type, sizeof(d.tp_idx_of_type));
+    memcpy(d.d_values, s->d_values, sizeof(d.d_values));
+    std::map<uint32_t, std::pair<uint32_t, uint32_t>> by_units;        // units -> (offset, count): degrees often share them
+    for (uint32_t j = 0; j < s->n_d; ++j) {
+        const uint32_t D = s->d_values[j];
+        if (D < 1) return SAILOR_E_RANGE;
+        const uint32_t units = mixed_units(s->granularity, D);
+        if (units > SAILOR_MIX_UNITS_MAX) return SAILOR_E_RANGE;
+        auto it = by_units.find(units);
+        if (it == by_units.end()) {
+            const uint32_t off = (uint32_t)mt.combs.size();
+            list_combinations(h.T, units, mt.combs);
+            it = by_units.emplace(units, std::make_pair(off, (uint32_t)mt.combs.size() - off)).first;
+        }
+        d.comb_off[j] = it->second.first;
+        d.n_comb[j] = it->second.second;
+    }
+    const uint64_t n_config = (uint64_t)s->n_p * s->n_mbs * s->n_rc * s->n_d;
+    if (n_config > (1u << 16)) return SAILOR_E_RANGE;
+    mt.n_config = (uint32_t)n_config;
+    mt.flat_base.assign(n_config + 1, 0);
+    unsigned __int128 run = 0;
+    for (uint32_t c = 0; c < n_config; ++c) {
+        mt.flat_base[c] = (uint64_t)run;
+        const MixedConfig k = mixed_config_of(d, c);
+        const unsigned __int128 radix = (unsigned __int128)h.Z * d.n_comb[k.di];
+        unsigned __int128 block = 1;
+        for (uint32_t q = 0; q < k.nseg; ++q) {
+            block *= radix;
+            if (block >> 63) return SAILOR_E_RANGE;
+        }
+        run += block;
+        if (run >> 63) return SAILOR_E_RANGE;
+    }
+    mt.flat_base[n_config] = (uint64_t)run;
+    return SAILOR_OK;
+}
+
+}  // namespace
+
+static int plan_mixed_impl(sailor_ctx* ctx, const sailor_mixed_space* s, const sailor_objective* o, uint32_t k,
+                           sailor_mixed_result* topk, uint32_t* n_found, sailor_stats* stats) {
+    if (!ctx || !s || !o || !topk || !n_found || k == 0) return SAILOR_E_ARG;
+    if (k > SAILOR_K_MAX || o->kind > SAILOR_OBJ_MAX_THROUGHPUT_PER_USD) return SAILOR_E_RANGE;
+    if (o->flags != 0 || o->budget_factor_over_cheapest > 0.0 || std::isnan(o->budget_usd_per_iter) ||
+        std::isnan(o->min_iters_per_s) || std::isnan(o->budget_factor_over_cheapest))
+        return SAILOR_E_ARG;
+    MixedTables mt;
+    int rc = build_mixed_tables(ctx, s, mt);
+    if (rc) return rc;
+    const uint64_t n_total = mt.flat_base[mt.n_config];
+    DeviceGuard guard(ctx->device);
+    const uint32_t R = ctx->hdr.R;
+    const size_t smem = ctx->hdr.static_bytes + sizeof(unsigned long long) * MIXS_WARPS * R + sizeof(sailor_mixed_plan) * MIXS_WARPS;
+    const uint64_t want_blocks = (n_total + MIXS_WARPS - 1) / MIXS_WARPS;
+    const uint32_t grid = (uint32_t)std::min<uint64_t>(std::max<uint64_t>(want_blocks, 1), (uint64_t)ctx->sm_count * 4);
+    const size_t total = padded(mt.combs.size() * 8) + padded(mt.flat_base.size() * 8) + padded(sizeof(Hit) * SAILOR_K_MAX * grid) +
+                         padded(sizeof(sailor_mixed_result) * SAILOR_K_MAX) + padded(9 * 8) + 1024;
+    if (total > ctx->mix_bytes) {
+        CU(ctx, stream_sync(ctx));
+        cudaFree(ctx->d_mix);
+        ctx->d_mix = nullptr;
+        ctx->mix_bytes = 0;
+        cudaError_t e = cudaMalloc(&ctx->d_mix, total);
+        if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
+        ctx->mix_bytes = total;
+    }
+    Bump bump{ctx->d_mix};
+    uint64_t* d_combs = bump.take<uint64_t>(mt.combs.size());
+    uint64_t* d_base = bump.take<uint64_t>(mt.flat_base.size());
+    Hit* d_partial = bump.take<Hit>((size_t)SAILOR_K_MAX * grid);
+    sailor_mixed_result* d_results = bump.take<sailor_mixed_result>(SAILOR_K_MAX);
+    unsigned long long* d_counters = bump.take<unsigned long long>(9);
+
+    CU(ctx, cudaMemcpyAsync(d_combs, mt.combs.data(), mt.combs.size() * 8, cudaMemcpyHostToDevice, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(d_base, mt.flat_base.data(), mt.flat_base.size() * 8, cudaMemcpyHostToDevice, ctx->stream));
+    CU(ctx, cudaMemsetAsync(d_counters, 0, 9 * 8, ctx->stream));
+    CU(ctx, cudaMemsetAsync(d_counters + 6, 0x7f, 8, ctx->stream));           // the cheapest cost starts above every cost
+    CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
+    MixedSearchParams mp;
+    memset(&mp, 0, sizeof(mp));
+    mp.blob = ctx->d_blob; mp.avail = ctx->d_avail; mp.cfg_flat_base = d_base; mp.combs = d_combs; mp.partial = d_partial;
+    mp.counters = d_counters; mp.results = d_results; mp.sp = mt.desc; mp.n_config = mt.n_config; mp.k = k; mp.obj = o->kind;
+    mp.n_partial = grid; mp.n_total = n_total; mp.budget = o->budget_usd_per_iter; mp.min_rate = o->min_iters_per_s;
+    plan_mixed_kernel<<<grid, MIXS_THREADS, smem, ctx->stream>>>(mp);
+    CU(ctx, cudaGetLastError());
+    mixed_finish_kernel<<<1, MIXS_THREADS, smem, ctx->stream>>>(mp);
+    CU(ctx, cudaGetLastError());
+    CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
+    unsigned long long counters[9];
+    std::vector<sailor_mixed_result> host_out(k);
+    CU(ctx, cudaMemcpyAsync(counters, d_counters, sizeof(counters), cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(host_out.data(), d_results, sizeof(sailor_mixed_result) * k, cudaMemcpyDeviceToHost, ctx->stream));
+    CU(ctx, stream_sync(ctx));                                 // also: the host tables are pageable
+    if (counters[7]) return SAILOR_E_DEVICE;
+    if (counters[8] > k) return SAILOR_E_DEVICE;
+    *n_found = (uint32_t)counters[8];
+    memcpy(topk, host_out.data(), sizeof(sailor_mixed_result) * counters[8]);
+    if (stats) {
+        memset(stats, 0, sizeof(*stats));
+        stats->n_total = counters[0];
+        stats->n_invalid = counters[1];
+        stats->n_oom = counters[2];
+        stats->n_over_avail = counters[3];
+        stats->n_over_constraint = counters[4];
+        stats->n_feasible = counters[5];
+        stats->budget_used = o->budget_usd_per_iter;
+        double mc;
+        memcpy(&mc, &counters[6], sizeof(mc));
+        stats->min_feasible_cost = counters[5] ? mc : 0.0;
+        CU(ctx, cudaEventElapsedTime(&stats->kernel_ms, ctx->ev0, ctx->ev1));
+        stats->n_launches = 2;
+        stats->n_configs = stats->n_configs_evaluated = mt.n_config;
+    }
+    return SAILOR_OK;
+}
+
+extern "C" int sailor_mixed_space_size(const sailor_ctx* ctx, const sailor_mixed_space* s, uint64_t* n_out) {
+    if (!n_out) return SAILOR_E_ARG;
+    try {
+        MixedTables mt;
+        const int rc = build_mixed_tables(ctx, s, mt);
+        if (rc) return rc;
+        *n_out = mt.flat_base[mt.n_config];
+        return SAILOR_OK;
+    } catch (const std::bad_alloc&) { return SAILOR_E_NOMEM; } catch (...) { return SAILOR_E_ARG; }
+}
+
+extern "C" int sailor_mixed_decode(const sailor_ctx* ctx, const sailor_mixed_space* s, uint64_t flat, sailor_mixed_plan* out) {
+    if (!out) return SAILOR_E_ARG;
+    try {
+        MixedTables mt;
+        const int rc = build_mixed_tables(ctx, s, mt);
+        if (rc) return rc;
+        if (flat >= mt.flat_base[mt.n_config]) return SAILOR_E_RANGE;
+        const uint32_t c = (uint32_t)(std::upper_bound(mt.flat_base.begin(), mt.flat_base.end(), flat) - mt.flat_base.begin()) - 1;
+        const MixedConfig k = mixed_config_of(mt.desc, c);
+        const uint64_t radix = (uint64_t)ctx->hdr.Z * mt.desc.n_comb[k.di];
+        uint64_t rem = flat - mt.flat_base[c], digit[SAILOR_SEG_MAX] = {0, 0, 0, 0};
+        for (uint32_t q = k.nseg; q-- > 0;) { digit[q] = rem % radix; rem /= radix; }
+        memset(out, 0, sizeof(*out));
+        out->P = (uint8_t)k.P; out->mbs_idx = (uint8_t)k.mi; out->rc = (uint8_t)k.rc; out->D = (uint16_t)k.D;
+        for (uint32_t i = 0; i < k.P; ++i) mixed_build_stage(mt.desc, k, ctx->hdr.T, mt.combs.data(), digit, i, &out->stage[i]);
+        return SAILOR_OK;
+    } catch (const std::bad_alloc&) { return SAILOR_E_NOMEM; } catch (...) { return SAILOR_E_ARG; }
+}
+
+extern "C" int sailor_plan_mixed(sailor_ctx* ctx, const sailor_mixed_space* s, const sailor_objective* o, uint32_t k,
+                                 sailor_mixed_result* topk, uint32_t* n_found, sailor_stats* stats) {
+    try {
+        return plan_mixed_impl(ctx, s, o, k, topk, n_found, stats);
+    } catch (const std::bad_alloc&) { return SAILOR_E_NOMEM; } catch (...) { return SAILOR_E_ARG; }
 }
 
 // ---- sustained issue rates (measurement) ---------------------------------------------------------------
