@@ -231,9 +231,13 @@ typedef struct sailor_stats {
     uint64_t n_skipped;         /* candidates of configurations early termination never reached */
     uint32_t n_configs;         /* configurations (P, mbs, tp, rc, D) of the space           */
     uint32_t n_configs_evaluated;   /* of which looked at (all of them without DEGREE_ORDER) */
-    float    h2d_ms;            /* device time of the last availability upload (CUDA events
-                                   around the copy in sailor_set_availability)               */
-    float    d2h_ms;            /* device time of this call's result read-back               */
+    float    h2d_ms;            /* device time of the last availability upload to device memory
+                                   (CUDA events around the copy; sailor_plan itself carries the
+                                   snapshot in its launch parameters and needs no such copy: the
+                                   entry points that read it through a pointer trigger one)     */
+    float    d2h_ms;            /* device time of this call's result read-back; 0 where the
+                                   kernel writes the results straight into pinned host memory
+                                   (sailor_plan, sailor_plan_range)                             */
 } sailor_stats;
 
 typedef struct sailor_ctx sailor_ctx;     /* opaque; owns device copies of the tables       */
@@ -252,7 +256,9 @@ int sailor_create(const sailor_model* m, const sailor_profile* p, const sailor_c
 int sailor_destroy(sailor_ctx* ctx);      /* NULL is accepted                               */
 
 /* Replace the availability snapshot (Sec. 4: "current availability of hardware resources").
- * `avail` is a HOST array [zone][type] of GPU counts.  The only per-snapshot upload. */
+ * `avail` is a HOST array [zone][type] of GPU counts, copied before the call returns.  It is the only
+ * per-snapshot input: a search carries it to the device in its launch parameters; the device copy read by
+ * sailor_simulate*, sailor_plan_dp and sailor_plan_mixed is refreshed when one of them is next called. */
 int sailor_set_availability(sailor_ctx* ctx, const uint16_t* avail);
 
 /* Simulate n explicit plans (Sec. 4.3).  Inputs and outputs are all HOST pointers when

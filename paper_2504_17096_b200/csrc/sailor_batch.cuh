@@ -3,8 +3,8 @@
 // A record costs 72 bytes in and 28 bytes out, so the batch is bound by HBM only if a record takes a few hundred
 // instructions.  Three things keep it there:
 //   - everything a stretch of equal stages needs (f + b, update time, gradient bytes, memory with and without an
-//     in-flight microbatch, the GPU's capacity) sits in ONE 48-byte table entry per (stage make-up, GPU type, tp,
-//     mbs, rc), formed once per context with the same functions and operation order as a stage-by-stage walk;
+//     in-flight microbatch) sits in ONE 32-byte table entry (one memory sector) per (stage make-up, GPU type, tp,
+//     mbs, rc), the gradient bytes in a table per (stage make-up, tp), both formed once per context with the same functions and operation order as a stage-by-stage walk;
 //   - the doubled one-way message time of every link (inside a node, between nodes, between zones) is tabulated
 //     per microbatch size, so a stage boundary is one or two loads and at most one maximum;
 //   - index arithmetic is 32 bits wide and the per-digit GPU counters are 16-bit saturating.
@@ -16,15 +16,13 @@
 
 namespace sailor {
 
-struct alignas(16) PieceRec {        // one per (composition, type, tp index, mbs index, rc)
+struct alignas(32) PieceRec {        // one per (composition, type, tp index, mbs index, rc): one 32-byte sector
     double fb;                       // f + b (+ f with recomputation) of a stage of this make-up
     double upd;                      // its update time
-    double grad;                     // gradient bytes of one worker, as a double
     uint64_t mem0r;                  // model + working bytes + the type's reserved bytes
     uint64_t mem1;                   // bytes kept per in-flight microbatch
-    uint64_t cap;                    // the type's capacity
 };
-static_assert(sizeof(PieceRec) == 48, "three 16-byte loads");
+static_assert(sizeof(PieceRec) == 32, "two 16-byte loads from one sector");
 
 __host__ __device__ inline size_t piece_count(const TabHdr& h) {
     return (size_t)4 * h.chain_len * h.T * h.n_tp * h.n_mbs * 2;
@@ -53,10 +51,8 @@ __global__ void batch_tables_kernel(unsigned char* blob) {
         PieceRec r;
         r.fb = add_rn(st.f, b);
         r.upd = st.u;
-        r.grad = (double)(ceil_div64(one.params, h->tp_values[tpi]) * h->grad_bytes);
         r.mem0r = zero.mem + h->reserved[g];
         r.mem1 = one.mem - zero.mem;
-        r.cap = h->capacity[g];
         out[x] = r;
     }
     double* intra2 = reinterpret_cast<double*>(blob + h->off_lnk_intra2);
@@ -84,6 +80,7 @@ struct BatchConst {
     uint32_t tp_values[SAILOR_TP_MAX];
     uint32_t mbs_values[SAILOR_MBS_MAX];
     uint32_t gpn[SAILOR_T_MAX];
+    uint64_t cap[SAILOR_T_MAX];
     uint64_t p2p[SAILOR_MBS_MAX];
     uint32_t avail[R_MAX];
     double price_s[R_MAX];
@@ -174,6 +171,7 @@ __device__ __forceinline__ BatchOut simulate_batch_record(const BatchConst& k, c
         const bool intra_dp = (uint64_t)D * tp <= k.gpn[g];
         const double ar_alpha = intra_dp ? k.intra_a[d] : k.inter_a[d], ar_inv = intra_dp ? k.intra_i[d] : k.inter_i[d];
         const uint32_t ent = ((g * k.n_tp + tpi) * k.n_mbs + mi) * 2 + rc;        // entry within a composition
+        const uint64_t cap = k.cap[g];
         while (i < run_end) {
             const bool e = (i == 0) && k.has_embed, hd = (i == P - 1) && k.has_head;
             // the piece ends with the run, after the embedding stage, where the extra blocks run out, before the head stage
@@ -186,11 +184,10 @@ __device__ __forceinline__ BatchOut simulate_batch_record(const BatchConst& k, c
             const uint32_t comp = ((e ? 2u : 0u) + (hd ? 1u : 0u)) * k.chain_len + base + (i < extra ? 1u : 0u);
             const PieceRec* pr = piece + (size_t)comp * k.piece_stride + ent;
             const double2 a0 = __ldg(reinterpret_cast<const double2*>(pr));                // fb, upd
-            const ulonglong2 a1 = __ldg(reinterpret_cast<const ulonglong2*>(pr) + 1);      // grad, mem0r
-            const ulonglong2 a2 = __ldg(reinterpret_cast<const ulonglong2*>(pr) + 2);      // mem1, cap
+            const ulonglong2 a1 = __ldg(reinterpret_cast<const ulonglong2*>(pr) + 1);      // mem0r, mem1
             const double fb = a0.x;
             if (D > 1) {
-                const double grad = __longlong_as_double((long long)a1.x);
+                const double grad = __ldg(&v.cmp_grad[comp * k.n_tp + tpi]);
                 const double volume = mul_rn(coef, grad);
                 double t;
                 if (k.has_poly) {
@@ -200,8 +197,8 @@ __device__ __forceinline__ BatchOut simulate_batch_record(const BatchConst& k, c
                 max_sync = dmax(max_sync, add_rn(t, mul_rn(steps, ar_alpha)));
             }
             const uint64_t left = P - i, inflight = left < n_b ? left : n_b;
-            const uint64_t m = a1.y + inflight * a2.x;
-            oom |= m > a2.y;
+            const uint64_t m = a1.x + inflight * a1.y;
+            oom |= m > cap;
             peak = m > peak ? m : peak;
             max_u = dmax(max_u, a0.y);
             const bool closes = piece_end == run_end;          // the piece's last stage sends to the next run, or is the final stage
@@ -274,7 +271,7 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
     }
     if (tid < SAILOR_TP_MAX) k.tp_values[tid] = h->tp_values[tid];
     if (tid < SAILOR_MBS_MAX) { k.mbs_values[tid] = h->mbs_values[tid]; k.p2p[tid] = tid < h->n_mbs ? v.p2p[tid] : 0; }
-    if (tid < SAILOR_T_MAX) k.gpn[tid] = h->gpn[tid];
+    if (tid < SAILOR_T_MAX) { k.gpn[tid] = h->gpn[tid]; k.cap[tid] = h->capacity[tid]; }
     if (tid < h->R) {
         k.avail[tid] = avail[tid];
         k.price_s[tid] = v.price_s[tid];

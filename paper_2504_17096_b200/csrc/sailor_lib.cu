@@ -174,11 +174,12 @@ struct sailor_ctx {
     int sm_count = 0;
     TabHdr hdr;                            // host copy of the header
     unsigned char* d_blob = nullptr;
-    uint16_t* d_avail = nullptr;
-    uint16_t* h_avail = nullptr;           // pinned
+    uint16_t* d_avail = nullptr;           // device copy for the kernels that take a pointer (brought up to date lazily)
+    uint16_t* h_avail = nullptr;           // pinned; the snapshot last set
+    bool avail_dirty = false;              // d_avail is older than h_avail
+    PlanOut* d_out_mapped = nullptr;       // device address of h_out (mapped pinned memory)
     Ctrl* d_ctrl = nullptr;
     unsigned int* d_sim_error = nullptr;   // error word of the explicit-batch kernels
-    PlanOut* d_out = nullptr;
     PlanOut* h_out = nullptr;              // pinned
     bool ctrl_dirty = true;                // the counters must be cleared from the host (first call, or after a failed one)
     uint64_t sync_epoch = 1;               // stream synchronisations by this context so far
@@ -403,7 +404,7 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
             PlanParams pp;
             memset(&pp, 0, sizeof(pp));
             pp.blob = ctx->d_blob;
-            pp.avail = ctx->d_avail;
+            memcpy(pp.avail, ctx->h_avail, sizeof(pp.avail));
             pp.ctrl = ctx->d_ctrl;
             pp.cfg_flat_base = sc.d_flat_base;
             pp.sp = d;
@@ -502,7 +503,7 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
     PlanParams pp;
     memset(&pp, 0, sizeof(pp));
     pp.blob = ctx->d_blob;
-    pp.avail = ctx->d_avail;
+    memcpy(pp.avail, ctx->h_avail, sizeof(pp.avail));
     pp.cfg_chunk_start = sc.d_chunk_start;
     pp.cfg_flat_base = sc.d_flat_base;
     pp.ctrl = ctx->d_ctrl;
@@ -522,7 +523,7 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
     pp.p_max = sc.p_max;
     pp.budget = budget;
     pp.min_rate = min_rate;
-    pp.out = ctx->d_out;
+    pp.out = ctx->d_out_mapped;        // the block that ends the pass writes the results straight into pinned host memory
     pp.finish = 1;
     pp.next_budget_factor = next_budget_factor;
     pp.cost_only = next_budget_factor > 0.0 ? 1u : 0u;
@@ -623,6 +624,18 @@ int finish_host_batch(sailor_ctx* ctx) {
         CU(ctx, cudaMemsetAsync(ctx->d_sim_error, 0, sizeof(unsigned int), ctx->stream));
         return SAILOR_E_DEVICE;
     }
+    return SAILOR_OK;
+}
+
+// The device copy of the availability snapshot, for kernels that read it through a pointer.
+int upload_availability(sailor_ctx* ctx) {
+    if (!ctx->avail_dirty) return SAILOR_OK;
+    CU(ctx, cudaEventRecord(ctx->evh0, ctx->stream));
+    CU(ctx, cudaMemcpyAsync(ctx->d_avail, ctx->h_avail, ctx->hdr.R * sizeof(uint16_t), cudaMemcpyHostToDevice, ctx->stream));
+    CU(ctx, cudaEventRecord(ctx->evh1, ctx->stream));
+    ctx->avail_epoch = ctx->sync_epoch;
+    ctx->h2d_fresh = true;
+    ctx->avail_dirty = false;
     return SAILOR_OK;
 }
 
@@ -766,6 +779,7 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     h.off_cmp_mem = put<uint64_t>(blob, nullptr, cmp_mem);
     h.off_cmp_fb = put<double>(blob, nullptr, cmp_fb);
     h.off_cmp_upd = put<double>(blob, nullptr, cmp_upd);
+    blob.resize((blob.size() + 31) & ~(size_t)31);         // a table entry is one 32-byte sector
     h.off_piece = put<PieceRec>(blob, nullptr, cmp_fb);
     h.off_lnk_intra2 = put<double>(blob, nullptr, R * n_mbs);
     h.off_lnk_inter2 = put<double>(blob, nullptr, R * n_mbs);
@@ -793,8 +807,9 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     memset(ctx->h_avail, 0, R_MAX * sizeof(uint16_t));       // availability starts at zero on both sides
     CUF(cudaMalloc(&ctx->d_ctrl, sizeof(Ctrl)));
     CUF(cudaMalloc(&ctx->d_sim_error, sizeof(unsigned int)));
-    CUF(cudaMalloc(&ctx->d_out, sizeof(PlanOut)));
-    CUF(cudaMallocHost(&ctx->h_out, sizeof(PlanOut)));
+    CUF(cudaHostAlloc(&ctx->h_out, sizeof(PlanOut), cudaHostAllocMapped));
+    CUF(cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->d_out_mapped), ctx->h_out, 0));
+    memset(ctx->h_out, 0, sizeof(PlanOut));
     CUF(cudaMalloc(&ctx->d_partial, sizeof(Hit) * SAILOR_K_MAX * ctx->max_grid));
     CUF(cudaMalloc(&ctx->d_partial_n, sizeof(uint32_t) * ctx->max_grid));
     CUF(cudaEventCreate(&ctx->ev0));
@@ -806,7 +821,6 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     CUF(cudaMemsetAsync(ctx->d_avail, 0, R_MAX * sizeof(uint16_t), ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_ctrl, 0, sizeof(Ctrl), ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_sim_error, 0, sizeof(unsigned int), ctx->stream));
-    CUF(cudaMemsetAsync(ctx->d_out, 0, sizeof(PlanOut), ctx->stream));
     {
         const uint32_t n_threads = 4 * T * n_tp * n_mbs + 2 * T * n_tp;
         chain_kernel<<<(n_threads + 127) / 128, 128, 0, ctx->stream>>>(ctx->d_blob);
@@ -839,7 +853,6 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFreeHost(ctx->h_avail);
     cudaFree(ctx->d_ctrl);
     cudaFree(ctx->d_sim_error);
-    cudaFree(ctx->d_out);
     cudaFreeHost(ctx->h_out);
     cudaFree(ctx->d_partial);
     cudaFree(ctx->d_partial_n);
@@ -863,15 +876,12 @@ int sailor_destroy(sailor_ctx* ctx) {
 int sailor_set_availability(sailor_ctx* ctx, const uint16_t* avail) {
     if (!ctx || !avail) return SAILOR_E_ARG;
     DeviceGuard guard(ctx->device);
-    // the pinned staging buffer may still feed the previous copy, unless the stream has been synchronised since
+    // A search takes the snapshot along in its launch parameters; the device copy that the other kernels read
+    // through a pointer is brought up to date when one of them is next enqueued (upload_availability).  The pinned
+    // buffer may still feed such a copy, unless the stream has been synchronised since.
     if (ctx->avail_epoch == ctx->sync_epoch) CU(ctx, stream_sync(ctx));
     memcpy(ctx->h_avail, avail, ctx->hdr.R * sizeof(uint16_t));
-    CU(ctx, cudaEventRecord(ctx->evh0, ctx->stream));
-    CU(ctx, cudaMemcpyAsync(ctx->d_avail, ctx->h_avail, ctx->hdr.R * sizeof(uint16_t), cudaMemcpyHostToDevice,
-                            ctx->stream));
-    CU(ctx, cudaEventRecord(ctx->evh1, ctx->stream));
-    ctx->avail_epoch = ctx->sync_epoch;
-    ctx->h2d_fresh = true;
+    ctx->avail_dirty = true;
     return SAILOR_OK;
 }
 
@@ -908,6 +918,10 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
         sailor_plan_rec* dp = reinterpret_cast<sailor_plan_rec*>(base + 32 * n);
         CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_plan_rec), cudaMemcpyHostToDevice, ctx->stream));
         d_plans = dp;
+    }
+    {
+        const int rc_up = upload_availability(ctx);
+        if (rc_up) return rc_up;
     }
     const uint64_t tiles = (n + BATCH_POOL - 1) / BATCH_POOL;
     const uint64_t cap = (uint64_t)ctx->sm_count * 12;         // three resident blocks per SM, four pools each at least
@@ -965,6 +979,10 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
         sailor_mixed_plan* dp = reinterpret_cast<sailor_mixed_plan*>(base + 32 * n);
         CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_mixed_plan), cudaMemcpyHostToDevice, ctx->stream));
         d_plans = dp;
+    }
+    {
+        const int rc_up = upload_availability(ctx);
+        if (rc_up) return rc_up;
     }
     const uint64_t tiles = (n + SIM_THREADS / 32 - 1) / (SIM_THREADS / 32);     // a warp per plan
     const uint64_t cap = (uint64_t)ctx->sm_count * 32;
@@ -1025,7 +1043,7 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
         CU(ctx, cudaMemsetAsync(&ctx->d_ctrl->min_cost_bits, 0x7f, 2 * sizeof(unsigned long long), ctx->stream));
     }
     ctx->ctrl_dirty = true;            // until this call has gone through
-    CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
+    if (stats) CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
     const bool two_pass = o->budget_factor_over_cheapest > 0.0;
     // a whole-space search with pruning on walks only the prefixes the survey found live
     const bool live = !(o->flags & SAILOR_FLAG_EVAL_ALL) && flat_lo == 0 && flat_hi == total;
@@ -1039,15 +1057,9 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
     rc = enqueue_pass(ctx, o->kind, o->budget_usd_per_iter, two_pass, o->min_iters_per_s, o->flags, flat_lo,
                       flat_hi, live, k, 0.0, &launches, &launched);
     if (rc) return rc;
-    CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
-    if (launched) {
-        CU(ctx, cudaMemcpyAsync(ctx->h_out, ctx->d_out, sizeof(Ctrl) + sizeof(sailor_result) * k, cudaMemcpyDeviceToHost,
-                                ctx->stream));
-        if (stats) CU(ctx, cudaEventRecord(ctx->ev2, ctx->stream));
-    } else {
-        memset(&ctx->h_out->ctrl, 0, sizeof(Ctrl));           // an empty range: nothing ran, nothing was found
-    }
-    CU(ctx, stream_sync(ctx));
+    if (stats) CU(ctx, cudaEventRecord(ctx->ev1, ctx->stream));
+    if (!launched) memset(&ctx->h_out->ctrl, 0, sizeof(Ctrl));    // an empty range: nothing ran, nothing was found
+    CU(ctx, stream_sync(ctx));                                      // the results are in h_out once the kernels are done
     ctx->ctrl_dirty = false;
     const Ctrl& cr = ctx->h_out->ctrl;
     if (cr.error) return SAILOR_E_DEVICE;
@@ -1077,9 +1089,8 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
         CU(ctx, cudaEventElapsedTime(&ms, ctx->ev0, ctx->ev1));
         stats->kernel_ms = ms;
         stats->n_launches = launches;
-        stats->d2h_ms = 0.f;
-        if (launched) CU(ctx, cudaEventElapsedTime(&stats->d2h_ms, ctx->ev1, ctx->ev2));
-        if (ctx->h2d_fresh) {              // the upload was enqueued before this search and is complete by now
+        stats->d2h_ms = 0.f;               // no copy of its own: the results were written in place
+        if (ctx->h2d_fresh) {              // an upload for another entry point was enqueued before this search: complete by now
             CU(ctx, cudaEventElapsedTime(&ctx->h2d_ms, ctx->evh0, ctx->evh1));
             ctx->h2d_fresh = false;
         }
@@ -1151,7 +1162,7 @@ int enqueue_pass_noalloc(sailor_ctx* ctx, NoAllocScratch* sc, const SpaceDesc& d
     PlanParams pp;
     memset(&pp, 0, sizeof(pp));
     pp.blob = ctx->d_blob;
-    pp.avail = ctx->d_avail;
+    memcpy(pp.avail, ctx->h_avail, sizeof(pp.avail));
     pp.cfg_chunk_start = sc->cfg_chunk_start;
     pp.cfg_flat_base = sc->cfg_flat_base;
     pp.ctrl = &sc->ctrl;
@@ -1395,6 +1406,10 @@ static int plan_dp_budget_impl(sailor_ctx* ctx, const SpaceDesc& d, const sailor
     unsigned long long* d_counters = bump.take<unsigned long long>(5);
 
     uint32_t launches = 0;
+    {
+        const int rc_up = upload_availability(ctx);
+        if (rc_up) return rc_up;
+    }
     CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
     CU(ctx, cudaMemsetAsync(d_tabs, 0, tab_bytes, ctx->stream));
     CU(ctx, cudaMemsetAsync(d_counters, 0, 40, ctx->stream));
@@ -1694,6 +1709,10 @@ static int plan_dp_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_zon
     unsigned long long* d_counters = bump.take<unsigned long long>(3);
 
     uint32_t launches = 0;
+    {
+        const int rc_up = upload_availability(ctx);
+        if (rc_up) return rc_up;
+    }
     CU(ctx, cudaEventRecord(ctx->ev0, ctx->stream));
     CU(ctx, cudaMemsetAsync(d_tabs, 0, tab_bytes, ctx->stream));
     CU(ctx, cudaMemsetAsync(d_counters, 0, 24, ctx->stream));
@@ -1984,6 +2003,10 @@ static int plan_mixed_impl(sailor_ctx* ctx, const sailor_mixed_space* s, const s
     sailor_mixed_result* d_results = bump.take<sailor_mixed_result>(SAILOR_K_MAX);
     unsigned long long* d_counters = bump.take<unsigned long long>(9);
 
+    {
+        const int rc_up = upload_availability(ctx);
+        if (rc_up) return rc_up;
+    }
     CU(ctx, cudaMemcpyAsync(d_combs, mt.combs.data(), mt.combs.size() * 8, cudaMemcpyHostToDevice, ctx->stream));
     CU(ctx, cudaMemcpyAsync(d_base, mt.flat_base.data(), mt.flat_base.size() * 8, cudaMemcpyHostToDevice, ctx->stream));
     CU(ctx, cudaMemsetAsync(d_counters, 0, 9 * 8, ctx->stream));

@@ -58,7 +58,8 @@ constexpr unsigned long long COST_BITS_START = 0x7ff0000000000000ull;   // +inf:
 
 struct PlanParams {
     const unsigned char* blob;
-    const uint16_t* avail;
+    uint16_t avail[R_MAX];             // the availability snapshot rides in the launch parameters: a search needs no
+                                       // copy of its own before it, and 128 bytes are well within the parameter space
     const uint32_t* cfg_chunk_start;   // [n_config + 1]
     const uint64_t* cfg_flat_base;     // [n_config]
     Ctrl* ctrl;

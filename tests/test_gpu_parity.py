@@ -376,8 +376,10 @@ def test_plan_argument_errors(make_ctx):
 
 
 def test_stats_report_transfer_times_and_launches(make_ctx):
-    """One launch per pass (the search kernel's last block merges), and the device times of the availability
-    upload and of the result read-back beside the kernel time."""
+    """One launch per pass (the search kernel's last block merges).  A search carries the snapshot in its launch
+    parameters and its kernel writes the results into pinned host memory, so it has no copies of its own to time;
+    the device copy of the snapshot that the batch simulator reads is uploaded when that is next called, and its
+    device time is then reported."""
     w = W.config2()
     cx = make_ctx(w)
     obj = B.make_objective(w)
@@ -385,10 +387,19 @@ def test_stats_report_transfer_times_and_launches(make_ctx):
     B.sailor_set_availability(cx.ctx, w.avail)
     res, st = B.sailor_plan(cx.ctx, cx.space, obj, 4)
     assert st.n_launches == 2 and len(res) == 4           # two passes: cheapest plan, then the budget
-    assert 0.0 < st.h2d_ms < 5.0 and 0.0 < st.d2h_ms < 5.0 and 0.0 < st.kernel_ms < 50.0
+    assert st.d2h_ms == 0.0 and 0.0 < st.kernel_ms < 50.0
     res1, st1 = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, factor=0.0), 4)
     assert st1.n_launches == 1
-    assert st1.h2d_ms == st.h2d_ms                        # no new upload: the last one's time stays
+    # the batch simulator reads the snapshot through a pointer: its next call uploads it, the search after reports it
+    recs = W.random_plans(w, 100, seed=3)
+    half = (w.avail // 2).astype(np.uint16)
+    B.sailor_set_availability(cx.ctx, half)
+    gpu = B.sailor_simulate(cx.ctx, B.pack_records(recs))
+    assert_sim_equal(gpu, Oracle(w, half).simulate_records(recs), "after a new snapshot")
+    _, st2 = B.sailor_plan(cx.ctx, cx.space, obj, 4)
+    assert 0.0 < st2.h2d_ms < 5.0
+    _, st3 = B.sailor_plan(cx.ctx, cx.space, obj, 4)
+    assert st3.h2d_ms == st2.h2d_ms                       # no new upload: the last one's time stays
 
 
 def test_issue_rate_measurement_is_plausible(torch_cuda):
