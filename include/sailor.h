@@ -197,6 +197,16 @@ typedef struct sailor_space {
 #define SAILOR_FLAG_DEGREE_ORDER 2u
 #define SAILOR_FLAG_MIN_TP_ONLY  4u
 
+/* SAILOR_FLAG_F32_SCREEN.  Every candidate is first evaluated in binary32 (from tables rounded once per
+ * configuration); a prefix with all its last digits is evaluated again in binary64, exactly as without the flag,
+ * only when its best binary32 score comes within 1e-4 (relative) of the score a candidate must beat to enter the
+ * top-k, or its cheapest binary32 cost within 1e-4 of the cheapest cost known.  The binary32 evaluation is off by
+ * less than 1.4e-5 (relative; at most 96 stages), so the returned plans, scores, counts and min_feasible_cost are
+ * the ones the search returns without the flag, bit for bit; only the time differs.  Searches without a budget, a
+ * throughput floor or a budget factor only, and not with SAILOR_FLAG_DEGREE_ORDER (E_ARG); not in
+ * sailor_plan_noalloc. */
+#define SAILOR_FLAG_F32_SCREEN   8u
+
 typedef struct sailor_objective {
     uint32_t kind;
     uint32_t flags;

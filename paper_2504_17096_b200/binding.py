@@ -16,7 +16,7 @@ KINDS, T_MAX, Z_MAX, TP_MAX, MBS_MAX, P_MAX, RUN_MAX, SEG_MAX, K_MAX, NP_MAX, ND
 OK, E_ARG, E_RANGE, E_CUDA, E_NOMEM, E_DEVICE = 0, -1, -2, -3, -4, -5
 ST_INVALID, ST_OVER_AVAIL, ST_OOM, ST_BAD_RECORD = 1, 2, 4, 32
 OBJ_MAX_THROUGHPUT, OBJ_MIN_COST, OBJ_MAX_THROUGHPUT_PER_USD = 0, 1, 2
-FLAG_EVAL_ALL, FLAG_DEGREE_ORDER, FLAG_MIN_TP_ONLY = 1, 2, 4
+FLAG_EVAL_ALL, FLAG_DEGREE_ORDER, FLAG_MIN_TP_ONLY, FLAG_F32_SCREEN = 1, 2, 4, 8
 DP_FLAG_INDEX_DENSE, DP_FLAG_INDEX_COMPACT, DP_FLAG_ENUM_BY_TYPE, DP_FLAG_ENUM_BY_ENTRY = 0x100, 0x200, 0x400, 0x800
 DP_FLAG_BUDGET_LOOP, DP_BUDGET_P_MAX = 0x1000, 32
 

@@ -144,7 +144,7 @@ struct SpaceCache {
     std::vector<uint64_t> flat_base;
     uint32_t* d_chunk_start = nullptr;
     uint64_t* d_flat_base = nullptr;
-    size_t smem = 0;
+    size_t smem = 0, smem_screen = 0;      // dynamic shared memory of a search block, without and with the binary32 tables
     // chunks of live prefixes only (see survey_kernel), for whole-space searches with pruning on
     uint32_t* d_live_start = nullptr;      // [n_config + 1]
     uint32_t live_chunks = 0;
@@ -189,7 +189,7 @@ struct sailor_ctx {
     Hit* d_partial = nullptr;
     uint32_t* d_partial_n = nullptr;
     uint32_t max_grid = 0;                 // capacity of the partial-result buffers
-    uint32_t grid_of[12] = {0};            // resident blocks per kernel variant, for the cached space
+    uint32_t grid_of[15] = {0};            // resident blocks per kernel variant, for the cached space
     SpaceCache space;
     cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr, evh0 = nullptr, evh1 = nullptr;
     // explicit-batch staging (grow-only)
@@ -432,6 +432,7 @@ int prepare_space(sailor_ctx* ctx, const sailor_space* s) {
     sc.chunk_start.swap(cs);
     sc.flat_base.swap(fb);
     sc.smem = smem;
+    sc.smem_screen = plan_smem_bytes(ctx->hdr.static_bytes, p_max, ctx->hdr.T, ctx->hdr.Z, (uint32_t)n_config, true);
     sc.valid = true;
     for (uint32_t& g : ctx->grid_of) g = 0;
     return SAILOR_OK;
@@ -451,9 +452,11 @@ uint32_t chunk_of(const sailor_ctx* ctx, uint64_t f) {
 
 using PlanKernel = void (*)(const PlanParams);
 
-constexpr int PLAN_VARIANTS = 12;      // objective x constraint x fused
+constexpr int PLAN_VARIANTS = 15;      // objective x constraint x fused, then the three screened kernels
 
-uint32_t variant_of(uint32_t obj, bool constr, bool fused) { return (obj * 2 + (constr ? 1 : 0)) * 2 + (fused ? 1 : 0); }
+uint32_t variant_of(uint32_t obj, bool constr, bool fused, bool screen = false) {
+    return screen ? 12 + obj : (obj * 2 + (constr ? 1 : 0)) * 2 + (fused ? 1 : 0);
+}
 
 template <bool FUSED>
 PlanKernel pick_kernel_of(uint32_t obj, bool constr) {
@@ -464,7 +467,11 @@ PlanKernel pick_kernel_of(uint32_t obj, bool constr) {
     }
 }
 
-PlanKernel pick_kernel(uint32_t obj, bool constr, bool fused) {
+PlanKernel pick_kernel(uint32_t obj, bool constr, bool fused, bool screen = false) {
+    if (screen)        // unconstrained searches only; they end their pass in finish_kernel
+        return obj == SAILOR_OBJ_MAX_THROUGHPUT ? plan_kernel<0, false, false, true>
+               : obj == SAILOR_OBJ_MIN_COST     ? plan_kernel<1, false, false, true>
+                                                : plan_kernel<2, false, false, true>;
     return fused ? pick_kernel_of<true>(obj, constr) : pick_kernel_of<false>(obj, constr);
 }
 
@@ -547,15 +554,19 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
     if (pp.chunk_hi > pp.chunk_lo) {
         const uint32_t n_chunks = waves ? sc.live_chunks : pp.chunk_hi - pp.chunk_lo;
         const bool constr = budget_from_ctrl || budget > 0.0 || min_rate > 0.0;
-        const bool fused = n_chunks <= FUSED_CHUNKS_PER_BLOCK * 2u * (uint32_t)ctx->sm_count;
-        PlanKernel kern = pick_kernel(obj, constr, fused);
-        const uint32_t variant = variant_of(obj, constr, fused);
+        const bool screen = (flags & SAILOR_FLAG_F32_SCREEN) != 0;
+        const bool fused = !screen && n_chunks <= FUSED_CHUNKS_PER_BLOCK * 2u * (uint32_t)ctx->sm_count;
+        PlanKernel kern = pick_kernel(obj, constr, fused, screen);
+        const uint32_t variant = variant_of(obj, constr, fused, screen);
+        const size_t smem_k = screen ? sc.smem_screen : sc.smem;
+        if (smem_k > (size_t)PLAN_SMEM_CEILING) return SAILOR_E_RANGE;
+        pp.screen = screen ? 1u : 0u;
         uint32_t& resident = ctx->grid_of[variant];
         if (resident == 0) {       // once per (space, kernel variant): size the grid
             int rc_opt = smem_optin(ctx, kern, variant);
             if (rc_opt) return rc_opt;
             int per_sm = 0;
-            CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, sc.smem));
+            CU(ctx, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, PLAN_THREADS, smem_k));
             if (per_sm < 1) return SAILOR_E_RANGE;
             resident = (uint32_t)per_sm * (uint32_t)ctx->sm_count;
             if (resident > ctx->max_grid) resident = ctx->max_grid;
@@ -564,7 +575,7 @@ int enqueue_pass(sailor_ctx* ctx, uint32_t obj, double budget, bool budget_from_
         const uint32_t batch = n_chunks / (grid * 32u);
         pp.batch = batch < 1 ? 1 : (batch > 16 ? 16 : batch);
         if (!waves) {
-            kern<<<grid, PLAN_THREADS, sc.smem, ctx->stream>>>(pp);
+            kern<<<grid, PLAN_THREADS, smem_k, ctx->stream>>>(pp);
             CU(ctx, cudaGetLastError());
             ++*n_launches;
         } else {
@@ -1022,7 +1033,12 @@ static int plan_range_impl(sailor_ctx* ctx, const sailor_space* s, const sailor_
     if (std::isnan(o->budget_usd_per_iter) || std::isnan(o->min_iters_per_s) ||
         std::isnan(o->budget_factor_over_cheapest))
         return SAILOR_E_ARG;
-    if (o->flags & ~(SAILOR_FLAG_EVAL_ALL | SAILOR_FLAG_DEGREE_ORDER | SAILOR_FLAG_MIN_TP_ONLY)) return SAILOR_E_ARG;
+    if (o->flags & ~(SAILOR_FLAG_EVAL_ALL | SAILOR_FLAG_DEGREE_ORDER | SAILOR_FLAG_MIN_TP_ONLY | SAILOR_FLAG_F32_SCREEN))
+        return SAILOR_E_ARG;
+    if ((o->flags & SAILOR_FLAG_F32_SCREEN) &&
+        (o->budget_usd_per_iter > 0.0 || o->min_iters_per_s > 0.0 || o->budget_factor_over_cheapest > 0.0 ||
+         (o->flags & SAILOR_FLAG_DEGREE_ORDER)))
+        return SAILOR_E_ARG;                                   // the screen covers unconstrained searches
     DeviceGuard guard(ctx->device);
     int rc = prepare_space(ctx, s);
     if (rc) return rc;

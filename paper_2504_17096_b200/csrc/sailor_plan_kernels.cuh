@@ -24,6 +24,9 @@ constexpr int PLAN_WARPS = PLAN_THREADS / 32;
 #ifndef PLAN_MIN_BLOCKS
 #define PLAN_MIN_BLOCKS 2
 #endif
+#ifndef PLAN_SCREEN_BLOCKS
+#define PLAN_SCREEN_BLOCKS 3        // resident blocks per SM the screened kernels are compiled for (binary32 state is half as wide)
+#endif
 constexpr unsigned FULL = 0xffffffffu;
 constexpr uint32_t WAIT_LIMIT = 1u << 22;   // bound of every spin-wait in this file
 
@@ -82,6 +85,7 @@ struct PlanParams {
     uint32_t finish;                   // this launch ends a pass: its last block merges the lists and writes `out`
     double next_budget_factor;         // > 0: the finishing block writes ctrl->budget = factor * best cost (next pass)
     uint32_t cost_only;                // the pass only looks for the cheapest feasible cost (no lists, no result records)
+    uint32_t screen;                   // candidates are first evaluated in binary32 (SCREEN kernels): sizes the shared tables
     const uint4* cfg_cache;            // non-null: the per-configuration tables, built once per space (cfg_cache_kernel)
     uint32_t cache_head16, cache_arr16;    // 16-byte words of a cached record: CfgShared head, then the arrays
     double budget;                     // <= 0: none
@@ -193,6 +197,22 @@ struct alignas(16) SegRec {                  // one per (segment, digit); 64 byt
     double rate;                 // D * tp * price per second of one stage
 };
 
+// The binary32 screen (optional search mode): every candidate is first evaluated in binary32 from rounded copies of
+// the tables; an item (a prefix with all its last digits) is evaluated again in binary64, exactly as without the
+// screen, only when its best binary32 score comes within SCREEN_BAND of the score a candidate must beat to enter
+// the top-k, or its cheapest binary32 cost within SCREEN_BAND of the cheapest cost known.  A binary32 evaluation
+// rounds each table entry once (2^-24) and adds at most P + 4 positive terms (each addition 2^-24), multiplies
+// twice and, for throughput per cost, once more: a relative error below (P + 12) * 2^-24 < 7e-6 for P <= 96 in time
+// and cost, below 1.4e-5 in their product.  The band is 1e-4, so every candidate whose exact score could enter the
+// list (or whose exact cost could be the cheapest) is looked at exactly: lists, counts and statistics are the
+// exact search's, bit for bit.
+constexpr double SCREEN_BAND = 1e-4;
+
+struct alignas(16) SegRec32 {                // SegRec rounded to binary32; 32 bytes
+    float v[N_RUNS];
+    float tmax, sync, upd, rate;
+};
+
 struct alignas(16) CfgShared {
     // scalars (written by thread 0 / the build, read by all)
     Config cfg;
@@ -226,6 +246,7 @@ struct alignas(16) CfgShared {
     uint64_t params[SAILOR_P_MAX];
     unsigned long long stat[7];
     unsigned long long thr_bits;     // the block's copy of Ctrl::thr_bits, lowered by its own warps as their lists fill
+    unsigned long long minc_bits;    // screened search: the cheapest exact cost the block's warps have seen (ordered bits)
     uint64_t mbar;
 };
 
@@ -238,13 +259,23 @@ struct CfgArrays {               // pointers into dynamic shared memory
     uint32_t* availv;            // [R]
     uint32_t* tz;                // [R]      type | zone << 8 of a digit
     uint32_t* chunk_tab;         // [n_config + 1] copy of the chunk offsets (spaces of fewer than PLAN_CFG_SMEM configurations)
+    SegRec32* rec32;             // screened search: rec, c2x, commx rounded to binary32 (same shapes and padding)
+    float* c2x32;
+    float* commx32;
 };
 
 constexpr uint32_t PLAN_CFG_SMEM = 4096;
 
-__host__ __device__ inline size_t plan_smem_bytes(uint32_t static_bytes, uint32_t p_max, uint32_t T, uint32_t Z, uint32_t n_config) {
+__host__ __device__ inline size_t plan_screen_bytes(uint32_t T, uint32_t Z) {
+    const size_t R = (size_t)T * Z;
+    return sizeof(SegRec32) * (SAILOR_SEG_MAX * R + PLAN_PAD) + sizeof(float) * ((R + PLAN_PAD) * R + (R + PLAN_PAD) * Z) + 32;
+}
+
+__host__ __device__ inline size_t plan_smem_bytes(uint32_t static_bytes, uint32_t p_max, uint32_t T, uint32_t Z, uint32_t n_config,
+                                                  bool screen = false) {
     const size_t R = (size_t)T * Z;
     size_t n = static_bytes;
+    if (screen) n += plan_screen_bytes(T, Z);
     if (n_config < 4096) n += sizeof(uint32_t) * ((size_t)n_config + 1);
     n += sizeof(SegRec) * (SAILOR_SEG_MAX * R + PLAN_PAD);               // padding digits, see walk_fast
     n += sizeof(double) * ((R + PLAN_PAD) * R + (R + PLAN_PAD) * Z + (size_t)SAILOR_SEG_MAX * T + 2 * (size_t)p_max * T);
@@ -263,7 +294,7 @@ __host__ __device__ inline uint32_t cache_arr16(uint32_t T, uint32_t Z) {
 }
 
 __device__ __forceinline__ void carve(unsigned char* dyn, uint32_t static_bytes, uint32_t p_max, uint32_t T,
-                                      uint32_t Z, CfgArrays& a) {
+                                      uint32_t Z, CfgArrays& a, uint32_t n_config = 0, bool screen = false) {
     const uint32_t R = T * Z;
     a.rec = reinterpret_cast<SegRec*>(dyn + static_bytes);           // static_bytes is a multiple of 16
     double* p = reinterpret_cast<double*>(a.rec + (size_t)SAILOR_SEG_MAX * R + PLAN_PAD);
@@ -275,6 +306,32 @@ __device__ __forceinline__ void carve(unsigned char* dyn, uint32_t static_bytes,
     a.availv = reinterpret_cast<uint32_t*>(p);
     a.tz = a.availv + R;
     a.chunk_tab = a.tz + R;
+    a.rec32 = nullptr;
+    a.c2x32 = a.commx32 = nullptr;
+    if (screen) {
+        uintptr_t at = reinterpret_cast<uintptr_t>(a.chunk_tab + (n_config < PLAN_CFG_SMEM ? n_config + 1 : 0));
+        at = (at + 15) & ~(uintptr_t)15;
+        a.rec32 = reinterpret_cast<SegRec32*>(at);
+        a.c2x32 = reinterpret_cast<float*>(a.rec32 + (size_t)SAILOR_SEG_MAX * R + PLAN_PAD);
+        a.commx32 = a.c2x32 + (size_t)(R + PLAN_PAD) * R;
+    }
+}
+
+// The binary32 copies of the tables of the configuration just built or loaded.  Called by the whole block; ends
+// synchronised.
+__device__ __forceinline__ void round_config32(const CfgArrays& a, uint32_t R, uint32_t Z) {
+    const uint32_t tid = threadIdx.x;
+    for (uint32_t x = tid; x < SAILOR_SEG_MAX * R + PLAN_PAD; x += PLAN_THREADS) {
+        const SegRec& r = a.rec[x];
+        SegRec32 q;
+        for (int j = 0; j < N_RUNS; ++j) q.v[j] = __double2float_rn(r.v[j]);
+        q.tmax = __double2float_rn(r.tmax); q.sync = __double2float_rn(r.sync);
+        q.upd = __double2float_rn(r.upd); q.rate = __double2float_rn(r.rate);
+        a.rec32[x] = q;
+    }
+    for (uint32_t x = tid; x < (R + PLAN_PAD) * R; x += PLAN_THREADS) a.c2x32[x] = __double2float_rn(a.c2x[x]);
+    for (uint32_t x = tid; x < (R + PLAN_PAD) * Z; x += PLAN_THREADS) a.commx32[x] = __double2float_rn(a.commx[x]);
+    __syncthreads();
 }
 
 // Run of stage i: 0 = stage 0 with the embedding, 1 = one extra block, 2 = plain, 3 = final stage.
@@ -585,6 +642,87 @@ __device__ __forceinline__ void eval_candidates(const CfgShared& cs, const ItemS
     }
 }
 
+// ---- the binary32 screen: the same walk from the rounded tables ---------------------------------------------
+__device__ __forceinline__ float fadd(float a, float b) { return __fadd_rn(a, b); }
+__device__ __forceinline__ float fmul(float a, float b) { return __fmul_rn(a, b); }
+__device__ __forceinline__ float fmaxf_sel(float a, float b) { return fmaxf(a, b); }      // one instruction in binary32; no NaN occurs
+
+struct ItemState32 {
+    float acc, mx, sy, up, rate, cc, fb_b;
+    const SegRec32* recs;
+    const float* c2x_col;
+    const float* comm_col;
+};
+
+template <int NSEG, int N2, int W>
+__device__ __forceinline__ void eval_candidates32(const CfgShared& cs, const ItemState32& it, uint32_t Z, uint32_t R,
+                                                  uint32_t d, float nb, float (&t_iter)[W], float (&cost)[W]) {
+    constexpr uint32_t last = NSEG - 1;
+    const SegRec32* rc = it.recs + d;
+    float t_sum[W], t_max[W], c_comm[W], r[W];
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+        t_sum[w] = it.acc; t_max[w] = it.mx; c_comm[w] = it.cc; r[w] = it.rate;
+        if (NSEG > 1) {
+            const float tb = fadd(it.fb_b, it.c2x_col[(d + w) * R]);
+            t_sum[w] = fadd(t_sum[w], tb);
+            t_max[w] = fmaxf_sel(t_max[w], tb);
+            c_comm[w] = fadd(c_comm[w], it.comm_col[(d + w) * Z]);
+        }
+    }
+#define SAILOR_STAGE32(RUN)                                                        \
+    _Pragma("unroll") for (int w = 0; w < W; ++w) {                                \
+        t_sum[w] = fadd(t_sum[w], rc[w].v[RUN]);                                   \
+        r[w] = fadd(r[w], rc[w].rate);                                             \
+    }
+    if (N2 >= 0) {
+#pragma unroll
+        for (int j = 0; j < N2; ++j) { SAILOR_STAGE32(2) }
+        SAILOR_STAGE32(3)
+    } else {
+        const uint32_t n0 = cs.n_run[last][0], n1 = cs.n_run[last][1], n2 = cs.n_run[last][2], n3 = cs.n_run[last][3];
+        if (n0) { SAILOR_STAGE32(0) }
+        for (uint32_t j = 0; j < n1; ++j) { SAILOR_STAGE32(1) }
+        uint32_t j = n2;
+        for (; j >= 4; j -= 4) { SAILOR_STAGE32(2) SAILOR_STAGE32(2) SAILOR_STAGE32(2) SAILOR_STAGE32(2) }
+        if (j & 2) { SAILOR_STAGE32(2) SAILOR_STAGE32(2) }
+        if (j & 1) { SAILOR_STAGE32(2) }
+        if (n3) { SAILOR_STAGE32(3) }
+    }
+#undef SAILOR_STAGE32
+#pragma unroll
+    for (int w = 0; w < W; ++w) {
+        t_max[w] = fmaxf_sel(t_max[w], rc[w].tmax);
+        const float t_pp = fadd(t_sum[w], fmul(nb, t_max[w]));
+        t_iter[w] = fadd(fadd(t_pp, fmaxf_sel(it.sy, rc[w].sync)), fmaxf_sel(it.up, rc[w].upd));
+        cost[w] = fadd(fmul(r[w], t_iter[w]), c_comm[w]);
+    }
+}
+
+// Binary32 pass over the candidates of one item: the lane's best score and cheapest cost, both approximate.
+template <int NSEG, int OBJ, int N2>
+__device__ __forceinline__ void walk_fast32(const CfgShared& cs, const ItemState32& it, uint64_t ok, uint64_t walk,
+                                            uint32_t Z, uint32_t R, float& best, float& min_cost) {
+    const float nb = (float)cs.n_b;
+    constexpr uint32_t U = PLAN_DIGITS_PER_STEP;
+    for (uint32_t half = 0; half * 32 < R; ++half) {
+        const uint32_t wm = (uint32_t)(walk >> (32 * half)), om = (uint32_t)(ok >> (32 * half));
+        const uint32_t d_end = min(R - 32 * half, 32u);
+        for (uint32_t dd = 0; dd < d_end; dd += U) {
+            if (!((wm >> dd) & ((1u << U) - 1u))) continue;   // warp-uniform
+            float t[U], c[U];
+            eval_candidates32<NSEG, N2, (int)U>(cs, it, Z, R, 32 * half + dd, nb, t, c);
+#pragma unroll
+            for (uint32_t u = 0; u < U; ++u) {
+                const bool g = (om >> (dd + u)) & 1u;
+                const float sc = OBJ == SAILOR_OBJ_MAX_THROUGHPUT ? t[u] : OBJ == SAILOR_OBJ_MIN_COST ? c[u] : fmul(t[u], c[u]);
+                min_cost = fminf(min_cost, g ? c[u] : min_cost);
+                best = fminf(best, g ? sc : best);
+            }
+        }
+    }
+}
+
 template <int OBJ>
 __device__ __forceinline__ double score_of(double t_iter, double cost) {
     return OBJ == SAILOR_OBJ_MAX_THROUGHPUT ? t_iter : OBJ == SAILOR_OBJ_MIN_COST ? cost : mul_rn(t_iter, cost);
@@ -634,7 +772,7 @@ __device__ __forceinline__ void walk_fast(const PlanParams& pp, const CfgShared&
 template <int NSEG, int OBJ, bool CONSTR, int N2>
 __device__ __forceinline__ void walk_offer(const PlanParams& pp, const CfgShared& cs, const ItemState& it,
                                            uint32_t Z, uint32_t R, double budget, uint64_t item_flat,
-                                           WarpTopK& top, uint32_t lane, double outer_thr) {
+                                           WarpTopK& top, uint32_t lane, double outer_thr, double& min_cost) {
     const double nb = (double)cs.n_b;
     for (uint32_t d = 0; d < R; ++d) {
         if (!((it.walk >> d) & 1ull)) continue;               // warp-uniform
@@ -643,6 +781,7 @@ __device__ __forceinline__ void walk_offer(const PlanParams& pp, const CfgShared
         const double t = t1[0], c = c1[0];
         const bool good = ((it.ok >> d) & 1ull) && within<CONSTR>(pp, budget, t, c);
         const double score = score_of<OBJ>(t, c);
+        min_cost = (good && c < min_cost) ? c : min_cost;      // (the fast pass of the exact search has seen it already)
         const bool want = good && score <= top.thr_score && score <= outer_thr;
         if (__any_sync(FULL, want)) top.offer(want, score, item_flat + d, pp.k, lane);
     }
@@ -651,7 +790,7 @@ __device__ __forceinline__ void walk_offer(const PlanParams& pp, const CfgShared
 // One item per lane: fixed prefix digits, walk the last segment's digit.
 // N2 >= 0 fixes the shape of the last segment at compile time (N2 plain stages, then the final
 // stage, nothing else), which makes the candidate loop straight-line code; N2 < 0 is the general form.
-template <int NSEG, int OBJ, bool CONSTR, int N2>
+template <int NSEG, int OBJ, bool CONSTR, int N2, bool SCREEN>
 __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared& cs, const CfgArrays& a,
                                           uint32_t T, uint32_t Z, uint32_t R, uint32_t q, bool active,
                                           uint64_t item_flat, double budget, WarpTopK& top, Counters& cnt,
@@ -788,6 +927,32 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     it.c2x_col = a.c2x + d_prev;
     it.comm_col = a.commx + z_prev;
 
+    if (SCREEN) {
+        // binary32 first; the item is walked exactly only if it may hold a member of the top-k or the cheapest plan
+        ItemState32 s32;
+        s32.acc = __double2float_rn(acc); s32.mx = __double2float_rn(mx); s32.sy = __double2float_rn(sy);
+        s32.up = __double2float_rn(up); s32.rate = __double2float_rn(rate); s32.cc = __double2float_rn(cc);
+        s32.fb_b = __double2float_rn(it.fb_b);
+        s32.recs = a.rec32 + last * R;
+        s32.c2x_col = a.c2x32 + d_prev;
+        s32.comm_col = a.commx32 + z_prev;
+        const float f_inf = __int_as_float(0x7f800000);
+        float best32 = f_inf, minc32 = f_inf;
+        walk_fast32<NSEG, OBJ, N2>(cs, s32, ok, walk, Z, R, best32, minc32);
+        const double outer_thr = __longlong_as_double((long long)*reinterpret_cast<const volatile unsigned long long*>(&cs.thr_bits));
+        const double outer_minc = __longlong_as_double((long long)*reinterpret_cast<const volatile unsigned long long*>(&cs.minc_bits));
+        const double thr = top.thr_score < outer_thr ? top.thr_score : outer_thr;
+        const bool need = best32 < f_inf && ((double)best32 <= thr * (1.0 + SCREEN_BAND) || (double)minc32 <= outer_minc * (1.0 + SCREEN_BAND));
+        if (__any_sync(FULL, need)) {
+            const double before = top.thr_score, mc_before = cnt.min_cost;
+            walk_offer<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, item_flat, top, lane, outer_thr, cnt.min_cost);
+            if (lane == 0 && top.thr_score < before)
+                atomicMin(const_cast<unsigned long long*>(&cs.thr_bits), (unsigned long long)__double_as_longlong(top.thr_score));
+            if (cnt.min_cost < mc_before)
+                atomicMin(const_cast<unsigned long long*>(&cs.minc_bits), (unsigned long long)__double_as_longlong(cnt.min_cost));
+        }
+        return;
+    }
     // fast pass: no votes, no list updates; each lane keeps its item's best score
     double best = make_inf();
     uint32_t feas = 0;
@@ -803,7 +968,7 @@ __device__ __forceinline__ void run_items(const PlanParams& pp, const CfgShared&
     const double outer_thr = __longlong_as_double((long long)*reinterpret_cast<const volatile unsigned long long*>(&cs.thr_bits));
     if (!pp.cost_only && __any_sync(FULL, best < make_inf() && best <= top.thr_score && best <= outer_thr)) {   // best == inf: no feasible candidate
         const double before = top.thr_score;
-        walk_offer<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, item_flat, top, lane, outer_thr);
+        walk_offer<NSEG, OBJ, CONSTR, N2>(pp, cs, it, Z, R, budget, item_flat, top, lane, outer_thr, cnt.min_cost);
         if (lane == 0 && top.thr_score < before)
             atomicMin(const_cast<unsigned long long*>(&cs.thr_bits), (unsigned long long)__double_as_longlong(top.thr_score));
     }
@@ -955,8 +1120,9 @@ __device__ __noinline__ void finish_pass(const PlanParams& pp, const TabView& v,
 // FUSED: the block that hands in its list last also ends the pass (one launch per pass: what small searches, bound
 // by launch and hand-over latencies, want).  Not FUSED: the lists are left for finish_kernel (the call inside the
 // kernel costs the candidate loop a few registers, which long searches would pay for in every iteration).
-template <int OBJ, bool CONSTR, bool FUSED>
-__global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(const __grid_constant__ PlanParams pp) {
+// SCREEN: candidates are evaluated in binary32 first (unconstrained searches; see SCREEN_BAND).
+template <int OBJ, bool CONSTR, bool FUSED, bool SCREEN = false>
+__global__ void __launch_bounds__(PLAN_THREADS, SCREEN ? PLAN_SCREEN_BLOCKS : PLAN_MIN_BLOCKS) plan_kernel(const __grid_constant__ PlanParams pp) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ CfgShared cs;
     __shared__ Hit s_hits[PLAN_WARPS][SAILOR_K_MAX];
@@ -976,10 +1142,11 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
     v.bind(dyn, pp.blob);
     const uint32_t T = v.h->T, Z = v.h->Z, R = v.h->R;
     CfgArrays a;
-    carve(dyn, static_bytes, pp.p_max, T, Z, a);
+    carve(dyn, static_bytes, pp.p_max, T, Z, a, pp.n_config, SCREEN);
 
     if (tid == 0) {
         cs.cur_config = 0xffffffffu;
+        cs.minc_bits = COST_BITS_START;
         cs.magic = (uint32_t)(0x100000000ull / (gh->R ? gh->R : 1u)) + 1u;      // for x / R, see CfgShared
     }
     if (tid < 7) cs.stat[tid] = 0;
@@ -1066,6 +1233,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
                 __syncthreads();
                 if (pp.cfg_cache) load_config(pp, cs, a, R, c);
                 else build_config(pp, v, cs, a, c);
+                if (SCREEN) round_config32(a, R, Z);
             }
             const uint32_t q = (ch - chunk_start[c]) * PLAN_THREADS + tid;    // < R^3 + 256 <= 2^18 + 256
             const bool active = q < (cs.packed ? cs.live_items : cs.n_items);
@@ -1084,7 +1252,7 @@ __global__ void __launch_bounds__(PLAN_THREADS, PLAN_MIN_BLOCKS) plan_kernel(con
             // the bulk of every space has four segments: pick the straight-line loop for its common shapes
             const int fixed = (cs.n_run[3][0] == 0 && cs.n_run[3][1] == 0 && cs.n_run[3][3] == 1 && cs.n_run[3][2] <= 3)
                                   ? (int)cs.n_run[3][2] : -1;
-#define SAILOR_RUN(NS, NF) run_items<NS, OBJ, CONSTR, NF>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane)
+#define SAILOR_RUN(NS, NF) run_items<NS, OBJ, CONSTR, NF, SCREEN>(pp, cs, a, T, Z, R, q, active, item_flat, budget, top, cnt, lane)
             switch (cs.cfg.nseg) {
                 case 1: SAILOR_RUN(1, -1); break;
                 case 2: SAILOR_RUN(2, -1); break;

@@ -370,7 +370,7 @@ def test_plan_argument_errors(make_ctx):
     bad = B.make_space(w)
     bad.seg_max = 5
     assert L.sailor_plan(cx.ctx, C.byref(bad), C.byref(obj), 1, res, C.byref(n), None) == B.E_RANGE
-    for flags in (8, 0x100, 1 << 31):                    # flags this entry point does not know
+    for flags in (16, 0x100, 1 << 31):                   # flags this entry point does not know
         odd = B.make_objective(w, flags=flags)
         assert L.sailor_plan(cx.ctx, C.byref(cx.space), C.byref(odd), 1, res, C.byref(n), None) == B.E_ARG
 
@@ -400,6 +400,55 @@ def test_stats_report_transfer_times_and_launches(make_ctx):
     assert 0.0 < st2.h2d_ms < 5.0
     _, st3 = B.sailor_plan(cx.ctx, cx.space, obj, 4)
     assert st3.h2d_ms == st2.h2d_ms                       # no new upload: the last one's time stays
+
+
+def _same_search(a, b, what):
+    (res_a, st_a), (res_b, st_b) = a, b
+    assert [(r.flat, r.score, r.t_iter, r.cost, r.peak_mem, r.status) for r in res_a] == \
+           [(r.flat, r.score, r.t_iter, r.cost, r.peak_mem, r.status) for r in res_b], what
+    assert {k: getattr(st_a, k) for k in COUNT_KEYS} == {k: getattr(st_b, k) for k in COUNT_KEYS}, what
+    assert st_a.min_feasible_cost == st_b.min_feasible_cost, what
+
+
+def test_f32_screen_returns_the_exact_search(make_ctx):
+    """SAILOR_FLAG_F32_SCREEN evaluates every candidate in binary32 first and walks an item exactly only when it may
+    matter: lists, scores, counts and the cheapest cost must be those of the exact search, bit for bit, and the
+    oracle's."""
+    rng = W.SplitMix64(77)
+    for case in range(10):                                   # tiny spaces against the oracle, all objectives
+        T, Z = rng.randint(1, 4), rng.randint(1, 3)
+        w = W.tiny(seed=300 + case, n_types=T, n_zones=Z, L=rng.randint(2, 9), seg_max=rng.randint(1, 4),
+                   objective=case % 3, alpha=rng.uniform() * 1e-4)
+        cx = make_ctx(w)
+        o = Oracle(w)
+        n = o.space_size()
+        k = rng.randint(1, 32)
+        lo, hi = (0, n) if case % 2 else (rng.randint(0, n // 2), rng.randint(n // 2, n))
+        for extra in (0, B.FLAG_EVAL_ALL):
+            hits, counts = o.search(w.objective, k, lo=lo, hi=hi)
+            res, st = B.sailor_plan_range(cx.ctx, cx.space, B.make_objective(w, flags=B.FLAG_F32_SCREEN | extra), lo, hi, k)
+            assert_plan_equal(res, st, hits, counts, o, f"case {case} flags={extra}")
+    for cfg, k in ((1, 32), (6, 16), (3, 16)):               # workloads: against the exact search (itself checked above)
+        w = W.CONFIGS[cfg]()
+        cx = make_ctx(w)
+        kw = dict(budget=0.0, min_rate=0.0, factor=0.0)
+        for extra in (0, B.FLAG_EVAL_ALL, B.FLAG_MIN_TP_ONLY):
+            exact = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=extra, **kw), k)
+            screened = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=extra | B.FLAG_F32_SCREEN, **kw), k)
+            _same_search(exact, screened, f"cfg{cfg} flags={extra}")
+    w = W.config5()
+    cx = make_ctx(w)
+    for extra in (0, B.FLAG_EVAL_ALL):
+        exact = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=extra), 32)
+        screened = B.sailor_plan(cx.ctx, cx.space, B.make_objective(w, flags=extra | B.FLAG_F32_SCREEN), 32)
+        _same_search(exact, screened, f"cfg5 flags={extra}")
+    # the screen is for unconstrained searches
+    L = B.load()
+    res = (B.Result * 4)()
+    nf = C.c_uint32()
+    for bad in (B.make_objective(w, flags=B.FLAG_F32_SCREEN, budget=1.0), B.make_objective(w, flags=B.FLAG_F32_SCREEN, min_rate=1.0),
+                B.make_objective(w, flags=B.FLAG_F32_SCREEN, factor=1.2), B.make_objective(w, flags=B.FLAG_F32_SCREEN | B.FLAG_DEGREE_ORDER)):
+        assert L.sailor_plan(cx.ctx, C.byref(cx.space), C.byref(bad), 4, res, C.byref(nf), None) == B.E_ARG
 
 
 def test_issue_rate_measurement_is_plausible(torch_cuda):
