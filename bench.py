@@ -15,7 +15,8 @@ Hooks for the profiling commands quoted under profiles/ (they change what is run
 timed): `--only-p P ...` keeps only those pipeline depths of the workload (a small case for ncu),
 `--dp-only` runs just the dynamic-programming search, `--dp-workspace-gib` bounds its tables, `--sim-only`
 runs just the explicit-batch kernels,
-`--no-cpu` / `--no-aux` drop the oracle leg / the secondary measurements, and
+`--f32-screen` times the search with the binary32 screen on, `--no-cpu` / `--no-aux` drop the oracle leg / the
+secondary measurements, and
 `--write-counters LOG.csv` turns an ncu `--csv` log of one plan_kernel launch into the counter file
 the roofline figure reads (stamped with a hash of the kernel sources it was captured on).
 """
@@ -263,6 +264,51 @@ def cold_search(B, torch, dev, w, flags: int = 0) -> dict:
     return {"create_s": t1 - t0, "first_search_s": t2 - t1, "cold_search_s": t2 - t0, "found": len(res)}
 
 
+def dp_budget_loop(B, ctx, w, budget: float) -> dict:
+    """The per-stage recursion steered by the budget (Sec. 4.2.3) next to the plain check of the budget on the
+    unlimited recursion's plans: workload 2 with pipelines of up to 8 stages, every zone order."""
+    sub = W.config2()
+    sub.p_values = [p for p in sub.p_values if p <= 8]
+    sp = B.make_space(sub)
+    orders = B.all_zone_orders(sub.n_zones)
+    out = {"budget": budget, "problems": None}
+    for name, loop in (("check_only", False), ("budget_loop", True)):
+        B.sailor_plan_dp(ctx, sp, orders, K_TOP, budget=budget, budget_loop=loop)
+        ts = []
+        for _ in range(3):
+            t0 = time.perf_counter()
+            res, st = B.sailor_plan_dp(ctx, sp, orders, K_TOP, budget=budget, budget_loop=loop)
+            ts.append(time.perf_counter() - t0)
+        out["problems"] = int(st.n_problems)
+        out[name] = {"search_s": statistics.median(ts), "kernel_ms": st.kernel_ms, "with_a_plan": int(st.n_solved),
+                     "within_budget": int(st.n_solved - st.n_over_constraint), "unfinished": int(st.n_unfinished),
+                     "calls_or_entries": int(st.n_states), "best_t_iter": res[0].t_iter if res else None}
+    return out
+
+
+def mixed_search(B, ctx, w) -> dict:
+    """Search over plans whose stages mix GPU types among their replicas: workload 2's model and cluster, two
+    pipeline depths, replicas split in quarters, next to the same space with one type per stage."""
+    sub = W.config2()
+    sub.p_values, sub.mbs_idx, sub.d_values = [2, 4], [sub.mbs_idx[1]], [4, 8]
+    tps = [0, 1, 2]
+    obj = B.Objective(W.OBJ_MAX_THROUGHPUT, 0, 0.0, 0.0, 0.0)
+    out = {}
+    for name, gran in (("one_type_per_stage", 1), ("quarters", 4)):
+        sp = B.make_mixed_space(sub, gran, tps)
+        B.sailor_plan_mixed(ctx, sp, obj, K_TOP)
+        ts = []
+        for _ in range(3):
+            t0 = time.perf_counter()
+            res, st = B.sailor_plan_mixed(ctx, sp, obj, K_TOP)
+            ts.append(time.perf_counter() - t0)
+        out[name] = {"candidates": int(st.n_total), "feasible": int(st.n_feasible), "search_s": statistics.median(ts),
+                     "kernel_ms": st.kernel_ms, "plans_per_s": st.n_total / (st.kernel_ms / 1e3),
+                     "best_t_iter": res[0].t_iter if res else None,
+                     "best_mixes_types": bool(res and any(s.n_groups > 1 for s in res[0].plan.stage[: res[0].plan.P]))}
+    return out
+
+
 def explicit_batches(B, torch, dev) -> dict:
     """sailor_simulate / sailor_simulate_mixed on batches resident in HBM (larger than L2), CUDA events."""
     out = {}
@@ -354,6 +400,9 @@ def aux_measurements(B, torch, dev, oracle_cfg4=None) -> dict:
                                 "cold_search_s": cold["cold_search_s"], "cold": cold}
             out[f"cfg{cfg}"]["pruning_modes"] = pruning_modes(B, ctx, w, sp)
             out[f"cfg{cfg}"]["dp"] = dp_search(B, ctx, w, sp)
+            if cfg == 2:
+                out["cfg2"]["dp_budget_loop"] = dp_budget_loop(B, ctx, w, st.budget_used)
+                out["cfg2"]["mixed_search"] = mixed_search(B, ctx, w)
         finally:
             B.sailor_destroy(ctx)
     out.update(explicit_batches(B, torch, dev))
@@ -475,7 +524,7 @@ def run_ours(args) -> None:
     stream = torch.cuda.current_stream()
     ctx = B.sailor_create(w, local, stream.cuda_stream)
     space = B.make_space(w)
-    obj = B.make_objective(w, flags=B.FLAG_EVAL_ALL)
+    obj = B.make_objective(w, flags=B.FLAG_EVAL_ALL | (B.FLAG_F32_SCREEN if args.f32_screen else 0))
     n = B.sailor_space_size(ctx, space)
     lo, hi = (sharding.split_by_cost(sharding.subspace_costs(w), world, rank) if split else (0, n))
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than the 126 MB L2
@@ -568,7 +617,8 @@ def run_ours(args) -> None:
         rates = B.sailor_measure_issue_rates(local, stream.cuda_stream, 5)
         sm_max = float(peaks.get("sm_max_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0)
         units_x_clock = rates.sm_count * ISSUE_PER_SM * sm_max * 1e6                 # warp-instructions/s
-        counters, why_not = (read_counters(w.name) if world == 1 else (None, "counters are of a whole-space launch"))
+        counters, why_not = (read_counters(w.name) if world == 1 and not args.f32_screen
+                             else (None, "counters are of a whole-space launch of the binary64 search"))
         roofline = {"bound": "alu", "unit": "warp-inst/s", "achieved": None, "peak": rates.ffma_warp_inst_per_s,
                     "frac": None, "traffic": None,
                     "peak_kind": "measured: FP32 multiply-add stream, 8 chains per thread, 4 x 256 threads per SM",
@@ -625,10 +675,23 @@ def run_ours(args) -> None:
                                                     "pruning_modes": pruning_modes(B, ctx, w, space),
                                                     "dp": dp_search(B, ctx, w, space)}
             aux[args.workload + "_every_candidate"] = {"cold": cold_search(B, torch, local, w, B.FLAG_EVAL_ALL)}
+            # the same search with the binary32 screen: identical results, the second figure
+            obs = B.make_objective(w, flags=B.FLAG_EVAL_ALL | B.FLAG_F32_SCREEN)
+            for _ in range(3):
+                B.sailor_plan(ctx, space, obs, K_TOP)
+            km = []
+            for _ in range(10):
+                flush.fill_(1)
+                rs, sts = B.sailor_plan(ctx, space, obs, K_TOP)
+                km.append(sts.kernel_ms)
+            aux[args.workload + "_f32_screen"] = {
+                "kernel_ms": statistics.median(km), "candidates_per_s": n / (statistics.median(km) / 1e3),
+                "same_results": [(r.flat, r.score) for r in rs] == [(int(f), sc) for sc, f in top] if not split else None}
         line = {"metric": METRIC, "value": total / dev_s, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": 1e3 * dev_s / args.steps, "higher_is_better": True,
                 "scaling": "strong" if split else "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-                "config": {"workload": w.name, "candidates": n, "top_k": K_TOP, "mode": "every candidate evaluated",
+                "config": {"workload": w.name, "candidates": n, "top_k": K_TOP,
+                           "mode": "every candidate evaluated" + (" (binary32 screen, binary64 re-score)" if args.f32_screen else ""),
                            "objective": w.objective, "l2": "flushed between timed iterations (256 MiB write)",
                            "parallelism": ("1 gpu" if world == 1 else
                                            f"one space split into {world} flat-index ranges of equal estimated cost, "
@@ -661,6 +724,7 @@ def main() -> None:
     ap.add_argument("--dp-workspace-gib", type=float, default=8.0, help="table workspace of --dp-only")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-aux", action="store_true")
+    ap.add_argument("--f32-screen", action="store_true", help="time the search with the binary32 screen on (for profiling)")
     ap.add_argument("--replicas", action="store_true", help="N > 1: every rank searches the whole space (weak scaling)")
     ap.add_argument("--write-counters", default=None, metavar="NCU_CSV", help="write the counter file from an ncu --csv log")
     args = ap.parse_args()
