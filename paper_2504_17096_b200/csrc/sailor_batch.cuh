@@ -7,7 +7,9 @@
 //     mbs, rc), the gradient bytes in a table per (stage make-up, tp), both formed once per context with the same functions and operation order as a stage-by-stage walk;
 //   - the doubled one-way message time of every link (inside a node, between nodes, between zones) is tabulated
 //     per microbatch size, so a stage boundary is one or two loads and at most one maximum;
-//   - index arithmetic is 32 bits wide and the per-digit GPU counters are 16-bit saturating.
+//   - index arithmetic is 32 bits wide, and the GPUs a plan takes of a (zone, type) are added up over its runs only
+//     when a run repeats an earlier run's (zone, type): no per-thread counters, so little shared memory and a large L1
+//     for the table entries.
 // The sums whose order of additions is part of the result (stage times, price rate, transfer cost) are still
 // added one stage after the other, exactly as simulate_runs does, so both give the same bits.
 #pragma once
@@ -92,21 +94,17 @@ constexpr int BATCH_THREADS = 256;
 constexpr uint32_t BATCH_POOL = 512;             // records a block stages and orders at a time
 constexpr uint32_t REC_WORDS = sizeof(sailor_plan_rec) / 8;
 
-__host__ __device__ inline size_t batch_smem_bytes(uint32_t R) {
-    return sizeof(uint16_t) * (size_t)R * BATCH_THREADS;      // per-thread 16-bit GPU counters, [digit][thread]
-}
-
 struct BatchOut {
     double t_iter, cost;
     uint64_t peak;
     uint32_t status;
 };
 
-// One record, held as nine 64-bit words at `w` (shared memory).  `cnt` = this thread's counters (digit d at
-// cnt[d * BATCH_THREADS]).  Follows simulate_runs operation by operation where roundings are concerned.
+// One record, held as nine 64-bit words at `w` (shared memory).  Follows simulate_runs operation by operation
+// where roundings are concerned.
 __device__ __forceinline__ BatchOut simulate_batch_record(const BatchConst& k, const TabView& v, const PieceRec* __restrict__ piece,
                                                           const double* __restrict__ intra2, const double* __restrict__ inter2,
-                                                          const double* __restrict__ zone2, const uint64_t* w, uint16_t* cnt) {
+                                                          const double* __restrict__ zone2, const uint64_t* w) {
     BatchOut o;
     o.t_iter = o.cost = make_nan();
     o.peak = 0;
@@ -130,13 +128,15 @@ __device__ __forceinline__ BatchOut simulate_batch_record(const BatchConst& k, c
         if (ok) {
             const uint32_t tp = k.tp_values[tpi], d = z * k.T + g;
             if (tp > k.gpn[g] || !((k.heads_ok >> tpi) & 1u)) status |= SAILOR_ST_INVALID;
-            const uint64_t have = ((seen >> d) & 1ull) ? cnt[d * BATCH_THREADS] : 0u;
-            const uint64_t sum = have + (uint64_t)D * tp * n;
+            uint64_t sum = (uint64_t)D * tp * n;            // GPUs this run takes of its (zone, type) ...
+            if ((seen >> d) & 1ull)                          // ... and, rarely, what earlier runs took of the same
+                for (uint32_t q2 = 0; q2 < q; ++q2) {
+                    const uint32_t r2 = run_of_q(q2);
+                    const uint32_t t2 = (r2 >> 16) & 0xff;
+                    if ((r2 & 0xffff) == (r & 0xffff) && t2 < k.n_tp) sum += (uint64_t)D * k.tp_values[t2] * (r2 >> 24);
+                }
             seen |= 1ull << d;
-            // availability is 16 bits wide: a count beyond that is over whatever is available, and stays so
-            const uint32_t kept = sum > 0xffffull ? 0xffffu : (uint32_t)sum;
-            cnt[d * BATCH_THREADS] = (uint16_t)kept;
-            if (sum > k.avail[d]) status |= SAILOR_ST_OVER_AVAIL;
+            if (sum > k.avail[d]) status |= SAILOR_ST_OVER_AVAIL;     // the total only grows from run to run
         }
     }
     if (bad || tot != P) return o;
@@ -252,7 +252,6 @@ __global__ void __launch_bounds__(BATCH_THREADS, 3)
 simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
                 const sailor_plan_rec* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
                 uint64_t* __restrict__ peak_mem, double* __restrict__ cost, uint32_t* __restrict__ status) {
-    extern __shared__ __align__(16) unsigned char dyn[];      // the counters
     __shared__ BatchConst k;
     __shared__ uint64_t recs[BATCH_POOL * REC_WORDS];
     __shared__ uint32_t hist[128];
@@ -284,7 +283,6 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
     const double* inter2 = reinterpret_cast<const double*>(blob + h->off_lnk_inter2);
     const double* zone2 = reinterpret_cast<const double*>(blob + h->off_lnk_zone2);
     const uint64_t* src = reinterpret_cast<const uint64_t*>(plans);
-    uint16_t* counters = reinterpret_cast<uint16_t*>(dyn) + tid;                     // [digit][thread]
     for (uint64_t pool = (uint64_t)blockIdx.x * BATCH_POOL; pool < n; pool += (uint64_t)gridDim.x * BATCH_POOL) {
         const uint32_t cnt = (uint32_t)(n - pool < BATCH_POOL ? n - pool : BATCH_POOL);
         __syncthreads();
@@ -337,7 +335,7 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
             const uint32_t slot = grp * 32 + lane;
             if (slot < cnt) {
                 const uint32_t mine = perm[slot];
-                const BatchOut o = simulate_batch_record(k, v, piece, intra2, inter2, zone2, &recs[mine * REC_WORDS], counters);
+                const BatchOut o = simulate_batch_record(k, v, piece, intra2, inter2, zone2, &recs[mine * REC_WORDS]);
                 if (t_iter) __stcs(&t_iter[pool + mine], o.t_iter);
                 if (peak_mem) __stcs(&peak_mem[pool + mine], o.peak);
                 if (cost) __stcs(&cost[pool + mine], o.cost);

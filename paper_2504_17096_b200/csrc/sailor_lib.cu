@@ -845,7 +845,6 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     }
     CUF(cudaStreamSynchronize(ctx->stream));           // `blob` is pageable host memory
     // both kernels stage the static tables in dynamic shared memory; the create-time limit is 96 KB
-    CUF(cudaFuncSetAttribute(simulate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)batch_smem_bytes(R_MAX)));
     CUF(cudaFuncSetAttribute(simulate_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
     CUF(cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 8) * 1024));
     CUF(cudaFuncSetAttribute(plan_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 16) * 1024));
@@ -937,7 +936,7 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
     const uint64_t tiles = (n + BATCH_POOL - 1) / BATCH_POOL;
     const uint64_t cap = (uint64_t)ctx->sm_count * 12;         // three resident blocks per SM, four pools each at least
     const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
-    simulate_kernel<<<grid, BATCH_THREADS, batch_smem_bytes(ctx->hdr.R), ctx->stream>>>(
+    simulate_kernel<<<grid, BATCH_THREADS, 0, ctx->stream>>>(
         ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s);
     CU(ctx, cudaGetLastError());
     if (!on_device) {
