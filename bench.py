@@ -349,17 +349,17 @@ def explicit_batches(B, torch, dev) -> dict:
             out[key] = {"plans": n, "mean_stages": mean_p, "kernel_ms": ms, "plans_per_s": n / ms * 1e3,
                         "hbm_gb_per_s": n * 100 / ms / 1e6}
             del d_plans, t, c, m, st
-        # plans whose stages mix GPU types among their replicas: 648 B in + 28 B out per plan
-        base = B.pack_mixed_plans(W.random_mixed_plans(w, 1 << 14, seed=13))
+        # plans whose stages mix GPU types among their replicas, up to 32 stages each: 648 B in + 28 B out per plan
+        base = B.pack_mixed_plans(W.random_mixed_plans(w, 1 << 14, seed=13), stages=32)
         reps = 64
         n = base.size * reps                                           # 1.05e6 plans, 680 MB: larger than L2
-        d_plans = torch.from_numpy(base.view(np.uint8).reshape(-1, 648).copy()).cuda().repeat(reps, 1).contiguous()
+        d_plans = torch.from_numpy(base.view(np.uint8).reshape(-1, base.itemsize).copy()).cuda().repeat(reps, 1).contiguous()
         t = torch.empty(n, dtype=torch.float64, device="cuda")
         c = torch.empty(n, dtype=torch.float64, device="cuda")
         m = torch.empty(n, dtype=torch.int64, device="cuda")
         st = torch.empty(n, dtype=torch.int32, device="cuda")
         call = lambda: B.sailor_simulate_mixed_device(ctx, d_plans.data_ptr(), n, t.data_ptr(), m.data_ptr(),
-                                                      c.data_ptr(), st.data_ptr())
+                                                      c.data_ptr(), st.data_ptr(), record_bytes=base.itemsize)
         for _ in range(3):
             call()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -370,7 +370,8 @@ def explicit_batches(B, torch, dev) -> dict:
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / 5
         out["simulate_mixed_cfg5"] = {"plans": n, "mean_stages": float(base["P"].astype(np.float64).mean()),
-                                      "kernel_ms": ms, "plans_per_s": n / ms * 1e3, "hbm_gb_per_s": n * 676 / ms / 1e6}
+                                      "kernel_ms": ms, "plans_per_s": n / ms * 1e3,
+                                      "hbm_gb_per_s": n * (base.itemsize + 28) / ms / 1e6}
         del d_plans, t, c, m, st
     finally:
         B.sailor_destroy(ctx)

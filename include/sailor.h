@@ -355,7 +355,7 @@ int sailor_plan_noalloc(sailor_ctx* ctx, const sailor_space* s, const sailor_obj
  *   - memory is checked per group; the update time is the largest over stages and groups; the price
  *     rate adds (double)(count*tp) * price per second group after group, stage after stage.
  * A plan with one group in every stage gives bit-identical results to sailor_simulate. */
-#define SAILOR_MIX_P_MAX       32
+#define SAILOR_MIX_P_MAX       96    /* the deepest pipeline of the plain simulator's workloads */
 #define SAILOR_MIX_GROUPS_MAX  4
 
 typedef struct sailor_replica_group {
@@ -369,7 +369,7 @@ typedef struct sailor_mixed_stage {
     sailor_replica_group group[SAILOR_MIX_GROUPS_MAX];
 } sailor_mixed_stage;
 
-typedef struct sailor_mixed_plan {      /* 648 bytes; arrays must be 8-byte aligned                  */
+typedef struct sailor_mixed_plan {      /* 1928 bytes (only the first P stages are read); 8-byte aligned */
     uint8_t  P;                         /* 1 .. SAILOR_MIX_P_MAX                                      */
     uint8_t  mbs_idx, rc, _pad;
     uint16_t D;                         /* >= 1                                                       */
@@ -382,6 +382,14 @@ typedef struct sailor_mixed_plan {      /* 648 bytes; arrays must be 8-byte alig
  * SAILOR_ST_BAD_RECORD an index outside its table or n_groups / P outside their limits. */
 int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint64_t n, int on_device,
                           double* t_iter, uint64_t* peak_mem, double* cost, uint32_t* status);
+
+/* The same for records cut short, so that a batch of shallow plans need not carry SAILOR_MIX_P_MAX stages each:
+ * record j starts at (const char*)plans + j * record_bytes and holds the 8-byte head of a sailor_mixed_plan and its
+ * first (record_bytes - 8) / sizeof(sailor_mixed_stage) stages.  record_bytes is a multiple of 8 from 32 to
+ * sizeof(sailor_mixed_plan), else SAILOR_E_ARG.  A plan with more stages than its record holds is refused
+ * (host records: SAILOR_E_RANGE; device records: SAILOR_ST_BAD_RECORD and NaN for that plan). */
+int sailor_simulate_mixed_strided(sailor_ctx* ctx, const void* plans, uint64_t n, uint32_t record_bytes, int on_device,
+                                  double* t_iter, uint64_t* peak_mem, double* cost, uint32_t* status);
 
 /* ---- searching over such plans (Sec. 4.2.2 "Implementation": per stage, the planner generates the resource
  * combinations of different GPU types that give the stage its D replicas) ---------------------------------

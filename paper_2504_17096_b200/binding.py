@@ -22,7 +22,7 @@ DP_FLAG_BUDGET_LOOP, DP_BUDGET_P_MAX = 0x1000, 32
 
 EXPORTS = ("sailor_create", "sailor_destroy", "sailor_set_availability", "sailor_simulate",
            "sailor_space_size", "sailor_decode", "sailor_plan", "sailor_plan_range", "sailor_plan_noalloc",
-           "sailor_plan_dp", "sailor_simulate_mixed", "sailor_mixed_space_size", "sailor_mixed_decode",
+           "sailor_plan_dp", "sailor_simulate_mixed", "sailor_simulate_mixed_strided", "sailor_mixed_space_size", "sailor_mixed_decode",
            "sailor_plan_mixed", "sailor_measure_issue_rates", "sailor_strerror",
            "sailor_last_cuda_error")
 
@@ -119,21 +119,34 @@ REC_DTYPE = np.dtype([("P", "u1"), ("mbs_idx", "u1"), ("rc", "u1"), ("n_runs", "
 assert REC_DTYPE.itemsize == 72
 
 
-MIX_P_MAX, MIX_GROUPS_MAX = 32, 4
+MIX_P_MAX, MIX_GROUPS_MAX = 96, 4
 MIX_GROUP_DTYPE = np.dtype([("type", "u1"), ("tp_idx", "u1"), ("count", "<u2")])
 MIX_STAGE_DTYPE = np.dtype([("zone", "u1"), ("n_groups", "u1"), ("_pad", "<u2"), ("group", MIX_GROUP_DTYPE, (MIX_GROUPS_MAX,))])
-MIX_DTYPE = np.dtype([("P", "u1"), ("mbs_idx", "u1"), ("rc", "u1"), ("_pad", "u1"), ("D", "<u2"), ("_pad2", "<u2"),
-                      ("stage", MIX_STAGE_DTYPE, (MIX_P_MAX,))])
-assert MIX_DTYPE.itemsize == 648
 
 
-def pack_mixed_plans(plans) -> np.ndarray:
+def mixed_dtype(stages: int) -> np.dtype:
+    """Record of a plan with mixed replicas that has room for `stages` stages (an even number up to MIX_P_MAX, so that
+    the record is a multiple of 8 bytes): the head of sailor_mixed_plan and its first stages."""
+    if stages < 2 or stages > MIX_P_MAX or stages % 2:
+        raise ValueError("stages per record: an even number from 2 to %d" % MIX_P_MAX)
+    return np.dtype([("P", "u1"), ("mbs_idx", "u1"), ("rc", "u1"), ("_pad", "u1"), ("D", "<u2"), ("_pad2", "<u2"),
+                     ("stage", MIX_STAGE_DTYPE, (stages,))])
+
+
+MIX_DTYPE = mixed_dtype(MIX_P_MAX)
+assert MIX_DTYPE.itemsize == 1928 and mixed_dtype(32).itemsize == 648
+
+
+def pack_mixed_plans(plans, stages: int = 0) -> np.ndarray:
     """List of dicts {"P", "mbs_idx", "rc", "D", "stages": [{"zone", "groups": [(type, tp_idx, count), ...]}]}
-    -> array of 648-byte records."""
-    out = np.zeros(len(plans), dtype=MIX_DTYPE)
+    -> array of records with room for `stages` stages each (0: the deepest plan of the list, rounded up to even)."""
+    deepest = max([p["P"] for p in plans], default=1)
+    if deepest > MIX_P_MAX:
+        raise ValueError("at most %d stages" % MIX_P_MAX)
+    out = np.zeros(len(plans), dtype=mixed_dtype(stages or max(2, deepest + deepest % 2)))
     for j, p in enumerate(plans):
-        if p["P"] > MIX_P_MAX:
-            raise ValueError("at most %d stages" % MIX_P_MAX)
+        if p["P"] > out.dtype["stage"].shape[0]:
+            raise ValueError("a plan of %d stages in records of %d" % (p["P"], out.dtype["stage"].shape[0]))
         out["P"][j], out["mbs_idx"][j], out["rc"][j], out["D"][j] = p["P"], p["mbs_idx"], p["rc"], p["D"]
         for i, st in enumerate(p["stages"]):
             if len(st["groups"]) > MIX_GROUPS_MAX:
@@ -178,7 +191,7 @@ class MixedResult(C.Structure):
                 ("score", C.c_double), ("status", C.c_uint32), ("_pad", C.c_uint32), ("plan", MixedPlan)]
 
 
-assert C.sizeof(MixedPlan) == 648 and C.sizeof(MixedResult) == 696 and C.sizeof(MixedSpace) == 152
+assert C.sizeof(MixedPlan) == 1928 and C.sizeof(MixedResult) == 1976 and C.sizeof(MixedSpace) == 152
 
 
 class SailorError(RuntimeError):
@@ -208,6 +221,7 @@ def load() -> C.CDLL:
     L.sailor_set_availability.argtypes = [vp, _u16p]
     L.sailor_simulate.argtypes = [vp, vp, C.c_uint64, C.c_int, vp, vp, vp, vp]
     L.sailor_simulate_mixed.argtypes = [vp, vp, C.c_uint64, C.c_int, vp, vp, vp, vp]
+    L.sailor_simulate_mixed_strided.argtypes = [vp, vp, C.c_uint64, C.c_uint32, C.c_int, vp, vp, vp, vp]
     L.sailor_space_size.argtypes = [vp, C.POINTER(Space), _u64p]
     L.sailor_decode.argtypes = [vp, C.POINTER(Space), C.c_uint64, C.POINTER(PlanRec)]
     L.sailor_plan.argtypes = [vp, C.POINTER(Space), C.POINTER(Objective), C.c_uint32, C.POINTER(Result), _u32p,
@@ -341,21 +355,30 @@ def sailor_simulate_device(ctx, plans_ptr: int, n: int, t_iter_ptr: int, peak_me
 
 
 def sailor_simulate_mixed(ctx, plans: np.ndarray):
-    """Plans with mixed replicas (MIX_DTYPE array, see pack_mixed_plans) in, (t_iter, peak_mem, cost, status) out."""
-    plans = np.ascontiguousarray(plans, dtype=MIX_DTYPE)
+    """Plans with mixed replicas (an array of a mixed_dtype, see pack_mixed_plans) in, (t_iter, peak_mem, cost, status)
+    out.  Records shorter than sailor_mixed_plan go through sailor_simulate_mixed_strided."""
+    plans = np.ascontiguousarray(plans)
+    if "stage" not in (plans.dtype.names or ()) or plans.dtype != mixed_dtype(plans.dtype["stage"].shape[0]):
+        raise TypeError("an array made by pack_mixed_plans is wanted")
     n = plans.size
     t, c = np.empty(n, np.float64), np.empty(n, np.float64)
     m, s = np.empty(n, np.uint64), np.empty(n, np.uint32)
-    _check(load().sailor_simulate_mixed(ctx, plans.ctypes.data, n, 0, t.ctypes.data, m.ctypes.data, c.ctypes.data,
-                                        s.ctypes.data), "sailor_simulate_mixed", ctx)
+    if plans.dtype.itemsize == C.sizeof(MixedPlan):
+        rc = load().sailor_simulate_mixed(ctx, plans.ctypes.data, n, 0, t.ctypes.data, m.ctypes.data, c.ctypes.data, s.ctypes.data)
+    else:
+        rc = load().sailor_simulate_mixed_strided(ctx, plans.ctypes.data, n, plans.dtype.itemsize, 0, t.ctypes.data,
+                                                  m.ctypes.data, c.ctypes.data, s.ctypes.data)
+    _check(rc, "sailor_simulate_mixed", ctx)
     return t, m, c, s
 
 
 def sailor_simulate_mixed_device(ctx, plans_ptr: int, n: int, t_iter_ptr: int, peak_mem_ptr: int, cost_ptr: int,
-                                 status_ptr: int) -> None:
-    """Device path of sailor_simulate_mixed: raw device pointers; only enqueues work."""
-    _check(load().sailor_simulate_mixed(ctx, plans_ptr, n, 1, t_iter_ptr or None, peak_mem_ptr or None, cost_ptr or None,
-                                        status_ptr or None), "sailor_simulate_mixed", ctx)
+                                 status_ptr: int, record_bytes: int = 0) -> None:
+    """Device path of sailor_simulate_mixed (record_bytes 0: whole sailor_mixed_plan records) and of
+    sailor_simulate_mixed_strided: raw device pointers; only enqueues work."""
+    _check(load().sailor_simulate_mixed_strided(ctx, plans_ptr, n, record_bytes or C.sizeof(MixedPlan), 1, t_iter_ptr or None,
+                                                peak_mem_ptr or None, cost_ptr or None, status_ptr or None),
+           "sailor_simulate_mixed", ctx)
 
 
 def sailor_space_size(ctx, space: Space) -> int:

@@ -99,15 +99,20 @@ __global__ void compose_kernel(unsigned char* blob) {
     }
 }
 
-// One warp per plan with mixed replicas (648-byte records, read in place, lane i reading stage i).  Tables in
-// shared memory, then R 64-bit GPU counters per warp.
-__global__ void __launch_bounds__(SIM_THREADS, 4)
+// One warp per plan with mixed replicas (records `stride` bytes apart holding `max_stages` stages, read in place,
+// lane i reading stage i).  Tables in shared memory, then R 64-bit GPU counters per warp.  Plans of up to 32 stages
+// are evaluated by the DEEP = false launch, which leaves deeper ones alone and notes in `deep_seen` that there are
+// some; the DEEP = true launch that follows returns at once when there are none and evaluates only those otherwise
+// (a lane then owns up to three stages; the state of that evaluation does not fit the registers of the first).
+template <bool DEEP>
+__global__ void __launch_bounds__(SIM_THREADS, DEEP ? 2 : 4)
 simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
-                      const sailor_mixed_plan* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
-                      uint64_t* __restrict__ peak_mem, double* __restrict__ cost, uint32_t* __restrict__ status,
-                      unsigned int* error) {
+                      const unsigned char* __restrict__ plans, uint32_t stride, uint32_t max_stages, uint64_t n,
+                      double* __restrict__ t_iter, uint64_t* __restrict__ peak_mem, double* __restrict__ cost,
+                      uint32_t* __restrict__ status, unsigned int* error, unsigned int* deep_seen) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ uint64_t mbar;
+    if (DEEP && *reinterpret_cast<volatile unsigned int*>(deep_seen) == 0) return;
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     constexpr uint32_t WARPS = SIM_THREADS / 32;
     const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(blob)->static_bytes;
@@ -121,7 +126,22 @@ simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __
     v.bind(dyn, blob);
     unsigned long long* counters = reinterpret_cast<unsigned long long*>(dyn + static_bytes) + (size_t)warp * v.h->R;
     for (uint64_t j = (uint64_t)blockIdx.x * WARPS + warp; j < n; j += (uint64_t)gridDim.x * WARPS) {
-        const SimOut o = simulate_mixed_warp(v, avail, plans[j], counters, lane);
+        const sailor_mixed_plan& r = *reinterpret_cast<const sailor_mixed_plan*>(plans + j * stride);
+        const uint32_t P = r.P;
+        SimOut o;
+        if (DEEP) {
+            if (P <= 32 || P > max_stages) continue;             // done by the first launch
+            o = simulate_mixed_tiles<SAILOR_MIX_P_MAX / 32>(v, avail, r, counters, lane);
+        } else if (P > max_stages) {                             // more stages than the record has room for
+            o.t_iter = o.cost = make_nan();
+            o.peak_mem = 0;
+            o.status = SAILOR_ST_BAD_RECORD;
+        } else if (P > 32) {
+            if (lane == 0) *reinterpret_cast<volatile unsigned int*>(deep_seen) = 1u;
+            continue;
+        } else {
+            o = simulate_mixed_warp(v, avail, r, counters, lane);
+        }
         if (lane == 0) {
             if (t_iter) t_iter[j] = o.t_iter;
             if (peak_mem) peak_mem[j] = o.peak_mem;
@@ -179,7 +199,7 @@ struct sailor_ctx {
     bool avail_dirty = false;              // d_avail is older than h_avail
     PlanOut* d_out_mapped = nullptr;       // device address of h_out (mapped pinned memory)
     Ctrl* d_ctrl = nullptr;
-    unsigned int* d_sim_error = nullptr;   // error word of the explicit-batch kernels
+    unsigned int* d_sim_error = nullptr;   // error word of the explicit-batch kernels, then the "deep plans seen" word
     PlanOut* h_out = nullptr;              // pinned
     bool ctrl_dirty = true;                // the counters must be cleared from the host (first call, or after a failed one)
     uint64_t sync_epoch = 1;               // stream synchronisations by this context so far
@@ -817,7 +837,7 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     CUF(cudaMallocHost(&ctx->h_avail, R_MAX * sizeof(uint16_t)));
     memset(ctx->h_avail, 0, R_MAX * sizeof(uint16_t));       // availability starts at zero on both sides
     CUF(cudaMalloc(&ctx->d_ctrl, sizeof(Ctrl)));
-    CUF(cudaMalloc(&ctx->d_sim_error, sizeof(unsigned int)));
+    CUF(cudaMalloc(&ctx->d_sim_error, 2 * sizeof(unsigned int)));
     CUF(cudaHostAlloc(&ctx->h_out, sizeof(PlanOut), cudaHostAllocMapped));
     CUF(cudaHostGetDevicePointer(reinterpret_cast<void**>(&ctx->d_out_mapped), ctx->h_out, 0));
     memset(ctx->h_out, 0, sizeof(PlanOut));
@@ -831,7 +851,7 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     CUF(cudaMemcpyAsync(ctx->d_blob, blob.data(), h.total_bytes, cudaMemcpyHostToDevice, ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_avail, 0, R_MAX * sizeof(uint16_t), ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_ctrl, 0, sizeof(Ctrl), ctx->stream));
-    CUF(cudaMemsetAsync(ctx->d_sim_error, 0, sizeof(unsigned int), ctx->stream));
+    CUF(cudaMemsetAsync(ctx->d_sim_error, 0, 2 * sizeof(unsigned int), ctx->stream));
     {
         const uint32_t n_threads = 4 * T * n_tp * n_mbs + 2 * T * n_tp;
         chain_kernel<<<(n_threads + 127) / 128, 128, 0, ctx->stream>>>(ctx->d_blob);
@@ -845,10 +865,12 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     }
     CUF(cudaStreamSynchronize(ctx->stream));           // `blob` is pageable host memory
     // both kernels stage the static tables in dynamic shared memory; the create-time limit is 96 KB
-    CUF(cudaFuncSetAttribute(simulate_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
+    CUF(cudaFuncSetAttribute(simulate_mixed_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
+    CUF(cudaFuncSetAttribute(simulate_mixed_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 64) * 1024));
     CUF(cudaFuncSetAttribute(finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 8) * 1024));
-    CUF(cudaFuncSetAttribute(plan_mixed_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 16) * 1024));
-    CUF(cudaFuncSetAttribute(mixed_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 16) * 1024));
+    CUF(cudaFuncSetAttribute(plan_mixed_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 24) * 1024));
+    CUF(cudaFuncSetAttribute(plan_mixed_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 24) * 1024));
+    CUF(cudaFuncSetAttribute(mixed_finish_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (96 + 24) * 1024));
 #undef CUF
     *out = ctx;
     return SAILOR_OK;
@@ -951,19 +973,32 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
 
 int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint64_t n, int on_device, double* t_iter,
                           uint64_t* peak_mem, double* cost, uint32_t* status) {
-    if (!ctx || (!plans && n)) return SAILOR_E_ARG;
+    return sailor_simulate_mixed_strided(ctx, plans, n, (uint32_t)sizeof(sailor_mixed_plan), on_device, t_iter, peak_mem,
+                                         cost, status);
+}
+
+int sailor_simulate_mixed_strided(sailor_ctx* ctx, const void* plans_v, uint64_t n, uint32_t record_bytes, int on_device,
+                                  double* t_iter, uint64_t* peak_mem, double* cost, uint32_t* status) {
+    constexpr uint32_t HEAD = (uint32_t)offsetof(sailor_mixed_plan, stage);
+    if (!ctx || (!plans_v && n)) return SAILOR_E_ARG;
+    if (record_bytes % 8 != 0 || record_bytes < HEAD + sizeof(sailor_mixed_stage) || record_bytes > sizeof(sailor_mixed_plan))
+        return SAILOR_E_ARG;
     if (n == 0) return SAILOR_OK;
+    const unsigned char* plans = static_cast<const unsigned char*>(plans_v);
     if ((uintptr_t)plans % 8 != 0) return SAILOR_E_ARG;
+    const uint32_t max_stages = (record_bytes - HEAD) / (uint32_t)sizeof(sailor_mixed_stage);
     DeviceGuard guard(ctx->device);
-    const sailor_mixed_plan* d_plans = plans;
+    const unsigned char* d_plans = plans;
+    bool any_deep = false;
     double *d_t = t_iter, *d_c = cost;
     uint64_t* d_m = peak_mem;
     uint32_t* d_s = status;
     if (!on_device) {
         const TabHdr& h = ctx->hdr;
         for (uint64_t j = 0; j < n; ++j) {
-            const sailor_mixed_plan& r = plans[j];
-            if (r.P < 1 || r.P > SAILOR_MIX_P_MAX || r.D < 1 || r.mbs_idx >= h.n_mbs) return SAILOR_E_RANGE;
+            const sailor_mixed_plan& r = *reinterpret_cast<const sailor_mixed_plan*>(plans + j * record_bytes);
+            if (r.P < 1 || r.P > max_stages || r.D < 1 || r.mbs_idx >= h.n_mbs) return SAILOR_E_RANGE;
+            any_deep = any_deep || r.P > 32;
             for (uint32_t i = 0; i < r.P; ++i) {
                 const sailor_mixed_stage& st = r.stage[i];
                 if (st.zone >= h.Z || st.n_groups < 1 || st.n_groups > SAILOR_MIX_GROUPS_MAX) return SAILOR_E_RANGE;
@@ -971,7 +1006,7 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
                     if (st.group[q].type >= h.T || st.group[q].tp_idx >= h.n_tp) return SAILOR_E_RANGE;
             }
         }
-        const size_t need = n * (sizeof(sailor_mixed_plan) + 32);
+        const size_t need = n * ((size_t)record_bytes + 32);
         if (need > ctx->stage_bytes) {
             CU(ctx, stream_sync(ctx));
             cudaFree(ctx->d_stage);
@@ -986,8 +1021,8 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
         d_c = reinterpret_cast<double*>(base + 8 * n);
         d_m = reinterpret_cast<uint64_t*>(base + 16 * n);
         d_s = reinterpret_cast<uint32_t*>(base + 24 * n);
-        sailor_mixed_plan* dp = reinterpret_cast<sailor_mixed_plan*>(base + 32 * n);
-        CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_mixed_plan), cudaMemcpyHostToDevice, ctx->stream));
+        unsigned char* dp = base + 32 * n;
+        CU(ctx, cudaMemcpyAsync(dp, plans, n * (size_t)record_bytes, cudaMemcpyHostToDevice, ctx->stream));
         d_plans = dp;
     }
     {
@@ -998,8 +1033,16 @@ int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint6
     const uint64_t cap = (uint64_t)ctx->sm_count * 32;
     const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
     const size_t smem = ctx->hdr.static_bytes + sizeof(unsigned long long) * (SIM_THREADS / 32) * ctx->hdr.R;
-    simulate_mixed_kernel<<<grid, SIM_THREADS, smem, ctx->stream>>>(ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s,
-                                                                     ctx->d_sim_error);
+    unsigned int* deep_seen = ctx->d_sim_error + 1;
+    if (max_stages > 32) CU(ctx, cudaMemsetAsync(deep_seen, 0, sizeof(unsigned int), ctx->stream));
+    simulate_mixed_kernel<false><<<grid, SIM_THREADS, smem, ctx->stream>>>(ctx->d_blob, ctx->d_avail, d_plans, record_bytes,
+                                                                            max_stages, n, d_t, d_m, d_c, d_s, ctx->d_sim_error,
+                                                                            deep_seen);
+    if (max_stages > 32 && (on_device || any_deep)) {            // the plans of more than 32 stages, if there are any
+        const uint64_t cap2 = (uint64_t)ctx->sm_count * 16;
+        simulate_mixed_kernel<true><<<(uint32_t)(tiles < cap2 ? tiles : cap2), SIM_THREADS, smem, ctx->stream>>>(
+            ctx->d_blob, ctx->d_avail, d_plans, record_bytes, max_stages, n, d_t, d_m, d_c, d_s, ctx->d_sim_error, deep_seen);
+    }
     CU(ctx, cudaGetLastError());
     if (!on_device) {
         if (t_iter) CU(ctx, cudaMemcpyAsync(t_iter, d_t, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
@@ -2032,7 +2075,10 @@ static int plan_mixed_impl(sailor_ctx* ctx, const sailor_mixed_space* s, const s
     mp.blob = ctx->d_blob; mp.avail = ctx->d_avail; mp.cfg_flat_base = d_base; mp.combs = d_combs; mp.partial = d_partial;
     mp.counters = d_counters; mp.results = d_results; mp.sp = mt.desc; mp.n_config = mt.n_config; mp.k = k; mp.obj = o->kind;
     mp.n_partial = grid; mp.n_total = n_total; mp.budget = o->budget_usd_per_iter; mp.min_rate = o->min_iters_per_s;
-    plan_mixed_kernel<<<grid, MIXS_THREADS, smem, ctx->stream>>>(mp);
+    bool deep = false;                                           // pipelines of more than 32 stages in the space
+    for (uint32_t i = 0; i < s->n_p; ++i) deep = deep || s->p_values[i] > 32;
+    if (deep) plan_mixed_kernel<true><<<grid, MIXS_THREADS, smem, ctx->stream>>>(mp);
+    else plan_mixed_kernel<false><<<grid, MIXS_THREADS, smem, ctx->stream>>>(mp);
     CU(ctx, cudaGetLastError());
     mixed_finish_kernel<<<1, MIXS_THREADS, smem, ctx->stream>>>(mp);
     CU(ctx, cudaGetLastError());

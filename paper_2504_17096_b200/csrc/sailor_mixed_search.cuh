@@ -4,7 +4,7 @@
 // A combination is a tuple of units per GPU type (see sailor.h); the host lists the combinations of every degree
 // of the space once per call (descending lexicographic order) and the device looks them up.  A candidate is
 // (P, mbs, rc, D) and one (zone, combination) per segment; one warp builds the candidate's record in shared memory
-// from its flat index, evaluates it with simulate_mixed_warp (lane = stage) and offers it to its top-k list, which
+// from its flat index, evaluates it with simulate_mixed_plan (a lane per stage) and offers it to its top-k list, which
 // here is a warp-uniform insertion.  Blocks leave their lists for mixed_finish_kernel, which merges them and writes
 // the winners out with their records.
 #pragma once
@@ -15,7 +15,7 @@
 namespace sailor {
 
 constexpr uint32_t MIX_UNITS_MAX = 16;
-static_assert(SAILOR_MIX_P_MAX == 32, "one lane per stage, and every lane writes one stage of the record");
+static_assert(SAILOR_MIX_P_MAX % 32 == 0, "every lane writes SAILOR_MIX_P_MAX / 32 stages of the record");
 
 struct MixedSpaceDesc {
     uint32_t n_p, n_mbs, n_rc, n_d, seg_max, granularity;
@@ -107,14 +107,18 @@ __device__ __forceinline__ void mixed_candidate(const MixedSearchParams& mp, uin
         plan->P = (uint8_t)k.P; plan->mbs_idx = (uint8_t)k.mi; plan->rc = (uint8_t)k.rc; plan->_pad = 0;
         plan->D = (uint16_t)k.D; plan->_pad2 = 0;
     }
-    if (lane < k.P) mixed_build_stage(mp.sp, k, T, mp.combs, digit, lane, &plan->stage[lane]);
-    else {                                                     // stages past the last are all zero, as the host decoder leaves them
-        uint32_t* z = reinterpret_cast<uint32_t*>(&plan->stage[lane]);
-        for (uint32_t x = 0; x < sizeof(sailor_mixed_stage) / 4; ++x) z[x] = 0;
+    for (uint32_t i = lane; i < SAILOR_MIX_P_MAX; i += 32) {
+        if (i < k.P) mixed_build_stage(mp.sp, k, T, mp.combs, digit, i, &plan->stage[i]);
+        else {                                                 // stages past the last are all zero, as the host decoder leaves them
+            uint32_t* z = reinterpret_cast<uint32_t*>(&plan->stage[i]);
+            for (uint32_t x = 0; x < sizeof(sailor_mixed_stage) / 4; ++x) z[x] = 0;
+        }
     }
     __syncwarp();
 }
 
+// DEEP: the space has pipelines of more than 32 stages (the evaluation then goes through the tiled variant).
+template <bool DEEP>
 __global__ void __launch_bounds__(MIXS_THREADS, 2) plan_mixed_kernel(const __grid_constant__ MixedSearchParams mp) {
     extern __shared__ __align__(16) unsigned char dyn[];      // static tables, then per-warp counters, then per-warp records
     __shared__ uint64_t mbar;
@@ -139,7 +143,7 @@ __global__ void __launch_bounds__(MIXS_THREADS, 2) plan_mixed_kernel(const __gri
     const uint64_t stride = (uint64_t)gridDim.x * MIXS_WARPS;
     for (uint64_t flat = (uint64_t)blockIdx.x * MIXS_WARPS + warp; flat < mp.n_total; flat += stride) {
         mixed_candidate(mp, T, Z, flat, plan, lane);
-        const SimOut o = simulate_mixed_warp(v, mp.avail, *plan, cnt, lane);
+        const SimOut o = DEEP ? simulate_mixed_plan(v, mp.avail, *plan, cnt, lane) : simulate_mixed_warp(v, mp.avail, *plan, cnt, lane);
         __syncwarp();                                          // the record and the counters are reused by the next candidate
         // every candidate falls in exactly one class: invalid, out of memory, over availability, over the constraint, feasible
         n_class[0]++;
@@ -218,14 +222,14 @@ __global__ void __launch_bounds__(MIXS_THREADS) mixed_finish_kernel(const __grid
     for (uint32_t j = warp; j < s_n; j += MIXS_WARPS) {
         const uint64_t flat = s_hits[0][j].flat;
         mixed_candidate(mp, T, Z, flat, plan, lane);
-        const SimOut o = simulate_mixed_warp(v, mp.avail, *plan, cnt, lane);
+        const SimOut o = simulate_mixed_plan(v, mp.avail, *plan, cnt, lane);
         __syncwarp();
         sailor_mixed_result* r = mp.results + j;
         if (lane == 0) {
             r->flat = flat; r->t_iter = o.t_iter; r->cost = o.cost; r->peak_mem = o.peak_mem;
             r->score = s_hits[0][j].score; r->status = o.status; r->_pad = 0;
         }
-        // the record, word by word (648 bytes = 81 words of 8)
+        // the record, word by word
         const uint64_t* src = reinterpret_cast<const uint64_t*>(plan);
         uint64_t* dst = reinterpret_cast<uint64_t*>(&r->plan);
         for (uint32_t x = lane; x < sizeof(sailor_mixed_plan) / 8; x += 32) dst[x] = src[x];

@@ -83,6 +83,51 @@ def test_mixed_tiny_with_latency_polynomials_and_recomputation():
         assert_equal(gpu, Oracle(w).simulate_mixed_batch(plans), w.name)
 
 
+@pytest.mark.parametrize("cfg", [0, 5])
+def test_deep_mixed_plans_match_oracle(cfg):
+    """Plans of up to 96 stages (a lane owns up to three stages): the full records and records cut to the deepest plan."""
+    w = W.CONFIGS[cfg]() if cfg else W.tiny(seed=23, n_types=8, n_zones=8, L=96, p_values=[96, 65, 64, 33, 32, 5],
+                                            d_values=(1, 2, 5, 64), gbs=640)
+    plans = W.random_mixed_plans(w, 4001, seed=500 + cfg, p_max=96)
+    depths = [p["P"] for p in plans]
+    assert max(depths) > 64 and sum(1 for d in depths if 32 < d <= 64) > 0 and min(depths) <= 32
+    orc = Oracle(w).simulate_mixed_batch(plans)
+    with Ctx(w) as cx:
+        assert_equal(B.sailor_simulate_mixed(cx.ctx, B.pack_mixed_plans(plans, stages=B.MIX_P_MAX)), orc, f"cfg{cfg} full records")
+        assert_equal(B.sailor_simulate_mixed(cx.ctx, B.pack_mixed_plans(plans)), orc, f"cfg{cfg} cut records")
+        # the boundaries of the lane tiles, one plan each
+        edge = [p for p in plans if p["P"] in (31, 32, 33, 63, 64, 65, 95, 96)]
+        if edge:
+            assert_equal(B.sailor_simulate_mixed(cx.ctx, B.pack_mixed_plans(edge)), Oracle(w).simulate_mixed_batch(edge), "tile edges")
+
+
+def test_mixed_record_sizes():
+    """sailor_simulate_mixed_strided: record sizes it takes, and a plan deeper than its record."""
+    import torch
+    w = W.config1()
+    plans = [p for p in W.random_mixed_plans(w, 800, seed=9) if p["P"] <= 8]
+    orc = Oracle(w).simulate_mixed_batch(plans)
+    with Ctx(w) as cx:
+        for stages in (8, 10, 32, 96):
+            assert_equal(B.sailor_simulate_mixed(cx.ctx, B.pack_mixed_plans(plans, stages=stages)), orc, f"{stages} stages per record")
+        L = B.load()
+        packed = B.pack_mixed_plans(plans, stages=8)
+        out = np.empty(len(plans)); st = np.empty(len(plans), np.uint32)
+        for bad_bytes in (0, 24, 28, 36, 1936):
+            assert L.sailor_simulate_mixed_strided(cx.ctx, packed.ctypes.data, len(plans), bad_bytes, 0, out.ctypes.data, None, None,
+                                                   st.ctypes.data) == B.E_ARG
+        deep = packed[:3].copy()
+        deep["P"][1] = 9                                 # more stages than the record holds
+        with pytest.raises(B.SailorError) as e:
+            B.sailor_simulate_mixed(cx.ctx, deep)
+        assert e.value.code == B.E_RANGE
+        d = torch.from_numpy(deep.view(np.uint8).reshape(3, deep.itemsize).copy()).cuda()
+        ds = torch.zeros(3, dtype=torch.int32, device="cuda"); dt = torch.zeros(3, dtype=torch.float64, device="cuda")
+        B.sailor_simulate_mixed_device(cx.ctx, d.data_ptr(), 3, dt.data_ptr(), 0, 0, ds.data_ptr(), record_bytes=deep.itemsize)
+        torch.cuda.synchronize()
+        assert ds.cpu().tolist()[1] == B.ST_BAD_RECORD and ds.cpu().tolist()[0] == int(orc[0][0]) and math.isnan(dt.cpu().tolist()[1])
+
+
 def test_mixed_with_one_group_equals_sailor_simulate():
     """No mixing: the same numbers as the run-length records of sailor_simulate."""
     w = W.config2()
@@ -116,10 +161,11 @@ def test_mixed_device_pointers_empty_and_bad_records():
         t, m, c, s = B.sailor_simulate_mixed(cx.ctx, np.zeros(0, dtype=B.MIX_DTYPE))
         assert t.size == 0
         n = packed.size
-        d = torch.from_numpy(packed.view(np.uint8).reshape(n, 648).copy()).cuda()
+        d = torch.from_numpy(packed.view(np.uint8).reshape(n, packed.itemsize).copy()).cuda()
         dt = torch.empty(n, dtype=torch.float64, device="cuda"); dc = torch.empty(n, dtype=torch.float64, device="cuda")
         dm = torch.empty(n, dtype=torch.int64, device="cuda"); ds = torch.empty(n, dtype=torch.int32, device="cuda")
-        B.sailor_simulate_mixed_device(cx.ctx, d.data_ptr(), n, dt.data_ptr(), dm.data_ptr(), dc.data_ptr(), ds.data_ptr())
+        B.sailor_simulate_mixed_device(cx.ctx, d.data_ptr(), n, dt.data_ptr(), dm.data_ptr(), dc.data_ptr(), ds.data_ptr(),
+                                       record_bytes=packed.itemsize)
         torch.cuda.synchronize()
         gpu = (dt.cpu().numpy(), dm.cpu().numpy().view(np.uint64), dc.cpu().numpy(), ds.cpu().numpy().view(np.uint32))
         assert_equal(gpu, Oracle(w).simulate_mixed_batch(plans), "device pointers")
@@ -129,9 +175,9 @@ def test_mixed_device_pointers_empty_and_bad_records():
         with pytest.raises(B.SailorError) as e:
             B.sailor_simulate_mixed(cx.ctx, bad)
         assert e.value.code == B.E_RANGE
-        d2 = torch.from_numpy(bad.view(np.uint8).reshape(2, 648).copy()).cuda()
+        d2 = torch.from_numpy(bad.view(np.uint8).reshape(2, bad.itemsize).copy()).cuda()
         st = torch.zeros(2, dtype=torch.int32, device="cuda"); tt = torch.zeros(2, dtype=torch.float64, device="cuda")
-        B.sailor_simulate_mixed_device(cx.ctx, d2.data_ptr(), 2, tt.data_ptr(), 0, 0, st.data_ptr())
+        B.sailor_simulate_mixed_device(cx.ctx, d2.data_ptr(), 2, tt.data_ptr(), 0, 0, st.data_ptr(), record_bytes=bad.itemsize)
         torch.cuda.synchronize()
         assert st.cpu().tolist()[1] == B.ST_BAD_RECORD and not (st.cpu().tolist()[0] & B.ST_BAD_RECORD)
         assert math.isnan(tt.cpu().tolist()[1])

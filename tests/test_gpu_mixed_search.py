@@ -53,6 +53,10 @@ def _cases():
     yield W.tiny(seed=5, n_types=3, n_zones=1, L=6, p_values=[2, 3], d_values=(4, 6), seg_max=3, gbs=48), 4, [1, 0, 0]
     yield W.tiny(seed=6, n_types=3, n_zones=2, L=4, p_values=[2, 4], d_values=(2, 4), seg_max=2), 4, [0, 0, 1]
     yield W.tiny(seed=11, n_types=4, n_zones=2, L=8, p_values=[3, 8], d_values=(3, 8), seg_max=2, gbs=48), 4, [0, 1, 0, 1]
+    deep = W.tiny(seed=13, n_types=3, n_zones=2, L=80, p_values=[5, 40, 80], d_values=(2, 4), seg_max=2, gbs=64)
+    deep.avail = deep.avail * 30                      # room for pipelines of 40 and 80 stages (a lane owns two or three)
+    deep.name += "-deep"
+    yield deep, 2, [0, 0, 1]
 
 
 @pytest.mark.parametrize("w,gran,tps", list(_cases()), ids=lambda x: getattr(x, "name", None))
@@ -131,7 +135,7 @@ def test_mixed_search_argument_checks():
         assert L.sailor_plan_mixed(cx.ctx, C.byref(sp), C.byref(ok), 33, res, C.byref(n), None) == B.E_RANGE
         for bad in (B.Objective(0, B.FLAG_EVAL_ALL, 0.0, 0.0, 0.0), B.Objective(0, 0, 0.0, 0.0, 1.2)):
             assert L.sailor_plan_mixed(cx.ctx, C.byref(sp), C.byref(bad), 4, res, C.byref(n), None) == B.E_ARG
-        deep = B.make_mixed_space(w, 2, [0, 0], p_values=[33])
+        deep = B.make_mixed_space(w, 2, [0, 0], p_values=[B.MIX_P_MAX + 1])
         assert L.sailor_plan_mixed(cx.ctx, C.byref(deep), C.byref(ok), 4, res, C.byref(n), None) == B.E_RANGE
         fine = B.make_mixed_space(w, 5, [0, 0], d_values=[17])          # 17 replicas one by one: more units than the limit
         assert L.sailor_plan_mixed(cx.ctx, C.byref(fine), C.byref(ok), 4, res, C.byref(n), None) == B.E_RANGE
