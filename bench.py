@@ -348,7 +348,23 @@ def explicit_batches(B, torch, dev) -> dict:
             mean_p = float(base["P"].astype(np.float64).mean())
             out[key] = {"plans": n, "mean_stages": mean_p, "kernel_ms": ms, "plans_per_s": n / ms * 1e3,
                         "hbm_gb_per_s": n * 100 / ms / 1e6}
-            del d_plans, t, c, m, st
+            # the same batch through the host path: records and results in pinned host memory, copies inside the call
+            h_plans = d_plans.cpu().pin_memory()
+            ht = torch.empty(n, dtype=torch.float64).pin_memory(); hc = torch.empty(n, dtype=torch.float64).pin_memory()
+            hm = torch.empty(n, dtype=torch.int64).pin_memory(); hs = torch.empty(n, dtype=torch.int32).pin_memory()
+            host_call = lambda: B.sailor_simulate_host(ctx, h_plans.data_ptr(), n, ht.data_ptr(), hm.data_ptr(),
+                                                       hc.data_ptr(), hs.data_ptr())
+            host_call()
+            ts = []
+            for _ in range(3):
+                t0 = time.perf_counter()
+                host_call()
+                ts.append(time.perf_counter() - t0)
+            torch.cuda.synchronize()
+            same = bool(torch.equal(ht.view(torch.int64), t.cpu().view(torch.int64)) and torch.equal(hs, st.cpu()))
+            out[key].update({"host_call_ms": statistics.median(ts) * 1e3, "host_plans_per_s": n / statistics.median(ts),
+                             "host_pcie_gb_per_s": n * 100 / statistics.median(ts) / 1e9, "host_equals_device": same})
+            del d_plans, t, c, m, st, h_plans, ht, hc, hm, hs
         # plans whose stages mix GPU types among their replicas, up to 32 stages each: 648 B in + 28 B out per plan
         base = B.pack_mixed_plans(W.random_mixed_plans(w, 1 << 14, seed=13), stages=32)
         reps = 64

@@ -347,6 +347,13 @@ def sailor_simulate(ctx, plans: np.ndarray):
     return t, m, c, s
 
 
+def sailor_simulate_host(ctx, plans_ptr: int, n: int, t_iter_ptr: int, peak_mem_ptr: int, cost_ptr: int,
+                         status_ptr: int) -> None:
+    """Host path on raw host pointers (e.g. pinned buffers): copies in, simulates, copies out, returns when done."""
+    _check(load().sailor_simulate(ctx, plans_ptr, n, 0, t_iter_ptr or None, peak_mem_ptr or None, cost_ptr or None,
+                                  status_ptr or None), "sailor_simulate", ctx)
+
+
 def sailor_simulate_device(ctx, plans_ptr: int, n: int, t_iter_ptr: int, peak_mem_ptr: int, cost_ptr: int,
                            status_ptr: int) -> None:
     """Device path: raw device pointers (e.g. torch tensors' data_ptr()); only enqueues work."""

@@ -90,7 +90,9 @@ struct BatchConst {
     double intra_a[R_MAX], intra_i[R_MAX], inter_a[R_MAX], inter_i[R_MAX];
 };
 
+constexpr unsigned int SIM_ERR_DEVICE = 1u, SIM_ERR_BAD_RECORD = 2u;   // bits of the batch kernels' error word
 constexpr int BATCH_THREADS = 256;
+constexpr int BATCH_BLOCKS_PER_SM = 3;
 constexpr uint32_t BATCH_POOL = 512;             // records a block stages and orders at a time
 constexpr uint32_t REC_WORDS = sizeof(sailor_plan_rec) / 8;
 
@@ -248,10 +250,11 @@ __device__ __forceinline__ BatchOut simulate_batch_record(const BatchConst& k, c
 // stage count (the work of a record grows with both; any order gives the same results), and its warps take groups
 // of 32 similar records from the pool, longest first, until it is empty.  Results leave as four
 // structure-of-arrays streams.
-__global__ void __launch_bounds__(BATCH_THREADS, 3)
+__global__ void __launch_bounds__(BATCH_THREADS, BATCH_BLOCKS_PER_SM)
 simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
                 const sailor_plan_rec* __restrict__ plans, uint64_t n, double* __restrict__ t_iter,
-                uint64_t* __restrict__ peak_mem, double* __restrict__ cost, uint32_t* __restrict__ status) {
+                uint64_t* __restrict__ peak_mem, double* __restrict__ cost, uint32_t* __restrict__ status,
+                unsigned int* bad_flag) {                      // not null: set SIM_ERR_BAD_RECORD there when a record is refused
     __shared__ BatchConst k;
     __shared__ uint64_t recs[BATCH_POOL * REC_WORDS];
     __shared__ uint32_t hist[128];
@@ -340,6 +343,7 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
                 if (peak_mem) __stcs(&peak_mem[pool + mine], o.peak);
                 if (cost) __stcs(&cost[pool + mine], o.cost);
                 if (status) __stcs(&status[pool + mine], o.status);
+                if (bad_flag && (o.status & SAILOR_ST_BAD_RECORD)) atomicOr(bad_flag, SIM_ERR_BAD_RECORD);
             }
             __syncwarp();
         }

@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(SIM_THREADS, DEEP ? 2 : 4)
 simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restrict__ avail,
                       const unsigned char* __restrict__ plans, uint32_t stride, uint32_t max_stages, uint64_t n,
                       double* __restrict__ t_iter, uint64_t* __restrict__ peak_mem, double* __restrict__ cost,
-                      uint32_t* __restrict__ status, unsigned int* error, unsigned int* deep_seen) {
+                      uint32_t* __restrict__ status, unsigned int* error, unsigned int* deep_seen, uint32_t report_bad) {
     extern __shared__ __align__(16) unsigned char dyn[];
     __shared__ uint64_t mbar;
     if (DEEP && *reinterpret_cast<volatile unsigned int*>(deep_seen) == 0) return;
@@ -117,7 +117,7 @@ simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __
     constexpr uint32_t WARPS = SIM_THREADS / 32;
     const uint32_t static_bytes = reinterpret_cast<const TabHdr*>(blob)->static_bytes;
     if (!bulk_load(dyn, blob, static_bytes, &mbar)) {
-        if (tid == 0) atomicExch(error, 1u);
+        if (tid == 0) atomicOr(error, SIM_ERR_DEVICE);
         for (uint32_t x = tid; x < static_bytes / 16; x += SIM_THREADS)
             reinterpret_cast<uint4*>(dyn)[x] = reinterpret_cast<const uint4*>(blob)[x];
         __syncthreads();
@@ -147,6 +147,7 @@ simulate_mixed_kernel(const unsigned char* __restrict__ blob, const uint16_t* __
             if (peak_mem) peak_mem[j] = o.peak_mem;
             if (cost) cost[j] = o.cost;
             if (status) status[j] = o.status;
+            if (report_bad && (o.status & SAILOR_ST_BAD_RECORD)) atomicOr(error, SIM_ERR_BAD_RECORD);
         }
         __syncwarp();
     }
@@ -212,6 +213,8 @@ struct sailor_ctx {
     uint32_t grid_of[15] = {0};            // resident blocks per kernel variant, for the cached space
     SpaceCache space;
     cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr, evh0 = nullptr, evh1 = nullptr;
+    cudaStream_t out_stream = nullptr;     // results of a host batch leave on it while the next chunk comes in
+    cudaEvent_t ev_chunk = nullptr, ev_join = nullptr;
     // explicit-batch staging (grow-only)
     unsigned char* d_stage = nullptr;
     size_t stage_bytes = 0;
@@ -653,9 +656,70 @@ int finish_host_batch(sailor_ctx* ctx) {
     CU(ctx, stream_sync(ctx));
     if (*h_err) {
         CU(ctx, cudaMemsetAsync(ctx->d_sim_error, 0, sizeof(unsigned int), ctx->stream));
-        return SAILOR_E_DEVICE;
+        return (*h_err & SIM_ERR_DEVICE) ? SAILOR_E_DEVICE : SAILOR_E_RANGE;
     }
     return SAILOR_OK;
+}
+
+// A host-side batch: records of `rec_bytes` in, four result arrays out (any may be NULL).  The batch goes through
+// the device in chunks: a chunk's records are copied in and evaluated on the context's stream, its results leave
+// on a second stream while the next chunk comes in, so that the two directions of the host link carry data at
+// the same time.  Records are checked by the kernel that reads them (`launch` passes the error word along, and a
+// record outside its tables sets SIM_ERR_BAD_RECORD in it).  `launch(d_records, m, d_t, d_m, d_c, d_s)` enqueues
+// the evaluation of m records on the context's stream.
+constexpr uint64_t HOST_CHUNK = 1u << 19;
+int upload_availability(sailor_ctx* ctx);
+
+template <class Launch>
+int host_batch(sailor_ctx* ctx, const unsigned char* recs, size_t rec_bytes, uint64_t n, double* t_iter, uint64_t* peak_mem,
+               double* cost, uint32_t* status, Launch launch) {
+    const size_t need = n * (rec_bytes + 32);
+    if (need > ctx->stage_bytes) {
+        CU(ctx, stream_sync(ctx));
+        cudaFree(ctx->d_stage);
+        ctx->d_stage = nullptr;
+        ctx->stage_bytes = 0;
+        cudaError_t e = cudaMalloc(&ctx->d_stage, need);
+        if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
+        ctx->stage_bytes = need;
+    }
+    unsigned char* base = ctx->d_stage;
+    double* d_t = reinterpret_cast<double*>(base);
+    double* d_c = reinterpret_cast<double*>(base + 8 * n);
+    uint64_t* d_m = reinterpret_cast<uint64_t*>(base + 16 * n);
+    uint32_t* d_s = reinterpret_cast<uint32_t*>(base + 24 * n);
+    unsigned char* d_recs = base + 32 * n;
+    {
+        const int rc_up = upload_availability(ctx);
+        if (rc_up) return rc_up;
+    }
+    const bool split = n > HOST_CHUNK;
+    cudaStream_t out = split ? ctx->out_stream : ctx->stream;
+    int rc = SAILOR_OK;
+    cudaError_t ce = cudaSuccess;
+    for (uint64_t off = 0; off < n && ce == cudaSuccess && rc == SAILOR_OK; off += HOST_CHUNK) {
+        const uint64_t m = n - off < HOST_CHUNK ? n - off : HOST_CHUNK;
+        ce = cudaMemcpyAsync(d_recs + off * rec_bytes, recs + off * rec_bytes, m * rec_bytes, cudaMemcpyHostToDevice, ctx->stream);
+        if (ce != cudaSuccess) break;
+        rc = launch(d_recs + off * rec_bytes, m, d_t + off, d_m + off, d_c + off, d_s + off);
+        if (rc != SAILOR_OK) break;
+        if (split) {
+            if ((ce = cudaEventRecord(ctx->ev_chunk, ctx->stream)) != cudaSuccess) break;
+            if ((ce = cudaStreamWaitEvent(out, ctx->ev_chunk, 0)) != cudaSuccess) break;
+        }
+        if (t_iter && ce == cudaSuccess) ce = cudaMemcpyAsync(t_iter + off, d_t + off, 8 * m, cudaMemcpyDeviceToHost, out);
+        if (cost && ce == cudaSuccess) ce = cudaMemcpyAsync(cost + off, d_c + off, 8 * m, cudaMemcpyDeviceToHost, out);
+        if (peak_mem && ce == cudaSuccess) ce = cudaMemcpyAsync(peak_mem + off, d_m + off, 8 * m, cudaMemcpyDeviceToHost, out);
+        if (status && ce == cudaSuccess) ce = cudaMemcpyAsync(status + off, d_s + off, 4 * m, cudaMemcpyDeviceToHost, out);
+    }
+    if (split) {                   // whatever happened, the context's stream waits for what the second one was given
+        cudaError_t cj = cudaEventRecord(ctx->ev_join, out);
+        if (cj == cudaSuccess) cj = cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0);
+        if (cj != cudaSuccess) { cudaStreamSynchronize(out); if (ce == cudaSuccess) ce = cj; }
+    }
+    const int rc_end = finish_host_batch(ctx);                 // waits for everything enqueued above
+    if (ce != cudaSuccess) { ctx->last_cuda = (int)ce; return SAILOR_E_CUDA; }
+    return rc != SAILOR_OK ? rc : rc_end;
 }
 
 // The device copy of the availability snapshot, for kernels that read it through a pointer.
@@ -668,19 +732,6 @@ int upload_availability(sailor_ctx* ctx) {
     ctx->h2d_fresh = true;
     ctx->avail_dirty = false;
     return SAILOR_OK;
-}
-
-int validate_host_record(const sailor_ctx* ctx, const sailor_plan_rec& r) {
-    const TabHdr& h = ctx->hdr;
-    if (r.P < 1 || r.P > SAILOR_P_MAX || r.n_runs < 1 || r.n_runs > SAILOR_RUN_MAX || r.D < 1) return SAILOR_E_RANGE;
-    if (r.mbs_idx >= h.n_mbs) return SAILOR_E_RANGE;
-    uint32_t tot = 0;
-    for (uint32_t q = 0; q < r.n_runs; ++q) {
-        if (r.run[q].type >= h.T || r.run[q].zone >= h.Z || r.run[q].tp_idx >= h.n_tp || r.run[q].n_stages < 1)
-            return SAILOR_E_RANGE;
-        tot += r.run[q].n_stages;
-    }
-    return tot == r.P ? SAILOR_OK : SAILOR_E_RANGE;
 }
 
 }  // namespace
@@ -848,6 +899,9 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     CUF(cudaEventCreate(&ctx->ev2));
     CUF(cudaEventCreate(&ctx->evh0));
     CUF(cudaEventCreate(&ctx->evh1));
+    CUF(cudaStreamCreateWithFlags(&ctx->out_stream, cudaStreamNonBlocking));
+    CUF(cudaEventCreateWithFlags(&ctx->ev_chunk, cudaEventDisableTiming));
+    CUF(cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming));
     CUF(cudaMemcpyAsync(ctx->d_blob, blob.data(), h.total_bytes, cudaMemcpyHostToDevice, ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_avail, 0, R_MAX * sizeof(uint16_t), ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_ctrl, 0, sizeof(Ctrl), ctx->stream));
@@ -899,8 +953,9 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->d_stage);
     cudaFree(ctx->d_mix);
     cudaFree(ctx->d_dp);
-    for (cudaEvent_t e : {ctx->ev0, ctx->ev1, ctx->ev2, ctx->evh0, ctx->evh1})
+    for (cudaEvent_t e : {ctx->ev0, ctx->ev1, ctx->ev2, ctx->evh0, ctx->evh1, ctx->ev_chunk, ctx->ev_join})
         if (e) cudaEventDestroy(e);
+    if (ctx->out_stream) cudaStreamDestroy(ctx->out_stream);
     delete ctx;
     return SAILOR_OK;
 }
@@ -923,52 +978,25 @@ int sailor_simulate(sailor_ctx* ctx, const sailor_plan_rec* plans, uint64_t n, i
     if (n == 0) return SAILOR_OK;
     if ((uintptr_t)plans % 8 != 0) return SAILOR_E_ARG;
     DeviceGuard guard(ctx->device);
-    const sailor_plan_rec* d_plans = plans;
-    double *d_t = t_iter, *d_c = cost;
-    uint64_t* d_m = peak_mem;
-    uint32_t* d_s = status;
-    if (!on_device) {
-        for (uint64_t j = 0; j < n; ++j) {
-            const int rc = validate_host_record(ctx, plans[j]);
-            if (rc) return rc;
-        }
-        const size_t need = n * (sizeof(sailor_plan_rec) + 32);
-        if (need > ctx->stage_bytes) {
-            CU(ctx, stream_sync(ctx));
-            cudaFree(ctx->d_stage);
-            ctx->d_stage = nullptr;
-            ctx->stage_bytes = 0;
-            cudaError_t e = cudaMalloc(&ctx->d_stage, need);
-            if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
-            ctx->stage_bytes = need;
-        }
-        unsigned char* base = ctx->d_stage;
-        d_t = reinterpret_cast<double*>(base);
-        d_c = reinterpret_cast<double*>(base + 8 * n);
-        d_m = reinterpret_cast<uint64_t*>(base + 16 * n);
-        d_s = reinterpret_cast<uint32_t*>(base + 24 * n);
-        sailor_plan_rec* dp = reinterpret_cast<sailor_plan_rec*>(base + 32 * n);
-        CU(ctx, cudaMemcpyAsync(dp, plans, n * sizeof(sailor_plan_rec), cudaMemcpyHostToDevice, ctx->stream));
-        d_plans = dp;
-    }
+    auto launch = [ctx](const sailor_plan_rec* d_plans, uint64_t m, double* d_t, uint64_t* d_m, double* d_c, uint32_t* d_s,
+                        unsigned int* bad_flag) {
+        const uint64_t tiles = (m + BATCH_POOL - 1) / BATCH_POOL;
+        const uint64_t cap = (uint64_t)ctx->sm_count * BATCH_BLOCKS_PER_SM * 4;   // the resident blocks, four pools each at least
+        const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
+        simulate_kernel<<<grid, BATCH_THREADS, 0, ctx->stream>>>(ctx->d_blob, ctx->d_avail, d_plans, m, d_t, d_m, d_c, d_s, bad_flag);
+        CU(ctx, cudaGetLastError());
+        return (int)SAILOR_OK;
+    };
+    if (!on_device)                                               // records are checked by the kernel (SIM_ERR_BAD_RECORD)
+        return host_batch(ctx, reinterpret_cast<const unsigned char*>(plans), sizeof(sailor_plan_rec), n, t_iter, peak_mem, cost,
+                          status, [&](const unsigned char* d_recs, uint64_t m, double* d_t, uint64_t* d_m, double* d_c, uint32_t* d_s) {
+                              return launch(reinterpret_cast<const sailor_plan_rec*>(d_recs), m, d_t, d_m, d_c, d_s, ctx->d_sim_error);
+                          });
     {
         const int rc_up = upload_availability(ctx);
         if (rc_up) return rc_up;
     }
-    const uint64_t tiles = (n + BATCH_POOL - 1) / BATCH_POOL;
-    const uint64_t cap = (uint64_t)ctx->sm_count * 12;         // three resident blocks per SM, four pools each at least
-    const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
-    simulate_kernel<<<grid, BATCH_THREADS, 0, ctx->stream>>>(
-        ctx->d_blob, ctx->d_avail, d_plans, n, d_t, d_m, d_c, d_s);
-    CU(ctx, cudaGetLastError());
-    if (!on_device) {
-        if (t_iter) CU(ctx, cudaMemcpyAsync(t_iter, d_t, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        if (cost) CU(ctx, cudaMemcpyAsync(cost, d_c, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        if (peak_mem) CU(ctx, cudaMemcpyAsync(peak_mem, d_m, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        if (status) CU(ctx, cudaMemcpyAsync(status, d_s, 4 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        return finish_host_batch(ctx);
-    }
-    return SAILOR_OK;
+    return launch(plans, n, t_iter, peak_mem, cost, status, nullptr);
 }
 
 int sailor_simulate_mixed(sailor_ctx* ctx, const sailor_mixed_plan* plans, uint64_t n, int on_device, double* t_iter,
@@ -988,70 +1016,37 @@ int sailor_simulate_mixed_strided(sailor_ctx* ctx, const void* plans_v, uint64_t
     if ((uintptr_t)plans % 8 != 0) return SAILOR_E_ARG;
     const uint32_t max_stages = (record_bytes - HEAD) / (uint32_t)sizeof(sailor_mixed_stage);
     DeviceGuard guard(ctx->device);
-    const unsigned char* d_plans = plans;
-    bool any_deep = false;
-    double *d_t = t_iter, *d_c = cost;
-    uint64_t* d_m = peak_mem;
-    uint32_t* d_s = status;
-    if (!on_device) {
-        const TabHdr& h = ctx->hdr;
-        for (uint64_t j = 0; j < n; ++j) {
-            const sailor_mixed_plan& r = *reinterpret_cast<const sailor_mixed_plan*>(plans + j * record_bytes);
-            if (r.P < 1 || r.P > max_stages || r.D < 1 || r.mbs_idx >= h.n_mbs) return SAILOR_E_RANGE;
-            any_deep = any_deep || r.P > 32;
-            for (uint32_t i = 0; i < r.P; ++i) {
-                const sailor_mixed_stage& st = r.stage[i];
-                if (st.zone >= h.Z || st.n_groups < 1 || st.n_groups > SAILOR_MIX_GROUPS_MAX) return SAILOR_E_RANGE;
-                for (uint32_t q = 0; q < st.n_groups; ++q)
-                    if (st.group[q].type >= h.T || st.group[q].tp_idx >= h.n_tp) return SAILOR_E_RANGE;
-            }
+    auto launch = [ctx, record_bytes, max_stages](const unsigned char* d_plans, uint64_t m, double* d_t, uint64_t* d_m, double* d_c,
+                                                  uint32_t* d_s, uint32_t report_bad) {
+        const uint64_t tiles = (m + SIM_THREADS / 32 - 1) / (SIM_THREADS / 32);     // a warp per plan
+        const uint64_t cap = (uint64_t)ctx->sm_count * 32;
+        const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
+        const size_t smem = ctx->hdr.static_bytes + sizeof(unsigned long long) * (SIM_THREADS / 32) * ctx->hdr.R;
+        unsigned int* deep_seen = ctx->d_sim_error + 1;
+        if (max_stages > 32) CU(ctx, cudaMemsetAsync(deep_seen, 0, sizeof(unsigned int), ctx->stream));
+        simulate_mixed_kernel<false><<<grid, SIM_THREADS, smem, ctx->stream>>>(ctx->d_blob, ctx->d_avail, d_plans, record_bytes,
+                                                                                max_stages, m, d_t, d_m, d_c, d_s, ctx->d_sim_error,
+                                                                                deep_seen, report_bad);
+        CU(ctx, cudaGetLastError());
+        if (max_stages > 32) {                                   // the plans of more than 32 stages, if the first launch saw any
+            const uint64_t cap2 = (uint64_t)ctx->sm_count * 16;
+            simulate_mixed_kernel<true><<<(uint32_t)(tiles < cap2 ? tiles : cap2), SIM_THREADS, smem, ctx->stream>>>(
+                ctx->d_blob, ctx->d_avail, d_plans, record_bytes, max_stages, m, d_t, d_m, d_c, d_s, ctx->d_sim_error, deep_seen,
+                report_bad);
+            CU(ctx, cudaGetLastError());
         }
-        const size_t need = n * ((size_t)record_bytes + 32);
-        if (need > ctx->stage_bytes) {
-            CU(ctx, stream_sync(ctx));
-            cudaFree(ctx->d_stage);
-            ctx->d_stage = nullptr;
-            ctx->stage_bytes = 0;
-            cudaError_t e = cudaMalloc(&ctx->d_stage, need);
-            if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
-            ctx->stage_bytes = need;
-        }
-        unsigned char* base = ctx->d_stage;
-        d_t = reinterpret_cast<double*>(base);
-        d_c = reinterpret_cast<double*>(base + 8 * n);
-        d_m = reinterpret_cast<uint64_t*>(base + 16 * n);
-        d_s = reinterpret_cast<uint32_t*>(base + 24 * n);
-        unsigned char* dp = base + 32 * n;
-        CU(ctx, cudaMemcpyAsync(dp, plans, n * (size_t)record_bytes, cudaMemcpyHostToDevice, ctx->stream));
-        d_plans = dp;
-    }
+        return (int)SAILOR_OK;
+    };
+    if (!on_device)                                               // records are checked by the kernel (SIM_ERR_BAD_RECORD)
+        return host_batch(ctx, plans, record_bytes, n, t_iter, peak_mem, cost, status,
+                          [&](const unsigned char* d_recs, uint64_t m, double* d_t, uint64_t* d_m, double* d_c, uint32_t* d_s) {
+                              return launch(d_recs, m, d_t, d_m, d_c, d_s, 1u);
+                          });
     {
         const int rc_up = upload_availability(ctx);
         if (rc_up) return rc_up;
     }
-    const uint64_t tiles = (n + SIM_THREADS / 32 - 1) / (SIM_THREADS / 32);     // a warp per plan
-    const uint64_t cap = (uint64_t)ctx->sm_count * 32;
-    const uint32_t grid = (uint32_t)(tiles < cap ? tiles : cap);
-    const size_t smem = ctx->hdr.static_bytes + sizeof(unsigned long long) * (SIM_THREADS / 32) * ctx->hdr.R;
-    unsigned int* deep_seen = ctx->d_sim_error + 1;
-    if (max_stages > 32) CU(ctx, cudaMemsetAsync(deep_seen, 0, sizeof(unsigned int), ctx->stream));
-    simulate_mixed_kernel<false><<<grid, SIM_THREADS, smem, ctx->stream>>>(ctx->d_blob, ctx->d_avail, d_plans, record_bytes,
-                                                                            max_stages, n, d_t, d_m, d_c, d_s, ctx->d_sim_error,
-                                                                            deep_seen);
-    if (max_stages > 32 && (on_device || any_deep)) {            // the plans of more than 32 stages, if there are any
-        const uint64_t cap2 = (uint64_t)ctx->sm_count * 16;
-        simulate_mixed_kernel<true><<<(uint32_t)(tiles < cap2 ? tiles : cap2), SIM_THREADS, smem, ctx->stream>>>(
-            ctx->d_blob, ctx->d_avail, d_plans, record_bytes, max_stages, n, d_t, d_m, d_c, d_s, ctx->d_sim_error, deep_seen);
-    }
-    CU(ctx, cudaGetLastError());
-    if (!on_device) {
-        if (t_iter) CU(ctx, cudaMemcpyAsync(t_iter, d_t, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        if (cost) CU(ctx, cudaMemcpyAsync(cost, d_c, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        if (peak_mem) CU(ctx, cudaMemcpyAsync(peak_mem, d_m, 8 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        if (status) CU(ctx, cudaMemcpyAsync(status, d_s, 4 * n, cudaMemcpyDeviceToHost, ctx->stream));
-        return finish_host_batch(ctx);
-    }
-    return SAILOR_OK;
+    return launch(plans, n, t_iter, peak_mem, cost, status, 0u);
 }
 
 int sailor_space_size(const sailor_ctx* ctx, const sailor_space* s, uint64_t* n_out) {

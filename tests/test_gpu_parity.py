@@ -143,6 +143,30 @@ def test_simulate_empty_and_bad_records(make_ctx, torch_cuda):
     torch.cuda.synchronize()
     assert st.cpu().tolist()[1] == B.ST_BAD_RECORD and (st.cpu().tolist()[0] & B.ST_BAD_RECORD) == 0
     assert math.isnan(tt.cpu().tolist()[1])
+    # a refused device record does not make a later host call fail, and a refused host batch leaves nothing behind
+    t, m, c, s = B.sailor_simulate(cx.ctx, B.pack_records(good))
+    assert s[0] == Oracle(w).simulate_records(good)[0][0]
+    # the host batch with a bad record in it: E_RANGE, results written, the bad one flagged
+    L = B.load()
+    out_t = np.zeros(2); out_s = np.zeros(2, np.uint32)
+    assert L.sailor_simulate(cx.ctx, both.ctypes.data, 2, 0, out_t.ctypes.data, None, None, out_s.ctypes.data) == B.E_RANGE
+    assert out_s[1] == B.ST_BAD_RECORD and out_s[0] == s[0] and math.isnan(out_t[1]) and out_t[0] == t[0]
+    assert L.sailor_simulate(cx.ctx, both.ctypes.data, 1, 0, out_t.ctypes.data, None, None, out_s.ctypes.data) == B.OK
+
+
+def test_simulate_host_batch_in_chunks(make_ctx):
+    """A host batch larger than the chunk the library moves at a time (2^19 records): every record's results are the
+    oracle's, whichever chunk it was in, and a ragged last chunk."""
+    w = W.config2()
+    cx = make_ctx(w)
+    recs = W.random_plans(w, 6007, seed=77, max_runs=8, hetero_tp=True)
+    base = B.pack_records(recs)
+    reps = (3 * (1 << 19)) // 6007 // 2 + 1                         # about 1.5 chunks ... plus a tail
+    big = np.tile(base, reps)[: (1 << 19) + 200_003]
+    t, m, c, s = B.sailor_simulate(cx.ctx, big)
+    so, to, co, mo = Oracle(w).simulate_records(recs)
+    idx = np.arange(big.size) % 6007
+    assert_sim_equal((t, m, c, s), (so[idx], to[idx], co[idx], mo[idx]), "host batch in chunks")
 
 
 # ---- enumeration ---------------------------------------------------------------------------------
