@@ -32,7 +32,9 @@ def subspace_costs(w) -> List[Tuple[int, float]]:
     return out
 
 
-COST_FIXED, COST_PER_STAGE = 9.0, 1.0
+# Fitted to the search times of workload 5's sub-spaces of equal size (pipelines of 4, 6, 8, 12, 16 stages: 1, 1, 2, 3, 4
+# stages in the last segment; 2.67, 2.69, 2.87, 3.03, 3.11 ms on one B200): time = 2.53 + 0.15 x stages.
+COST_FIXED, COST_PER_STAGE = 17.0, 1.0
 
 
 def split_by_cost(parts: Sequence[Tuple[int, float]], world: int, rank: int) -> Tuple[int, int]:
