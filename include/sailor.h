@@ -277,8 +277,9 @@ int sailor_set_availability(sailor_ctx* ctx, const uint16_t* avail);
  * arrays of n; any of them may be NULL.  t_iter and cost are NaN when SAILOR_ST_INVALID
  * or SAILOR_ST_BAD_RECORD is set; peak_mem is the maximum over stages of the per-GPU peak
  * (with N_b taken as floor(gbs / (D*mbs))).  A different tp per run is accepted (Sec. 4.4).
- * Host batches of more than 2^19 records go through the device in chunks, results coming back while the next
- * chunk goes in.  Records are checked on the device, by the kernel that reads them.
+ * Host batches go through the device in chunks (2^19 records or 64 MB of records, whichever is less), results
+ * coming back while the next chunk goes in; the library stages at most three chunks at a time, whatever n is.
+ * Records are checked on the device, by the kernel that reads them.
  * Errors: E_ARG (null ctx/plans, unaligned plans), E_RANGE (host records only: an index
  * outside its table, n_runs or P outside limits, run lengths not summing to P; the outputs are
  * written all the same, the refused records with SAILOR_ST_BAD_RECORD and NaN), E_CUDA. */

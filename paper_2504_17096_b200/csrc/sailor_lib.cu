@@ -214,7 +214,7 @@ struct sailor_ctx {
     SpaceCache space;
     cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr, evh0 = nullptr, evh1 = nullptr;
     cudaStream_t out_stream = nullptr;     // results of a host batch leave on it while the next chunk comes in
-    cudaEvent_t ev_chunk = nullptr, ev_join = nullptr;
+    cudaEvent_t ev_chunk = nullptr, ev_join = nullptr, ev_slot[3] = {nullptr, nullptr, nullptr};
     // explicit-batch staging (grow-only)
     unsigned char* d_stage = nullptr;
     size_t stage_bytes = 0;
@@ -662,18 +662,27 @@ int finish_host_batch(sailor_ctx* ctx) {
 }
 
 // A host-side batch: records of `rec_bytes` in, four result arrays out (any may be NULL).  The batch goes through
-// the device in chunks: a chunk's records are copied in and evaluated on the context's stream, its results leave
-// on a second stream while the next chunk comes in, so that the two directions of the host link carry data at
-// the same time.  Records are checked by the kernel that reads them (`launch` passes the error word along, and a
-// record outside its tables sets SIM_ERR_BAD_RECORD in it).  `launch(d_records, m, d_t, d_m, d_c, d_s)` enqueues
-// the evaluation of m records on the context's stream.
-constexpr uint64_t HOST_CHUNK = 1u << 19;
+// the device in chunks that take turns in HOST_SLOTS staging slots: a chunk's records are copied in and evaluated
+// on the context's stream, its results leave on a second stream while the next chunk comes in, so that the two
+// directions of the host link carry data at the same time; a slot is filled again only after its results have
+// left.  The staging memory therefore does not grow with the batch beyond HOST_SLOTS chunks.  Records are checked
+// by the kernel that reads them (`launch` passes the error word along, and a record outside its tables sets
+// SIM_ERR_BAD_RECORD in it).  `launch(d_records, m, d_t, d_m, d_c, d_s)` enqueues the evaluation of m records on
+// the context's stream.
+constexpr uint64_t HOST_CHUNK_RECORDS = 1u << 19, HOST_CHUNK_BYTES = 1u << 26;
+constexpr uint32_t HOST_SLOTS = 3;
 int upload_availability(sailor_ctx* ctx);
 
 template <class Launch>
 int host_batch(sailor_ctx* ctx, const unsigned char* recs, size_t rec_bytes, uint64_t n, double* t_iter, uint64_t* peak_mem,
                double* cost, uint32_t* status, Launch launch) {
-    const size_t need = n * (rec_bytes + 32);
+    uint64_t chunk = HOST_CHUNK_BYTES / rec_bytes;             // records per chunk: 64 MB of records, 2^19 at most
+    chunk = chunk > HOST_CHUNK_RECORDS ? HOST_CHUNK_RECORDS : chunk;
+    const bool split = n > chunk;
+    const uint64_t slot_records = split ? chunk : n;
+    const size_t slot_bytes = (slot_records * (rec_bytes + 32) + 255) / 256 * 256;
+    const uint64_t n_chunks = (n + chunk - 1) / chunk;
+    const size_t need = slot_bytes * (split ? (n_chunks < HOST_SLOTS ? n_chunks : HOST_SLOTS) : 1);
     if (need > ctx->stage_bytes) {
         CU(ctx, stream_sync(ctx));
         cudaFree(ctx->d_stage);
@@ -683,34 +692,38 @@ int host_batch(sailor_ctx* ctx, const unsigned char* recs, size_t rec_bytes, uin
         if (e != cudaSuccess) { ctx->last_cuda = (int)e; return SAILOR_E_NOMEM; }
         ctx->stage_bytes = need;
     }
-    unsigned char* base = ctx->d_stage;
-    double* d_t = reinterpret_cast<double*>(base);
-    double* d_c = reinterpret_cast<double*>(base + 8 * n);
-    uint64_t* d_m = reinterpret_cast<uint64_t*>(base + 16 * n);
-    uint32_t* d_s = reinterpret_cast<uint32_t*>(base + 24 * n);
-    unsigned char* d_recs = base + 32 * n;
     {
         const int rc_up = upload_availability(ctx);
         if (rc_up) return rc_up;
     }
-    const bool split = n > HOST_CHUNK;
     cudaStream_t out = split ? ctx->out_stream : ctx->stream;
     int rc = SAILOR_OK;
     cudaError_t ce = cudaSuccess;
-    for (uint64_t off = 0; off < n && ce == cudaSuccess && rc == SAILOR_OK; off += HOST_CHUNK) {
-        const uint64_t m = n - off < HOST_CHUNK ? n - off : HOST_CHUNK;
-        ce = cudaMemcpyAsync(d_recs + off * rec_bytes, recs + off * rec_bytes, m * rec_bytes, cudaMemcpyHostToDevice, ctx->stream);
+    uint64_t c = 0;
+    for (uint64_t off = 0; off < n && ce == cudaSuccess && rc == SAILOR_OK; off += chunk, ++c) {
+        const uint64_t m = n - off < chunk ? n - off : chunk;
+        const uint32_t slot = (uint32_t)(c % HOST_SLOTS);
+        unsigned char* base = ctx->d_stage + (split ? slot * slot_bytes : 0);
+        double* d_t = reinterpret_cast<double*>(base);
+        double* d_c = reinterpret_cast<double*>(base + 8 * slot_records);
+        uint64_t* d_m = reinterpret_cast<uint64_t*>(base + 16 * slot_records);
+        uint32_t* d_s = reinterpret_cast<uint32_t*>(base + 24 * slot_records);
+        unsigned char* d_recs = base + 32 * slot_records;
+        if (split && c >= HOST_SLOTS)                          // the slot's earlier results have to be out first
+            if ((ce = cudaStreamWaitEvent(ctx->stream, ctx->ev_slot[slot], 0)) != cudaSuccess) break;
+        ce = cudaMemcpyAsync(d_recs, recs + off * rec_bytes, m * rec_bytes, cudaMemcpyHostToDevice, ctx->stream);
         if (ce != cudaSuccess) break;
-        rc = launch(d_recs + off * rec_bytes, m, d_t + off, d_m + off, d_c + off, d_s + off);
+        rc = launch(d_recs, m, d_t, d_m, d_c, d_s);
         if (rc != SAILOR_OK) break;
         if (split) {
             if ((ce = cudaEventRecord(ctx->ev_chunk, ctx->stream)) != cudaSuccess) break;
             if ((ce = cudaStreamWaitEvent(out, ctx->ev_chunk, 0)) != cudaSuccess) break;
         }
-        if (t_iter && ce == cudaSuccess) ce = cudaMemcpyAsync(t_iter + off, d_t + off, 8 * m, cudaMemcpyDeviceToHost, out);
-        if (cost && ce == cudaSuccess) ce = cudaMemcpyAsync(cost + off, d_c + off, 8 * m, cudaMemcpyDeviceToHost, out);
-        if (peak_mem && ce == cudaSuccess) ce = cudaMemcpyAsync(peak_mem + off, d_m + off, 8 * m, cudaMemcpyDeviceToHost, out);
-        if (status && ce == cudaSuccess) ce = cudaMemcpyAsync(status + off, d_s + off, 4 * m, cudaMemcpyDeviceToHost, out);
+        if (t_iter && ce == cudaSuccess) ce = cudaMemcpyAsync(t_iter + off, d_t, 8 * m, cudaMemcpyDeviceToHost, out);
+        if (cost && ce == cudaSuccess) ce = cudaMemcpyAsync(cost + off, d_c, 8 * m, cudaMemcpyDeviceToHost, out);
+        if (peak_mem && ce == cudaSuccess) ce = cudaMemcpyAsync(peak_mem + off, d_m, 8 * m, cudaMemcpyDeviceToHost, out);
+        if (status && ce == cudaSuccess) ce = cudaMemcpyAsync(status + off, d_s, 4 * m, cudaMemcpyDeviceToHost, out);
+        if (split && ce == cudaSuccess) ce = cudaEventRecord(ctx->ev_slot[slot], out);
     }
     if (split) {                   // whatever happened, the context's stream waits for what the second one was given
         cudaError_t cj = cudaEventRecord(ctx->ev_join, out);
@@ -902,6 +915,7 @@ static int create_impl(const sailor_model* m, const sailor_profile* p, const sai
     CUF(cudaStreamCreateWithFlags(&ctx->out_stream, cudaStreamNonBlocking));
     CUF(cudaEventCreateWithFlags(&ctx->ev_chunk, cudaEventDisableTiming));
     CUF(cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming));
+    for (cudaEvent_t& e : ctx->ev_slot) CUF(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
     CUF(cudaMemcpyAsync(ctx->d_blob, blob.data(), h.total_bytes, cudaMemcpyHostToDevice, ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_avail, 0, R_MAX * sizeof(uint16_t), ctx->stream));
     CUF(cudaMemsetAsync(ctx->d_ctrl, 0, sizeof(Ctrl), ctx->stream));
@@ -953,7 +967,8 @@ int sailor_destroy(sailor_ctx* ctx) {
     cudaFree(ctx->d_stage);
     cudaFree(ctx->d_mix);
     cudaFree(ctx->d_dp);
-    for (cudaEvent_t e : {ctx->ev0, ctx->ev1, ctx->ev2, ctx->evh0, ctx->evh1, ctx->ev_chunk, ctx->ev_join})
+    for (cudaEvent_t e : {ctx->ev0, ctx->ev1, ctx->ev2, ctx->evh0, ctx->evh1, ctx->ev_chunk, ctx->ev_join, ctx->ev_slot[0],
+                          ctx->ev_slot[1], ctx->ev_slot[2]})
         if (e) cudaEventDestroy(e);
     if (ctx->out_stream) cudaStreamDestroy(ctx->out_stream);
     delete ctx;

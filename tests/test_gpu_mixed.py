@@ -128,6 +128,19 @@ def test_mixed_record_sizes():
         assert ds.cpu().tolist()[1] == B.ST_BAD_RECORD and ds.cpu().tolist()[0] == int(orc[0][0]) and math.isnan(dt.cpu().tolist()[1])
 
 
+def test_mixed_host_batch_in_chunks():
+    """A host batch of more chunks than staging slots (64 MB of records a chunk, three slots), deep plans among them."""
+    w = W.config5()
+    plans = W.random_mixed_plans(w, 3001, seed=31, p_max=96)
+    base = B.pack_mixed_plans(plans, stages=B.MIX_P_MAX)            # 1 928 B a record: 34 807 records a chunk
+    n = 5 * 34_807 + 1_234
+    big = np.tile(base, n // 3001 + 1)[:n]
+    so, to, co, mo = Oracle(w).simulate_mixed_batch(plans)
+    idx = np.arange(n) % 3001
+    with Ctx(w) as cx:
+        assert_equal(B.sailor_simulate_mixed(cx.ctx, big), (so[idx], to[idx], co[idx], mo[idx]), "mixed host batch in chunks")
+
+
 def test_mixed_with_one_group_equals_sailor_simulate():
     """No mixing: the same numbers as the run-length records of sailor_simulate."""
     w = W.config2()

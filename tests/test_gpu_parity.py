@@ -155,14 +155,14 @@ def test_simulate_empty_and_bad_records(make_ctx, torch_cuda):
 
 
 def test_simulate_host_batch_in_chunks(make_ctx):
-    """A host batch larger than the chunk the library moves at a time (2^19 records): every record's results are the
-    oracle's, whichever chunk it was in, and a ragged last chunk."""
+    """A host batch larger than what the library stages at a time (chunks of 2^19 records taking turns in three
+    slots): every record's results are the oracle's, whichever chunk and slot it went through; a ragged last chunk."""
     w = W.config2()
     cx = make_ctx(w)
     recs = W.random_plans(w, 6007, seed=77, max_runs=8, hetero_tp=True)
     base = B.pack_records(recs)
-    reps = (3 * (1 << 19)) // 6007 // 2 + 1                         # about 1.5 chunks ... plus a tail
-    big = np.tile(base, reps)[: (1 << 19) + 200_003]
+    n = 4 * (1 << 19) + 200_003                                     # five chunks: slots 0 and 1 are used twice
+    big = np.tile(base, n // 6007 + 1)[:n]
     t, m, c, s = B.sailor_simulate(cx.ctx, big)
     so, to, co, mo = Oracle(w).simulate_records(recs)
     idx = np.arange(big.size) % 6007
