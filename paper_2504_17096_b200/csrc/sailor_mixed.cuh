@@ -47,24 +47,28 @@ __device__ inline SimOut simulate_mixed_warp(const TabView& v, const uint16_t* _
     if (P < 1 || P > 32 || D < 1 || mi >= h->n_mbs) return o;
     const bool mine = lane < P;
 
-    // this lane's stage
-    uint32_t zone = 0, ng = 0, gtype[SAILOR_MIX_GROUPS_MAX], gtpi[SAILOR_MIX_GROUPS_MAX], gcount[SAILOR_MIX_GROUPS_MAX];
-#pragma unroll
-    for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q) gtype[q] = gtpi[q] = gcount[q] = 0;
+    // this lane's stage; group q as one word (type | tp_idx << 8 | count << 16), two words to a register pair, so
+    // that the loops over a stage's groups need not be unrolled (the kernel waits on instruction fetch)
+    uint32_t zone = 0, ng = 0;
+    uint64_t g01 = 0, g23 = 0;
+    auto group_word = [&](uint32_t q) { return (uint32_t)((q & 2u ? g23 : g01) >> (32u * (q & 1u))); };
     bool bad = false;
     if (mine) {
         const sailor_mixed_stage& s = r.stage[lane];
         zone = s.zone;
         ng = s.n_groups;
         bad = zone >= Z || ng < 1 || ng > SAILOR_MIX_GROUPS_MAX;
-#pragma unroll
-        for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q)
-            if (!bad && q < ng) {
-                gtype[q] = s.group[q].type; gtpi[q] = s.group[q].tp_idx; gcount[q] = s.group[q].count;
+        if (!bad) {
+            const uint32_t* g32 = reinterpret_cast<const uint32_t*>(&s.group[0]);      // a group is four bytes
+            const uint32_t w0 = g32[0], w1 = ng > 1 ? g32[1] : 0u, w2 = ng > 2 ? g32[2] : 0u, w3 = ng > 3 ? g32[3] : 0u;
+            g01 = (uint64_t)w0 | (uint64_t)w1 << 32;
+            g23 = (uint64_t)w2 | (uint64_t)w3 << 32;
+#pragma unroll 1
+            for (uint32_t q = 0; q < ng; ++q) {
+                const uint32_t gq = group_word(q);
+                bad = bad || (gq & 0xff) >= T || ((gq >> 8) & 0xff) >= h->n_tp;
             }
-#pragma unroll
-        for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q)
-            if (q < ng) bad = bad || gtype[q] >= T || gtpi[q] >= h->n_tp;
+        }
     }
     if (__any_sync(MIX_FULL, bad)) return o;
 
@@ -79,9 +83,7 @@ __device__ inline SimOut simulate_mixed_warp(const TabView& v, const uint16_t* _
     __syncwarp();
     const double steps = (double)(2 * (uint64_t)(D - 1));
     const double coef = steps / (double)D;
-    double sync_l = 0.0, upd_l = 0.0, term[SAILOR_MIX_GROUPS_MAX];
-#pragma unroll
-    for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q) term[q] = 0.0;
+    double sync_l = 0.0, upd_l = 0.0;
     uint64_t peak_l = 0;
     size_t comp = 0;
     if (mine) {
@@ -93,41 +95,39 @@ __device__ inline SimOut simulate_mixed_warp(const TabView& v, const uint16_t* _
         comp = (size_t)((e ? 2u : 0u) + (hd ? 1u : 0u)) * h->chain_len + nb;
         uint64_t replicas = 0;
         double gradbytes = 0.0;
-#pragma unroll
-        for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q)
-            if (q < ng) {
-                const uint32_t tp = h->tp_values[gtpi[q]];
-                replicas += gcount[q];
-                if (gcount[q] == 0 || tp > h->gpn[gtype[q]] || h->heads % tp != 0) status |= SAILOR_ST_INVALID;
-                atomicAdd(cnt + zone * T + gtype[q], (unsigned long long)gcount[q] * tp);
-                const size_t ct = comp * h->n_tp + gtpi[q];
-                const uint64_t* mm = v.cmp_mem + ((ct * h->n_mbs + mi) * 2 + rc) * 2;
-                const uint64_t m = mm[0] + inflight * mm[1] + h->reserved[gtype[q]];
-                if (m > h->capacity[gtype[q]]) status |= SAILOR_ST_OOM;
-                peak_l = m > peak_l ? m : peak_l;
-                gradbytes = dmax(gradbytes, v.cmp_grad[ct]);      // the ring moves the largest shard (smallest tp)
-            }
+#pragma unroll 1
+        for (uint32_t q = 0; q < ng; ++q) {
+            const uint32_t gq = group_word(q), ty = gq & 0xff, ti = (gq >> 8) & 0xff, cn = gq >> 16;
+            const uint32_t tp = h->tp_values[ti];
+            replicas += cn;
+            if (cn == 0 || tp > h->gpn[ty] || h->heads % tp != 0) status |= SAILOR_ST_INVALID;
+            atomicAdd(cnt + zone * T + ty, (unsigned long long)cn * tp);
+            const size_t ct = comp * h->n_tp + ti;
+            const uint64_t* mm = v.cmp_mem + ((ct * h->n_mbs + mi) * 2 + rc) * 2;
+            const uint64_t m = mm[0] + inflight * mm[1] + h->reserved[ty];
+            if (m > h->capacity[ty]) status |= SAILOR_ST_OOM;
+            peak_l = m > peak_l ? m : peak_l;
+            gradbytes = dmax(gradbytes, v.cmp_grad[ct]);          // the ring moves the largest shard (smallest tp)
+        }
         if (replicas != D) status |= SAILOR_ST_INVALID;
-#pragma unroll
-        for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q)
-            if (q < ng) {
-                const uint32_t d = zone * T + gtype[q], tp = h->tp_values[gtpi[q]];
-                upd_l = dmax(upd_l, v.cmp_upd[(comp * T + gtype[q]) * h->n_tp + gtpi[q]]);
-                if (D > 1) {
-                    const bool intra = ng == 1 && (uint64_t)D * tp <= h->gpn[gtype[q]];
-                    sync_l = dmax(sync_l, allreduce_bytes_time(v, d, intra, gradbytes, D, steps, coef));
-                }
-                term[q] = mul_rn((double)((uint32_t)gcount[q] * tp), v.price_s[d]);
+#pragma unroll 1
+        for (uint32_t q = 0; q < ng; ++q) {
+            const uint32_t gq = group_word(q), ty = gq & 0xff, ti = (gq >> 8) & 0xff;
+            const uint32_t d = zone * T + ty, tp = h->tp_values[ti];
+            upd_l = dmax(upd_l, v.cmp_upd[(comp * T + ty) * h->n_tp + ti]);
+            if (D > 1) {
+                const bool intra = ng == 1 && (uint64_t)D * tp <= h->gpn[ty];
+                sync_l = dmax(sync_l, allreduce_bytes_time(v, d, intra, gradbytes, D, steps, coef));
             }
+        }
     }
     __syncwarp();                                                // the counters are complete
     if (mine) {
-#pragma unroll
-        for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q)
-            if (q < ng) {
-                const uint32_t d = zone * T + gtype[q];
-                if (cnt[d] > avail[d]) status |= SAILOR_ST_OVER_AVAIL;
-            }
+#pragma unroll 1
+        for (uint32_t q = 0; q < ng; ++q) {
+            const uint32_t d = zone * T + (group_word(q) & 0xff);
+            if (cnt[d] > avail[d]) status |= SAILOR_ST_OVER_AVAIL;
+        }
     }
     status = __reduce_or_sync(MIX_FULL, status);
     o.peak_mem = warp_max_u64(peak_l);
@@ -136,21 +136,17 @@ __device__ inline SimOut simulate_mixed_warp(const TabView& v, const uint16_t* _
     const double max_sync = warp_max_f64(sync_l), max_u = warp_max_f64(upd_l);
     double rate = 0.0;                                           // stage after stage, group after group
     for (uint32_t i = 0; i < P; ++i) {
-        const uint32_t ng_i = __shfl_sync(MIX_FULL, ng, i);
-#pragma unroll
-        for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q) {
-            const double tq = __shfl_sync(MIX_FULL, term[q], i);
-            if (q < ng_i) rate = add_rn(rate, tq);
+        const uint32_t ng_i = __shfl_sync(MIX_FULL, ng, i), z_i = __shfl_sync(MIX_FULL, zone, i);
+        const uint64_t a01 = __shfl_sync(MIX_FULL, (unsigned long long)g01, i), a23 = __shfl_sync(MIX_FULL, (unsigned long long)g23, i);
+#pragma unroll 1
+        for (uint32_t q = 0; q < ng_i; ++q) {                    // every lane forms the same term (warp-uniform)
+            const uint32_t gq = (uint32_t)((q & 2u ? a23 : a01) >> (32u * (q & 1u)));
+            const uint32_t cn = gq >> 16, tp = h->tp_values[(gq >> 8) & 0xff];
+            rate = add_rn(rate, mul_rn((double)(cn * tp), v.price_s[z_i * T + (gq & 0xff)]));
         }
     }
 
     // the pipelines: from one group boundary to the next all replicas see the same groups
-    uint32_t upto[SAILOR_MIX_GROUPS_MAX];                        // replicas up to and including group q of this stage
-    {
-        uint32_t run = 0;
-#pragma unroll
-        for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q) { run += gcount[q]; upto[q] = run; }
-    }
     const double msg = (double)v.p2p[mi];
     const uint32_t z2 = __shfl_down_sync(MIX_FULL, zone, 1);     // zone of the next stage
     const bool sends = mine && lane + 1 < P;
@@ -158,13 +154,14 @@ __device__ inline SimOut simulate_mixed_warp(const TabView& v, const uint16_t* _
     uint32_t k = 0;
     while (k < D) {
         // group of replica k in this lane's stage
-        uint32_t g = gtype[0], tpi = gtpi[0], cn = gcount[0], nxt = upto[0];
+        uint32_t cur = (uint32_t)g01, nxt = cur >> 16;
 #pragma unroll
         for (uint32_t q = 1; q < SAILOR_MIX_GROUPS_MAX; ++q)
-            if (q < ng && k >= upto[q - 1]) { g = gtype[q]; tpi = gtpi[q]; cn = gcount[q]; nxt = upto[q]; }
+            if (q < ng && k >= nxt) { cur = group_word(q); nxt += cur >> 16; }
+        const uint32_t g = cur & 0xff, tpi = (cur >> 8) & 0xff, cn = cur >> 16;
         const uint32_t next = __reduce_min_sync(MIX_FULL, mine ? nxt : D);
-        const uint32_t g2 = __shfl_down_sync(MIX_FULL, g, 1), tpi2 = __shfl_down_sync(MIX_FULL, tpi, 1),
-                       cn2 = __shfl_down_sync(MIX_FULL, cn, 1);
+        const uint32_t cur2 = __shfl_down_sync(MIX_FULL, cur, 1);
+        const uint32_t g2 = cur2 & 0xff, tpi2 = (cur2 >> 8) & 0xff, cn2 = cur2 >> 16;
         double t = 0.0;
         if (mine) {
             const double fb = v.cmp_fb[(((comp * T + g) * h->n_tp + tpi) * h->n_mbs + mi) * 2 + rc];
