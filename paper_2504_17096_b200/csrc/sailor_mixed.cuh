@@ -167,16 +167,20 @@ __device__ inline SimOut simulate_mixed_warp(const TabView& v, const uint16_t* _
             const double fb = v.cmp_fb[(((comp * T + g) * h->n_tp + tpi) * h->n_mbs + mi) * 2 + rc];
             double c = 0.0;
             if (sends) {
-                const uint32_t z = zone;
-                if (z != z2) {
-                    c = link_time(v.zone_a[z * Z + z2], v.zone_i[z * Z + z2], v.zone_p, z * Z + z2, msg);
-                } else if (g == g2 && (uint64_t)cn * h->tp_values[tpi] + (uint64_t)cn2 * h->tp_values[tpi2] <= h->gpn[g]) {
-                    const uint32_t d = z * T + g;
-                    c = link_time(v.intra_a[d], v.intra_i[d], v.intra_p, d, msg);
-                } else {
-                    const uint32_t d = z * T + g, d2 = z * T + g2;
-                    c = dmax(link_time(v.inter_a[d], v.inter_i[d], v.inter_p, d, msg),
-                             link_time(v.inter_a[d2], v.inter_i[d2], v.inter_p, d2, msg));
+                // which link: its parameters are picked first, so that the link model is in the code once (twice for
+                // the inter-node link between unlike types, whose slower end counts)
+                const uint32_t z = zone, d = z * T + g;
+                const bool cross = z != z2;
+                const bool intra = !cross && g == g2 &&
+                                   (uint64_t)cn * h->tp_values[tpi] + (uint64_t)cn2 * h->tp_values[tpi2] <= h->gpn[g];
+                const uint32_t idx = cross ? z * Z + z2 : d;
+                const double* la = cross ? v.zone_a : intra ? v.intra_a : v.inter_a;
+                const double* li = cross ? v.zone_i : intra ? v.intra_i : v.inter_i;
+                const double* lp = cross ? v.zone_p : intra ? v.intra_p : v.inter_p;
+                c = link_time(la[idx], li[idx], lp, idx, msg);
+                if (!cross && !intra && g2 != g) {
+                    const uint32_t d2 = z * T + g2;
+                    c = dmax(c, link_time(v.inter_a[d2], v.inter_i[d2], v.inter_p, d2, msg));
                 }
             }
             t = add_rn(fb, mul_rn(2.0, c));
