@@ -19,19 +19,23 @@ namespace sailor {
 
 constexpr uint32_t MIX_FULL = 0xffffffffu;
 
-__device__ __forceinline__ double warp_max_f64(double x) {
-#pragma unroll
-    for (uint32_t o = 16; o; o >>= 1) x = dmax(x, __shfl_xor_sync(MIX_FULL, x, o));
-    return x;
+// Largest of the warp's 64-bit values by two 32-bit warp maxima: the high words, then the low words of the lanes
+// that hold the largest high word.
+__device__ __forceinline__ uint64_t warp_max_u64(uint64_t x) {
+    const uint32_t hi = (uint32_t)(x >> 32), lo = (uint32_t)x;
+    const uint32_t mh = __reduce_max_sync(MIX_FULL, hi);
+    const uint32_t ml = __reduce_max_sync(MIX_FULL, hi == mh ? lo : 0u);
+    return (uint64_t)mh << 32 | ml;
 }
 
-__device__ __forceinline__ uint64_t warp_max_u64(uint64_t x) {
-#pragma unroll
-    for (uint32_t o = 16; o; o >>= 1) {
-        const uint64_t y = __shfl_xor_sync(MIX_FULL, (unsigned long long)x, o);
-        x = y > x ? y : x;
-    }
-    return x;
+// Largest of the warp's binary64 values (none is a NaN): the bit patterns, mapped so that unsigned order is numeric
+// order (sign bit flipped for positive values, all bits for negative ones), go through warp_max_u64.
+__device__ __forceinline__ double warp_max_f64(double x) {
+    uint64_t b = (uint64_t)__double_as_longlong(x);
+    b ^= (b >> 63) ? ~0ull : 0x8000000000000000ull;
+    uint64_t m = warp_max_u64(b);
+    m ^= (m >> 63) ? 0x8000000000000000ull : ~0ull;
+    return __longlong_as_double((long long)m);
 }
 
 // `cnt` points to this warp's per-digit GPU counters (R of them, shared memory).  Every lane of the warp
@@ -74,9 +78,16 @@ __device__ inline SimOut simulate_mixed_warp(const TabView& v, const uint16_t* _
 
     uint32_t status = 0;
     const uint64_t dm = (uint64_t)D * h->mbs_values[mi];
-    if (h->gbs % dm != 0) status |= SAILOR_ST_INVALID;
-    const uint64_t n_b = h->gbs / dm;
-    const uint32_t base = h->n_blocks / P, extra = h->n_blocks % P;
+    uint64_t n_b;
+    if (((h->gbs | dm) >> 32) == 0) {                            // the usual case: a 32-bit division
+        const uint32_t q32 = (uint32_t)h->gbs / (uint32_t)dm;
+        n_b = q32;
+        if (q32 * (uint32_t)dm != (uint32_t)h->gbs) status |= SAILOR_ST_INVALID;
+    } else {
+        n_b = h->gbs / dm;
+        if (n_b * dm != h->gbs) status |= SAILOR_ST_INVALID;
+    }
+    const uint32_t base = h->n_blocks / P, extra = h->n_blocks - base * P;
 
     // validity, resources, memory per group, update time, synchronisation, price-rate terms: all stages at once
     for (uint32_t d = lane; d < R; d += 32) cnt[d] = 0;
@@ -134,15 +145,19 @@ __device__ inline SimOut simulate_mixed_warp(const TabView& v, const uint16_t* _
     o.status = status;
     if (status & SAILOR_ST_INVALID) return o;
     const double max_sync = warp_max_f64(sync_l), max_u = warp_max_f64(upd_l);
+    double term[SAILOR_MIX_GROUPS_MAX];                          // this stage's price-rate terms
+#pragma unroll
+    for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q) {
+        const uint32_t gq = group_word(q);                       // zero beyond the stage's groups: type 0, no replicas
+        term[q] = mul_rn((double)((gq >> 16) * h->tp_values[(gq >> 8) & 0xff]), v.price_s[zone * T + (gq & 0xff)]);
+    }
     double rate = 0.0;                                           // stage after stage, group after group
     for (uint32_t i = 0; i < P; ++i) {
-        const uint32_t ng_i = __shfl_sync(MIX_FULL, ng, i), z_i = __shfl_sync(MIX_FULL, zone, i);
-        const uint64_t a01 = __shfl_sync(MIX_FULL, (unsigned long long)g01, i), a23 = __shfl_sync(MIX_FULL, (unsigned long long)g23, i);
-#pragma unroll 1
-        for (uint32_t q = 0; q < ng_i; ++q) {                    // every lane forms the same term (warp-uniform)
-            const uint32_t gq = (uint32_t)((q & 2u ? a23 : a01) >> (32u * (q & 1u)));
-            const uint32_t cn = gq >> 16, tp = h->tp_values[(gq >> 8) & 0xff];
-            rate = add_rn(rate, mul_rn((double)(cn * tp), v.price_s[z_i * T + (gq & 0xff)]));
+        const uint32_t ng_i = __shfl_sync(MIX_FULL, ng, i);
+#pragma unroll
+        for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q) {
+            const double tq = __shfl_sync(MIX_FULL, term[q], i);
+            if (q < ng_i) rate = add_rn(rate, tq);
         }
     }
 
