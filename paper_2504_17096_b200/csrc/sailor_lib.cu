@@ -2142,8 +2142,9 @@ extern "C" int sailor_mixed_decode(const sailor_ctx* ctx, const sailor_mixed_spa
         const uint32_t c = (uint32_t)(std::upper_bound(mt.flat_base.begin(), mt.flat_base.end(), flat) - mt.flat_base.begin()) - 1;
         const MixedConfig k = mixed_config_of(mt.desc, c);
         const uint64_t radix = (uint64_t)ctx->hdr.Z * mt.desc.n_comb[k.di];
-        uint64_t rem = flat - mt.flat_base[c], digit[SAILOR_SEG_MAX] = {0, 0, 0, 0};
-        for (uint32_t q = k.nseg; q-- > 0;) { digit[q] = rem % radix; rem /= radix; }
+        uint64_t rem = flat - mt.flat_base[c];
+        uint32_t digit[SAILOR_SEG_MAX] = {0, 0, 0, 0};
+        for (uint32_t q = k.nseg; q-- > 0;) { digit[q] = (uint32_t)(rem % radix); rem /= radix; }
         memset(out, 0, sizeof(*out));
         out->P = (uint8_t)k.P; out->mbs_idx = (uint8_t)k.mi; out->rc = (uint8_t)k.rc; out->D = (uint16_t)k.D;
         for (uint32_t i = 0; i < k.P; ++i) mixed_build_stage(mt.desc, k, ctx->hdr.T, mt.combs.data(), digit, i, &out->stage[i]);

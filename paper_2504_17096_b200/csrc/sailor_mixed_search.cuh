@@ -33,7 +33,7 @@ __host__ __device__ inline uint32_t mixed_units(uint32_t granularity, uint32_t D
 }
 
 // Configuration c = ((p * n_mbs + mbs) * n_rc + rc) * n_d + d (positions in the space's lists).
-struct MixedConfig { uint32_t P, mi, rc, D, di, nseg; };
+struct MixedConfig { uint32_t P, mi, rc, D, di, nseg, per_unit; };   // per_unit: replicas in one unit of a combination
 
 __host__ __device__ inline MixedConfig mixed_config_of(const MixedSpaceDesc& s, uint32_t c) {
     MixedConfig k;
@@ -46,20 +46,21 @@ __host__ __device__ inline MixedConfig mixed_config_of(const MixedSpaceDesc& s, 
     k.rc = s.rc_values[ri];
     k.D = s.d_values[k.di];
     k.nseg = k.P < s.seg_max ? k.P : s.seg_max;
+    k.per_unit = k.D / mixed_units(s.granularity, k.D);
     return k;
 }
 
 // Stage i of the candidate whose segment digits are `digit` (zone * n_comb + combination): its record.
 // `combs` holds one 64-bit word per combination, byte g = units on type g.
 __host__ __device__ inline void mixed_build_stage(const MixedSpaceDesc& s, const MixedConfig& k, uint32_t T,
-                                                  const uint64_t* combs, const uint64_t* digit, uint32_t i,
+                                                  const uint64_t* combs, const uint32_t* digit, uint32_t i,
                                                   sailor_mixed_stage* out) {
     const uint32_t n_comb = s.n_comb[k.di];
-    const uint64_t dg = digit[(uint64_t)i * k.nseg / k.P];
-    const uint64_t word = combs[s.comb_off[k.di] + (uint32_t)(dg % n_comb)];
-    const uint32_t per_unit = k.D / mixed_units(s.granularity, k.D);
+    const uint32_t dg = digit[i * k.nseg / k.P], zone = dg / n_comb;       // a digit is below Z * n_comb < 2^32
+    const uint64_t word = combs[s.comb_off[k.di] + (dg - zone * n_comb)];
+    const uint32_t per_unit = k.per_unit;
     sailor_mixed_stage st;
-    st.zone = (uint8_t)(dg / n_comb);
+    st.zone = (uint8_t)zone;
     st.n_groups = 0;
     st._pad = 0;
     for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q) { st.group[q].type = 0; st.group[q].tp_idx = 0; st.group[q].count = 0; }
@@ -91,23 +92,46 @@ struct MixedSearchParams {
 constexpr int MIXS_THREADS = 256;
 constexpr int MIXS_WARPS = MIXS_THREADS / 32;
 
-// The record of candidate `flat` into `plan` (shared memory, one per warp), by all lanes of the warp.
+// The record of candidate `flat` into `plan` (shared memory, one per warp), by all lanes of the warp.  WHOLE: the
+// stages past the last are zeroed as well (a record that leaves the device); the evaluation reads the first P only.
+// The configuration of a warp's previous candidate (a warp's candidates are a grid stride apart and mostly stay
+// inside one configuration): tried first, decoded anew only when the index has left it.
+struct MixedCursor {
+    uint32_t cfg = ~0u;
+    uint64_t lo = 1, hi = 0;             // flat indices [lo, hi) of the configuration
+    MixedConfig k;
+};
+
+template <bool WHOLE>
 __device__ __forceinline__ void mixed_candidate(const MixedSearchParams& mp, uint32_t T, uint32_t Z, uint64_t flat,
-                                                sailor_mixed_plan* plan, uint32_t lane) {
-    uint32_t lo = 0, hi = mp.n_config;                       // the configuration whose block holds the index
-    while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (mp.cfg_flat_base[mid] <= flat) lo = mid; else hi = mid;
+                                                sailor_mixed_plan* plan, uint32_t lane, MixedCursor& cur) {
+    if (!(cur.lo <= flat && flat < cur.hi)) {
+        uint32_t lo = 0, hi = mp.n_config;                   // the configuration whose block holds the index
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (mp.cfg_flat_base[mid] <= flat) lo = mid; else hi = mid;
+        }
+        cur.cfg = lo;
+        cur.lo = mp.cfg_flat_base[lo];
+        cur.hi = mp.cfg_flat_base[lo + 1];
+        cur.k = mixed_config_of(mp.sp, lo);
     }
-    const MixedConfig k = mixed_config_of(mp.sp, lo);
+    const MixedConfig& k = cur.k;
     const uint64_t radix = (uint64_t)Z * mp.sp.n_comb[k.di];
-    uint64_t rem = flat - mp.cfg_flat_base[lo], digit[SAILOR_SEG_MAX] = {0, 0, 0, 0};
-    for (uint32_t s = k.nseg; s-- > 0;) { digit[s] = rem % radix; rem /= radix; }
+    uint64_t rem = flat - cur.lo;
+    uint32_t digit[SAILOR_SEG_MAX] = {0, 0, 0, 0};
+    if ((rem >> 32) == 0) {                                  // the usual case: 32-bit divisions
+        uint32_t r32 = (uint32_t)rem;
+        const uint32_t rx = (uint32_t)radix;
+        for (uint32_t s = k.nseg; s-- > 0;) { const uint32_t q = r32 / rx; digit[s] = r32 - q * rx; r32 = q; }
+    } else {
+        for (uint32_t s = k.nseg; s-- > 0;) { digit[s] = (uint32_t)(rem % radix); rem /= radix; }
+    }
     if (lane == 0) {
         plan->P = (uint8_t)k.P; plan->mbs_idx = (uint8_t)k.mi; plan->rc = (uint8_t)k.rc; plan->_pad = 0;
         plan->D = (uint16_t)k.D; plan->_pad2 = 0;
     }
-    for (uint32_t i = lane; i < SAILOR_MIX_P_MAX; i += 32) {
+    for (uint32_t i = lane; i < (WHOLE ? (uint32_t)SAILOR_MIX_P_MAX : k.P); i += 32) {
         if (i < k.P) mixed_build_stage(mp.sp, k, T, mp.combs, digit, i, &plan->stage[i]);
         else {                                                 // stages past the last are all zero, as the host decoder leaves them
             uint32_t* z = reinterpret_cast<uint32_t*>(&plan->stage[i]);
@@ -141,8 +165,9 @@ __global__ void __launch_bounds__(MIXS_THREADS, 2) plan_mixed_kernel(const __gri
     unsigned long long n_class[6] = {0, 0, 0, 0, 0, 0};
     double min_cost = make_inf();
     const uint64_t stride = (uint64_t)gridDim.x * MIXS_WARPS;
+    MixedCursor cur;                                           // configuration of this warp's previous candidate
     for (uint64_t flat = (uint64_t)blockIdx.x * MIXS_WARPS + warp; flat < mp.n_total; flat += stride) {
-        mixed_candidate(mp, T, Z, flat, plan, lane);
+        mixed_candidate<false>(mp, T, Z, flat, plan, lane, cur);
         const SimOut o = DEEP ? simulate_mixed_plan(v, mp.avail, *plan, cnt, lane) : simulate_mixed_warp(v, mp.avail, *plan, cnt, lane);
         __syncwarp();                                          // the record and the counters are reused by the next candidate
         // every candidate falls in exactly one class: invalid, out of memory, over availability, over the constraint, feasible
@@ -221,7 +246,8 @@ __global__ void __launch_bounds__(MIXS_THREADS) mixed_finish_kernel(const __grid
     __syncthreads();
     for (uint32_t j = warp; j < s_n; j += MIXS_WARPS) {
         const uint64_t flat = s_hits[0][j].flat;
-        mixed_candidate(mp, T, Z, flat, plan, lane);
+        MixedCursor cur;
+        mixed_candidate<true>(mp, T, Z, flat, plan, lane, cur);
         const SimOut o = simulate_mixed_plan(v, mp.avail, *plan, cnt, lane);
         __syncwarp();
         sailor_mixed_result* r = mp.results + j;
