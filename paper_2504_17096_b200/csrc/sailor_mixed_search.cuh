@@ -58,21 +58,23 @@ __host__ __device__ inline void mixed_build_stage(const MixedSpaceDesc& s, const
     const uint32_t n_comb = s.n_comb[k.di];
     const uint32_t dg = digit[i * k.nseg / k.P], zone = dg / n_comb;       // a digit is below Z * n_comb < 2^32
     const uint64_t word = combs[s.comb_off[k.di] + (dg - zone * n_comb)];
-    const uint32_t per_unit = k.per_unit;
-    sailor_mixed_stage st;
-    st.zone = (uint8_t)zone;
-    st.n_groups = 0;
-    st._pad = 0;
-    for (uint32_t q = 0; q < SAILOR_MIX_GROUPS_MAX; ++q) { st.group[q].type = 0; st.group[q].tp_idx = 0; st.group[q].count = 0; }
+    // the stage as five 32-bit words (little-endian fields): zone | n_groups << 8, then type | tp_idx << 8 | count << 16
+    // per group; the non-empty types in ascending order take the groups
+    uint32_t gw[SAILOR_MIX_GROUPS_MAX] = {0, 0, 0, 0}, n_groups = 0;
     for (uint32_t g = 0; g < T; ++g) {
         const uint32_t units = (uint32_t)(word >> (8 * g)) & 0xffu;
-        if (!units || st.n_groups >= SAILOR_MIX_GROUPS_MAX) continue;
-        st.group[st.n_groups].type = (uint8_t)g;
-        st.group[st.n_groups].tp_idx = s.tp_idx_of_type[g];
-        st.group[st.n_groups].count = (uint16_t)(units * per_unit);
-        st.n_groups++;
+        if (!units || n_groups >= SAILOR_MIX_GROUPS_MAX) continue;
+        const uint32_t grp = g | (uint32_t)s.tp_idx_of_type[g] << 8 | (units * k.per_unit & 0xffffu) << 16;
+        gw[0] = n_groups == 0 ? grp : gw[0];
+        gw[1] = n_groups == 1 ? grp : gw[1];
+        gw[2] = n_groups == 2 ? grp : gw[2];
+        gw[3] = n_groups == 3 ? grp : gw[3];
+        n_groups++;
     }
-    *out = st;
+    static_assert(sizeof(sailor_mixed_stage) == 20 && SAILOR_MIX_GROUPS_MAX == 4, "five words a stage");
+    uint32_t* w = reinterpret_cast<uint32_t*>(out);
+    w[0] = (zone & 0xffu) | n_groups << 8;
+    w[1] = gw[0]; w[2] = gw[1]; w[3] = gw[2]; w[4] = gw[3];
 }
 
 struct MixedSearchParams {
