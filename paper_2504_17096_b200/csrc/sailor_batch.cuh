@@ -257,7 +257,7 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
                 unsigned int* bad_flag) {                      // not null: set SIM_ERR_BAD_RECORD there when a record is refused
     __shared__ BatchConst k;
     __shared__ uint64_t recs[BATCH_POOL * REC_WORDS];
-    __shared__ uint32_t hist[128];
+    __shared__ uint32_t hist[256];
     __shared__ uint16_t perm[BATCH_POOL];
     __shared__ uint32_t next_group;
     const uint32_t tid = threadIdx.x, lane = tid & 31;
@@ -290,7 +290,7 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
         const uint32_t cnt = (uint32_t)(n - pool < BATCH_POOL ? n - pool : BATCH_POOL);
         __syncthreads();
         for (uint32_t x = tid; x < cnt * REC_WORDS; x += BATCH_THREADS) recs[x] = __ldcs(&src[pool * REC_WORDS + x]);
-        if (tid < 128) hist[tid] = 0;
+        hist[tid] = 0;
         if (tid == 0) next_group = 0;
         __syncthreads();
         // counting sort, most work first: by run count (byte 3 of a record), then by stage count (byte 0)
@@ -302,16 +302,16 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
             if (x < cnt) {
                 const uint32_t w0 = (uint32_t)recs[x * REC_WORDS];
                 const uint32_t P = w0 & 0xff, nr = w0 >> 24;
-                const uint32_t work = (nr > 15u ? 15u : nr) * 8u + (P > 95u ? 7u : P / 12u);
-                key[u] = 127u - work;
+                const uint32_t work = (nr > 15u ? 15u : nr) * 16u + (P > 95u ? 15u : P / 6u);
+                key[u] = 255u - work;
                 rank[u] = atomicAdd(&hist[key[u]], 1u);
             }
         }
         __syncthreads();
-        if (tid < 32) {                                        // exclusive scan of the 128 bins by one warp
-            uint32_t h4[4], sum = 0;
+        if (tid < 32) {                                        // exclusive scan of the 256 bins by one warp
+            uint32_t h4[8], sum = 0;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) { h4[q] = hist[tid * 4 + q]; sum += h4[q]; }
+            for (int q = 0; q < 8; ++q) { h4[q] = hist[tid * 8 + q]; sum += h4[q]; }
             uint32_t incl = sum;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -320,7 +320,7 @@ simulate_kernel(const unsigned char* __restrict__ blob, const uint16_t* __restri
             }
             uint32_t at = incl - sum;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) { hist[tid * 4 + q] = at; at += h4[q]; }
+            for (int q = 0; q < 8; ++q) { hist[tid * 8 + q] = at; at += h4[q]; }
         }
         __syncthreads();
 #pragma unroll
