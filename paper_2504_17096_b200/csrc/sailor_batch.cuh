@@ -95,6 +95,7 @@ constexpr int BATCH_THREADS = 256;
 constexpr int BATCH_BLOCKS_PER_SM = 3;
 constexpr uint32_t BATCH_POOL = 512;             // records a block stages and orders at a time
 constexpr uint32_t REC_WORDS = sizeof(sailor_plan_rec) / 8;
+static_assert(BATCH_POOL % BATCH_THREADS == 0, "every thread ranks BATCH_POOL / BATCH_THREADS records of a pool: a pool that is not a multiple leaves records unranked");
 
 struct BatchOut {
     double t_iter, cost;
